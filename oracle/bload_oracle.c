@@ -1,0 +1,333 @@
+/*
+ * bload_oracle.c -- TEST INFRASTRUCTURE, not part of the product.
+ *
+ * A plain, slow, single-threaded CPU statement of BLoad's ragged-to-block
+ * packing (Methods section of the paper, its Fig. "Our proposed padding
+ * approach" and the caption of its pseudocode figure).  It exists so that the
+ * GPU library can be compared with it element by element.  It shares no code
+ * with the GPU library and must never be called from the product path: only
+ * the tests, the smoke check and the benchmark's CPU-baseline leg use it.
+ *
+ * Everything is written with linear scans, per-slot loops and memcpy so that a
+ * reader can check each function against the paper by eye.
+ *
+ * Pins (what each function is checked against, in tests that need no GPU):
+ *   philox4x64_10      numpy's Philox bit generator (same published algorithm)
+ *   oracle_pick        Python big-integer arithmetic
+ *   offsets            numpy.cumsum (textbook exclusive prefix sum)
+ *   L_dict order       Python sorted() on (T, h, i)
+ *   fill rule          exhaustive enumeration of the choice tree on tiny inputs
+ *                      (reachable set, exact probabilities, chi-square),
+ *                      maximality and no-drop/no-split invariants, the toy
+ *                      dataset of the paper (8 videos, lengths 2..6)
+ *   stats              closed forms; the paper's Table I "0 padding" count
+ *   metadata/pack/unpack  numpy fancy-index gather built from the tables,
+ *                      round trip, pad bytes
+ *   Parity unpinned: the paper's "block_pad" padding count of Table I (block
+ *   length of that run is not stated and the rule is random) and its
+ *   time-per-epoch figures.
+ */
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+#define ORACLE_OK 0
+#define ORACLE_ERR_ARG (-1)
+#define ORACLE_ERR_LENGTH (-2)
+#define ORACLE_ERR_NOMEM (-3)
+#define ORACLE_ERR_POLICY (-4)
+
+/* ------------------------------------------------------------------------ */
+/* Counter-based random numbers: Philox-4x64-10 (Salmon, Moraes, Dror, Shaw, */
+/* "Parallel random numbers: as easy as 1, 2, 3", SC'11).                    */
+/* ------------------------------------------------------------------------ */
+
+static void mul_hi_lo(uint64_t a, uint64_t b, uint64_t *hi, uint64_t *lo)
+{
+    unsigned __int128 p = (unsigned __int128)a * (unsigned __int128)b;
+    *hi = (uint64_t)(p >> 64);
+    *lo = (uint64_t)p;
+}
+
+void oracle_philox4x64_10(const uint64_t ctr_in[4], const uint64_t key_in[2], uint64_t out[4])
+{
+    const uint64_t mult0 = 0xD2E7470EE14C6C93ULL, mult1 = 0xCA5A826395121157ULL;
+    const uint64_t weyl0 = 0x9E3779B97F4A7C15ULL, weyl1 = 0xBB67AE8584CAA73BULL;
+    uint64_t c[4] = {ctr_in[0], ctr_in[1], ctr_in[2], ctr_in[3]};
+    uint64_t k[2] = {key_in[0], key_in[1]};
+    for (int round = 0; round < 10; ++round) {
+        uint64_t hi0, lo0, hi1, lo1;
+        if (round > 0) { k[0] += weyl0; k[1] += weyl1; }
+        mul_hi_lo(mult0, c[0], &hi0, &lo0);
+        mul_hi_lo(mult1, c[2], &hi1, &lo1);
+        uint64_t n0 = hi1 ^ c[1] ^ k[0];
+        uint64_t n1 = lo1;
+        uint64_t n2 = hi0 ^ c[3] ^ k[1];
+        uint64_t n3 = lo0;
+        c[0] = n0; c[1] = n1; c[2] = n2; c[3] = n3;
+    }
+    out[0] = c[0]; out[1] = c[1]; out[2] = c[2]; out[3] = c[3];
+}
+
+/* Two streams of the generator: key = (seed, stream), counter = (index,0,0,0),
+ * first output word is used. */
+#define STREAM_KEYS 1ULL
+#define STREAM_DRAWS 2ULL
+
+/* h_i: the shuffle key that orders sequences of equal length inside L_dict. */
+uint32_t oracle_seq_key(uint64_t seed, int64_t i)
+{
+    uint64_t c[4] = {(uint64_t)i, 0, 0, 0}, k[2] = {seed, STREAM_KEYS}, o[4];
+    oracle_philox4x64_10(c, k, o);
+    return (uint32_t)(o[0] >> 32);
+}
+
+/* u_k: the 64-bit random word of the k-th draw of the fill loop. */
+uint64_t oracle_draw_word(uint64_t seed, int64_t k)
+{
+    uint64_t c[4] = {(uint64_t)k, 0, 0, 0}, kk[2] = {seed, STREAM_DRAWS}, o[4];
+    oracle_philox4x64_10(c, kk, o);
+    return o[0];
+}
+
+/* Map a 64-bit word to an index in [0, m): floor(u * m / 2^64). */
+uint64_t oracle_pick(uint64_t u, uint64_t m)
+{
+    return (uint64_t)(((unsigned __int128)u * (unsigned __int128)m) >> 64);
+}
+
+/* ------------------------------------------------------------------------ */
+/* Ragged offsets: offsets[i] = T_0 + ... + T_{i-1}; offsets[n] = sum T.     */
+/* (Problem statement: N samples of T_i frames stored back to back.)         */
+/* ------------------------------------------------------------------------ */
+void oracle_offsets(const int32_t *lengths, int64_t n, int64_t *offsets)
+{
+    int64_t acc = 0;
+    for (int64_t i = 0; i < n; ++i) { offsets[i] = acc; acc += lengths[i]; }
+    offsets[n] = acc;
+}
+
+/* ------------------------------------------------------------------------ */
+/* Plan: block construction (Methods, first paragraph) and the table of      */
+/* start indices (Methods, second paragraph).                                */
+/* ------------------------------------------------------------------------ */
+typedef struct {
+    const int32_t *lengths; /* in  [n] */
+    int64_t n;
+    int32_t t_block;
+    uint64_t seed;
+    uint32_t policy; /* 0 = uniform over the unused sequences that fit */
+    /* outputs, all caller-allocated */
+    int64_t *offsets;         /* [n+1] */
+    int32_t *seg_seq;         /* [n]   sequence placed by the k-th draw */
+    int32_t *seg_block;       /* [n]   block it went to */
+    int32_t *seg_start;       /* [n]   first slot it occupies in that block */
+    int32_t *block_seg_begin; /* [n+1] k of the first draw of each block (CSR) */
+    int32_t *block_fill;      /* [n]   occupied slots of each block */
+    int32_t *seq_block;       /* [n]   inverse: block of sequence i */
+    int32_t *seq_start;       /* [n]   inverse: first slot of sequence i */
+    /* scalars */
+    int64_t n_blocks, sum_t, t_max, first_bad;
+    uint64_t checksum;
+    int64_t max_segs_per_block;
+} oracle_plan_t;
+
+typedef struct { int32_t len; uint32_t h; int32_t id; } ldict_entry_t;
+
+static int ldict_cmp(const void *pa, const void *pb)
+{
+    const ldict_entry_t *a = (const ldict_entry_t *)pa, *b = (const ldict_entry_t *)pb;
+    if (a->len != b->len) return a->len < b->len ? -1 : 1;
+    if (a->h != b->h) return a->h < b->h ? -1 : 1;
+    if (a->id != b->id) return a->id < b->id ? -1 : 1;
+    return 0;
+}
+
+static uint64_t fmix64(uint64_t x)
+{ /* the 64-bit finaliser of MurmurHash3 (public domain, A. Appleby) */
+    x ^= x >> 33; x *= 0xff51afd7ed558ccdULL;
+    x ^= x >> 33; x *= 0xc4ceb9fe1a85ec53ULL;
+    x ^= x >> 33;
+    return x;
+}
+
+int oracle_plan(oracle_plan_t *p)
+{
+    const int64_t n = p->n;
+    const int32_t tb = p->t_block;
+    p->n_blocks = 0; p->sum_t = 0; p->t_max = 0; p->first_bad = -1;
+    p->checksum = 0; p->max_segs_per_block = 0;
+    if (n < 1 || n > 0x7fffffffLL || tb < 1) return ORACLE_ERR_ARG;
+    if (p->policy != 0) return ORACLE_ERR_POLICY;
+
+    /* Precondition of the method: 1 <= T_i <= block length. */
+    for (int64_t i = 0; i < n; ++i) {
+        if (p->lengths[i] < 1 || p->lengths[i] > tb) { p->first_bad = i; return ORACLE_ERR_LENGTH; }
+    }
+    oracle_offsets(p->lengths, n, p->offsets);
+    p->sum_t = p->offsets[n];
+    for (int64_t i = 0; i < n; ++i) if (p->lengths[i] > p->t_max) p->t_max = p->lengths[i];
+
+    /* L_dict: for every length, the sequences of that length in (h_i, i) order. */
+    ldict_entry_t *dict = (ldict_entry_t *)malloc((size_t)n * sizeof *dict);
+    int64_t *first = (int64_t *)calloc((size_t)tb + 2, sizeof *first);  /* first[l]: where length l begins in dict */
+    int64_t *unused = (int64_t *)calloc((size_t)tb + 2, sizeof *unused); /* unused[l]: entries of length l not yet drawn */
+    if (!dict || !first || !unused) { free(dict); free(first); free(unused); return ORACLE_ERR_NOMEM; }
+    for (int64_t i = 0; i < n; ++i) {
+        dict[i].len = p->lengths[i];
+        dict[i].h = oracle_seq_key(p->seed, i);
+        dict[i].id = (int32_t)i;
+        unused[p->lengths[i]] += 1;
+    }
+    qsort(dict, (size_t)n, sizeof *dict, ldict_cmp);
+    first[1] = 0;
+    for (int32_t l = 1; l <= tb; ++l) first[l + 1] = first[l] + unused[l];
+
+    int64_t k = 0;      /* draws made so far */
+    int64_t b = 0;      /* current block */
+    while (k < n) {
+        int32_t remaining = tb, start = 0;
+        p->block_seg_begin[b] = (int32_t)k;
+        for (;;) {
+            /* m: unused sequences that still fit */
+            int64_t m = 0;
+            for (int32_t l = 1; l <= remaining; ++l) m += unused[l];
+            if (m == 0) break;
+            /* Random_*(): the j-th of them, counted in order of length */
+            uint64_t j = oracle_pick(oracle_draw_word(p->seed, k), (uint64_t)m);
+            int32_t l = 1;
+            int64_t run = unused[1];
+            while ((uint64_t)run <= j) { l += 1; run += unused[l]; }
+            /* first unused entry of L_dict[l] */
+            int64_t taken = (first[l + 1] - first[l]) - unused[l];
+            int32_t id = dict[first[l] + taken].id;
+            unused[l] -= 1;
+            p->seg_seq[k] = id;
+            p->seg_block[k] = (int32_t)b;
+            p->seg_start[k] = start;
+            p->seq_block[id] = (int32_t)b;
+            p->seq_start[id] = start;
+            start += l;
+            remaining -= l;
+            k += 1;
+        }
+        p->block_fill[b] = start; /* slots [start, t_block) are padding */
+        int64_t segs = k - p->block_seg_begin[b];
+        if (segs > p->max_segs_per_block) p->max_segs_per_block = segs;
+        b += 1;
+    }
+    p->block_seg_begin[b] = (int32_t)k;
+    p->n_blocks = b;
+
+    /* Order-independent 64-bit digest of the segment list. */
+    uint64_t sum = 0;
+    for (int64_t q = 0; q < n; ++q) {
+        uint64_t where = ((uint64_t)(uint32_t)p->seg_block[q] << 32) | (uint64_t)(uint32_t)p->seg_start[q];
+        sum += fmix64(where * 0x9E3779B97F4A7C15ULL + (uint64_t)(uint32_t)p->seg_seq[q]);
+    }
+    p->checksum = sum;
+
+    free(dict); free(first); free(unused);
+    return ORACLE_OK;
+}
+
+/* ------------------------------------------------------------------------ */
+/* Per-slot metadata for blocks [block_begin, block_begin + block_count).     */
+/* Blocks at or beyond n_blocks are filler: all padding.                      */
+/* ------------------------------------------------------------------------ */
+typedef struct {
+    int64_t n, n_blocks;
+    int32_t t_block;
+    const int64_t *offsets;
+    const int32_t *seg_seq, *seg_start, *block_seg_begin;
+} oracle_tables_t;
+
+int oracle_metadata(const oracle_tables_t *t, int64_t block_begin, int64_t block_count,
+                    int32_t *seq_id, int32_t *pos, uint8_t *reset, uint8_t *valid)
+{
+    if (block_begin < 0 || block_count < 0) return ORACLE_ERR_ARG;
+    for (int64_t q = 0; q < block_count; ++q) {
+        int64_t b = block_begin + q;
+        int32_t *sid = seq_id + q * t->t_block, *ps = pos + q * t->t_block;
+        uint8_t *rs = reset + q * t->t_block, *vd = valid + q * t->t_block;
+        for (int32_t s = 0; s < t->t_block; ++s) { sid[s] = -1; ps[s] = -1; rs[s] = 0; vd[s] = 0; }
+        if (b >= t->n_blocks) continue;
+        for (int32_t k = t->block_seg_begin[b]; k < t->block_seg_begin[b + 1]; ++k) {
+            int32_t id = t->seg_seq[k];
+            int64_t len = t->offsets[id + 1] - t->offsets[id];
+            for (int64_t f = 0; f < len; ++f) {
+                int64_t s = t->seg_start[k] + f;
+                sid[s] = id; ps[s] = (int32_t)f; vd[s] = 1; rs[s] = (f == 0);
+            }
+        }
+    }
+    return ORACLE_OK;
+}
+
+/* dense[q, s, :] = store[offsets[id] + f, :] on valid slots, pad_byte elsewhere. */
+int oracle_pack(const oracle_tables_t *t, const uint8_t *store, int64_t frame_bytes,
+                int64_t block_begin, int64_t block_count, uint8_t *dense, uint8_t pad_byte)
+{
+    if (block_begin < 0 || block_count < 0 || frame_bytes < 1) return ORACLE_ERR_ARG;
+    int32_t *sid = (int32_t *)malloc(sizeof(int32_t) * (size_t)t->t_block);
+    int32_t *ps = (int32_t *)malloc(sizeof(int32_t) * (size_t)t->t_block);
+    uint8_t *rs = (uint8_t *)malloc((size_t)t->t_block), *vd = (uint8_t *)malloc((size_t)t->t_block);
+    if (!sid || !ps || !rs || !vd) { free(sid); free(ps); free(rs); free(vd); return ORACLE_ERR_NOMEM; }
+    for (int64_t q = 0; q < block_count; ++q) {
+        oracle_metadata(t, block_begin + q, 1, sid, ps, rs, vd);
+        for (int32_t s = 0; s < t->t_block; ++s) {
+            uint8_t *dst = dense + ((size_t)q * (size_t)t->t_block + (size_t)s) * (size_t)frame_bytes;
+            if (vd[s]) memcpy(dst, store + (size_t)(t->offsets[sid[s]] + ps[s]) * (size_t)frame_bytes, (size_t)frame_bytes);
+            else memset(dst, pad_byte, (size_t)frame_bytes);
+        }
+    }
+    free(sid); free(ps); free(rs); free(vd);
+    return ORACLE_OK;
+}
+
+/* ragged_out[offsets[id] + f, :] = dense_out[q, s, :] on valid slots; padding ignored. */
+int oracle_unpack(const oracle_tables_t *t, const uint8_t *dense_out, int64_t frame_bytes,
+                  int64_t block_begin, int64_t block_count, uint8_t *ragged_out)
+{
+    if (block_begin < 0 || block_count < 0 || frame_bytes < 1) return ORACLE_ERR_ARG;
+    int32_t *sid = (int32_t *)malloc(sizeof(int32_t) * (size_t)t->t_block);
+    int32_t *ps = (int32_t *)malloc(sizeof(int32_t) * (size_t)t->t_block);
+    uint8_t *rs = (uint8_t *)malloc((size_t)t->t_block), *vd = (uint8_t *)malloc((size_t)t->t_block);
+    if (!sid || !ps || !rs || !vd) { free(sid); free(ps); free(rs); free(vd); return ORACLE_ERR_NOMEM; }
+    for (int64_t q = 0; q < block_count; ++q) {
+        oracle_metadata(t, block_begin + q, 1, sid, ps, rs, vd);
+        for (int32_t s = 0; s < t->t_block; ++s) {
+            if (!vd[s]) continue;
+            memcpy(ragged_out + (size_t)(t->offsets[sid[s]] + ps[s]) * (size_t)frame_bytes,
+                   dense_out + ((size_t)q * (size_t)t->t_block + (size_t)s) * (size_t)frame_bytes, (size_t)frame_bytes);
+        }
+    }
+    free(sid); free(ps); free(rs); free(vd);
+    return ORACLE_OK;
+}
+
+/* ------------------------------------------------------------------------ */
+/* Padding statistics (closed forms).                                         */
+/*   naive  : every sample padded to the longest one: N*T_max - sum T         */
+/*   packed : n_blocks*T_block - sum T                                         */
+/* ------------------------------------------------------------------------ */
+typedef struct {
+    int64_t n, sum_t, t_max, t_block, n_blocks;
+    int64_t pad_packed, pad_naive_tmax, pad_naive_tblock, min_blocks;
+    double frac_packed, frac_naive_tmax, frac_naive_tblock, reduction_vs_tmax, mean_segs_per_block;
+} oracle_stats_t;
+
+int oracle_stats(oracle_stats_t *s)
+{
+    if (s->n < 1 || s->t_block < 1 || s->sum_t < 1 || s->n_blocks < 0) return ORACLE_ERR_ARG;
+    s->pad_packed = s->n_blocks * s->t_block - s->sum_t;
+    s->pad_naive_tmax = s->n * s->t_max - s->sum_t;
+    s->pad_naive_tblock = s->n * s->t_block - s->sum_t;
+    s->min_blocks = (s->sum_t + s->t_block - 1) / s->t_block;
+    s->frac_packed = s->n_blocks ? (double)s->pad_packed / (double)(s->n_blocks * s->t_block) : 0.0;
+    s->frac_naive_tmax = s->t_max ? (double)s->pad_naive_tmax / (double)(s->n * s->t_max) : 0.0;
+    s->frac_naive_tblock = (double)s->pad_naive_tblock / (double)(s->n * s->t_block);
+    s->reduction_vs_tmax = s->pad_packed > 0 ? (double)s->pad_naive_tmax / (double)s->pad_packed : 0.0;
+    s->mean_segs_per_block = s->n_blocks ? (double)s->n / (double)s->n_blocks : 0.0;
+    return ORACLE_OK;
+}

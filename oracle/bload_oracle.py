@@ -1,0 +1,206 @@
+"""ctypes front end of the CPU oracle (``bload_oracle.c``).
+
+TEST INFRASTRUCTURE.  Only the tests, the smoke check and the benchmark's CPU
+baseline may import this module; the GPU library never does, and this module
+never imports the GPU package.  All arrays are numpy arrays in host memory.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+import subprocess
+from dataclasses import dataclass
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "bload_oracle.c")
+_SO = os.path.join(_HERE, "libbload_oracle.so")
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with gcc (no CUDA involved)."""
+    if force or not os.path.exists(_SO) or os.path.getmtime(_SO) < os.path.getmtime(_SRC):
+        tmp = _SO + ".tmp%d" % os.getpid()
+        subprocess.check_call(["gcc", "-O2", "-std=c11", "-Wall", "-Wextra", "-shared", "-fPIC", _SRC, "-o", tmp])
+        os.replace(tmp, _SO)
+    return _SO
+
+
+class _PlanStruct(C.Structure):
+    _fields_ = [
+        ("lengths", C.c_void_p), ("n", C.c_int64), ("t_block", C.c_int32), ("seed", C.c_uint64),
+        ("policy", C.c_uint32),
+        ("offsets", C.c_void_p), ("seg_seq", C.c_void_p), ("seg_block", C.c_void_p), ("seg_start", C.c_void_p),
+        ("block_seg_begin", C.c_void_p), ("block_fill", C.c_void_p), ("seq_block", C.c_void_p),
+        ("seq_start", C.c_void_p),
+        ("n_blocks", C.c_int64), ("sum_t", C.c_int64), ("t_max", C.c_int64), ("first_bad", C.c_int64),
+        ("checksum", C.c_uint64), ("max_segs_per_block", C.c_int64),
+    ]
+
+
+class _TablesStruct(C.Structure):
+    _fields_ = [
+        ("n", C.c_int64), ("n_blocks", C.c_int64), ("t_block", C.c_int32),
+        ("offsets", C.c_void_p), ("seg_seq", C.c_void_p), ("seg_start", C.c_void_p),
+        ("block_seg_begin", C.c_void_p),
+    ]
+
+
+class _StatsStruct(C.Structure):
+    _fields_ = [(k, C.c_int64) for k in ("n", "sum_t", "t_max", "t_block", "n_blocks", "pad_packed",
+                                          "pad_naive_tmax", "pad_naive_tblock", "min_blocks")] + \
+               [(k, C.c_double) for k in ("frac_packed", "frac_naive_tmax", "frac_naive_tblock",
+                                          "reduction_vs_tmax", "mean_segs_per_block")]
+
+
+def lib():
+    global _lib
+    if _lib is None:
+        build()
+        L = C.CDLL(_SO)
+        L.oracle_philox4x64_10.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p]
+        L.oracle_philox4x64_10.restype = None
+        L.oracle_seq_key.argtypes = [C.c_uint64, C.c_int64]
+        L.oracle_seq_key.restype = C.c_uint32
+        L.oracle_draw_word.argtypes = [C.c_uint64, C.c_int64]
+        L.oracle_draw_word.restype = C.c_uint64
+        L.oracle_pick.argtypes = [C.c_uint64, C.c_uint64]
+        L.oracle_pick.restype = C.c_uint64
+        L.oracle_offsets.argtypes = [C.c_void_p, C.c_int64, C.c_void_p]
+        L.oracle_offsets.restype = None
+        L.oracle_plan.argtypes = [C.POINTER(_PlanStruct)]
+        L.oracle_plan.restype = C.c_int
+        L.oracle_metadata.argtypes = [C.POINTER(_TablesStruct), C.c_int64, C.c_int64] + [C.c_void_p] * 4
+        L.oracle_metadata.restype = C.c_int
+        L.oracle_pack.argtypes = [C.POINTER(_TablesStruct), C.c_void_p, C.c_int64, C.c_int64, C.c_int64,
+                                  C.c_void_p, C.c_uint8]
+        L.oracle_pack.restype = C.c_int
+        L.oracle_unpack.argtypes = [C.POINTER(_TablesStruct), C.c_void_p, C.c_int64, C.c_int64, C.c_int64,
+                                    C.c_void_p]
+        L.oracle_unpack.restype = C.c_int
+        L.oracle_stats.argtypes = [C.POINTER(_StatsStruct)]
+        L.oracle_stats.restype = C.c_int
+        _lib = L
+    return _lib
+
+
+def _p(a: np.ndarray) -> int:
+    return a.ctypes.data
+
+
+def philox4x64_10(ctr, key) -> np.ndarray:
+    c = np.asarray(ctr, dtype=np.uint64).copy()
+    k = np.asarray(key, dtype=np.uint64).copy()
+    o = np.zeros(4, dtype=np.uint64)
+    lib().oracle_philox4x64_10(_p(c), _p(k), _p(o))
+    return o
+
+
+def seq_key(seed: int, i: int) -> int:
+    return int(lib().oracle_seq_key(seed, i))
+
+
+def draw_word(seed: int, k: int) -> int:
+    return int(lib().oracle_draw_word(seed, k))
+
+
+def pick(u: int, m: int) -> int:
+    return int(lib().oracle_pick(u, m))
+
+
+def offsets(lengths: np.ndarray) -> np.ndarray:
+    lengths = np.ascontiguousarray(lengths, dtype=np.int32)
+    out = np.zeros(lengths.size + 1, dtype=np.int64)
+    lib().oracle_offsets(_p(lengths), lengths.size, _p(out))
+    return out
+
+
+@dataclass
+class OraclePlan:
+    status: int
+    n: int
+    t_block: int
+    seed: int
+    n_blocks: int
+    sum_t: int
+    t_max: int
+    first_bad: int
+    checksum: int
+    max_segs_per_block: int
+    lengths: np.ndarray
+    offsets: np.ndarray
+    seg_seq: np.ndarray
+    seg_block: np.ndarray
+    seg_start: np.ndarray
+    block_seg_begin: np.ndarray
+    block_fill: np.ndarray
+    seq_block: np.ndarray
+    seq_start: np.ndarray
+
+    def _tables(self) -> _TablesStruct:
+        return _TablesStruct(self.n, self.n_blocks, self.t_block, _p(self.offsets), _p(self.seg_seq),
+                             _p(self.seg_start), _p(self.block_seg_begin))
+
+
+def plan(lengths: np.ndarray, t_block: int, seed: int, policy: int = 0) -> OraclePlan:
+    lengths = np.ascontiguousarray(lengths, dtype=np.int32)
+    n = int(lengths.size)
+    m = max(n, 1)
+    a = dict(offsets=np.zeros(m + 1, np.int64), seg_seq=np.zeros(m, np.int32), seg_block=np.zeros(m, np.int32),
+             seg_start=np.zeros(m, np.int32), block_seg_begin=np.zeros(m + 1, np.int32),
+             block_fill=np.zeros(m, np.int32), seq_block=np.zeros(m, np.int32), seq_start=np.zeros(m, np.int32))
+    s = _PlanStruct(lengths=_p(lengths), n=n, t_block=t_block, seed=seed, policy=policy,
+                    **{k: _p(v) for k, v in a.items()})
+    rc = lib().oracle_plan(C.byref(s))
+    nb = int(s.n_blocks)
+    a["block_seg_begin"] = a["block_seg_begin"][: nb + 1]
+    a["block_fill"] = a["block_fill"][:nb]
+    return OraclePlan(status=rc, n=n, t_block=t_block, seed=seed, n_blocks=nb, sum_t=int(s.sum_t),
+                      t_max=int(s.t_max), first_bad=int(s.first_bad), checksum=int(s.checksum),
+                      max_segs_per_block=int(s.max_segs_per_block), lengths=lengths, **a)
+
+
+def metadata(p: OraclePlan, block_begin: int, block_count: int):
+    shape = (block_count, p.t_block)
+    seq_id = np.empty(shape, np.int32)
+    pos = np.empty(shape, np.int32)
+    reset = np.empty(shape, np.uint8)
+    valid = np.empty(shape, np.uint8)
+    t = p._tables()
+    rc = lib().oracle_metadata(C.byref(t), block_begin, block_count, _p(seq_id), _p(pos), _p(reset), _p(valid))
+    assert rc == 0, rc
+    return seq_id, pos, reset, valid
+
+
+def pack(p: OraclePlan, store: np.ndarray, frame_bytes: int, block_begin: int, block_count: int,
+         pad_byte: int = 0) -> np.ndarray:
+    """store: uint8 view of the flat ragged frame store, sum_t * frame_bytes bytes."""
+    store = np.ascontiguousarray(store).view(np.uint8).reshape(-1)
+    assert store.size == p.sum_t * frame_bytes
+    dense = np.empty((block_count, p.t_block, frame_bytes), np.uint8)
+    t = p._tables()
+    rc = lib().oracle_pack(C.byref(t), _p(store), frame_bytes, block_begin, block_count, _p(dense), pad_byte)
+    assert rc == 0, rc
+    return dense
+
+
+def unpack(p: OraclePlan, dense_out: np.ndarray, frame_bytes: int, block_begin: int, block_count: int,
+           ragged_out: np.ndarray) -> np.ndarray:
+    """Scatter valid slots of dense_out (blocks block_begin..) into ragged_out (uint8, in place)."""
+    dense_out = np.ascontiguousarray(dense_out).view(np.uint8).reshape(-1)
+    assert dense_out.size == block_count * p.t_block * frame_bytes
+    assert ragged_out.dtype == np.uint8 and ragged_out.flags.c_contiguous
+    assert ragged_out.size == p.sum_t * frame_bytes
+    t = p._tables()
+    rc = lib().oracle_unpack(C.byref(t), _p(dense_out), frame_bytes, block_begin, block_count, _p(ragged_out))
+    assert rc == 0, rc
+    return ragged_out
+
+
+def stats(n: int, sum_t: int, t_max: int, t_block: int, n_blocks: int) -> dict:
+    s = _StatsStruct(n=n, sum_t=sum_t, t_max=t_max, t_block=t_block, n_blocks=n_blocks)
+    rc = lib().oracle_stats(C.byref(s))
+    assert rc == 0, rc
+    return {k: getattr(s, k) for k, _ in _StatsStruct._fields_}
