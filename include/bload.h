@@ -1,0 +1,182 @@
+/*
+ * bload.h -- C ABI of libbload: BLoad's ragged-to-block packing on one NVIDIA B200 (sm_100a).
+ *
+ * The paper ("BLoad: Enhancing Neural Network Training with Efficient Sequential Data Handling",
+ * section Methods) trains on N sequences of T_i frames without padding each to the longest one:
+ * randomly sampled sequences are concatenated into blocks of a fixed number of frames, the tail
+ * of a block that cannot be filled exactly is padded with zeros, and a table records the slot at
+ * which each new sequence starts inside its block.  This library computes that assignment on the
+ * GPU (bload_plan), materialises dense [blocks, t_block, frame] batches and their per-slot
+ * metadata from a flat ragged frame store (bload_pack), scatters per-frame outputs back to the
+ * ragged order (bload_unpack), and reports padding statistics (bload_stats).
+ *
+ * Conventions
+ *   - "d_" pointers are DEVICE pointers; all others are HOST pointers.
+ *   - The caller owns every buffer.  The library allocates no device memory and keeps no state
+ *     between calls; a plan is position independent (tables addressed by byte offsets) and can
+ *     be copied or saved as a blob of bload_sizes_t.plan_bytes bytes.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = default stream).
+ *   - Every function returns BLOAD_OK (0) or a negative BLOAD_ERR_* code.  Errors that the host
+ *     can detect launch nothing.  Nothing aborts, throws or traps.
+ *   - Frames are opaque byte strings of `frame_bytes` bytes; they are moved bit for bit.
+ */
+#ifndef BLOAD_H_
+#define BLOAD_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#if defined(__GNUC__)
+#define BLOAD_API __attribute__((visibility("default")))
+#else
+#define BLOAD_API
+#endif
+
+#define BLOAD_OK 0
+#define BLOAD_ERR_NULL (-1)        /* a required pointer is NULL */
+#define BLOAD_ERR_ARG (-2)         /* n < 1, t_block < 1, frame_bytes < 1, bad block range, ... */
+#define BLOAD_ERR_LENGTH (-3)      /* some T_i outside [1, t_block]; index in info.first_bad_index */
+#define BLOAD_ERR_WORKSPACE (-4)   /* plan or work buffer smaller than bload_plan_sizes says */
+#define BLOAD_ERR_ALIGN (-5)       /* a device pointer is not aligned as documented */
+#define BLOAD_ERR_UNSUPPORTED (-6) /* t_block above BLOAD_MAX_T_BLOCK, unknown policy */
+#define BLOAD_ERR_CUDA (-7)        /* a CUDA runtime call or launch failed */
+#define BLOAD_ERR_TIMEOUT (-8)     /* a bounded device-side wait expired */
+#define BLOAD_ERR_PLAN (-9)        /* info/plan do not describe a finished plan */
+
+#define BLOAD_MAX_T_BLOCK 32768
+#define BLOAD_POLICY_UNIFORM_SEQUENCES 0u /* every unused sequence that fits is equally likely */
+
+/* Sizes and table offsets for a problem of n sequences (host only, no GPU call). */
+typedef struct {
+    size_t plan_bytes; /* bytes of the plan buffer */
+    size_t work_bytes; /* bytes of the scratch buffer bload_plan needs (contents are garbage afterwards) */
+    int64_t max_blocks; /* upper bound on n_blocks (= n); the tables below have room for it */
+    /* byte offsets of the tables inside the plan buffer (each 256-byte aligned) */
+    size_t off_offsets;         /* int64 [n+1]  first frame of sequence i in the ragged store; [n] = sum T */
+    size_t off_seg_seq;         /* int32 [n]    sequence placed by the k-th draw (segments in placement order) */
+    size_t off_seg_block;       /* int32 [n]    block of segment k */
+    size_t off_seg_start;       /* int32 [n]    first slot of segment k in its block: the paper's start-index table */
+    size_t off_seg_src;         /* int64 [n]    first frame of segment k in the ragged store (= offsets[seg_seq[k]]) */
+    size_t off_block_seg_begin; /* int32 [max_blocks+1]  CSR: segments of block b are [begin[b], begin[b+1]) */
+    size_t off_block_fill;      /* int32 [max_blocks]    occupied slots of block b; slots beyond are padding */
+    size_t off_seq_block;       /* int32 [n]    inverse table: block of sequence i */
+    size_t off_seq_start;       /* int32 [n]    inverse table: first slot of sequence i */
+} bload_sizes_t;
+
+/* Scalars of a finished plan (host). */
+typedef struct {
+    int32_t status;  /* BLOAD_OK or the error the planner found */
+    int32_t t_block; /* block length in frames */
+    int64_t n;       /* sequences */
+    int64_t n_blocks;
+    int64_t sum_t;   /* total frames */
+    int64_t t_max;   /* longest sequence */
+    int64_t first_bad_index; /* first i with T_i outside [1, t_block], else -1 */
+    uint64_t checksum;       /* order-independent digest of (block, start, sequence) over all segments */
+    int64_t max_segs_per_block;
+    uint64_t seed;
+    uint32_t policy;
+    uint32_t reserved_;
+} bload_plan_info_t;
+
+typedef struct {
+    int64_t n, sum_t, t_max, t_block, n_blocks;
+    int64_t pad_packed;       /* n_blocks * t_block - sum_t */
+    int64_t pad_naive_tmax;   /* n * t_max - sum_t  (every sample padded to the longest) */
+    int64_t pad_naive_tblock; /* n * t_block - sum_t */
+    int64_t min_blocks;       /* ceil(sum_t / t_block): no packing can use fewer blocks */
+    double frac_packed;       /* pad_packed / (n_blocks * t_block) */
+    double frac_naive_tmax;   /* pad_naive_tmax / (n * t_max) */
+    double frac_naive_tblock;
+    double reduction_vs_tmax; /* pad_naive_tmax / pad_packed (0 when pad_packed == 0) */
+    double mean_segs_per_block;
+    int64_t max_segs_per_block;
+} bload_stats_t;
+
+/*
+ * bload_plan_sizes -- buffer sizes and table offsets for n sequences and blocks of t_block frames.
+ * Host only.  Errors: NULL out, n < 1 or n >= 2^31, t_block < 1 (ARG), t_block > BLOAD_MAX_T_BLOCK
+ * (UNSUPPORTED).
+ */
+BLOAD_API int bload_plan_sizes(int64_t n, int32_t t_block, bload_sizes_t* out);
+
+/*
+ * bload_plan -- block construction (paper, Methods, first paragraph; caption of the pseudocode
+ * figure) and the table of start indices (Methods, second paragraph).
+ *
+ * Blocks are built one after another.  While some unused sequence is no longer than the room left
+ * in the open block, one of them is drawn uniformly at random and appended (the paper's Random_*()
+ * over L_dict); when none fits, the rest of the block is padding and the next block is opened.
+ * Randomness comes from the counter-based generator Philox-4x64-10 keyed by `seed`, so the plan is
+ * a pure function of (lengths, t_block, seed, policy).
+ *
+ *   d_lengths  device int32[n], 4-byte aligned; every T_i must satisfy 1 <= T_i <= t_block
+ *   d_plan     device buffer of plan_bytes bytes, 256-byte aligned; receives the tables
+ *   d_work     device scratch of work_bytes bytes, 256-byte aligned
+ *   info       host out; filled after ONE synchronisation of `stream` (the only one in the library)
+ *
+ * Returns info->status.  On BLOAD_ERR_LENGTH the tables are undefined and first_bad_index is set.
+ */
+BLOAD_API int bload_plan(const int32_t* d_lengths, int64_t n, int32_t t_block, uint64_t seed, uint32_t policy,
+               void* d_plan, size_t plan_bytes, void* d_work, size_t work_bytes, void* stream,
+               bload_plan_info_t* info);
+
+/*
+ * bload_pack -- dense batches and per-slot metadata for blocks [block_begin, block_begin+block_count)
+ * (paper, Methods: concatenate the sequences of a block, pad the rest with zeros; the start table).
+ *
+ *   d_dense[q, s, :] = d_store[(offsets[id] + f) * frame_bytes ...]  if slot s of block block_begin+q
+ *                      holds frame f of sequence id;  pad_byte repeated frame_bytes times otherwise
+ *   d_seq_id[q, s] = id or -1     d_pos[q, s] = f or -1
+ *   d_reset[q, s]  = 1 at the first slot of every sequence, else 0 (where carried state must be reset)
+ *   d_valid[q, s]  = 1 on frames, 0 on padding
+ *
+ * Blocks at or beyond n_blocks are filler (all padding, all flags 0, ids -1) so that a caller can
+ * round an epoch up to whole batches.  d_store is the flat ragged store (sum_t * frame_bytes bytes,
+ * sequence i at frame offsets[i]); d_dense is [block_count, t_block, frame_bytes] row major.
+ * d_store and d_dense must be 16-byte aligned.  d_dense and each of the four metadata outputs may be
+ * NULL (that output is skipped).  Asynchronous on `stream`; no host synchronisation.
+ * Errors: NULL plan/info/store (when d_dense is given), ARG (frame_bytes < 1, negative range,
+ * block_begin + block_count >= 2^31), ALIGN, PLAN (info->status != 0), CUDA.
+ */
+BLOAD_API int bload_pack(const void* d_plan, const bload_plan_info_t* info, const void* d_store, int64_t frame_bytes,
+               int64_t block_begin, int64_t block_count, void* d_dense, int32_t* d_seq_id, int32_t* d_pos,
+               uint8_t* d_reset, uint8_t* d_valid, uint8_t pad_byte, void* stream);
+
+/*
+ * bload_unpack -- inverse of bload_pack for per-frame outputs: for every valid slot of the given
+ * blocks, d_ragged_out[(offsets[id] + f) * out_frame_bytes ...] = d_dense_out[q, s, :].  Padding
+ * slots and filler blocks are ignored; frames of sequences outside the block range are not touched.
+ * The paper does not describe this step; it is defined as the exact inverse of the gather above.
+ * Both buffers 16-byte aligned.  Asynchronous on `stream`.
+ */
+BLOAD_API int bload_unpack(const void* d_plan, const bload_plan_info_t* info, const void* d_dense_out,
+                 int64_t out_frame_bytes, int64_t block_begin, int64_t block_count, void* d_ragged_out,
+                 void* stream);
+
+/*
+ * bload_stats -- padding statistics from the scalars of a plan (host only; closed forms).
+ * pad_naive_tmax is the "0 padding" row of the paper's Table I, pad_packed its "block_pad" row.
+ */
+BLOAD_API int bload_stats(const bload_plan_info_t* info, bload_stats_t* out);
+
+/*
+ * bload_plan_stage_times -- device time, in milliseconds, that the most recent bload_plan call of
+ * this thread spent in each stage: [0] validate + scan + keys, [1] key sort, [2] fill rule,
+ * [3] inverse tables.  Host only; for benchmarking.  Returns BLOAD_ERR_PLAN when no plan was timed.
+ * Timing is enabled by bload_set_plan_timing(1) (off by default; it adds event records only).
+ */
+BLOAD_API int bload_set_plan_timing(int enable);
+BLOAD_API int bload_plan_stage_times(float out_ms[4]);
+
+BLOAD_API const char* bload_strerror(int code);
+BLOAD_API int bload_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* BLOAD_H_ */

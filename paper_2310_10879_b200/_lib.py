@@ -1,0 +1,200 @@
+"""ctypes binding of libbload.so: argument marshalling only.
+
+Every step of the path runs inside the library's CUDA kernels; torch is used for device memory
+and streams.  There is no CPU fallback: if the shared library is missing, loading raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from dataclasses import dataclass
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libbload.so")
+
+OK = 0
+ERR_NULL, ERR_ARG, ERR_LENGTH, ERR_WORKSPACE, ERR_ALIGN = -1, -2, -3, -4, -5
+ERR_UNSUPPORTED, ERR_CUDA, ERR_TIMEOUT, ERR_PLAN = -6, -7, -8, -9
+MAX_T_BLOCK = 32768
+
+EXPORTS = ("bload_plan_sizes", "bload_plan", "bload_pack", "bload_unpack", "bload_stats",
+           "bload_set_plan_timing", "bload_plan_stage_times", "bload_strerror", "bload_version")
+
+
+class Sizes(C.Structure):
+    _fields_ = [("plan_bytes", C.c_size_t), ("work_bytes", C.c_size_t), ("max_blocks", C.c_int64)] + \
+               [(k, C.c_size_t) for k in ("off_offsets", "off_seg_seq", "off_seg_block", "off_seg_start",
+                                          "off_seg_src", "off_block_seg_begin", "off_block_fill",
+                                          "off_seq_block", "off_seq_start")]
+
+
+class PlanInfo(C.Structure):
+    _fields_ = [("status", C.c_int32), ("t_block", C.c_int32), ("n", C.c_int64), ("n_blocks", C.c_int64),
+                ("sum_t", C.c_int64), ("t_max", C.c_int64), ("first_bad_index", C.c_int64),
+                ("checksum", C.c_uint64), ("max_segs_per_block", C.c_int64), ("seed", C.c_uint64),
+                ("policy", C.c_uint32), ("reserved_", C.c_uint32)]
+
+
+class Stats(C.Structure):
+    _fields_ = [(k, C.c_int64) for k in ("n", "sum_t", "t_max", "t_block", "n_blocks", "pad_packed",
+                                          "pad_naive_tmax", "pad_naive_tblock", "min_blocks")] + \
+               [(k, C.c_double) for k in ("frac_packed", "frac_naive_tmax", "frac_naive_tblock",
+                                          "reduction_vs_tmax", "mean_segs_per_block")] + \
+               [("max_segs_per_block", C.c_int64)]
+
+
+class BloadError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__("%s: %s (%d)" % (where, strerror(code), code))
+
+
+_lib = None
+
+
+def load() -> C.CDLL:
+    """Load libbload.so.  Raises if it has not been built (python -m paper_2310_10879_b200.build)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise RuntimeError("libbload.so is missing at %s: build it with `python -m paper_2310_10879_b200.build` "
+                           "(there is no CPU fallback)" % LIB_PATH)
+    L = C.CDLL(LIB_PATH)
+    vp, i64, i32, u64, u32, u8 = C.c_void_p, C.c_int64, C.c_int32, C.c_uint64, C.c_uint32, C.c_uint8
+    L.bload_plan_sizes.argtypes = [i64, i32, C.POINTER(Sizes)]
+    L.bload_plan.argtypes = [vp, i64, i32, u64, u32, vp, C.c_size_t, vp, C.c_size_t, vp, C.POINTER(PlanInfo)]
+    L.bload_pack.argtypes = [vp, C.POINTER(PlanInfo), vp, i64, i64, i64, vp, vp, vp, vp, vp, u8, vp]
+    L.bload_unpack.argtypes = [vp, C.POINTER(PlanInfo), vp, i64, i64, i64, vp, vp]
+    L.bload_stats.argtypes = [C.POINTER(PlanInfo), C.POINTER(Stats)]
+    L.bload_set_plan_timing.argtypes = [C.c_int]
+    L.bload_plan_stage_times.argtypes = [C.POINTER(C.c_float * 4)]
+    L.bload_strerror.argtypes = [C.c_int]
+    L.bload_strerror.restype = C.c_char_p
+    L.bload_version.argtypes = []
+    for name in EXPORTS:
+        if name != "bload_strerror":
+            getattr(L, name).restype = C.c_int
+    _lib = L
+    return L
+
+
+def strerror(code: int) -> str:
+    return load().bload_strerror(code).decode()
+
+
+def _ptr(t) -> int | None:
+    return None if t is None else t.data_ptr()
+
+
+def _stream(stream) -> int | None:
+    import torch
+    s = torch.cuda.current_stream() if stream is None else stream
+    return s.cuda_stream or None
+
+
+def bload_plan_sizes(n: int, t_block: int) -> Sizes:
+    s = Sizes()
+    rc = load().bload_plan_sizes(n, t_block, C.byref(s))
+    if rc:
+        raise BloadError(rc, "bload_plan_sizes")
+    return s
+
+
+@dataclass
+class Plan:
+    """A device plan: the raw buffer, its host scalars, and typed views of its tables (device tensors
+    that alias the buffer)."""
+    buf: "object"
+    info: PlanInfo
+    sizes: Sizes
+
+    def _view(self, off: int, count: int, dtype):
+        import torch
+        esz = torch.empty((), dtype=dtype).element_size()
+        return self.buf[off: off + count * esz].view(dtype)
+
+    @property
+    def n(self): return int(self.info.n)
+    @property
+    def t_block(self): return int(self.info.t_block)
+    @property
+    def n_blocks(self): return int(self.info.n_blocks)
+    @property
+    def sum_t(self): return int(self.info.sum_t)
+
+    def tables(self) -> dict:
+        import torch
+        n, nb, s = self.n, self.n_blocks, self.sizes
+        return dict(
+            offsets=self._view(s.off_offsets, n + 1, torch.int64),
+            seg_seq=self._view(s.off_seg_seq, n, torch.int32),
+            seg_block=self._view(s.off_seg_block, n, torch.int32),
+            seg_start=self._view(s.off_seg_start, n, torch.int32),
+            seg_src=self._view(s.off_seg_src, n, torch.int64),
+            block_seg_begin=self._view(s.off_block_seg_begin, nb + 1, torch.int32),
+            block_fill=self._view(s.off_block_fill, nb, torch.int32),
+            seq_block=self._view(s.off_seq_block, n, torch.int32),
+            seq_start=self._view(s.off_seq_start, n, torch.int32),
+        )
+
+
+def bload_plan(lengths, t_block: int, seed: int, policy: int = 0, stream=None, work=None, plan_buf=None,
+               check: bool = True) -> Plan:
+    """lengths: CUDA int32 tensor [n].  Returns a Plan whose tables live in device memory."""
+    import torch
+    if not lengths.is_cuda or lengths.dtype != torch.int32 or not lengths.is_contiguous():
+        raise TypeError("lengths must be a contiguous CUDA int32 tensor")
+    n = lengths.numel()
+    sizes = bload_plan_sizes(n, t_block)
+    dev = lengths.device
+    if plan_buf is None:
+        plan_buf = torch.empty(sizes.plan_bytes, dtype=torch.uint8, device=dev)
+    if work is None:
+        work = torch.empty(sizes.work_bytes, dtype=torch.uint8, device=dev)
+    info = PlanInfo()
+    rc = load().bload_plan(lengths.data_ptr(), n, t_block, seed, policy, plan_buf.data_ptr(), plan_buf.numel(),
+                           work.data_ptr(), work.numel(), _stream(stream), C.byref(info))
+    if rc and check:
+        err = BloadError(rc, "bload_plan")
+        err.info = info
+        raise err
+    return Plan(plan_buf, info, sizes)
+
+
+def bload_pack(plan: Plan, store, frame_bytes: int, block_begin: int, block_count: int, dense=None, seq_id=None,
+               pos=None, reset=None, valid=None, pad_byte: int = 0, stream=None) -> None:
+    """store: CUDA tensor holding the flat ragged frames; dense/seq_id/pos/reset/valid: CUDA outputs or None."""
+    rc = load().bload_pack(plan.buf.data_ptr(), C.byref(plan.info), _ptr(store), frame_bytes, block_begin,
+                           block_count, _ptr(dense), _ptr(seq_id), _ptr(pos), _ptr(reset), _ptr(valid), pad_byte,
+                           _stream(stream))
+    if rc:
+        raise BloadError(rc, "bload_pack")
+
+
+def bload_unpack(plan: Plan, dense_out, out_frame_bytes: int, block_begin: int, block_count: int, ragged_out,
+                 stream=None) -> None:
+    rc = load().bload_unpack(plan.buf.data_ptr(), C.byref(plan.info), _ptr(dense_out), out_frame_bytes, block_begin,
+                             block_count, _ptr(ragged_out), _stream(stream))
+    if rc:
+        raise BloadError(rc, "bload_unpack")
+
+
+def bload_stats(info: PlanInfo) -> dict:
+    s = Stats()
+    rc = load().bload_stats(C.byref(info), C.byref(s))
+    if rc:
+        raise BloadError(rc, "bload_stats")
+    return {k: getattr(s, k) for k, _ in Stats._fields_}
+
+
+def bload_set_plan_timing(enable: bool) -> None:
+    load().bload_set_plan_timing(1 if enable else 0)
+
+
+def bload_plan_stage_times() -> list[float]:
+    out = (C.c_float * 4)()
+    rc = load().bload_plan_stage_times(C.byref(out))
+    if rc:
+        raise BloadError(rc, "bload_plan_stage_times")
+    return [float(x) for x in out]

@@ -1,0 +1,232 @@
+// C ABI of libbload: argument checks, buffer layouts, launches.  See include/bload.h.
+#include <string.h>
+
+#include "bload_internal.cuh"
+
+namespace bload {
+
+void plan_layout(int64_t n, bload_sizes_t* s)
+{
+    size_t off = kHeaderBytes;
+    auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes); return o; };
+    const size_t un = (size_t)n;
+    s->max_blocks = n;
+    s->off_offsets = take(sizeof(int64_t) * (un + 1));
+    s->off_seg_seq = take(sizeof(int32_t) * un);
+    s->off_seg_block = take(sizeof(int32_t) * un);
+    s->off_seg_start = take(sizeof(int32_t) * un);
+    s->off_seg_src = take(sizeof(int64_t) * un);
+    s->off_block_seg_begin = take(sizeof(int32_t) * (un + 1));
+    s->off_block_fill = take(sizeof(int32_t) * un);
+    s->off_seq_block = take(sizeof(int32_t) * un);
+    s->off_seq_start = take(sizeof(int32_t) * un);
+    s->plan_bytes = off;
+}
+
+PlanView plan_view(void* d_plan, int64_t n)
+{
+    bload_sizes_t s;
+    plan_layout(n, &s);
+    char* b = static_cast<char*>(d_plan);
+    PlanView v;
+    v.hdr = reinterpret_cast<PlanHeader*>(b);
+    v.offsets = reinterpret_cast<int64_t*>(b + s.off_offsets);
+    v.seg_seq = reinterpret_cast<int32_t*>(b + s.off_seg_seq);
+    v.seg_block = reinterpret_cast<int32_t*>(b + s.off_seg_block);
+    v.seg_start = reinterpret_cast<int32_t*>(b + s.off_seg_start);
+    v.seg_src = reinterpret_cast<int64_t*>(b + s.off_seg_src);
+    v.block_seg_begin = reinterpret_cast<int32_t*>(b + s.off_block_seg_begin);
+    v.block_fill = reinterpret_cast<int32_t*>(b + s.off_block_fill);
+    v.seq_block = reinterpret_cast<int32_t*>(b + s.off_seq_block);
+    v.seq_start = reinterpret_cast<int32_t*>(b + s.off_seq_start);
+    return v;
+}
+
+namespace {
+thread_local bool g_timing = false;
+thread_local bool g_have_times = false;
+thread_local float g_stage_ms[4] = {0, 0, 0, 0};
+
+inline bool aligned(const void* p, uintptr_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
+
+int check_sizes(int64_t n, int32_t t_block)
+{
+    if (n < 1 || n > 0x7fffffffLL || t_block < 1) return BLOAD_ERR_ARG;
+    if (t_block > BLOAD_MAX_T_BLOCK) return BLOAD_ERR_UNSUPPORTED;
+    return BLOAD_OK;
+}
+
+int check_plan_args(const void* d_plan, const bload_plan_info_t* info, int64_t frame_bytes, int64_t block_begin,
+                    int64_t block_count)
+{
+    if (!d_plan || !info) return BLOAD_ERR_NULL;
+    if (info->status != BLOAD_OK || info->n < 1 || info->t_block < 1 || info->n_blocks < 1) return BLOAD_ERR_PLAN;
+    if (frame_bytes < 1 || block_begin < 0 || block_count < 0) return BLOAD_ERR_ARG;
+    if (block_begin + block_count > 0x7fffffffLL) return BLOAD_ERR_ARG;
+    if (!aligned(d_plan, kAlign)) return BLOAD_ERR_ALIGN;
+    return BLOAD_OK;
+}
+}  // namespace
+
+}  // namespace bload
+
+using namespace bload;
+
+extern "C" {
+
+int bload_version(void) { return 1; }
+
+const char* bload_strerror(int code)
+{
+    switch (code) {
+        case BLOAD_OK: return "ok";
+        case BLOAD_ERR_NULL: return "a required pointer is NULL";
+        case BLOAD_ERR_ARG: return "argument out of range";
+        case BLOAD_ERR_LENGTH: return "a sequence length is outside [1, t_block]";
+        case BLOAD_ERR_WORKSPACE: return "plan or work buffer too small";
+        case BLOAD_ERR_ALIGN: return "device pointer not aligned as required";
+        case BLOAD_ERR_UNSUPPORTED: return "unsupported t_block or policy";
+        case BLOAD_ERR_CUDA: return "CUDA call failed";
+        case BLOAD_ERR_TIMEOUT: return "bounded device wait expired";
+        case BLOAD_ERR_PLAN: return "plan is missing, unfinished or failed";
+        default: return "unknown error code";
+    }
+}
+
+int bload_plan_sizes(int64_t n, int32_t t_block, bload_sizes_t* out)
+{
+    if (!out) return BLOAD_ERR_NULL;
+    memset(out, 0, sizeof *out);
+    int rc = check_sizes(n, t_block);
+    if (rc) return rc;
+    plan_layout(n, out);
+    out->work_bytes = work_layout(n, t_block, nullptr, nullptr);
+    return BLOAD_OK;
+}
+
+int bload_set_plan_timing(int enable)
+{
+    g_timing = enable != 0;
+    return BLOAD_OK;
+}
+
+int bload_plan_stage_times(float out_ms[4])
+{
+    if (!out_ms) return BLOAD_ERR_NULL;
+    if (!g_have_times) return BLOAD_ERR_PLAN;
+    for (int i = 0; i < 4; ++i) out_ms[i] = g_stage_ms[i];
+    return BLOAD_OK;
+}
+
+int bload_plan(const int32_t* d_lengths, int64_t n, int32_t t_block, uint64_t seed, uint32_t policy, void* d_plan,
+               size_t plan_bytes, void* d_work, size_t work_bytes, void* stream, bload_plan_info_t* info)
+{
+    if (!info) return BLOAD_ERR_NULL;
+    memset(info, 0, sizeof *info);
+    info->first_bad_index = -1;
+    info->n = n; info->t_block = t_block; info->seed = seed; info->policy = policy;
+    auto fail = [&](int rc) { info->status = rc; return rc; };
+    if (!d_lengths || !d_plan || !d_work) return fail(BLOAD_ERR_NULL);
+    int rc = check_sizes(n, t_block);
+    if (rc) return fail(rc);
+    if (policy != BLOAD_POLICY_UNIFORM_SEQUENCES) return fail(BLOAD_ERR_UNSUPPORTED);
+    bload_sizes_t sz;
+    plan_layout(n, &sz);
+    WorkView wv;
+    const size_t need_work = work_layout(n, t_block, d_work, &wv);
+    if (plan_bytes < sz.plan_bytes || work_bytes < need_work) return fail(BLOAD_ERR_WORKSPACE);
+    if (!aligned(d_plan, kAlign) || !aligned(d_work, kAlign) || !aligned(d_lengths, 4)) return fail(BLOAD_ERR_ALIGN);
+
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    PlanView pv = plan_view(d_plan, n);
+    cudaEvent_t ev[5];
+    bool timing = g_timing;
+    if (timing)
+        for (int i = 0; i < 5; ++i)
+            if (cudaEventCreate(&ev[i]) != cudaSuccess) { timing = false; break; }
+    cudaError_t ce = launch_plan(d_lengths, n, t_block, seed, policy, pv, wv, st, timing ? ev : nullptr);
+    PlanHeader h;
+    if (ce == cudaSuccess) ce = cudaMemcpyAsync(&h, pv.hdr, sizeof h, cudaMemcpyDeviceToHost, st);
+    if (ce == cudaSuccess) ce = cudaStreamSynchronize(st);
+    if (timing) {
+        if (ce == cudaSuccess) {
+            for (int i = 0; i < 4; ++i) cudaEventElapsedTime(&g_stage_ms[i], ev[i], ev[i + 1]);
+            g_have_times = true;
+        }
+        for (int i = 0; i < 5; ++i) cudaEventDestroy(ev[i]);
+    }
+    if (ce != cudaSuccess) { (void)cudaGetLastError(); return fail(BLOAD_ERR_CUDA); }
+
+    info->status = h.status;
+    info->n_blocks = h.n_blocks;
+    info->sum_t = h.sum_t;
+    info->t_max = h.t_max;
+    info->first_bad_index = h.first_bad == ~0ULL ? -1 : (int64_t)h.first_bad;
+    info->checksum = h.checksum;
+    info->max_segs_per_block = h.max_segs;
+    if (h.status == BLOAD_OK && h.magic != kPlanMagic) return fail(BLOAD_ERR_PLAN);
+    return info->status;
+}
+
+int bload_pack(const void* d_plan, const bload_plan_info_t* info, const void* d_store, int64_t frame_bytes,
+               int64_t block_begin, int64_t block_count, void* d_dense, int32_t* d_seq_id, int32_t* d_pos,
+               uint8_t* d_reset, uint8_t* d_valid, uint8_t pad_byte, void* stream)
+{
+    int rc = check_plan_args(d_plan, info, frame_bytes, block_begin, block_count);
+    if (rc) return rc;
+    if (block_count == 0) return BLOAD_OK;
+    if (d_dense && !d_store) return BLOAD_ERR_NULL;
+    if (d_dense && (!aligned(d_dense, 16) || !aligned(d_store, 16))) return BLOAD_ERR_ALIGN;
+    if (!aligned(d_seq_id, 4) || !aligned(d_pos, 4)) return BLOAD_ERR_ALIGN;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    PlanView pv = plan_view(const_cast<void*>(d_plan), info->n);
+    cudaError_t ce = cudaSuccess;
+    if (d_seq_id || d_pos || d_reset || d_valid)
+        ce = launch_metadata(pv, info->t_block, block_begin, block_count, d_seq_id, d_pos, d_reset, d_valid, st);
+    if (ce == cudaSuccess && d_dense)
+        ce = launch_copy(false, pv, info->t_block, frame_bytes, block_begin, block_count,
+                         static_cast<const uint8_t*>(d_store), static_cast<uint8_t*>(d_dense), nullptr,
+                         info->sum_t * frame_bytes, pad_byte, st);
+    if (ce != cudaSuccess) { (void)cudaGetLastError(); return BLOAD_ERR_CUDA; }
+    return BLOAD_OK;
+}
+
+int bload_unpack(const void* d_plan, const bload_plan_info_t* info, const void* d_dense_out, int64_t out_frame_bytes,
+                 int64_t block_begin, int64_t block_count, void* d_ragged_out, void* stream)
+{
+    int rc = check_plan_args(d_plan, info, out_frame_bytes, block_begin, block_count);
+    if (rc) return rc;
+    if (block_count == 0) return BLOAD_OK;
+    if (!d_dense_out || !d_ragged_out) return BLOAD_ERR_NULL;
+    if (!aligned(d_dense_out, 16) || !aligned(d_ragged_out, 16)) return BLOAD_ERR_ALIGN;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    PlanView pv = plan_view(const_cast<void*>(d_plan), info->n);
+    cudaError_t ce = launch_copy(true, pv, info->t_block, out_frame_bytes, block_begin, block_count, nullptr,
+                                 const_cast<uint8_t*>(static_cast<const uint8_t*>(d_dense_out)),
+                                 static_cast<uint8_t*>(d_ragged_out), info->sum_t * out_frame_bytes, 0, st);
+    if (ce != cudaSuccess) { (void)cudaGetLastError(); return BLOAD_ERR_CUDA; }
+    return BLOAD_OK;
+}
+
+int bload_stats(const bload_plan_info_t* info, bload_stats_t* out)
+{
+    if (!info || !out) return BLOAD_ERR_NULL;
+    memset(out, 0, sizeof *out);
+    if (info->status != BLOAD_OK || info->n < 1 || info->t_block < 1 || info->n_blocks < 1 || info->sum_t < 1)
+        return BLOAD_ERR_PLAN;
+    const int64_t n = info->n, s = info->sum_t, tb = info->t_block, nb = info->n_blocks, tm = info->t_max;
+    out->n = n; out->sum_t = s; out->t_max = tm; out->t_block = tb; out->n_blocks = nb;
+    out->pad_packed = nb * tb - s;
+    out->pad_naive_tmax = n * tm - s;
+    out->pad_naive_tblock = n * tb - s;
+    out->min_blocks = (s + tb - 1) / tb;
+    out->frac_packed = (double)out->pad_packed / (double)(nb * tb);
+    out->frac_naive_tmax = tm > 0 ? (double)out->pad_naive_tmax / (double)(n * tm) : 0.0;
+    out->frac_naive_tblock = (double)out->pad_naive_tblock / (double)(n * tb);
+    out->reduction_vs_tmax = out->pad_packed > 0 ? (double)out->pad_naive_tmax / (double)out->pad_packed : 0.0;
+    out->mean_segs_per_block = (double)n / (double)nb;
+    out->max_segs_per_block = info->max_segs_per_block;
+    return BLOAD_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,77 @@
+// Internal declarations shared by the translation units of libbload (GPU path only).
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "bload.h"
+
+namespace bload {
+
+constexpr uint64_t kPlanMagic = 0x424c6f6164763031ULL;  // "BLoadv01"
+constexpr size_t kAlign = 256;
+constexpr int kHeaderBytes = 256;
+
+// First 256 bytes of a plan buffer.
+struct PlanHeader {
+    uint64_t magic;
+    int64_t n;
+    int64_t n_blocks;
+    int64_t sum_t;
+    unsigned long long first_bad;  // ULLONG_MAX while no bad length was seen
+    unsigned long long checksum;
+    uint64_t seed;
+    int32_t t_block;
+    int32_t t_max;
+    int32_t status;
+    int32_t max_segs;
+    uint32_t policy;
+    uint32_t pad_[45];
+};
+static_assert(sizeof(PlanHeader) == kHeaderBytes, "header is 256 bytes");
+
+// Device view of the tables of a plan (pointers resolved on the host from the offsets).
+struct PlanView {
+    PlanHeader* hdr;
+    int64_t* offsets;
+    int32_t* seg_seq;
+    int32_t* seg_block;
+    int32_t* seg_start;
+    int64_t* seg_src;
+    int32_t* block_seg_begin;
+    int32_t* block_fill;
+    int32_t* seq_block;
+    int32_t* seq_start;
+};
+
+// Scratch layout of bload_plan.
+struct WorkView {
+    uint64_t* key_a;      // [n] sort keys (T << 32 | h), ping
+    uint64_t* key_b;      // [n] pong
+    int32_t* id_a;        // [n] payload ids, ping
+    int32_t* id_b;        // [n] pong
+    uint64_t* draw_u;     // [n] random word of draw k
+    int4* draw_rec;       // [n] per draw: {length, unused count of that length before the draw, block, start}
+    int64_t* partial;     // [chunks] per-chunk sums of lengths
+    uint32_t* digit_hist; // [256 * chunks] per-chunk digit counts of one sort pass
+    int32_t* bucket_end;  // [t_block + 1] sequences with length <= l
+};
+
+constexpr int kChunk = 2048;  // elements per CTA in scan / sort kernels (256 threads x 8)
+
+inline size_t align_up(size_t x, size_t a = kAlign) { return (x + a - 1) / a * a; }
+inline int64_t chunks_of(int64_t n) { return (n + kChunk - 1) / kChunk; }
+
+size_t work_layout(int64_t n, int32_t t_block, void* base, WorkView* w);
+void plan_layout(int64_t n, bload_sizes_t* s);
+PlanView plan_view(void* d_plan, int64_t n);
+
+// launchers (each returns a cudaError_t from cudaPeekAtLastError)
+cudaError_t launch_plan(const int32_t* d_lengths, int64_t n, int32_t t_block, uint64_t seed, uint32_t policy,
+                        const PlanView& pv, const WorkView& wv, cudaStream_t st, cudaEvent_t* ev /*5 or null*/);
+cudaError_t launch_metadata(const PlanView& pv, int32_t t_block, int64_t block_begin, int64_t block_count,
+                            int32_t* seq_id, int32_t* pos, uint8_t* reset, uint8_t* valid, cudaStream_t st);
+cudaError_t launch_copy(bool unpack, const PlanView& pv, int32_t t_block, int64_t frame_bytes, int64_t block_begin,
+                        int64_t block_count, const uint8_t* ragged_in, uint8_t* dense, uint8_t* ragged_out,
+                        int64_t ragged_bytes, uint8_t pad_byte, cudaStream_t st);
+
+}  // namespace bload

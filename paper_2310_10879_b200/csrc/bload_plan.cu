@@ -1,0 +1,488 @@
+// Planner kernels: ragged offsets, shuffle keys, key sort, the fill rule, inverse tables.
+//
+// The paper's block construction (Methods, first paragraph; caption of the pseudocode figure):
+// open a block, draw a random unused sequence among those that still fit (Random_*() over L_dict),
+// append it, repeat until nothing fits, pad, open the next block.  On the device this becomes
+//   1. validate + exclusive scan of the lengths (ragged offsets), one Philox word per sequence
+//      (shuffle key h_i) and one per draw (u_k);
+//   2. a stable LSD radix sort of the ids by (T_i, h_i): L_dict as one array, buckets by length,
+//      each bucket pre-shuffled;
+//   3. the fill rule itself, a chain of n dependent draws run by one warp over a two-level table of
+//      running counts kept in shared memory;
+//   4. a parallel pass that resolves draws to sequence ids and writes the inverse tables.
+#include <limits.h>
+
+#include "bload_internal.cuh"
+
+namespace bload {
+
+namespace {
+
+constexpr unsigned kFull = 0xffffffffu;
+constexpr unsigned long long kNoBad = ULLONG_MAX;
+
+// ---- Philox-4x64-10 (Salmon et al., SC'11): counter (idx,0,0,0), key (seed, stream); word 0 ----
+__device__ __forceinline__ uint64_t philox_word0(uint64_t idx, uint64_t seed, uint64_t stream)
+{
+    const uint64_t M0 = 0xD2E7470EE14C6C93ULL, M1 = 0xCA5A826395121157ULL;
+    const uint64_t W0 = 0x9E3779B97F4A7C15ULL, W1 = 0xBB67AE8584CAA73BULL;
+    uint64_t c0 = idx, c1 = 0, c2 = 0, c3 = 0, k0 = seed, k1 = stream;
+#pragma unroll
+    for (int r = 0; r < 10; ++r) {
+        if (r) { k0 += W0; k1 += W1; }
+        uint64_t hi0 = __umul64hi(M0, c0), lo0 = M0 * c0;
+        uint64_t hi1 = __umul64hi(M1, c2), lo1 = M1 * c2;
+        c0 = hi1 ^ c1 ^ k0;
+        c1 = lo1;
+        c2 = hi0 ^ c3 ^ k1;
+        c3 = lo0;
+    }
+    return c0;
+}
+
+// ---- block-wide exclusive scan over 256 threads (8 warps) ----
+template <typename T>
+__device__ __forceinline__ T warp_inclusive(T v)
+{
+    const int lane = threadIdx.x & 31;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        T o = __shfl_up_sync(kFull, v, d);
+        if (lane >= d) v += o;
+    }
+    return v;
+}
+
+template <typename T, int WARPS>
+__device__ __forceinline__ T block_exclusive(T v, T* warp_tot /*[WARPS] shared*/, T* total)
+{
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    T inc = warp_inclusive(v);
+    if (lane == 31) warp_tot[w] = inc;
+    __syncthreads();
+    T base = 0, tot = 0;
+#pragma unroll
+    for (int i = 0; i < WARPS; ++i) {
+        T x = warp_tot[i];
+        if (i < w) base += x;
+        tot += x;
+    }
+    __syncthreads();
+    *total = tot;
+    return base + inc - v;
+}
+
+__global__ void k0_init(PlanHeader* h, int64_t n, int32_t t_block, uint64_t seed, uint32_t policy)
+{
+    if (threadIdx.x == 0 && blockIdx.x == 0) {
+        h->magic = 0;  // set when the plan is complete
+        h->n = n;
+        h->n_blocks = 0;
+        h->sum_t = 0;
+        h->first_bad = kNoBad;
+        h->checksum = 0;
+        h->seed = seed;
+        h->t_block = t_block;
+        h->t_max = 0;
+        h->status = BLOAD_OK;
+        h->max_segs = 0;
+        h->policy = policy;
+    }
+}
+
+// per-chunk sum of lengths, global max, first index with T outside [1, t_block]
+__global__ void __launch_bounds__(256) k1_reduce(const int32_t* __restrict__ len, int64_t n, int32_t t_block,
+                                                 int64_t* __restrict__ partial, PlanHeader* h)
+{
+    __shared__ int64_t s_sum[8];
+    __shared__ int s_max[8];
+    __shared__ unsigned long long s_bad[8];
+    const int64_t base = (int64_t)blockIdx.x * kChunk;
+    int64_t sum = 0;
+    int mx = 0;
+    unsigned long long bad = kNoBad;
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+        int64_t i = base + e * 256 + threadIdx.x;
+        if (i < n) {
+            int t = len[i];
+            if (t < 1 || t > t_block) { if ((unsigned long long)i < bad) bad = (unsigned long long)i; }
+            sum += t;
+            mx = max(mx, t);
+        }
+    }
+#pragma unroll
+    for (int d = 16; d; d >>= 1) {
+        sum += __shfl_xor_sync(kFull, sum, d);
+        mx = max(mx, __shfl_xor_sync(kFull, mx, d));
+        unsigned long long ob = __shfl_xor_sync(kFull, bad, d);
+        bad = ob < bad ? ob : bad;
+    }
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    if (lane == 0) { s_sum[w] = sum; s_max[w] = mx; s_bad[w] = bad; }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        for (int i = 1; i < 8; ++i) { sum += s_sum[i]; mx = max(mx, s_max[i]); bad = s_bad[i] < bad ? s_bad[i] : bad; }
+        partial[blockIdx.x] = sum;
+        atomicMax(&h->t_max, mx);
+        if (bad != kNoBad) atomicMin(&h->first_bad, bad);
+    }
+}
+
+// exclusive scan of the per-chunk sums (one CTA), total to the header, status on bad input
+__global__ void __launch_bounds__(1024) k1_scan_partials(int64_t* __restrict__ partial, int64_t chunks, PlanHeader* h)
+{
+    __shared__ int64_t s_tot[32];
+    int64_t carry = 0;
+    for (int64_t lo = 0; lo < chunks; lo += 1024) {
+        int64_t i = lo + threadIdx.x;
+        int64_t v = i < chunks ? partial[i] : 0, tot;
+        int64_t ex = block_exclusive<int64_t, 32>(v, s_tot, &tot);
+        if (i < chunks) partial[i] = carry + ex;
+        carry += tot;
+    }
+    if (threadIdx.x == 0) {
+        h->sum_t = carry;
+        if (h->first_bad != kNoBad) h->status = BLOAD_ERR_LENGTH;
+    }
+}
+
+// offsets[i], sort key (T_i << 32 | h_i), payload id, random word of draw i
+__global__ void __launch_bounds__(256) k1_offsets_keys(const int32_t* __restrict__ len, int64_t n, uint64_t seed,
+                                                       const int64_t* __restrict__ partial,
+                                                       int64_t* __restrict__ offsets, uint64_t* __restrict__ key,
+                                                       int32_t* __restrict__ id, uint64_t* __restrict__ draw_u,
+                                                       const PlanHeader* h)
+{
+    __shared__ int64_t s_tot[8];
+    if (h->first_bad != kNoBad) return;
+    const int64_t base = (int64_t)blockIdx.x * kChunk + (int64_t)threadIdx.x * 8;
+    int t[8];
+    int64_t sum = 0;
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+        t[e] = (base + e < n) ? len[base + e] : 0;
+        sum += t[e];
+    }
+    int64_t tot;
+    int64_t run = partial[blockIdx.x] + block_exclusive<int64_t, 8>(sum, s_tot, &tot);
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+        int64_t i = base + e;
+        if (i < n) {
+            offsets[i] = run;
+            run += t[e];
+            uint32_t hkey = (uint32_t)(philox_word0((uint64_t)i, seed, 1ULL) >> 32);
+            key[i] = ((uint64_t)(uint32_t)t[e] << 32) | hkey;
+            id[i] = (int32_t)i;
+            draw_u[i] = philox_word0((uint64_t)i, seed, 2ULL);
+            if (i == n - 1) offsets[n] = run;
+        }
+    }
+}
+
+// ---- stable LSD radix sort, 8-bit digits, chunk = 2048 keys per CTA ----
+__global__ void __launch_bounds__(256) k3_hist(const uint64_t* __restrict__ key, int64_t n, int shift, int64_t chunks,
+                                               uint32_t* __restrict__ hist, const PlanHeader* h)
+{
+    __shared__ uint32_t s_h[256];
+    if (h->first_bad != kNoBad) return;
+    s_h[threadIdx.x] = 0;
+    __syncthreads();
+    const int64_t base = (int64_t)blockIdx.x * kChunk;
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+        int64_t i = base + e * 256 + threadIdx.x;
+        if (i < n) atomicAdd(&s_h[(unsigned)(key[i] >> shift) & 255u], 1u);
+    }
+    __syncthreads();
+    hist[(int64_t)threadIdx.x * chunks + blockIdx.x] = s_h[threadIdx.x];
+}
+
+__global__ void __launch_bounds__(1024) k3_scan(uint32_t* __restrict__ hist, int64_t total, const PlanHeader* h)
+{
+    __shared__ uint32_t s_tot[32];
+    if (h->first_bad != kNoBad) return;
+    uint32_t carry = 0;
+    for (int64_t lo = 0; lo < total; lo += 1024) {
+        int64_t i = lo + threadIdx.x;
+        uint32_t v = i < total ? hist[i] : 0, tot;
+        uint32_t ex = block_exclusive<uint32_t, 32>(v, s_tot, &tot);
+        if (i < total) hist[i] = carry + ex;
+        carry += tot;
+    }
+}
+
+__global__ void __launch_bounds__(256) k3_scatter(const uint64_t* __restrict__ key_in, const int32_t* __restrict__ id_in,
+                                                  uint64_t* __restrict__ key_out, int32_t* __restrict__ id_out,
+                                                  int64_t n, int shift, int64_t chunks,
+                                                  const uint32_t* __restrict__ hist, const PlanHeader* h)
+{
+    __shared__ uint32_t s_cnt[8][256];
+    if (h->first_bad != kNoBad) return;
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    for (int i = threadIdx.x; i < 8 * 256; i += 256) (&s_cnt[0][0])[i] = 0;
+    __syncthreads();
+    // warp w ranks its 256 consecutive keys, 32 at a time, in input order
+    const int64_t wbase = (int64_t)blockIdx.x * kChunk + w * 256;
+    uint64_t k[8];
+    int32_t v[8];
+    uint32_t rank[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+        int64_t i = wbase + e * 32 + lane;
+        bool ok = i < n;
+        k[e] = ok ? key_in[i] : 0;
+        v[e] = ok ? id_in[i] : 0;
+        unsigned d = (unsigned)(k[e] >> shift) & 255u;
+        unsigned tag = ok ? d : (256u + lane);
+        unsigned peers = __match_any_sync(kFull, tag);
+        unsigned before = __popc(peers & ((1u << lane) - 1u));
+        uint32_t prev = ok ? s_cnt[w][d] : 0;
+        __syncwarp();
+        if (ok && before == 0) s_cnt[w][d] = prev + __popc(peers);
+        __syncwarp();
+        rank[e] = prev + before;
+    }
+    __syncthreads();
+    {
+        const int d = threadIdx.x;
+        uint32_t run = hist[(int64_t)d * chunks + blockIdx.x];
+#pragma unroll
+        for (int ww = 0; ww < 8; ++ww) {
+            uint32_t c = s_cnt[ww][d];
+            s_cnt[ww][d] = run;
+            run += c;
+        }
+    }
+    __syncthreads();
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+        int64_t i = wbase + e * 32 + lane;
+        if (i < n) {
+            unsigned d = (unsigned)(k[e] >> shift) & 255u;
+            uint32_t p = s_cnt[w][d] + rank[e];
+            key_out[p] = k[e];
+            id_out[p] = v[e];
+        }
+    }
+}
+
+// bucket_end[l] = number of sequences with length <= l, l = 0..t_block, from the sorted keys
+__global__ void __launch_bounds__(256) k3_buckets(const uint64_t* __restrict__ key, int64_t n, int32_t t_block,
+                                                  int32_t* __restrict__ bucket_end, const PlanHeader* h)
+{
+    if (h->first_bad != kNoBad) return;
+    int64_t p = (int64_t)blockIdx.x * 256 + threadIdx.x;
+    if (p >= n) return;
+    int t = (int)(key[p] >> 32);
+    if (p == 0)
+        for (int l = 0; l < t; ++l) bucket_end[l] = 0;
+    int tn = (p + 1 < n) ? (int)(key[p + 1] >> 32) : t_block + 1;
+    for (int l = t; l < tn; ++l) bucket_end[l] = (int32_t)(p + 1);
+}
+
+// ---- the fill rule: one warp, n dependent draws ----
+// Shared memory holds running counts of UNUSED sequences as inclusive prefix sums:
+//   P0[g]        sequences with length <= 256*(g+1)           (128 entries)
+//   P1[g][i]     sequences with length in (256*g, 256*g+i+1]   (groups of 256 lengths)
+// so that "how many fit in r slots" is two reads and "the j-th of them in order of length" is two
+// compare-and-count steps; a draw then decrements the entries at and after the chosen length.
+__global__ void __launch_bounds__(256, 1) k4_fill(PlanView pv, const int32_t* __restrict__ bucket_end,
+                                                  const uint64_t* __restrict__ draw_u, int4* __restrict__ draw_rec,
+                                                  int64_t n64, int32_t L)
+{
+    extern __shared__ __align__(16) int32_t sm[];
+    int32_t* P0 = sm;
+    int32_t* P1 = sm + 128;
+    if (pv.hdr->first_bad != kNoBad) return;
+    const int G = (L + 255) >> 8;
+    for (int idx = threadIdx.x; idx < G * 256; idx += blockDim.x) {
+        int g = idx >> 8;
+        int hi = min(idx + 1, L);
+        P1[idx] = bucket_end[hi] - bucket_end[g << 8];
+    }
+    for (int g = threadIdx.x; g < 128; g += blockDim.x) P0[g] = bucket_end[min((g + 1) << 8, L)];
+    __syncthreads();
+    if (threadIdx.x >= 32) return;
+
+    const int lane = threadIdx.x;
+    const int n = (int)n64;
+    int4 p0 = reinterpret_cast<int4*>(P0)[lane];
+    int k = 0, b = 0, room = L, start = 0;
+    if (lane == 0) pv.block_seg_begin[0] = 0;
+    uint64_t u_next = draw_u[0];
+    while (k < n) {
+        int m = 0;
+        if (room > 0) {
+            int y = room - 1, gy = y >> 8;
+            m = P1[y] + (gy ? P0[gy - 1] : 0);
+        }
+        if (m == 0) {  // nothing fits: the rest of the block is padding
+            if (lane == 0) { pv.block_fill[b] = start; pv.block_seg_begin[b + 1] = k; }
+            ++b; room = L; start = 0;
+            continue;
+        }
+        const uint64_t u = u_next;
+        if (k + 1 < n) u_next = draw_u[k + 1];
+        const int j = (int)__umul64hi(u, (uint64_t)(unsigned)m);  // floor(u * m / 2^64)
+        int c = (p0.x <= j) + (p0.y <= j) + (p0.z <= j) + (p0.w <= j);
+        const int g = __reduce_add_sync(kFull, c);
+        const int j1 = j - (g ? P0[g - 1] : 0);
+        int4* row = reinterpret_cast<int4*>(P1 + (g << 8));
+        int4 va = row[2 * lane], vb = row[2 * lane + 1];
+        c = (va.x <= j1) + (va.y <= j1) + (va.z <= j1) + (va.w <= j1) + (vb.x <= j1) + (vb.y <= j1) + (vb.z <= j1) +
+            (vb.w <= j1);
+        const int i = __reduce_add_sync(kFull, c);
+        const int len = (g << 8) + i + 1;
+        int prev = __shfl_up_sync(kFull, vb.w, 1);
+        if (lane == 0) prev = 0;
+        const int owner = i >> 3, e = i & 7;
+        if (lane == owner) {
+            int cur = e == 0 ? va.x : e == 1 ? va.y : e == 2 ? va.z : e == 3 ? va.w : e == 4 ? vb.x : e == 5 ? vb.y : e == 6 ? vb.z : vb.w;
+            int prv = e == 0 ? prev : e == 1 ? va.x : e == 2 ? va.y : e == 3 ? va.z : e == 4 ? va.w : e == 5 ? vb.x : e == 6 ? vb.y : vb.z;
+            draw_rec[k] = make_int4(len, cur - prv, b, start);
+        }
+        {
+            const int f = 4 * lane;
+            p0.x -= (f + 0 >= g); p0.y -= (f + 1 >= g); p0.z -= (f + 2 >= g); p0.w -= (f + 3 >= g);
+            if (f + 3 >= g) reinterpret_cast<int4*>(P0)[lane] = p0;
+        }
+        if (lane >= owner) {
+            const int f = 8 * lane;
+            va.x -= (f + 0 >= i); va.y -= (f + 1 >= i); va.z -= (f + 2 >= i); va.w -= (f + 3 >= i);
+            vb.x -= (f + 4 >= i); vb.y -= (f + 5 >= i); vb.z -= (f + 6 >= i); vb.w -= (f + 7 >= i);
+            row[2 * lane] = va; row[2 * lane + 1] = vb;
+        }
+        __syncwarp();
+        room -= len; start += len; ++k;
+    }
+    if (lane == 0) {
+        pv.block_fill[b] = start;
+        pv.block_seg_begin[b + 1] = k;
+        pv.hdr->n_blocks = b + 1;
+    }
+}
+
+__device__ __forceinline__ uint64_t fmix64(uint64_t x)
+{  // 64-bit finaliser of MurmurHash3
+    x ^= x >> 33; x *= 0xff51afd7ed558ccdULL;
+    x ^= x >> 33; x *= 0xc4ceb9fe1a85ec53ULL;
+    x ^= x >> 33;
+    return x;
+}
+
+// resolve draws to sequence ids; segment list, inverse tables, digest, widest block
+__global__ void __launch_bounds__(256) k5_tables(PlanView pv, const int4* __restrict__ draw_rec,
+                                                 const int32_t* __restrict__ bucket_end,
+                                                 const int32_t* __restrict__ sorted_id, int64_t n)
+{
+    __shared__ unsigned long long s_sum[8];
+    __shared__ int s_max[8];
+    if (pv.hdr->first_bad != kNoBad) return;
+    const int64_t k = (int64_t)blockIdx.x * 256 + threadIdx.x;
+    unsigned long long term = 0;
+    int segs = 0;
+    if (k < n) {
+        int4 r = draw_rec[k];
+        int id = sorted_id[bucket_end[r.x] - r.y];
+        pv.seg_seq[k] = id;
+        pv.seg_block[k] = r.z;
+        pv.seg_start[k] = r.w;
+        pv.seg_src[k] = pv.offsets[id];
+        pv.seq_block[id] = r.z;
+        pv.seq_start[id] = r.w;
+        uint64_t where = ((uint64_t)(uint32_t)r.z << 32) | (uint64_t)(uint32_t)r.w;
+        term = fmix64(where * 0x9E3779B97F4A7C15ULL + (uint64_t)(uint32_t)id);
+        if (k < pv.hdr->n_blocks) segs = pv.block_seg_begin[k + 1] - pv.block_seg_begin[k];
+    }
+#pragma unroll
+    for (int d = 16; d; d >>= 1) {
+        term += __shfl_xor_sync(kFull, term, d);
+        segs = max(segs, __shfl_xor_sync(kFull, segs, d));
+    }
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    if (lane == 0) { s_sum[w] = term; s_max[w] = segs; }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        for (int i = 1; i < 8; ++i) { term += s_sum[i]; segs = max(segs, s_max[i]); }
+        atomicAdd(&pv.hdr->checksum, term);
+        atomicMax(&pv.hdr->max_segs, segs);
+    }
+}
+
+__global__ void k5_finish(PlanHeader* h)
+{
+    if (threadIdx.x == 0 && blockIdx.x == 0 && h->first_bad == kNoBad) h->magic = kPlanMagic;
+}
+
+}  // namespace
+
+size_t work_layout(int64_t n, int32_t t_block, void* base, WorkView* w)
+{
+    size_t off = 0;
+    auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes); return o; };
+    const int64_t chunks = chunks_of(n);
+    size_t o_ka = take(sizeof(uint64_t) * n), o_kb = take(sizeof(uint64_t) * n);
+    size_t o_ia = take(sizeof(int32_t) * n), o_ib = take(sizeof(int32_t) * n);
+    size_t o_u = take(sizeof(uint64_t) * n), o_rec = take(sizeof(int4) * n);
+    size_t o_part = take(sizeof(int64_t) * chunks), o_hist = take(sizeof(uint32_t) * 256 * chunks);
+    size_t o_be = take(sizeof(int32_t) * ((size_t)t_block + 1));
+    if (w) {
+        char* b = static_cast<char*>(base);
+        w->key_a = reinterpret_cast<uint64_t*>(b + o_ka);
+        w->key_b = reinterpret_cast<uint64_t*>(b + o_kb);
+        w->id_a = reinterpret_cast<int32_t*>(b + o_ia);
+        w->id_b = reinterpret_cast<int32_t*>(b + o_ib);
+        w->draw_u = reinterpret_cast<uint64_t*>(b + o_u);
+        w->draw_rec = reinterpret_cast<int4*>(b + o_rec);
+        w->partial = reinterpret_cast<int64_t*>(b + o_part);
+        w->digit_hist = reinterpret_cast<uint32_t*>(b + o_hist);
+        w->bucket_end = reinterpret_cast<int32_t*>(b + o_be);
+    }
+    return off;
+}
+
+cudaError_t launch_plan(const int32_t* d_lengths, int64_t n, int32_t t_block, uint64_t seed, uint32_t policy,
+                        const PlanView& pv, const WorkView& wv, cudaStream_t st, cudaEvent_t* ev)
+{
+    const int64_t chunks = chunks_of(n);
+    const unsigned gc = (unsigned)chunks;
+    if (ev) cudaEventRecord(ev[0], st);
+    k0_init<<<1, 32, 0, st>>>(pv.hdr, n, t_block, seed, policy);
+    k1_reduce<<<gc, 256, 0, st>>>(d_lengths, n, t_block, wv.partial, pv.hdr);
+    k1_scan_partials<<<1, 1024, 0, st>>>(wv.partial, chunks, pv.hdr);
+    k1_offsets_keys<<<gc, 256, 0, st>>>(d_lengths, n, seed, wv.partial, pv.offsets, wv.key_a, wv.id_a, wv.draw_u, pv.hdr);
+    if (ev) cudaEventRecord(ev[1], st);
+
+    // digits: 4 of the shuffle key, then as many as the block length needs
+    int t_bits = 0;
+    while ((1 << t_bits) <= t_block) ++t_bits;
+    const int passes = 4 + (t_bits + 7) / 8;
+    uint64_t *kin = wv.key_a, *kout = wv.key_b;
+    int32_t *iin = wv.id_a, *iout = wv.id_b;
+    for (int p = 0; p < passes; ++p) {
+        const int shift = 8 * p;
+        k3_hist<<<gc, 256, 0, st>>>(kin, n, shift, chunks, wv.digit_hist, pv.hdr);
+        k3_scan<<<1, 1024, 0, st>>>(wv.digit_hist, 256 * chunks, pv.hdr);
+        k3_scatter<<<gc, 256, 0, st>>>(kin, iin, kout, iout, n, shift, chunks, wv.digit_hist, pv.hdr);
+        uint64_t* tk = kin; kin = kout; kout = tk;
+        int32_t* ti = iin; iin = iout; iout = ti;
+    }
+    k3_buckets<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(kin, n, t_block, wv.bucket_end, pv.hdr);
+    if (ev) cudaEventRecord(ev[2], st);
+
+    const int G = (t_block + 255) >> 8;
+    const size_t smem = sizeof(int32_t) * (128 + (size_t)G * 256);
+    cudaError_t e = cudaFuncSetAttribute(k4_fill, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    k4_fill<<<1, 256, smem, st>>>(pv, wv.bucket_end, wv.draw_u, wv.draw_rec, n, t_block);
+    if (ev) cudaEventRecord(ev[3], st);
+
+    k5_tables<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(pv, wv.draw_rec, wv.bucket_end, iin, n);
+    k5_finish<<<1, 32, 0, st>>>(pv.hdr);
+    if (ev) cudaEventRecord(ev[4], st);
+    return cudaPeekAtLastError();
+}
+
+}  // namespace bload

@@ -1,0 +1,87 @@
+"""GPU parity at the full sizes of the three large evaluation configurations, in the launch
+configuration the benchmark times (one whole-epoch call per direction).  The plan is compared with
+the oracle table by table; packed and unpacked bytes are compared on sampled blocks, which the
+oracle computes one by one, plus size-independent properties (pad bytes, untouched canaries)."""
+import numpy as np
+import pytest
+import torch
+
+import gpu_util as G
+import paper_2310_10879_b200 as B
+from oracle import bload_oracle as O
+from paper_2310_10879_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+
+
+def _sample_blocks(n_blocks, k, seed):
+    rng = np.random.default_rng(seed)
+    pick = set(int(x) for x in rng.choice(n_blocks, size=min(k, n_blocks), replace=False))
+    pick |= {0, n_blocks - 1}
+    return sorted(pick)
+
+
+def _run(name, n_sample):
+    w = W.WORKLOADS[name]
+    T = W.lengths(w)
+    op = O.plan(T, w.t_block, w.seed)
+    plan = G.gpu_plan(T, w.t_block, w.seed)
+    G.assert_plan_equal(plan, op)
+    fb, ofb, tb, nb = w.frame_bytes, w.out_frame_bytes, w.t_block, op.n_blocks
+    store = W.payload_torch(w, op.sum_t, G.DEV)
+    store_u8 = store.view(torch.uint8).reshape(-1)
+    dense = G.Guarded(nb * tb * fb)
+    B.bload_pack(plan, store_u8, fb, 0, nb, dense=dense.t, pad_byte=0)
+    torch.cuda.synchronize()
+    dense.check()
+    store_h = store_u8.cpu().numpy()
+    blocks = _sample_blocks(nb, n_sample, 3)
+    d3 = dense.t.view(nb, tb * fb)
+    for b in blocks:
+        want = O.pack(op, store_h, fb, b, 1, 0).reshape(-1)
+        assert np.array_equal(d3[b].cpu().numpy(), want), "block %d" % b
+    # property at any size: the pad region of every block is zero and counts pad_packed frames
+    fill = torch.from_numpy(op.block_fill.astype(np.int64)).to(G.DEV)
+    slot = torch.arange(tb, device=G.DEV)
+    step = max(1, (1 << 28) // (tb * fb))
+    nonzero_pad = 0
+    for lo in range(0, nb, step):
+        chunk = dense.t.view(nb, tb, fb)[lo:lo + step]
+        padmask = slot[None, :] >= fill[lo:lo + step, None]
+        nonzero_pad += int((chunk.ne(0).any(dim=2) & padmask).sum())
+    assert nonzero_pad == 0
+    # round trip of the input itself (same frame size): unpack(pack(x)) == x, every byte
+    back = G.Guarded(op.sum_t * fb, 0x5A)
+    B.bload_unpack(plan, dense.t, fb, 0, nb, back.t)
+    torch.cuda.synchronize(); back.check()
+    assert torch.equal(back.t, store_u8)
+    del back, dense, d3
+    # unpack of a per-frame output (fp32 of the same shape for the bf16 workload)
+    if ofb != fb:
+        del store, store_u8
+        torch.cuda.empty_cache()
+        out = W.payload_torch(w, nb * tb, G.DEV, out=True)          # dense per-frame outputs
+        out_u8 = out.view(torch.uint8).reshape(nb, tb * ofb)
+        rag = G.Guarded(op.sum_t * ofb, 0x5A)
+        B.bload_unpack(plan, out_u8, ofb, 0, nb, rag.t)
+        torch.cuda.synchronize(); rag.check()
+        want = np.empty(op.sum_t * ofb, np.uint8)                   # pages are touched only where written
+        for b in blocks[:4]:
+            O.unpack(op, out_u8[b].cpu().numpy(), ofb, b, 1, want)
+            for k in range(op.block_seg_begin[b], op.block_seg_begin[b + 1]):
+                s = int(op.seg_seq[k]); lo, hi = int(op.offsets[s]) * ofb, int(op.offsets[s + 1]) * ofb
+                assert np.array_equal(rag.t[lo:hi].cpu().numpy(), want[lo:hi]), "sequence %d" % s
+    st = B.bload_stats(plan.info)
+    assert st["pad_packed"] == nb * tb - op.sum_t and st["pad_naive_tmax"] == op.n * op.t_max - op.sum_t
+
+
+def test_full_size_raw_frames():
+    _run("raw_frames", 3)
+
+
+def test_full_size_tokens():
+    _run("tokens", 300)
+
+
+def test_full_size_heavy_tail_bf16_with_fp32_outputs():
+    _run("heavy_tail_bf16", 6)

@@ -1,0 +1,216 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the CPU oracle, bit for bit."""
+import ctypes as C
+
+import numpy as np
+import pytest
+import torch
+
+import gpu_util as G
+import paper_2310_10879_b200 as B
+from oracle import bload_oracle as O
+from paper_2310_10879_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+
+
+def test_toy8_of_the_paper():
+    for seed in range(20):
+        for fb in (12288, 1):
+            G.full_parity(W.TOY8_LENGTHS, W.TOY8_T_BLOCK, seed, fb, payload_seed=seed)
+
+
+def test_config_toy_video():
+    w = W.WORKLOADS["toy_video"]
+    plan, op = G.full_parity(W.lengths(w), w.t_block, w.seed, w.frame_bytes)
+    # batches of 8 blocks, the last one rounded up with filler blocks
+    store = W.payload_torch(w, op.sum_t, G.DEV).view(torch.uint8).reshape(-1)
+    store_h = store.cpu().numpy()
+    for b0 in range(0, op.n_blocks, w.batch_blocks):
+        res, _ = G.gpu_pack_all(plan, store, w.frame_bytes, b0, w.batch_blocks, 0)
+        assert np.array_equal(res["dense"], O.pack(op, store_h, w.frame_bytes, b0, w.batch_blocks, 0))
+        for name, want in zip(("seq_id", "pos", "reset", "valid"), O.metadata(op, b0, w.batch_blocks)):
+            assert np.array_equal(res[name], want)
+
+
+def test_config_features_fp16():
+    w = W.WORKLOADS["features_fp16"]
+    G.full_parity(W.lengths(w), w.t_block, w.seed, w.frame_bytes)
+
+
+def test_config_raw_frames_scaled():
+    w = W.scaled(W.WORKLOADS["raw_frames"], 40)
+    G.full_parity(W.lengths(w), w.t_block, w.seed, w.frame_bytes, extra_blocks=1)
+
+
+def test_config_tokens_scaled():
+    w = W.scaled(W.WORKLOADS["tokens"], 30000)
+    G.full_parity(W.lengths(w), w.t_block, w.seed, w.frame_bytes)
+
+
+def test_config_heavy_tail_scaled_with_fp32_outputs():
+    w = W.scaled(W.WORKLOADS["heavy_tail_bf16"], 1200)
+    G.full_parity(W.lengths(w), w.t_block, w.seed, w.frame_bytes, out_fb=w.out_frame_bytes, extra_blocks=1)
+
+
+def test_dataset_shaped_lengths():
+    w = W.WORKLOADS["video_dataset_shape"]
+    plan, op = G.full_parity(W.lengths(w), w.t_block, w.seed, w.frame_bytes)
+    s = B.bload_stats(plan.info)
+    assert s == {**O.stats(op.n, op.sum_t, op.t_max, op.t_block, op.n_blocks),
+                 "max_segs_per_block": op.max_segs_per_block}
+
+
+@pytest.mark.parametrize("fb", [1, 2, 3, 4, 6, 8, 12, 20, 24, 48, 100, 1000, 4100])
+@pytest.mark.parametrize("pad", [0, 0x7F])
+def test_frame_sizes_and_alignments(fb, pad):
+    """Frame sizes that are not multiples of 16 exercise every relative misalignment of source and
+    destination runs (byte, 2-, 4-, 8-byte granules) and the head/tail handling."""
+    rng = np.random.default_rng(fb * 31 + pad)
+    tb = int(rng.integers(5, 200))
+    T = rng.integers(1, tb + 1, size=int(rng.integers(1, 300))).astype(np.int32)
+    G.full_parity(T, tb, int(rng.integers(0, 1 << 40)), fb, out_fb=fb + (fb % 3), pad=pad)
+
+
+@pytest.mark.parametrize("case", ["one", "all_full", "all_ones", "block_of_one", "max_t_block", "many_short",
+                                  "two_lengths"])
+def test_degenerate_plans(case):
+    rng = np.random.default_rng(1)
+    if case == "one":
+        T, tb = np.array([5], np.int32), 9
+    elif case == "all_full":
+        T, tb = np.full(300, 17, np.int32), 17
+    elif case == "all_ones":
+        T, tb = np.ones(5000, np.int32), 33
+    elif case == "block_of_one":
+        T, tb = np.ones(70, np.int32), 1
+    elif case == "max_t_block":
+        tb = 32768
+        T = np.concatenate([rng.integers(1, tb + 1, size=40), [tb, tb, 1, 1, 255, 256, 257]]).astype(np.int32)
+    elif case == "many_short":
+        T, tb = rng.integers(1, 4, size=9000).astype(np.int32), 4096      # thousands of segments per block
+    else:
+        T, tb = rng.choice([3, 700], size=4097).astype(np.int32), 1000
+    G.full_parity(T, tb, 77, 8 if case in ("max_t_block", "many_short") else 20)
+
+
+@pytest.mark.parametrize("n", [1, 2, 31, 32, 33, 255, 256, 257, 2047, 2048, 2049, 4096, 70001])
+def test_plan_sizes_around_tile_boundaries(n):
+    rng = np.random.default_rng(n)
+    tb = 300
+    T = rng.integers(1, tb + 1, size=n).astype(np.int32)
+    for seed in (0, 2**63 + 11):
+        G.assert_plan_equal(G.gpu_plan(T, tb, seed), O.plan(T, tb, seed))
+
+
+def test_many_seeds_small():
+    T = W.lengths(W.WORKLOADS["features_fp16"])[:200]
+    for seed in range(40):
+        G.assert_plan_equal(G.gpu_plan(T, 1000, seed), O.plan(T, 1000, seed))
+
+
+def test_block_ranges_and_partial_unpack():
+    w = W.scaled(W.WORKLOADS["features_fp16"], 400)
+    T = W.lengths(w)
+    op = O.plan(T, w.t_block, 9)
+    plan = G.gpu_plan(T, w.t_block, 9)
+    fb = 40
+    store = torch.randint(0, 256, (op.sum_t * fb,), dtype=torch.uint8, device=G.DEV)
+    store_h = store.cpu().numpy()
+    for b0, cnt in [(0, 1), (3, 4), (op.n_blocks - 1, 1), (op.n_blocks - 1, 3), (op.n_blocks + 5, 2), (2, 0)]:
+        res, _ = G.gpu_pack_all(plan, store, fb, b0, cnt, 0x33)
+        assert np.array_equal(res["dense"], O.pack(op, store_h, fb, b0, cnt, 0x33))
+        for name, want in zip(("seq_id", "pos", "reset", "valid"), O.metadata(op, b0, cnt)):
+            assert np.array_equal(res[name], want)
+        dense_out = torch.randint(0, 256, (cnt * w.t_block * fb,), dtype=torch.uint8, device=G.DEV)
+        rag = G.Guarded(op.sum_t * fb, 0x5A)
+        B.bload_unpack(plan, dense_out, fb, b0, cnt, rag.t)
+        torch.cuda.synchronize(); rag.check()
+        want = np.full(op.sum_t * fb, 0x5A, np.uint8)
+        O.unpack(op, dense_out.cpu().numpy(), fb, b0, cnt, want)
+        assert np.array_equal(rag.t.cpu().numpy(), want)
+
+
+def test_metadata_only_and_dense_only_calls():
+    T = W.lengths(W.scaled(W.WORKLOADS["features_fp16"], 100))
+    op = O.plan(T, 1000, 4); plan = G.gpu_plan(T, 1000, 4)
+    valid = torch.zeros(op.n_blocks * 1000, dtype=torch.uint8, device=G.DEV)
+    B.bload_pack(plan, None, 16, 0, op.n_blocks, valid=valid)
+    assert np.array_equal(valid.cpu().numpy().reshape(op.n_blocks, 1000), O.metadata(op, 0, op.n_blocks)[3])
+    # odd t_block and unaligned metadata pointers take the scalar path
+    T = np.array([3, 4, 2, 7, 1, 6], np.int32)
+    op = O.plan(T, 7, 1); plan = G.gpu_plan(T, 7, 1)
+    raw = torch.zeros(op.n_blocks * 7 + 3, dtype=torch.uint8, device=G.DEV)
+    B.bload_pack(plan, None, 16, 0, op.n_blocks, reset=raw[1:1 + op.n_blocks * 7])
+    assert np.array_equal(raw[1:1 + op.n_blocks * 7].cpu().numpy().reshape(op.n_blocks, 7),
+                          O.metadata(op, 0, op.n_blocks)[2])
+
+
+def test_bad_lengths_are_reported_not_faulted():
+    for T, tb, bad in [([3, 0, 2], 4, 1), ([3, 4, 5, 2], 4, 2), ([3, -1], 4, 1)]:
+        plan = G.gpu_plan(np.array(T, np.int32), tb, 0, check=False)
+        op = O.plan(np.array(T, np.int32), tb, 0)
+        assert plan.info.status == B._lib.ERR_LENGTH and op.status != 0
+        assert plan.info.first_bad_index == bad == op.first_bad
+        with pytest.raises(B.BloadError):
+            B.bload_pack(plan, torch.zeros(64, dtype=torch.uint8, device=G.DEV), 1, 0, 1,
+                         dense=torch.zeros(64, dtype=torch.uint8, device=G.DEV))
+    big = np.ones(5000, np.int32); big[4321] = 9
+    plan = G.gpu_plan(big, 8, 0, check=False)
+    assert plan.info.first_bad_index == 4321
+    # the context is still healthy
+    G.assert_plan_equal(G.gpu_plan(np.ones(10, np.int32), 8, 0), O.plan(np.ones(10, np.int32), 8, 0))
+
+
+def test_host_detected_errors_launch_nothing():
+    L = B.load()
+    e = B._lib
+    d_len = torch.ones(16, dtype=torch.int32, device=G.DEV)
+    sz = B.bload_plan_sizes(16, 8)
+    plan_buf = torch.zeros(sz.plan_bytes + 256, dtype=torch.uint8, device=G.DEV)
+    work = torch.zeros(sz.work_bytes + 256, dtype=torch.uint8, device=G.DEV)
+    info = B.PlanInfo()
+
+    def call(lengths=d_len.data_ptr(), n=16, tb=8, policy=0, plan=plan_buf.data_ptr(), pb=sz.plan_bytes,
+             wk=work.data_ptr(), wb=sz.work_bytes):
+        return L.bload_plan(lengths, n, tb, 0, policy, plan, pb, wk, wb, None, C.byref(info))
+
+    assert call(lengths=None) == e.ERR_NULL and call(plan=None) == e.ERR_NULL and call(wk=None) == e.ERR_NULL
+    assert call(n=0) == e.ERR_ARG and call(tb=0) == e.ERR_ARG
+    assert call(tb=e.MAX_T_BLOCK + 1) == e.ERR_UNSUPPORTED and call(policy=3) == e.ERR_UNSUPPORTED
+    assert call(pb=sz.plan_bytes - 1) == e.ERR_WORKSPACE and call(wb=sz.work_bytes - 1) == e.ERR_WORKSPACE
+    assert call(plan=plan_buf.data_ptr() + 8) == e.ERR_ALIGN and call(wk=work.data_ptr() + 16) == e.ERR_ALIGN
+    assert call() == 0
+    p = B.Plan(plan_buf, info, sz)
+    x = torch.zeros(4096, dtype=torch.uint8, device=G.DEV)
+    for kwargs, code in [(dict(frame_bytes=0), e.ERR_ARG), (dict(block_begin=-1), e.ERR_ARG),
+                         (dict(block_count=-1), e.ERR_ARG), (dict(block_begin=2**31 - 1, block_count=1), e.ERR_ARG)]:
+        a = dict(frame_bytes=1, block_begin=0, block_count=1); a.update(kwargs)
+        with pytest.raises(B.BloadError) as ei:
+            B.bload_pack(p, x, a["frame_bytes"], a["block_begin"], a["block_count"], dense=x)
+        assert ei.value.code == code
+        with pytest.raises(B.BloadError) as ei:
+            B.bload_unpack(p, x, a["frame_bytes"], a["block_begin"], a["block_count"], x)
+        assert ei.value.code == code
+    with pytest.raises(B.BloadError) as ei:
+        B.bload_pack(p, x[4:], 1, 0, 1, dense=x)
+    assert ei.value.code == e.ERR_ALIGN
+    with pytest.raises(B.BloadError) as ei:
+        B.bload_unpack(p, x, 1, 0, 1, x[8:])
+    assert ei.value.code == e.ERR_ALIGN
+    with pytest.raises(B.BloadError) as ei:
+        B.bload_pack(p, None, 1, 0, 1, dense=x)
+    assert ei.value.code == e.ERR_NULL
+    torch.cuda.synchronize()
+
+
+def test_plan_on_a_side_stream_and_reuse_of_buffers():
+    T = W.lengths(W.scaled(W.WORKLOADS["tokens"], 5000))
+    d_len = torch.from_numpy(T).to(G.DEV)
+    sz = B.bload_plan_sizes(T.size, 4096)
+    plan_buf = torch.empty(sz.plan_bytes, dtype=torch.uint8, device=G.DEV)
+    work = torch.empty(sz.work_bytes, dtype=torch.uint8, device=G.DEV)
+    s = torch.cuda.Stream()
+    for seed in (1, 2, 1):
+        with torch.cuda.stream(s):
+            plan = B.bload_plan(d_len, 4096, seed, work=work, plan_buf=plan_buf)
+        G.assert_plan_equal(plan, O.plan(T, 4096, seed))
