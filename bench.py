@@ -1,0 +1,385 @@
+#!/usr/bin/env python
+"""Benchmark of the BLoad packing path on B200.
+
+One step = one pass of the whole path over one epoch of a synthetic workload: plan (validate,
+scan, keys, sort, fill rule, inverse tables), per-slot metadata, pack of all blocks, unpack of a
+per-frame output of all blocks, statistics.  Prints ONE JSON line.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
+
+With N > 1 (under torchrun) every rank runs an independent replica of the same workload on its own
+GPU ("replicas only": the path has no exchange step); time is the maximum over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "pack+unpack GB/s (algorithmic bytes of the pack and unpack copies / time of the whole step)"
+UNIT = "GB/s"
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+
+
+# ----------------------------------------------------------------------------------------------
+def algorithmic_bytes(sum_t: int, n_blocks: int, t_block: int, fb: int, ofb: int) -> dict:
+    """pack reads every frame once and writes every slot (padding included); unpack reads and
+    writes every frame once (pad slots are not read); metadata writes 10 bytes per slot."""
+    return dict(pack=sum_t * fb + n_blocks * t_block * fb, unpack=2 * sum_t * ofb, meta=10 * n_blocks * t_block)
+
+
+def measured_peak() -> tuple[float, str]:
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(p) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.Q,
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([x.strip() for x in line.split(",")])
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.thread.join(timeout=2)
+        sm, mx, reasons, pw = [], [], set(), []
+        for r in self.rows:
+            try:
+                sm.append(float(r[0])); mx.append(float(r[1])); pw.append(float(r[2]))
+                for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), r[3:7]):
+                    if v.lower().startswith("active"):
+                        reasons.add(name)
+            except Exception:
+                pass
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "power_w_max": max(pw) if pw else None, "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def dist_max(x: float, device=None) -> float:
+    """Maximum of a per-rank scalar over all ranks (identity without a process group)."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()):
+        return x
+    t = torch.tensor([x], dtype=torch.float64, device=device or "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def aggregate(units_per_rank: float, world: int, seconds_max: float) -> float:
+    """Whole-job throughput of `world` independent replicas: all units / slowest rank's time."""
+    return units_per_rank * world / seconds_max
+
+
+# ----------------------------------------------------------------------------------------------
+def cpu_oracle_sample(w, target_blocks: int) -> dict:
+    """Time the CPU oracle, as it stands, on a bounded sample of the workload: the full plan, then
+    metadata + pack + unpack of `target_blocks` consecutive blocks (single thread)."""
+    import numpy as np
+    from oracle import bload_oracle as O
+    from paper_2310_10879_b200 import workloads as W
+    T = W.lengths(w)
+    t0 = time.perf_counter()
+    op = O.plan(T, w.t_block, w.seed)
+    t_plan = time.perf_counter() - t0
+    fb, ofb, tb = w.frame_bytes, w.out_frame_bytes, w.t_block
+    cnt = min(target_blocks, op.n_blocks)
+    b0 = (op.n_blocks - cnt) // 2
+    # host store: only the frames of the sampled blocks' sequences are touched (rest stays untouched virtual memory)
+    store = np.empty(op.sum_t * fb, np.uint8)
+    frames = 0
+    rng = np.random.default_rng(1)
+    for k in range(op.block_seg_begin[b0], op.block_seg_begin[b0 + cnt]):
+        s = int(op.seg_seq[k]); lo, hi = int(op.offsets[s]) * fb, int(op.offsets[s + 1]) * fb
+        store[lo:hi] = rng.integers(0, 256, size=1, dtype=np.uint8)[0]
+        frames += int(op.offsets[s + 1] - op.offsets[s])
+    dense_out = np.ones(cnt * tb * ofb, np.uint8)
+    ragged_out = np.empty(op.sum_t * ofb, np.uint8)
+    for k in range(op.block_seg_begin[b0], op.block_seg_begin[b0 + cnt]):  # fault the output pages in before timing
+        s = int(op.seg_seq[k]); ragged_out[int(op.offsets[s]) * ofb:int(op.offsets[s + 1]) * ofb] = 0
+    t0 = time.perf_counter(); O.metadata(op, b0, cnt); t_meta = time.perf_counter() - t0
+    t0 = time.perf_counter(); O.pack(op, store, fb, b0, cnt, 0); t_pack = time.perf_counter() - t0
+    t0 = time.perf_counter(); O.unpack(op, dense_out, ofb, b0, cnt, ragged_out); t_unpack = time.perf_counter() - t0
+    frac = cnt / op.n_blocks
+    by = dict(pack=frames * fb + cnt * tb * fb, unpack=2 * frames * ofb)
+    t_total = t_plan * frac + t_meta + t_pack + t_unpack
+    return dict(value=(by["pack"] + by["unpack"]) / t_total / 1e9, unit=UNIT, cores=1, kind="oracle",
+                sample="full plan (N=%d, %.3f s, charged pro rata) + metadata/pack/unpack of %d of %d blocks "
+                       "(%d frames); pack %.2f GB/s, unpack %.2f GB/s, single thread"
+                       % (op.n, t_plan, cnt, op.n_blocks, frames, by["pack"] / t_pack / 1e9, by["unpack"] / t_unpack / 1e9),
+                seconds=t_plan + t_meta + t_pack + t_unpack, frames_per_s=frames / t_total,
+                plan_s=t_plan, _bytes=by["pack"] + by["unpack"], _t=t_total)
+
+
+def run_reference(args, w) -> dict:
+    """The reference arm: the CPU oracle on this machine's host cores, a bounded sample per step."""
+    times, last = [], None
+    for i in range(args.warmup + args.steps):
+        r = cpu_oracle_sample(w, max(1, args.ref_blocks // 4))
+        if i >= args.warmup:
+            times.append(r["_t"])
+        last = r
+    t = sum(times) / len(times)
+    value = last["_bytes"] / t / 1e9
+    cb = {k: v for k, v in last.items() if not k.startswith("_")}
+    cb["value"] = value
+    return {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": t * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "u8", "data": "synthetic",
+            "config": config_of(w, None), "cpu_baseline": cb,
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+
+
+def config_of(w, extra) -> dict:
+    c = {"workload": "configs[%d] %s: N=%d, lengths %s, frame %d B (%s), T_block=%d, unpack of %d B/frame outputs; "
+                     "one whole-epoch call per direction" % (w.index, w.name, w.n, w.dist, w.frame_bytes, w.payload,
+                                                             w.t_block, w.out_frame_bytes),
+         "batch_blocks": w.batch_blocks, "l2": "inputs larger than L2 (no flush needed)", "seed": w.seed}
+    if extra:
+        c.update(extra)
+    return c
+
+
+# ----------------------------------------------------------------------------------------------
+def run_gpu(args, w) -> dict:
+    import torch
+    import torch.distributed as dist
+
+    import paper_2310_10879_b200 as B
+    from paper_2310_10879_b200 import workloads as W
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: there is no CPU fallback of the packing path")
+    B.load()
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1 and not dist.is_initialized():
+        dist.init_process_group("nccl", device_id=dev)
+
+    T = W.lengths(w)
+    fb, ofb, tb = w.frame_bytes, w.out_frame_bytes, w.t_block
+    d_len = torch.from_numpy(T).to(dev)
+    sizes = B.bload_plan_sizes(T.size, tb)
+    plan_buf = torch.empty(sizes.plan_bytes, dtype=torch.uint8, device=dev)
+    work = torch.empty(sizes.work_bytes, dtype=torch.uint8, device=dev)
+    plan = B.bload_plan(d_len, tb, w.seed, work=work, plan_buf=plan_buf)
+    nb, sum_t = plan.n_blocks, plan.sum_t
+    by = algorithmic_bytes(sum_t, nb, tb, fb, ofb)
+
+    store = W.payload_torch(w, sum_t, dev).view(torch.uint8).reshape(-1)
+    dense = torch.empty(nb * tb * fb, dtype=torch.uint8, device=dev)
+    seq_id = torch.empty(nb * tb, dtype=torch.int32, device=dev)
+    pos = torch.empty(nb * tb, dtype=torch.int32, device=dev)
+    reset = torch.empty(nb * tb, dtype=torch.uint8, device=dev)
+    valid = torch.empty(nb * tb, dtype=torch.uint8, device=dev)
+    dense_out = W.payload_torch(w, nb * tb, dev, out=True).view(torch.uint8).reshape(-1)
+    ragged_out = torch.empty(sum_t * ofb, dtype=torch.uint8, device=dev)
+
+    B.bload_set_plan_timing(True)
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+
+    def step(rec=None):
+        e = [ev() for _ in range(5)] if rec is not None else None
+        if e: e[0].record()
+        p = B.bload_plan(d_len, tb, w.seed, work=work, plan_buf=plan_buf)
+        if e: e[1].record()
+        B.bload_pack(p, None, fb, 0, nb, seq_id=seq_id, pos=pos, reset=reset, valid=valid)
+        if e: e[2].record()
+        B.bload_pack(p, store, fb, 0, nb, dense=dense)
+        if e: e[3].record()
+        B.bload_unpack(p, dense_out, ofb, 0, nb, ragged_out)
+        if e: e[4].record()
+        st = B.bload_stats(p.info)
+        if rec is not None:
+            rec.append((e, B.bload_plan_stage_times(), st))
+        return st
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        step()
+    barrier()
+    sampler = ClockSampler(local)
+    sampler.start()
+    launches0 = B.bload_kernel_launches()
+    rec = []
+    t_begin, t_end = ev(), ev()
+    barrier()
+    t_begin.record()
+    for _ in range(args.steps):
+        stats = step(rec)
+    t_end.record()
+    barrier()
+    launches = B.bload_kernel_launches() - launches0
+    seconds = dist_max(t_begin.elapsed_time(t_end) / 1e3, dev)
+    clocks = sampler.stop()
+
+    def avg(i):
+        return sum(r[0][i].elapsed_time(r[0][i + 1]) for r in rec) / len(rec)
+    plan_ms, meta_ms, pack_ms, unpack_ms = avg(0), avg(1), avg(2), avg(3)
+    stage = [sum(r[1][i] for r in rec) / len(rec) for i in range(4)]
+    step_s = seconds / args.steps
+    value = aggregate(by["pack"] + by["unpack"], world, step_s) / 1e9
+
+    # ---- end to end through the same calls with HOST buffers (pinned), copies inside the timed region
+    e2e = None
+    if not args.no_e2e:
+        h_len = torch.from_numpy(T).pin_memory()
+        h_store = torch.empty(store.numel(), dtype=torch.uint8, pin_memory=True); h_store.copy_(store)
+        h_dense = torch.empty(dense.numel(), dtype=torch.uint8, pin_memory=True)
+        h_meta = [torch.empty(x.numel(), dtype=x.dtype, pin_memory=True) for x in (seq_id, pos, reset, valid)]
+        h_dense_out = torch.empty(dense_out.numel(), dtype=torch.uint8, pin_memory=True); h_dense_out.copy_(dense_out)
+        h_ragged_out = torch.empty(ragged_out.numel(), dtype=torch.uint8, pin_memory=True)
+        h2d = h_len.numel() * 4 + h_store.numel() + h_dense_out.numel()
+        d2h = h_dense.numel() + sum(x.numel() * x.element_size() for x in h_meta) + h_ragged_out.numel()
+
+        def e2e_step():
+            d_len.copy_(h_len, non_blocking=True)
+            store.copy_(h_store, non_blocking=True)
+            p = B.bload_plan(d_len, tb, w.seed, work=work, plan_buf=plan_buf)
+            B.bload_pack(p, store, fb, 0, nb, dense=dense, seq_id=seq_id, pos=pos, reset=reset, valid=valid)
+            h_dense.copy_(dense, non_blocking=True)
+            for h, d in zip(h_meta, (seq_id, pos, reset, valid)):
+                h.copy_(d, non_blocking=True)
+            dense_out.copy_(h_dense_out, non_blocking=True)
+            B.bload_unpack(p, dense_out, ofb, 0, nb, ragged_out)
+            h_ragged_out.copy_(ragged_out, non_blocking=True)
+            return B.bload_stats(p.info)
+
+        e2e_step()
+        barrier()
+        a, b_ = ev(), ev()
+        a.record()
+        for _ in range(args.e2e_steps):
+            e2e_step()
+        b_.record()
+        barrier()
+        e2e_s = dist_max(a.elapsed_time(b_) / 1e3, dev) / args.e2e_steps
+        e2e = {"value": aggregate(by["pack"] + by["unpack"], world, e2e_s) / 1e9, "unit": UNIT,
+               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": e2e_s * 1e3,
+               "steps": args.e2e_steps}
+        del h_store, h_dense, h_dense_out, h_ragged_out
+
+    if rank != 0:
+        return {}
+
+    peak, peak_kind = measured_peak()
+    kernels = {"k7_copy<unpack>": (unpack_ms, by["unpack"]), "k7_copy<pack>": (pack_ms, by["pack"]),
+               "k4_fill": (stage[2], None)}
+    dom = max(("k7_copy<unpack>", "k7_copy<pack>"), key=lambda k: kernels[k][0])
+    d_ms, d_bytes = kernels[dom]
+    achieved = d_bytes / (d_ms / 1e3) / 1e9
+    roofline = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "GB/s",
+                "frac": achieved / peak, "peak_kind": "of " + peak_kind, "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
+                "traffic": TRAFFIC.get((w.name, dom)), "launch_ms": d_ms, "algorithmic_bytes_per_launch": d_bytes}
+
+    out = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+           "ms_per_step": step_s * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+           "dtype": "u8", "data": "synthetic", "config": config_of(w, {"parallelism": "replicas only"}),
+           "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline,
+           "frames_per_s": aggregate(sum_t, world, step_s),
+           "kernels": {
+               "pack_copy": {"ms": pack_ms, "GB/s": by["pack"] / pack_ms / 1e6, "frac_measured": by["pack"] / pack_ms / 1e6 / peak,
+                             "frac_nominal": by["pack"] / pack_ms / 1e6 / NOMINAL_HBM_GBS, "frames_per_s": sum_t / pack_ms * 1e3},
+               "unpack_copy": {"ms": unpack_ms, "GB/s": by["unpack"] / unpack_ms / 1e6,
+                               "frac_measured": by["unpack"] / unpack_ms / 1e6 / peak,
+                               "frac_nominal": by["unpack"] / unpack_ms / 1e6 / NOMINAL_HBM_GBS,
+                               "frames_per_s": sum_t / unpack_ms * 1e3},
+               "metadata": {"ms": meta_ms, "GB/s": by["meta"] / meta_ms / 1e6},
+               "plan": {"ms": plan_ms, "scan_keys_ms": stage[0], "sort_ms": stage[1], "fill_ms": stage[2],
+                        "tables_ms": stage[3], "draws_per_s": T.size / stage[2] * 1e3 if stage[2] > 0 else None}},
+           "padding": {"n": stats["n"], "sum_t": stats["sum_t"], "t_max": stats["t_max"], "n_blocks": stats["n_blocks"],
+                       "min_blocks": stats["min_blocks"], "frac_packed": stats["frac_packed"],
+                       "frac_naive_tmax": stats["frac_naive_tmax"], "frac_naive_tblock": stats["frac_naive_tblock"],
+                       "reduction_vs_tmax": stats["reduction_vs_tmax"]}}
+    if not args.no_cpu and world == 1:
+        cb = cpu_oracle_sample(w, args.ref_blocks)
+        out["cpu_baseline"] = {k: v for k, v in cb.items() if not k.startswith("_")}
+    else:
+        out["cpu_baseline"] = None
+    return out
+
+
+# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the committed ncu captures
+# under profiles/; null where the kernel has changed since the counters were taken.
+TRAFFIC: dict = {}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="bload", choices=["bload", "reference"])
+    ap.add_argument("--workload", default="heavy_tail_bf16")
+    ap.add_argument("--n", type=int, default=0, help="override the number of sequences (small profiling cases)")
+    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--ref-blocks", type=int, default=24, help="blocks in the CPU oracle's sample")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "bload" else args.warmup
+
+    from paper_2310_10879_b200 import workloads as W
+    w = W.WORKLOADS[args.workload]
+    if args.n:
+        w = W.scaled(w, args.n)
+
+    if args.impl == "reference":
+        if int(os.environ.get("RANK", "0")) == 0:
+            print(json.dumps(run_reference(args, w)), flush=True)
+        return
+    out = run_gpu(args, w)
+    if out:
+        print(json.dumps(out), flush=True)
+    import torch.distributed as dist
+    if dist.is_available() and dist.is_initialized():
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

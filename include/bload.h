@@ -13,7 +13,8 @@
  * Conventions
  *   - "d_" pointers are DEVICE pointers; all others are HOST pointers.
  *   - The caller owns every buffer.  The library allocates no device memory and keeps no state
- *     between calls; a plan is position independent (tables addressed by byte offsets) and can
+ *     between calls (apart from the benchmarking counters at the end of this file); a plan is
+ *     position independent (tables addressed by byte offsets) and can
  *     be copied or saved as a blob of bload_sizes_t.plan_bytes bytes.
  *   - `stream` is a cudaStream_t passed as void* (NULL = default stream).
  *   - Every function returns BLOAD_OK (0) or a negative BLOAD_ERR_* code.  Errors that the host
@@ -172,6 +173,12 @@ BLOAD_API int bload_stats(const bload_plan_info_t* info, bload_stats_t* out);
  */
 BLOAD_API int bload_set_plan_timing(int enable);
 BLOAD_API int bload_plan_stage_times(float out_ms[4]);
+
+/*
+ * bload_kernel_launches -- number of kernels this library has launched in this process so far
+ * (all threads).  Host only; lets a benchmark report how many launches a timed region contained.
+ */
+BLOAD_API int64_t bload_kernel_launches(void);
 
 BLOAD_API const char* bload_strerror(int code);
 BLOAD_API int bload_version(void);

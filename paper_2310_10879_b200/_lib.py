@@ -18,7 +18,8 @@ ERR_UNSUPPORTED, ERR_CUDA, ERR_TIMEOUT, ERR_PLAN = -6, -7, -8, -9
 MAX_T_BLOCK = 32768
 
 EXPORTS = ("bload_plan_sizes", "bload_plan", "bload_pack", "bload_unpack", "bload_stats",
-           "bload_set_plan_timing", "bload_plan_stage_times", "bload_strerror", "bload_version")
+           "bload_set_plan_timing", "bload_plan_stage_times", "bload_kernel_launches", "bload_strerror",
+           "bload_version")
 
 
 class Sizes(C.Structure):
@@ -72,9 +73,11 @@ def load() -> C.CDLL:
     L.bload_strerror.argtypes = [C.c_int]
     L.bload_strerror.restype = C.c_char_p
     L.bload_version.argtypes = []
+    L.bload_kernel_launches.argtypes = []
     for name in EXPORTS:
-        if name != "bload_strerror":
+        if name not in ("bload_strerror", "bload_kernel_launches"):
             getattr(L, name).restype = C.c_int
+    L.bload_kernel_launches.restype = C.c_int64
     _lib = L
     return L
 
@@ -198,3 +201,7 @@ def bload_plan_stage_times() -> list[float]:
     if rc:
         raise BloadError(rc, "bload_plan_stage_times")
     return [float(x) for x in out]
+
+
+def bload_kernel_launches() -> int:
+    return int(load().bload_kernel_launches())

@@ -1,6 +1,8 @@
 // C ABI of libbload: argument checks, buffer layouts, launches.  See include/bload.h.
 #include <string.h>
 
+#include <atomic>
+
 #include "bload_internal.cuh"
 
 namespace bload {
@@ -42,6 +44,9 @@ PlanView plan_view(void* d_plan, int64_t n)
     return v;
 }
 
+static std::atomic<long long> g_launches{0};
+void count_launches(int k) { g_launches.fetch_add(k, std::memory_order_relaxed); }
+
 namespace {
 thread_local bool g_timing = false;
 thread_local bool g_have_times = false;
@@ -75,6 +80,8 @@ using namespace bload;
 extern "C" {
 
 int bload_version(void) { return 1; }
+
+int64_t bload_kernel_launches(void) { return (int64_t)g_launches.load(std::memory_order_relaxed); }
 
 const char* bload_strerror(int code)
 {

@@ -197,6 +197,7 @@ cudaError_t launch_copy(bool unpack, const PlanView& pv, int32_t t_block, int64_
     else
         k7_copy<false><<<grid, 256, 0, st>>>(pv, t_block, frame_bytes, block_begin, block_count, ragged_in, dense,
                                               ragged_bytes, sub, spb, pad_byte);
+    count_launches(1);
     return cudaPeekAtLastError();
 }
 

@@ -65,6 +65,9 @@ size_t work_layout(int64_t n, int32_t t_block, void* base, WorkView* w);
 void plan_layout(int64_t n, bload_sizes_t* s);
 PlanView plan_view(void* d_plan, int64_t n);
 
+// every kernel launch of the library goes through this counter (see bload_kernel_launches)
+void count_launches(int k);
+
 // launchers (each returns a cudaError_t from cudaPeekAtLastError)
 cudaError_t launch_plan(const int32_t* d_lengths, int64_t n, int32_t t_block, uint64_t seed, uint32_t policy,
                         const PlanView& pv, const WorkView& wv, cudaStream_t st, cudaEvent_t* ev /*5 or null*/);

@@ -92,6 +92,7 @@ cudaError_t launch_metadata(const PlanView& pv, int32_t t_block, int64_t block_b
         k6_metadata<4, true><<<grid, 256, 0, st>>>(pv, t_block, block_begin, block_count, gpb, seq_id, pos, reset, valid);
     else
         k6_metadata<4, false><<<grid, 256, 0, st>>>(pv, t_block, block_begin, block_count, gpb, seq_id, pos, reset, valid);
+    count_launches(1);
     return cudaPeekAtLastError();
 }
 

@@ -481,6 +481,7 @@ cudaError_t launch_plan(const int32_t* d_lengths, int64_t n, int32_t t_block, ui
 
     k5_tables<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(pv, wv.draw_rec, wv.bucket_end, iin, n);
     k5_finish<<<1, 32, 0, st>>>(pv.hdr);
+    count_launches(4 + 3 * passes + 1 + 1 + 2);
     if (ev) cudaEventRecord(ev[4], st);
     return cudaPeekAtLastError();
 }
