@@ -7,8 +7,8 @@
 //      (shuffle key h_i) and one per draw (u_k);
 //   2. a stable LSD radix sort of the ids by (T_i, h_i): L_dict as one array, buckets by length,
 //      each bucket pre-shuffled;
-//   3. the fill rule itself, a chain of n dependent draws run by one warp over a two-level table of
-//      running counts kept in shared memory;
+//   3. the fill rule itself, a chain of n dependent draws run by one warp over a three-level table
+//      of running counts kept in shared memory;
 //   4. a parallel pass that resolves draws to sequence ids and writes the inverse tables.
 #include <limits.h>
 
@@ -283,79 +283,80 @@ __global__ void __launch_bounds__(256) k3_buckets(const uint64_t* __restrict__ k
 }
 
 // ---- the fill rule: one warp, n dependent draws ----
-// Shared memory holds running counts of UNUSED sequences as inclusive prefix sums:
-//   P0[g]        sequences with length <= 256*(g+1)           (128 entries)
-//   P1[g][i]     sequences with length in (256*g, 256*g+i+1]   (groups of 256 lengths)
-// so that "how many fit in r slots" is two reads and "the j-th of them in order of length" is two
-// compare-and-count steps; a draw then decrements the entries at and after the chosen length.
+// Shared memory holds running counts of UNUSED sequences as a three-level, 32-ary table of inclusive
+// prefix sums over the lengths (leaf x stands for length x + 1; x = a*1024 + b*32 + c):
+//   Q0[a]          sequences with x < (a+1)*1024                         (32 entries, also one per lane)
+//   Q1[a][b]       sequences with a*1024 <= x < a*1024 + (b+1)*32         (32 x 32)
+//   Q2[a*32+b][c]  sequences with (a*32+b)*32 <= x <= (a*32+b)*32 + c     (one row of 32 per 32 lengths)
+// "How many fit in r slots" is three reads; "the j-th of them in order of length" is one
+// compare + ballot + popcount per level with one entry per lane; a draw then decrements the entries
+// at and after the chosen digit in one row per level.
 __global__ void __launch_bounds__(256, 1) k4_fill(PlanView pv, const int32_t* __restrict__ bucket_end,
                                                   const uint64_t* __restrict__ draw_u, int4* __restrict__ draw_rec,
                                                   int64_t n64, int32_t L)
 {
     extern __shared__ __align__(16) int32_t sm[];
-    int32_t* P0 = sm;
-    int32_t* P1 = sm + 128;
+    int32_t* Q0 = sm;              // [32]
+    int32_t* Q1 = sm + 32;         // [32][32]
+    int32_t* Q2 = sm + 32 + 1024;  // [rows][32], rows = ceil(L / 32)
     if (pv.hdr->first_bad != kNoBad) return;
-    const int G = (L + 255) >> 8;
-    for (int idx = threadIdx.x; idx < G * 256; idx += blockDim.x) {
-        int g = idx >> 8;
-        int hi = min(idx + 1, L);
-        P1[idx] = bucket_end[hi] - bucket_end[g << 8];
-    }
-    for (int g = threadIdx.x; g < 128; g += blockDim.x) P0[g] = bucket_end[min((g + 1) << 8, L)];
+    const int rows = (L + 31) >> 5;
+    auto upto = [&](int l) { return bucket_end[min(l, L)]; };  // sequences with length <= l
+    for (int idx = threadIdx.x; idx < rows * 32; idx += blockDim.x) Q2[idx] = upto(idx + 1) - upto(idx & ~31);
+    for (int idx = threadIdx.x; idx < 1024; idx += blockDim.x) Q1[idx] = upto((idx + 1) << 5) - upto((idx >> 5) << 10);
+    if (threadIdx.x < 32) Q0[threadIdx.x] = upto((threadIdx.x + 1) << 10);
     __syncthreads();
     if (threadIdx.x >= 32) return;
 
     const int lane = threadIdx.x;
     const int n = (int)n64;
-    int4 p0 = reinterpret_cast<int4*>(P0)[lane];
+    int q0 = Q0[lane];
     int k = 0, b = 0, room = L, start = 0;
     if (lane == 0) pv.block_seg_begin[0] = 0;
-    uint64_t u_next = draw_u[0];
+    // random words of 32 draws at a time, one per lane, the next 32 prefetched
+    uint64_t u_cur = lane < n ? draw_u[lane] : 0;
+    uint64_t u_nxt = 32 + lane < n ? draw_u[32 + lane] : 0;
     while (k < n) {
+        const uint64_t u = __shfl_sync(kFull, u_cur, k & 31);
         int m = 0;
         if (room > 0) {
-            int y = room - 1, gy = y >> 8;
-            m = P1[y] + (gy ? P0[gy - 1] : 0);
+            const int y = room - 1, ya = y >> 10, yb = (y >> 5) & 31;
+            m = Q2[y] + (yb ? Q1[(ya << 5) + yb - 1] : 0) + (ya ? Q0[ya - 1] : 0);
         }
         if (m == 0) {  // nothing fits: the rest of the block is padding
             if (lane == 0) { pv.block_fill[b] = start; pv.block_seg_begin[b + 1] = k; }
             ++b; room = L; start = 0;
             continue;
         }
-        const uint64_t u = u_next;
-        if (k + 1 < n) u_next = draw_u[k + 1];
-        const int j = (int)__umul64hi(u, (uint64_t)(unsigned)m);  // floor(u * m / 2^64)
-        int c = (p0.x <= j) + (p0.y <= j) + (p0.z <= j) + (p0.w <= j);
-        const int g = __reduce_add_sync(kFull, c);
-        const int j1 = j - (g ? P0[g - 1] : 0);
-        int4* row = reinterpret_cast<int4*>(P1 + (g << 8));
-        int4 va = row[2 * lane], vb = row[2 * lane + 1];
-        c = (va.x <= j1) + (va.y <= j1) + (va.z <= j1) + (va.w <= j1) + (vb.x <= j1) + (vb.y <= j1) + (vb.z <= j1) +
-            (vb.w <= j1);
-        const int i = __reduce_add_sync(kFull, c);
-        const int len = (g << 8) + i + 1;
-        int prev = __shfl_up_sync(kFull, vb.w, 1);
-        if (lane == 0) prev = 0;
-        const int owner = i >> 3, e = i & 7;
-        if (lane == owner) {
-            int cur = e == 0 ? va.x : e == 1 ? va.y : e == 2 ? va.z : e == 3 ? va.w : e == 4 ? vb.x : e == 5 ? vb.y : e == 6 ? vb.z : vb.w;
-            int prv = e == 0 ? prev : e == 1 ? va.x : e == 2 ? va.y : e == 3 ? va.z : e == 4 ? va.w : e == 5 ? vb.x : e == 6 ? vb.y : vb.z;
-            draw_rec[k] = make_int4(len, cur - prv, b, start);
-        }
-        {
-            const int f = 4 * lane;
-            p0.x -= (f + 0 >= g); p0.y -= (f + 1 >= g); p0.z -= (f + 2 >= g); p0.w -= (f + 3 >= g);
-            if (f + 3 >= g) reinterpret_cast<int4*>(P0)[lane] = p0;
-        }
-        if (lane >= owner) {
-            const int f = 8 * lane;
-            va.x -= (f + 0 >= i); va.y -= (f + 1 >= i); va.z -= (f + 2 >= i); va.w -= (f + 3 >= i);
-            vb.x -= (f + 4 >= i); vb.y -= (f + 5 >= i); vb.z -= (f + 6 >= i); vb.w -= (f + 7 >= i);
-            row[2 * lane] = va; row[2 * lane + 1] = vb;
-        }
+        // j = floor(u * m / 2^64), m < 2^31, from 32-bit pieces
+        int j = (int)(((uint64_t)(uint32_t)(u >> 32) * (uint32_t)m + __umulhi((uint32_t)u, (uint32_t)m)) >> 32);
+        // level 0
+        const int a = __popc(__ballot_sync(kFull, q0 <= j));
+        const int q1 = Q1[(a << 5) + lane];
+        int base = __shfl_sync(kFull, q0, (a - 1) & 31);
+        j -= a ? base : 0;
+        // level 1
+        const int bb = __popc(__ballot_sync(kFull, q1 <= j));
+        const int row = (a << 5) + bb;
+        const int q2 = Q2[(row << 5) + lane];
+        base = __shfl_sync(kFull, q1, (bb - 1) & 31);
+        j -= bb ? base : 0;
+        // level 2
+        const int c = __popc(__ballot_sync(kFull, q2 <= j));
+        const int len = (row << 5) + c + 1;
+        // decrement the running counts at and after the chosen digits
+        if (lane >= a) { --q0; Q0[lane] = q0; }
+        if (lane >= bb) Q1[(a << 5) + lane] = q1 - 1;
+        if (lane >= c) Q2[(row << 5) + lane] = q2 - 1;
+        int below = __shfl_up_sync(kFull, q2, 1);
+        if (lane == 0) below = 0;
+        if (lane == c) draw_rec[k] = make_int4(len, q2 - below, b, start);  // q2 - below: unused of this length
         __syncwarp();
         room -= len; start += len; ++k;
+        if ((k & 31) == 0) {
+            u_cur = u_nxt;
+            u_nxt = k + 32 + lane < n ? draw_u[k + 32 + lane] : 0;
+        }
     }
     if (lane == 0) {
         pv.block_fill[b] = start;
@@ -472,8 +473,7 @@ cudaError_t launch_plan(const int32_t* d_lengths, int64_t n, int32_t t_block, ui
     k3_buckets<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(kin, n, t_block, wv.bucket_end, pv.hdr);
     if (ev) cudaEventRecord(ev[2], st);
 
-    const int G = (t_block + 255) >> 8;
-    const size_t smem = sizeof(int32_t) * (128 + (size_t)G * 256);
+    const size_t smem = sizeof(int32_t) * (32 + 1024 + (size_t)((t_block + 31) / 32) * 32);
     cudaError_t e = cudaFuncSetAttribute(k4_fill, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     k4_fill<<<1, 256, smem, st>>>(pv, wv.bucket_end, wv.draw_u, wv.draw_rec, n, t_block);
