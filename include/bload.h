@@ -166,6 +166,42 @@ BLOAD_API int bload_unpack(const void* d_plan, const bload_plan_info_t* info, co
 BLOAD_API int bload_stats(const bload_plan_info_t* info, bload_stats_t* out);
 
 /*
+ * bload_plan_static -- bload_plan for callers that must not, or cannot, allocate device memory.
+ * (The paper has no counterpart of this call; it is a packaging variant of bload_plan and computes
+ * exactly the same plan.)
+ *
+ * bload_plan needs a scratch buffer from its caller.  A data-loading thread that lives next to a
+ * training job usually cannot get one: the framework's caching allocator has already taken the
+ * device's memory, so a new cudaMalloc may fail, and even when it succeeds it can stall every
+ * stream on the device while the driver serves it.  The same goes for loops that are simply
+ * forbidden to touch the allocator.  This entry point keeps its scratch in a fixed array of
+ * BLOAD_STATIC_SCRATCH_BYTES bytes inside the library image, so it calls no cudaMalloc, no
+ * cudaFree and no allocating routine of any library.  The price: every GPU that loads the
+ * library holds those bytes until the process exits, and the problem size is capped.
+ *
+ *   d_lengths, n, t_block, seed, policy, d_plan, plan_bytes, stream, info: as for bload_plan
+ *   (the caller still provides the input and the plan buffer; only d_work/work_bytes are gone).
+ *
+ * Limits and errors: n > BLOAD_STATIC_MAX_N, or a (n, t_block) whose scratch need exceeds the
+ * array, returns BLOAD_ERR_WORKSPACE ("buffer too small") and launches nothing; use bload_plan
+ * with your own buffer for larger problems.  All other errors are those of bload_plan.
+ *
+ * First call on a device: the library looks up the device address of its array (the current
+ * device must be the one the buffers live on).  Make that first call outside any stream capture.
+ *
+ * Sharing: all calls on a device use the same array and it keeps whatever the last call left.
+ * The planner overwrites every scratch table it reads, so nothing has to be cleared between
+ * calls; but two calls whose kernels overlap on the GPU (different streams or threads) race on
+ * the array and produce garbage.  Run them one after the other, as this call itself does: like
+ * bload_plan it synchronises `stream` once before it returns.
+ */
+#define BLOAD_STATIC_MAX_N 65536
+#define BLOAD_STATIC_SCRATCH_BYTES (4u << 20)
+BLOAD_API int bload_plan_static(const int32_t* d_lengths, int64_t n, int32_t t_block, uint64_t seed,
+                                uint32_t policy, void* d_plan, size_t plan_bytes, void* stream,
+                                bload_plan_info_t* info);
+
+/*
  * bload_plan_stage_times -- device time, in milliseconds, that the most recent bload_plan call of
  * this thread spent in each stage: [0] validate + scan + keys, [1] key sort, [2] fill rule,
  * [3] inverse tables.  Host only; for benchmarking.  Returns BLOAD_ERR_PLAN when no plan was timed.

@@ -205,3 +205,35 @@ def bload_plan_stage_times() -> list[float]:
 
 def bload_kernel_launches() -> int:
     return int(load().bload_kernel_launches())
+
+
+STATIC_MAX_N = 65536
+
+
+def bload_plan_static(lengths, t_block: int, seed: int, policy: int = 0, stream=None, plan_buf=None,
+                      check: bool = True) -> Plan:
+    """bload_plan without a caller-provided scratch buffer, for callers that cannot allocate device
+    memory (for example a loader thread beside a training job whose allocator owns the device).
+    The library's built-in scratch array is used instead, which caps n at STATIC_MAX_N; calls that
+    overlap on the GPU race on that array.  Pass a pre-made `plan_buf` to avoid every allocation;
+    without one this wrapper (not the library) allocates the plan buffer with torch."""
+    import torch
+    if not lengths.is_cuda or lengths.dtype != torch.int32 or not lengths.is_contiguous():
+        raise TypeError("lengths must be a contiguous CUDA int32 tensor")
+    L = load()
+    fn = L.bload_plan_static
+    fn.argtypes = [C.c_void_p, C.c_int64, C.c_int32, C.c_uint64, C.c_uint32, C.c_void_p, C.c_size_t, C.c_void_p,
+                   C.POINTER(PlanInfo)]
+    fn.restype = C.c_int
+    n = lengths.numel()
+    sizes = bload_plan_sizes(n, t_block)
+    if plan_buf is None:
+        plan_buf = torch.empty(sizes.plan_bytes, dtype=torch.uint8, device=lengths.device)
+    info = PlanInfo()
+    rc = fn(lengths.data_ptr(), n, t_block, seed, policy, plan_buf.data_ptr(), plan_buf.numel(), _stream(stream),
+            C.byref(info))
+    if rc and check:
+        err = BloadError(rc, "bload_plan_static")
+        err.info = info
+        raise err
+    return Plan(plan_buf, info, sizes)
