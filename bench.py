@@ -68,7 +68,11 @@ class ClockSampler:
 
     def _read(self):
         for line in self.proc.stdout:
-            self.rows.append([x.strip() for x in line.split(",")])
+            self.rows.append([time.monotonic()] + [x.strip() for x in line.split(",")])
+
+    def mark(self):
+        """Start of the timed region: only samples taken after this moment are reported."""
+        self.t_mark = time.monotonic()
 
     def stop(self) -> dict:
         if self.proc is None:
@@ -80,7 +84,9 @@ class ClockSampler:
             self.proc.kill()
         self.thread.join(timeout=2)
         sm, mx, reasons, pw = [], [], set(), []
-        for r in self.rows:
+        t_mark = getattr(self, "t_mark", 0.0)
+        rows = [r[1:] for r in self.rows if r[0] >= t_mark] or [r[1:] for r in self.rows[-1:]]
+        for r in rows:
             try:
                 sm.append(float(r[0])); mx.append(float(r[1])); pw.append(float(r[2]))
                 for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), r[3:7]):
@@ -109,50 +115,72 @@ def aggregate(units_per_rank: float, world: int, seconds_max: float) -> float:
 
 
 # ----------------------------------------------------------------------------------------------
-def cpu_oracle_sample(w, target_blocks: int) -> dict:
-    """Time the CPU oracle, as it stands, on a bounded sample of the workload: the full plan, then
-    metadata + pack + unpack of `target_blocks` consecutive blocks (single thread)."""
-    import numpy as np
-    from oracle import bload_oracle as O
-    from paper_2310_10879_b200 import workloads as W
-    T = W.lengths(w)
-    t0 = time.perf_counter()
-    op = O.plan(T, w.t_block, w.seed)
-    t_plan = time.perf_counter() - t0
-    fb, ofb, tb = w.frame_bytes, w.out_frame_bytes, w.t_block
-    cnt = min(target_blocks, op.n_blocks)
-    b0 = (op.n_blocks - cnt) // 2
-    # host store: only the frames of the sampled blocks' sequences are touched (rest stays untouched virtual memory)
-    store = np.empty(op.sum_t * fb, np.uint8)
-    frames = 0
-    rng = np.random.default_rng(1)
-    for k in range(op.block_seg_begin[b0], op.block_seg_begin[b0 + cnt]):
-        s = int(op.seg_seq[k]); lo, hi = int(op.offsets[s]) * fb, int(op.offsets[s + 1]) * fb
-        store[lo:hi] = rng.integers(0, 256, size=1, dtype=np.uint8)[0]
-        frames += int(op.offsets[s + 1] - op.offsets[s])
-    dense_out = np.ones(cnt * tb * ofb, np.uint8)
-    ragged_out = np.empty(op.sum_t * ofb, np.uint8)
-    for k in range(op.block_seg_begin[b0], op.block_seg_begin[b0 + cnt]):  # fault the output pages in before timing
-        s = int(op.seg_seq[k]); ragged_out[int(op.offsets[s]) * ofb:int(op.offsets[s + 1]) * ofb] = 0
-    t0 = time.perf_counter(); O.metadata(op, b0, cnt); t_meta = time.perf_counter() - t0
-    t0 = time.perf_counter(); O.pack(op, store, fb, b0, cnt, 0); t_pack = time.perf_counter() - t0
-    t0 = time.perf_counter(); O.unpack(op, dense_out, ofb, b0, cnt, ragged_out); t_unpack = time.perf_counter() - t0
-    frac = cnt / op.n_blocks
-    by = dict(pack=frames * fb + cnt * tb * fb, unpack=2 * frames * ofb)
-    t_total = t_plan * frac + t_meta + t_pack + t_unpack
-    return dict(value=(by["pack"] + by["unpack"]) / t_total / 1e9, unit=UNIT, cores=1, kind="oracle",
-                sample="full plan (N=%d, %.3f s, charged pro rata) + metadata/pack/unpack of %d of %d blocks "
-                       "(%d frames); pack %.2f GB/s, unpack %.2f GB/s, single thread"
-                       % (op.n, t_plan, cnt, op.n_blocks, frames, by["pack"] / t_pack / 1e9, by["unpack"] / t_unpack / 1e9),
-                seconds=t_plan + t_meta + t_pack + t_unpack, frames_per_s=frames / t_total,
-                plan_s=t_plan, _bytes=by["pack"] + by["unpack"], _t=t_total)
+class CpuOracleSample:
+    """The CPU oracle, as it stands, on a bounded sample of the workload: the full plan, then
+    metadata + pack + unpack of `target_blocks` consecutive blocks (0 = all), single thread.
+    Buffers are set up once; run() times one pass."""
+
+    def __init__(self, w, target_blocks: int):
+        import numpy as np
+        from oracle import bload_oracle as O
+        from paper_2310_10879_b200 import workloads as W
+        self.O, self.w = O, w
+        self.T = W.lengths(w)
+        op = self.plan()
+        fb, ofb, tb = w.frame_bytes, w.out_frame_bytes, w.t_block
+        self.cnt = cnt = min(target_blocks, op.n_blocks) if target_blocks > 0 else op.n_blocks
+        self.b0 = b0 = (op.n_blocks - cnt) // 2
+        # host store: only the frames of the sampled blocks' sequences are touched (the rest stays untouched
+        # virtual memory); the output pages are faulted in before timing
+        self.store = np.empty(op.sum_t * fb, np.uint8)
+        self.ragged_out = np.empty(op.sum_t * ofb, np.uint8)
+        self.frames = 0
+        for k in range(op.block_seg_begin[b0], op.block_seg_begin[b0 + cnt]):
+            s = int(op.seg_seq[k]); lo, hi = int(op.offsets[s]), int(op.offsets[s + 1])
+            self.store[lo * fb:hi * fb] = (s * 37 + 11) & 255
+            self.ragged_out[lo * ofb:hi * ofb] = 0
+            self.frames += hi - lo
+        self.dense_out = np.ones(cnt * tb * ofb, np.uint8)
+        self.bytes = dict(pack=self.frames * fb + cnt * tb * fb, unpack=2 * self.frames * ofb)
+
+    def plan(self):
+        t0 = time.perf_counter()
+        self.op = self.O.plan(self.T, self.w.t_block, self.w.seed)
+        self.t_plan = time.perf_counter() - t0
+        return self.op
+
+    def run(self) -> dict:
+        O, w, op = self.O, self.w, self.plan()
+        fb, ofb = w.frame_bytes, w.out_frame_bytes
+        t0 = time.perf_counter(); O.metadata(op, self.b0, self.cnt); t_meta = time.perf_counter() - t0
+        t0 = time.perf_counter(); O.pack(op, self.store, fb, self.b0, self.cnt, 0); t_pack = time.perf_counter() - t0
+        t0 = time.perf_counter(); O.unpack(op, self.dense_out, ofb, self.b0, self.cnt, self.ragged_out)
+        t_unpack = time.perf_counter() - t0
+        by = self.bytes
+        t_total = self.t_plan * self.cnt / op.n_blocks + t_meta + t_pack + t_unpack
+        return dict(value=(by["pack"] + by["unpack"]) / t_total / 1e9, unit=UNIT, cores=1, kind="oracle",
+                    sample="full plan (N=%d, %.3f s, charged pro rata) + metadata/pack/unpack of %d of %d blocks "
+                           "(%d frames); pack %.2f GB/s, unpack %.2f GB/s, single thread"
+                           % (op.n, self.t_plan, self.cnt, op.n_blocks, self.frames, by["pack"] / t_pack / 1e9,
+                              by["unpack"] / t_unpack / 1e9),
+                    seconds=self.t_plan + t_meta + t_pack + t_unpack, frames_per_s=self.frames / t_total,
+                    plan_s=self.t_plan, _bytes=by["pack"] + by["unpack"], _t=t_total)
 
 
 def run_reference(args, w) -> dict:
-    """The reference arm: the CPU oracle on this machine's host cores, a bounded sample per step."""
+    """The reference arm: the CPU oracle on this machine's host cores, a bounded sample per step.  The
+    sample (blocks per step) is sized from a 2-block calibration so that the whole run of
+    warmup + steps stays near two minutes."""
+    blocks = args.ref_blocks
+    if blocks <= 0:
+        cal = CpuOracleSample(w, 2).run()
+        per_block = max(cal["seconds"] - cal["plan_s"], 1e-3) / 2
+        budget = 100.0 / max(1, args.warmup + args.steps) - cal["plan_s"]
+        blocks = int(max(1, min(budget / per_block, 64)))
+    sample = CpuOracleSample(w, blocks)
     times, last = [], None
     for i in range(args.warmup + args.steps):
-        r = cpu_oracle_sample(w, max(1, args.ref_blocks // 4))
+        r = sample.run()
         if i >= args.warmup:
             times.append(r["_t"])
         last = r
@@ -240,15 +268,16 @@ def run_gpu(args, w) -> dict:
             dist.barrier()
         torch.cuda.synchronize()
 
+    sampler = ClockSampler(local)
+    sampler.start()
     for _ in range(args.warmup):
         step()
     barrier()
-    sampler = ClockSampler(local)
-    sampler.start()
     launches0 = B.bload_kernel_launches()
     rec = []
     t_begin, t_end = ev(), ev()
     barrier()
+    sampler.mark()
     t_begin.record()
     for _ in range(args.steps):
         stats = step(rec)
@@ -337,7 +366,7 @@ def run_gpu(args, w) -> dict:
                        "frac_naive_tmax": stats["frac_naive_tmax"], "frac_naive_tblock": stats["frac_naive_tblock"],
                        "reduction_vs_tmax": stats["reduction_vs_tmax"]}}
     if not args.no_cpu and world == 1:
-        cb = cpu_oracle_sample(w, args.ref_blocks)
+        cb = CpuOracleSample(w, args.ref_blocks).run()
         out["cpu_baseline"] = {k: v for k, v in cb.items() if not k.startswith("_")}
     else:
         out["cpu_baseline"] = None
@@ -352,13 +381,15 @@ TRAFFIC: dict = {}
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="bload", choices=["bload", "reference"])
     ap.add_argument("--workload", default="heavy_tail_bf16")
     ap.add_argument("--n", type=int, default=0, help="override the number of sequences (small profiling cases)")
     ap.add_argument("--e2e-steps", type=int, default=3)
-    ap.add_argument("--ref-blocks", type=int, default=24, help="blocks in the CPU oracle's sample")
+    ap.add_argument("--ref-blocks", type=int, default=0,
+                    help="blocks in the CPU oracle's sample (0 = all blocks for the CPU baseline; sized from a "
+                         "calibration run for --impl reference)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     args = ap.parse_args()
