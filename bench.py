@@ -386,6 +386,7 @@ def main():
     ap.add_argument("--impl", default="bload", choices=["bload", "reference"])
     ap.add_argument("--workload", default="heavy_tail_bf16")
     ap.add_argument("--n", type=int, default=0, help="override the number of sequences (small profiling cases)")
+    ap.add_argument("--frame-bytes", type=int, default=0, help="override the frame size of the workload (experiments)")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--ref-blocks", type=int, default=0,
                     help="blocks in the CPU oracle's sample (0 = all blocks for the CPU baseline; sized from a "
@@ -399,6 +400,9 @@ def main():
     w = W.WORKLOADS[args.workload]
     if args.n:
         w = W.scaled(w, args.n)
+    if args.frame_bytes:
+        from dataclasses import replace
+        w = replace(w, frame_bytes=args.frame_bytes, out_frame_bytes=args.frame_bytes, payload="u8")
 
     if args.impl == "reference":
         if int(os.environ.get("RANK", "0")) == 0:

@@ -10,7 +10,7 @@ import os
 from dataclasses import dataclass
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libbload.so")
+LIB_PATH = os.environ.get("BLOAD_LIBRARY") or os.path.join(_HERE, "libbload.so")  # override: a build to compare
 
 OK = 0
 ERR_NULL, ERR_ARG, ERR_LENGTH, ERR_WORKSPACE, ERR_ALIGN = -1, -2, -3, -4, -5

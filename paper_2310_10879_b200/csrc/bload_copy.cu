@@ -178,6 +178,286 @@ __global__ void __launch_bounds__(256) k7_copy(PlanView pv, int32_t t_block, int
     }
 }
 
+
+// ------------------------------------------------------------------------------------------------
+// Staged variant for small frames whose size is a multiple of 4 bytes (token ids, short feature
+// vectors): runs are short and start at arbitrary 4-byte offsets, so the register path above keeps too
+// few bytes in flight.  Here every warp owns a ring of shared-memory stages, each the image of one
+// sub-tile of the DENSE side:
+//   pack    gather the runs into the stage with asynchronous copies (cp.async, 16 bytes where source
+//           and stage are mutually aligned, else 4 bytes), pad with shared-memory stores, then write
+//           the finished sub-tile with one bulk copy shared -> global (cp.async.bulk);
+//   unpack  load the valid part of the sub-tile with 16-byte cp.async, then scatter it to the ragged
+//           side with coalesced word (or vector) stores.
+// The loads of item i are in flight while item i-1 is completed, and nothing waits on a flag: the only
+// waits are cp.async.wait_group / cp.async.bulk.wait_group, which end when the hardware copies end.
+// Requires frame_bytes % 4 == 0 and (t_block * frame_bytes) % 16 == 0.
+// Tuning of the two directions (swept on B200 with the 4-byte token workload): bytes per stage, warps
+// per CTA, stages per warp, consecutive sub-tiles of a block handled by one warp.  More, smaller stages
+// mean more resident warps; the kernels are limited by per-warp instruction latency, not by bytes in flight.
+#ifndef BLOAD_PACK_CFG
+#define BLOAD_PACK_CFG 8192, 4, 2, 2
+#endif
+#ifndef BLOAD_UNPACK_CFG
+#define BLOAD_UNPACK_CFG 4096, 8, 2, 4
+#endif
+template <int BYTES, int WARPS, int STAGES, int GROUP>
+struct StageCfgT {
+    static constexpr int kBytes = BYTES, kWarps = WARPS, kStages = STAGES, kGroup = GROUP;
+    static_assert(BYTES % 512 == 0 && STAGES >= 2 && GROUP >= 1, "stage configuration");
+};
+template <bool UNPACK> struct StageCfg : StageCfgT<BLOAD_PACK_CFG> {};
+template <> struct StageCfg<true> : StageCfgT<BLOAD_UNPACK_CFG> {};
+constexpr int64_t kStagedMaxFrameBytes = 256;
+
+__device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void cp_async4(uint32_t s, const void* g)
+{
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(s), "l"(g) : "memory");
+}
+__device__ __forceinline__ void cp_async16(uint32_t s, const void* g)
+{
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(s), "l"(g) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void bulk_store(void* g, uint32_t s, uint32_t bytes)
+{
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(g), "r"(s), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory"); }
+
+// four copies of `sz` bytes, 32 lanes apart, with immediate offsets
+#define BLOAD_CP4X(op, sz, s, g, st)                                                                                \
+    asm volatile(op " [%0], [%1], " #sz ";\n\t" op " [%0+" #st "], [%1+" #st "], " #sz ";\n\t"                       \
+                 op " [%0+2*" #st "], [%1+2*" #st "], " #sz ";\n\t" op " [%0+3*" #st "], [%1+3*" #st "], " #sz ";"   \
+                 ::"r"(s), "l"(g) : "memory")
+
+// asynchronous gather of n bytes (n % 4 == 0, both addresses 4-byte aligned) into shared memory
+__device__ __forceinline__ void warp_gather_async(uint32_t sd, const uint8_t* __restrict__ gs, int n, int lane)
+{
+    if (((sd ^ (uint32_t)reinterpret_cast<uintptr_t>(gs)) & 15u) == 0) {
+        int hw = (int)(((16u - (sd & 15u)) & 15u) >> 2);
+        if (hw * 4 > n) hw = n >> 2;
+        if (lane < hw) cp_async4(sd + 4 * lane, gs + 4 * lane);
+        sd += 4 * hw; gs += 4 * hw; n -= 4 * hw;
+        const int nv = n >> 4;
+        {
+            uint32_t s = sd + 16 * lane;
+            const uint8_t* g = gs + 16 * lane;
+            int rem = nv - lane;  // vectors left for this lane, 32 apart
+            for (; rem > 96; rem -= 128, s += 2048, g += 2048) BLOAD_CP4X("cp.async.cg.shared.global", 16, s, g, 512);
+            for (; rem > 0; rem -= 32, s += 512, g += 512) cp_async16(s, g);
+        }
+        const int tw = (n - (nv << 4)) >> 2;
+        if (lane < tw) cp_async4(sd + (nv << 4) + 4 * lane, gs + (nv << 4) + 4 * lane);
+    } else {
+        uint32_t s = sd + 4 * lane;
+        const uint8_t* g = gs + 4 * lane;
+        int rem = (n >> 2) - lane;  // words left for this lane, 32 apart
+        for (; rem > 96; rem -= 128, s += 512, g += 512) BLOAD_CP4X("cp.async.ca.shared.global", 4, s, g, 128);
+        for (; rem > 0; rem -= 32, s += 128, g += 128) cp_async4(s, g);
+    }
+}
+
+template <int WS>
+__device__ __forceinline__ void scatter_vectors(uint4* __restrict__ d, const uint4* __restrict__ a, int nv, int lane)
+{
+    int i = lane;
+    for (; i + 96 < nv; i += 128) {  // four output vectors in flight per lane
+        uint4 lo[4], hi[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) { lo[u] = a[i + 32 * u]; if (WS) hi[u] = a[i + 32 * u + 1]; }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) st_stream(d + i + 32 * u, WS ? splice<WS>(lo[u], hi[u], 0) : lo[u]);
+    }
+    for (; i < nv; i += 32) st_stream(d + i, WS ? splice<WS>(a[i], a[i + 1], 0) : a[i]);
+}
+
+// scatter of n bytes (n % 4 == 0, 4-byte aligned) from shared memory to global memory, with 16-byte
+// stores on the global side; a misaligned shared-memory source is read as two aligned vectors per
+// output vector (the second may reach up to 12 bytes past the run: the stage area has 16 spare bytes)
+__device__ __forceinline__ void warp_scatter(uint8_t* __restrict__ gd, const uint8_t* __restrict__ ss, int n, int lane)
+{
+    int hw = (int)(((16u - (unsigned)(reinterpret_cast<uintptr_t>(gd) & 15u)) & 15u) >> 2);
+    if (hw * 4 > n) hw = n >> 2;
+    if (lane < hw) reinterpret_cast<uint32_t*>(gd)[lane] = reinterpret_cast<const uint32_t*>(ss)[lane];
+    gd += 4 * hw; ss += 4 * hw; n -= 4 * hw;
+    const int nv = n >> 4;
+    uint4* d = reinterpret_cast<uint4*>(gd);
+    const int ws = (int)((smem_addr(ss) & 15u) >> 2);  // word shift of the source, 0..3
+    const uint4* a = reinterpret_cast<const uint4*>(ss - 4 * ws);
+    switch (ws) {
+        case 0: scatter_vectors<0>(d, a, nv, lane); break;
+        case 1: scatter_vectors<1>(d, a, nv, lane); break;
+        case 2: scatter_vectors<2>(d, a, nv, lane); break;
+        default: scatter_vectors<3>(d, a, nv, lane); break;
+    }
+    const int tw = (n - (nv << 4)) >> 2;
+    if (lane < tw) reinterpret_cast<uint32_t*>(gd + (nv << 4))[lane] = reinterpret_cast<const uint32_t*>(ss + (nv << 4))[lane];
+}
+
+// What a warp has to remember about a sub-tile between its two phases.
+struct StagedItem {
+    int64_t dense_off;  // byte offset of [lo, hi) inside the dense buffer
+    int lo;             // byte offset inside the block (blocks of the staged path are < 2^31 bytes)
+    int nbytes;         // hi - lo
+    int valid;          // bytes of [lo, hi) that hold frames (the rest is padding)
+    bool fresh;         // first sub-tile of its group: the run walker restarts from the fields below
+    int k, k1, fill;    // first overlapping segment, end of the block's segments, occupied slots
+    int w_st;           // lane's entry of the 32-segment window starting at k: start slot ...
+    int64_t w_src;      // ... and first source frame
+};
+struct GroupHeader { int k0, k1, fill; };
+// Position of a warp in the segment list while it walks consecutive sub-tiles of one block.
+struct RunWalker { int k, kw, k1, fill, w_st; int64_t w_src; };
+
+template <bool UNPACK>
+__global__ void __launch_bounds__(StageCfg<UNPACK>::kWarps * 32) k8_staged(PlanView pv, int32_t t_block, int64_t frame_bytes,
+                                                             int64_t block_begin, uint32_t groups,
+                                                             const uint8_t* __restrict__ src_base,
+                                                             uint8_t* __restrict__ dst_base, uint32_t groups_per_block,
+                                                             uint8_t pad)
+{
+    // A group is kStageGroup consecutive sub-tiles of one block, handled by one warp so that the
+    // position in the segment list carries over from one sub-tile to the next.
+    // groups = blocks of this launch * groups_per_block < 2^31 (the launcher splits larger calls).
+    using Cfg = StageCfg<UNPACK>;
+    constexpr int NST = Cfg::kStages, kStageBytes = Cfg::kBytes, kStageWarps = Cfg::kWarps, kStageGroup = Cfg::kGroup;
+    extern __shared__ __align__(128) uint8_t stage_mem[];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    uint8_t* my_stages = stage_mem + (size_t)warp * NST * kStageBytes;
+    const uint32_t warps = gridDim.x * kStageWarps;
+    const int fb = (int)frame_bytes;
+    const int block_bytes = t_block * fb;
+    const int64_t n_blocks = pv.hdr->n_blocks;
+
+    // the three scalars of a group's block; loaded one group ahead so that their latency is hidden
+    auto load_header = [&](uint32_t g) {
+        GroupHeader h{0, 0, 0};
+        const int64_t b = block_begin + g / groups_per_block;
+        if (g < groups && b < n_blocks) {
+            h.k0 = pv.block_seg_begin[b];
+            h.k1 = pv.block_seg_begin[b + 1];
+            h.fill = pv.block_fill[b];
+        }
+        return h;
+    };
+    RunWalker wk{0, 0, 0, 0, 0, 0};
+    // walk the runs of a sub-tile; f(offset inside the sub-tile, byte offset in the ragged buffer, bytes)
+    auto for_each_run = [&](const StagedItem& it, auto&& f) {
+        if (it.fresh) { wk.k = wk.kw = it.k; wk.k1 = it.k1; wk.fill = it.fill; wk.w_st = it.w_st; wk.w_src = it.w_src; }
+        const int hi = it.lo + it.valid;
+        int cur = it.lo;
+        while (cur < hi) {
+            if (wk.k - wk.kw == 31) {
+                wk.kw = wk.k;
+                wk.w_st = (wk.kw + lane < wk.k1) ? pv.seg_start[wk.kw + lane] : wk.fill;
+                wk.w_src = (wk.kw + lane < wk.k1) ? pv.seg_src[wk.kw + lane] : 0;
+            }
+            const int st = __shfl_sync(kFull, wk.w_st, wk.k - wk.kw);
+            const int nx = __shfl_sync(kFull, wk.w_st, wk.k - wk.kw + 1);
+            const int64_t src_frame = __shfl_sync(kFull, wk.w_src, wk.k - wk.kw);
+            const int seg_e = nx * fb;
+            const int pe = min(seg_e, hi);
+            f(cur - it.lo, src_frame * fb + (cur - st * fb), pe - cur);
+            cur = pe;
+            if (pe == seg_e) ++wk.k;  // a run cut by the end of the sub-tile continues in the next one
+        }
+    };
+    // second phase of an item whose loads have landed in `stage`
+    auto complete = [&](const StagedItem& it, uint8_t* stage) {
+        if (!UNPACK) {
+            fence_proxy_async();  // stage was written through the generic proxy, the bulk copy reads it through the async proxy
+            __syncwarp();
+            if (lane == 0) { bulk_store(dst_base + it.dense_off, smem_addr(stage), (uint32_t)it.nbytes); bulk_commit(); }
+        } else {
+            __syncwarp();
+            for_each_run(it, [&](int off, int64_t rag, int n) { warp_scatter(dst_base + rag, stage + off, n, lane); });
+            __syncwarp();  // all lanes are done reading before the stage is refilled
+        }
+    };
+
+    StagedItem prev;
+    bool have_prev = false;
+    int s = 0, s_prev = 0;
+    uint32_t g = blockIdx.x * kStageWarps + warp;
+    GroupHeader h_next = load_header(g);
+    int wn_st = 0;          // prefetched window of the next group (when it starts at the top of a block)
+    int64_t wn_src = 0;
+    bool wn_valid = false;
+    for (; g < groups; g += warps) {
+        const GroupHeader h = h_next;
+        h_next = load_header(g + warps);
+        const uint32_t q = g / groups_per_block;
+        const int first = (int)(g - q * groups_per_block) * kStageGroup;
+        const int fill_bytes = h.fill * fb;
+        int k = h.k0, w_st = wn_st;
+        int64_t w_src = wn_src;
+        if (!wn_valid) {
+            const int lo0 = first * kStageBytes;
+            if (lo0 != 0 && lo0 < fill_bytes) k = warp_find_segment(pv.seg_start, h.k0, h.k1, lo0 / fb, lane);
+            w_st = (k + lane < h.k1) ? pv.seg_start[k + lane] : h.fill;
+            w_src = (k + lane < h.k1) ? pv.seg_src[k + lane] : 0;
+        }
+        wn_valid = false;
+#pragma unroll 1
+        for (int j = 0; j < kStageGroup; ++j) {
+            StagedItem it;
+            it.lo = (first + j) * kStageBytes;
+            if (it.lo >= block_bytes) break;
+            it.nbytes = min(kStageBytes, block_bytes - it.lo);
+            it.dense_off = (int64_t)q * block_bytes + it.lo;
+            it.valid = it.lo < fill_bytes ? min(it.nbytes, fill_bytes - it.lo) : 0;
+            it.fresh = j == 0;
+            it.k = k; it.k1 = h.k1; it.fill = h.fill; it.w_st = w_st; it.w_src = w_src;
+            if ((j == kStageGroup - 1 || it.lo + kStageBytes >= block_bytes) && g + warps < groups &&
+                (g + warps) % groups_per_block == 0) {
+                // the next group opens a block: its window does not need a search, fetch it now
+                wn_st = (h_next.k0 + lane < h_next.k1) ? pv.seg_start[h_next.k0 + lane] : h_next.fill;
+                wn_src = (h_next.k0 + lane < h_next.k1) ? pv.seg_src[h_next.k0 + lane] : 0;
+                wn_valid = true;
+            }
+            uint8_t* stage = my_stages + (size_t)s * kStageBytes;
+            const uint32_t sa = smem_addr(stage);
+            if (!UNPACK) {
+                // the bulk store that last read this stage (NST items ago) must have finished reading it
+                if (lane == 0) bulk_wait_read<NST - 2>();
+                __syncwarp();
+                for_each_run(it, [&](int off, int64_t rag, int n) { warp_gather_async(sa + off, src_base + rag, n, lane); });
+                // padding: words up to the next 16-byte boundary, then vectors (valid % 4 == 0, nbytes % 16 == 0)
+                const uint32_t p4 = 0x01010101u * pad;
+                const int firstv = min((it.valid + 15) & ~15, it.nbytes);
+                if (lane < ((firstv - it.valid) >> 2)) *reinterpret_cast<uint32_t*>(stage + it.valid + 4 * lane) = p4;
+                for (int o = firstv + 16 * lane; o < it.nbytes; o += 512) *reinterpret_cast<uint4*>(stage + o) = make_uint4(p4, p4, p4, p4);
+            } else {
+                // whole vectors of the valid part: the sub-tile is 16-byte aligned and sized
+                uint32_t sp = sa + 16 * lane;
+                const uint8_t* gp = src_base + it.dense_off + 16 * lane;
+                int rem = ((it.valid + 15) >> 4) - lane;
+                for (; rem > 96; rem -= 128, sp += 2048, gp += 2048) BLOAD_CP4X("cp.async.cg.shared.global", 16, sp, gp, 512);
+                for (; rem > 0; rem -= 32, sp += 512, gp += 512) cp_async16(sp, gp);
+            }
+            cp_async_commit();
+            if (have_prev) {
+                cp_async_wait<1>();  // everything but the group just committed has landed
+                complete(prev, my_stages + (size_t)s_prev * kStageBytes);
+            }
+            prev = it; have_prev = true; s_prev = s;
+            s = (s + 1 == NST) ? 0 : s + 1;
+        }
+    }
+    if (have_prev) {
+        cp_async_wait<0>();
+        complete(prev, my_stages + (size_t)s_prev * kStageBytes);
+    }
+    if (!UNPACK && lane == 0) bulk_wait_read<0>();  // shared memory must outlive the reads of the last stores
+}
+
 }  // namespace
 
 cudaError_t launch_copy(bool unpack, const PlanView& pv, int32_t t_block, int64_t frame_bytes, int64_t block_begin,
@@ -186,6 +466,37 @@ cudaError_t launch_copy(bool unpack, const PlanView& pv, int32_t t_block, int64_
 {
     if (block_count == 0) return cudaSuccess;
     const int64_t block_bytes = (int64_t)t_block * frame_bytes;
+    count_launches(1);
+    // small word-granular frames: staged kernel; everything else: register path
+    if (frame_bytes % 4 == 0 && block_bytes % 16 == 0 && frame_bytes <= kStagedMaxFrameBytes) {
+        const int stage_bytes = unpack ? StageCfg<true>::kBytes : StageCfg<false>::kBytes;
+        const int stage_warps = unpack ? StageCfg<true>::kWarps : StageCfg<false>::kWarps;
+        const int nst = unpack ? StageCfg<true>::kStages : StageCfg<false>::kStages;
+        const int group = unpack ? StageCfg<true>::kGroup : StageCfg<false>::kGroup;
+        const int64_t spb = (block_bytes + stage_bytes - 1) / stage_bytes;
+        const int64_t gpb = (spb + group - 1) / group;  // groups of sub-tiles per block
+        const size_t smem = (size_t)stage_warps * nst * stage_bytes + 16;  // 16 spare bytes: see warp_scatter
+        const int per_sm = (int)((227 * 1024) / (smem + 1024));
+        cudaError_t e = unpack ? cudaFuncSetAttribute(k8_staged<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)
+                               : cudaFuncSetAttribute(k8_staged<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        // 32-bit group arithmetic on the device: at most 2^31 - 1 groups per launch
+        const int64_t max_blocks = 0x7fffffffLL / gpb;
+        for (int64_t done = 0; done < block_count; done += max_blocks) {
+            const int64_t cnt = block_count - done < max_blocks ? block_count - done : max_blocks;
+            const int64_t groups = cnt * gpb;
+            const int64_t want = (groups + stage_warps - 1) / stage_warps;
+            const unsigned grid = (unsigned)(want < 148 * per_sm ? want : 148 * per_sm);
+            uint8_t* d = dense + done * block_bytes;
+            if (unpack)
+                k8_staged<true><<<grid, stage_warps * 32, smem, st>>>(pv, t_block, frame_bytes, block_begin + done,
+                                                                     (uint32_t)groups, d, ragged_out, (uint32_t)gpb, pad_byte);
+            else
+                k8_staged<false><<<grid, stage_warps * 32, smem, st>>>(pv, t_block, frame_bytes, block_begin + done,
+                                                                      (uint32_t)groups, ragged_in, d, (uint32_t)gpb, pad_byte);
+        }
+        return cudaPeekAtLastError();
+    }
     const int64_t sub = 16384;
     const int64_t spb = (block_bytes + sub - 1) / sub;
     const int64_t items = block_count * spb;
@@ -197,7 +508,6 @@ cudaError_t launch_copy(bool unpack, const PlanView& pv, int32_t t_block, int64_
     else
         k7_copy<false><<<grid, 256, 0, st>>>(pv, t_block, frame_bytes, block_begin, block_count, ragged_in, dense,
                                               ragged_bytes, sub, spb, pad_byte);
-    count_launches(1);
     return cudaPeekAtLastError();
 }
 

@@ -214,3 +214,23 @@ def test_plan_on_a_side_stream_and_reuse_of_buffers():
         with torch.cuda.stream(s):
             plan = B.bload_plan(d_len, 4096, seed, work=work, plan_buf=plan_buf)
         G.assert_plan_equal(plan, O.plan(T, 4096, seed))
+
+
+@pytest.mark.parametrize("tb,fb,tmax", [(4, 4, 4), (64, 4, 64), (1000, 16, 9), (4096, 4, 4096), (4096, 8, 40),
+                                        (20000, 36, 3000), (20000, 4, 20000), (700, 256, 300), (32768, 12, 5000),
+                                        (5000, 64, 2), (2048, 20, 2048)])
+def test_small_word_sized_frames_take_the_staged_path(tb, fb, tmax):
+    """Frames of 4..256 bytes (multiples of 4) with 16-byte-multiple blocks go through the shared-memory
+    staged kernels: many sub-tiles per block, runs cut by sub-tile ends, more than 32 runs per sub-tile,
+    pad-only sub-tiles, filler blocks, a non-zero pad byte."""
+    assert (tb * fb) % 16 == 0
+    rng = np.random.default_rng(tb * 131 + fb)
+    n = int(min(4000, max(3, 6_000_000 // (tmax * fb))))
+    T = rng.integers(1, tmax + 1, size=n).astype(np.int32)
+    T[rng.integers(0, n)] = tmax
+    plan, op = G.full_parity(T, tb, 5, fb, out_fb=fb, pad=0xA7, extra_blocks=2)
+    # a sub-range in the middle, as a training loop would request batch by batch
+    if op.n_blocks > 3:
+        store = torch.randint(0, 256, (op.sum_t * fb,), dtype=torch.uint8, device=G.DEV)
+        res, _ = G.gpu_pack_all(plan, store, fb, 1, 2, 0, meta=False)
+        assert np.array_equal(res["dense"], O.pack(op, store.cpu().numpy(), fb, 1, 2, 0))
