@@ -193,7 +193,7 @@ int bload_pack(const void* d_plan, const bload_plan_info_t* info, const void* d_
     if (ce == cudaSuccess && d_dense)
         ce = launch_copy(false, pv, info->t_block, frame_bytes, block_begin, block_count,
                          static_cast<const uint8_t*>(d_store), static_cast<uint8_t*>(d_dense), nullptr,
-                         info->sum_t * frame_bytes, pad_byte, st);
+                         info->sum_t * frame_bytes, pad_byte, st, info->n, info->n_blocks);
     if (ce != cudaSuccess) { (void)cudaGetLastError(); return BLOAD_ERR_CUDA; }
     return BLOAD_OK;
 }
@@ -210,7 +210,8 @@ int bload_unpack(const void* d_plan, const bload_plan_info_t* info, const void* 
     PlanView pv = plan_view(const_cast<void*>(d_plan), info->n);
     cudaError_t ce = launch_copy(true, pv, info->t_block, out_frame_bytes, block_begin, block_count, nullptr,
                                  const_cast<uint8_t*>(static_cast<const uint8_t*>(d_dense_out)),
-                                 static_cast<uint8_t*>(d_ragged_out), info->sum_t * out_frame_bytes, 0, st);
+                                 static_cast<uint8_t*>(d_ragged_out), info->sum_t * out_frame_bytes, 0, st, info->n,
+                                 info->n_blocks);
     if (ce != cudaSuccess) { (void)cudaGetLastError(); return BLOAD_ERR_CUDA; }
     return BLOAD_OK;
 }

@@ -458,15 +458,128 @@ __global__ void __launch_bounds__(StageCfg<UNPACK>::kWarps * 32) k8_staged(PlanV
     if (!UNPACK && lane == 0) bulk_wait_read<0>();  // shared memory must outlive the reads of the last stores
 }
 
+
+// ------------------------------------------------------------------------------------------------
+// Whole-plan unpack for small word-sized frames, tiled on the RAGGED side.  When every block of the
+// plan is unpacked, the ragged output is one contiguous buffer that is written completely, so it can
+// be produced exactly like a pack: cut it into sub-tiles, gather each sub-tile's runs (now read from
+// their blocks in the dense buffer, through the inverse tables seq_block / seq_start) into a
+// shared-memory stage with cp.async, and write the stage with one bulk copy.  Every warp owns a
+// contiguous range of sub-tiles: it locates its first sequence once (32-way search of `offsets`)
+// and then only walks forward, 32 sequences per window.
+__device__ __forceinline__ int warp_find_sequence(const int64_t* __restrict__ offsets, int n, int64_t frame, int lane)
+{   // largest i in [0, n) with offsets[i] <= frame (offsets[0] == 0)
+    int lo = 0, hi = n;
+    while (hi - lo > 1) {
+        const int step = (hi - lo + 31) >> 5;
+        const int64_t idx = (int64_t)lo + (int64_t)lane * step;
+        const bool p = idx < hi && offsets[idx] <= frame;
+        const int c = __popc(__ballot_sync(kFull, p));
+        const int nlo = lo + (c - 1) * step;
+        hi = min(hi, nlo + step);
+        lo = nlo;
+    }
+    return lo;
+}
+
+__global__ void __launch_bounds__(StageCfg<false>::kWarps * 32) k9_unpack_ragged(PlanView pv, int32_t n, int32_t t_block,
+                                                                               int64_t frame_bytes, int64_t sum_t,
+                                                                               const uint8_t* __restrict__ dense,
+                                                                               uint8_t* __restrict__ ragged,
+                                                                               int64_t tiles, int64_t tiles_per_warp)
+{
+    using Cfg = StageCfg<false>;
+    constexpr int NST = Cfg::kStages, kStageBytes = Cfg::kBytes, kStageWarps = Cfg::kWarps;
+    extern __shared__ __align__(128) uint8_t stage_mem[];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    uint8_t* my_stages = stage_mem + (size_t)warp * NST * kStageBytes;
+    const int64_t gw = (int64_t)blockIdx.x * kStageWarps + warp;
+    const int64_t t_begin = gw * tiles_per_warp;
+    const int64_t t_end = min(t_begin + tiles_per_warp, tiles);
+    if (t_begin >= t_end) return;
+    const int64_t total = sum_t * frame_bytes;
+
+    // window of 32 sequences from kw: first frame in the ragged order, first frame in the dense buffer
+    int i = warp_find_sequence(pv.offsets, n, (t_begin * kStageBytes) / frame_bytes, lane);
+    int kw = i;
+    int64_t w_off = 0, w_src = 0;
+    auto load_window = [&]() {
+        const int s = kw + lane;
+        w_off = s < n ? pv.offsets[s] : sum_t;  // the entry after the last sequence closes it
+        w_src = s < n ? (int64_t)pv.seq_block[s] * t_block + pv.seq_start[s] : 0;
+    };
+    load_window();
+
+    int64_t prev_lo = 0;
+    int prev_n = 0, s = 0, s_prev = 0;
+    bool have_prev = false;
+    auto complete = [&](int64_t lo, int nbytes, uint8_t* stage) {
+        fence_proxy_async();
+        __syncwarp();
+        const int n16 = nbytes & ~15;
+        if (lane == 0 && n16) { bulk_store(ragged + lo, smem_addr(stage), (uint32_t)n16); bulk_commit(); }
+        if (lane < nbytes - n16) ragged[lo + n16 + lane] = stage[n16 + lane];  // last tile only: total % 16 bytes
+    };
+    for (int64_t t = t_begin; t < t_end; ++t) {
+        uint8_t* stage = my_stages + (size_t)s * kStageBytes;
+        const uint32_t sa = smem_addr(stage);
+        const int64_t lo = t * kStageBytes;
+        const int nbytes = (int)min((int64_t)kStageBytes, total - lo);
+        if (lane == 0) bulk_wait_read<NST - 2>();  // the store that last read this stage has finished reading
+        __syncwarp();
+        int64_t cur = lo;
+        const int64_t hi = lo + nbytes;
+        while (cur < hi) {
+            if (i - kw == 31) { kw = i; load_window(); }
+            const int64_t off = __shfl_sync(kFull, w_off, i - kw);
+            const int64_t nxt = __shfl_sync(kFull, w_off, i - kw + 1);
+            const int64_t src = __shfl_sync(kFull, w_src, i - kw);
+            const int64_t seq_e = nxt * frame_bytes;
+            const int64_t pe = min(seq_e, hi);
+            warp_gather_async(sa + (uint32_t)(cur - lo), dense + src * frame_bytes + (cur - off * frame_bytes), (int)(pe - cur), lane);
+            cur = pe;
+            if (pe == seq_e) ++i;
+        }
+        cp_async_commit();
+        if (have_prev) {
+            cp_async_wait<1>();
+            complete(prev_lo, prev_n, my_stages + (size_t)s_prev * kStageBytes);
+        }
+        prev_lo = lo; prev_n = nbytes; have_prev = true; s_prev = s;
+        s = (s + 1 == NST) ? 0 : s + 1;
+    }
+    cp_async_wait<0>();
+    complete(prev_lo, prev_n, my_stages + (size_t)s_prev * kStageBytes);
+    __syncwarp();
+    if (lane == 0) bulk_wait_read<0>();
+}
+
 }  // namespace
 
 cudaError_t launch_copy(bool unpack, const PlanView& pv, int32_t t_block, int64_t frame_bytes, int64_t block_begin,
                         int64_t block_count, const uint8_t* ragged_in, uint8_t* dense, uint8_t* ragged_out,
-                        int64_t ragged_bytes, uint8_t pad_byte, cudaStream_t st)
+                        int64_t ragged_bytes, uint8_t pad_byte, cudaStream_t st, int64_t n, int64_t n_blocks)
 {
     if (block_count == 0) return cudaSuccess;
     const int64_t block_bytes = (int64_t)t_block * frame_bytes;
     count_launches(1);
+    // whole-plan unpack of small word-sized frames: tile the (contiguous, fully written) ragged side
+    if (unpack && frame_bytes % 4 == 0 && frame_bytes <= kStagedMaxFrameBytes && block_begin == 0 &&
+        block_count >= n_blocks && ragged_bytes > 0) {
+        using Cfg = StageCfg<false>;
+        const size_t smem = (size_t)Cfg::kWarps * Cfg::kStages * Cfg::kBytes + 16;
+        const int per_sm = (int)((227 * 1024) / (smem + 1024));
+        cudaError_t e = cudaFuncSetAttribute(k9_unpack_ragged, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        const int64_t tiles = (ragged_bytes + Cfg::kBytes - 1) / Cfg::kBytes;
+        const int64_t max_warps = (int64_t)148 * per_sm * Cfg::kWarps;
+        const int64_t tpw = (tiles + max_warps - 1) / max_warps;           // contiguous sub-tiles per warp
+        const int64_t warps = (tiles + tpw - 1) / tpw;
+        const unsigned grid = (unsigned)((warps + Cfg::kWarps - 1) / Cfg::kWarps);
+        k9_unpack_ragged<<<grid, Cfg::kWarps * 32, smem, st>>>(pv, (int32_t)n, t_block, frame_bytes, ragged_bytes / frame_bytes,
+                                                              dense, ragged_out, tiles, tpw);
+        return cudaPeekAtLastError();
+    }
     // small word-granular frames: staged kernel; everything else: register path
     if (frame_bytes % 4 == 0 && block_bytes % 16 == 0 && frame_bytes <= kStagedMaxFrameBytes) {
         const int stage_bytes = unpack ? StageCfg<true>::kBytes : StageCfg<false>::kBytes;

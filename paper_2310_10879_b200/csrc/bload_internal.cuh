@@ -75,6 +75,6 @@ cudaError_t launch_metadata(const PlanView& pv, int32_t t_block, int64_t block_b
                             int32_t* seq_id, int32_t* pos, uint8_t* reset, uint8_t* valid, cudaStream_t st);
 cudaError_t launch_copy(bool unpack, const PlanView& pv, int32_t t_block, int64_t frame_bytes, int64_t block_begin,
                         int64_t block_count, const uint8_t* ragged_in, uint8_t* dense, uint8_t* ragged_out,
-                        int64_t ragged_bytes, uint8_t pad_byte, cudaStream_t st);
+                        int64_t ragged_bytes, uint8_t pad_byte, cudaStream_t st, int64_t n, int64_t n_blocks);
 
 }  // namespace bload

@@ -234,3 +234,15 @@ def test_small_word_sized_frames_take_the_staged_path(tb, fb, tmax):
         store = torch.randint(0, 256, (op.sum_t * fb,), dtype=torch.uint8, device=G.DEV)
         res, _ = G.gpu_pack_all(plan, store, fb, 1, 2, 0, meta=False)
         assert np.array_equal(res["dense"], O.pack(op, store.cpu().numpy(), fb, 1, 2, 0))
+
+
+@pytest.mark.parametrize("tb,fb,lengths", [(6, 4, [2, 2, 3, 3, 4, 5, 6, 6]), (7, 12, [1]), (9, 20, [9, 1, 1]),
+                                           (5, 4, [1, 1, 1]), (3000, 4, None), (1234, 36, None)])
+def test_whole_plan_unpack_of_word_sized_frames(tb, fb, lengths):
+    """Unpacking every block of a plan with small word-sized frames takes the ragged-side tiled kernel:
+    totals that are not multiples of 16 bytes, totals below one vector, block sizes that are not
+    multiples of 16 bytes, many warps with one sub-tile each."""
+    rng = np.random.default_rng(tb + fb)
+    T = np.array(lengths, np.int32) if lengths else rng.integers(1, tb + 1, size=5000).astype(np.int32)
+    G.full_parity(T, tb, 3, fb, out_fb=fb, pad=0x11, extra_blocks=0)
+    G.full_parity(T, tb, 4, fb, out_fb=fb, pad=0, extra_blocks=3)
