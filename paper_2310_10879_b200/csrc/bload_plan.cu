@@ -298,7 +298,8 @@ __global__ void __launch_bounds__(256, 1) k4_fill(PlanView pv, const int32_t* __
     extern __shared__ __align__(16) int32_t sm[];
     int32_t* Q0 = sm;              // [32]
     int32_t* Q1 = sm + 32;         // [32][32]
-    int32_t* Q2 = sm + 32 + 1024;  // [rows][32], rows = ceil(L / 32)
+    int32_t* Q2 = sm + 32 + 1024 + 128;  // [rows][32], rows = ceil(L / 32)
+    int4* ring = reinterpret_cast<int4*>(sm + 32 + 1024);  // [32] records of the last draws
     if (pv.hdr->first_bad != kNoBad) return;
     const int rows = (L + 31) >> 5;
     auto upto = [&](int l) { return bucket_end[min(l, L)]; };  // sequences with length <= l
@@ -348,16 +349,21 @@ __global__ void __launch_bounds__(256, 1) k4_fill(PlanView pv, const int32_t* __
         if (lane >= a) { --q0; Q0[lane] = q0; }
         if (lane >= bb) Q1[(a << 5) + lane] = q1 - 1;
         if (lane >= c) Q2[(row << 5) + lane] = q2 - 1;
+        // the draw's record goes to a 32-entry ring in shared memory and leaves 32 at a time, one per lane:
+        // a global store inside the chain costs about 55 cycles per draw
         int below = __shfl_up_sync(kFull, q2, 1);
         if (lane == 0) below = 0;
-        if (lane == c) draw_rec[k] = make_int4(len, q2 - below, b, start);  // q2 - below: unused of this length
+        if (lane == c) ring[k & 31] = make_int4(len, q2 - below, b, start);  // q2 - below: unused of this length
         __syncwarp();
         room -= len; start += len; ++k;
         if ((k & 31) == 0) {
+            draw_rec[k - 32 + lane] = ring[lane];
             u_cur = u_nxt;
             u_nxt = k + 32 + lane < n ? draw_u[k + 32 + lane] : 0;
+            __syncwarp();
         }
     }
+    if (lane < (n & 31)) draw_rec[(n & ~31) + lane] = ring[lane];
     if (lane == 0) {
         pv.block_fill[b] = start;
         pv.block_seg_begin[b + 1] = k;
@@ -473,7 +479,7 @@ cudaError_t launch_plan(const int32_t* d_lengths, int64_t n, int32_t t_block, ui
     k3_buckets<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(kin, n, t_block, wv.bucket_end, pv.hdr);
     if (ev) cudaEventRecord(ev[2], st);
 
-    const size_t smem = sizeof(int32_t) * (32 + 1024 + (size_t)((t_block + 31) / 32) * 32);
+    const size_t smem = sizeof(int32_t) * (32 + 1024 + 128 + (size_t)((t_block + 31) / 32) * 32);
     cudaError_t e = cudaFuncSetAttribute(k4_fill, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     k4_fill<<<1, 256, smem, st>>>(pv, wv.bucket_end, wv.draw_u, wv.draw_rec, n, t_block);
