@@ -294,6 +294,51 @@ def run_gpu(args, w) -> dict:
     step_s = seconds / args.steps
     value = aggregate(by["pack"] + by["unpack"], world, step_s) / 1e9
 
+    # ---- batch-by-batch use: one pack call (metadata + dense) per training batch of w.batch_blocks blocks,
+    # the last batch rounded up with filler blocks; the output buffers of one batch are reused
+    bb = w.batch_blocks
+    n_batches = (nb + bb - 1) // bb
+    per_batch = None
+    if n_batches * bb * tb * fb <= dense.numel() + bb * tb * fb:
+        b_dense = torch.empty(bb * tb * fb, dtype=torch.uint8, device=dev)
+        b_meta = [torch.empty(bb * tb, dtype=d, device=dev) for d in (torch.int32, torch.int32, torch.uint8, torch.uint8)]
+        reps = max(1, min(n_batches, 4000))
+
+        def batch_loop():
+            for i in range(reps):
+                B.bload_pack(plan, store, fb, i * bb, bb, dense=b_dense, seq_id=b_meta[0], pos=b_meta[1],
+                             reset=b_meta[2], valid=b_meta[3])
+        batch_loop()
+        torch.cuda.synchronize()
+        a, b_ = ev(), ev()
+        a.record(); batch_loop(); b_.record()
+        torch.cuda.synchronize()
+        ms = a.elapsed_time(b_)
+        per_batch = {"batch_blocks": bb, "batches_timed": reps, "us_per_call": ms * 1e3 / reps,
+                     "GB/s": (2 * bb * tb * fb) * reps / ms / 1e6, "launches_per_call": 2}
+        # the same loop captured once in a CUDA graph and replayed (the calls are asynchronous and allocate nothing)
+        try:
+            side = torch.cuda.Stream()
+            side.wait_stream(torch.cuda.current_stream())
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.stream(side):
+                with torch.cuda.graph(graph, stream=side):
+                    batch_loop()
+            torch.cuda.current_stream().wait_stream(side)
+            graph.replay()
+            torch.cuda.synchronize()
+            a, b_ = ev(), ev()
+            a.record(); graph.replay(); b_.record()
+            torch.cuda.synchronize()
+            gms = a.elapsed_time(b_)
+            per_batch["graph_us_per_call"] = gms * 1e3 / reps
+            per_batch["graph_GB/s"] = (2 * bb * tb * fb) * reps / gms / 1e6
+            del graph
+        except Exception as exc:  # capture is an optimisation of the measurement, not part of the path
+            per_batch["graph_us_per_call"] = None
+            per_batch["graph_error"] = str(exc)[:200]
+        del b_dense, b_meta
+
     # ---- end to end through the same calls with HOST buffers (pinned), copies inside the timed region
     e2e = None
     if not args.no_e2e:
@@ -350,7 +395,7 @@ def run_gpu(args, w) -> dict:
            "ms_per_step": step_s * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
            "dtype": "u8", "data": "synthetic", "config": config_of(w, {"parallelism": "replicas only"}),
            "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline,
-           "frames_per_s": aggregate(sum_t, world, step_s),
+           "frames_per_s": aggregate(sum_t, world, step_s), "per_batch_pack": per_batch,
            "kernels": {
                "pack_copy": {"ms": pack_ms, "GB/s": by["pack"] / pack_ms / 1e6, "frac_measured": by["pack"] / pack_ms / 1e6 / peak,
                              "frac_nominal": by["pack"] / pack_ms / 1e6 / NOMINAL_HBM_GBS, "frames_per_s": sum_t / pack_ms * 1e3},
