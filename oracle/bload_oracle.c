@@ -116,7 +116,8 @@ typedef struct {
     int64_t n;
     int32_t t_block;
     uint64_t seed;
-    uint32_t policy; /* 0 = uniform over the unused sequences that fit */
+    uint32_t policy; /* 0 = uniform over the unused sequences that fit; 1 = uniform over the LENGTHS (keys of
+                        L_dict) that fit and still have an unused sequence */
     /* outputs, all caller-allocated */
     int64_t *offsets;         /* [n+1] */
     int32_t *seg_seq;         /* [n]   sequence placed by the k-th draw */
@@ -158,7 +159,7 @@ int oracle_plan(oracle_plan_t *p)
     p->n_blocks = 0; p->sum_t = 0; p->t_max = 0; p->first_bad = -1;
     p->checksum = 0; p->max_segs_per_block = 0;
     if (n < 1 || n > 0x7fffffffLL || tb < 1) return ORACLE_ERR_ARG;
-    if (p->policy != 0) return ORACLE_ERR_POLICY;
+    if (p->policy > 1) return ORACLE_ERR_POLICY;
 
     /* Precondition of the method: 1 <= T_i <= block length. */
     for (int64_t i = 0; i < n; ++i) {
@@ -189,15 +190,26 @@ int oracle_plan(oracle_plan_t *p)
         int32_t remaining = tb, start = 0;
         p->block_seg_begin[b] = (int32_t)k;
         for (;;) {
-            /* m: unused sequences that still fit */
-            int64_t m = 0;
-            for (int32_t l = 1; l <= remaining; ++l) m += unused[l];
-            if (m == 0) break;
-            /* Random_*(): the j-th of them, counted in order of length */
-            uint64_t j = oracle_pick(oracle_draw_word(p->seed, k), (uint64_t)m);
             int32_t l = 1;
-            int64_t run = unused[1];
-            while ((uint64_t)run <= j) { l += 1; run += unused[l]; }
+            if (p->policy == 0) {
+                /* m: unused sequences that still fit */
+                int64_t m = 0;
+                for (int32_t q = 1; q <= remaining; ++q) m += unused[q];
+                if (m == 0) break;
+                /* Random_*(): the j-th of them, counted in order of length */
+                uint64_t j = oracle_pick(oracle_draw_word(p->seed, k), (uint64_t)m);
+                int64_t run = unused[1];
+                while ((uint64_t)run <= j) { l += 1; run += unused[l]; }
+            } else {
+                /* m: keys of L_dict (lengths) that fit and are not exhausted */
+                int64_t m = 0;
+                for (int32_t q = 1; q <= remaining; ++q) m += unused[q] > 0;
+                if (m == 0) break;
+                /* Random_*(): the j-th such key in increasing order, then an entry of its list */
+                uint64_t j = oracle_pick(oracle_draw_word(p->seed, k), (uint64_t)m);
+                int64_t run = unused[1] > 0;
+                while ((uint64_t)run <= j) { l += 1; run += unused[l] > 0; }
+            }
             /* first unused entry of L_dict[l] */
             int64_t taken = (first[l + 1] - first[l]) - unused[l];
             int32_t id = dict[first[l] + taken].id;

@@ -11,8 +11,10 @@ from functools import lru_cache
 from itertools import combinations
 
 
-def outcome_distribution(lengths, t_block):
-    """dict: outcome -> exact probability; outcome = tuple of blocks, block = tuple of lengths."""
+def outcome_distribution(lengths, t_block, policy=0):
+    """dict: outcome -> exact probability; outcome = tuple of blocks, block = tuple of lengths.
+    policy 0: every unused sequence that fits is equally likely (P(length l) = count[l] / m);
+    policy 1: every LENGTH that fits and is not exhausted is equally likely (P = 1 / #such lengths)."""
     start = tuple(sorted(lengths))
 
     @lru_cache(maxsize=None)
@@ -28,7 +30,7 @@ def outcome_distribution(lengths, t_block):
             return out
         m = len(fit)
         for l in sorted(set(fit)):
-            pl = Fraction(fit.count(l), m)
+            pl = Fraction(fit.count(l), m) if policy == 0 else Fraction(1, len(set(fit)))
             rest = list(left)
             rest.remove(l)
             for tail, p in rec(tuple(rest), room - l).items():

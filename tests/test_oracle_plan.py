@@ -207,6 +207,7 @@ def test_bad_inputs_are_rejected():
     assert O.plan(np.array([1], np.int32), 0, 0).status != 0
     assert O.plan(np.array([], np.int32), 4, 0).status != 0
     assert O.plan(np.array([1], np.int32), 4, 0, policy=7).status != 0
+    assert O.plan(np.array([1], np.int32), 4, 0, policy=1).status == 0
 
 
 def test_checker_rejects_planted_mistakes():
@@ -238,3 +239,65 @@ def test_checker_rejects_planted_mistakes():
     sst = np.empty_like(p.seq_start); sst[p.seg_seq] = st
     if fill.max() <= p.t_block:
         broken(block_seg_begin=bsb, seg_block=sb, seg_start=st, block_fill=fill, seq_block=sblk, seq_start=sst)
+
+
+# ---- policy 1: the other reading of "a random entry of L_dict": a random KEY (length) that fits ----
+
+@pytest.mark.parametrize("lengths,t_block", [
+    ([2, 2, 2, 2, 3, 6, 6, 6], 6),
+    ([1, 1, 1, 1, 1, 4, 5], 5),
+    ([4, 3, 3, 3, 2, 1, 1, 1], 7),
+])
+def test_policy1_outcome_frequencies_match_uniform_over_lengths(lengths, t_block):
+    T = np.array(lengths, np.int32)
+    dist = brute.outcome_distribution(lengths, t_block, policy=1)
+    other = brute.outcome_distribution(lengths, t_block, policy=0)
+    tv = 0.5 * sum(abs(float(dist.get(k, 0)) - float(other.get(k, 0))) for k in set(dist) | set(other))
+    assert tv > 0.05                                     # the two readings really differ on this input
+    n_seeds = 10000
+    seen = {}
+    for seed in range(n_seeds):
+        p = O.plan(T, t_block, seed, policy=1)
+        _check(p)
+        k = brute.outcome_of_plan(T, p.n_blocks, p.seg_seq, p.block_seg_begin)
+        assert k in dist, k
+        seen[k] = seen.get(k, 0) + 1
+    keys = sorted(dist, key=lambda k: -dist[k])
+    exp = np.array([float(dist[k]) * n_seeds for k in keys])
+    obs = np.array([seen.get(k, 0) for k in keys], dtype=float)
+    big = exp >= 5
+    e = np.append(exp[big], exp[~big].sum()) if (~big).any() else exp
+    o = np.append(obs[big], obs[~big].sum()) if (~big).any() else obs
+    keep = e > 0
+    stat = float(((o[keep] - e[keep]) ** 2 / e[keep]).sum())
+    assert stat < chi2.ppf(0.9999, keep.sum() - 1), (stat, keep.sum())
+
+
+def test_policy1_first_draw_is_uniform_over_lengths_not_sequences():
+    T = np.array([1] * 9 + [2], np.int32)        # nine sequences of length 1, one of length 2
+    hits = sum(int(T[O.plan(T, 4, seed, policy=1).seg_seq[0]] == 2) for seed in range(4000))
+    assert 1800 < hits < 2200                     # 1/2 under policy 1 (it would be 1/10 under policy 0)
+    hits0 = sum(int(T[O.plan(T, 4, seed, policy=0).seg_seq[0]] == 2) for seed in range(4000))
+    assert 300 < hits0 < 500
+
+
+@pytest.mark.parametrize("name", ["toy_video", "features_fp16", "heavy_tail_bf16", "video_dataset_shape"])
+def test_policy1_invariants_on_workloads(name):
+    w = W.WORKLOADS[name]
+    T = W.lengths(w)
+    p = O.plan(T, w.t_block, seed=w.seed, policy=1)
+    _check(p)
+    q = O.plan(T, w.t_block, seed=w.seed, policy=0)
+    assert not np.array_equal(p.seg_seq, q.seg_seq)
+
+
+def test_policy1_random_small_cases_stay_in_reachable_set():
+    rng = np.random.default_rng(12)
+    for _ in range(40):
+        n = int(rng.integers(1, 8)); tb = int(rng.integers(1, 10))
+        T = rng.integers(1, tb + 1, size=n).astype(np.int32)
+        dist = brute.outcome_distribution([int(x) for x in T], tb, policy=1)
+        for seed in range(15):
+            p = O.plan(T, tb, seed, policy=1)
+            _check(p)
+            assert brute.outcome_of_plan(T, p.n_blocks, p.seg_seq, p.block_seg_begin) in dist
