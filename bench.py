@@ -28,6 +28,7 @@ if ROOT not in sys.path:
 METRIC = "pack+unpack GB/s (algorithmic bytes of the pack and unpack copies / time of the whole step)"
 UNIT = "GB/s"
 NOMINAL_HBM_GBS = 8000.0
+POLICY = 0  # fill policy of this run (set from --policy)
 FALLBACK_HBM_GBS = 6650.0
 
 
@@ -145,7 +146,7 @@ class CpuOracleSample:
 
     def plan(self):
         t0 = time.perf_counter()
-        self.op = self.O.plan(self.T, self.w.t_block, self.w.seed)
+        self.op = self.O.plan(self.T, self.w.t_block, self.w.seed, POLICY)
         self.t_plan = time.perf_counter() - t0
         return self.op
 
@@ -200,7 +201,8 @@ def config_of(w, extra) -> dict:
     c = {"workload": "configs[%d] %s: N=%d, lengths %s, frame %d B (%s), T_block=%d, unpack of %d B/frame outputs; "
                      "one whole-epoch call per direction" % (w.index, w.name, w.n, w.dist, w.frame_bytes, w.payload,
                                                              w.t_block, w.out_frame_bytes),
-         "batch_blocks": w.batch_blocks, "l2": "inputs larger than L2 (no flush needed)", "seed": w.seed}
+         "batch_blocks": w.batch_blocks, "l2": "inputs larger than L2 (no flush needed)", "seed": w.seed,
+         "policy": POLICY}
     if extra:
         c.update(extra)
     return c
@@ -231,7 +233,7 @@ def run_gpu(args, w) -> dict:
     sizes = B.bload_plan_sizes(T.size, tb)
     plan_buf = torch.empty(sizes.plan_bytes, dtype=torch.uint8, device=dev)
     work = torch.empty(sizes.work_bytes, dtype=torch.uint8, device=dev)
-    plan = B.bload_plan(d_len, tb, w.seed, work=work, plan_buf=plan_buf)
+    plan = B.bload_plan(d_len, tb, w.seed, policy=args.policy, work=work, plan_buf=plan_buf)
     nb, sum_t = plan.n_blocks, plan.sum_t
     by = algorithmic_bytes(sum_t, nb, tb, fb, ofb)
 
@@ -250,7 +252,7 @@ def run_gpu(args, w) -> dict:
     def step(rec=None):
         e = [ev() for _ in range(5)] if rec is not None else None
         if e: e[0].record()
-        p = B.bload_plan(d_len, tb, w.seed, work=work, plan_buf=plan_buf)
+        p = B.bload_plan(d_len, tb, w.seed, policy=args.policy, work=work, plan_buf=plan_buf)
         if e: e[1].record()
         B.bload_pack(p, None, fb, 0, nb, seq_id=seq_id, pos=pos, reset=reset, valid=valid)
         if e: e[2].record()
@@ -354,7 +356,7 @@ def run_gpu(args, w) -> dict:
         def e2e_step():
             d_len.copy_(h_len, non_blocking=True)
             store.copy_(h_store, non_blocking=True)
-            p = B.bload_plan(d_len, tb, w.seed, work=work, plan_buf=plan_buf)
+            p = B.bload_plan(d_len, tb, w.seed, policy=args.policy, work=work, plan_buf=plan_buf)
             B.bload_pack(p, store, fb, 0, nb, dense=dense, seq_id=seq_id, pos=pos, reset=reset, valid=valid)
             h_dense.copy_(dense, non_blocking=True)
             for h, d in zip(h_meta, (seq_id, pos, reset, valid)):
@@ -436,6 +438,7 @@ def main():
     ap.add_argument("--impl", default="bload", choices=["bload", "reference"])
     ap.add_argument("--workload", default="heavy_tail_bf16")
     ap.add_argument("--n", type=int, default=0, help="override the number of sequences (small profiling cases)")
+    ap.add_argument("--policy", type=int, default=0, help="fill policy: 0 uniform over sequences, 1 uniform over lengths")
     ap.add_argument("--frame-bytes", type=int, default=0, help="override the frame size of the workload (experiments)")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--ref-blocks", type=int, default=0,
@@ -446,6 +449,8 @@ def main():
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "bload" else args.warmup
 
+    global POLICY
+    POLICY = args.policy
     from paper_2310_10879_b200 import workloads as W
     w = W.WORKLOADS[args.workload]
     if args.n:

@@ -50,6 +50,8 @@ extern "C" {
 
 #define BLOAD_MAX_T_BLOCK 32768
 #define BLOAD_POLICY_UNIFORM_SEQUENCES 0u /* every unused sequence that fits is equally likely */
+#define BLOAD_POLICY_UNIFORM_LENGTHS 1u   /* every length (key of L_dict) that fits and is not exhausted is equally
+                                             likely, then the next unused sequence of that length; needs n < 2^26 */
 
 /* Sizes and table offsets for a problem of n sequences (host only, no GPU call). */
 typedef struct {

@@ -136,7 +136,8 @@ int bload_plan(const int32_t* d_lengths, int64_t n, int32_t t_block, uint64_t se
     if (!d_lengths || !d_plan || !d_work) return fail(BLOAD_ERR_NULL);
     int rc = check_sizes(n, t_block);
     if (rc) return fail(rc);
-    if (policy != BLOAD_POLICY_UNIFORM_SEQUENCES) return fail(BLOAD_ERR_UNSUPPORTED);
+    if (policy > BLOAD_POLICY_UNIFORM_LENGTHS) return fail(BLOAD_ERR_UNSUPPORTED);
+    if (policy == BLOAD_POLICY_UNIFORM_LENGTHS && n >= (1LL << 26)) return fail(BLOAD_ERR_UNSUPPORTED);
     bload_sizes_t sz;
     plan_layout(n, &sz);
     WorkView wv;

@@ -371,6 +371,109 @@ __global__ void __launch_bounds__(256, 1) k4_fill(PlanView pv, const int32_t* __
     }
 }
 
+// Policy 1: every LENGTH that fits and still has an unused sequence is equally likely (the other reading
+// of "a random entry of L_dict": a random key of the dictionary).  Same three-level table, but it counts
+// non-exhausted lengths instead of sequences, and a leaf word packs two fields:
+//   bits 0..5   inclusive count of non-exhausted lengths in its row up to this leaf (0..32)
+//   bits 6..31  unused sequences of this length (hence n < 2^26 for this policy)
+// Most draws change only the chosen leaf's count; the prefix fields move when a length runs out.
+__global__ void __launch_bounds__(256, 1) k4_fill_lengths(PlanView pv, const int32_t* __restrict__ bucket_end,
+                                                          const uint64_t* __restrict__ draw_u,
+                                                          int4* __restrict__ draw_rec, int64_t n64, int32_t L)
+{
+    extern __shared__ __align__(16) int32_t sm[];
+    int32_t* Q0 = sm;
+    int32_t* Q1 = sm + 32;
+    int4* ring = reinterpret_cast<int4*>(sm + 32 + 1024);
+    int32_t* Q2 = sm + 32 + 1024 + 128;
+    if (pv.hdr->first_bad != kNoBad) return;
+    const int rows = (L + 31) >> 5;
+    auto upto = [&](int l) { return bucket_end[min(l, L)]; };
+    // leaves: one thread per row, 32 leaves in order
+    for (int r = threadIdx.x; r < rows; r += blockDim.x) {
+        int live = 0;
+        for (int c = 0; c < 32; ++c) {
+            const int x = (r << 5) + c;
+            const int cnt = x < L ? upto(x + 1) - upto(x) : 0;
+            live += cnt > 0;
+            Q2[x] = (int32_t)(((uint32_t)cnt << 6) | (uint32_t)live);
+        }
+    }
+    __syncthreads();
+    // rows of a top group: one thread per group
+    if (threadIdx.x < 32) {
+        int run = 0;
+        for (int b = 0; b < 32; ++b) {
+            const int r = (threadIdx.x << 5) + b;
+            run += r < rows ? (Q2[(r << 5) + 31] & 63) : 0;
+            Q1[(threadIdx.x << 5) + b] = run;
+        }
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int run = 0;
+        for (int a = 0; a < 32; ++a) { run += Q1[(a << 5) + 31]; Q0[a] = run; }
+    }
+    __syncthreads();
+    if (threadIdx.x >= 32) return;
+
+    const int lane = threadIdx.x;
+    const int n = (int)n64;
+    int q0 = Q0[lane];
+    int k = 0, b = 0, room = L, start = 0;
+    if (lane == 0) pv.block_seg_begin[0] = 0;
+    uint64_t u_cur = lane < n ? draw_u[lane] : 0;
+    uint64_t u_nxt = 32 + lane < n ? draw_u[32 + lane] : 0;
+    while (k < n) {
+        const uint64_t u = __shfl_sync(kFull, u_cur, k & 31);
+        int m = 0;  // lengths that fit and are not exhausted
+        if (room > 0) {
+            const int y = room - 1, ya = y >> 10, yb = (y >> 5) & 31;
+            m = (Q2[y] & 63) + (yb ? Q1[(ya << 5) + yb - 1] : 0) + (ya ? Q0[ya - 1] : 0);
+        }
+        if (m == 0) {
+            if (lane == 0) { pv.block_fill[b] = start; pv.block_seg_begin[b + 1] = k; }
+            ++b; room = L; start = 0;
+            continue;
+        }
+        int j = (int)(((uint64_t)(uint32_t)(u >> 32) * (uint32_t)m + __umulhi((uint32_t)u, (uint32_t)m)) >> 32);
+        const int a = __popc(__ballot_sync(kFull, q0 <= j));
+        const int q1 = Q1[(a << 5) + lane];
+        int base = __shfl_sync(kFull, q0, (a - 1) & 31);
+        j -= a ? base : 0;
+        const int bb = __popc(__ballot_sync(kFull, q1 <= j));
+        const int row = (a << 5) + bb;
+        const int q2 = Q2[(row << 5) + lane];
+        base = __shfl_sync(kFull, q1, (bb - 1) & 31);
+        j -= bb ? base : 0;
+        const int c = __popc(__ballot_sync(kFull, (q2 & 63) <= j));
+        const int len = (row << 5) + c + 1;
+        const int cnt = (int)((uint32_t)__shfl_sync(kFull, q2, c) >> 6);  // unused sequences of the chosen length, >= 1
+        if (cnt == 1) {  // the length runs out: it leaves the prefix counts of all three levels
+            if (lane >= a) { --q0; Q0[lane] = q0; }
+            if (lane >= bb) Q1[(a << 5) + lane] = q1 - 1;
+            if (lane >= c) Q2[(row << 5) + lane] = (lane == c ? q2 - 64 : q2) - 1;
+        } else if (lane == c) {
+            Q2[(row << 5) + lane] = q2 - 64;
+        }
+        if (lane == c) ring[k & 31] = make_int4(len, cnt, b, start);
+        __syncwarp();
+        room -= len; start += len; ++k;
+        if ((k & 31) == 0) {
+            draw_rec[k - 32 + lane] = ring[lane];
+            u_cur = u_nxt;
+            u_nxt = k + 32 + lane < n ? draw_u[k + 32 + lane] : 0;
+            __syncwarp();
+        }
+    }
+    if (lane < (n & 31)) draw_rec[(n & ~31) + lane] = ring[lane];
+    if (lane == 0) {
+        pv.block_fill[b] = start;
+        pv.block_seg_begin[b + 1] = k;
+        pv.hdr->n_blocks = b + 1;
+    }
+}
+
 __device__ __forceinline__ uint64_t fmix64(uint64_t x)
 {  // 64-bit finaliser of MurmurHash3
     x ^= x >> 33; x *= 0xff51afd7ed558ccdULL;
@@ -480,9 +583,10 @@ cudaError_t launch_plan(const int32_t* d_lengths, int64_t n, int32_t t_block, ui
     if (ev) cudaEventRecord(ev[2], st);
 
     const size_t smem = sizeof(int32_t) * (32 + 1024 + 128 + (size_t)((t_block + 31) / 32) * 32);
-    cudaError_t e = cudaFuncSetAttribute(k4_fill, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    auto fill = policy == BLOAD_POLICY_UNIFORM_LENGTHS ? k4_fill_lengths : k4_fill;
+    cudaError_t e = cudaFuncSetAttribute(fill, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    k4_fill<<<1, 256, smem, st>>>(pv, wv.bucket_end, wv.draw_u, wv.draw_rec, n, t_block);
+    fill<<<1, 256, smem, st>>>(pv, wv.bucket_end, wv.draw_u, wv.draw_rec, n, t_block);
     if (ev) cudaEventRecord(ev[3], st);
 
     k5_tables<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(pv, wv.draw_rec, wv.bucket_end, iin, n);

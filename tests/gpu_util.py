@@ -11,9 +11,9 @@ DEV = "cuda:0"
 GUARD = 4096  # canary bytes on both sides of every output
 
 
-def gpu_plan(lengths: np.ndarray, t_block: int, seed: int, check=True):
+def gpu_plan(lengths: np.ndarray, t_block: int, seed: int, check=True, policy=0):
     d_len = torch.from_numpy(np.ascontiguousarray(lengths, dtype=np.int32)).to(DEV)
-    return B.bload_plan(d_len, t_block, seed, check=check)
+    return B.bload_plan(d_len, t_block, seed, policy=policy, check=check)
 
 
 def host_tables(plan) -> dict:
@@ -91,10 +91,10 @@ def first_diff(a: np.ndarray, b: np.ndarray):
 
 
 def full_parity(lengths: np.ndarray, t_block: int, seed: int, fb: int, out_fb: int | None = None, pad: int = 0,
-                extra_blocks: int = 2, payload_seed: int = 5):
+                extra_blocks: int = 2, payload_seed: int = 5, policy: int = 0):
     """plan + metadata + pack + unpack of ALL blocks (plus filler blocks) against the oracle."""
-    op = O.plan(lengths, t_block, seed)
-    plan = gpu_plan(lengths, t_block, seed)
+    op = O.plan(lengths, t_block, seed, policy)
+    plan = gpu_plan(lengths, t_block, seed, policy=policy)
     assert_plan_equal(plan, op)
     g = torch.Generator(device=DEV); g.manual_seed(payload_seed)
     store = torch.randint(0, 256, (op.sum_t * fb,), dtype=torch.uint8, device=DEV, generator=g)

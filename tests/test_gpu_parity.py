@@ -177,6 +177,7 @@ def test_host_detected_errors_launch_nothing():
     assert call(lengths=None) == e.ERR_NULL and call(plan=None) == e.ERR_NULL and call(wk=None) == e.ERR_NULL
     assert call(n=0) == e.ERR_ARG and call(tb=0) == e.ERR_ARG
     assert call(tb=e.MAX_T_BLOCK + 1) == e.ERR_UNSUPPORTED and call(policy=3) == e.ERR_UNSUPPORTED
+    assert call(policy=1) == 0
     assert call(pb=sz.plan_bytes - 1) == e.ERR_WORKSPACE and call(wb=sz.work_bytes - 1) == e.ERR_WORKSPACE
     assert call(plan=plan_buf.data_ptr() + 8) == e.ERR_ALIGN and call(wk=work.data_ptr() + 16) == e.ERR_ALIGN
     assert call() == 0
@@ -246,3 +247,30 @@ def test_whole_plan_unpack_of_word_sized_frames(tb, fb, lengths):
     T = np.array(lengths, np.int32) if lengths else rng.integers(1, tb + 1, size=5000).astype(np.int32)
     G.full_parity(T, tb, 3, fb, out_fb=fb, pad=0x11, extra_blocks=0)
     G.full_parity(T, tb, 4, fb, out_fb=fb, pad=0, extra_blocks=3)
+
+
+# ---- policy 1: uniform over the lengths that fit ----
+
+@pytest.mark.parametrize("name,n", [("toy_video", None), ("features_fp16", None), ("tokens", 30000),
+                                    ("heavy_tail_bf16", 20000), ("video_dataset_shape", None)])
+def test_policy1_plans_match_the_oracle(name, n):
+    w = W.WORKLOADS[name]
+    if n:
+        w = W.scaled(w, n)
+    T = W.lengths(w)
+    for seed in (w.seed, 7):
+        G.assert_plan_equal(G.gpu_plan(T, w.t_block, seed, policy=1), O.plan(T, w.t_block, seed, policy=1))
+
+
+def test_policy1_small_and_degenerate_cases():
+    rng = np.random.default_rng(3)
+    G.full_parity(W.TOY8_LENGTHS, W.TOY8_T_BLOCK, 2, 8, policy=1)
+    for T, tb in [(np.array([5], np.int32), 9), (np.full(300, 17, np.int32), 17), (np.ones(5000, np.int32), 33),
+                  (np.ones(70, np.int32), 1), (rng.integers(1, 4, size=9000).astype(np.int32), 4096),
+                  (np.concatenate([rng.integers(1, 32769, size=40), [32768, 32768, 1, 1, 1024, 1025]]).astype(np.int32), 32768),
+                  (rng.choice([3, 700], size=4097).astype(np.int32), 1000)]:
+        for seed in (0, 11):
+            G.assert_plan_equal(G.gpu_plan(T, tb, seed, policy=1), O.plan(T, tb, seed, policy=1))
+    for n in (1, 31, 32, 33, 2049, 70001):
+        T = rng.integers(1, 301, size=n).astype(np.int32)
+        G.assert_plan_equal(G.gpu_plan(T, 300, 5, policy=1), O.plan(T, 300, 5, policy=1))
