@@ -353,17 +353,33 @@ def run_gpu(args, w) -> dict:
         h2d = h_len.numel() * 4 + h_store.numel() + h_dense_out.numel()
         d2h = h_dense.numel() + sum(x.numel() * x.element_size() for x in h_meta) + h_ragged_out.numel()
 
+        s_in, s_out = torch.cuda.Stream(), torch.cuda.Stream()
+
         def e2e_step():
+            # three streams: host->device copies, the library's kernels, device->host copies.  The plan needs
+            # only the lengths, so it runs while the store is still arriving; the dense batches leave while
+            # the per-frame outputs arrive (PCIe is full duplex).
+            cur = torch.cuda.current_stream()
+            s_in.wait_stream(cur); s_out.wait_stream(cur)
             d_len.copy_(h_len, non_blocking=True)
-            store.copy_(h_store, non_blocking=True)
+            with torch.cuda.stream(s_in):
+                store.copy_(h_store, non_blocking=True)
+                ev_store = s_in.record_event()
+                dense_out.copy_(h_dense_out, non_blocking=True)
+                ev_outputs = s_in.record_event()
             p = B.bload_plan(d_len, tb, w.seed, policy=args.policy, work=work, plan_buf=plan_buf)
+            cur.wait_event(ev_store)
             B.bload_pack(p, store, fb, 0, nb, dense=dense, seq_id=seq_id, pos=pos, reset=reset, valid=valid)
-            h_dense.copy_(dense, non_blocking=True)
-            for h, d in zip(h_meta, (seq_id, pos, reset, valid)):
-                h.copy_(d, non_blocking=True)
-            dense_out.copy_(h_dense_out, non_blocking=True)
+            ev_packed = cur.record_event()
+            with torch.cuda.stream(s_out):
+                s_out.wait_event(ev_packed)
+                h_dense.copy_(dense, non_blocking=True)
+                for h, d in zip(h_meta, (seq_id, pos, reset, valid)):
+                    h.copy_(d, non_blocking=True)
+            cur.wait_event(ev_outputs)
             B.bload_unpack(p, dense_out, ofb, 0, nb, ragged_out)
             h_ragged_out.copy_(ragged_out, non_blocking=True)
+            cur.wait_stream(s_out)
             return B.bload_stats(p.info)
 
         e2e_step()
