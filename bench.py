@@ -407,7 +407,9 @@ def run_gpu(args, w) -> dict:
     achieved = d_bytes / (d_ms / 1e3) / 1e9
     roofline = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "GB/s",
                 "frac": achieved / peak, "peak_kind": "of " + peak_kind, "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
-                "traffic": TRAFFIC.get((w.name, dom)) if not (args.n or args.frame_bytes) else None, "launch_ms": d_ms, "algorithmic_bytes_per_launch": d_bytes}
+                "traffic": TRAFFIC.get((w.name, dom)) if not (args.n or args.frame_bytes) else None,
+                "note": "largest HBM-bound kernel of the step; the planner's fill rule (k4_fill, %.2f ms) is a latency-bound "
+                        "chain of dependent draws on one warp and is reported in kernels.plan as time and draws/s" % stage[2], "launch_ms": d_ms, "algorithmic_bytes_per_launch": d_bytes}
 
     out = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
            "ms_per_step": step_s * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,

@@ -58,6 +58,15 @@ def load() -> C.CDLL:
     global _lib
     if _lib is not None:
         return _lib
+    if "BLOAD_LIBRARY" not in os.environ:
+        # a missing or stale in-tree library is (re)built from the CUDA sources; if that is impossible, fail loudly
+        try:
+            from . import build as _build
+            _build.build()
+        except Exception as exc:
+            if not os.path.exists(LIB_PATH):
+                raise RuntimeError("libbload.so is missing at %s and could not be built (%s): there is no CPU "
+                                   "fallback" % (LIB_PATH, exc)) from exc
     if not os.path.exists(LIB_PATH):
         raise RuntimeError("libbload.so is missing at %s: build it with `python -m paper_2310_10879_b200.build` "
                            "(there is no CPU fallback)" % LIB_PATH)
