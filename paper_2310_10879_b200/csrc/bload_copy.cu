@@ -180,18 +180,19 @@ __global__ void __launch_bounds__(256) k7_copy(PlanView pv, int32_t t_block, int
 
 
 // ------------------------------------------------------------------------------------------------
-// Staged variant for small frames whose size is a multiple of 4 bytes (token ids, short feature
+// Staged kernels for small frames whose size is a multiple of 4 bytes (token ids, short feature
 // vectors): runs are short and start at arbitrary 4-byte offsets, so the register path above keeps too
-// few bytes in flight.  Here every warp owns a ring of shared-memory stages, each the image of one
-// sub-tile of the DENSE side:
-//   pack    gather the runs into the stage with asynchronous copies (cp.async, 16 bytes where source
-//           and stage are mutually aligned, else 4 bytes), pad with shared-memory stores, then write
-//           the finished sub-tile with one bulk copy shared -> global (cp.async.bulk);
-//   unpack  load the valid part of the sub-tile with 16-byte cp.async, then scatter it to the ragged
-//           side with coalesced word (or vector) stores.
+// few bytes in flight.  Here every warp owns a small ring of shared-memory stages, each the image of
+// one aligned sub-tile:
+//   k10_pack_contig    sub-tiles of the dense side: gather the runs into the stage with cp.async (16
+//                      bytes where source and stage are mutually aligned, else 4 bytes), pad with
+//                      shared-memory stores, write the sub-tile with one bulk copy (cp.async.bulk);
+//   k9_unpack_ragged   whole-plan unpack, sub-tiles of the ragged side: same gather, from the blocks;
+//   k8_unpack_staged   unpack of a block sub-range, sub-tiles of the dense side: load the valid part
+//                      with 16-byte cp.async, scatter it to the ragged side with 16-byte stores.
 // The loads of item i are in flight while item i-1 is completed, and nothing waits on a flag: the only
 // waits are cp.async.wait_group / cp.async.bulk.wait_group, which end when the hardware copies end.
-// Requires frame_bytes % 4 == 0 and (t_block * frame_bytes) % 16 == 0.
+// Requires frame_bytes % 4 == 0 (and, on the dense side, (t_block * frame_bytes) % 16 == 0).
 // Tuning of the two directions (swept on B200 with the 4-byte token workload): bytes per stage, warps
 // per CTA, stages per warp, consecutive sub-tiles of a block handled by one warp.  More, smaller stages
 // mean more resident warps; the kernels are limited by per-warp instruction latency, not by bytes in flight.
@@ -209,6 +210,10 @@ struct StageCfgT {
 template <bool UNPACK> struct StageCfg : StageCfgT<BLOAD_PACK_CFG> {};
 template <> struct StageCfg<true> : StageCfgT<BLOAD_UNPACK_CFG> {};
 constexpr int64_t kStagedMaxFrameBytes = 256;
+#ifndef BLOAD_PACK_CHUNK_TILES
+#define BLOAD_PACK_CHUNK_TILES 4
+#endif
+constexpr int64_t kPackChunkTiles = BLOAD_PACK_CHUNK_TILES;  // consecutive sub-tiles a warp packs before it jumps ahead
 
 __device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 __device__ __forceinline__ void cp_async4(uint32_t s, const void* g)
@@ -316,8 +321,7 @@ struct GroupHeader { int k0, k1, fill; };
 // Position of a warp in the segment list while it walks consecutive sub-tiles of one block.
 struct RunWalker { int k, kw, k1, fill, w_st; int64_t w_src; };
 
-template <bool UNPACK>
-__global__ void __launch_bounds__(StageCfg<UNPACK>::kWarps * 32) k8_staged(PlanView pv, int32_t t_block, int64_t frame_bytes,
+__global__ void __launch_bounds__(StageCfg<true>::kWarps * 32) k8_unpack_staged(PlanView pv, int32_t t_block, int64_t frame_bytes,
                                                              int64_t block_begin, uint32_t groups,
                                                              const uint8_t* __restrict__ src_base,
                                                              uint8_t* __restrict__ dst_base, uint32_t groups_per_block,
@@ -326,7 +330,7 @@ __global__ void __launch_bounds__(StageCfg<UNPACK>::kWarps * 32) k8_staged(PlanV
     // A group is kStageGroup consecutive sub-tiles of one block, handled by one warp so that the
     // position in the segment list carries over from one sub-tile to the next.
     // groups = blocks of this launch * groups_per_block < 2^31 (the launcher splits larger calls).
-    using Cfg = StageCfg<UNPACK>;
+    using Cfg = StageCfg<true>;
     constexpr int NST = Cfg::kStages, kStageBytes = Cfg::kBytes, kStageWarps = Cfg::kWarps, kStageGroup = Cfg::kGroup;
     extern __shared__ __align__(128) uint8_t stage_mem[];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -371,15 +375,9 @@ __global__ void __launch_bounds__(StageCfg<UNPACK>::kWarps * 32) k8_staged(PlanV
     };
     // second phase of an item whose loads have landed in `stage`
     auto complete = [&](const StagedItem& it, uint8_t* stage) {
-        if (!UNPACK) {
-            fence_proxy_async();  // stage was written through the generic proxy, the bulk copy reads it through the async proxy
-            __syncwarp();
-            if (lane == 0) { bulk_store(dst_base + it.dense_off, smem_addr(stage), (uint32_t)it.nbytes); bulk_commit(); }
-        } else {
-            __syncwarp();
-            for_each_run(it, [&](int off, int64_t rag, int n) { warp_scatter(dst_base + rag, stage + off, n, lane); });
-            __syncwarp();  // all lanes are done reading before the stage is refilled
-        }
+        __syncwarp();
+        for_each_run(it, [&](int off, int64_t rag, int n) { warp_scatter(dst_base + rag, stage + off, n, lane); });
+        __syncwarp();  // all lanes are done reading before the stage is refilled
     };
 
     StagedItem prev;
@@ -424,17 +422,7 @@ __global__ void __launch_bounds__(StageCfg<UNPACK>::kWarps * 32) k8_staged(PlanV
             }
             uint8_t* stage = my_stages + (size_t)s * kStageBytes;
             const uint32_t sa = smem_addr(stage);
-            if (!UNPACK) {
-                // the bulk store that last read this stage (NST items ago) must have finished reading it
-                if (lane == 0) bulk_wait_read<NST - 2>();
-                __syncwarp();
-                for_each_run(it, [&](int off, int64_t rag, int n) { warp_gather_async(sa + off, src_base + rag, n, lane); });
-                // padding: words up to the next 16-byte boundary, then vectors (valid % 4 == 0, nbytes % 16 == 0)
-                const uint32_t p4 = 0x01010101u * pad;
-                const int firstv = min((it.valid + 15) & ~15, it.nbytes);
-                if (lane < ((firstv - it.valid) >> 2)) *reinterpret_cast<uint32_t*>(stage + it.valid + 4 * lane) = p4;
-                for (int o = firstv + 16 * lane; o < it.nbytes; o += 512) *reinterpret_cast<uint4*>(stage + o) = make_uint4(p4, p4, p4, p4);
-            } else {
+            {
                 // whole vectors of the valid part: the sub-tile is 16-byte aligned and sized
                 uint32_t sp = sa + 16 * lane;
                 const uint8_t* gp = src_base + it.dense_off + 16 * lane;
@@ -455,7 +443,6 @@ __global__ void __launch_bounds__(StageCfg<UNPACK>::kWarps * 32) k8_staged(PlanV
         cp_async_wait<0>();
         complete(prev, my_stages + (size_t)s_prev * kStageBytes);
     }
-    if (!UNPACK && lane == 0) bulk_wait_read<0>();  // shared memory must outlive the reads of the last stores
 }
 
 
@@ -554,6 +541,106 @@ __global__ void __launch_bounds__(StageCfg<false>::kWarps * 32) k9_unpack_ragged
     if (lane == 0) bulk_wait_read<0>();
 }
 
+// ------------------------------------------------------------------------------------------------
+// Pack for small word-sized frames with a contiguous range of dense sub-tiles per warp (the pack-side
+// twin of k9_unpack_ragged): the warp locates its first segment once and then walks forward through
+// the segment list, which runs on from one block to the next; only `fill` and the segment end of each
+// new block are read, one block ahead.  Blocks at or beyond n_blocks are written as padding.
+__global__ void __launch_bounds__(StageCfg<false>::kWarps * 32) k10_pack_contig(PlanView pv, int32_t n, int32_t t_block,
+                                                                              int64_t frame_bytes, int64_t block_begin,
+                                                                              const uint8_t* __restrict__ store,
+                                                                              uint8_t* __restrict__ dense, int64_t tiles,
+                                                                              int64_t tiles_per_warp, int32_t subs_per_block,
+                                                                              uint8_t pad)
+{
+    using Cfg = StageCfg<false>;
+    constexpr int NST = Cfg::kStages, kStageBytes = Cfg::kBytes, kStageWarps = Cfg::kWarps;
+    extern __shared__ __align__(128) uint8_t stage_mem[];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    uint8_t* my_stages = stage_mem + (size_t)warp * NST * kStageBytes;
+    const int64_t gw = (int64_t)blockIdx.x * kStageWarps + warp;
+    const int64_t n_warps = (int64_t)gridDim.x * kStageWarps;
+    const int fb = (int)frame_bytes;
+    const int block_bytes = t_block * fb;
+    const int64_t n_blocks = pv.hdr->n_blocks;
+    auto seg_end_of = [&](int64_t b) { return b < n_blocks ? pv.block_seg_begin[b + 1] : 0; };
+    auto fill_of = [&](int64_t b) { return b < n_blocks ? pv.block_fill[b] * fb : 0; };
+    int64_t prev_off = 0;
+    int prev_n = 0, s = 0, s_prev = 0;
+    bool have_prev = false;
+    auto complete = [&](int64_t off, int nbytes, uint8_t* stage) {
+        fence_proxy_async();
+        __syncwarp();
+        if (lane == 0) { bulk_store(dense + off, smem_addr(stage), (uint32_t)nbytes); bulk_commit(); }
+    };
+    const uint32_t p4 = 0x01010101u * pad;
+    // the warp takes chunks of `tiles_per_warp` consecutive sub-tiles, chunk after chunk, grid-strided
+    for (int64_t t_begin = gw * tiles_per_warp; t_begin < tiles; t_begin += n_warps * tiles_per_warp) {
+    const int64_t t_end = min(t_begin + tiles_per_warp, tiles);
+    int64_t q = t_begin / subs_per_block;            // block of this call the warp is in
+    int sub = (int)(t_begin - q * subs_per_block);   // sub-tile inside it
+    // current block: end of its segments and occupied bytes; the same two scalars of the next block
+    int k1 = seg_end_of(block_begin + q), fill_bytes = fill_of(block_begin + q);
+    int k1_next = seg_end_of(block_begin + q + 1), fill_next = fill_of(block_begin + q + 1);
+    // position in the segment list and a window of 32 segments from kw (raw start slots, source frames)
+    int k = (block_begin + q) < n_blocks ? pv.block_seg_begin[block_begin + q] : 0;
+    if (sub != 0 && sub * kStageBytes < fill_bytes)
+        k = warp_find_segment(pv.seg_start, k, k1, (sub * kStageBytes) / fb, lane);
+    int kw = k, w_st = 0;
+    int64_t w_src = 0;
+    auto load_window = [&]() {
+        const int si = kw + lane;
+        w_st = si < n ? pv.seg_start[si] : 0;
+        w_src = si < n ? pv.seg_src[si] : 0;
+    };
+    load_window();
+    for (int64_t t = t_begin; t < t_end; ++t) {
+        uint8_t* stage = my_stages + (size_t)s * kStageBytes;
+        const uint32_t sa = smem_addr(stage);
+        const int lo = sub * kStageBytes;
+        const int nbytes = min(kStageBytes, block_bytes - lo);
+        const int valid = lo < fill_bytes ? min(nbytes, fill_bytes - lo) : 0;
+        if (lane == 0) bulk_wait_read<NST - 2>();  // the store that last read this stage has finished reading
+        __syncwarp();
+        int cur = lo;
+        const int hi = lo + valid;
+        while (cur < hi) {
+            if ((unsigned)(k - kw) >= 31u) { kw = k; load_window(); }
+            const int st = __shfl_sync(kFull, w_st, k - kw);
+            int nx = __shfl_sync(kFull, w_st, k - kw + 1);
+            const int64_t src = __shfl_sync(kFull, w_src, k - kw);
+            const int seg_e = (k + 1 < k1) ? nx * fb : fill_bytes;  // the block's last run ends where its frames end
+            const int pe = min(seg_e, hi);
+            warp_gather_async(sa + (uint32_t)(cur - lo), store + src * fb + (cur - st * fb), pe - cur, lane);
+            cur = pe;
+            if (pe == seg_e) ++k;
+        }
+        // padding: words up to the next 16-byte boundary, then vectors (valid % 4 == 0, nbytes % 16 == 0)
+        const int firstv = min((valid + 15) & ~15, nbytes);
+        if (lane < ((firstv - valid) >> 2)) *reinterpret_cast<uint32_t*>(stage + valid + 4 * lane) = p4;
+        for (int o = firstv + 16 * lane; o < nbytes; o += 512) *reinterpret_cast<uint4*>(stage + o) = make_uint4(p4, p4, p4, p4);
+        cp_async_commit();
+        if (have_prev) {
+            cp_async_wait<1>();
+            complete(prev_off, prev_n, my_stages + (size_t)s_prev * kStageBytes);
+        }
+        prev_off = q * (int64_t)block_bytes + lo; prev_n = nbytes; have_prev = true; s_prev = s;
+        s = (s + 1 == NST) ? 0 : s + 1;
+        if (++sub == subs_per_block) {  // next block: its segments follow directly in the list
+            sub = 0; ++q;
+            k = k1;  // (already there unless the warp started inside the padding of the block it leaves)
+            k1 = k1_next; fill_bytes = fill_next;
+            k1_next = seg_end_of(block_begin + q + 1); fill_next = fill_of(block_begin + q + 1);
+        }
+    }
+    }
+    if (!have_prev) return;
+    cp_async_wait<0>();
+    complete(prev_off, prev_n, my_stages + (size_t)s_prev * kStageBytes);
+    __syncwarp();
+    if (lane == 0) bulk_wait_read<0>();
+}
+
 }  // namespace
 
 cudaError_t launch_copy(bool unpack, const PlanView& pv, int32_t t_block, int64_t frame_bytes, int64_t block_begin,
@@ -563,6 +650,25 @@ cudaError_t launch_copy(bool unpack, const PlanView& pv, int32_t t_block, int64_
     if (block_count == 0) return cudaSuccess;
     const int64_t block_bytes = (int64_t)t_block * frame_bytes;
     count_launches(1);
+    // pack of small word-sized frames: contiguous ranges of dense sub-tiles per warp
+    if (!unpack && frame_bytes % 4 == 0 && block_bytes % 16 == 0 && frame_bytes <= kStagedMaxFrameBytes) {
+        using Cfg = StageCfg<false>;
+        const size_t smem = (size_t)Cfg::kWarps * Cfg::kStages * Cfg::kBytes + 16;
+        const int per_sm = (int)((227 * 1024) / (smem + 1024));
+        cudaError_t e = cudaFuncSetAttribute(k10_pack_contig, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        const int64_t spb = (block_bytes + Cfg::kBytes - 1) / Cfg::kBytes;
+        const int64_t tiles = block_count * spb;
+        const int64_t max_warps = (int64_t)148 * per_sm * Cfg::kWarps;
+        int64_t tpw = (tiles + max_warps - 1) / max_warps;
+        if (tpw > kPackChunkTiles) tpw = kPackChunkTiles;  // chunks are grid-strided beyond this size
+        int64_t warps = (tiles + tpw - 1) / tpw;
+        if (warps > max_warps) warps = max_warps;
+        const unsigned grid = (unsigned)((warps + Cfg::kWarps - 1) / Cfg::kWarps);
+        k10_pack_contig<<<grid, Cfg::kWarps * 32, smem, st>>>(pv, (int32_t)n, t_block, frame_bytes, block_begin, ragged_in,
+                                                             dense, tiles, tpw, (int32_t)spb, pad_byte);
+        return cudaPeekAtLastError();
+    }
     // whole-plan unpack of small word-sized frames: tile the (contiguous, fully written) ragged side
     if (unpack && frame_bytes % 4 == 0 && frame_bytes <= kStagedMaxFrameBytes && block_begin == 0 &&
         block_count >= n_blocks && ragged_bytes > 0) {
@@ -580,33 +686,24 @@ cudaError_t launch_copy(bool unpack, const PlanView& pv, int32_t t_block, int64_
                                                               dense, ragged_out, tiles, tpw);
         return cudaPeekAtLastError();
     }
-    // small word-granular frames: staged kernel; everything else: register path
-    if (frame_bytes % 4 == 0 && block_bytes % 16 == 0 && frame_bytes <= kStagedMaxFrameBytes) {
-        const int stage_bytes = unpack ? StageCfg<true>::kBytes : StageCfg<false>::kBytes;
-        const int stage_warps = unpack ? StageCfg<true>::kWarps : StageCfg<false>::kWarps;
-        const int nst = unpack ? StageCfg<true>::kStages : StageCfg<false>::kStages;
-        const int group = unpack ? StageCfg<true>::kGroup : StageCfg<false>::kGroup;
-        const int64_t spb = (block_bytes + stage_bytes - 1) / stage_bytes;
-        const int64_t gpb = (spb + group - 1) / group;  // groups of sub-tiles per block
-        const size_t smem = (size_t)stage_warps * nst * stage_bytes + 16;  // 16 spare bytes: see warp_scatter
+    // block sub-ranges of small word-sized frames, unpack direction: staged kernel over the dense side
+    if (unpack && frame_bytes % 4 == 0 && block_bytes % 16 == 0 && frame_bytes <= kStagedMaxFrameBytes) {
+        using Cfg = StageCfg<true>;
+        const int64_t spb = (block_bytes + Cfg::kBytes - 1) / Cfg::kBytes;
+        const int64_t gpb = (spb + Cfg::kGroup - 1) / Cfg::kGroup;  // groups of sub-tiles per block
+        const size_t smem = (size_t)Cfg::kWarps * Cfg::kStages * Cfg::kBytes + 16;  // 16 spare bytes: see warp_scatter
         const int per_sm = (int)((227 * 1024) / (smem + 1024));
-        cudaError_t e = unpack ? cudaFuncSetAttribute(k8_staged<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)
-                               : cudaFuncSetAttribute(k8_staged<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        cudaError_t e = cudaFuncSetAttribute(k8_unpack_staged, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
         // 32-bit group arithmetic on the device: at most 2^31 - 1 groups per launch
         const int64_t max_blocks = 0x7fffffffLL / gpb;
         for (int64_t done = 0; done < block_count; done += max_blocks) {
             const int64_t cnt = block_count - done < max_blocks ? block_count - done : max_blocks;
             const int64_t groups = cnt * gpb;
-            const int64_t want = (groups + stage_warps - 1) / stage_warps;
+            const int64_t want = (groups + Cfg::kWarps - 1) / Cfg::kWarps;
             const unsigned grid = (unsigned)(want < 148 * per_sm ? want : 148 * per_sm);
-            uint8_t* d = dense + done * block_bytes;
-            if (unpack)
-                k8_staged<true><<<grid, stage_warps * 32, smem, st>>>(pv, t_block, frame_bytes, block_begin + done,
-                                                                     (uint32_t)groups, d, ragged_out, (uint32_t)gpb, pad_byte);
-            else
-                k8_staged<false><<<grid, stage_warps * 32, smem, st>>>(pv, t_block, frame_bytes, block_begin + done,
-                                                                      (uint32_t)groups, ragged_in, d, (uint32_t)gpb, pad_byte);
+            k8_unpack_staged<<<grid, Cfg::kWarps * 32, smem, st>>>(pv, t_block, frame_bytes, block_begin + done, (uint32_t)groups,
+                                                                 dense + done * block_bytes, ragged_out, (uint32_t)gpb, pad_byte);
         }
         return cudaPeekAtLastError();
     }
