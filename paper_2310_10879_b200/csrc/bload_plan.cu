@@ -283,35 +283,45 @@ __global__ void __launch_bounds__(256) k3_buckets(const uint64_t* __restrict__ k
 }
 
 // ---- the fill rule: one warp, n dependent draws ----
-// Shared memory holds running counts of UNUSED sequences as a three-level, 32-ary table of inclusive
-// prefix sums over the lengths (leaf x stands for length x + 1; x = a*1024 + b*32 + c):
-//   Q0[a]          sequences with x < (a+1)*1024                         (32 entries, also one per lane)
-//   Q1[a][b]       sequences with a*1024 <= x < a*1024 + (b+1)*32         (32 x 32)
-//   Q2[a*32+b][c]  sequences with (a*32+b)*32 <= x <= (a*32+b)*32 + c     (one row of 32 per 32 lengths)
+// Shared memory holds running counts of UNUSED sequences as a three-level, 32-ary table of prefix sums
+// over the lengths (leaf x stands for length x + 1; x = a*1024 + b*32 + c).  Every row has 33 entries:
+// entry 0 is zero and entry i+1 is the inclusive sum up to digit i, so that the same row serves as
+// inclusive prefix (read at digit+1) and exclusive prefix (read at digit) without a select or a shuffle,
+// and rows of 33 words fall on distinct banks:
+//   Q0[a+1]            sequences with x < (a+1)*1024
+//   Q1[a][b+1]         sequences with a*1024 <= x < a*1024 + (b+1)*32
+//   Q2[a*32+b][c+1]    sequences with (a*32+b)*32 <= x <= (a*32+b)*32 + c
 // "How many fit in r slots" is three reads; "the j-th of them in order of length" is one
 // compare + ballot + popcount per level with one entry per lane; a draw then decrements the entries
 // at and after the chosen digit in one row per level.
+constexpr int kQ1Off = 36, kRingOff = kQ1Off + 32 * 33, kQ2Off = kRingOff + 128;  // in 32-bit words; ring 16-byte aligned
+static_assert(kRingOff % 4 == 0, "ring alignment");
+
 __global__ void __launch_bounds__(256, 1) k4_fill(PlanView pv, const int32_t* __restrict__ bucket_end,
                                                   const uint64_t* __restrict__ draw_u, int4* __restrict__ draw_rec,
                                                   int64_t n64, int32_t L)
 {
     extern __shared__ __align__(16) int32_t sm[];
-    int32_t* Q0 = sm;              // [32]
-    int32_t* Q1 = sm + 32;         // [32][32]
-    int32_t* Q2 = sm + 32 + 1024 + 128;  // [rows][32], rows = ceil(L / 32)
-    int4* ring = reinterpret_cast<int4*>(sm + 32 + 1024);  // [32] records of the last draws
+    int32_t* Q0 = sm;                                      // [33]
+    int32_t* Q1 = sm + kQ1Off;                             // [32][33]
+    int4* ring = reinterpret_cast<int4*>(sm + kRingOff);   // [32] records of the last draws
+    int32_t* Q2 = sm + kQ2Off;                             // [rows][33], rows = ceil(L / 32)
     if (pv.hdr->first_bad != kNoBad) return;
     const int rows = (L + 31) >> 5;
     auto upto = [&](int l) { return bucket_end[min(l, L)]; };  // sequences with length <= l
-    for (int idx = threadIdx.x; idx < rows * 32; idx += blockDim.x) Q2[idx] = upto(idx + 1) - upto(idx & ~31);
-    for (int idx = threadIdx.x; idx < 1024; idx += blockDim.x) Q1[idx] = upto((idx + 1) << 5) - upto((idx >> 5) << 10);
-    if (threadIdx.x < 32) Q0[threadIdx.x] = upto((threadIdx.x + 1) << 10);
+    for (int idx = threadIdx.x; idx < rows * 32; idx += blockDim.x)
+        Q2[(idx >> 5) * 33 + (idx & 31) + 1] = upto(idx + 1) - upto(idx & ~31);
+    for (int r = threadIdx.x; r < rows; r += blockDim.x) Q2[r * 33] = 0;
+    for (int idx = threadIdx.x; idx < 1024; idx += blockDim.x)
+        Q1[(idx >> 5) * 33 + (idx & 31) + 1] = upto((idx + 1) << 5) - upto((idx >> 5) << 10);
+    if (threadIdx.x < 32) { Q1[threadIdx.x * 33] = 0; Q0[threadIdx.x + 1] = upto((threadIdx.x + 1) << 10); }
+    if (threadIdx.x == 0) Q0[0] = 0;
     __syncthreads();
     if (threadIdx.x >= 32) return;
 
     const int lane = threadIdx.x;
     const int n = (int)n64;
-    int q0 = Q0[lane];
+    int q0 = Q0[lane + 1];
     int k = 0, b = 0, room = L, start = 0;
     if (lane == 0) pv.block_seg_begin[0] = 0;
     // random words of 32 draws at a time, one per lane, the next 32 prefetched
@@ -319,11 +329,8 @@ __global__ void __launch_bounds__(256, 1) k4_fill(PlanView pv, const int32_t* __
     uint64_t u_nxt = 32 + lane < n ? draw_u[32 + lane] : 0;
     while (k < n) {
         const uint64_t u = __shfl_sync(kFull, u_cur, k & 31);
-        int m = 0;
-        if (room > 0) {
-            const int y = room - 1, ya = y >> 10, yb = (y >> 5) & 31;
-            m = Q2[y] + (yb ? Q1[(ya << 5) + yb - 1] : 0) + (ya ? Q0[ya - 1] : 0);
-        }
+        const int y = room - 1, ya = y >> 10, yr = y >> 5;
+        const int m = room > 0 ? Q2[yr * 33 + (y & 31) + 1] + Q1[ya * 33 + (yr & 31)] + Q0[ya] : 0;
         if (m == 0) {  // nothing fits: the rest of the block is padding
             if (lane == 0) { pv.block_fill[b] = start; pv.block_seg_begin[b + 1] = k; }
             ++b; room = L; start = 0;
@@ -333,26 +340,23 @@ __global__ void __launch_bounds__(256, 1) k4_fill(PlanView pv, const int32_t* __
         int j = (int)(((uint64_t)(uint32_t)(u >> 32) * (uint32_t)m + __umulhi((uint32_t)u, (uint32_t)m)) >> 32);
         // level 0
         const int a = __popc(__ballot_sync(kFull, q0 <= j));
-        const int q1 = Q1[(a << 5) + lane];
-        int base = __shfl_sync(kFull, q0, (a - 1) & 31);
-        j -= a ? base : 0;
+        const int q1 = Q1[a * 33 + lane + 1];
+        j -= Q0[a];
         // level 1
         const int bb = __popc(__ballot_sync(kFull, q1 <= j));
         const int row = (a << 5) + bb;
-        const int q2 = Q2[(row << 5) + lane];
-        base = __shfl_sync(kFull, q1, (bb - 1) & 31);
-        j -= bb ? base : 0;
+        const int q2 = Q2[row * 33 + lane + 1];
+        const int below = Q2[row * 33 + lane];
+        j -= Q1[a * 33 + bb];
         // level 2
         const int c = __popc(__ballot_sync(kFull, q2 <= j));
         const int len = (row << 5) + c + 1;
         // decrement the running counts at and after the chosen digits
-        if (lane >= a) { --q0; Q0[lane] = q0; }
-        if (lane >= bb) Q1[(a << 5) + lane] = q1 - 1;
-        if (lane >= c) Q2[(row << 5) + lane] = q2 - 1;
+        if (lane >= a) { --q0; Q0[lane + 1] = q0; }
+        if (lane >= bb) Q1[a * 33 + lane + 1] = q1 - 1;
+        if (lane >= c) Q2[row * 33 + lane + 1] = q2 - 1;
         // the draw's record goes to a 32-entry ring in shared memory and leaves 32 at a time, one per lane:
         // a global store inside the chain costs about 55 cycles per draw
-        int below = __shfl_up_sync(kFull, q2, 1);
-        if (lane == 0) below = 0;
         if (lane == c) ring[k & 31] = make_int4(len, q2 - below, b, start);  // q2 - below: unused of this length
         __syncwarp();
         room -= len; start += len; ++k;
@@ -382,10 +386,10 @@ __global__ void __launch_bounds__(256, 1) k4_fill_lengths(PlanView pv, const int
                                                           int4* __restrict__ draw_rec, int64_t n64, int32_t L)
 {
     extern __shared__ __align__(16) int32_t sm[];
-    int32_t* Q0 = sm;
-    int32_t* Q1 = sm + 32;
-    int4* ring = reinterpret_cast<int4*>(sm + 32 + 1024);
-    int32_t* Q2 = sm + 32 + 1024 + 128;
+    int32_t* Q0 = sm;                                      // [33], entry 0 is zero (see k4_fill)
+    int32_t* Q1 = sm + kQ1Off;                             // [32][33]
+    int4* ring = reinterpret_cast<int4*>(sm + kRingOff);
+    int32_t* Q2 = sm + kQ2Off;                             // [rows][32] packed leaf words (rows are not shifted)
     if (pv.hdr->first_bad != kNoBad) return;
     const int rows = (L + 31) >> 5;
     auto upto = [&](int l) { return bucket_end[min(l, L)]; };
@@ -406,31 +410,31 @@ __global__ void __launch_bounds__(256, 1) k4_fill_lengths(PlanView pv, const int
         for (int b = 0; b < 32; ++b) {
             const int r = (threadIdx.x << 5) + b;
             run += r < rows ? (Q2[(r << 5) + 31] & 63) : 0;
-            Q1[(threadIdx.x << 5) + b] = run;
+            Q1[threadIdx.x * 33 + b + 1] = run;
         }
+        Q1[threadIdx.x * 33] = 0;
     }
     __syncthreads();
     if (threadIdx.x == 0) {
         int run = 0;
-        for (int a = 0; a < 32; ++a) { run += Q1[(a << 5) + 31]; Q0[a] = run; }
+        Q0[0] = 0;
+        for (int a = 0; a < 32; ++a) { run += Q1[a * 33 + 32]; Q0[a + 1] = run; }
     }
     __syncthreads();
     if (threadIdx.x >= 32) return;
 
     const int lane = threadIdx.x;
     const int n = (int)n64;
-    int q0 = Q0[lane];
+    int q0 = Q0[lane + 1];
     int k = 0, b = 0, room = L, start = 0;
     if (lane == 0) pv.block_seg_begin[0] = 0;
     uint64_t u_cur = lane < n ? draw_u[lane] : 0;
     uint64_t u_nxt = 32 + lane < n ? draw_u[32 + lane] : 0;
     while (k < n) {
         const uint64_t u = __shfl_sync(kFull, u_cur, k & 31);
-        int m = 0;  // lengths that fit and are not exhausted
-        if (room > 0) {
-            const int y = room - 1, ya = y >> 10, yb = (y >> 5) & 31;
-            m = (Q2[y] & 63) + (yb ? Q1[(ya << 5) + yb - 1] : 0) + (ya ? Q0[ya - 1] : 0);
-        }
+        const int y = room - 1, ya = y >> 10;
+        // lengths that fit and are not exhausted
+        const int m = room > 0 ? (Q2[y] & 63) + Q1[ya * 33 + ((y >> 5) & 31)] + Q0[ya] : 0;
         if (m == 0) {
             if (lane == 0) { pv.block_fill[b] = start; pv.block_seg_begin[b + 1] = k; }
             ++b; room = L; start = 0;
@@ -438,20 +442,18 @@ __global__ void __launch_bounds__(256, 1) k4_fill_lengths(PlanView pv, const int
         }
         int j = (int)(((uint64_t)(uint32_t)(u >> 32) * (uint32_t)m + __umulhi((uint32_t)u, (uint32_t)m)) >> 32);
         const int a = __popc(__ballot_sync(kFull, q0 <= j));
-        const int q1 = Q1[(a << 5) + lane];
-        int base = __shfl_sync(kFull, q0, (a - 1) & 31);
-        j -= a ? base : 0;
+        const int q1 = Q1[a * 33 + lane + 1];
+        j -= Q0[a];
         const int bb = __popc(__ballot_sync(kFull, q1 <= j));
         const int row = (a << 5) + bb;
         const int q2 = Q2[(row << 5) + lane];
-        base = __shfl_sync(kFull, q1, (bb - 1) & 31);
-        j -= bb ? base : 0;
+        j -= Q1[a * 33 + bb];
         const int c = __popc(__ballot_sync(kFull, (q2 & 63) <= j));
         const int len = (row << 5) + c + 1;
         const int cnt = (int)((uint32_t)__shfl_sync(kFull, q2, c) >> 6);  // unused sequences of the chosen length, >= 1
         if (cnt == 1) {  // the length runs out: it leaves the prefix counts of all three levels
-            if (lane >= a) { --q0; Q0[lane] = q0; }
-            if (lane >= bb) Q1[(a << 5) + lane] = q1 - 1;
+            if (lane >= a) { --q0; Q0[lane + 1] = q0; }
+            if (lane >= bb) Q1[a * 33 + lane + 1] = q1 - 1;
             if (lane >= c) Q2[(row << 5) + lane] = (lane == c ? q2 - 64 : q2) - 1;
         } else if (lane == c) {
             Q2[(row << 5) + lane] = q2 - 64;
@@ -582,7 +584,7 @@ cudaError_t launch_plan(const int32_t* d_lengths, int64_t n, int32_t t_block, ui
     k3_buckets<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(kin, n, t_block, wv.bucket_end, pv.hdr);
     if (ev) cudaEventRecord(ev[2], st);
 
-    const size_t smem = sizeof(int32_t) * (32 + 1024 + 128 + (size_t)((t_block + 31) / 32) * 32);
+    const size_t smem = sizeof(int32_t) * (kQ2Off + (size_t)((t_block + 31) / 32) * 33);
     auto fill = policy == BLOAD_POLICY_UNIFORM_LENGTHS ? k4_fill_lengths : k4_fill;
     cudaError_t e = cudaFuncSetAttribute(fill, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
