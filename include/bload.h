@@ -129,6 +129,23 @@ BLOAD_API int bload_plan(const int32_t* d_lengths, int64_t n, int32_t t_block, u
                bload_plan_info_t* info);
 
 /*
+ * bload_plan_async / bload_plan_finish -- bload_plan split in two, for callers that keep several plans
+ * in flight.  The fill rule is a chain of dependent draws that occupies one warp of one SM, so plans
+ * for different epochs (seeds) cost almost nothing extra when they run side by side on different
+ * streams, and a plan for the next epoch can run under the pack/unpack traffic of the current one.
+ *
+ * bload_plan_async checks its arguments exactly like bload_plan, enqueues the planner on `stream` and
+ * returns without synchronising (BLOAD_OK means "enqueued").  Each plan in flight needs its own d_plan
+ * and d_work.  bload_plan_finish copies the plan's scalars to the host on `stream`, synchronises that
+ * stream and fills `info` (all fields, taken from the plan itself); it returns info->status, and
+ * BLOAD_ERR_PLAN if the buffer does not hold a finished plan.  The paper has no counterpart (it builds
+ * its blocks on the host).
+ */
+BLOAD_API int bload_plan_async(const int32_t* d_lengths, int64_t n, int32_t t_block, uint64_t seed, uint32_t policy,
+                               void* d_plan, size_t plan_bytes, void* d_work, size_t work_bytes, void* stream);
+BLOAD_API int bload_plan_finish(const void* d_plan, void* stream, bload_plan_info_t* info);
+
+/*
  * bload_pack -- dense batches and per-slot metadata for blocks [block_begin, block_begin+block_count)
  * (paper, Methods: concatenate the sequences of a block, pad the rest with zeros; the start table).
  *

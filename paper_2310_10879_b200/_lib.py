@@ -17,7 +17,7 @@ ERR_NULL, ERR_ARG, ERR_LENGTH, ERR_WORKSPACE, ERR_ALIGN = -1, -2, -3, -4, -5
 ERR_UNSUPPORTED, ERR_CUDA, ERR_TIMEOUT, ERR_PLAN = -6, -7, -8, -9
 MAX_T_BLOCK = 32768
 
-EXPORTS = ("bload_plan_sizes", "bload_plan", "bload_pack", "bload_unpack", "bload_stats",
+EXPORTS = ("bload_plan_sizes", "bload_plan", "bload_plan_async", "bload_plan_finish", "bload_pack", "bload_unpack", "bload_stats",
            "bload_set_plan_timing", "bload_plan_stage_times", "bload_kernel_launches", "bload_strerror",
            "bload_version")
 
@@ -74,6 +74,8 @@ def load() -> C.CDLL:
     vp, i64, i32, u64, u32, u8 = C.c_void_p, C.c_int64, C.c_int32, C.c_uint64, C.c_uint32, C.c_uint8
     L.bload_plan_sizes.argtypes = [i64, i32, C.POINTER(Sizes)]
     L.bload_plan.argtypes = [vp, i64, i32, u64, u32, vp, C.c_size_t, vp, C.c_size_t, vp, C.POINTER(PlanInfo)]
+    L.bload_plan_async.argtypes = [vp, i64, i32, u64, u32, vp, C.c_size_t, vp, C.c_size_t, vp]
+    L.bload_plan_finish.argtypes = [vp, vp, C.POINTER(PlanInfo)]
     L.bload_pack.argtypes = [vp, C.POINTER(PlanInfo), vp, i64, i64, i64, vp, vp, vp, vp, vp, u8, vp]
     L.bload_unpack.argtypes = [vp, C.POINTER(PlanInfo), vp, i64, i64, i64, vp, vp]
     L.bload_stats.argtypes = [C.POINTER(PlanInfo), C.POINTER(Stats)]
@@ -169,6 +171,35 @@ def bload_plan(lengths, t_block: int, seed: int, policy: int = 0, stream=None, w
                            work.data_ptr(), work.numel(), _stream(stream), C.byref(info))
     if rc and check:
         err = BloadError(rc, "bload_plan")
+        err.info = info
+        raise err
+    return Plan(plan_buf, info, sizes)
+
+
+def bload_plan_async(lengths, t_block: int, seed: int, policy: int = 0, stream=None, work=None, plan_buf=None):
+    """Enqueue a plan without waiting for it.  Returns (plan_buf, work, sizes); keep all three alive and
+    call bload_plan_finish(plan_buf, sizes, stream) to obtain the Plan."""
+    import torch
+    if not lengths.is_cuda or lengths.dtype != torch.int32 or not lengths.is_contiguous():
+        raise TypeError("lengths must be a contiguous CUDA int32 tensor")
+    n = lengths.numel()
+    sizes = bload_plan_sizes(n, t_block)
+    if plan_buf is None:
+        plan_buf = torch.empty(sizes.plan_bytes, dtype=torch.uint8, device=lengths.device)
+    if work is None:
+        work = torch.empty(sizes.work_bytes, dtype=torch.uint8, device=lengths.device)
+    rc = load().bload_plan_async(lengths.data_ptr(), n, t_block, seed, policy, plan_buf.data_ptr(), plan_buf.numel(),
+                                 work.data_ptr(), work.numel(), _stream(stream))
+    if rc:
+        raise BloadError(rc, "bload_plan_async")
+    return plan_buf, work, sizes
+
+
+def bload_plan_finish(plan_buf, sizes: Sizes, stream=None, check: bool = True) -> Plan:
+    info = PlanInfo()
+    rc = load().bload_plan_finish(plan_buf.data_ptr(), _stream(stream), C.byref(info))
+    if rc and check:
+        err = BloadError(rc, "bload_plan_finish")
         err.info = info
         raise err
     return Plan(plan_buf, info, sizes)

@@ -176,6 +176,51 @@ int bload_plan(const int32_t* d_lengths, int64_t n, int32_t t_block, uint64_t se
     return info->status;
 }
 
+int bload_plan_async(const int32_t* d_lengths, int64_t n, int32_t t_block, uint64_t seed, uint32_t policy, void* d_plan,
+                     size_t plan_bytes, void* d_work, size_t work_bytes, void* stream)
+{
+    if (!d_lengths || !d_plan || !d_work) return BLOAD_ERR_NULL;
+    int rc = check_sizes(n, t_block);
+    if (rc) return rc;
+    if (policy > BLOAD_POLICY_UNIFORM_LENGTHS) return BLOAD_ERR_UNSUPPORTED;
+    if (policy == BLOAD_POLICY_UNIFORM_LENGTHS && n >= (1LL << 26)) return BLOAD_ERR_UNSUPPORTED;
+    bload_sizes_t sz;
+    plan_layout(n, &sz);
+    WorkView wv;
+    const size_t need_work = work_layout(n, t_block, d_work, &wv);
+    if (plan_bytes < sz.plan_bytes || work_bytes < need_work) return BLOAD_ERR_WORKSPACE;
+    if (!aligned(d_plan, kAlign) || !aligned(d_work, kAlign) || !aligned(d_lengths, 4)) return BLOAD_ERR_ALIGN;
+    cudaError_t ce = launch_plan(d_lengths, n, t_block, seed, policy, plan_view(d_plan, n), wv,
+                                 static_cast<cudaStream_t>(stream), nullptr);
+    if (ce != cudaSuccess) { (void)cudaGetLastError(); return BLOAD_ERR_CUDA; }
+    return BLOAD_OK;
+}
+
+int bload_plan_finish(const void* d_plan, void* stream, bload_plan_info_t* info)
+{
+    if (!info) return BLOAD_ERR_NULL;
+    memset(info, 0, sizeof *info);
+    info->first_bad_index = -1;
+    auto fail = [&](int rc) { info->status = rc; return rc; };
+    if (!d_plan) return fail(BLOAD_ERR_NULL);
+    if (!aligned(d_plan, kAlign)) return fail(BLOAD_ERR_ALIGN);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    PlanHeader h;
+    cudaError_t ce = cudaMemcpyAsync(&h, d_plan, sizeof h, cudaMemcpyDeviceToHost, st);
+    if (ce == cudaSuccess) ce = cudaStreamSynchronize(st);
+    if (ce != cudaSuccess) { (void)cudaGetLastError(); return fail(BLOAD_ERR_CUDA); }
+    info->n = h.n; info->t_block = h.t_block; info->seed = h.seed; info->policy = h.policy;
+    info->status = h.status;
+    info->n_blocks = h.n_blocks;
+    info->sum_t = h.sum_t;
+    info->t_max = h.t_max;
+    info->first_bad_index = h.first_bad == ~0ULL ? -1 : (int64_t)h.first_bad;
+    info->checksum = h.checksum;
+    info->max_segs_per_block = h.max_segs;
+    if (h.status == BLOAD_OK && h.magic != kPlanMagic) return fail(BLOAD_ERR_PLAN);
+    return info->status;
+}
+
 int bload_pack(const void* d_plan, const bload_plan_info_t* info, const void* d_store, int64_t frame_bytes,
                int64_t block_begin, int64_t block_count, void* d_dense, int32_t* d_seq_id, int32_t* d_pos,
                uint8_t* d_reset, uint8_t* d_valid, uint8_t pad_byte, void* stream)
