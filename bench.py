@@ -296,6 +296,59 @@ def run_gpu(args, w) -> dict:
     step_s = seconds / args.steps
     value = aggregate(by["pack"] + by["unpack"], world, step_s) / 1e9
 
+    # ---- the same work as a two-stage pipeline: the plan of epoch e+1 runs on a side stream (one warp of one SM)
+    # under the metadata/pack/unpack traffic of epoch e; and eight plans side by side on eight streams
+    pipelined = None
+    if not args.no_pipeline:
+        side = torch.cuda.Stream()
+        main = torch.cuda.current_stream()
+        bufs = [torch.empty(sizes.plan_bytes, dtype=torch.uint8, device=dev) for _ in range(2)]
+        work2 = torch.empty(sizes.work_bytes, dtype=torch.uint8, device=dev)
+
+        def pipeline(steps):
+            side.wait_stream(main)
+            B.bload_plan_async(d_len, tb, w.seed, policy=args.policy, stream=side, work=work2, plan_buf=bufs[0])
+            p = B.bload_plan_finish(bufs[0], sizes, stream=side)
+            done = [None, None]
+            for i in range(steps):
+                nxt = (i + 1) % 2
+                if done[nxt] is not None:
+                    side.wait_event(done[nxt])          # the copies that read this plan buffer have finished
+                B.bload_plan_async(d_len, tb, w.seed, policy=args.policy, stream=side, work=work2, plan_buf=bufs[nxt])
+                B.bload_pack(p, None, fb, 0, nb, seq_id=seq_id, pos=pos, reset=reset, valid=valid)
+                B.bload_pack(p, store, fb, 0, nb, dense=dense)
+                B.bload_unpack(p, dense_out, ofb, 0, nb, ragged_out)
+                done[i % 2] = main.record_event()
+                p = B.bload_plan_finish(bufs[nxt], sizes, stream=side)   # the host waits for the plan only
+                B.bload_stats(p.info)
+            main.wait_stream(side)
+
+        pipeline(3)
+        torch.cuda.synchronize()
+        psteps = max(10, min(args.steps, 100))
+        a, b_ = ev(), ev()
+        a.record(); pipeline(psteps); b_.record()
+        torch.cuda.synchronize()
+        pms = a.elapsed_time(b_) / psteps
+        streams8 = [torch.cuda.Stream() for _ in range(8)]
+        jobs8 = [(torch.empty(sizes.plan_bytes, dtype=torch.uint8, device=dev),
+                  torch.empty(sizes.work_bytes, dtype=torch.uint8, device=dev)) for _ in range(8)]
+
+        def eight():
+            for e, (st8, (pb, wk)) in enumerate(zip(streams8, jobs8)):
+                st8.wait_stream(main)
+                B.bload_plan_async(d_len, tb, w.seed + e, policy=args.policy, stream=st8, work=wk, plan_buf=pb)
+            for st8, (pb, wk) in zip(streams8, jobs8):
+                B.bload_plan_finish(pb, sizes, stream=st8)
+        eight()
+        torch.cuda.synchronize()
+        t0 = time.perf_counter(); eight(); torch.cuda.synchronize(); t8 = (time.perf_counter() - t0) * 1e3
+        pipelined = {"ms_per_step": pms, "value": (by["pack"] + by["unpack"]) / pms / 1e6, "unit": UNIT, "steps": psteps,
+                     "what": "plan of epoch e+1 on a side stream under metadata+pack+unpack of epoch e (every step still "
+                             "plans, packs and unpacks one whole epoch)",
+                     "eight_plans_side_by_side_ms": t8, "plans_per_s": 8e3 / t8}
+        del bufs, work2, jobs8
+
     # ---- batch-by-batch use: one pack call (metadata + dense) per training batch of w.batch_blocks blocks,
     # the last batch rounded up with filler blocks; the output buffers of one batch are reused
     bb = w.batch_blocks
@@ -415,7 +468,7 @@ def run_gpu(args, w) -> dict:
            "ms_per_step": step_s * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
            "dtype": "u8", "data": "synthetic", "config": config_of(w, {"parallelism": "replicas only"}),
            "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline,
-           "frames_per_s": aggregate(sum_t, world, step_s), "per_batch_pack": per_batch,
+           "frames_per_s": aggregate(sum_t, world, step_s), "per_batch_pack": per_batch, "pipelined": pipelined,
            "kernels": {
                "pack_copy": {"ms": pack_ms, "GB/s": by["pack"] / pack_ms / 1e6, "frac_measured": by["pack"] / pack_ms / 1e6 / peak,
                              "frac_nominal": by["pack"] / pack_ms / 1e6 / NOMINAL_HBM_GBS, "frames_per_s": sum_t / pack_ms * 1e3},
@@ -463,6 +516,7 @@ def main():
                     help="blocks in the CPU oracle's sample (0 = all blocks for the CPU baseline; sized from a "
                          "calibration run for --impl reference)")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-pipeline", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "bload" else args.warmup
