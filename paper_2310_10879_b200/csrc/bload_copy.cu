@@ -209,7 +209,9 @@ struct StageCfgT {
 };
 template <bool UNPACK> struct StageCfg : StageCfgT<BLOAD_PACK_CFG> {};
 template <> struct StageCfg<true> : StageCfgT<BLOAD_UNPACK_CFG> {};
-constexpr int64_t kStagedMaxFrameBytes = 256;
+// the staged kernels win while the average run (T_i * frame_bytes) is short; measured cross-over on B200 at about
+// 16 KB (1.4 KB runs: 6.0 against 3.8 TB/s; 14 KB: 5.9 against 5.8; 23 KB: 6.15 against 6.36)
+constexpr int64_t kStagedMaxRunBytes = 16384;
 #ifndef BLOAD_PACK_CHUNK_TILES
 #define BLOAD_PACK_CHUNK_TILES 4
 #endif
@@ -651,7 +653,8 @@ cudaError_t launch_copy(bool unpack, const PlanView& pv, int32_t t_block, int64_
     const int64_t block_bytes = (int64_t)t_block * frame_bytes;
     count_launches(1);
     // pack of small word-sized frames: contiguous ranges of dense sub-tiles per warp
-    if (!unpack && frame_bytes % 4 == 0 && block_bytes % 16 == 0 && frame_bytes <= kStagedMaxFrameBytes) {
+    const bool short_runs = frame_bytes % 4 == 0 && n > 0 && ragged_bytes / n <= kStagedMaxRunBytes && block_bytes < (1LL << 31);
+    if (!unpack && short_runs && block_bytes % 16 == 0) {
         using Cfg = StageCfg<false>;
         const size_t smem = (size_t)Cfg::kWarps * Cfg::kStages * Cfg::kBytes + 16;
         const int per_sm = (int)((227 * 1024) / (smem + 1024));
@@ -670,8 +673,7 @@ cudaError_t launch_copy(bool unpack, const PlanView& pv, int32_t t_block, int64_
         return cudaPeekAtLastError();
     }
     // whole-plan unpack of small word-sized frames: tile the (contiguous, fully written) ragged side
-    if (unpack && frame_bytes % 4 == 0 && frame_bytes <= kStagedMaxFrameBytes && block_begin == 0 &&
-        block_count >= n_blocks && ragged_bytes > 0) {
+    if (unpack && short_runs && block_begin == 0 && block_count >= n_blocks && ragged_bytes > 0) {
         using Cfg = StageCfg<false>;
         const size_t smem = (size_t)Cfg::kWarps * Cfg::kStages * Cfg::kBytes + 16;
         const int per_sm = (int)((227 * 1024) / (smem + 1024));
@@ -687,7 +689,7 @@ cudaError_t launch_copy(bool unpack, const PlanView& pv, int32_t t_block, int64_
         return cudaPeekAtLastError();
     }
     // block sub-ranges of small word-sized frames, unpack direction: staged kernel over the dense side
-    if (unpack && frame_bytes % 4 == 0 && block_bytes % 16 == 0 && frame_bytes <= kStagedMaxFrameBytes) {
+    if (unpack && short_runs && block_bytes % 16 == 0) {
         using Cfg = StageCfg<true>;
         const int64_t spb = (block_bytes + Cfg::kBytes - 1) / Cfg::kBytes;
         const int64_t gpb = (spb + Cfg::kGroup - 1) / Cfg::kGroup;  // groups of sub-tiles per block

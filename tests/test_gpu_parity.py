@@ -219,10 +219,11 @@ def test_plan_on_a_side_stream_and_reuse_of_buffers():
 
 @pytest.mark.parametrize("tb,fb,tmax", [(4, 4, 4), (64, 4, 64), (1000, 16, 9), (4096, 4, 4096), (4096, 8, 40),
                                         (20000, 36, 3000), (20000, 4, 20000), (700, 256, 300), (32768, 12, 5000),
-                                        (5000, 64, 2), (2048, 20, 2048)])
+                                        (5000, 64, 2), (2048, 20, 2048), (64, 1024, 8), (100, 4096, 3), (37, 16384, 1),
+                                        (300, 2052, 6)])
 def test_small_word_sized_frames_take_the_staged_path(tb, fb, tmax):
-    """Frames of 4..256 bytes (multiples of 4) with 16-byte-multiple blocks go through the shared-memory
-    staged kernels: many sub-tiles per block, runs cut by sub-tile ends, more than 32 runs per sub-tile,
+    """Word-sized frames whose runs are short on average (up to 16 KB) and whose blocks are multiples of 16 bytes go
+    through the shared-memory staged kernels, the rest through the register path: many sub-tiles per block, runs cut by sub-tile ends, more than 32 runs per sub-tile,
     pad-only sub-tiles, filler blocks, a non-zero pad byte."""
     assert (tb * fb) % 16 == 0
     rng = np.random.default_rng(tb * 131 + fb)
