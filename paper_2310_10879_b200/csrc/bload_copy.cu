@@ -52,21 +52,28 @@ __device__ __forceinline__ uint4 splice(uint4 a, uint4 b, int bits)
     return o;
 }
 
-template <int WS, int U>
+// Loads of the realigning path: neighbouring lanes (and the two loads of one lane) touch the same 32-byte
+// sectors.  Measured on B200 with 64..1028-byte frames: letting them allocate in L1 helps when the source is
+// the dense side (unpack, +3..6 %) and costs when it is the ragged store (pack, -3..5 %), so the direction chooses.
+template <bool CACHED>
+__device__ __forceinline__ uint4 ld_shared_sector(const uint4* p) { return CACHED ? __ldg(p) : __ldcs(p); }
+
+template <int WS, int U, bool CACHED>
 __device__ __forceinline__ void warp_copy_shifted(uint4* __restrict__ d, const uint4* __restrict__ a, int64_t nv, int bits, int lane)
 {
     int64_t i = lane;
     for (; i + 32 * (U - 1) < nv; i += 32 * U) {
         uint4 lo[U], hi[U];
 #pragma unroll
-        for (int u = 0; u < U; ++u) { lo[u] = ld_stream(a + i + 32 * u); hi[u] = ld_stream(a + i + 32 * u + 1); }
+        for (int u = 0; u < U; ++u) { lo[u] = ld_shared_sector<CACHED>(a + i + 32 * u); hi[u] = ld_shared_sector<CACHED>(a + i + 32 * u + 1); }
 #pragma unroll
         for (int u = 0; u < U; ++u) st_stream(d + i + 32 * u, splice<WS>(lo[u], hi[u], bits));
     }
-    for (; i < nv; i += 32) st_stream(d + i, splice<WS>(ld_stream(a + i), ld_stream(a + i + 1), bits));
+    for (; i < nv; i += 32) st_stream(d + i, splice<WS>(ld_shared_sector<CACHED>(a + i), ld_shared_sector<CACHED>(a + i + 1), bits));
 }
 
 // Copy n bytes; s_limit is the end of the whole source buffer (no load goes beyond it).
+template <bool CACHED>
 __device__ __forceinline__ void warp_copy(uint8_t* __restrict__ d, const uint8_t* __restrict__ s, int64_t n,
                                           const uint8_t* s_limit, int lane)
 {
@@ -86,10 +93,10 @@ __device__ __forceinline__ void warp_copy(uint8_t* __restrict__ d, const uint8_t
         uint4* dv = reinterpret_cast<uint4*>(d);
         const uint4* av = reinterpret_cast<const uint4*>(a);
         switch (sh >> 2) {
-            case 0: warp_copy_shifted<0, 4>(dv, av, nv, bits, lane); break;
-            case 1: warp_copy_shifted<1, 4>(dv, av, nv, bits, lane); break;
-            case 2: warp_copy_shifted<2, 4>(dv, av, nv, bits, lane); break;
-            default: warp_copy_shifted<3, 4>(dv, av, nv, bits, lane); break;
+            case 0: warp_copy_shifted<0, 4, CACHED>(dv, av, nv, bits, lane); break;
+            case 1: warp_copy_shifted<1, 4, CACHED>(dv, av, nv, bits, lane); break;
+            case 2: warp_copy_shifted<2, 4, CACHED>(dv, av, nv, bits, lane); break;
+            default: warp_copy_shifted<3, 4, CACHED>(dv, av, nv, bits, lane); break;
         }
     }
     for (int64_t t = (nv << 4) + lane; t < n; t += 32) d[t] = s[t];
@@ -166,9 +173,9 @@ __global__ void __launch_bounds__(256) k7_copy(PlanView pv, int32_t t_block, int
                     const int64_t pe = min((int64_t)nx * frame_bytes, hi);
                     const int64_t rag = src_frame * frame_bytes + (cur - seg_b);
                     if (UNPACK)
-                        warp_copy(dst_base + rag, src_base + dense_off + cur, pe - cur, s_limit, lane);
+                        warp_copy<true>(dst_base + rag, src_base + dense_off + cur, pe - cur, s_limit, lane);
                     else
-                        warp_copy(dst_base + dense_off + cur, src_base + rag, pe - cur, s_limit, lane);
+                        warp_copy<false>(dst_base + dense_off + cur, src_base + rag, pe - cur, s_limit, lane);
                     cur = pe;
                     ++k;
                 }
