@@ -117,7 +117,8 @@ typedef struct {
     int32_t t_block;
     uint64_t seed;
     uint32_t policy; /* 0 = uniform over the unused sequences that fit; 1 = uniform over the LENGTHS (keys of
-                        L_dict) that fit and still have an unused sequence */
+                        L_dict) that fit and still have an unused sequence; 2 = best fit decreasing, a
+                        deterministic comparison strategy that is NOT the paper's rule */
     /* outputs, all caller-allocated */
     int64_t *offsets;         /* [n+1] */
     int32_t *seg_seq;         /* [n]   sequence placed by the k-th draw */
@@ -159,7 +160,7 @@ int oracle_plan(oracle_plan_t *p)
     p->n_blocks = 0; p->sum_t = 0; p->t_max = 0; p->first_bad = -1;
     p->checksum = 0; p->max_segs_per_block = 0;
     if (n < 1 || n > 0x7fffffffLL || tb < 1) return ORACLE_ERR_ARG;
-    if (p->policy > 1) return ORACLE_ERR_POLICY;
+    if (p->policy > 2) return ORACLE_ERR_POLICY;
 
     /* Precondition of the method: 1 <= T_i <= block length. */
     for (int64_t i = 0; i < n; ++i) {
@@ -186,6 +187,55 @@ int oracle_plan(oracle_plan_t *p)
 
     int64_t k = 0;      /* draws made so far */
     int64_t b = 0;      /* current block */
+    if (p->policy == 2) {
+        /* Best fit decreasing (textbook bin packing heuristic): sequences in decreasing order of length
+         * (the reverse of the L_dict order); each goes to the open block whose free room is the smallest
+         * that still holds it -- among blocks with equal room, the one that has had that room longest --
+         * or opens a new block when none has room.  head/tail/next: one FIFO of blocks per room value. */
+        int32_t *head = (int32_t *)malloc(sizeof(int32_t) * ((size_t)tb + 1));
+        int32_t *tail = (int32_t *)malloc(sizeof(int32_t) * ((size_t)tb + 1));
+        int32_t *next = (int32_t *)malloc(sizeof(int32_t) * (size_t)n);
+        int32_t *item_block = (int32_t *)malloc(sizeof(int32_t) * (size_t)n);
+        int32_t *item_start = (int32_t *)malloc(sizeof(int32_t) * (size_t)n);
+        if (!head || !tail || !next || !item_block || !item_start) {
+            free(head); free(tail); free(next); free(item_block); free(item_start);
+            free(dict); free(first); free(unused);
+            return ORACLE_ERR_NOMEM;
+        }
+        for (int32_t r = 0; r <= tb; ++r) head[r] = tail[r] = -1;
+        for (int64_t t = 0; t < n; ++t) {
+            const int32_t l = dict[n - 1 - t].len;
+            int32_t r = l;
+            while (r <= tb && head[r] < 0) ++r;          /* smallest room >= l among the open blocks */
+            int32_t blk, start;
+            if (r > tb) { blk = (int32_t)b++; start = 0; r = tb; p->block_fill[blk] = 0; }
+            else { blk = head[r]; head[r] = next[blk]; if (head[r] < 0) tail[r] = -1; start = tb - r; }
+            const int32_t room = r - l;                   /* a block without room left is never looked at again */
+            if (room > 0) {
+                next[blk] = -1;
+                if (tail[room] >= 0) next[tail[room]] = blk; else head[room] = blk;
+                tail[room] = blk;
+            }
+            item_block[t] = blk; item_start[t] = start;
+            p->block_fill[blk] = start + l;
+        }
+        /* segment list: blocks in opening order, inside a block in placement order */
+        for (int64_t q = 0; q <= b; ++q) p->block_seg_begin[q] = 0;
+        for (int64_t t = 0; t < n; ++t) p->block_seg_begin[item_block[t] + 1] += 1;
+        for (int64_t q = 0; q < b; ++q) {
+            if (p->block_seg_begin[q + 1] > p->max_segs_per_block) p->max_segs_per_block = p->block_seg_begin[q + 1];
+            p->block_seg_begin[q + 1] += p->block_seg_begin[q];
+        }
+        int32_t *cursor = next;                           /* reuse: next free position of each block */
+        for (int64_t q = 0; q < b; ++q) cursor[q] = p->block_seg_begin[q];
+        for (int64_t t = 0; t < n; ++t) {
+            const int32_t id = dict[n - 1 - t].id, blk = item_block[t], pos = cursor[blk]++;
+            p->seg_seq[pos] = id; p->seg_block[pos] = blk; p->seg_start[pos] = item_start[t];
+            p->seq_block[id] = blk; p->seq_start[id] = item_start[t];
+        }
+        free(head); free(tail); free(next); free(item_block); free(item_start);
+        k = n;
+    }
     while (k < n) {
         int32_t remaining = tb, start = 0;
         p->block_seg_begin[b] = (int32_t)k;
@@ -228,7 +278,7 @@ int oracle_plan(oracle_plan_t *p)
         if (segs > p->max_segs_per_block) p->max_segs_per_block = segs;
         b += 1;
     }
-    p->block_seg_begin[b] = (int32_t)k;
+    if (p->policy != 2) p->block_seg_begin[b] = (int32_t)k;
     p->n_blocks = b;
 
     /* Order-independent 64-bit digest of the segment list. */

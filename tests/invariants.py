@@ -22,7 +22,9 @@ def _req(cond, msg):
 
 
 def check_plan(lengths, t_block, n_blocks, offsets, seg_seq, seg_block, seg_start, block_seg_begin,
-               block_fill, seq_block, seq_start):
+               block_fill, seq_block, seq_start, maximal=True):
+    """maximal=False skips I5, which belongs to the paper's rule (a block is closed only when nothing that is
+    left fits) and does not hold for strategies that keep several blocks open."""
     T = np.asarray(lengths, dtype=np.int64)
     n = T.size
     seg_seq = np.asarray(seg_seq)[:n].astype(np.int64)
@@ -54,12 +56,13 @@ def check_plan(lengths, t_block, n_blocks, offsets, seg_seq, seg_block, seg_star
     # I5: everything placed after block b was too long for the room left in b
     min_len_block = np.minimum.reduceat(seg_len, bsb[:-1])
     suffix_min = np.minimum.accumulate(min_len_block[::-1])[::-1]
-    if n_blocks > 1:
+    if n_blocks > 1 and maximal:
         _req(np.all(suffix_min[1:] > t_block - fill[:-1]), "I5: a later sequence would have fitted")
         _req(np.all(fill[:-1] + fill[1:] > t_block), "I5': adjacent blocks could merge")
     s = int(T.sum())
     _req(-(-s // t_block) <= n_blocks, "fewer blocks than the volume bound")
-    _req(n_blocks < 2 * s / t_block + 1, "I5'': too many blocks")
+    if maximal:
+        _req(n_blocks < 2 * s / t_block + 1, "I5'': too many blocks")
     return True
 
 
