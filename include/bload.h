@@ -50,6 +50,8 @@ extern "C" {
 
 #define BLOAD_MAX_T_BLOCK 32768
 #define BLOAD_POLICY_UNIFORM_SEQUENCES 0u /* every unused sequence that fits is equally likely */
+#define BLOAD_POLICY_BEST_FIT_DECREASING 2u /* NOT the paper's rule: the textbook best-fit-decreasing heuristic, a
+                                             deterministic low-padding comparison (seed only orders equal lengths) */
 #define BLOAD_POLICY_UNIFORM_LENGTHS 1u   /* every length (key of L_dict) that fits and is not exhausted is equally
                                              likely, then the next unused sequence of that length; needs n < 2^26 */
 
@@ -115,7 +117,9 @@ BLOAD_API int bload_plan_sizes(int64_t n, int32_t t_block, bload_sizes_t* out);
  * in the open block, one of them is drawn uniformly at random and appended (the paper's Random_*()
  * over L_dict); when none fits, the rest of the block is padding and the next block is opened.
  * Randomness comes from the counter-based generator Philox-4x64-10 keyed by `seed`, so the plan is
- * a pure function of (lengths, t_block, seed, policy).
+ * a pure function of (lengths, t_block, seed, policy).  `policy` selects the reading of "random entry"
+ * (BLOAD_POLICY_UNIFORM_SEQUENCES, the default, or BLOAD_POLICY_UNIFORM_LENGTHS) or the deterministic
+ * comparison strategy BLOAD_POLICY_BEST_FIT_DECREASING, which is not the paper's rule.
  *
  *   d_lengths  device int32[n], 4-byte aligned; every T_i must satisfy 1 <= T_i <= t_block
  *   d_plan     device buffer of plan_bytes bytes, 256-byte aligned; receives the tables

@@ -107,7 +107,7 @@ int bload_plan_sizes(int64_t n, int32_t t_block, bload_sizes_t* out)
     int rc = check_sizes(n, t_block);
     if (rc) return rc;
     plan_layout(n, out);
-    out->work_bytes = work_layout(n, t_block, nullptr, nullptr);
+    out->work_bytes = work_layout(n, t_block, nullptr, nullptr) + bfd_layout(n, t_block, nullptr, nullptr);
     return BLOAD_OK;
 }
 
@@ -136,12 +136,14 @@ int bload_plan(const int32_t* d_lengths, int64_t n, int32_t t_block, uint64_t se
     if (!d_lengths || !d_plan || !d_work) return fail(BLOAD_ERR_NULL);
     int rc = check_sizes(n, t_block);
     if (rc) return fail(rc);
-    if (policy > BLOAD_POLICY_UNIFORM_LENGTHS) return fail(BLOAD_ERR_UNSUPPORTED);
+    if (policy > BLOAD_POLICY_BEST_FIT_DECREASING) return fail(BLOAD_ERR_UNSUPPORTED);
     if (policy == BLOAD_POLICY_UNIFORM_LENGTHS && n >= (1LL << 26)) return fail(BLOAD_ERR_UNSUPPORTED);
     bload_sizes_t sz;
     plan_layout(n, &sz);
     WorkView wv;
-    const size_t need_work = work_layout(n, t_block, d_work, &wv);
+    BfdView bv;
+    size_t need_work = work_layout(n, t_block, d_work, &wv);  // the size bload_plan_sizes reports covers every policy
+    need_work += bfd_layout(n, t_block, static_cast<char*>(d_work) + need_work, &bv);
     if (plan_bytes < sz.plan_bytes || work_bytes < need_work) return fail(BLOAD_ERR_WORKSPACE);
     if (!aligned(d_plan, kAlign) || !aligned(d_work, kAlign) || !aligned(d_lengths, 4)) return fail(BLOAD_ERR_ALIGN);
 
@@ -152,7 +154,7 @@ int bload_plan(const int32_t* d_lengths, int64_t n, int32_t t_block, uint64_t se
     if (timing)
         for (int i = 0; i < 5; ++i)
             if (cudaEventCreate(&ev[i]) != cudaSuccess) { timing = false; break; }
-    cudaError_t ce = launch_plan(d_lengths, n, t_block, seed, policy, pv, wv, st, timing ? ev : nullptr);
+    cudaError_t ce = launch_plan(d_lengths, n, t_block, seed, policy, pv, wv, st, timing ? ev : nullptr, &bv);
     PlanHeader h;
     if (ce == cudaSuccess) ce = cudaMemcpyAsync(&h, pv.hdr, sizeof h, cudaMemcpyDeviceToHost, st);
     if (ce == cudaSuccess) ce = cudaStreamSynchronize(st);
@@ -182,16 +184,18 @@ int bload_plan_async(const int32_t* d_lengths, int64_t n, int32_t t_block, uint6
     if (!d_lengths || !d_plan || !d_work) return BLOAD_ERR_NULL;
     int rc = check_sizes(n, t_block);
     if (rc) return rc;
-    if (policy > BLOAD_POLICY_UNIFORM_LENGTHS) return BLOAD_ERR_UNSUPPORTED;
+    if (policy > BLOAD_POLICY_BEST_FIT_DECREASING) return BLOAD_ERR_UNSUPPORTED;
     if (policy == BLOAD_POLICY_UNIFORM_LENGTHS && n >= (1LL << 26)) return BLOAD_ERR_UNSUPPORTED;
     bload_sizes_t sz;
     plan_layout(n, &sz);
     WorkView wv;
-    const size_t need_work = work_layout(n, t_block, d_work, &wv);
+    BfdView bv;
+    size_t need_work = work_layout(n, t_block, d_work, &wv);  // the size bload_plan_sizes reports covers every policy
+    need_work += bfd_layout(n, t_block, static_cast<char*>(d_work) + need_work, &bv);
     if (plan_bytes < sz.plan_bytes || work_bytes < need_work) return BLOAD_ERR_WORKSPACE;
     if (!aligned(d_plan, kAlign) || !aligned(d_work, kAlign) || !aligned(d_lengths, 4)) return BLOAD_ERR_ALIGN;
     cudaError_t ce = launch_plan(d_lengths, n, t_block, seed, policy, plan_view(d_plan, n), wv,
-                                 static_cast<cudaStream_t>(stream), nullptr);
+                                 static_cast<cudaStream_t>(stream), nullptr, &bv);
     if (ce != cudaSuccess) { (void)cudaGetLastError(); return BLOAD_ERR_CUDA; }
     return BLOAD_OK;
 }

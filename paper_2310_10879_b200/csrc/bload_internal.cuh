@@ -65,12 +65,38 @@ size_t work_layout(int64_t n, int32_t t_block, void* base, WorkView* w);
 void plan_layout(int64_t n, bload_sizes_t* s);
 PlanView plan_view(void* d_plan, int64_t n);
 
+// Extra scratch of the best-fit-decreasing planner (policy 2), placed after the WorkView region.
+struct BfdView {
+    int2* rec;            // [n] per item in placement order: {room it was taken from (0 = new block), room it left}
+    uint64_t* ek_a;       // [n] event sort keys, ping
+    uint64_t* ek_b;       // [n] pong
+    int32_t* ei_a;        // [n] event payload (item index), ping
+    int32_t* ei_b;        // [n] pong
+    int32_t* put_item;    // [n] items ordered by (room they left, time)
+    int32_t* jump_a;      // [n] predecessor pointers, ping
+    int32_t* jump_b;      // [n] pong
+    int32_t* blk;         // [n] block of item t
+    int32_t* put_end;     // [t_block + 1] items that left a room <= r
+    int32_t* take_end;    // [t_block + 1] items that took a room <= r (room 0 = opened a new block)
+};
+size_t bfd_layout(int64_t n, int32_t t_block, void* base, BfdView* v);
+
+// stable LSD radix sort of (key, id) pairs on `digits` 8-bit digits starting at bit `first_shift`; the sorted
+// arrays are returned in *k_out / *i_out (one of the two ping-pong pairs); and counts of keys by their high word
+cudaError_t plan_radix_sort(uint64_t* ka, int32_t* ia, uint64_t* kb, int32_t* ib, int64_t n, int first_shift, int digits,
+                            uint32_t* hist, const PlanHeader* hdr, cudaStream_t st, uint64_t** k_out, int32_t** i_out);
+cudaError_t plan_key_buckets(const uint64_t* sorted_keys, int64_t n, int32_t max_value, int32_t* bucket_end,
+                             const PlanHeader* hdr, cudaStream_t st);
+cudaError_t launch_bfd(const PlanView& pv, const WorkView& wv, const BfdView& bv, const uint64_t* sorted_key,
+                       const int32_t* sorted_id, int64_t n, int32_t t_block, cudaStream_t st);
+
 // every kernel launch of the library goes through this counter (see bload_kernel_launches)
 void count_launches(int k);
 
 // launchers (each returns a cudaError_t from cudaPeekAtLastError)
 cudaError_t launch_plan(const int32_t* d_lengths, int64_t n, int32_t t_block, uint64_t seed, uint32_t policy,
-                        const PlanView& pv, const WorkView& wv, cudaStream_t st, cudaEvent_t* ev /*5 or null*/);
+                        const PlanView& pv, const WorkView& wv, cudaStream_t st, cudaEvent_t* ev /*5 or null*/,
+                        const BfdView* bv = nullptr /*policy 2 only*/);
 cudaError_t launch_metadata(const PlanView& pv, int32_t t_block, int64_t block_begin, int64_t block_count,
                             int32_t* seq_id, int32_t* pos, uint8_t* reset, uint8_t* valid, cudaStream_t st);
 cudaError_t launch_copy(bool unpack, const PlanView& pv, int32_t t_block, int64_t frame_bytes, int64_t block_begin,

@@ -555,8 +555,36 @@ size_t work_layout(int64_t n, int32_t t_block, void* base, WorkView* w)
     return off;
 }
 
+cudaError_t plan_radix_sort(uint64_t* ka, int32_t* ia, uint64_t* kb, int32_t* ib, int64_t n, int first_shift, int digits,
+                            uint32_t* hist, const PlanHeader* hdr, cudaStream_t st, uint64_t** k_out, int32_t** i_out)
+{
+    const int64_t chunks = chunks_of(n);
+    const unsigned gc = (unsigned)chunks;
+    uint64_t *kin = ka, *kout = kb;
+    int32_t *iin = ia, *iout = ib;
+    for (int p = 0; p < digits; ++p) {
+        const int shift = first_shift + 8 * p;
+        k3_hist<<<gc, 256, 0, st>>>(kin, n, shift, chunks, hist, hdr);
+        k3_scan<<<1, 1024, 0, st>>>(hist, 256 * chunks, hdr);
+        k3_scatter<<<gc, 256, 0, st>>>(kin, iin, kout, iout, n, shift, chunks, hist, hdr);
+        uint64_t* tk = kin; kin = kout; kout = tk;
+        int32_t* ti = iin; iin = iout; iout = ti;
+    }
+    count_launches(3 * digits);
+    *k_out = kin; *i_out = iin;
+    return cudaPeekAtLastError();
+}
+
+cudaError_t plan_key_buckets(const uint64_t* sorted_keys, int64_t n, int32_t max_value, int32_t* bucket_end,
+                             const PlanHeader* hdr, cudaStream_t st)
+{
+    k3_buckets<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(sorted_keys, n, max_value, bucket_end, hdr);
+    count_launches(1);
+    return cudaPeekAtLastError();
+}
+
 cudaError_t launch_plan(const int32_t* d_lengths, int64_t n, int32_t t_block, uint64_t seed, uint32_t policy,
-                        const PlanView& pv, const WorkView& wv, cudaStream_t st, cudaEvent_t* ev)
+                        const PlanView& pv, const WorkView& wv, cudaStream_t st, cudaEvent_t* ev, const BfdView* bv)
 {
     const int64_t chunks = chunks_of(n);
     const unsigned gc = (unsigned)chunks;
@@ -584,6 +612,12 @@ cudaError_t launch_plan(const int32_t* d_lengths, int64_t n, int32_t t_block, ui
     k3_buckets<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(kin, n, t_block, wv.bucket_end, pv.hdr);
     if (ev) cudaEventRecord(ev[2], st);
 
+    if (policy == BLOAD_POLICY_BEST_FIT_DECREASING) {  // a different planner from here on (see bload_bfd.cu)
+        count_launches(4 + 3 * passes + 1);
+        cudaError_t eb = bv ? launch_bfd(pv, wv, *bv, kin, iin, n, t_block, st) : cudaErrorInvalidValue;
+        if (ev) { cudaEventRecord(ev[3], st); cudaEventRecord(ev[4], st); }
+        return eb;
+    }
     const size_t smem = sizeof(int32_t) * (kQ2Off + (size_t)((t_block + 31) / 32) * 33);
     auto fill = policy == BLOAD_POLICY_UNIFORM_LENGTHS ? k4_fill_lengths : k4_fill;
     cudaError_t e = cudaFuncSetAttribute(fill, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);

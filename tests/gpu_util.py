@@ -20,7 +20,7 @@ def host_tables(plan) -> dict:
     return {k: v.cpu().numpy() for k, v in plan.tables().items()}
 
 
-def assert_plan_equal(plan, op):
+def assert_plan_equal(plan, op, maximal=None):
     """GPU plan vs oracle plan: every table and scalar, bit exact; plus the validity checker."""
     i = plan.info
     assert i.status == 0 and op.status == 0
@@ -36,8 +36,11 @@ def assert_plan_equal(plan, op):
             raise AssertionError("%s differs first at %d: gpu %s oracle %s" % (name, bad, a[bad], b[bad]))
     assert np.array_equal(t["seg_src"], op.offsets[op.seg_seq.astype(np.int64)])
     assert i.checksum == op.checksum and i.max_segs_per_block == op.max_segs_per_block
+    if maximal is None:
+        maximal = i.policy != 2            # best fit decreasing keeps several blocks open
     invariants.check_plan(op.lengths, i.t_block, i.n_blocks, t["offsets"], t["seg_seq"], t["seg_block"],
-                          t["seg_start"], t["block_seg_begin"], t["block_fill"], t["seq_block"], t["seq_start"])
+                          t["seg_start"], t["block_seg_begin"], t["block_fill"], t["seq_block"], t["seq_start"],
+                          maximal=maximal)
 
 
 class Guarded:

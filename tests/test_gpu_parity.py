@@ -275,3 +275,37 @@ def test_policy1_small_and_degenerate_cases():
     for n in (1, 31, 32, 33, 2049, 70001):
         T = rng.integers(1, 301, size=n).astype(np.int32)
         G.assert_plan_equal(G.gpu_plan(T, 300, 5, policy=1), O.plan(T, 300, 5, policy=1))
+
+
+# ---- policy 2: best fit decreasing (deterministic comparison strategy) ----
+
+@pytest.mark.parametrize("name,n", [("toy_video", None), ("features_fp16", None), ("raw_frames", None), ("tokens", 50000),
+                                    ("heavy_tail_bf16", 20000), ("video_dataset_shape", None)])
+def test_policy2_plans_match_the_oracle(name, n):
+    w = W.WORKLOADS[name]
+    if n:
+        w = W.scaled(w, n)
+    T = W.lengths(w)
+    for seed in (w.seed, 7):
+        G.assert_plan_equal(G.gpu_plan(T, w.t_block, seed, policy=2), O.plan(T, w.t_block, seed, policy=2))
+
+
+def test_policy2_small_and_degenerate_cases():
+    rng = np.random.default_rng(4)
+    G.full_parity(W.TOY8_LENGTHS, W.TOY8_T_BLOCK, 2, 8, policy=2)
+    G.full_parity(rng.integers(1, 60, size=700).astype(np.int32), 64, 3, 20, policy=2)
+    for T, tb in [(np.array([5], np.int32), 9), (np.full(300, 17, np.int32), 17), (np.ones(5000, np.int32), 33),
+                  (np.ones(70, np.int32), 1), (rng.integers(1, 4, size=9000).astype(np.int32), 4096),
+                  (np.concatenate([rng.integers(1, 32769, size=40), [32768, 32768, 1, 1, 1024, 1025]]).astype(np.int32), 32768),
+                  (rng.choice([3, 700], size=4097).astype(np.int32), 1000), (np.array([2, 1, 1], np.int32), 2)]:
+        for seed in (0, 11):
+            G.assert_plan_equal(G.gpu_plan(T, tb, seed, policy=2), O.plan(T, tb, seed, policy=2))
+    for n in (1, 31, 32, 33, 2049, 70001):
+        T = rng.integers(1, 301, size=n).astype(np.int32)
+        G.assert_plan_equal(G.gpu_plan(T, 300, 5, policy=2), O.plan(T, 300, 5, policy=2))
+
+
+def test_policy2_full_size_tokens():
+    w = W.WORKLOADS["tokens"]
+    T = W.lengths(w)
+    G.assert_plan_equal(G.gpu_plan(T, w.t_block, w.seed, policy=2), O.plan(T, w.t_block, w.seed, policy=2))
