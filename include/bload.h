@@ -225,6 +225,25 @@ BLOAD_API int bload_plan_static(const int32_t* d_lengths, int64_t n, int32_t t_b
                                 bload_plan_info_t* info);
 
 /*
+ * bload_rank_range -- the share of one data-parallel rank, host only.
+ *
+ * The paper's motivation (section "Problem Statement and Current Limitations"): with data-parallel
+ * training every process must run the same number of equally long iterations, or gradient
+ * synchronisation stalls without an error.  Blocks all have t_block slots, so it is enough to give
+ * every rank the same number of blocks: ranks take contiguous ranges of `per_rank` blocks, where
+ * per_rank is ceil(n_blocks / world_size) rounded up to a whole number of batches of `batch_blocks`.
+ * Ranges may reach beyond n_blocks; bload_pack writes such blocks as padding (filler) and
+ * bload_unpack ignores them, so every rank can run the same loop.  No communication is involved:
+ * each rank computes the same plan from the same seed and packs only its range.
+ *
+ * out_begin / out_count receive the rank's first block and its number of blocks (equal for all ranks).
+ * Errors: NULL outputs, n_blocks < 1, world_size < 1, rank outside [0, world_size), batch_blocks < 1,
+ * or a range that would not fit a 31-bit block index (BLOAD_ERR_ARG).
+ */
+BLOAD_API int bload_rank_range(int64_t n_blocks, int32_t world_size, int32_t rank, int32_t batch_blocks,
+                               int64_t* out_begin, int64_t* out_count);
+
+/*
  * bload_plan_stage_times -- device time, in milliseconds, that the most recent bload_plan call of
  * this thread spent in each stage: [0] validate + scan + keys, [1] key sort, [2] fill rule,
  * [3] inverse tables.  Host only; for benchmarking.  Returns BLOAD_ERR_PLAN when no plan was timed.

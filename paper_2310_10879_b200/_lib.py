@@ -17,7 +17,7 @@ ERR_NULL, ERR_ARG, ERR_LENGTH, ERR_WORKSPACE, ERR_ALIGN = -1, -2, -3, -4, -5
 ERR_UNSUPPORTED, ERR_CUDA, ERR_TIMEOUT, ERR_PLAN = -6, -7, -8, -9
 MAX_T_BLOCK = 32768
 
-EXPORTS = ("bload_plan_sizes", "bload_plan", "bload_plan_async", "bload_plan_finish", "bload_pack", "bload_unpack", "bload_stats",
+EXPORTS = ("bload_plan_sizes", "bload_plan", "bload_plan_async", "bload_plan_finish", "bload_rank_range", "bload_pack", "bload_unpack", "bload_stats",
            "bload_set_plan_timing", "bload_plan_stage_times", "bload_kernel_launches", "bload_strerror",
            "bload_version")
 
@@ -76,6 +76,7 @@ def load() -> C.CDLL:
     L.bload_plan.argtypes = [vp, i64, i32, u64, u32, vp, C.c_size_t, vp, C.c_size_t, vp, C.POINTER(PlanInfo)]
     L.bload_plan_async.argtypes = [vp, i64, i32, u64, u32, vp, C.c_size_t, vp, C.c_size_t, vp]
     L.bload_plan_finish.argtypes = [vp, vp, C.POINTER(PlanInfo)]
+    L.bload_rank_range.argtypes = [i64, i32, i32, i32, C.POINTER(i64), C.POINTER(i64)]
     L.bload_pack.argtypes = [vp, C.POINTER(PlanInfo), vp, i64, i64, i64, vp, vp, vp, vp, vp, u8, vp]
     L.bload_unpack.argtypes = [vp, C.POINTER(PlanInfo), vp, i64, i64, i64, vp, vp]
     L.bload_stats.argtypes = [C.POINTER(PlanInfo), C.POINTER(Stats)]
@@ -277,3 +278,13 @@ def bload_plan_static(lengths, t_block: int, seed: int, policy: int = 0, stream=
         err.info = info
         raise err
     return Plan(plan_buf, info, sizes)
+
+
+def bload_rank_range(n_blocks: int, world_size: int, rank: int, batch_blocks: int = 1) -> tuple[int, int]:
+    """(first block, number of blocks) of one data-parallel rank; the same count on every rank, rounded up to whole
+    batches (blocks beyond n_blocks are packed as padding)."""
+    b, c = C.c_int64(), C.c_int64()
+    rc = load().bload_rank_range(n_blocks, world_size, rank, batch_blocks, C.byref(b), C.byref(c))
+    if rc:
+        raise BloadError(rc, "bload_rank_range")
+    return int(b.value), int(c.value)

@@ -266,6 +266,20 @@ int bload_unpack(const void* d_plan, const bload_plan_info_t* info, const void* 
     return BLOAD_OK;
 }
 
+int bload_rank_range(int64_t n_blocks, int32_t world_size, int32_t rank, int32_t batch_blocks, int64_t* out_begin,
+                     int64_t* out_count)
+{
+    if (!out_begin || !out_count) return BLOAD_ERR_NULL;
+    *out_begin = 0; *out_count = 0;
+    if (n_blocks < 1 || world_size < 1 || rank < 0 || rank >= world_size || batch_blocks < 1) return BLOAD_ERR_ARG;
+    const int64_t share = (n_blocks + world_size - 1) / world_size;
+    const int64_t per_rank = (share + batch_blocks - 1) / batch_blocks * batch_blocks;
+    if (per_rank * world_size > 0x7fffffffLL) return BLOAD_ERR_ARG;
+    *out_begin = per_rank * rank;
+    *out_count = per_rank;
+    return BLOAD_OK;
+}
+
 int bload_stats(const bload_plan_info_t* info, bload_stats_t* out)
 {
     if (!info || !out) return BLOAD_ERR_NULL;

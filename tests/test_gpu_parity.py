@@ -309,3 +309,26 @@ def test_policy2_full_size_tokens():
     w = W.WORKLOADS["tokens"]
     T = W.lengths(w)
     G.assert_plan_equal(G.gpu_plan(T, w.t_block, w.seed, policy=2), O.plan(T, w.t_block, w.seed, policy=2))
+
+
+def test_rank_ranges_pack_and_unpack_like_the_whole():
+    """Three data-parallel ranks, emulated one after the other on one GPU (they share nothing and wait for nothing):
+    each packs its equal share of blocks, filler blocks included; together the shares are the whole epoch."""
+    w = W.scaled(W.WORKLOADS["features_fp16"], 500)
+    T = W.lengths(w)
+    fb, tb, world, batch = 48, w.t_block, 3, 4
+    op = O.plan(T, tb, 21)
+    plan = G.gpu_plan(T, tb, 21)
+    store = torch.randint(0, 256, (op.sum_t * fb,), dtype=torch.uint8, device=G.DEV)
+    store_h = store.cpu().numpy()
+    back = torch.full((op.sum_t * fb,), 0x5A, dtype=torch.uint8, device=G.DEV)
+    covered = 0
+    for rank in range(world):
+        b0, cnt = B.bload_rank_range(op.n_blocks, world, rank, batch)
+        res, dense = G.gpu_pack_all(plan, store, fb, b0, cnt, 0)
+        assert np.array_equal(res["dense"], O.pack(op, store_h, fb, b0, cnt, 0))
+        assert np.array_equal(res["valid"], O.metadata(op, b0, cnt)[3])
+        B.bload_unpack(plan, dense.t, fb, b0, cnt, back)
+        covered += cnt
+    torch.cuda.synchronize()
+    assert covered >= op.n_blocks and torch.equal(back, store)
