@@ -79,3 +79,33 @@ def test_async_errors_and_unfinished_buffers():
     pb, wk, s3 = B.bload_plan_async(bad, 4, 0)
     p = B.bload_plan_finish(pb, s3, check=False)
     assert p.info.status == _lib.ERR_LENGTH and p.info.first_bad_index == 1
+
+
+def test_pack_and_unpack_of_two_plans_on_two_streams_at_once():
+    """Two independent epochs handled concurrently on two streams (separate plans and buffers): the kernels keep no
+    state outside their arguments, so both results must be exact."""
+    w = W.scaled(W.WORKLOADS["features_fp16"], 600)
+    T = W.lengths(w)
+    fb = 64
+    d_len = torch.from_numpy(T).to(G.DEV)
+    jobs = []
+    for e in range(2):
+        s = torch.cuda.Stream()
+        s.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(s):
+            plan = B.bload_plan(d_len, w.t_block, 50 + e, policy=e)
+            op = O.plan(T, w.t_block, 50 + e, policy=e)
+            store = torch.randint(0, 256, (op.sum_t * fb,), dtype=torch.uint8, device=G.DEV)
+            dense = torch.empty(op.n_blocks * w.t_block * fb, dtype=torch.uint8, device=G.DEV)
+            back = torch.empty_like(store)
+        jobs.append((s, plan, op, store, dense, back))
+    for _ in range(3):                       # interleave the launches of the two streams
+        for s, plan, op, store, dense, back in jobs:
+            with torch.cuda.stream(s):
+                B.bload_pack(plan, store, fb, 0, op.n_blocks, dense=dense)
+                B.bload_unpack(plan, dense, fb, 0, op.n_blocks, back)
+    torch.cuda.synchronize()
+    for s, plan, op, store, dense, back in jobs:
+        assert np.array_equal(dense.cpu().numpy().reshape(op.n_blocks, w.t_block, fb),
+                              O.pack(op, store.cpu().numpy(), fb, 0, op.n_blocks, 0))
+        assert torch.equal(back, store)
