@@ -99,6 +99,18 @@ class ClockSampler:
                 "power_w_max": max(pw) if pw else None, "samples": len(sm), "reasons": sorted(reasons)}
 
 
+def host_memory_available() -> float:
+    """Bytes of host memory that can still be allocated (MemAvailable of /proc/meminfo; +inf if unknown)."""
+    try:
+        with open("/proc/meminfo") as f:
+            for line in f:
+                if line.startswith("MemAvailable:"):
+                    return float(line.split()[1]) * 1024.0
+    except Exception:
+        pass
+    return float("inf")
+
+
 def dist_max(x: float, device=None) -> float:
     """Maximum of a per-rank scalar over all ranks (identity without a process group)."""
     import torch
@@ -396,7 +408,10 @@ def run_gpu(args, w) -> dict:
 
     # ---- end to end through the same calls with HOST buffers (pinned), copies inside the timed region
     e2e = None
-    if not args.no_e2e:
+    e2e_need = T.size * 4 + store.numel() + dense_out.numel() + dense.numel() + 10 * nb * tb + ragged_out.numel()
+    if not args.no_e2e and host_memory_available() < 1.3 * e2e_need * max(1, int(os.environ.get("LOCAL_WORLD_SIZE", world))):
+        e2e = {"value": None, "unit": UNIT, "skipped": "not enough free host memory for the pinned buffers of all local ranks"}
+    elif not args.no_e2e:
         h_len = torch.from_numpy(T).pin_memory()
         h_store = torch.empty(store.numel(), dtype=torch.uint8, pin_memory=True); h_store.copy_(store)
         h_dense = torch.empty(dense.numel(), dtype=torch.uint8, pin_memory=True)
@@ -484,7 +499,11 @@ def run_gpu(args, w) -> dict:
                        "frac_naive_tmax": stats["frac_naive_tmax"], "frac_naive_tblock": stats["frac_naive_tblock"],
                        "reduction_vs_tmax": stats["reduction_vs_tmax"]}}
     if not args.no_cpu and world == 1:
-        cb = CpuOracleSample(w, args.ref_blocks).run()
+        blocks = args.ref_blocks
+        need = (fb + ofb) * (sum_t + nb * tb) * 1.3          # host arrays of a whole-workload sample
+        if blocks <= 0 and host_memory_available() < need:
+            blocks = max(1, int(nb * host_memory_available() / need / 1.5))
+        cb = CpuOracleSample(w, blocks).run()
         out["cpu_baseline"] = {k: v for k, v in cb.items() if not k.startswith("_")}
     else:
         out["cpu_baseline"] = None
