@@ -298,6 +298,7 @@ def run_gpu(args, w) -> dict:
     t_end.record()
     barrier()
     launches = B.bload_kernel_launches() - launches0
+    B.bload_set_plan_timing(False)   # stage events are only needed above (and they cost the end-to-end loop its copy overlap)
     seconds = dist_max(t_begin.elapsed_time(t_end) / 1e3, dev)
     clocks = sampler.stop()
 
@@ -366,7 +367,7 @@ def run_gpu(args, w) -> dict:
     bb = w.batch_blocks
     n_batches = (nb + bb - 1) // bb
     per_batch = None
-    if n_batches * bb * tb * fb <= dense.numel() + bb * tb * fb:
+    if not args.no_batch and n_batches * bb * tb * fb <= dense.numel() + bb * tb * fb:
         b_dense = torch.empty(bb * tb * fb, dtype=torch.uint8, device=dev)
         b_meta = [torch.empty(bb * tb, dtype=d, device=dev) for d in (torch.int32, torch.int32, torch.uint8, torch.uint8)]
         reps = max(1, min(n_batches, 4000))
@@ -536,6 +537,7 @@ def main():
                          "calibration run for --impl reference)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-pipeline", action="store_true")
+    ap.add_argument("--no-batch", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "bload" else args.warmup

@@ -247,7 +247,9 @@ BLOAD_API int bload_rank_range(int64_t n_blocks, int32_t world_size, int32_t ran
  * bload_plan_stage_times -- device time, in milliseconds, that the most recent bload_plan call of
  * this thread spent in each stage: [0] validate + scan + keys, [1] key sort, [2] fill rule,
  * [3] inverse tables.  Host only; for benchmarking.  Returns BLOAD_ERR_PLAN when no plan was timed.
- * Timing is enabled by bload_set_plan_timing(1) (off by default; it adds event records only).
+ * Timing is enabled by bload_set_plan_timing(1) (off by default).  It creates, records and destroys five
+ * events per plan; on the test machine that was enough to keep host<->device copies on other streams from
+ * overlapping, so switch it on only around the plans whose stages are to be timed.
  */
 BLOAD_API int bload_set_plan_timing(int enable);
 BLOAD_API int bload_plan_stage_times(float out_ms[4]);
