@@ -52,7 +52,7 @@ struct WorkView {
     uint64_t* draw_u;     // [n] random word of draw k
     int4* draw_rec;       // [n] per draw: {length, unused count of that length before the draw, block, start}
     int64_t* partial;     // [chunks] per-chunk sums of lengths
-    uint32_t* digit_hist; // [256 * chunks] per-chunk digit counts of one sort pass
+    uint32_t* digit_hist; // [256 * (chunks + 1)] per-chunk digit counts of one sort pass, then the 256 digit totals
     int32_t* bucket_end;  // [t_block + 1] sequences with length <= l
 };
 

@@ -199,18 +199,23 @@ __global__ void __launch_bounds__(256) k3_hist(const uint64_t* __restrict__ key,
     hist[(int64_t)threadIdx.x * chunks + blockIdx.x] = s_h[threadIdx.x];
 }
 
-__global__ void __launch_bounds__(1024) k3_scan(uint32_t* __restrict__ hist, int64_t total, const PlanHeader* h)
+// per digit: exclusive scan of its row of per-chunk counts (one warp per digit), row total to hist[256*chunks + d];
+// the offsets of the digits themselves (a 256-entry scan of those totals) are formed by every scatter CTA
+__global__ void __launch_bounds__(1024) k3_scan(uint32_t* __restrict__ hist, int64_t chunks, const PlanHeader* h)
 {
-    __shared__ uint32_t s_tot[32];
     if (h->first_bad != kNoBad) return;
+    const int lane = threadIdx.x & 31;
+    const int d = (int)((blockIdx.x * blockDim.x + threadIdx.x) >> 5);  // 8 CTAs x 32 warps = 256 digits
+    uint32_t* row = hist + (int64_t)d * chunks;
     uint32_t carry = 0;
-    for (int64_t lo = 0; lo < total; lo += 1024) {
-        int64_t i = lo + threadIdx.x;
-        uint32_t v = i < total ? hist[i] : 0, tot;
-        uint32_t ex = block_exclusive<uint32_t, 32>(v, s_tot, &tot);
-        if (i < total) hist[i] = carry + ex;
-        carry += tot;
+    for (int64_t lo = 0; lo < chunks; lo += 32) {
+        const int64_t i = lo + lane;
+        const uint32_t v = i < chunks ? row[i] : 0;
+        const uint32_t inc = warp_inclusive(v);
+        if (i < chunks) row[i] = carry + inc - v;
+        carry += __shfl_sync(kFull, inc, 31);
     }
+    if (lane == 0) hist[256 * chunks + d] = carry;
 }
 
 __global__ void __launch_bounds__(256) k3_scatter(const uint64_t* __restrict__ key_in, const int32_t* __restrict__ id_in,
@@ -219,6 +224,7 @@ __global__ void __launch_bounds__(256) k3_scatter(const uint64_t* __restrict__ k
                                                   const uint32_t* __restrict__ hist, const PlanHeader* h)
 {
     __shared__ uint32_t s_cnt[8][256];
+    __shared__ uint32_t s_tot[8];
     if (h->first_bad != kNoBad) return;
     const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
     for (int i = threadIdx.x; i < 8 * 256; i += 256) (&s_cnt[0][0])[i] = 0;
@@ -247,7 +253,9 @@ __global__ void __launch_bounds__(256) k3_scatter(const uint64_t* __restrict__ k
     __syncthreads();
     {
         const int d = threadIdx.x;
-        uint32_t run = hist[(int64_t)d * chunks + blockIdx.x];
+        uint32_t all;
+        const uint32_t digit_base = block_exclusive<uint32_t, 8>(hist[256 * chunks + d], s_tot, &all);  // keys with a smaller digit
+        uint32_t run = digit_base + hist[(int64_t)d * chunks + blockIdx.x];
 #pragma unroll
         for (int ww = 0; ww < 8; ++ww) {
             uint32_t c = s_cnt[ww][d];
@@ -538,7 +546,7 @@ size_t work_layout(int64_t n, int32_t t_block, void* base, WorkView* w)
     size_t o_ka = take(sizeof(uint64_t) * n), o_kb = take(sizeof(uint64_t) * n);
     size_t o_ia = take(sizeof(int32_t) * n), o_ib = take(sizeof(int32_t) * n);
     size_t o_u = take(sizeof(uint64_t) * n), o_rec = take(sizeof(int4) * n);
-    size_t o_part = take(sizeof(int64_t) * chunks), o_hist = take(sizeof(uint32_t) * 256 * chunks);
+    size_t o_part = take(sizeof(int64_t) * chunks), o_hist = take(sizeof(uint32_t) * 256 * (chunks + 1));
     size_t o_be = take(sizeof(int32_t) * ((size_t)t_block + 1));
     if (w) {
         char* b = static_cast<char*>(base);
@@ -565,7 +573,7 @@ cudaError_t plan_radix_sort(uint64_t* ka, int32_t* ia, uint64_t* kb, int32_t* ib
     for (int p = 0; p < digits; ++p) {
         const int shift = first_shift + 8 * p;
         k3_hist<<<gc, 256, 0, st>>>(kin, n, shift, chunks, hist, hdr);
-        k3_scan<<<1, 1024, 0, st>>>(hist, 256 * chunks, hdr);
+        k3_scan<<<8, 1024, 0, st>>>(hist, chunks, hdr);
         k3_scatter<<<gc, 256, 0, st>>>(kin, iin, kout, iout, n, shift, chunks, hist, hdr);
         uint64_t* tk = kin; kin = kout; kout = tk;
         int32_t* ti = iin; iin = iout; iout = ti;
@@ -604,7 +612,7 @@ cudaError_t launch_plan(const int32_t* d_lengths, int64_t n, int32_t t_block, ui
     for (int p = 0; p < passes; ++p) {
         const int shift = 8 * p;
         k3_hist<<<gc, 256, 0, st>>>(kin, n, shift, chunks, wv.digit_hist, pv.hdr);
-        k3_scan<<<1, 1024, 0, st>>>(wv.digit_hist, 256 * chunks, pv.hdr);
+        k3_scan<<<8, 1024, 0, st>>>(wv.digit_hist, chunks, pv.hdr);
         k3_scatter<<<gc, 256, 0, st>>>(kin, iin, kout, iout, n, shift, chunks, wv.digit_hist, pv.hdr);
         uint64_t* tk = kin; kin = kout; kout = tk;
         int32_t* ti = iin; iin = iout; iout = ti;
