@@ -318,7 +318,7 @@ def run_gpu(args, w) -> dict:
     # under the metadata/pack/unpack traffic of epoch e; and eight plans side by side on eight streams
     pipelined = None
     if not args.no_pipeline:
-        side = torch.cuda.Stream()
+        side = torch.cuda.Stream(priority=-1)   # the planner's small kernels go ahead of queued copy CTAs
         main = torch.cuda.current_stream()
         bufs = [torch.empty(sizes.plan_bytes, dtype=torch.uint8, device=dev) for _ in range(2)]
         work2 = torch.empty(sizes.work_bytes, dtype=torch.uint8, device=dev)

@@ -720,7 +720,10 @@ cudaError_t launch_copy(bool unpack, const PlanView& pv, int32_t t_block, int64_
     const int64_t spb = (block_bytes + sub - 1) / sub;
     const int64_t items = block_count * spb;
     const int64_t want = (items + 7) / 8;
-    const unsigned grid = (unsigned)(want < 148 * 8 ? want : 148 * 8);
+    // one sub-tile per warp, as many CTAs as that takes: measured 1 % faster than a persistent grid of 148 x 8
+    // CTAs (6.63 / 6.65 against 6.54 / 6.59 TB/s) and kinder to small kernels of other streams, which then
+    // find free slots between short-lived CTAs; the grid-stride loop only matters beyond 2^31 - 1 CTAs
+    const unsigned grid = (unsigned)(want < 0x7fffffffLL ? want : 0x7fffffffLL);
     if (unpack)
         k7_copy<true><<<grid, 256, 0, st>>>(pv, t_block, frame_bytes, block_begin, block_count, dense, ragged_out,
                                              block_count * block_bytes, sub, spb, pad_byte);
