@@ -23,6 +23,12 @@
  *   stats              closed forms; the paper's Table I "0 padding" count
  *   metadata/pack/unpack  numpy fancy-index gather built from the tables,
  *                      round trip, pad bytes
+ *   carry_prev         shifting every sequence by one frame in the ragged store and
+ *                      packing that gives the same bytes
+ *   reset_state        a running sum carried through the slots with resets equals the
+ *                      per-sequence numpy.cumsum after unpacking
+ *   valid_sum          packing per-frame integers and summing the frames equals the sum
+ *                      over the ragged array (exact in double)
  *   Parity unpinned: the paper's "block_pad" padding count of Table I (block
  *   length of that run is not stated and the rule is random) and its
  *   time-per-epoch figures.
@@ -364,6 +370,79 @@ int oracle_unpack(const oracle_tables_t *t, const uint8_t *dense_out, int64_t fr
                    dense_out + ((size_t)q * (size_t)t->t_block + (size_t)s) * (size_t)frame_bytes, (size_t)frame_bytes);
         }
     }
+    free(sid); free(ps); free(rs); free(vd);
+    return ORACLE_OK;
+}
+
+/* ------------------------------------------------------------------------ */
+/* Consumer side of the start table (Methods, second paragraph): a recurrent  */
+/* model feeds information of frame t-1 into frame t and must discard it       */
+/* wherever a new sequence starts inside a block.                              */
+/* ------------------------------------------------------------------------ */
+
+/* prev[q, s, :] = dense[q, s-1, :] where slot s holds frame f >= 1 of a sequence (the frame before
+ * it belongs to the same sequence); fill_byte where it holds a first frame, padding, or the block
+ * is filler.  This is "what frame t receives from frame t-1" for a whole batch at once. */
+int oracle_carry_prev(const oracle_tables_t *t, const uint8_t *dense, int64_t frame_bytes,
+                      int64_t block_begin, int64_t block_count, uint8_t *prev, uint8_t fill_byte)
+{
+    if (block_begin < 0 || block_count < 0 || frame_bytes < 1) return ORACLE_ERR_ARG;
+    int32_t *sid = (int32_t *)malloc(sizeof(int32_t) * (size_t)t->t_block);
+    int32_t *ps = (int32_t *)malloc(sizeof(int32_t) * (size_t)t->t_block);
+    uint8_t *rs = (uint8_t *)malloc((size_t)t->t_block), *vd = (uint8_t *)malloc((size_t)t->t_block);
+    if (!sid || !ps || !rs || !vd) { free(sid); free(ps); free(rs); free(vd); return ORACLE_ERR_NOMEM; }
+    for (int64_t q = 0; q < block_count; ++q) {
+        oracle_metadata(t, block_begin + q, 1, sid, ps, rs, vd);
+        for (int32_t s = 0; s < t->t_block; ++s) {
+            size_t at = ((size_t)q * (size_t)t->t_block + (size_t)s) * (size_t)frame_bytes;
+            if (vd[s] && !rs[s]) memcpy(prev + at, dense + at - (size_t)frame_bytes, (size_t)frame_bytes);
+            else memset(prev + at, fill_byte, (size_t)frame_bytes);
+        }
+    }
+    free(sid); free(ps); free(rs); free(vd);
+    return ORACLE_OK;
+}
+
+/* One step of a recurrence that walks the slots of a batch in order: before slot `slot` is
+ * processed, row q of the carried state is replaced by `init` (zeros when init is NULL) unless a
+ * sequence continues at that slot, i.e. on a first frame, on padding and in filler blocks.
+ * Rows whose sequence continues are left as they are. */
+int oracle_reset_state(const oracle_tables_t *t, int64_t block_begin, int64_t block_count, int32_t slot,
+                       uint8_t *state, int64_t state_bytes, const uint8_t *init)
+{
+    if (block_begin < 0 || block_count < 0 || state_bytes < 1 || slot < 0 || slot >= t->t_block) return ORACLE_ERR_ARG;
+    int32_t *sid = (int32_t *)malloc(sizeof(int32_t) * (size_t)t->t_block);
+    int32_t *ps = (int32_t *)malloc(sizeof(int32_t) * (size_t)t->t_block);
+    uint8_t *rs = (uint8_t *)malloc((size_t)t->t_block), *vd = (uint8_t *)malloc((size_t)t->t_block);
+    if (!sid || !ps || !rs || !vd) { free(sid); free(ps); free(rs); free(vd); return ORACLE_ERR_NOMEM; }
+    for (int64_t q = 0; q < block_count; ++q) {
+        oracle_metadata(t, block_begin + q, 1, sid, ps, rs, vd);
+        if (vd[slot] && !rs[slot]) continue;
+        if (init) memcpy(state + (size_t)q * (size_t)state_bytes, init, (size_t)state_bytes);
+        else memset(state + (size_t)q * (size_t)state_bytes, 0, (size_t)state_bytes);
+    }
+    free(sid); free(ps); free(rs); free(vd);
+    return ORACLE_OK;
+}
+
+/* Sum (in double precision, slot order) and count of per-slot float values over the frames of the
+ * given blocks; padding and filler blocks contribute nothing (a loss must not see them). */
+int oracle_valid_sum(const oracle_tables_t *t, int64_t block_begin, int64_t block_count, const float *values,
+                     double *sum, int64_t *count)
+{
+    if (block_begin < 0 || block_count < 0) return ORACLE_ERR_ARG;
+    int32_t *sid = (int32_t *)malloc(sizeof(int32_t) * (size_t)t->t_block);
+    int32_t *ps = (int32_t *)malloc(sizeof(int32_t) * (size_t)t->t_block);
+    uint8_t *rs = (uint8_t *)malloc((size_t)t->t_block), *vd = (uint8_t *)malloc((size_t)t->t_block);
+    if (!sid || !ps || !rs || !vd) { free(sid); free(ps); free(rs); free(vd); return ORACLE_ERR_NOMEM; }
+    double acc = 0.0;
+    int64_t cnt = 0;
+    for (int64_t q = 0; q < block_count; ++q) {
+        oracle_metadata(t, block_begin + q, 1, sid, ps, rs, vd);
+        for (int32_t s = 0; s < t->t_block; ++s)
+            if (vd[s]) { acc += (double)values[(size_t)q * (size_t)t->t_block + (size_t)s]; ++cnt; }
+    }
+    *sum = acc; *count = cnt;
     free(sid); free(ps); free(rs); free(vd);
     return ORACLE_OK;
 }

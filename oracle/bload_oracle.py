@@ -80,6 +80,15 @@ def lib():
         L.oracle_unpack.argtypes = [C.POINTER(_TablesStruct), C.c_void_p, C.c_int64, C.c_int64, C.c_int64,
                                     C.c_void_p]
         L.oracle_unpack.restype = C.c_int
+        L.oracle_carry_prev.argtypes = [C.POINTER(_TablesStruct), C.c_void_p, C.c_int64, C.c_int64, C.c_int64,
+                                        C.c_void_p, C.c_uint8]
+        L.oracle_carry_prev.restype = C.c_int
+        L.oracle_reset_state.argtypes = [C.POINTER(_TablesStruct), C.c_int64, C.c_int64, C.c_int32, C.c_void_p,
+                                         C.c_int64, C.c_void_p]
+        L.oracle_reset_state.restype = C.c_int
+        L.oracle_valid_sum.argtypes = [C.POINTER(_TablesStruct), C.c_int64, C.c_int64, C.c_void_p,
+                                       C.POINTER(C.c_double), C.POINTER(C.c_int64)]
+        L.oracle_valid_sum.restype = C.c_int
         L.oracle_stats.argtypes = [C.POINTER(_StatsStruct)]
         L.oracle_stats.restype = C.c_int
         _lib = L
@@ -197,6 +206,45 @@ def unpack(p: OraclePlan, dense_out: np.ndarray, frame_bytes: int, block_begin: 
     rc = lib().oracle_unpack(C.byref(t), _p(dense_out), frame_bytes, block_begin, block_count, _p(ragged_out))
     assert rc == 0, rc
     return ragged_out
+
+
+def carry_prev(p: OraclePlan, dense: np.ndarray, frame_bytes: int, block_begin: int, block_count: int,
+               fill_byte: int = 0) -> np.ndarray:
+    """What every slot receives from the slot before it: the previous frame of the same sequence, or fill."""
+    dense = np.ascontiguousarray(dense).view(np.uint8).reshape(-1)
+    assert dense.size == block_count * p.t_block * frame_bytes
+    prev = np.empty((block_count, p.t_block, frame_bytes), np.uint8)
+    t = p._tables()
+    rc = lib().oracle_carry_prev(C.byref(t), _p(dense), frame_bytes, block_begin, block_count, _p(prev), fill_byte)
+    assert rc == 0, rc
+    return prev
+
+
+def reset_state(p: OraclePlan, block_begin: int, block_count: int, slot: int, state: np.ndarray,
+                init: np.ndarray | None = None) -> np.ndarray:
+    """In place: rows of `state` ([block_count, state_bytes] uint8) whose block starts a sequence, or has no frame,
+    at `slot` are replaced by `init` (zeros when None)."""
+    assert state.dtype == np.uint8 and state.flags.c_contiguous and state.shape[0] == block_count
+    sb = state.size // max(block_count, 1)
+    if init is not None:
+        init = np.ascontiguousarray(init).view(np.uint8).reshape(-1)
+        assert init.size == sb
+    t = p._tables()
+    rc = lib().oracle_reset_state(C.byref(t), block_begin, block_count, slot, _p(state), sb,
+                                  _p(init) if init is not None else None)
+    assert rc == 0, rc
+    return state
+
+
+def valid_sum(p: OraclePlan, block_begin: int, block_count: int, values: np.ndarray) -> tuple[float, int]:
+    """(sum in double precision, number) of the float32 per-slot values that sit on frames."""
+    values = np.ascontiguousarray(values, dtype=np.float32).reshape(-1)
+    assert values.size == block_count * p.t_block
+    s, c = C.c_double(), C.c_int64()
+    t = p._tables()
+    rc = lib().oracle_valid_sum(C.byref(t), block_begin, block_count, _p(values), C.byref(s), C.byref(c))
+    assert rc == 0, rc
+    return float(s.value), int(c.value)
 
 
 def stats(n: int, sum_t: int, t_max: int, t_block: int, n_blocks: int) -> dict:
