@@ -183,6 +183,59 @@ BLOAD_API int bload_unpack(const void* d_plan, const bload_plan_info_t* info, co
                  void* stream);
 
 /*
+ * Consumer side of the start table (paper, Methods, second paragraph, and its figure of the DDS
+ * architecture): a recurrent model feeds information of frame t-1 into frame t, and the table of
+ * start indices tells it where that information belongs to another sequence and has to be
+ * discarded.  The three calls below apply the table on the GPU, straight from the plan.
+ *
+ * bload_carry_prev -- what every slot receives from the slot before it, for a whole batch at once:
+ *
+ *   d_prev[q, s, :] = d_dense[q, s-1, :]   if slot s of block block_begin+q holds frame f >= 1 of a
+ *                                          sequence (slot s-1 then holds frame f-1 of the same one)
+ *                   = fill_byte repeated   on the first frame of every sequence, on padding and in
+ *                                          filler blocks (nothing is carried over there)
+ *
+ * d_dense and d_prev are [block_count, t_block, frame_bytes] row major, 16-byte aligned, and must
+ * not be the same buffer (ARG) nor overlap.  Frames are opaque bytes.  Asynchronous on `stream`.
+ * Errors as for bload_pack.
+ */
+BLOAD_API int bload_carry_prev(const void* d_plan, const bload_plan_info_t* info, const void* d_dense,
+                               int64_t frame_bytes, int64_t block_begin, int64_t block_count, void* d_prev,
+                               uint8_t fill_byte, void* stream);
+
+/*
+ * bload_reset_state -- one step of a recurrence that walks the slots of a batch in order.  Call it
+ * before slot `slot` is processed: row q of the carried state (d_state, [block_count, state_bytes]
+ * row major, opaque bytes) is overwritten with the initial state unless a sequence continues at that
+ * slot of block block_begin+q, that is, on the first frame of a sequence, on padding and in filler
+ * blocks.  Rows whose sequence continues are not touched.  d_init points to state_bytes bytes of
+ * initial state (device, 16-byte aligned) or is NULL for zeros.  Asynchronous on `stream`.
+ * Errors: NULL plan/info/state, ARG (state_bytes < 1, slot outside [0, t_block), bad range), ALIGN,
+ * PLAN, CUDA.
+ */
+BLOAD_API int bload_reset_state(const void* d_plan, const bload_plan_info_t* info, int64_t block_begin,
+                                int64_t block_count, int32_t slot, void* d_state, int64_t state_bytes,
+                                const void* d_init, void* stream);
+
+/*
+ * bload_valid_sum -- masked reduction of per-slot values (a per-frame loss, say): padding slots and
+ * filler blocks hold no frame and must not count.
+ *
+ *   d_block_sum[q] = sum over the frames s of block block_begin+q of d_values[q, s]      (double)
+ *   d_total[0]     = sum over q of d_block_sum[q];  d_total[1] = number of frames in the range
+ *
+ * d_values is float32 [block_count, t_block] (4-byte aligned; 16-byte aligned rows are read as
+ * vectors); d_block_sum is double[block_count]; d_total is double[2] or NULL (skipped).  Sums are
+ * accumulated in double precision in a fixed order, so repeated calls give identical bits; against a
+ * sum taken in another order the difference is bounded by block rounding, about 1e-15 of the sum of
+ * magnitudes.  A mean over frames is d_total[0] / d_total[1].  Asynchronous on `stream`.
+ * Errors: NULL plan/info/values/block_sum, ARG (bad range), ALIGN, PLAN, CUDA.
+ */
+BLOAD_API int bload_valid_sum(const void* d_plan, const bload_plan_info_t* info, const float* d_values,
+                              int64_t block_begin, int64_t block_count, double* d_block_sum, double* d_total,
+                              void* stream);
+
+/*
  * bload_stats -- padding statistics from the scalars of a plan (host only; closed forms).
  * pad_naive_tmax is the "0 padding" row of the paper's Table I, pad_packed its "block_pad" row.
  */

@@ -18,6 +18,7 @@ ERR_UNSUPPORTED, ERR_CUDA, ERR_TIMEOUT, ERR_PLAN = -6, -7, -8, -9
 MAX_T_BLOCK = 32768
 
 EXPORTS = ("bload_plan_sizes", "bload_plan", "bload_plan_async", "bload_plan_finish", "bload_rank_range", "bload_pack", "bload_unpack", "bload_stats",
+           "bload_carry_prev", "bload_reset_state", "bload_valid_sum",
            "bload_set_plan_timing", "bload_plan_stage_times", "bload_kernel_launches", "bload_strerror",
            "bload_version")
 
@@ -80,6 +81,9 @@ def load() -> C.CDLL:
     L.bload_pack.argtypes = [vp, C.POINTER(PlanInfo), vp, i64, i64, i64, vp, vp, vp, vp, vp, u8, vp]
     L.bload_unpack.argtypes = [vp, C.POINTER(PlanInfo), vp, i64, i64, i64, vp, vp]
     L.bload_stats.argtypes = [C.POINTER(PlanInfo), C.POINTER(Stats)]
+    L.bload_carry_prev.argtypes = [vp, C.POINTER(PlanInfo), vp, i64, i64, i64, vp, u8, vp]
+    L.bload_reset_state.argtypes = [vp, C.POINTER(PlanInfo), i64, i64, i32, vp, i64, vp, vp]
+    L.bload_valid_sum.argtypes = [vp, C.POINTER(PlanInfo), vp, i64, i64, vp, vp, vp]
     L.bload_set_plan_timing.argtypes = [C.c_int]
     L.bload_plan_stage_times.argtypes = [C.POINTER(C.c_float * 4)]
     L.bload_strerror.argtypes = [C.c_int]
@@ -222,6 +226,33 @@ def bload_unpack(plan: Plan, dense_out, out_frame_bytes: int, block_begin: int, 
                              block_count, _ptr(ragged_out), _stream(stream))
     if rc:
         raise BloadError(rc, "bload_unpack")
+
+
+def bload_carry_prev(plan: Plan, dense, frame_bytes: int, block_begin: int, block_count: int, prev,
+                     fill_byte: int = 0, stream=None) -> None:
+    """prev[q, s] = dense[q, s-1] where a sequence continues at slot s, fill_byte elsewhere (CUDA tensors)."""
+    rc = load().bload_carry_prev(plan.buf.data_ptr(), C.byref(plan.info), _ptr(dense), frame_bytes, block_begin,
+                                 block_count, _ptr(prev), fill_byte, _stream(stream))
+    if rc:
+        raise BloadError(rc, "bload_carry_prev")
+
+
+def bload_reset_state(plan: Plan, block_begin: int, block_count: int, slot: int, state, state_bytes: int,
+                      init=None, stream=None) -> None:
+    """Re-initialise, in place, the rows of `state` whose block does not continue a sequence at `slot`."""
+    rc = load().bload_reset_state(plan.buf.data_ptr(), C.byref(plan.info), block_begin, block_count, slot,
+                                  _ptr(state), state_bytes, _ptr(init), _stream(stream))
+    if rc:
+        raise BloadError(rc, "bload_reset_state")
+
+
+def bload_valid_sum(plan: Plan, values, block_begin: int, block_count: int, block_sum, total=None,
+                    stream=None) -> None:
+    """block_sum[q] (float64 CUDA tensor) = sum of the float32 values on the frames of block q; total = [sum, frames]."""
+    rc = load().bload_valid_sum(plan.buf.data_ptr(), C.byref(plan.info), _ptr(values), block_begin, block_count,
+                                _ptr(block_sum), _ptr(total), _stream(stream))
+    if rc:
+        raise BloadError(rc, "bload_valid_sum")
 
 
 def bload_stats(info: PlanInfo) -> dict:

@@ -266,6 +266,59 @@ int bload_unpack(const void* d_plan, const bload_plan_info_t* info, const void* 
     return BLOAD_OK;
 }
 
+int bload_carry_prev(const void* d_plan, const bload_plan_info_t* info, const void* d_dense, int64_t frame_bytes,
+                     int64_t block_begin, int64_t block_count, void* d_prev, uint8_t fill_byte, void* stream)
+{
+    int rc = check_plan_args(d_plan, info, frame_bytes, block_begin, block_count);
+    if (rc) return rc;
+    if (block_count == 0) return BLOAD_OK;
+    if (!d_dense || !d_prev) return BLOAD_ERR_NULL;
+    if (d_dense == d_prev) return BLOAD_ERR_ARG;
+    if (!aligned(d_dense, 16) || !aligned(d_prev, 16)) return BLOAD_ERR_ALIGN;
+    cudaError_t ce = launch_carry_prev(plan_view(const_cast<void*>(d_plan), info->n), info->t_block, frame_bytes,
+                                       block_begin, block_count, static_cast<const uint8_t*>(d_dense),
+                                       static_cast<uint8_t*>(d_prev), fill_byte, static_cast<cudaStream_t>(stream));
+    if (ce != cudaSuccess) { (void)cudaGetLastError(); return BLOAD_ERR_CUDA; }
+    return BLOAD_OK;
+}
+
+int bload_reset_state(const void* d_plan, const bload_plan_info_t* info, int64_t block_begin, int64_t block_count,
+                      int32_t slot, void* d_state, int64_t state_bytes, const void* d_init, void* stream)
+{
+    int rc = check_plan_args(d_plan, info, state_bytes, block_begin, block_count);
+    if (rc) return rc;
+    if (slot < 0 || slot >= info->t_block) return BLOAD_ERR_ARG;
+    if (block_count == 0) return BLOAD_OK;
+    if (!d_state) return BLOAD_ERR_NULL;
+    if (!aligned(d_init, 16)) return BLOAD_ERR_ALIGN;
+    cudaError_t ce = launch_reset_state(plan_view(const_cast<void*>(d_plan), info->n), block_begin, block_count, slot,
+                                        static_cast<uint8_t*>(d_state), state_bytes, static_cast<const uint8_t*>(d_init),
+                                        static_cast<cudaStream_t>(stream));
+    if (ce != cudaSuccess) { (void)cudaGetLastError(); return BLOAD_ERR_CUDA; }
+    return BLOAD_OK;
+}
+
+int bload_valid_sum(const void* d_plan, const bload_plan_info_t* info, const float* d_values, int64_t block_begin,
+                    int64_t block_count, double* d_block_sum, double* d_total, void* stream)
+{
+    int rc = check_plan_args(d_plan, info, 1, block_begin, block_count);
+    if (rc) return rc;
+    if (!d_values || !d_block_sum) return BLOAD_ERR_NULL;
+    if (!aligned(d_values, 4) || !aligned(d_block_sum, 8) || !aligned(d_total, 8)) return BLOAD_ERR_ALIGN;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (block_count == 0) {  // an empty range sums to zero over zero frames
+        if (d_total && cudaMemsetAsync(d_total, 0, 2 * sizeof(double), st) != cudaSuccess) {
+            (void)cudaGetLastError();
+            return BLOAD_ERR_CUDA;
+        }
+        return BLOAD_OK;
+    }
+    cudaError_t ce = launch_valid_sum(plan_view(const_cast<void*>(d_plan), info->n), info->t_block, block_begin, block_count,
+                                      d_values, d_block_sum, d_total, st);
+    if (ce != cudaSuccess) { (void)cudaGetLastError(); return BLOAD_ERR_CUDA; }
+    return BLOAD_OK;
+}
+
 int bload_rank_range(int64_t n_blocks, int32_t world_size, int32_t rank, int32_t batch_blocks, int64_t* out_begin,
                      int64_t* out_count)
 {

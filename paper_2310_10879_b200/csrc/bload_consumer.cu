@@ -1,0 +1,202 @@
+// Consumer side of the start table (paper, Methods, second paragraph): a recurrent model hands
+// information of frame t-1 to frame t and has to discard it wherever a new sequence starts inside a
+// block.  Three kernels use the plan's segment list for that, without per-slot metadata:
+//   k11_carry_prev   prev[q, s, :] = dense[q, s-1, :] where a sequence continues at slot s, a fill byte
+//                    elsewhere: one shifted, segmented memcpy over the whole batch (HBM bound);
+//   k12_reset_state  one step of a slot-by-slot recurrence: rows of the carried state whose block does
+//                    not continue a sequence at the given slot are re-initialised;
+//   k13_valid_sum    per-block sums of per-slot float values over frames only (padding masked out),
+//                    in double precision and in a fixed order, plus their total.
+#include "bload_internal.cuh"
+#include "bload_warp_copy.cuh"
+
+namespace bload {
+
+namespace {
+
+using namespace wc;
+
+// Same decomposition as the pack kernel: the output is cut into sub-tiles of `sub_bytes`, a warp owns one.
+// Inside a segment that occupies bytes [seg_b, seg_e) of its block, the first frame receives the fill byte and
+// every later byte x receives dense[x - frame_bytes]; everything behind the last segment is fill.
+__global__ void __launch_bounds__(256, 3) k11_carry_prev(PlanView pv, int32_t t_block, int64_t frame_bytes, int64_t block_begin,
+                                                      int64_t block_count, const uint8_t* __restrict__ dense,
+                                                      uint8_t* __restrict__ prev, int64_t sub_bytes, int64_t subs_per_block,
+                                                      uint8_t fill_byte)
+{
+    const int lane = threadIdx.x & 31;
+    const int64_t warps = ((int64_t)gridDim.x * blockDim.x) >> 5;
+    const int64_t items = block_count * subs_per_block;
+    const int64_t block_bytes = (int64_t)t_block * frame_bytes;
+    const int64_t n_blocks = pv.hdr->n_blocks;
+    const uint8_t* s_limit = dense + block_count * block_bytes;
+
+    for (int64_t item = (((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5); item < items; item += warps) {
+        const int64_t q = item / subs_per_block;
+        const int64_t lo = (item - q * subs_per_block) * sub_bytes;
+        const int64_t hi = min(lo + sub_bytes, block_bytes);
+        const int64_t b = block_begin + q;
+        const int64_t dense_off = q * block_bytes;
+        int64_t cur = lo;
+        if (b < n_blocks) {
+            const int k0 = pv.block_seg_begin[b], k1 = pv.block_seg_begin[b + 1];
+            const int fill = pv.block_fill[b];
+            if (cur < (int64_t)fill * frame_bytes) {
+                int k = warp_find_segment(pv.seg_start, k0, k1, (int)(cur / frame_bytes), lane);
+                int kw = k;  // lanes hold the start slots of segments kw .. kw+31
+                int w_st = (kw + lane < k1) ? pv.seg_start[kw + lane] : fill;
+                while (cur < hi && k < k1) {
+                    if (k - kw == 31) {
+                        kw = k;
+                        w_st = (kw + lane < k1) ? pv.seg_start[kw + lane] : fill;
+                    }
+                    const int st = __shfl_sync(kFull, w_st, k - kw);
+                    const int nx = __shfl_sync(kFull, w_st, k - kw + 1);
+                    const int64_t first_e = min(((int64_t)st + 1) * frame_bytes, hi);  // end of the first frame
+                    const int64_t seg_e = min((int64_t)nx * frame_bytes, hi);
+                    if (cur < first_e) {
+                        warp_fill(prev + dense_off + cur, first_e - cur, fill_byte, lane);
+                        cur = first_e;
+                    }
+                    if (cur < seg_e) {
+                        warp_copy<true>(prev + dense_off + cur, dense + dense_off + cur - frame_bytes, seg_e - cur, s_limit, lane);
+                        cur = seg_e;
+                    }
+                    ++k;
+                }
+            }
+        }
+        if (cur < hi) warp_fill(prev + dense_off + cur, hi - cur, fill_byte, lane);
+    }
+}
+
+// A warp owns `sub_bytes` of one row of the state.  It decides from the plan whether a sequence continues at
+// `slot` of the row's block (then the row is left alone) and otherwise writes the initial state over its part.
+__global__ void __launch_bounds__(256) k12_reset_state(PlanView pv, int64_t block_begin, int64_t block_count, int32_t slot,
+                                                       uint8_t* __restrict__ state, int64_t state_bytes,
+                                                       const uint8_t* __restrict__ init, int64_t sub_bytes,
+                                                       int64_t subs_per_row)
+{
+    const int lane = threadIdx.x & 31;
+    const int64_t warps = ((int64_t)gridDim.x * blockDim.x) >> 5;
+    const int64_t items = block_count * subs_per_row;
+    const int64_t n_blocks = pv.hdr->n_blocks;
+    for (int64_t item = (((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5); item < items; item += warps) {
+        const int64_t q = item / subs_per_row;
+        const int64_t lo = (item - q * subs_per_row) * sub_bytes;
+        const int64_t hi = min(lo + sub_bytes, state_bytes);
+        const int64_t b = block_begin + q;
+        bool continues = false;
+        if (b < n_blocks && slot < pv.block_fill[b]) {
+            const int k = warp_find_segment(pv.seg_start, pv.block_seg_begin[b], pv.block_seg_begin[b + 1], slot, lane);
+            continues = pv.seg_start[k] != slot;
+        }
+        if (continues) continue;
+        uint8_t* d = state + q * state_bytes + lo;
+        if (init) warp_copy<true>(d, init + lo, hi - lo, init + state_bytes, lane);
+        else warp_fill(d, hi - lo, 0, lane);
+    }
+}
+
+constexpr int kSumThreads = 256;
+
+// Fixed-order sum of one double per thread over a CTA of kSumThreads threads; the result is valid in thread 0.
+__device__ __forceinline__ double cta_sum(double v, double* sh)
+{
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) v += __shfl_down_sync(kFull, v, d);
+    if ((threadIdx.x & 31) == 0) sh[threadIdx.x >> 5] = v;
+    __syncthreads();
+    double t = 0.0;
+    if (threadIdx.x == 0)
+        for (int w = 0; w < kSumThreads / 32; ++w) t += sh[w];
+    __syncthreads();
+    return t;
+}
+
+// One CTA per block: the frames of a block are its first block_fill slots, so the mask needs no segment search.
+__global__ void __launch_bounds__(kSumThreads) k13_valid_sum(PlanView pv, int32_t t_block, int64_t block_begin,
+                                                             const float* __restrict__ values,
+                                                             double* __restrict__ block_sum)
+{
+    __shared__ double sh[kSumThreads / 32];
+    const int64_t q = blockIdx.x;
+    const int64_t b = block_begin + q;
+    const int fill = b < pv.hdr->n_blocks ? pv.block_fill[b] : 0;
+    const float* row = values + q * (int64_t)t_block;
+    double acc = 0.0;
+    if ((reinterpret_cast<uintptr_t>(row) & 15u) == 0) {
+        const int nv = fill >> 2;
+        const float4* r4 = reinterpret_cast<const float4*>(row);
+        for (int i = threadIdx.x; i < nv; i += kSumThreads) {
+            const float4 v = __ldcs(r4 + i);
+            acc += ((double)v.x + (double)v.y) + ((double)v.z + (double)v.w);
+        }
+        for (int i = (nv << 2) + threadIdx.x; i < fill; i += kSumThreads) acc += (double)row[i];
+    } else {
+        for (int i = threadIdx.x; i < fill; i += kSumThreads) acc += (double)row[i];
+    }
+    const double t = cta_sum(acc, sh);
+    if (threadIdx.x == 0) block_sum[q] = t;
+}
+
+// total[0] = sum of the block sums, total[1] = number of frames in the range; one CTA, fixed order.
+__global__ void __launch_bounds__(kSumThreads) k13_total(PlanView pv, int64_t block_begin, int64_t block_count,
+                                                         const double* __restrict__ block_sum, double* __restrict__ total)
+{
+    __shared__ double sh[kSumThreads / 32];
+    const int64_t n_blocks = pv.hdr->n_blocks;
+    double s = 0.0, c = 0.0;
+    for (int64_t q = threadIdx.x; q < block_count; q += kSumThreads) {
+        s += block_sum[q];
+        if (block_begin + q < n_blocks) c += (double)pv.block_fill[block_begin + q];
+    }
+    const double ts = cta_sum(s, sh);
+    const double tc = cta_sum(c, sh);
+    if (threadIdx.x == 0) { total[0] = ts; total[1] = tc; }
+}
+
+unsigned grid_for_items(int64_t items)
+{
+    const int64_t want = (items + 7) / 8;  // CTAs of 8 warps, one item per warp
+    return (unsigned)(want < 0x7fffffffLL ? want : 0x7fffffffLL);
+}
+
+}  // namespace
+
+cudaError_t launch_carry_prev(const PlanView& pv, int32_t t_block, int64_t frame_bytes, int64_t block_begin,
+                              int64_t block_count, const uint8_t* dense, uint8_t* prev, uint8_t fill_byte, cudaStream_t st)
+{
+    if (block_count == 0) return cudaSuccess;
+    const int64_t block_bytes = (int64_t)t_block * frame_bytes;
+    const int64_t sub = 16384;
+    const int64_t spb = (block_bytes + sub - 1) / sub;
+    count_launches(1);
+    k11_carry_prev<<<grid_for_items(block_count * spb), 256, 0, st>>>(pv, t_block, frame_bytes, block_begin, block_count,
+                                                                     dense, prev, sub, spb, fill_byte);
+    return cudaPeekAtLastError();
+}
+
+cudaError_t launch_reset_state(const PlanView& pv, int64_t block_begin, int64_t block_count, int32_t slot, uint8_t* state,
+                               int64_t state_bytes, const uint8_t* init, cudaStream_t st)
+{
+    if (block_count == 0) return cudaSuccess;
+    const int64_t sub = 16384;
+    const int64_t spr = (state_bytes + sub - 1) / sub;
+    count_launches(1);
+    k12_reset_state<<<grid_for_items(block_count * spr), 256, 0, st>>>(pv, block_begin, block_count, slot, state, state_bytes,
+                                                                      init, sub, spr);
+    return cudaPeekAtLastError();
+}
+
+cudaError_t launch_valid_sum(const PlanView& pv, int32_t t_block, int64_t block_begin, int64_t block_count,
+                             const float* values, double* block_sum, double* total, cudaStream_t st)
+{
+    if (block_count == 0) return cudaSuccess;
+    count_launches(total ? 2 : 1);
+    k13_valid_sum<<<(unsigned)block_count, kSumThreads, 0, st>>>(pv, t_block, block_begin, values, block_sum);
+    if (total) k13_total<<<1, kSumThreads, 0, st>>>(pv, block_begin, block_count, block_sum, total);
+    return cudaPeekAtLastError();
+}
+
+}  // namespace bload
