@@ -412,6 +412,41 @@ def run_gpu(args, w) -> dict:
             per_batch["graph_error"] = str(exc)[:200]
         del b_dense, b_meta
 
+    # ---- consumer side of the start table (not part of the step): the shifted copy over the whole epoch, the
+    # masked sum of a per-slot loss, and the per-slot state reset of a batch
+    consumer = None
+    if not args.no_consumer:
+        def timed(fn, reps):
+            for _ in range(3):
+                fn()
+            torch.cuda.synchronize()
+            a, b_ = ev(), ev()
+            a.record()
+            for _ in range(reps):
+                fn()
+            b_.record()
+            torch.cuda.synchronize()
+            return a.elapsed_time(b_) / reps
+        prev = torch.empty_like(dense)
+        ms = timed(lambda: B.bload_carry_prev(plan, dense, fb, 0, nb, prev), 20)
+        cp_bytes = (sum_t - T.size) * fb + nb * tb * fb
+        del prev
+        vals = torch.empty(nb * tb, dtype=torch.float32, device=dev).normal_()
+        bsum = torch.empty(nb, dtype=torch.float64, device=dev)
+        tot = torch.empty(2, dtype=torch.float64, device=dev)
+        ms_sum = timed(lambda: B.bload_valid_sum(plan, vals, 0, nb, bsum, tot), 20)
+        bb = min(w.batch_blocks, nb)
+        state = torch.zeros(bb * 4096, dtype=torch.uint8, device=dev)
+        ms_reset = timed(lambda: B.bload_reset_state(plan, 0, bb, tb // 2, state, 4096), 200)
+        consumer = {"carry_prev": {"ms": ms, "GB/s": cp_bytes / ms / 1e6, "algorithmic_bytes": cp_bytes,
+                                   "what": "prev[q,s] = dense[q,s-1] inside sequences, fill elsewhere, all blocks; "
+                                           "bytes = (sum_t - n) frames read + n_blocks*t_block frames written"},
+                    "valid_sum": {"ms": ms_sum, "GB/s": 4 * sum_t / ms_sum / 1e6, "slots": nb * tb,
+                                  "what": "fp32 per-slot values, frames only, per-block and total sums in double; "
+                                          "bytes = 4 per frame read"},
+                    "reset_state": {"us_per_call": ms_reset * 1e3, "batch_blocks": bb, "state_bytes": 4096}}
+        del vals, bsum, tot, state
+
     # ---- end to end through the same calls with HOST buffers (pinned), copies inside the timed region
     e2e = None
     e2e_need = T.size * 4 + store.numel() + dense_out.numel() + dense.numel() + 10 * nb * tb + ragged_out.numel()
@@ -489,7 +524,7 @@ def run_gpu(args, w) -> dict:
            "ms_per_step": step_s * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
            "dtype": "u8", "data": "synthetic", "config": config_of(w, {"parallelism": "replicas only"}),
            "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline,
-           "frames_per_s": aggregate(sum_t, world, step_s), "per_batch_pack": per_batch, "pipelined": pipelined,
+           "frames_per_s": aggregate(sum_t, world, step_s), "per_batch_pack": per_batch, "pipelined": pipelined, "consumer": consumer,
            "kernels": {
                "pack_copy": {"ms": pack_ms, "GB/s": by["pack"] / pack_ms / 1e6, "frac_measured": by["pack"] / pack_ms / 1e6 / peak,
                              "frac_nominal": by["pack"] / pack_ms / 1e6 / NOMINAL_HBM_GBS, "frames_per_s": sum_t / pack_ms * 1e3},
@@ -544,6 +579,7 @@ def main():
     ap.add_argument("--no-pipeline", action="store_true")
     ap.add_argument("--no-batch", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--no-consumer", action="store_true")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "bload" else args.warmup
 
