@@ -23,6 +23,8 @@
  *   stats              closed forms; the paper's Table I "0 padding" count
  *   metadata/pack/unpack  numpy fancy-index gather built from the tables,
  *                      round trip, pad bytes
+ *   pack_repeat_last   numpy gather with pad slots mapped to the block's last frame; with one
+ *                      sequence per block, the paper's naive repeat-last padding of each sample
  *   carry_prev         shifting every sequence by one frame in the ragged store and
  *                      packing that gives the same bytes
  *   reset_state        a running sum carried through the slots with resets equals the
@@ -348,6 +350,31 @@ int oracle_pack(const oracle_tables_t *t, const uint8_t *store, int64_t frame_by
             if (vd[s]) memcpy(dst, store + (size_t)(t->offsets[sid[s]] + ps[s]) * (size_t)frame_bytes, (size_t)frame_bytes);
             else memset(dst, pad_byte, (size_t)frame_bytes);
         }
+    }
+    free(sid); free(ps); free(rs); free(vd);
+    return ORACLE_OK;
+}
+
+/* The other padding the paper mentions (caption of its naive-padding figure: "adding 0's or repeating the
+ * last entry of the sequence"), applied to blocks: the padding slots of a block repeat the frame in the
+ * block's last occupied slot.  A filler block holds no frame and is filled with pad_byte. */
+int oracle_pack_repeat_last(const oracle_tables_t *t, const uint8_t *store, int64_t frame_bytes,
+                            int64_t block_begin, int64_t block_count, uint8_t *dense, uint8_t pad_byte)
+{
+    int rc = oracle_pack(t, store, frame_bytes, block_begin, block_count, dense, pad_byte);
+    if (rc != ORACLE_OK) return rc;
+    uint8_t *vd = (uint8_t *)malloc((size_t)t->t_block), *rs = (uint8_t *)malloc((size_t)t->t_block);
+    int32_t *sid = (int32_t *)malloc(sizeof(int32_t) * (size_t)t->t_block);
+    int32_t *ps = (int32_t *)malloc(sizeof(int32_t) * (size_t)t->t_block);
+    if (!sid || !ps || !rs || !vd) { free(sid); free(ps); free(rs); free(vd); return ORACLE_ERR_NOMEM; }
+    for (int64_t q = 0; q < block_count; ++q) {
+        oracle_metadata(t, block_begin + q, 1, sid, ps, rs, vd);
+        int32_t last = -1;
+        for (int32_t s = 0; s < t->t_block; ++s) if (vd[s]) last = s;
+        if (last < 0) continue;
+        uint8_t *row = dense + (size_t)q * (size_t)t->t_block * (size_t)frame_bytes;
+        for (int32_t s = last + 1; s < t->t_block; ++s)
+            memcpy(row + (size_t)s * (size_t)frame_bytes, row + (size_t)last * (size_t)frame_bytes, (size_t)frame_bytes);
     }
     free(sid); free(ps); free(rs); free(vd);
     return ORACLE_OK;

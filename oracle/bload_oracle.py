@@ -77,6 +77,8 @@ def lib():
         L.oracle_pack.argtypes = [C.POINTER(_TablesStruct), C.c_void_p, C.c_int64, C.c_int64, C.c_int64,
                                   C.c_void_p, C.c_uint8]
         L.oracle_pack.restype = C.c_int
+        L.oracle_pack_repeat_last.argtypes = L.oracle_pack.argtypes
+        L.oracle_pack_repeat_last.restype = C.c_int
         L.oracle_unpack.argtypes = [C.POINTER(_TablesStruct), C.c_void_p, C.c_int64, C.c_int64, C.c_int64,
                                     C.c_void_p]
         L.oracle_unpack.restype = C.c_int
@@ -191,6 +193,19 @@ def pack(p: OraclePlan, store: np.ndarray, frame_bytes: int, block_begin: int, b
     dense = np.empty((block_count, p.t_block, frame_bytes), np.uint8)
     t = p._tables()
     rc = lib().oracle_pack(C.byref(t), _p(store), frame_bytes, block_begin, block_count, _p(dense), pad_byte)
+    assert rc == 0, rc
+    return dense
+
+
+def pack_repeat_last(p: OraclePlan, store: np.ndarray, frame_bytes: int, block_begin: int, block_count: int,
+                     pad_byte: int = 0) -> np.ndarray:
+    """pack(), but the padding slots of a block repeat its last frame (filler blocks: pad_byte)."""
+    store = np.ascontiguousarray(store).view(np.uint8).reshape(-1)
+    assert store.size == p.sum_t * frame_bytes
+    dense = np.empty((block_count, p.t_block, frame_bytes), np.uint8)
+    t = p._tables()
+    rc = lib().oracle_pack_repeat_last(C.byref(t), _p(store), frame_bytes, block_begin, block_count, _p(dense),
+                                       pad_byte)
     assert rc == 0, rc
     return dense
 

@@ -124,3 +124,39 @@ def test_pack_is_a_gather_and_unpack_its_inverse(name, n, fb, pad):
     assert np.array_equal(o2[touched], frames[touched]) and np.all(o2[~touched] == 0x3C)
     # packing a sub-range equals the slice
     assert np.array_equal(O.pack(p, store, fb, lo, cnt, pad), dense[lo:lo + cnt])
+
+
+def test_pack_repeat_last_against_a_numpy_gather():
+    rng = np.random.default_rng(12)
+    for n, tb, fb in ((8, 6, 3), (60, 25, 16), (200, 64, 5)):
+        T = rng.integers(1, tb + 1, size=n).astype(np.int32)
+        p = O.plan(T, tb, 1000 + n)
+        store = rng.integers(0, 256, size=(p.sum_t, fb), dtype=np.uint8)
+        nb = p.n_blocks + 1
+        seq_id, pos, _, valid = O.metadata(p, 0, nb)
+        src = np.where(valid == 1, p.offsets[np.maximum(seq_id, 0)] + pos, -1)
+        want = np.full((nb, tb, fb), 0x42, np.uint8)
+        for q in range(nb):
+            fill = int(valid[q].sum())
+            if fill:
+                idx = src[q].copy()
+                idx[fill:] = idx[fill - 1]
+                want[q] = store[idx]
+        got = O.pack_repeat_last(p, store, fb, 0, nb, 0x42)
+        assert np.array_equal(got, want)
+        assert np.array_equal(O.pack_repeat_last(p, store, fb, 1, 2, 0x42), want[1:3])
+
+
+def test_pack_repeat_last_with_one_sequence_per_block_is_the_naive_padding_of_the_paper():
+    # lengths above half a block cannot share a block: every sample is padded on its own by repeating its last frame
+    rng = np.random.default_rng(13)
+    tb = 20
+    T = rng.integers(11, tb + 1, size=30).astype(np.int32)
+    p = O.plan(T, tb, 5)
+    assert p.n_blocks == T.size
+    store = rng.integers(0, 256, size=(p.sum_t, 7), dtype=np.uint8)
+    got = O.pack_repeat_last(p, store, 7, 0, p.n_blocks)
+    for b in range(p.n_blocks):
+        i = int(p.seg_seq[p.block_seg_begin[b]])
+        x = store[p.offsets[i]:p.offsets[i + 1]]
+        assert np.array_equal(got[b], np.concatenate([x, np.repeat(x[-1:], tb - len(x), axis=0)]))
