@@ -172,6 +172,20 @@ BLOAD_API int bload_pack(const void* d_plan, const bload_plan_info_t* info, cons
                uint8_t* d_reset, uint8_t* d_valid, uint8_t pad_byte, void* stream);
 
 /*
+ * bload_pack_repeat_last -- bload_pack with the other padding the paper mentions (caption of its figure
+ * of the naive padding solution: samples are padded "by adding 0's or repeating the last entry"): the
+ * padding slots of a block repeat the frame in the block's last occupied slot instead of holding
+ * pad_byte.  Filler blocks, which hold no frame, are still filled with pad_byte, and the metadata is
+ * that of bload_pack (padding stays valid = 0: the repeated frames are not data).  Same arguments,
+ * alignment rules and errors as bload_pack.  Runs the pack kernels and then one small kernel that
+ * rewrites the padding from the dense buffer itself, on the same stream.
+ */
+BLOAD_API int bload_pack_repeat_last(const void* d_plan, const bload_plan_info_t* info, const void* d_store,
+                                     int64_t frame_bytes, int64_t block_begin, int64_t block_count, void* d_dense,
+                                     int32_t* d_seq_id, int32_t* d_pos, uint8_t* d_reset, uint8_t* d_valid,
+                                     uint8_t pad_byte, void* stream);
+
+/*
  * bload_unpack -- inverse of bload_pack for per-frame outputs: for every valid slot of the given
  * blocks, d_ragged_out[(offsets[id] + f) * out_frame_bytes ...] = d_dense_out[q, s, :].  Padding
  * slots and filler blocks are ignored; frames of sequences outside the block range are not touched.

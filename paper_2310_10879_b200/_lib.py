@@ -18,7 +18,7 @@ ERR_UNSUPPORTED, ERR_CUDA, ERR_TIMEOUT, ERR_PLAN = -6, -7, -8, -9
 MAX_T_BLOCK = 32768
 
 EXPORTS = ("bload_plan_sizes", "bload_plan", "bload_plan_async", "bload_plan_finish", "bload_rank_range", "bload_pack", "bload_unpack", "bload_stats",
-           "bload_carry_prev", "bload_reset_state", "bload_valid_sum",
+           "bload_pack_repeat_last", "bload_carry_prev", "bload_reset_state", "bload_valid_sum",
            "bload_set_plan_timing", "bload_plan_stage_times", "bload_kernel_launches", "bload_strerror",
            "bload_version")
 
@@ -79,6 +79,7 @@ def load() -> C.CDLL:
     L.bload_plan_finish.argtypes = [vp, vp, C.POINTER(PlanInfo)]
     L.bload_rank_range.argtypes = [i64, i32, i32, i32, C.POINTER(i64), C.POINTER(i64)]
     L.bload_pack.argtypes = [vp, C.POINTER(PlanInfo), vp, i64, i64, i64, vp, vp, vp, vp, vp, u8, vp]
+    L.bload_pack_repeat_last.argtypes = L.bload_pack.argtypes
     L.bload_unpack.argtypes = [vp, C.POINTER(PlanInfo), vp, i64, i64, i64, vp, vp]
     L.bload_stats.argtypes = [C.POINTER(PlanInfo), C.POINTER(Stats)]
     L.bload_carry_prev.argtypes = [vp, C.POINTER(PlanInfo), vp, i64, i64, i64, vp, u8, vp]
@@ -211,9 +212,11 @@ def bload_plan_finish(plan_buf, sizes: Sizes, stream=None, check: bool = True) -
 
 
 def bload_pack(plan: Plan, store, frame_bytes: int, block_begin: int, block_count: int, dense=None, seq_id=None,
-               pos=None, reset=None, valid=None, pad_byte: int = 0, stream=None) -> None:
-    """store: CUDA tensor holding the flat ragged frames; dense/seq_id/pos/reset/valid: CUDA outputs or None."""
-    rc = load().bload_pack(plan.buf.data_ptr(), C.byref(plan.info), _ptr(store), frame_bytes, block_begin,
+               pos=None, reset=None, valid=None, pad_byte: int = 0, stream=None, repeat_last: bool = False) -> None:
+    """store: CUDA tensor holding the flat ragged frames; dense/seq_id/pos/reset/valid: CUDA outputs or None.
+    repeat_last: padding slots repeat the block's last frame (bload_pack_repeat_last) instead of pad_byte."""
+    fn = load().bload_pack_repeat_last if repeat_last else load().bload_pack
+    rc = fn(plan.buf.data_ptr(), C.byref(plan.info), _ptr(store), frame_bytes, block_begin,
                            block_count, _ptr(dense), _ptr(seq_id), _ptr(pos), _ptr(reset), _ptr(valid), pad_byte,
                            _stream(stream))
     if rc:

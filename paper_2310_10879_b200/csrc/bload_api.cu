@@ -248,6 +248,20 @@ int bload_pack(const void* d_plan, const bload_plan_info_t* info, const void* d_
     return BLOAD_OK;
 }
 
+int bload_pack_repeat_last(const void* d_plan, const bload_plan_info_t* info, const void* d_store, int64_t frame_bytes,
+                           int64_t block_begin, int64_t block_count, void* d_dense, int32_t* d_seq_id, int32_t* d_pos,
+                           uint8_t* d_reset, uint8_t* d_valid, uint8_t pad_byte, void* stream)
+{
+    int rc = bload_pack(d_plan, info, d_store, frame_bytes, block_begin, block_count, d_dense, d_seq_id, d_pos, d_reset,
+                        d_valid, pad_byte, stream);
+    if (rc || block_count == 0 || !d_dense) return rc;
+    cudaError_t ce = launch_repeat_last(plan_view(const_cast<void*>(d_plan), info->n), info->t_block, frame_bytes,
+                                        block_begin, block_count, static_cast<uint8_t*>(d_dense),
+                                        static_cast<cudaStream_t>(stream));
+    if (ce != cudaSuccess) { (void)cudaGetLastError(); return BLOAD_ERR_CUDA; }
+    return BLOAD_OK;
+}
+
 int bload_unpack(const void* d_plan, const bload_plan_info_t* info, const void* d_dense_out, int64_t out_frame_bytes,
                  int64_t block_begin, int64_t block_count, void* d_ragged_out, void* stream)
 {

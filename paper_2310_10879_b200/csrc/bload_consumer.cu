@@ -1,10 +1,11 @@
 // Consumer side of the start table (paper, Methods, second paragraph): a recurrent model hands
 // information of frame t-1 to frame t and has to discard it wherever a new sequence starts inside a
-// block.  Three kernels use the plan's segment list for that, without per-slot metadata:
+// block.  These kernels use the plan's segment list for that, without per-slot metadata:
 //   k11_carry_prev   prev[q, s, :] = dense[q, s-1, :] where a sequence continues at slot s, a fill byte
 //                    elsewhere: one shifted, segmented memcpy over the whole batch (HBM bound);
 //   k12_reset_state  one step of a slot-by-slot recurrence: rows of the carried state whose block does
 //                    not continue a sequence at the given slot are re-initialised;
+//   k14_repeat_last  the other padding the paper mentions: padding slots repeat the block's last frame;
 //   k13_valid_sum    per-block sums of per-slot float values over frames only (padding masked out),
 //                    in double precision and in a fixed order, plus their total.
 #include "bload_internal.cuh"
@@ -98,6 +99,38 @@ __global__ void __launch_bounds__(256) k12_reset_state(PlanView pv, int64_t bloc
     }
 }
 
+// Repeat-last padding, applied after the pack kernel has written the blocks: a warp owns a sub-tile of the dense
+// side and overwrites the part of it that lies in the padding of its block with copies of the block's last frame.
+__global__ void __launch_bounds__(256) k14_repeat_last(PlanView pv, int32_t t_block, int64_t frame_bytes, int64_t block_begin,
+                                                       int64_t block_count, uint8_t* __restrict__ dense, int64_t sub_bytes,
+                                                       int64_t subs_per_block)
+{
+    const int lane = threadIdx.x & 31;
+    const int64_t warps = ((int64_t)gridDim.x * blockDim.x) >> 5;
+    const int64_t items = block_count * subs_per_block;
+    const int64_t block_bytes = (int64_t)t_block * frame_bytes;
+    const int64_t n_blocks = pv.hdr->n_blocks;
+    for (int64_t item = (((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5); item < items; item += warps) {
+        const int64_t q = item / subs_per_block;
+        const int64_t b = block_begin + q;
+        if (b >= n_blocks) continue;  // a filler block has no frame to repeat
+        const int64_t pad_lo = (int64_t)pv.block_fill[b] * frame_bytes;
+        const int64_t lo = (item - q * subs_per_block) * sub_bytes;
+        const int64_t hi = min(lo + sub_bytes, block_bytes);
+        int64_t cur = max(lo, pad_lo);
+        if (cur >= hi || pad_lo == 0) continue;
+        uint8_t* row = dense + q * block_bytes;
+        const uint8_t* last = row + pad_lo - frame_bytes;
+        int64_t fo = cur % frame_bytes;  // offset inside the frame being written
+        while (cur < hi) {
+            const int64_t len = min(frame_bytes - fo, hi - cur);
+            warp_copy<true>(row + cur, last + fo, len, row + pad_lo, lane);
+            cur += len;
+            fo = 0;
+        }
+    }
+}
+
 constexpr int kSumThreads = 256;
 
 // Fixed-order sum of one double per thread over a CTA of kSumThreads threads; the result is valid in thread 0.
@@ -186,6 +219,19 @@ cudaError_t launch_reset_state(const PlanView& pv, int64_t block_begin, int64_t 
     count_launches(1);
     k12_reset_state<<<grid_for_items(block_count * spr), 256, 0, st>>>(pv, block_begin, block_count, slot, state, state_bytes,
                                                                       init, sub, spr);
+    return cudaPeekAtLastError();
+}
+
+cudaError_t launch_repeat_last(const PlanView& pv, int32_t t_block, int64_t frame_bytes, int64_t block_begin,
+                               int64_t block_count, uint8_t* dense, cudaStream_t st)
+{
+    if (block_count == 0) return cudaSuccess;
+    const int64_t block_bytes = (int64_t)t_block * frame_bytes;
+    const int64_t sub = 16384;
+    const int64_t spb = (block_bytes + sub - 1) / sub;
+    count_launches(1);
+    k14_repeat_last<<<grid_for_items(block_count * spb), 256, 0, st>>>(pv, t_block, frame_bytes, block_begin, block_count,
+                                                                      dense, sub, spb);
     return cudaPeekAtLastError();
 }
 

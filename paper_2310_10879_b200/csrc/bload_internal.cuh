@@ -107,6 +107,8 @@ cudaError_t launch_carry_prev(const PlanView& pv, int32_t t_block, int64_t frame
                               int64_t block_count, const uint8_t* dense, uint8_t* prev, uint8_t fill_byte, cudaStream_t st);
 cudaError_t launch_reset_state(const PlanView& pv, int64_t block_begin, int64_t block_count, int32_t slot, uint8_t* state,
                                int64_t state_bytes, const uint8_t* init, cudaStream_t st);
+cudaError_t launch_repeat_last(const PlanView& pv, int32_t t_block, int64_t frame_bytes, int64_t block_begin,
+                               int64_t block_count, uint8_t* dense, cudaStream_t st);
 cudaError_t launch_valid_sum(const PlanView& pv, int32_t t_block, int64_t block_begin, int64_t block_count,
                              const float* values, double* block_sum, double* total, cudaStream_t st);
 

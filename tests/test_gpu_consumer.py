@@ -1,4 +1,4 @@
-"""GPU parity of the consumer-side calls (bload_carry_prev, bload_reset_state, bload_valid_sum),
+"""GPU parity of the consumer-side calls (bload_carry_prev, bload_reset_state, bload_valid_sum) and of repeat-last padding,
 through the C ABI, against the CPU oracle: bytes bit for bit, sums within a stated bound."""
 import numpy as np
 import pytest
@@ -212,3 +212,39 @@ def test_consumer_calls_reject_bad_arguments():
     B.bload_valid_sum(plan, f, 0, 0, d, tot)
     torch.cuda.synchronize()
     assert tot.tolist() == [0.0, 0.0]
+
+
+@pytest.mark.parametrize("fb", [1, 4, 6, 16, 100, 4096, 40000])
+def test_pack_repeat_last_against_the_oracle(fb):
+    rng = np.random.default_rng(fb + 1)
+    tb = int(rng.integers(5, 90))
+    T = rng.integers(1, tb + 1, size=int(rng.integers(2, 150))).astype(np.int32)
+    plan, op = _both_plans(T, tb, int(rng.integers(0, 1 << 40)))
+    g = torch.Generator(device=G.DEV); g.manual_seed(fb)
+    store = torch.randint(0, 256, (op.sum_t * fb,), dtype=torch.uint8, device=G.DEV, generator=g)
+    store_h = store.cpu().numpy()
+    for b0, cnt in ((0, op.n_blocks + 2), (1, max(op.n_blocks - 1, 1))):
+        dense = G.Guarded(cnt * tb * fb)
+        valid = torch.empty(cnt * tb, dtype=torch.uint8, device=G.DEV)
+        B.bload_pack(plan, store, fb, b0, cnt, dense=dense.t, valid=valid, pad_byte=0x33, repeat_last=True)
+        torch.cuda.synchronize()
+        dense.check()
+        d = G.first_diff(dense.t.cpu().numpy(), O.pack_repeat_last(op, store_h, fb, b0, cnt, 0x33))
+        assert d is None, "repeat-last fb=%d: %s" % (fb, d)
+        assert np.array_equal(valid.cpu().numpy().reshape(cnt, tb), O.metadata(op, b0, cnt)[3])
+
+
+def test_pack_repeat_last_workloads():
+    for name, n in (("toy_video", 0), ("features_fp16", 0), ("tokens", 20000), ("heavy_tail_bf16", 1000)):
+        w = W.WORKLOADS[name]
+        if n:
+            w = W.scaled(w, n)
+        plan, op = _both_plans(W.lengths(w), w.t_block, w.seed)
+        store = W.payload_torch(w, op.sum_t, G.DEV).view(torch.uint8).reshape(-1)
+        cnt = op.n_blocks + 1
+        dense = G.Guarded(cnt * w.t_block * w.frame_bytes)
+        B.bload_pack(plan, store, w.frame_bytes, 0, cnt, dense=dense.t, repeat_last=True)
+        torch.cuda.synchronize()
+        dense.check()
+        d = G.first_diff(dense.t.cpu().numpy(), O.pack_repeat_last(op, store.cpu().numpy(), w.frame_bytes, 0, cnt, 0))
+        assert d is None, name + ": " + d
