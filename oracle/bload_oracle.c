@@ -25,6 +25,9 @@
  *                      round trip, pad bytes
  *   pack_repeat_last   numpy gather with pad slots mapped to the block's last frame; with one
  *                      sequence per block, the paper's naive repeat-last padding of each sample
+ *   byte_offsets       numpy.cumsum of T_i * F_i
+ *   pack_var/unpack_var  equal frame sizes reduce to pack/unpack; per-slot numpy construction from
+ *                      H_i x W_i images; round trip; padding bytes
  *   carry_prev         shifting every sequence by one frame in the ragged store and
  *                      packing that gives the same bytes
  *   reset_state        a running sum carried through the slots with resets equals the
@@ -395,6 +398,68 @@ int oracle_unpack(const oracle_tables_t *t, const uint8_t *dense_out, int64_t fr
             if (!vd[s]) continue;
             memcpy(ragged_out + (size_t)(t->offsets[sid[s]] + ps[s]) * (size_t)frame_bytes,
                    dense_out + ((size_t)q * (size_t)t->t_block + (size_t)s) * (size_t)frame_bytes, (size_t)frame_bytes);
+        }
+    }
+    free(sid); free(ps); free(rs); free(vd);
+    return ORACLE_OK;
+}
+
+/* ------------------------------------------------------------------------ */
+/* Frames whose size differs from sample to sample (problem statement: every   */
+/* sample has its own H, W and T).  Sequence i holds T_i frames of F_i bytes,  */
+/* back to back, at byte_offsets[i] of the store; a slot of a block has room   */
+/* for the largest frame and a smaller frame is followed by padding.           */
+/* ------------------------------------------------------------------------ */
+void oracle_byte_offsets(const int32_t *lengths, const int32_t *frame_bytes, int64_t n, int64_t *byte_offsets)
+{
+    int64_t run = 0;
+    for (int64_t i = 0; i < n; ++i) { byte_offsets[i] = run; run += (int64_t)lengths[i] * (int64_t)frame_bytes[i]; }
+    byte_offsets[n] = run;
+}
+
+int oracle_pack_var(const oracle_tables_t *t, const uint8_t *store, const int32_t *frame_bytes,
+                    const int64_t *byte_offsets, int64_t slot_bytes, int64_t block_begin, int64_t block_count,
+                    uint8_t *dense, uint8_t pad_byte)
+{
+    if (block_begin < 0 || block_count < 0 || slot_bytes < 1) return ORACLE_ERR_ARG;
+    for (int64_t i = 0; i < t->n; ++i) if (frame_bytes[i] < 1 || frame_bytes[i] > slot_bytes) return ORACLE_ERR_ARG;
+    int32_t *sid = (int32_t *)malloc(sizeof(int32_t) * (size_t)t->t_block);
+    int32_t *ps = (int32_t *)malloc(sizeof(int32_t) * (size_t)t->t_block);
+    uint8_t *rs = (uint8_t *)malloc((size_t)t->t_block), *vd = (uint8_t *)malloc((size_t)t->t_block);
+    if (!sid || !ps || !rs || !vd) { free(sid); free(ps); free(rs); free(vd); return ORACLE_ERR_NOMEM; }
+    for (int64_t q = 0; q < block_count; ++q) {
+        oracle_metadata(t, block_begin + q, 1, sid, ps, rs, vd);
+        for (int32_t s = 0; s < t->t_block; ++s) {
+            uint8_t *dst = dense + ((size_t)q * (size_t)t->t_block + (size_t)s) * (size_t)slot_bytes;
+            size_t have = 0;
+            if (vd[s]) {
+                have = (size_t)frame_bytes[sid[s]];
+                memcpy(dst, store + (size_t)byte_offsets[sid[s]] + (size_t)ps[s] * have, have);
+            }
+            memset(dst + have, pad_byte, (size_t)slot_bytes - have);
+        }
+    }
+    free(sid); free(ps); free(rs); free(vd);
+    return ORACLE_OK;
+}
+
+int oracle_unpack_var(const oracle_tables_t *t, const uint8_t *dense_out, const int32_t *frame_bytes,
+                      const int64_t *byte_offsets, int64_t slot_bytes, int64_t block_begin, int64_t block_count,
+                      uint8_t *ragged_out)
+{
+    if (block_begin < 0 || block_count < 0 || slot_bytes < 1) return ORACLE_ERR_ARG;
+    for (int64_t i = 0; i < t->n; ++i) if (frame_bytes[i] < 1 || frame_bytes[i] > slot_bytes) return ORACLE_ERR_ARG;
+    int32_t *sid = (int32_t *)malloc(sizeof(int32_t) * (size_t)t->t_block);
+    int32_t *ps = (int32_t *)malloc(sizeof(int32_t) * (size_t)t->t_block);
+    uint8_t *rs = (uint8_t *)malloc((size_t)t->t_block), *vd = (uint8_t *)malloc((size_t)t->t_block);
+    if (!sid || !ps || !rs || !vd) { free(sid); free(ps); free(rs); free(vd); return ORACLE_ERR_NOMEM; }
+    for (int64_t q = 0; q < block_count; ++q) {
+        oracle_metadata(t, block_begin + q, 1, sid, ps, rs, vd);
+        for (int32_t s = 0; s < t->t_block; ++s) {
+            if (!vd[s]) continue;
+            size_t have = (size_t)frame_bytes[sid[s]];
+            memcpy(ragged_out + (size_t)byte_offsets[sid[s]] + (size_t)ps[s] * have,
+                   dense_out + ((size_t)q * (size_t)t->t_block + (size_t)s) * (size_t)slot_bytes, have);
         }
     }
     free(sid); free(ps); free(rs); free(vd);

@@ -82,6 +82,14 @@ def lib():
         L.oracle_unpack.argtypes = [C.POINTER(_TablesStruct), C.c_void_p, C.c_int64, C.c_int64, C.c_int64,
                                     C.c_void_p]
         L.oracle_unpack.restype = C.c_int
+        L.oracle_byte_offsets.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p]
+        L.oracle_byte_offsets.restype = None
+        L.oracle_pack_var.argtypes = [C.POINTER(_TablesStruct), C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64,
+                                      C.c_int64, C.c_int64, C.c_void_p, C.c_uint8]
+        L.oracle_pack_var.restype = C.c_int
+        L.oracle_unpack_var.argtypes = [C.POINTER(_TablesStruct), C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64,
+                                        C.c_int64, C.c_int64, C.c_void_p]
+        L.oracle_unpack_var.restype = C.c_int
         L.oracle_carry_prev.argtypes = [C.POINTER(_TablesStruct), C.c_void_p, C.c_int64, C.c_int64, C.c_int64,
                                         C.c_void_p, C.c_uint8]
         L.oracle_carry_prev.restype = C.c_int
@@ -219,6 +227,45 @@ def unpack(p: OraclePlan, dense_out: np.ndarray, frame_bytes: int, block_begin: 
     assert ragged_out.size == p.sum_t * frame_bytes
     t = p._tables()
     rc = lib().oracle_unpack(C.byref(t), _p(dense_out), frame_bytes, block_begin, block_count, _p(ragged_out))
+    assert rc == 0, rc
+    return ragged_out
+
+
+def byte_offsets(lengths: np.ndarray, frame_bytes: np.ndarray) -> np.ndarray:
+    """int64[n+1]: first byte of sequence i in a store whose sequence i holds T_i frames of frame_bytes[i] bytes."""
+    lengths = np.ascontiguousarray(lengths, dtype=np.int32)
+    frame_bytes = np.ascontiguousarray(frame_bytes, dtype=np.int32)
+    assert lengths.size == frame_bytes.size
+    out = np.zeros(lengths.size + 1, dtype=np.int64)
+    lib().oracle_byte_offsets(_p(lengths), _p(frame_bytes), lengths.size, _p(out))
+    return out
+
+
+def pack_var(p: OraclePlan, store: np.ndarray, frame_bytes: np.ndarray, slot_bytes: int, block_begin: int,
+             block_count: int, pad_byte: int = 0) -> np.ndarray:
+    """pack() for per-sequence frame sizes: every slot has slot_bytes bytes, a smaller frame is followed by padding."""
+    frame_bytes = np.ascontiguousarray(frame_bytes, dtype=np.int32)
+    boff = byte_offsets(p.lengths, frame_bytes)
+    store = np.ascontiguousarray(store).view(np.uint8).reshape(-1)
+    assert store.size == int(boff[-1])
+    dense = np.empty((block_count, p.t_block, slot_bytes), np.uint8)
+    t = p._tables()
+    rc = lib().oracle_pack_var(C.byref(t), _p(store), _p(frame_bytes), _p(boff), slot_bytes, block_begin, block_count,
+                               _p(dense), pad_byte)
+    assert rc == 0, rc
+    return dense
+
+
+def unpack_var(p: OraclePlan, dense_out: np.ndarray, frame_bytes: np.ndarray, slot_bytes: int, block_begin: int,
+               block_count: int, ragged_out: np.ndarray) -> np.ndarray:
+    frame_bytes = np.ascontiguousarray(frame_bytes, dtype=np.int32)
+    boff = byte_offsets(p.lengths, frame_bytes)
+    dense_out = np.ascontiguousarray(dense_out).view(np.uint8).reshape(-1)
+    assert dense_out.size == block_count * p.t_block * slot_bytes
+    assert ragged_out.dtype == np.uint8 and ragged_out.flags.c_contiguous and ragged_out.size == int(boff[-1])
+    t = p._tables()
+    rc = lib().oracle_unpack_var(C.byref(t), _p(dense_out), _p(frame_bytes), _p(boff), slot_bytes, block_begin,
+                                 block_count, _p(ragged_out))
     assert rc == 0, rc
     return ragged_out
 

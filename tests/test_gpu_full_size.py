@@ -50,6 +50,18 @@ def _run(name, n_sample):
         padmask = slot[None, :] >= fill[lo:lo + step, None]
         nonzero_pad += int((chunk.ne(0).any(dim=2) & padmask).sum())
     assert nonzero_pad == 0
+    # per-slot metadata of the whole epoch in one call: sampled blocks against the oracle, and counts that hold at any
+    # size (one valid slot per frame, one reset flag per sequence, ids and positions -1 exactly on padding)
+    meta = [torch.empty(nb * tb, dtype=d, device=G.DEV) for d in (torch.int32, torch.int32, torch.uint8, torch.uint8)]
+    B.bload_pack(plan, None, fb, 0, nb, seq_id=meta[0], pos=meta[1], reset=meta[2], valid=meta[3])
+    torch.cuda.synchronize()
+    for b in blocks:
+        for got, want in zip(meta, O.metadata(op, b, 1)):
+            assert np.array_equal(got.view(nb, tb)[b].cpu().numpy(), want[0]), "metadata of block %d" % b
+    assert int(meta[3].sum(dtype=torch.int64)) == op.sum_t and int(meta[2].sum(dtype=torch.int64)) == op.n
+    assert int((meta[0] < 0).sum()) == nb * tb - op.sum_t and bool(((meta[0] < 0) == (meta[3] == 0)).all())
+    assert bool(((meta[1] == 0) == (meta[2] == 1)).all())
+    del meta
     # round trip of the input itself (same frame size): unpack(pack(x)) == x, every byte
     back = G.Guarded(op.sum_t * fb, 0x5A)
     B.bload_unpack(plan, dense.t, fb, 0, nb, back.t)
