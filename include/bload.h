@@ -197,6 +197,42 @@ BLOAD_API int bload_unpack(const void* d_plan, const bload_plan_info_t* info, co
                  void* stream);
 
 /*
+ * Frames whose size differs from sample to sample (paper, Problem Statement: each sample S_i has its
+ * own H, W and T).  Sequence i holds T_i frames of F_i = d_frame_bytes[i] bytes, back to back, at byte
+ * d_byte_offsets[i] of the store.  A slot of a block has slot_bytes bytes (at least the largest F_i);
+ * a frame sits at the start of its slot and the rest of the slot is padding.  The plan is the ordinary
+ * one (it depends only on the lengths), and per-slot metadata comes from bload_pack as before.  The
+ * paper does not say how frames of different sizes share a block; this layout (every frame on a
+ * canvas of the largest size, as opaque bytes) is the reading taken here.
+ *
+ * bload_var_offsets -- d_byte_offsets[i] = sum over j < i of T_j * F_j, for i = 0..n.  The array needs
+ * n + 3 elements: [n] = total bytes of the store, [n+1] = largest F_i, [n+2] = first i with F_i < 1
+ * or -1; the same three values are returned in `info` after one synchronisation of `stream`.
+ * Returns BLOAD_ERR_ARG when some F_i < 1.  d_lengths, d_frame_bytes: device int32[n].
+ *
+ * bload_pack_var / bload_unpack_var -- bload_pack / bload_unpack with per-sequence frame sizes:
+ *   d_dense[q, s, 0:F_id] = frame f of sequence id;  d_dense[q, s, F_id:slot_bytes] = pad_byte
+ *   d_ragged_out[byte_offsets[id] + f * F_id ...] = d_dense_out[q, s, 0:F_id]
+ * d_dense is [block_count, t_block, slot_bytes]; store, dense and ragged_out 16-byte aligned.
+ * Precondition: 1 <= F_i <= slot_bytes for every i (bload_var_offsets reports the largest); sizes
+ * outside that range are clamped on the device, which truncates frames but never leaves the buffers.
+ * Asynchronous on `stream`.  Errors as for bload_pack (slot_bytes in the place of frame_bytes).
+ */
+typedef struct {
+    int64_t total_bytes;     /* bytes of the ragged store */
+    int64_t max_frame_bytes; /* largest F_i: the smallest slot_bytes that holds every frame */
+    int64_t first_bad_index; /* first i with F_i < 1, else -1 */
+} bload_var_info_t;
+BLOAD_API int bload_var_offsets(const int32_t* d_lengths, const int32_t* d_frame_bytes, int64_t n,
+                                int64_t* d_byte_offsets, void* stream, bload_var_info_t* info);
+BLOAD_API int bload_pack_var(const void* d_plan, const bload_plan_info_t* info, const void* d_store,
+                             const int32_t* d_frame_bytes, const int64_t* d_byte_offsets, int64_t slot_bytes,
+                             int64_t block_begin, int64_t block_count, void* d_dense, uint8_t pad_byte, void* stream);
+BLOAD_API int bload_unpack_var(const void* d_plan, const bload_plan_info_t* info, const void* d_dense_out,
+                               const int32_t* d_frame_bytes, const int64_t* d_byte_offsets, int64_t slot_bytes,
+                               int64_t block_begin, int64_t block_count, void* d_ragged_out, void* stream);
+
+/*
  * Consumer side of the start table (paper, Methods, second paragraph, and its figure of the DDS
  * architecture): a recurrent model feeds information of frame t-1 into frame t, and the table of
  * start indices tells it where that information belongs to another sequence and has to be

@@ -18,7 +18,7 @@ ERR_UNSUPPORTED, ERR_CUDA, ERR_TIMEOUT, ERR_PLAN = -6, -7, -8, -9
 MAX_T_BLOCK = 32768
 
 EXPORTS = ("bload_plan_sizes", "bload_plan", "bload_plan_async", "bload_plan_finish", "bload_rank_range", "bload_pack", "bload_unpack", "bload_stats",
-           "bload_pack_repeat_last", "bload_carry_prev", "bload_reset_state", "bload_valid_sum",
+           "bload_pack_repeat_last", "bload_var_offsets", "bload_pack_var", "bload_unpack_var", "bload_carry_prev", "bload_reset_state", "bload_valid_sum",
            "bload_set_plan_timing", "bload_plan_stage_times", "bload_kernel_launches", "bload_strerror",
            "bload_version")
 
@@ -43,6 +43,10 @@ class Stats(C.Structure):
                [(k, C.c_double) for k in ("frac_packed", "frac_naive_tmax", "frac_naive_tblock",
                                           "reduction_vs_tmax", "mean_segs_per_block")] + \
                [("max_segs_per_block", C.c_int64)]
+
+
+class VarInfo(C.Structure):
+    _fields_ = [("total_bytes", C.c_int64), ("max_frame_bytes", C.c_int64), ("first_bad_index", C.c_int64)]
 
 
 class BloadError(RuntimeError):
@@ -82,6 +86,9 @@ def load() -> C.CDLL:
     L.bload_pack_repeat_last.argtypes = L.bload_pack.argtypes
     L.bload_unpack.argtypes = [vp, C.POINTER(PlanInfo), vp, i64, i64, i64, vp, vp]
     L.bload_stats.argtypes = [C.POINTER(PlanInfo), C.POINTER(Stats)]
+    L.bload_var_offsets.argtypes = [vp, vp, i64, vp, vp, C.POINTER(VarInfo)]
+    L.bload_pack_var.argtypes = [vp, C.POINTER(PlanInfo), vp, vp, vp, i64, i64, i64, vp, u8, vp]
+    L.bload_unpack_var.argtypes = [vp, C.POINTER(PlanInfo), vp, vp, vp, i64, i64, i64, vp, vp]
     L.bload_carry_prev.argtypes = [vp, C.POINTER(PlanInfo), vp, i64, i64, i64, vp, u8, vp]
     L.bload_reset_state.argtypes = [vp, C.POINTER(PlanInfo), i64, i64, i32, vp, i64, vp, vp]
     L.bload_valid_sum.argtypes = [vp, C.POINTER(PlanInfo), vp, i64, i64, vp, vp, vp]
@@ -229,6 +236,40 @@ def bload_unpack(plan: Plan, dense_out, out_frame_bytes: int, block_begin: int, 
                              block_count, _ptr(ragged_out), _stream(stream))
     if rc:
         raise BloadError(rc, "bload_unpack")
+
+
+def bload_var_offsets(lengths, frame_bytes, stream=None):
+    """Byte offsets of a store whose sequence i holds lengths[i] frames of frame_bytes[i] bytes (CUDA int32 tensors).
+    Returns (byte_offsets int64 CUDA tensor [n+3], VarInfo); the first n+1 entries are the offsets."""
+    import torch
+    n = lengths.numel()
+    out = torch.empty(n + 3, dtype=torch.int64, device=lengths.device)
+    info = VarInfo()
+    rc = load().bload_var_offsets(lengths.data_ptr(), frame_bytes.data_ptr(), n, out.data_ptr(), _stream(stream),
+                                  C.byref(info))
+    if rc:
+        err = BloadError(rc, "bload_var_offsets")
+        err.info = info
+        raise err
+    return out, info
+
+
+def bload_pack_var(plan: Plan, store, frame_bytes, byte_offsets, slot_bytes: int, block_begin: int, block_count: int,
+                   dense, pad_byte: int = 0, stream=None) -> None:
+    rc = load().bload_pack_var(plan.buf.data_ptr(), C.byref(plan.info), _ptr(store), _ptr(frame_bytes),
+                               _ptr(byte_offsets), slot_bytes, block_begin, block_count, _ptr(dense), pad_byte,
+                               _stream(stream))
+    if rc:
+        raise BloadError(rc, "bload_pack_var")
+
+
+def bload_unpack_var(plan: Plan, dense_out, frame_bytes, byte_offsets, slot_bytes: int, block_begin: int,
+                     block_count: int, ragged_out, stream=None) -> None:
+    rc = load().bload_unpack_var(plan.buf.data_ptr(), C.byref(plan.info), _ptr(dense_out), _ptr(frame_bytes),
+                                 _ptr(byte_offsets), slot_bytes, block_begin, block_count, _ptr(ragged_out),
+                                 _stream(stream))
+    if rc:
+        raise BloadError(rc, "bload_unpack_var")
 
 
 def bload_carry_prev(plan: Plan, dense, frame_bytes: int, block_begin: int, block_count: int, prev,

@@ -103,6 +103,10 @@ cudaError_t launch_copy(bool unpack, const PlanView& pv, int32_t t_block, int64_
                         int64_t block_count, const uint8_t* ragged_in, uint8_t* dense, uint8_t* ragged_out,
                         int64_t ragged_bytes, uint8_t pad_byte, cudaStream_t st, int64_t n, int64_t n_blocks);
 
+cudaError_t launch_var_offsets(const int32_t* lengths, const int32_t* frame_bytes, int64_t n, int64_t* out, cudaStream_t st);
+cudaError_t launch_copy_var(bool unpack, const PlanView& pv, int32_t t_block, int64_t slot_bytes, int64_t block_begin,
+                            int64_t block_count, const int32_t* frame_bytes, const int64_t* byte_offsets,
+                            const uint8_t* src, uint8_t* dst, uint8_t pad_byte, cudaStream_t st);
 cudaError_t launch_carry_prev(const PlanView& pv, int32_t t_block, int64_t frame_bytes, int64_t block_begin,
                               int64_t block_count, const uint8_t* dense, uint8_t* prev, uint8_t fill_byte, cudaStream_t st);
 cudaError_t launch_reset_state(const PlanView& pv, int64_t block_begin, int64_t block_count, int32_t slot, uint8_t* state,

@@ -1,0 +1,187 @@
+// Frames whose size differs from sample to sample (paper, Problem Statement: every sample S_i has its own
+// H, W and T).  Sequence i holds T_i frames of F_i bytes back to back; a slot of a block has room for the
+// largest frame, and a smaller frame sits at the start of its slot, followed by padding.
+//   k15_var_offsets  byte offset of every sequence in such a store (exclusive scan of T_i * F_i), with the
+//                    largest frame size and the first invalid size;
+//   k16_copy_var     pack / unpack with per-sequence frame sizes: the decomposition of the fixed-size copy
+//                    kernel (a warp owns a sub-tile of the dense side), walking slots inside each segment.
+#include "bload_internal.cuh"
+#include "bload_warp_copy.cuh"
+
+namespace bload {
+
+namespace {
+
+using namespace wc;
+
+constexpr int kScanThreads = 1024;
+
+// One CTA walks the sequences in chunks of kScanThreads with a running carry.  out[0..n) = first byte of each
+// sequence, out[n] = total bytes, out[n+1] = largest frame size, out[n+2] = first i with F_i < 1 (or -1).
+__global__ void __launch_bounds__(kScanThreads) k15_var_offsets(const int32_t* __restrict__ lengths,
+                                                                const int32_t* __restrict__ frame_bytes, int64_t n,
+                                                                int64_t* __restrict__ out)
+{
+    __shared__ int64_t warp_sum[kScanThreads / 32];
+    __shared__ int64_t carry_sh;
+    __shared__ int max_sh;
+    __shared__ unsigned long long bad_sh;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (threadIdx.x == 0) { carry_sh = 0; max_sh = 0; bad_sh = ~0ULL; }
+    __syncthreads();
+    int my_max = 0;
+    for (int64_t base = 0; base < n; base += kScanThreads) {
+        const int64_t i = base + threadIdx.x;
+        int64_t v = 0;
+        if (i < n) {
+            const int f = frame_bytes[i];
+            if (f < 1) atomicMin(&bad_sh, (unsigned long long)i);
+            my_max = max(my_max, f);
+            v = (int64_t)lengths[i] * (int64_t)max(f, 0);
+        }
+        int64_t incl = v;  // inclusive scan inside the warp
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const int64_t up = __shfl_up_sync(kFull, incl, d);
+            if (lane >= d) incl += up;
+        }
+        if (lane == 31) warp_sum[warp] = incl;
+        __syncthreads();
+        if (warp == 0) {
+            int64_t w = warp_sum[lane];
+#pragma unroll
+            for (int d = 1; d < 32; d <<= 1) {
+                const int64_t up = __shfl_up_sync(kFull, w, d);
+                if (lane >= d) w += up;
+            }
+            warp_sum[lane] = w;  // inclusive over warps
+        }
+        __syncthreads();
+        const int64_t carry = carry_sh;
+        const int64_t before = carry + (warp ? warp_sum[warp - 1] : 0) + (incl - v);
+        if (i < n) out[i] = before;
+        __syncthreads();
+        if (threadIdx.x == kScanThreads - 1) carry_sh = carry + warp_sum[kScanThreads / 32 - 1];
+        __syncthreads();
+    }
+    atomicMax(&max_sh, my_max);
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        out[n] = carry_sh;
+        out[n + 1] = max_sh;
+        out[n + 2] = bad_sh == ~0ULL ? -1 : (int64_t)bad_sh;
+    }
+}
+
+// A frame size is clamped to the slot size on the device, so a caller that breaks the documented precondition
+// (F_i <= slot_bytes) gets truncated frames but never an access outside the buffers.
+template <bool UNPACK>
+__global__ void __launch_bounds__(256, 2) k16_copy_var(PlanView pv, int32_t t_block, int64_t slot_bytes, int64_t block_begin,
+                                                       int64_t block_count, const int32_t* __restrict__ frame_bytes,
+                                                       const int64_t* __restrict__ byte_offsets,
+                                                       const uint8_t* __restrict__ src_base, uint8_t* __restrict__ dst_base,
+                                                       int64_t sub_bytes, int64_t subs_per_block, uint8_t pad)
+{
+    const int lane = threadIdx.x & 31;
+    const int64_t warps = ((int64_t)gridDim.x * blockDim.x) >> 5;
+    const int64_t items = block_count * subs_per_block;
+    const int64_t block_bytes = (int64_t)t_block * slot_bytes;
+    const int64_t n_blocks = pv.hdr->n_blocks;
+    const int64_t ragged_total = byte_offsets[pv.hdr->n];
+    const uint8_t* s_limit = src_base + (UNPACK ? block_count * block_bytes : ragged_total);
+
+    for (int64_t item = (((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5); item < items; item += warps) {
+        const int64_t q = item / subs_per_block;
+        const int64_t lo = (item - q * subs_per_block) * sub_bytes;
+        const int64_t hi = min(lo + sub_bytes, block_bytes);
+        const int64_t b = block_begin + q;
+        const int64_t dense_off = q * block_bytes;
+        int64_t cur = lo;
+        if (b < n_blocks) {
+            const int k0 = pv.block_seg_begin[b], k1 = pv.block_seg_begin[b + 1];
+            const int fill = pv.block_fill[b];
+            if (cur < (int64_t)fill * slot_bytes) {
+                int slot = (int)(cur / slot_bytes);
+                int64_t in = cur - (int64_t)slot * slot_bytes;  // offset inside the slot
+                int k = warp_find_segment(pv.seg_start, k0, k1, slot, lane);
+                int kw = k;  // lanes hold start slot, frame size and first byte of segments kw .. kw+31
+                int w_st = fill, w_fb = 1;
+                int64_t w_off = 0;
+                auto load_window = [&]() {
+                    w_st = fill; w_fb = 1; w_off = 0;
+                    if (kw + lane < k1) {
+                        const int id = pv.seg_seq[kw + lane];
+                        w_st = pv.seg_start[kw + lane];
+                        w_fb = (int)min((int64_t)max(frame_bytes[id], 1), slot_bytes);
+                        w_off = byte_offsets[id];
+                    }
+                };
+                load_window();
+                while (cur < hi && k < k1) {
+                    if (k - kw == 31) { kw = k; load_window(); }
+                    const int st = __shfl_sync(kFull, w_st, k - kw);
+                    const int nx = __shfl_sync(kFull, w_st, k - kw + 1);
+                    const int64_t fb = __shfl_sync(kFull, w_fb, k - kw);
+                    const int64_t off = __shfl_sync(kFull, w_off, k - kw);
+                    const int64_t seg_e = min((int64_t)nx * slot_bytes, hi);
+                    if (fb == slot_bytes) {  // frames fill their slots: the rest of the segment is one run
+                        const int64_t rag = off + (cur - (int64_t)st * slot_bytes);
+                        if (UNPACK) warp_copy<true>(dst_base + rag, src_base + dense_off + cur, seg_e - cur, s_limit, lane);
+                        else warp_copy<false>(dst_base + dense_off + cur, src_base + rag, seg_e - cur, s_limit, lane);
+                        in = 0;  // a segment ends on a slot boundary unless the tile ends first
+                        cur = seg_e;
+                    } else {
+                        while (cur < seg_e) {
+                            if (in < fb) {
+                                const int64_t len = min(fb - in, seg_e - cur);
+                                const int64_t rag = off + (int64_t)(slot - st) * fb + in;
+                                if (UNPACK) warp_copy<true>(dst_base + rag, src_base + dense_off + cur, len, s_limit, lane);
+                                else warp_copy<false>(dst_base + dense_off + cur, src_base + rag, len, s_limit, lane);
+                                cur += len; in += len;
+                            }
+                            if (cur < seg_e) {  // the padding behind the frame
+                                const int64_t len = min(slot_bytes - in, seg_e - cur);
+                                if (!UNPACK) warp_fill(dst_base + dense_off + cur, len, pad, lane);
+                                cur += len; in += len;
+                            }
+                            if (in == slot_bytes) { in = 0; ++slot; }
+                        }
+                    }
+                    if (cur == (int64_t)nx * slot_bytes) { ++k; slot = nx; in = 0; }
+                }
+            }
+        }
+        if (!UNPACK && cur < hi) warp_fill(dst_base + dense_off + cur, hi - cur, pad, lane);
+    }
+}
+
+}  // namespace
+
+cudaError_t launch_var_offsets(const int32_t* lengths, const int32_t* frame_bytes, int64_t n, int64_t* out, cudaStream_t st)
+{
+    count_launches(1);
+    k15_var_offsets<<<1, kScanThreads, 0, st>>>(lengths, frame_bytes, n, out);
+    return cudaPeekAtLastError();
+}
+
+cudaError_t launch_copy_var(bool unpack, const PlanView& pv, int32_t t_block, int64_t slot_bytes, int64_t block_begin,
+                            int64_t block_count, const int32_t* frame_bytes, const int64_t* byte_offsets,
+                            const uint8_t* src, uint8_t* dst, uint8_t pad_byte, cudaStream_t st)
+{
+    if (block_count == 0) return cudaSuccess;
+    const int64_t block_bytes = (int64_t)t_block * slot_bytes;
+    const int64_t sub = 16384;
+    const int64_t spb = (block_bytes + sub - 1) / sub;
+    const int64_t want = (block_count * spb + 7) / 8;
+    const unsigned grid = (unsigned)(want < 0x7fffffffLL ? want : 0x7fffffffLL);
+    count_launches(1);
+    if (unpack)
+        k16_copy_var<true><<<grid, 256, 0, st>>>(pv, t_block, slot_bytes, block_begin, block_count, frame_bytes, byte_offsets,
+                                                  src, dst, sub, spb, pad_byte);
+    else
+        k16_copy_var<false><<<grid, 256, 0, st>>>(pv, t_block, slot_bytes, block_begin, block_count, frame_bytes, byte_offsets,
+                                                   src, dst, sub, spb, pad_byte);
+    return cudaPeekAtLastError();
+}
+
+}  // namespace bload

@@ -1,0 +1,121 @@
+"""GPU parity of per-sample frame sizes (bload_var_offsets, bload_pack_var, bload_unpack_var), through the
+C ABI, against the CPU oracle, bit for bit."""
+import numpy as np
+import pytest
+import torch
+
+import gpu_util as G
+import paper_2310_10879_b200 as B
+from oracle import bload_oracle as O
+
+pytestmark = pytest.mark.gpu
+
+
+def _setup(T, F, tb, seed):
+    T = np.ascontiguousarray(T, np.int32); F = np.ascontiguousarray(F, np.int32)
+    op = O.plan(T, tb, seed)
+    plan = G.gpu_plan(T, tb, seed)
+    assert plan.info.checksum == op.checksum
+    d_T = torch.from_numpy(T).to(G.DEV); d_F = torch.from_numpy(F).to(G.DEV)
+    boff, info = B.bload_var_offsets(d_T, d_F)
+    want = O.byte_offsets(T, F)
+    assert np.array_equal(boff[:T.size + 1].cpu().numpy(), want)
+    assert (info.total_bytes, info.max_frame_bytes, info.first_bad_index) == (int(want[-1]), int(F.max()), -1)
+    return op, plan, d_F, boff, int(want[-1])
+
+
+def _parity(T, F, tb, seed, slot, pad=0x6B, ranges=None):
+    op, plan, d_F, boff, total = _setup(T, F, tb, seed)
+    g = torch.Generator(device=G.DEV); g.manual_seed(seed)
+    store = torch.randint(0, 256, (total,), dtype=torch.uint8, device=G.DEV, generator=g)
+    store_h = store.cpu().numpy()
+    for b0, cnt in ranges or ((0, op.n_blocks + 2), (1, max(op.n_blocks - 1, 1))):
+        dense = G.Guarded(cnt * tb * slot)
+        B.bload_pack_var(plan, store, d_F, boff, slot, b0, cnt, dense.t, pad_byte=pad)
+        torch.cuda.synchronize(); dense.check()
+        d = G.first_diff(dense.t.cpu().numpy(), O.pack_var(op, store_h, F, slot, b0, cnt, pad))
+        assert d is None, "pack_var slot=%d blocks [%d,+%d): %s" % (slot, b0, cnt, d)
+        dense_out = torch.randint(0, 256, (cnt * tb * slot,), dtype=torch.uint8, device=G.DEV, generator=g)
+        rag = G.Guarded(total, 0x5A)
+        B.bload_unpack_var(plan, dense_out, d_F, boff, slot, b0, cnt, rag.t)
+        torch.cuda.synchronize(); rag.check()
+        want = np.full(total, 0x5A, np.uint8)
+        O.unpack_var(op, dense_out.cpu().numpy(), F, slot, b0, cnt, want)
+        d = G.first_diff(rag.t.cpu().numpy(), want)
+        assert d is None, "unpack_var slot=%d blocks [%d,+%d): %s" % (slot, b0, cnt, d)
+    # round trip on the GPU alone
+    nb = op.n_blocks
+    dense = torch.empty(nb * tb * slot, dtype=torch.uint8, device=G.DEV)
+    back = torch.full((total,), 0x11, dtype=torch.uint8, device=G.DEV)
+    B.bload_pack_var(plan, store, d_F, boff, slot, 0, nb, dense)
+    B.bload_unpack_var(plan, dense, d_F, boff, slot, 0, nb, back)
+    torch.cuda.synchronize()
+    assert torch.equal(back, store)
+
+
+@pytest.mark.parametrize("fmax", [1, 3, 4, 16, 37, 100, 1000, 5000, 40000])
+def test_random_frame_sizes(fmax):
+    rng = np.random.default_rng(fmax)
+    tb = int(rng.integers(4, 60))
+    n = int(rng.integers(2, 120))
+    T = rng.integers(1, tb + 1, size=n)
+    F = rng.integers(1, fmax + 1, size=n)
+    _parity(T, F, tb, 7 + fmax, slot=fmax)
+    _parity(T, F, tb, 8 + fmax, slot=fmax + int(rng.integers(1, 40)))  # slots larger than every frame
+
+
+def test_images_of_different_sizes():
+    # H_i x W_i x 3 uint8 images on a canvas of the largest size; t_block spans several 16 KB sub-tiles per slot and
+    # several slots per sub-tile
+    rng = np.random.default_rng(2)
+    n, tb = 60, 24
+    T = rng.integers(1, tb + 1, size=n)
+    H = rng.integers(8, 97, size=n); Wd = rng.integers(8, 129, size=n)
+    F = H * Wd * 3
+    _parity(T, F, tb, 99, slot=96 * 128 * 3)
+
+
+def test_equal_sizes_match_the_fixed_size_calls():
+    rng = np.random.default_rng(5)
+    tb, fb = 50, 4096
+    T = rng.integers(1, tb + 1, size=200).astype(np.int32)
+    F = np.full(T.size, fb, np.int32)
+    op, plan, d_F, boff, total = _setup(T, F, tb, 3)
+    store = torch.randint(0, 256, (total,), dtype=torch.uint8, device=G.DEV)
+    nb = op.n_blocks + 1
+    a = torch.empty(nb * tb * fb, dtype=torch.uint8, device=G.DEV); b = torch.empty_like(a)
+    B.bload_pack_var(plan, store, d_F, boff, fb, 0, nb, a, pad_byte=9)
+    B.bload_pack(plan, store, fb, 0, nb, dense=b, pad_byte=9)
+    torch.cuda.synchronize()
+    assert torch.equal(a, b)
+
+
+def test_var_offsets_large_and_bad_sizes():
+    rng = np.random.default_rng(6)
+    n = 300_000
+    T = rng.integers(1, 4096, size=n).astype(np.int32)
+    F = rng.integers(1, 1 << 18, size=n).astype(np.int32)
+    d_T = torch.from_numpy(T).to(G.DEV); d_F = torch.from_numpy(F).to(G.DEV)
+    boff, info = B.bload_var_offsets(d_T, d_F)
+    want = O.byte_offsets(T, F)
+    assert int(want[-1]) > 1 << 40
+    assert np.array_equal(boff[:n + 1].cpu().numpy(), want) and info.max_frame_bytes == int(F.max())
+    F[1234] = 0; F[200_000] = -5
+    with pytest.raises(B.BloadError) as e:
+        B.bload_var_offsets(d_T, torch.from_numpy(F).to(G.DEV))
+    assert e.value.code == -2 and e.value.info.first_bad_index == 1234
+
+
+def test_var_calls_reject_bad_arguments():
+    T = np.array([3, 4, 5], np.int32); F = np.array([8, 16, 4], np.int32)
+    op, plan, d_F, boff, total = _setup(T, F, 8, 1)
+    buf = torch.zeros(1 << 12, dtype=torch.uint8, device=G.DEV)
+    for args, code in (((buf, d_F, boff, 0, 0, 1, buf), -2), ((buf, d_F, boff, 16, -1, 1, buf), -2),
+                       ((None, d_F, boff, 16, 0, 1, buf), -1), ((buf, None, boff, 16, 0, 1, buf), -1),
+                       ((buf[4:], d_F, boff, 16, 0, 1, buf), -5)):
+        with pytest.raises(B.BloadError) as e:
+            B.bload_pack_var(plan, *args)
+        assert e.value.code == code
+        with pytest.raises(B.BloadError) as e:
+            B.bload_unpack_var(plan, *args)
+        assert e.value.code == code
