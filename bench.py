@@ -438,13 +438,33 @@ def run_gpu(args, w) -> dict:
         bb = min(w.batch_blocks, nb)
         state = torch.zeros(bb * 4096, dtype=torch.uint8, device=dev)
         ms_reset = timed(lambda: B.bload_reset_state(plan, 0, bb, tb // 2, state, 4096), 200)
+        # per-sample frame sizes: the same lengths, frame sizes drawn from {1/4, 1/2, 3/4, 1} of the workload's frame
+        var = None
+        if fb >= 64:
+            import numpy as np
+            rngv = np.random.Generator(np.random.PCG64(w.seed + 77))
+            Fv = (rngv.integers(1, 5, size=T.size) * (fb // 4)).astype(np.int32)
+            d_Fv = torch.from_numpy(Fv).to(dev)
+            boff, vinfo = B.bload_var_offsets(d_len, d_Fv)
+            vstore = torch.empty(vinfo.total_bytes, dtype=torch.uint8, device=dev)
+            vstore.view(torch.int32)[:].random_() if vinfo.total_bytes % 4 == 0 else vstore.random_()
+            vback = torch.empty_like(vstore)
+            ms_p = timed(lambda: B.bload_pack_var(plan, vstore, d_Fv, boff, fb, 0, nb, dense), 10)
+            ms_u = timed(lambda: B.bload_unpack_var(plan, dense, d_Fv, boff, fb, 0, nb, vback), 10)
+            ok = bool(torch.equal(vback, vstore))
+            var = {"frame_bytes": "uniform over {1/4, 1/2, 3/4, 1} x %d" % fb, "slot_bytes": fb,
+                   "store_bytes": int(vinfo.total_bytes),
+                   "pack_ms": ms_p, "pack_GB/s": (vinfo.total_bytes + nb * tb * fb) / ms_p / 1e6,
+                   "unpack_ms": ms_u, "unpack_GB/s": 2 * vinfo.total_bytes / ms_u / 1e6, "round_trip_ok": ok}
+            del vstore, vback, boff
         consumer = {"carry_prev": {"ms": ms, "GB/s": cp_bytes / ms / 1e6, "algorithmic_bytes": cp_bytes,
                                    "what": "prev[q,s] = dense[q,s-1] inside sequences, fill elsewhere, all blocks; "
                                            "bytes = (sum_t - n) frames read + n_blocks*t_block frames written"},
                     "valid_sum": {"ms": ms_sum, "GB/s": 4 * sum_t / ms_sum / 1e6, "slots": nb * tb,
                                   "what": "fp32 per-slot values, frames only, per-block and total sums in double; "
                                           "bytes = 4 per frame read"},
-                    "reset_state": {"us_per_call": ms_reset * 1e3, "batch_blocks": bb, "state_bytes": 4096}}
+                    "reset_state": {"us_per_call": ms_reset * 1e3, "batch_blocks": bb, "state_bytes": 4096},
+                    "var_frames": var}
         del vals, bsum, tot, state
 
     # ---- end to end through the same calls with HOST buffers (pinned), copies inside the timed region
