@@ -348,7 +348,8 @@ int bload_carry_prev(const void* d_plan, const bload_plan_info_t* info, const vo
     if (!aligned(d_dense, 16) || !aligned(d_prev, 16)) return BLOAD_ERR_ALIGN;
     cudaError_t ce = launch_carry_prev(plan_view(const_cast<void*>(d_plan), info->n), info->t_block, frame_bytes,
                                        block_begin, block_count, static_cast<const uint8_t*>(d_dense),
-                                       static_cast<uint8_t*>(d_prev), fill_byte, static_cast<cudaStream_t>(stream));
+                                       static_cast<uint8_t*>(d_prev), fill_byte, static_cast<cudaStream_t>(stream), info->n,
+                                       info->sum_t);
     if (ce != cudaSuccess) { (void)cudaGetLastError(); return BLOAD_ERR_CUDA; }
     return BLOAD_OK;
 }

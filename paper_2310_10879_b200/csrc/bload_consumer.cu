@@ -198,13 +198,18 @@ unsigned grid_for_items(int64_t items)
 }  // namespace
 
 cudaError_t launch_carry_prev(const PlanView& pv, int32_t t_block, int64_t frame_bytes, int64_t block_begin,
-                              int64_t block_count, const uint8_t* dense, uint8_t* prev, uint8_t fill_byte, cudaStream_t st)
+                              int64_t block_count, const uint8_t* dense, uint8_t* prev, uint8_t fill_byte, cudaStream_t st,
+                              int64_t n, int64_t sum_t)
 {
     if (block_count == 0) return cudaSuccess;
     const int64_t block_bytes = (int64_t)t_block * frame_bytes;
     const int64_t sub = 16384;
     const int64_t spb = (block_bytes + sub - 1) / sub;
     count_launches(1);
+    // small word-sized frames in short runs: the staged pack kernel with the dense input as its source
+    cudaError_t staged_err = cudaSuccess;
+    if (staged_carry_prev(pv, t_block, frame_bytes, block_begin, block_count, dense, prev, fill_byte, st, n, sum_t, &staged_err))
+        return staged_err;
     k11_carry_prev<<<grid_for_items(block_count * spb), 256, 0, st>>>(pv, t_block, frame_bytes, block_begin, block_count,
                                                                      dense, prev, sub, spb, fill_byte);
     return cudaPeekAtLastError();

@@ -446,6 +446,8 @@ __global__ void __launch_bounds__(StageCfg<false>::kWarps * 32) k9_unpack_ragged
 // twin of k9_unpack_ragged): the warp locates its first segment once and then walks forward through
 // the segment list, which runs on from one block to the next; only `fill` and the segment end of each
 // new block are read, one block ahead.  Blocks at or beyond n_blocks are written as padding.
+// CARRY: the same walk produces bload_carry_prev for small frames (source = the dense input, one frame back).
+template <bool CARRY>
 __global__ void __launch_bounds__(StageCfg<false>::kWarps * 32) k10_pack_contig(PlanView pv, int32_t n, int32_t t_block,
                                                                               int64_t frame_bytes, int64_t block_begin,
                                                                               const uint8_t* __restrict__ store,
@@ -511,7 +513,17 @@ __global__ void __launch_bounds__(StageCfg<false>::kWarps * 32) k10_pack_contig(
             const int64_t src = __shfl_sync(kFull, w_src, k - kw);
             const int seg_e = (k + 1 < k1) ? nx * fb : fill_bytes;  // the block's last run ends where its frames end
             const int pe = min(seg_e, hi);
-            warp_gather_async(sa + (uint32_t)(cur - lo), store + src * fb + (cur - st * fb), pe - cur, lane);
+            if (CARRY) {
+                // `store` is the dense input: the first frame of a segment receives the fill pattern, every later byte
+                // the byte one frame before it in the same block
+                const int fe = min(st * fb + fb, pe);
+                for (int o = cur + 4 * lane; o < fe; o += 128) *reinterpret_cast<uint32_t*>(stage + (o - lo)) = p4;
+                cur = max(cur, fe);
+                if (cur < pe)
+                    warp_gather_async(sa + (uint32_t)(cur - lo), store + q * (int64_t)block_bytes + (cur - fb), pe - cur, lane);
+            } else {
+                warp_gather_async(sa + (uint32_t)(cur - lo), store + src * fb + (cur - st * fb), pe - cur, lane);
+            }
             cur = pe;
             if (pe == seg_e) ++k;
         }
@@ -543,6 +555,34 @@ __global__ void __launch_bounds__(StageCfg<false>::kWarps * 32) k10_pack_contig(
 
 }  // namespace
 
+// bload_carry_prev through the staged pack kernel; false when the frame size or the run lengths do not suit it.
+bool staged_carry_prev(const PlanView& pv, int32_t t_block, int64_t frame_bytes, int64_t block_begin, int64_t block_count,
+                       const uint8_t* dense, uint8_t* prev, uint8_t fill_byte, cudaStream_t st, int64_t n, int64_t sum_t,
+                       cudaError_t* err)
+{
+    const int64_t block_bytes = (int64_t)t_block * frame_bytes;
+    if (!(frame_bytes % 4 == 0 && n > 0 && sum_t * frame_bytes / n <= kStagedMaxRunBytes && block_bytes < (1LL << 31) &&
+          block_bytes % 16 == 0))
+        return false;
+    using Cfg = StageCfg<false>;
+    const size_t smem = (size_t)Cfg::kWarps * Cfg::kStages * Cfg::kBytes + 16;
+    const int per_sm = (int)((227 * 1024) / (smem + 1024));
+    *err = cudaFuncSetAttribute(k10_pack_contig<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (*err != cudaSuccess) return true;
+    const int64_t spb = (block_bytes + Cfg::kBytes - 1) / Cfg::kBytes;
+    const int64_t tiles = block_count * spb;
+    const int64_t max_warps = (int64_t)148 * per_sm * Cfg::kWarps;
+    int64_t tpw = (tiles + max_warps - 1) / max_warps;
+    if (tpw > kPackChunkTiles) tpw = kPackChunkTiles;
+    int64_t warps = (tiles + tpw - 1) / tpw;
+    if (warps > max_warps) warps = max_warps;
+    const unsigned grid = (unsigned)((warps + Cfg::kWarps - 1) / Cfg::kWarps);
+    k10_pack_contig<true><<<grid, Cfg::kWarps * 32, smem, st>>>(pv, (int32_t)n, t_block, frame_bytes, block_begin, dense, prev,
+                                                               tiles, tpw, (int32_t)spb, fill_byte);
+    *err = cudaPeekAtLastError();
+    return true;
+}
+
 cudaError_t launch_copy(bool unpack, const PlanView& pv, int32_t t_block, int64_t frame_bytes, int64_t block_begin,
                         int64_t block_count, const uint8_t* ragged_in, uint8_t* dense, uint8_t* ragged_out,
                         int64_t ragged_bytes, uint8_t pad_byte, cudaStream_t st, int64_t n, int64_t n_blocks)
@@ -556,7 +596,7 @@ cudaError_t launch_copy(bool unpack, const PlanView& pv, int32_t t_block, int64_
         using Cfg = StageCfg<false>;
         const size_t smem = (size_t)Cfg::kWarps * Cfg::kStages * Cfg::kBytes + 16;
         const int per_sm = (int)((227 * 1024) / (smem + 1024));
-        cudaError_t e = cudaFuncSetAttribute(k10_pack_contig, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        cudaError_t e = cudaFuncSetAttribute(k10_pack_contig<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
         const int64_t spb = (block_bytes + Cfg::kBytes - 1) / Cfg::kBytes;
         const int64_t tiles = block_count * spb;
@@ -566,7 +606,7 @@ cudaError_t launch_copy(bool unpack, const PlanView& pv, int32_t t_block, int64_
         int64_t warps = (tiles + tpw - 1) / tpw;
         if (warps > max_warps) warps = max_warps;
         const unsigned grid = (unsigned)((warps + Cfg::kWarps - 1) / Cfg::kWarps);
-        k10_pack_contig<<<grid, Cfg::kWarps * 32, smem, st>>>(pv, (int32_t)n, t_block, frame_bytes, block_begin, ragged_in,
+        k10_pack_contig<false><<<grid, Cfg::kWarps * 32, smem, st>>>(pv, (int32_t)n, t_block, frame_bytes, block_begin, ragged_in,
                                                              dense, tiles, tpw, (int32_t)spb, pad_byte);
         return cudaPeekAtLastError();
     }

@@ -108,7 +108,11 @@ cudaError_t launch_copy_var(bool unpack, const PlanView& pv, int32_t t_block, in
                             int64_t block_count, const int32_t* frame_bytes, const int64_t* byte_offsets,
                             const uint8_t* src, uint8_t* dst, uint8_t pad_byte, cudaStream_t st);
 cudaError_t launch_carry_prev(const PlanView& pv, int32_t t_block, int64_t frame_bytes, int64_t block_begin,
-                              int64_t block_count, const uint8_t* dense, uint8_t* prev, uint8_t fill_byte, cudaStream_t st);
+                              int64_t block_count, const uint8_t* dense, uint8_t* prev, uint8_t fill_byte, cudaStream_t st,
+                              int64_t n, int64_t sum_t);
+bool staged_carry_prev(const PlanView& pv, int32_t t_block, int64_t frame_bytes, int64_t block_begin, int64_t block_count,
+                       const uint8_t* dense, uint8_t* prev, uint8_t fill_byte, cudaStream_t st, int64_t n, int64_t sum_t,
+                       cudaError_t* err);
 cudaError_t launch_reset_state(const PlanView& pv, int64_t block_begin, int64_t block_count, int32_t slot, uint8_t* state,
                                int64_t state_bytes, const uint8_t* init, cudaStream_t st);
 cudaError_t launch_repeat_last(const PlanView& pv, int32_t t_block, int64_t frame_bytes, int64_t block_begin,

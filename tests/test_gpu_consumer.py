@@ -248,3 +248,19 @@ def test_pack_repeat_last_workloads():
         dense.check()
         d = G.first_diff(dense.t.cpu().numpy(), O.pack_repeat_last(op, store.cpu().numpy(), w.frame_bytes, 0, cnt, 0))
         assert d is None, name + ": " + d
+
+
+@pytest.mark.parametrize("fb,tb", [(4, 16), (4, 4096), (8, 64), (12, 1000), (16, 64), (32, 500), (100, 64), (256, 48),
+                                   (4, 8192)])
+def test_carry_prev_small_word_sized_frames_take_the_staged_kernel(fb, tb):
+    # frame sizes that are multiples of 4 in short runs with 16-byte block rows: stages of 8 KB, several per block or
+    # several blocks per stage, segments that start inside a stage, first frames that straddle two stages
+    rng = np.random.default_rng(fb * 1000 + tb)
+    n = int(rng.integers(50, 600))
+    T = np.minimum(rng.geometric(1.0 / max(2, tb // 6), size=n), tb).astype(np.int32)
+    plan, op = _both_plans(T, tb, int(rng.integers(0, 1 << 40)))
+    _carry_prev_parity(plan, op, fb, 0, op.n_blocks + 2, 0x00)
+    _carry_prev_parity(plan, op, fb, 0, op.n_blocks, 0xC3, seed=9)
+    if op.n_blocks > 4:
+        _carry_prev_parity(plan, op, fb, 3, op.n_blocks - 4, 0x5E)
+        _carry_prev_parity(plan, op, fb, op.n_blocks - 1, 5, 0x01)
