@@ -161,7 +161,15 @@ __global__ void __launch_bounds__(kSumThreads) k13_valid_sum(PlanView pv, int32_
     if ((reinterpret_cast<uintptr_t>(row) & 15u) == 0) {
         const int nv = fill >> 2;
         const float4* r4 = reinterpret_cast<const float4*>(row);
-        for (int i = threadIdx.x; i < nv; i += kSumThreads) {
+        int i = threadIdx.x;
+        for (; i + 3 * kSumThreads < nv; i += 4 * kSumThreads) {  // four loads in flight per thread
+            float4 v[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) v[u] = __ldcs(r4 + i + u * kSumThreads);
+#pragma unroll
+            for (int u = 0; u < 4; ++u) acc += ((double)v[u].x + (double)v[u].y) + ((double)v[u].z + (double)v[u].w);
+        }
+        for (; i < nv; i += kSumThreads) {
             const float4 v = __ldcs(r4 + i);
             acc += ((double)v.x + (double)v.y) + ((double)v.z + (double)v.w);
         }

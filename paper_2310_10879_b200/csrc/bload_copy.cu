@@ -94,19 +94,34 @@ __global__ void __launch_bounds__(256) k7_copy(PlanView pv, int32_t t_block, int
 // Tuning of the two directions (swept on B200 with the 4-byte token workload): bytes per stage, warps
 // per CTA, stages per warp, consecutive sub-tiles of a block handled by one warp.  More, smaller stages
 // mean more resident warps; the kernels are limited by per-warp instruction latency, not by bytes in flight.
-#ifndef BLOAD_PACK_CFG
-#define BLOAD_PACK_CFG 8192, 4, 2, 2
+#ifndef BLOAD_PACK_BYTES
+#define BLOAD_PACK_BYTES 8192
 #endif
-#ifndef BLOAD_UNPACK_CFG
-#define BLOAD_UNPACK_CFG 4096, 8, 2, 4
+#ifndef BLOAD_PACK_WARPS
+#define BLOAD_PACK_WARPS 4
+#endif
+#ifndef BLOAD_PACK_STAGES
+#define BLOAD_PACK_STAGES 2
+#endif
+#ifndef BLOAD_UNPACK_BYTES
+#define BLOAD_UNPACK_BYTES 4096
+#endif
+#ifndef BLOAD_UNPACK_WARPS
+#define BLOAD_UNPACK_WARPS 8
+#endif
+#ifndef BLOAD_UNPACK_STAGES
+#define BLOAD_UNPACK_STAGES 2
+#endif
+#ifndef BLOAD_UNPACK_GROUP
+#define BLOAD_UNPACK_GROUP 4
 #endif
 template <int BYTES, int WARPS, int STAGES, int GROUP>
 struct StageCfgT {
     static constexpr int kBytes = BYTES, kWarps = WARPS, kStages = STAGES, kGroup = GROUP;
     static_assert(BYTES % 512 == 0 && STAGES >= 2 && GROUP >= 1, "stage configuration");
 };
-template <bool UNPACK> struct StageCfg : StageCfgT<BLOAD_PACK_CFG> {};
-template <> struct StageCfg<true> : StageCfgT<BLOAD_UNPACK_CFG> {};
+template <bool UNPACK> struct StageCfg : StageCfgT<BLOAD_PACK_BYTES, BLOAD_PACK_WARPS, BLOAD_PACK_STAGES, 2> {};
+template <> struct StageCfg<true> : StageCfgT<BLOAD_UNPACK_BYTES, BLOAD_UNPACK_WARPS, BLOAD_UNPACK_STAGES, BLOAD_UNPACK_GROUP> {};
 // the staged kernels win while the average run (T_i * frame_bytes) is short; measured cross-over on B200 at about
 // 16 KB (1.4 KB runs: 6.0 against 3.8 TB/s; 14 KB: 5.9 against 5.8; 23 KB: 6.15 against 6.36)
 constexpr int64_t kStagedMaxRunBytes = 16384;
