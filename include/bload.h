@@ -150,6 +150,51 @@ BLOAD_API int bload_plan_async(const int32_t* d_lengths, int64_t n, int32_t t_bl
 BLOAD_API int bload_plan_finish(const void* d_plan, void* stream, bload_plan_info_t* info);
 
 /*
+ * bload_epoch -- plan, metadata, pack and unpack of one whole epoch in a single call, with the copies running
+ * while the plan is still being built.  Results are exactly those of
+ *     bload_plan(policy BLOAD_POLICY_UNIFORM_SEQUENCES) ; bload_pack(blocks 0 .. block_capacity) ;
+ *     bload_unpack(blocks 0 .. block_capacity)
+ * but the fill rule (a chain of dependent draws that keeps one warp busy and leaves the memory system idle) runs
+ * in chunks of about 1,250 draws on `stream`, and as soon as a chunk has closed its blocks their tables, metadata,
+ * pack and unpack are issued on `side_stream`, under the next chunk of the chain.  Only launch-order dependencies
+ * (events) are used; no kernel waits for another.  The paper has no counterpart (it builds blocks on the host).
+ *
+ *   io->d_store / frame_bytes / d_dense      pack (skipped when d_dense is NULL)
+ *   io->d_seq_id, d_pos, d_reset, d_valid    per-slot metadata, each may be NULL
+ *   io->d_dense_out / out_frame_bytes / d_ragged_out   unpack (skipped when d_dense_out is NULL)
+ *   io->block_capacity   rows (blocks) that d_dense, the metadata arrays and d_dense_out have; the number of
+ *                        blocks is only known when the plan is done, so give an upper bound (the previous epoch's
+ *                        count plus a margin, or 2 * sum_t / t_block + 1); rows beyond n_blocks are filler
+ *   d_work / work_bytes  as for bload_plan (bload_plan_sizes covers this call)
+ *   side_stream          a second stream of the same device, or NULL (then everything runs on `stream`, in order)
+ *
+ * Both streams are synchronised once before the call returns: on return `info` is filled and every output is
+ * complete.  Errors are those of bload_plan, bload_pack and bload_unpack; BLOAD_ERR_WORKSPACE is also returned when
+ * n_blocks exceeds block_capacity (the plan is complete and info->n_blocks tells how many rows are needed; blocks
+ * beyond the capacity were not packed).  With bload_set_plan_timing(1), bload_epoch_stage_times returns the device
+ * time of the last call, summed over chunks: [0] fill rule, [1] tables, [2] metadata, [3] pack, [4] unpack (ms).
+ */
+typedef struct {
+    const void* d_store;
+    int64_t frame_bytes;
+    void* d_dense;
+    int32_t* d_seq_id;
+    int32_t* d_pos;
+    uint8_t* d_reset;
+    uint8_t* d_valid;
+    const void* d_dense_out;
+    int64_t out_frame_bytes;
+    void* d_ragged_out;
+    int64_t block_capacity;
+    uint8_t pad_byte;
+    uint8_t reserved_[7];
+} bload_epoch_io_t;
+BLOAD_API int bload_epoch(const int32_t* d_lengths, int64_t n, int32_t t_block, uint64_t seed, void* d_plan,
+                          size_t plan_bytes, void* d_work, size_t work_bytes, const bload_epoch_io_t* io, void* stream,
+                          void* side_stream, bload_plan_info_t* info);
+BLOAD_API int bload_epoch_stage_times(float out_ms[5]);
+
+/*
  * bload_pack -- dense batches and per-slot metadata for blocks [block_begin, block_begin+block_count)
  * (paper, Methods: concatenate the sequences of a block, pad the rest with zeros; the start table).
  *

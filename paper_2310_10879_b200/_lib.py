@@ -17,7 +17,7 @@ ERR_NULL, ERR_ARG, ERR_LENGTH, ERR_WORKSPACE, ERR_ALIGN = -1, -2, -3, -4, -5
 ERR_UNSUPPORTED, ERR_CUDA, ERR_TIMEOUT, ERR_PLAN = -6, -7, -8, -9
 MAX_T_BLOCK = 32768
 
-EXPORTS = ("bload_plan_sizes", "bload_plan", "bload_plan_async", "bload_plan_finish", "bload_rank_range", "bload_pack", "bload_unpack", "bload_stats",
+EXPORTS = ("bload_plan_sizes", "bload_plan", "bload_plan_async", "bload_plan_finish", "bload_rank_range", "bload_pack", "bload_unpack", "bload_stats", "bload_epoch", "bload_epoch_stage_times",
            "bload_pack_repeat_last", "bload_var_offsets", "bload_pack_var", "bload_unpack_var", "bload_carry_prev", "bload_reset_state", "bload_valid_sum",
            "bload_set_plan_timing", "bload_plan_stage_times", "bload_kernel_launches", "bload_strerror",
            "bload_version")
@@ -43,6 +43,13 @@ class Stats(C.Structure):
                [(k, C.c_double) for k in ("frac_packed", "frac_naive_tmax", "frac_naive_tblock",
                                           "reduction_vs_tmax", "mean_segs_per_block")] + \
                [("max_segs_per_block", C.c_int64)]
+
+
+class EpochIO(C.Structure):
+    _fields_ = [("d_store", C.c_void_p), ("frame_bytes", C.c_int64), ("d_dense", C.c_void_p),
+                ("d_seq_id", C.c_void_p), ("d_pos", C.c_void_p), ("d_reset", C.c_void_p), ("d_valid", C.c_void_p),
+                ("d_dense_out", C.c_void_p), ("out_frame_bytes", C.c_int64), ("d_ragged_out", C.c_void_p),
+                ("block_capacity", C.c_int64), ("pad_byte", C.c_uint8), ("reserved_", C.c_uint8 * 7)]
 
 
 class VarInfo(C.Structure):
@@ -92,6 +99,9 @@ def load() -> C.CDLL:
     L.bload_carry_prev.argtypes = [vp, C.POINTER(PlanInfo), vp, i64, i64, i64, vp, u8, vp]
     L.bload_reset_state.argtypes = [vp, C.POINTER(PlanInfo), i64, i64, i32, vp, i64, vp, vp]
     L.bload_valid_sum.argtypes = [vp, C.POINTER(PlanInfo), vp, i64, i64, vp, vp, vp]
+    L.bload_epoch.argtypes = [vp, i64, i32, u64, vp, C.c_size_t, vp, C.c_size_t, C.POINTER(EpochIO), vp, vp,
+                              C.POINTER(PlanInfo)]
+    L.bload_epoch_stage_times.argtypes = [C.POINTER(C.c_float * 5)]
     L.bload_set_plan_timing.argtypes = [C.c_int]
     L.bload_plan_stage_times.argtypes = [C.POINTER(C.c_float * 4)]
     L.bload_strerror.argtypes = [C.c_int]
@@ -187,6 +197,43 @@ def bload_plan(lengths, t_block: int, seed: int, policy: int = 0, stream=None, w
         err.info = info
         raise err
     return Plan(plan_buf, info, sizes)
+
+
+def bload_epoch(lengths, t_block: int, seed: int, block_capacity: int, store=None, frame_bytes: int = 0, dense=None,
+                seq_id=None, pos=None, reset=None, valid=None, pad_byte: int = 0, dense_out=None,
+                out_frame_bytes: int = 0, ragged_out=None, stream=None, side_stream=None, work=None, plan_buf=None,
+                check: bool = True) -> Plan:
+    """Plan, metadata, pack and unpack of a whole epoch in one call; the copies of finished blocks run on
+    `side_stream` while the plan is still being built on `stream`.  Same results as bload_plan + bload_pack +
+    bload_unpack over blocks [0, block_capacity).  All outputs are complete when the call returns."""
+    import torch
+    if not lengths.is_cuda or lengths.dtype != torch.int32 or not lengths.is_contiguous():
+        raise TypeError("lengths must be a contiguous CUDA int32 tensor")
+    n = lengths.numel()
+    sizes = bload_plan_sizes(n, t_block)
+    if plan_buf is None:
+        plan_buf = torch.empty(sizes.plan_bytes, dtype=torch.uint8, device=lengths.device)
+    if work is None:
+        work = torch.empty(sizes.work_bytes, dtype=torch.uint8, device=lengths.device)
+    io = EpochIO(_ptr(store), frame_bytes, _ptr(dense), _ptr(seq_id), _ptr(pos), _ptr(reset), _ptr(valid),
+                 _ptr(dense_out), out_frame_bytes, _ptr(ragged_out), block_capacity, pad_byte)
+    info = PlanInfo()
+    side = None if side_stream is None else (side_stream.cuda_stream or None)
+    rc = load().bload_epoch(lengths.data_ptr(), n, t_block, seed, plan_buf.data_ptr(), plan_buf.numel(),
+                            work.data_ptr(), work.numel(), C.byref(io), _stream(stream), side, C.byref(info))
+    if rc and check:
+        err = BloadError(rc, "bload_epoch")
+        err.info = info
+        raise err
+    return Plan(plan_buf, info, sizes)
+
+
+def bload_epoch_stage_times() -> list[float]:
+    out = (C.c_float * 5)()
+    rc = load().bload_epoch_stage_times(C.byref(out))
+    if rc:
+        raise BloadError(rc, "bload_epoch_stage_times")
+    return [float(x) for x in out]
 
 
 def bload_plan_async(lengths, t_block: int, seed: int, policy: int = 0, stream=None, work=None, plan_buf=None):

@@ -51,6 +51,8 @@ namespace {
 thread_local bool g_timing = false;
 thread_local bool g_have_times = false;
 thread_local float g_stage_ms[4] = {0, 0, 0, 0};
+thread_local bool g_have_epoch_times = false;
+thread_local float g_epoch_ms[5] = {0, 0, 0, 0, 0};
 
 inline bool aligned(const void* p, uintptr_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
 
@@ -107,7 +109,9 @@ int bload_plan_sizes(int64_t n, int32_t t_block, bload_sizes_t* out)
     int rc = check_sizes(n, t_block);
     if (rc) return rc;
     plan_layout(n, out);
-    out->work_bytes = work_layout(n, t_block, nullptr, nullptr) + bfd_layout(n, t_block, nullptr, nullptr);
+    // policy 2 and bload_epoch (policy 0) place their extra scratch behind the common part; they never run together
+    const size_t extra_bfd = bfd_layout(n, t_block, nullptr, nullptr), extra_epoch = epoch_layout(t_block, nullptr, nullptr);
+    out->work_bytes = work_layout(n, t_block, nullptr, nullptr) + (extra_bfd > extra_epoch ? extra_bfd : extra_epoch);
     return BLOAD_OK;
 }
 
@@ -222,6 +226,155 @@ int bload_plan_finish(const void* d_plan, void* stream, bload_plan_info_t* info)
     info->checksum = h.checksum;
     info->max_segs_per_block = h.max_segs;
     if (h.status == BLOAD_OK && h.magic != kPlanMagic) return fail(BLOAD_ERR_PLAN);
+    return info->status;
+}
+
+int bload_epoch_stage_times(float out_ms[5])
+{
+    if (!out_ms) return BLOAD_ERR_NULL;
+    if (!g_have_epoch_times) return BLOAD_ERR_PLAN;
+    for (int i = 0; i < 5; ++i) out_ms[i] = g_epoch_ms[i];
+    return BLOAD_OK;
+}
+
+int bload_epoch(const int32_t* d_lengths, int64_t n, int32_t t_block, uint64_t seed, void* d_plan, size_t plan_bytes,
+                void* d_work, size_t work_bytes, const bload_epoch_io_t* io, void* stream, void* side_stream,
+                bload_plan_info_t* info)
+{
+    if (!info) return BLOAD_ERR_NULL;
+    memset(info, 0, sizeof *info);
+    info->first_bad_index = -1;
+    info->n = n; info->t_block = t_block; info->seed = seed; info->policy = BLOAD_POLICY_UNIFORM_SEQUENCES;
+    auto fail = [&](int rc) { info->status = rc; return rc; };
+    if (!d_lengths || !d_plan || !d_work || !io) return fail(BLOAD_ERR_NULL);
+    int rc = check_sizes(n, t_block);
+    if (rc) return fail(rc);
+    const bool do_pack = io->d_dense != nullptr, do_unpack = io->d_dense_out != nullptr;
+    const bool do_meta = io->d_seq_id || io->d_pos || io->d_reset || io->d_valid;
+    if (do_pack && !io->d_store) return fail(BLOAD_ERR_NULL);
+    if (do_unpack && !io->d_ragged_out) return fail(BLOAD_ERR_NULL);
+    if ((do_pack && io->frame_bytes < 1) || (do_unpack && io->out_frame_bytes < 1) || io->block_capacity < 1 ||
+        io->block_capacity > 0x7fffffffLL)
+        return fail(BLOAD_ERR_ARG);
+    if (do_pack && (!aligned(io->d_dense, 16) || !aligned(io->d_store, 16))) return fail(BLOAD_ERR_ALIGN);
+    if (do_unpack && (!aligned(io->d_dense_out, 16) || !aligned(io->d_ragged_out, 16))) return fail(BLOAD_ERR_ALIGN);
+    if (!aligned(io->d_seq_id, 4) || !aligned(io->d_pos, 4)) return fail(BLOAD_ERR_ALIGN);
+    bload_sizes_t sz;
+    plan_layout(n, &sz);
+    WorkView wv;
+    EpochView ev;
+    size_t need_work = work_layout(n, t_block, d_work, &wv);
+    need_work += epoch_layout(t_block, static_cast<char*>(d_work) + need_work, &ev);
+    if (plan_bytes < sz.plan_bytes || work_bytes < need_work) return fail(BLOAD_ERR_WORKSPACE);
+    if (!aligned(d_plan, kAlign) || !aligned(d_work, kAlign) || !aligned(d_lengths, 4)) return fail(BLOAD_ERR_ALIGN);
+
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    cudaStream_t side = side_stream ? static_cast<cudaStream_t>(side_stream) : st;
+    PlanView pv = plan_view(d_plan, n);
+    const int32_t cap = (int32_t)io->block_capacity;
+    // chunks of about 1,250 draws: fine enough that the last chunk's copies are a small tail, coarse enough that
+    // the launches and the hand-over of the fill rule's tables (a few microseconds per chunk) stay negligible
+    int chunks = (int)(n / 1250);
+    if (chunks < 1) chunks = 1;
+    if (chunks > 16) chunks = 16;
+    const bool timing = g_timing;
+    g_have_epoch_times = false;
+
+    // events: one per chunk to hand its blocks to the side stream, one to join; with timing, 2 + 5 more per chunk
+    constexpr int kPer = 8;
+    cudaEvent_t evs[kMaxEpochChunks * kPer + 1];
+    int n_ev = 0;
+    auto new_event = [&](bool timed) -> cudaEvent_t {
+        cudaEvent_t e = nullptr;
+        if (cudaEventCreateWithFlags(&e, timed ? cudaEventDefault : cudaEventDisableTiming) != cudaSuccess) return nullptr;
+        evs[n_ev++] = e;
+        return e;
+    };
+    auto destroy_events = [&]() { for (int i = 0; i < n_ev; ++i) cudaEventDestroy(evs[i]); };
+    struct ChunkEv { cudaEvent_t f0, f1, ready, t0, t1, t2, t3, t4; } ce_[kMaxEpochChunks];
+
+    cudaError_t ce = cudaMemsetAsync(ev.resume, 0, sizeof(FillResume), st);
+    int32_t* sorted_id = nullptr;
+    if (ce == cudaSuccess)
+        ce = launch_plan_front(d_lengths, n, t_block, seed, BLOAD_POLICY_UNIFORM_SEQUENCES, pv, wv, st, &sorted_id);
+    const int64_t dense_total = do_unpack ? io->block_capacity * (int64_t)t_block * io->out_frame_bytes : 0;
+    for (int c = 0; c < chunks && ce == cudaSuccess; ++c) {
+        ChunkEv& E = ce_[c];
+        E = ChunkEv{};
+        if (timing) { E.f0 = new_event(true); E.f1 = new_event(true); }
+        E.ready = new_event(false);
+        if (timing) { E.t0 = new_event(true); E.t1 = new_event(true); E.t2 = new_event(true); E.t3 = new_event(true); E.t4 = new_event(true); }
+        if (!E.ready || (timing && (!E.f0 || !E.f1 || !E.t0 || !E.t1 || !E.t2 || !E.t3 || !E.t4))) { ce = cudaErrorMemoryAllocation; break; }
+        const int32_t k_target = c + 1 == chunks ? (int32_t)n : (int32_t)((n * (c + 1)) / chunks);
+        if (timing) cudaEventRecord(E.f0, st);
+        ce = launch_fill_chunk(pv, wv, ev, n, t_block, k_target, cap, st);
+        if (timing) cudaEventRecord(E.f1, st);
+        if (ce != cudaSuccess) break;
+        cudaEventRecord(E.ready, st);
+        if (side != st) cudaStreamWaitEvent(side, E.ready, 0);
+        const int32_t* d_blocks = ev.resume->range[c];
+        const int32_t* d_draws = ev.resume->draw[c];
+        if (timing) cudaEventRecord(E.t0, side);
+        ce = launch_tables_chunk(pv, wv, sorted_id, n, d_draws, side);
+        if (timing) cudaEventRecord(E.t1, side);
+        if (ce == cudaSuccess && do_meta)
+            ce = launch_metadata(pv, t_block, 0, 0, io->d_seq_id, io->d_pos, io->d_reset, io->d_valid, side, d_blocks);
+        if (timing) cudaEventRecord(E.t2, side);
+        if (ce == cudaSuccess && do_pack)
+            ce = launch_copy_range(false, pv, t_block, io->frame_bytes, static_cast<const uint8_t*>(io->d_store),
+                                   static_cast<uint8_t*>(io->d_dense), 0 /*taken from the plan on the device*/, io->pad_byte, d_blocks, side);
+        if (timing) cudaEventRecord(E.t3, side);
+        if (ce == cudaSuccess && do_unpack)
+            ce = launch_copy_range(true, pv, t_block, io->out_frame_bytes, static_cast<const uint8_t*>(io->d_dense_out),
+                                   static_cast<uint8_t*>(io->d_ragged_out), dense_total, 0, d_blocks, side);
+        if (timing) cudaEventRecord(E.t4, side);
+    }
+    // filler blocks between the end of the plan and the end of the caller's buffers, then the plan is complete
+    if (ce == cudaSuccess) {
+        const int32_t* d_tail = ev.resume->range[kMaxEpochChunks];
+        if (do_meta) ce = launch_metadata(pv, t_block, 0, 0, io->d_seq_id, io->d_pos, io->d_reset, io->d_valid, side, d_tail);
+        if (ce == cudaSuccess && do_pack)
+            ce = launch_copy_range(false, pv, t_block, io->frame_bytes, static_cast<const uint8_t*>(io->d_store),
+                                   static_cast<uint8_t*>(io->d_dense), 0, io->pad_byte, d_tail, side);
+        if (ce == cudaSuccess) ce = launch_plan_finish(pv, side);
+    }
+    if (ce == cudaSuccess && side != st) {
+        cudaEvent_t join = new_event(false);
+        if (!join) ce = cudaErrorMemoryAllocation;
+        else { cudaEventRecord(join, side); cudaStreamWaitEvent(st, join, 0); }
+    }
+    PlanHeader h;
+    if (ce == cudaSuccess) ce = cudaMemcpyAsync(&h, pv.hdr, sizeof h, cudaMemcpyDeviceToHost, st);
+    if (ce == cudaSuccess) ce = cudaStreamSynchronize(st);
+    if (ce != cudaSuccess) {
+        (void)cudaGetLastError();
+        cudaStreamSynchronize(side); cudaStreamSynchronize(st);  // nothing may still use the events
+        destroy_events();
+        return fail(BLOAD_ERR_CUDA);
+    }
+    if (timing) {
+        for (int i = 0; i < 5; ++i) g_epoch_ms[i] = 0.f;
+        for (int c = 0; c < chunks; ++c) {
+            float ms = 0.f;
+            const ChunkEv& E = ce_[c];
+            if (cudaEventElapsedTime(&ms, E.f0, E.f1) == cudaSuccess) g_epoch_ms[0] += ms;
+            if (cudaEventElapsedTime(&ms, E.t0, E.t1) == cudaSuccess) g_epoch_ms[1] += ms;
+            if (cudaEventElapsedTime(&ms, E.t1, E.t2) == cudaSuccess) g_epoch_ms[2] += ms;
+            if (cudaEventElapsedTime(&ms, E.t2, E.t3) == cudaSuccess) g_epoch_ms[3] += ms;
+            if (cudaEventElapsedTime(&ms, E.t3, E.t4) == cudaSuccess) g_epoch_ms[4] += ms;
+        }
+        g_have_epoch_times = true;
+    }
+    destroy_events();
+    info->status = h.status;
+    info->n_blocks = h.n_blocks;
+    info->sum_t = h.sum_t;
+    info->t_max = h.t_max;
+    info->first_bad_index = h.first_bad == ~0ULL ? -1 : (int64_t)h.first_bad;
+    info->checksum = h.checksum;
+    info->max_segs_per_block = h.max_segs;
+    if (h.status == BLOAD_OK && h.magic != kPlanMagic) return fail(BLOAD_ERR_PLAN);
+    if (h.status == BLOAD_OK && h.n_blocks > io->block_capacity) return BLOAD_ERR_WORKSPACE;  // the plan itself is complete
     return info->status;
 }
 

@@ -23,17 +23,27 @@ namespace {
 
 using namespace wc;
 
+// `range` (device, or null): {first block, end block, end of the real blocks} replaces block_begin / block_count /
+// n_blocks when the blocks of a launch are decided on the device (a plan that is still being built); `out_base` is
+// the block that the first row of the dense buffer holds.
 template <bool UNPACK>
 __global__ void __launch_bounds__(256) k7_copy(PlanView pv, int32_t t_block, int64_t frame_bytes, int64_t block_begin,
                                                int64_t block_count, const uint8_t* __restrict__ src_base,
                                                uint8_t* __restrict__ dst_base, int64_t src_total_bytes,
-                                               int64_t sub_bytes, int64_t subs_per_block, uint8_t pad)
+                                               int64_t sub_bytes, int64_t subs_per_block, uint8_t pad,
+                                               const int32_t* __restrict__ range, int64_t out_base)
 {
     const int lane = threadIdx.x & 31;
     const int64_t warps = ((int64_t)gridDim.x * blockDim.x) >> 5;
+    int64_t n_blocks;
+    if (range) {
+        block_begin = range[0]; block_count = range[1] - range[0]; n_blocks = range[2];
+        if (!UNPACK) src_total_bytes = pv.hdr->sum_t * frame_bytes;  // the host does not know the size of the store yet
+    } else {
+        n_blocks = pv.hdr->n_blocks;
+    }
     const int64_t items = block_count * subs_per_block;
     const int64_t block_bytes = (int64_t)t_block * frame_bytes;
-    const int64_t n_blocks = pv.hdr->n_blocks;
     const uint8_t* s_limit = src_base + src_total_bytes;
 
     for (int64_t item = (((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5); item < items; item += warps) {
@@ -41,7 +51,7 @@ __global__ void __launch_bounds__(256) k7_copy(PlanView pv, int32_t t_block, int
         const int64_t lo = (item - q * subs_per_block) * sub_bytes;
         const int64_t hi = min(lo + sub_bytes, block_bytes);
         const int64_t b = block_begin + q;
-        const int64_t dense_off = q * block_bytes;  // of this block inside the dense buffer
+        const int64_t dense_off = (b - out_base) * block_bytes;  // of this block inside the dense buffer
         int64_t cur = lo;
         if (b < n_blocks) {
             const int k0 = pv.block_seg_begin[b], k1 = pv.block_seg_begin[b + 1];
@@ -672,10 +682,28 @@ cudaError_t launch_copy(bool unpack, const PlanView& pv, int32_t t_block, int64_
     const unsigned grid = (unsigned)(want < 0x7fffffffLL ? want : 0x7fffffffLL);
     if (unpack)
         k7_copy<true><<<grid, 256, 0, st>>>(pv, t_block, frame_bytes, block_begin, block_count, dense, ragged_out,
-                                             block_count * block_bytes, sub, spb, pad_byte);
+                                             block_count * block_bytes, sub, spb, pad_byte, nullptr, block_begin);
     else
         k7_copy<false><<<grid, 256, 0, st>>>(pv, t_block, frame_bytes, block_begin, block_count, ragged_in, dense,
-                                              ragged_bytes, sub, spb, pad_byte);
+                                              ragged_bytes, sub, spb, pad_byte, nullptr, block_begin);
+    return cudaPeekAtLastError();
+}
+
+// Register-path copy of the blocks named by a device-side range (see k7_copy): a fixed grid whose warps loop, because
+// the host does not know how many blocks the range holds.  The dense buffer starts at block 0.
+cudaError_t launch_copy_range(bool unpack, const PlanView& pv, int32_t t_block, int64_t frame_bytes, const uint8_t* src,
+                              uint8_t* dst, int64_t src_total_bytes, uint8_t pad_byte, const int32_t* d_range,
+                              cudaStream_t st)
+{
+    const int64_t block_bytes = (int64_t)t_block * frame_bytes;
+    const int64_t sub = 16384;
+    const int64_t spb = (block_bytes + sub - 1) / sub;
+    const unsigned grid = 148 * 3 * 4;  // three CTAs of this kernel are resident per SM; four rounds of them
+    count_launches(1);
+    if (unpack)
+        k7_copy<true><<<grid, 256, 0, st>>>(pv, t_block, frame_bytes, 0, 0, src, dst, src_total_bytes, sub, spb, pad_byte, d_range, 0);
+    else
+        k7_copy<false><<<grid, 256, 0, st>>>(pv, t_block, frame_bytes, 0, 0, src, dst, src_total_bytes, sub, spb, pad_byte, d_range, 0);
     return cudaPeekAtLastError();
 }
 

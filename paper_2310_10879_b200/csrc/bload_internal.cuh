@@ -56,6 +56,23 @@ struct WorkView {
     int32_t* bucket_end;  // [t_block + 1] sequences with length <= l
 };
 
+// State of a fill rule that runs in several launches (bload_epoch): where the chain stands, and for every launch
+// ("chunk") the blocks and draws it completed.  Lives in the scratch buffer, zeroed before the first chunk.
+constexpr int kMaxEpochChunks = 32;
+struct FillResume {
+    int32_t k, b, room, start;               // next draw, open block, room left in it, its next free slot
+    int32_t done, chunk;                     // all sequences placed; chunks run so far
+    int32_t pad_[2];
+    int32_t range[kMaxEpochChunks + 1][4];   // per chunk {first block, end block, end of the real blocks, 0}, clamped to
+                                             // the caller's capacity; row kMaxEpochChunks: the filler blocks behind the plan
+    int32_t draw[kMaxEpochChunks + 1][4];    // per chunk {first draw, end draw, first block, end block} (not clamped)
+};
+struct EpochView {
+    FillResume* resume;
+    int32_t* fill_tables;  // snapshot of the fill rule's shared-memory tables between chunks
+};
+size_t epoch_layout(int32_t t_block, void* base, EpochView* v);
+
 constexpr int kChunk = 2048;  // elements per CTA in scan / sort kernels (256 threads x 8)
 
 inline size_t align_up(size_t x, size_t a = kAlign) { return (x + a - 1) / a * a; }
@@ -98,10 +115,25 @@ cudaError_t launch_plan(const int32_t* d_lengths, int64_t n, int32_t t_block, ui
                         const PlanView& pv, const WorkView& wv, cudaStream_t st, cudaEvent_t* ev /*5 or null*/,
                         const BfdView* bv = nullptr /*policy 2 only*/);
 cudaError_t launch_metadata(const PlanView& pv, int32_t t_block, int64_t block_begin, int64_t block_count,
-                            int32_t* seq_id, int32_t* pos, uint8_t* reset, uint8_t* valid, cudaStream_t st);
+                            int32_t* seq_id, int32_t* pos, uint8_t* reset, uint8_t* valid, cudaStream_t st,
+                            const int32_t* d_range = nullptr);
 cudaError_t launch_copy(bool unpack, const PlanView& pv, int32_t t_block, int64_t frame_bytes, int64_t block_begin,
                         int64_t block_count, const uint8_t* ragged_in, uint8_t* dense, uint8_t* ragged_out,
                         int64_t ragged_bytes, uint8_t pad_byte, cudaStream_t st, int64_t n, int64_t n_blocks);
+// The pieces of the planner and the copies that bload_epoch strings together on two streams.  `d_range` points to
+// {first block, end block, end of the real blocks} in device memory: the blocks a launch covers are decided on the
+// device, so these launches use fixed grids whose CTAs loop.
+cudaError_t launch_plan_front(const int32_t* d_lengths, int64_t n, int32_t t_block, uint64_t seed, uint32_t policy,
+                              const PlanView& pv, const WorkView& wv, cudaStream_t st, int32_t** sorted_id);
+cudaError_t launch_fill_chunk(const PlanView& pv, const WorkView& wv, const EpochView& ev, int64_t n, int32_t t_block,
+                              int32_t k_target, int32_t filler_end, cudaStream_t st);
+cudaError_t launch_tables_chunk(const PlanView& pv, const WorkView& wv, const int32_t* sorted_id, int64_t n,
+                                const int32_t* d_draw_range /*{first draw, end draw, first block, end block}*/,
+                                cudaStream_t st);
+cudaError_t launch_plan_finish(const PlanView& pv, cudaStream_t st);
+cudaError_t launch_copy_range(bool unpack, const PlanView& pv, int32_t t_block, int64_t frame_bytes, const uint8_t* src,
+                              uint8_t* dst, int64_t src_total_bytes, uint8_t pad_byte, const int32_t* d_range,
+                              cudaStream_t st);
 
 cudaError_t launch_var_offsets(const int32_t* lengths, const int32_t* frame_bytes, int64_t n, int64_t* out, cudaStream_t st);
 cudaError_t launch_copy_var(bool unpack, const PlanView& pv, int32_t t_block, int64_t slot_bytes, int64_t block_begin,

@@ -18,11 +18,15 @@ template <bool VEC>
 __global__ void __launch_bounds__(kMetaThreads) k6_metadata(PlanView pv, int32_t t_block, int64_t block_begin,
                                                             int32_t block_count, int32_t* __restrict__ seq_id,
                                                             int32_t* __restrict__ pos, uint8_t* __restrict__ reset,
-                                                            uint8_t* __restrict__ valid)
+                                                            uint8_t* __restrict__ valid, const int32_t* __restrict__ range)
 {
     const int s0 = (int)blockIdx.x * kMetaChunk + (int)threadIdx.x * 4;
     if (s0 >= t_block) return;
-    const int64_t n_blocks = pv.hdr->n_blocks;
+    // `range` (device, or null): {first block, end block, end of the real blocks} of a plan that is still being built;
+    // the outputs then start at block 0
+    int64_t n_blocks, out_base = block_begin;
+    if (range) { block_begin = range[0]; block_count = range[1] - range[0]; n_blocks = range[2]; out_base = 0; }
+    else n_blocks = pv.hdr->n_blocks;
     const int32_t* __restrict__ seg_start = pv.seg_start;
     for (int q = blockIdx.y; q < block_count; q += gridDim.y) {
         const int64_t b = block_begin + q;
@@ -70,7 +74,7 @@ __global__ void __launch_bounds__(kMetaThreads) k6_metadata(PlanView pv, int32_t
                 }
             }
         }
-        const int64_t o = (int64_t)q * t_block + s0;
+        const int64_t o = (b - out_base) * t_block + s0;
         if (VEC) {  // t_block % 4 == 0 and aligned outputs: one vector per array
             if (seq_id) __stcs(reinterpret_cast<int4*>(seq_id + o), make_int4(sid[0], sid[1], sid[2], sid[3]));
             if (pos) __stcs(reinterpret_cast<int4*>(pos + o), make_int4(ps[0], ps[1], ps[2], ps[3]));
@@ -93,20 +97,22 @@ __global__ void __launch_bounds__(kMetaThreads) k6_metadata(PlanView pv, int32_t
 }  // namespace
 
 cudaError_t launch_metadata(const PlanView& pv, int32_t t_block, int64_t block_begin, int64_t block_count,
-                            int32_t* seq_id, int32_t* pos, uint8_t* reset, uint8_t* valid, cudaStream_t st)
+                            int32_t* seq_id, int32_t* pos, uint8_t* reset, uint8_t* valid, cudaStream_t st,
+                            const int32_t* d_range)
 {
-    if (block_count == 0) return cudaSuccess;
+    if (block_count == 0 && !d_range) return cudaSuccess;
     auto al = [](const void* p, uintptr_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; };
     const unsigned chunks = (unsigned)((t_block + kMetaChunk - 1) / kMetaChunk);
     // enough CTAs in flight to cover the machine several times over; beyond that a CTA loops over blocks
     int64_t rows = (148 * 64 + chunks - 1) / chunks;
-    if (rows > block_count) rows = block_count;
+    if (rows > block_count && !d_range) rows = block_count;
+    if (d_range && rows > 256) rows = 256;  // a chunk of a plan in progress holds a few blocks
     if (rows > 65535) rows = 65535;
     const dim3 grid(chunks, (unsigned)rows);
     if (t_block % 4 == 0 && al(seq_id, 16) && al(pos, 16) && al(reset, 4) && al(valid, 4))
-        k6_metadata<true><<<grid, kMetaThreads, 0, st>>>(pv, t_block, block_begin, (int32_t)block_count, seq_id, pos, reset, valid);
+        k6_metadata<true><<<grid, kMetaThreads, 0, st>>>(pv, t_block, block_begin, (int32_t)block_count, seq_id, pos, reset, valid, d_range);
     else
-        k6_metadata<false><<<grid, kMetaThreads, 0, st>>>(pv, t_block, block_begin, (int32_t)block_count, seq_id, pos, reset, valid);
+        k6_metadata<false><<<grid, kMetaThreads, 0, st>>>(pv, t_block, block_begin, (int32_t)block_count, seq_id, pos, reset, valid, d_range);
     count_launches(1);
     return cudaPeekAtLastError();
 }

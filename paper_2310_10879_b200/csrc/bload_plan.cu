@@ -305,9 +305,16 @@ __global__ void __launch_bounds__(256) k3_buckets(const uint64_t* __restrict__ k
 constexpr int kQ1Off = 36, kRingOff = kQ1Off + 32 * 33, kQ2Off = kRingOff + 128;  // in 32-bit words; ring 16-byte aligned
 static_assert(kRingOff % 4 == 0, "ring alignment");
 
+//
+// RESUME: the chain runs in several launches ("chunks") so that blocks which are already closed can be packed on
+// another stream while later ones are still being built.  A chunk stops at the first block that closes at or after
+// draw `k_target`, leaves its position in `rs` and its count tables in `snap`, and records the blocks and draws it
+// covered; the next launch picks both up.  Without RESUME the kernel is the single launch it always was.
+template <bool RESUME>
 __global__ void __launch_bounds__(256, 1) k4_fill(PlanView pv, const int32_t* __restrict__ bucket_end,
                                                   const uint64_t* __restrict__ draw_u, int4* __restrict__ draw_rec,
-                                                  int64_t n64, int32_t L)
+                                                  int64_t n64, int32_t L, FillResume* __restrict__ rs,
+                                                  int32_t* __restrict__ snap, int32_t k_target, int32_t filler_end)
 {
     extern __shared__ __align__(16) int32_t sm[];
     int32_t* Q0 = sm;                                      // [33]
@@ -316,25 +323,44 @@ __global__ void __launch_bounds__(256, 1) k4_fill(PlanView pv, const int32_t* __
     int32_t* Q2 = sm + kQ2Off;                             // [rows][33], rows = ceil(L / 32)
     if (pv.hdr->first_bad != kNoBad) return;
     const int rows = (L + 31) >> 5;
-    auto upto = [&](int l) { return bucket_end[min(l, L)]; };  // sequences with length <= l
-    for (int idx = threadIdx.x; idx < rows * 32; idx += blockDim.x)
-        Q2[(idx >> 5) * 33 + (idx & 31) + 1] = upto(idx + 1) - upto(idx & ~31);
-    for (int r = threadIdx.x; r < rows; r += blockDim.x) Q2[r * 33] = 0;
-    for (int idx = threadIdx.x; idx < 1024; idx += blockDim.x)
-        Q1[(idx >> 5) * 33 + (idx & 31) + 1] = upto((idx + 1) << 5) - upto((idx >> 5) << 10);
-    if (threadIdx.x < 32) { Q1[threadIdx.x * 33] = 0; Q0[threadIdx.x + 1] = upto((threadIdx.x + 1) << 10); }
-    if (threadIdx.x == 0) Q0[0] = 0;
+    const int chunk = RESUME ? rs->chunk : 0;
+    if (RESUME && rs->done) {  // an earlier chunk placed the last sequence: this one covers nothing
+        __syncthreads();       // every thread has read the state before thread 0 changes it
+        if (threadIdx.x == 0) {
+            const int e = rs->range[chunk - 1][1], d = rs->draw[chunk - 1][1], eb = rs->draw[chunk - 1][3];
+            rs->range[chunk][0] = e; rs->range[chunk][1] = e; rs->range[chunk][2] = e;
+            rs->draw[chunk][0] = d; rs->draw[chunk][1] = d; rs->draw[chunk][2] = eb; rs->draw[chunk][3] = eb;
+            rs->chunk = chunk + 1;
+        }
+        return;
+    }
+    if (RESUME && chunk > 0) {
+        const int words = kQ2Off + rows * 33;
+        for (int i = threadIdx.x; i < words; i += blockDim.x) sm[i] = snap[i];
+    } else {
+        auto upto = [&](int l) { return bucket_end[min(l, L)]; };  // sequences with length <= l
+        for (int idx = threadIdx.x; idx < rows * 32; idx += blockDim.x)
+            Q2[(idx >> 5) * 33 + (idx & 31) + 1] = upto(idx + 1) - upto(idx & ~31);
+        for (int r = threadIdx.x; r < rows; r += blockDim.x) Q2[r * 33] = 0;
+        for (int idx = threadIdx.x; idx < 1024; idx += blockDim.x)
+            Q1[(idx >> 5) * 33 + (idx & 31) + 1] = upto((idx + 1) << 5) - upto((idx >> 5) << 10);
+        if (threadIdx.x < 32) { Q1[threadIdx.x * 33] = 0; Q0[threadIdx.x + 1] = upto((threadIdx.x + 1) << 10); }
+        if (threadIdx.x == 0) Q0[0] = 0;
+    }
+    int k = 0, b = 0, room = L, start = 0;
+    if (RESUME && chunk > 0) { k = rs->k; b = rs->b; room = rs->room; start = rs->start; }
     __syncthreads();
     if (threadIdx.x >= 32) return;
 
     const int lane = threadIdx.x;
     const int n = (int)n64;
     int q0 = Q0[lane + 1];
-    int k = 0, b = 0, room = L, start = 0;
-    if (lane == 0) pv.block_seg_begin[0] = 0;
+    const int k_first = k, b_first = b;
+    int flush_from = k & 31;  // records of the first group below this lane were written by the previous chunk
+    if (lane == 0 && k == 0) pv.block_seg_begin[0] = 0;
     // random words of 32 draws at a time, one per lane, the next 32 prefetched
-    uint64_t u_cur = lane < n ? draw_u[lane] : 0;
-    uint64_t u_nxt = 32 + lane < n ? draw_u[32 + lane] : 0;
+    uint64_t u_cur = (k & ~31) + lane < n ? draw_u[(k & ~31) + lane] : 0;
+    uint64_t u_nxt = (k & ~31) + 32 + lane < n ? draw_u[(k & ~31) + 32 + lane] : 0;
     while (k < n) {
         const uint64_t u = __shfl_sync(kFull, u_cur, k & 31);
         const int y = room - 1, ya = y >> 10, yr = y >> 5;
@@ -342,6 +368,7 @@ __global__ void __launch_bounds__(256, 1) k4_fill(PlanView pv, const int32_t* __
         if (m == 0) {  // nothing fits: the rest of the block is padding
             if (lane == 0) { pv.block_fill[b] = start; pv.block_seg_begin[b + 1] = k; }
             ++b; room = L; start = 0;
+            if (RESUME && k >= k_target) break;
             continue;
         }
         // j = floor(u * m / 2^64), m < 2^31, from 32-bit pieces
@@ -369,17 +396,40 @@ __global__ void __launch_bounds__(256, 1) k4_fill(PlanView pv, const int32_t* __
         __syncwarp();
         room -= len; start += len; ++k;
         if ((k & 31) == 0) {
-            draw_rec[k - 32 + lane] = ring[lane];
+            if (!RESUME || lane >= flush_from) draw_rec[k - 32 + lane] = ring[lane];
+            flush_from = 0;
             u_cur = u_nxt;
             u_nxt = k + 32 + lane < n ? draw_u[k + 32 + lane] : 0;
             __syncwarp();
         }
     }
-    if (lane < (n & 31)) draw_rec[(n & ~31) + lane] = ring[lane];
-    if (lane == 0) {
+    if (lane < (k & 31) && lane >= flush_from) draw_rec[(k & ~31) + lane] = ring[lane];
+    const bool finished = k == n;
+    if (finished && lane == 0) {
         pv.block_fill[b] = start;
         pv.block_seg_begin[b + 1] = k;
         pv.hdr->n_blocks = b + 1;
+    }
+    if (RESUME) {
+        const int closed = finished ? b + 1 : b;  // blocks [b_first, closed) are complete now
+        __syncwarp();
+        const int words = kQ2Off + rows * 33;
+        if (!finished)
+            for (int i = lane; i < words; i += 32) snap[i] = sm[i];
+        if (lane == 0) {
+            rs->k = k; rs->b = b; rs->room = room; rs->start = start;
+            rs->done = finished ? 1 : 0;
+            // what the copies may touch is clamped to the rows the caller's buffers have (filler_end)
+            const int lo_c = min(b_first, filler_end), hi_c = min(closed, filler_end);
+            rs->range[chunk][0] = lo_c; rs->range[chunk][1] = hi_c; rs->range[chunk][2] = hi_c;
+            rs->draw[chunk][0] = k_first; rs->draw[chunk][1] = k; rs->draw[chunk][2] = b_first; rs->draw[chunk][3] = closed;
+            rs->chunk = chunk + 1;
+            if (finished) {  // the filler blocks between the end of the plan and the end of the caller's buffers
+                rs->range[kMaxEpochChunks][0] = hi_c;
+                rs->range[kMaxEpochChunks][1] = filler_end;
+                rs->range[kMaxEpochChunks][2] = hi_c;
+            }
+        }
     }
 }
 
@@ -492,18 +542,23 @@ __device__ __forceinline__ uint64_t fmix64(uint64_t x)
     return x;
 }
 
-// resolve draws to sequence ids; segment list, inverse tables, digest, widest block
+// resolve draws to sequence ids; segment list, inverse tables, digest, widest block.  With `draw_range` the kernel
+// covers the draws [draw_range[0], draw_range[1]) and the blocks [draw_range[2], draw_range[3]) of one chunk of
+// a plan that is still being built (every block has at least one draw, so the draw index doubles as block index).
 __global__ void __launch_bounds__(256) k5_tables(PlanView pv, const int4* __restrict__ draw_rec,
                                                  const int32_t* __restrict__ bucket_end,
-                                                 const int32_t* __restrict__ sorted_id, int64_t n)
+                                                 const int32_t* __restrict__ sorted_id, int64_t n,
+                                                 const int32_t* __restrict__ draw_range)
 {
     __shared__ unsigned long long s_sum[8];
     __shared__ int s_max[8];
     if (pv.hdr->first_bad != kNoBad) return;
-    const int64_t k = (int64_t)blockIdx.x * 256 + threadIdx.x;
+    const int64_t k_lo = draw_range ? draw_range[0] : 0, k_hi = draw_range ? draw_range[1] : n;
+    const int64_t b_lo = draw_range ? draw_range[2] : 0;
+    const int64_t b_hi = draw_range ? draw_range[3] : pv.hdr->n_blocks;
     unsigned long long term = 0;
     int segs = 0;
-    if (k < n) {
+    for (int64_t k = k_lo + (int64_t)blockIdx.x * 256 + threadIdx.x; k < k_hi; k += (int64_t)gridDim.x * 256) {
         int4 r = draw_rec[k];
         int id = sorted_id[bucket_end[r.x] - r.y];
         pv.seg_seq[k] = id;
@@ -513,8 +568,9 @@ __global__ void __launch_bounds__(256) k5_tables(PlanView pv, const int4* __rest
         pv.seq_block[id] = r.z;
         pv.seq_start[id] = r.w;
         uint64_t where = ((uint64_t)(uint32_t)r.z << 32) | (uint64_t)(uint32_t)r.w;
-        term = fmix64(where * 0x9E3779B97F4A7C15ULL + (uint64_t)(uint32_t)id);
-        if (k < pv.hdr->n_blocks) segs = pv.block_seg_begin[k + 1] - pv.block_seg_begin[k];
+        term += fmix64(where * 0x9E3779B97F4A7C15ULL + (uint64_t)(uint32_t)id);
+        const int64_t b = b_lo + (k - k_lo);
+        if (b < b_hi) segs = max(segs, pv.block_seg_begin[b + 1] - pv.block_seg_begin[b]);
     }
 #pragma unroll
     for (int d = 16; d; d >>= 1) {
@@ -526,8 +582,8 @@ __global__ void __launch_bounds__(256) k5_tables(PlanView pv, const int4* __rest
     __syncthreads();
     if (threadIdx.x == 0) {
         for (int i = 1; i < 8; ++i) { term += s_sum[i]; segs = max(segs, s_max[i]); }
-        atomicAdd(&pv.hdr->checksum, term);
-        atomicMax(&pv.hdr->max_segs, segs);
+        if (term) atomicAdd(&pv.hdr->checksum, term);
+        if (segs) atomicMax(&pv.hdr->max_segs, segs);
     }
 }
 
@@ -591,8 +647,24 @@ cudaError_t plan_key_buckets(const uint64_t* sorted_keys, int64_t n, int32_t max
     return cudaPeekAtLastError();
 }
 
-cudaError_t launch_plan(const int32_t* d_lengths, int64_t n, int32_t t_block, uint64_t seed, uint32_t policy,
-                        const PlanView& pv, const WorkView& wv, cudaStream_t st, cudaEvent_t* ev, const BfdView* bv)
+size_t epoch_layout(int32_t t_block, void* base, EpochView* v)
+{
+    size_t off = 0;
+    auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes); return o; };
+    const size_t o_rs = take(sizeof(FillResume));
+    const size_t o_tab = take(sizeof(int32_t) * (kQ2Off + (size_t)((t_block + 31) / 32) * 33));
+    if (v) {
+        char* b = static_cast<char*>(base);
+        v->resume = reinterpret_cast<FillResume*>(b + o_rs);
+        v->fill_tables = reinterpret_cast<int32_t*>(b + o_tab);
+    }
+    return off;
+}
+
+// validate + scan + keys + key sort + buckets; *sorted_id receives the array of ids sorted by (T, h)
+cudaError_t launch_plan_front(const int32_t* d_lengths, int64_t n, int32_t t_block, uint64_t seed, uint32_t policy,
+                              const PlanView& pv, const WorkView& wv, cudaStream_t st, int32_t** sorted_id,
+                              uint64_t** sorted_key, cudaEvent_t* ev)
 {
     const int64_t chunks = chunks_of(n);
     const unsigned gc = (unsigned)chunks;
@@ -619,23 +691,75 @@ cudaError_t launch_plan(const int32_t* d_lengths, int64_t n, int32_t t_block, ui
     }
     k3_buckets<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(kin, n, t_block, wv.bucket_end, pv.hdr);
     if (ev) cudaEventRecord(ev[2], st);
+    count_launches(4 + 3 * passes + 1);
+    *sorted_id = iin;
+    if (sorted_key) *sorted_key = kin;
+    return cudaPeekAtLastError();
+}
 
+cudaError_t launch_plan_front(const int32_t* d_lengths, int64_t n, int32_t t_block, uint64_t seed, uint32_t policy,
+                              const PlanView& pv, const WorkView& wv, cudaStream_t st, int32_t** sorted_id)
+{
+    return launch_plan_front(d_lengths, n, t_block, seed, policy, pv, wv, st, sorted_id, nullptr, nullptr);
+}
+
+static size_t fill_smem_bytes(int32_t t_block) { return sizeof(int32_t) * (kQ2Off + (size_t)((t_block + 31) / 32) * 33); }
+
+cudaError_t launch_fill_chunk(const PlanView& pv, const WorkView& wv, const EpochView& ev, int64_t n, int32_t t_block,
+                              int32_t k_target, int32_t filler_end, cudaStream_t st)
+{
+    const size_t smem = fill_smem_bytes(t_block);
+    cudaError_t e = cudaFuncSetAttribute(k4_fill<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    k4_fill<true><<<1, 256, smem, st>>>(pv, wv.bucket_end, wv.draw_u, wv.draw_rec, n, t_block, ev.resume, ev.fill_tables,
+                                         k_target, filler_end);
+    count_launches(1);
+    return cudaPeekAtLastError();
+}
+
+cudaError_t launch_tables_chunk(const PlanView& pv, const WorkView& wv, const int32_t* sorted_id, int64_t n,
+                                const int32_t* d_draw_range, cudaStream_t st)
+{
+    const int64_t want = (n + 255) / 256;
+    k5_tables<<<(unsigned)(want < 592 ? want : 592), 256, 0, st>>>(pv, wv.draw_rec, wv.bucket_end, sorted_id, n, d_draw_range);
+    count_launches(1);
+    return cudaPeekAtLastError();
+}
+
+cudaError_t launch_plan_finish(const PlanView& pv, cudaStream_t st)
+{
+    k5_finish<<<1, 32, 0, st>>>(pv.hdr);
+    count_launches(1);
+    return cudaPeekAtLastError();
+}
+
+cudaError_t launch_plan(const int32_t* d_lengths, int64_t n, int32_t t_block, uint64_t seed, uint32_t policy,
+                        const PlanView& pv, const WorkView& wv, cudaStream_t st, cudaEvent_t* ev, const BfdView* bv)
+{
+    int32_t* iin = nullptr;
+    uint64_t* kin = nullptr;
+    cudaError_t e = launch_plan_front(d_lengths, n, t_block, seed, policy, pv, wv, st, &iin, &kin, ev);
+    if (e != cudaSuccess) return e;
     if (policy == BLOAD_POLICY_BEST_FIT_DECREASING) {  // a different planner from here on (see bload_bfd.cu)
-        count_launches(4 + 3 * passes + 1);
         cudaError_t eb = bv ? launch_bfd(pv, wv, *bv, kin, iin, n, t_block, st) : cudaErrorInvalidValue;
         if (ev) { cudaEventRecord(ev[3], st); cudaEventRecord(ev[4], st); }
         return eb;
     }
-    const size_t smem = sizeof(int32_t) * (kQ2Off + (size_t)((t_block + 31) / 32) * 33);
-    auto fill = policy == BLOAD_POLICY_UNIFORM_LENGTHS ? k4_fill_lengths : k4_fill;
-    cudaError_t e = cudaFuncSetAttribute(fill, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
-    fill<<<1, 256, smem, st>>>(pv, wv.bucket_end, wv.draw_u, wv.draw_rec, n, t_block);
+    const size_t smem = fill_smem_bytes(t_block);
+    if (policy == BLOAD_POLICY_UNIFORM_LENGTHS) {
+        e = cudaFuncSetAttribute(k4_fill_lengths, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        k4_fill_lengths<<<1, 256, smem, st>>>(pv, wv.bucket_end, wv.draw_u, wv.draw_rec, n, t_block);
+    } else {
+        e = cudaFuncSetAttribute(k4_fill<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        k4_fill<false><<<1, 256, smem, st>>>(pv, wv.bucket_end, wv.draw_u, wv.draw_rec, n, t_block, nullptr, nullptr, 0, 0);
+    }
     if (ev) cudaEventRecord(ev[3], st);
 
-    k5_tables<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(pv, wv.draw_rec, wv.bucket_end, iin, n);
+    k5_tables<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(pv, wv.draw_rec, wv.bucket_end, iin, n, nullptr);
     k5_finish<<<1, 32, 0, st>>>(pv.hdr);
-    count_launches(4 + 3 * passes + 1 + 1 + 2);
+    count_launches(1 + 2);
     if (ev) cudaEventRecord(ev[4], st);
     return cudaPeekAtLastError();
 }
