@@ -367,6 +367,40 @@ def run_gpu(args, w) -> dict:
                      "eight_plans_side_by_side_ms": t8, "plans_per_s": 8e3 / t8}
         del bufs, work2, jobs8
 
+    # ---- the whole step as ONE call (bload_epoch): the fill rule in chunks on this stream, tables, metadata, pack and
+    # unpack of the blocks each chunk has closed on a side stream under the next chunk
+    fused = None
+    if not args.no_fused:
+        side2 = torch.cuda.Stream()
+        chain = torch.cuda.Stream(priority=-1)  # the chain's single CTA goes ahead of queued copy CTAs
+
+        def fused_step():
+            chain.wait_stream(torch.cuda.current_stream())
+            p = B.bload_epoch(d_len, tb, w.seed, nb, store=store, frame_bytes=fb, dense=dense, seq_id=seq_id, pos=pos,
+                              reset=reset, valid=valid, dense_out=dense_out, out_frame_bytes=ofb, ragged_out=ragged_out,
+                              stream=chain, side_stream=side2, work=work, plan_buf=plan_buf)
+            return B.bload_stats(p.info)
+        for _ in range(max(3, args.warmup)):
+            fused_step()
+        barrier()
+        a, b_ = ev(), ev()
+        a.record()
+        for _ in range(args.steps):
+            fused_step()
+        b_.record()
+        barrier()
+        f_s = dist_max(a.elapsed_time(b_) / 1e3, dev) / args.steps
+        B.bload_set_plan_timing(True)
+        fused_step()
+        st_ms = B.bload_epoch_stage_times()
+        B.bload_set_plan_timing(False)
+        fused = {"ms_per_step": f_s * 1e3, "value": aggregate(by["pack"] + by["unpack"], world, f_s) / 1e9, "unit": UNIT,
+                 "steps": args.steps,
+                 "what": "bload_epoch: one call per step = plan + metadata + pack + unpack of the whole epoch, copies of "
+                         "finished blocks on a side stream while the fill rule is still running",
+                 "stage_ms_summed_over_chunks": {"fill": st_ms[0], "tables": st_ms[1], "metadata": st_ms[2],
+                                                 "pack": st_ms[3], "unpack": st_ms[4]}}
+
     # ---- batch-by-batch use: one pack call (metadata + dense) per training batch of w.batch_blocks blocks,
     # the last batch rounded up with filler blocks; the output buffers of one batch are reused
     bb = w.batch_blocks
@@ -594,7 +628,7 @@ def run_gpu(args, w) -> dict:
            "ms_per_step": step_s * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
            "dtype": "u8", "data": "synthetic", "config": config_of(w, {"parallelism": "replicas only"}),
            "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline,
-           "frames_per_s": aggregate(sum_t, world, step_s), "per_batch_pack": per_batch, "pipelined": pipelined, "consumer": consumer,
+           "frames_per_s": aggregate(sum_t, world, step_s), "per_batch_pack": per_batch, "pipelined": pipelined, "fused_epoch": fused, "consumer": consumer,
            "kernels": {
                "pack_copy": {"ms": pack_ms, "GB/s": by["pack"] / pack_ms / 1e6, "frac_measured": by["pack"] / pack_ms / 1e6 / peak,
                              "frac_nominal": by["pack"] / pack_ms / 1e6 / NOMINAL_HBM_GBS, "frames_per_s": sum_t / pack_ms * 1e3},
@@ -650,6 +684,7 @@ def main():
     ap.add_argument("--no-batch", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--no-consumer", action="store_true")
+    ap.add_argument("--no-fused", action="store_true")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "bload" else args.warmup
 

@@ -147,7 +147,11 @@ int bload_plan(const int32_t* d_lengths, int64_t n, int32_t t_block, uint64_t se
     WorkView wv;
     BfdView bv;
     size_t need_work = work_layout(n, t_block, d_work, &wv);  // the size bload_plan_sizes reports covers every policy
-    need_work += bfd_layout(n, t_block, static_cast<char*>(d_work) + need_work, &bv);
+    {
+        const size_t extra_bfd = bfd_layout(n, t_block, static_cast<char*>(d_work) + need_work, &bv);
+        const size_t extra_epoch = epoch_layout(t_block, nullptr, nullptr);
+        need_work += extra_bfd > extra_epoch ? extra_bfd : extra_epoch;
+    }
     if (plan_bytes < sz.plan_bytes || work_bytes < need_work) return fail(BLOAD_ERR_WORKSPACE);
     if (!aligned(d_plan, kAlign) || !aligned(d_work, kAlign) || !aligned(d_lengths, 4)) return fail(BLOAD_ERR_ALIGN);
 
@@ -195,7 +199,11 @@ int bload_plan_async(const int32_t* d_lengths, int64_t n, int32_t t_block, uint6
     WorkView wv;
     BfdView bv;
     size_t need_work = work_layout(n, t_block, d_work, &wv);  // the size bload_plan_sizes reports covers every policy
-    need_work += bfd_layout(n, t_block, static_cast<char*>(d_work) + need_work, &bv);
+    {
+        const size_t extra_bfd = bfd_layout(n, t_block, static_cast<char*>(d_work) + need_work, &bv);
+        const size_t extra_epoch = epoch_layout(t_block, nullptr, nullptr);
+        need_work += extra_bfd > extra_epoch ? extra_bfd : extra_epoch;
+    }
     if (plan_bytes < sz.plan_bytes || work_bytes < need_work) return BLOAD_ERR_WORKSPACE;
     if (!aligned(d_plan, kAlign) || !aligned(d_work, kAlign) || !aligned(d_lengths, 4)) return BLOAD_ERR_ALIGN;
     cudaError_t ce = launch_plan(d_lengths, n, t_block, seed, policy, plan_view(d_plan, n), wv,
@@ -264,7 +272,11 @@ int bload_epoch(const int32_t* d_lengths, int64_t n, int32_t t_block, uint64_t s
     WorkView wv;
     EpochView ev;
     size_t need_work = work_layout(n, t_block, d_work, &wv);
-    need_work += epoch_layout(t_block, static_cast<char*>(d_work) + need_work, &ev);
+    {
+        const size_t extra_epoch = epoch_layout(t_block, static_cast<char*>(d_work) + need_work, &ev);
+        const size_t extra_bfd = bfd_layout(n, t_block, nullptr, nullptr);
+        need_work += extra_bfd > extra_epoch ? extra_bfd : extra_epoch;  // the one size bload_plan_sizes reports
+    }
     if (plan_bytes < sz.plan_bytes || work_bytes < need_work) return fail(BLOAD_ERR_WORKSPACE);
     if (!aligned(d_plan, kAlign) || !aligned(d_work, kAlign) || !aligned(d_lengths, 4)) return fail(BLOAD_ERR_ALIGN);
 

@@ -698,12 +698,16 @@ cudaError_t launch_copy_range(bool unpack, const PlanView& pv, int32_t t_block, 
     const int64_t block_bytes = (int64_t)t_block * frame_bytes;
     const int64_t sub = 16384;
     const int64_t spb = (block_bytes + sub - 1) / sub;
-    const unsigned grid = 148 * 3 * 4;  // three CTAs of this kernel are resident per SM; four rounds of them
+    // many short-lived CTAs rather than a few long ones: the next chunk of the fill rule (one CTA on the other stream)
+    // starts as soon as any CTA of this launch retires; a chunk holds some thousand sub-tiles, about one per warp
+    const unsigned grid = 148 * 3 * 32;
     count_launches(1);
     if (unpack)
-        k7_copy<true><<<grid, 256, 0, st>>>(pv, t_block, frame_bytes, 0, 0, src, dst, src_total_bytes, sub, spb, pad_byte, d_range, 0);
+        k7_copy<true><<<grid, 256, kBesideChainSmemBytes, st>>>(pv, t_block, frame_bytes, 0, 0, src, dst, src_total_bytes, sub, spb,
+                                                                pad_byte, d_range, 0);
     else
-        k7_copy<false><<<grid, 256, 0, st>>>(pv, t_block, frame_bytes, 0, 0, src, dst, src_total_bytes, sub, spb, pad_byte, d_range, 0);
+        k7_copy<false><<<grid, 256, kBesideChainSmemBytes, st>>>(pv, t_block, frame_bytes, 0, 0, src, dst, src_total_bytes, sub, spb,
+                                                                 pad_byte, d_range, 0);
     return cudaPeekAtLastError();
 }
 

@@ -67,6 +67,13 @@ struct FillResume {
                                              // the caller's capacity; row kMaxEpochChunks: the filler blocks behind the plan
     int32_t draw[kMaxEpochChunks + 1][4];    // per chunk {first draw, end draw, first block, end block} (not clamped)
 };
+// Occupancy control of bload_epoch: the chunks of the fill rule ask for kChainSmemBytes of shared memory (they need
+// far less) and every kernel that runs beside them asks for kBesideChainSmemBytes it never touches, so no CTA of
+// those kernels fits on the SM that runs the chain (227 KB per SM), while three of them still fit on any other SM.
+// A chain that shares its SM with copy warps was measured 30 % slower (its shared-memory loads queue behind their
+// global loads and stores).
+constexpr int kChainSmemBytes = 184 * 1024;
+constexpr int kBesideChainSmemBytes = 46 * 1024;  // below the 48 KB a launch may ask for without opting in, static use included
 struct EpochView {
     FillResume* resume;
     int32_t* fill_tables;  // snapshot of the fill rule's shared-memory tables between chunks

@@ -109,10 +109,11 @@ cudaError_t launch_metadata(const PlanView& pv, int32_t t_block, int64_t block_b
     if (d_range && rows > 256) rows = 256;  // a chunk of a plan in progress holds a few blocks
     if (rows > 65535) rows = 65535;
     const dim3 grid(chunks, (unsigned)rows);
+    const size_t smem = d_range ? kBesideChainSmemBytes : 0;  // beside a running fill rule: stay off its SM
     if (t_block % 4 == 0 && al(seq_id, 16) && al(pos, 16) && al(reset, 4) && al(valid, 4))
-        k6_metadata<true><<<grid, kMetaThreads, 0, st>>>(pv, t_block, block_begin, (int32_t)block_count, seq_id, pos, reset, valid, d_range);
+        k6_metadata<true><<<grid, kMetaThreads, smem, st>>>(pv, t_block, block_begin, (int32_t)block_count, seq_id, pos, reset, valid, d_range);
     else
-        k6_metadata<false><<<grid, kMetaThreads, 0, st>>>(pv, t_block, block_begin, (int32_t)block_count, seq_id, pos, reset, valid, d_range);
+        k6_metadata<false><<<grid, kMetaThreads, smem, st>>>(pv, t_block, block_begin, (int32_t)block_count, seq_id, pos, reset, valid, d_range);
     count_launches(1);
     return cudaPeekAtLastError();
 }

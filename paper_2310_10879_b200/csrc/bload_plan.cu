@@ -708,7 +708,8 @@ static size_t fill_smem_bytes(int32_t t_block) { return sizeof(int32_t) * (kQ2Of
 cudaError_t launch_fill_chunk(const PlanView& pv, const WorkView& wv, const EpochView& ev, int64_t n, int32_t t_block,
                               int32_t k_target, int32_t filler_end, cudaStream_t st)
 {
-    const size_t smem = fill_smem_bytes(t_block);
+    size_t smem = fill_smem_bytes(t_block);
+    if (smem < (size_t)kChainSmemBytes) smem = kChainSmemBytes;  // keeps other CTAs off this SM (see kChainSmemBytes)
     cudaError_t e = cudaFuncSetAttribute(k4_fill<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     k4_fill<true><<<1, 256, smem, st>>>(pv, wv.bucket_end, wv.draw_u, wv.draw_rec, n, t_block, ev.resume, ev.fill_tables,
@@ -721,7 +722,8 @@ cudaError_t launch_tables_chunk(const PlanView& pv, const WorkView& wv, const in
                                 const int32_t* d_draw_range, cudaStream_t st)
 {
     const int64_t want = (n + 255) / 256;
-    k5_tables<<<(unsigned)(want < 592 ? want : 592), 256, 0, st>>>(pv, wv.draw_rec, wv.bucket_end, sorted_id, n, d_draw_range);
+    k5_tables<<<(unsigned)(want < 592 ? want : 592), 256, kBesideChainSmemBytes, st>>>(pv, wv.draw_rec, wv.bucket_end, sorted_id, n,
+                                                                                        d_draw_range);
     count_launches(1);
     return cudaPeekAtLastError();
 }
