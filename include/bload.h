@@ -166,7 +166,9 @@ BLOAD_API int bload_plan_finish(const void* d_plan, void* stream, bload_plan_inf
  *                        blocks is only known when the plan is done, so give an upper bound (the previous epoch's
  *                        count plus a margin, or 2 * sum_t / t_block + 1); rows beyond n_blocks are filler
  *   d_work / work_bytes  as for bload_plan (bload_plan_sizes covers this call)
- *   side_stream          a second stream of the same device, or NULL (then everything runs on `stream`, in order)
+ *   side_stream          a second stream of the same device, or NULL (then everything runs on `stream`, in order);
+ *                        give `stream` the higher priority of the two, so that each chunk of the chain starts as
+ *                        soon as an SM has room for it
  *
  * Both streams are synchronised once before the call returns: on return `info` is filled and every output is
  * complete.  Errors are those of bload_plan, bload_pack and bload_unpack; BLOAD_ERR_WORKSPACE is also returned when

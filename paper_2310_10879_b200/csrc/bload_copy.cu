@@ -700,7 +700,7 @@ cudaError_t launch_copy_range(bool unpack, const PlanView& pv, int32_t t_block, 
     const int64_t spb = (block_bytes + sub - 1) / sub;
     // many short-lived CTAs rather than a few long ones: the next chunk of the fill rule (one CTA on the other stream)
     // starts as soon as any CTA of this launch retires; a chunk holds some thousand sub-tiles, about one per warp
-    const unsigned grid = 148 * 3 * 32;
+    const unsigned grid = 148 * 3 * 16;  // (2 to 32 rounds of resident CTAs measured alike)
     count_launches(1);
     if (unpack)
         k7_copy<true><<<grid, 256, kBesideChainSmemBytes, st>>>(pv, t_block, frame_bytes, 0, 0, src, dst, src_total_bytes, sub, spb,
