@@ -363,13 +363,15 @@ __global__ void __launch_bounds__(256, 1) k4_fill(PlanView pv, const int32_t* __
     // random words of 32 draws at a time, one per lane, the next 32 prefetched
     uint64_t u_cur = (k & ~31) + lane < n ? draw_u[(k & ~31) + lane] : 0;
     uint64_t u_nxt = (k & ~31) + 32 + lane < n ? draw_u[(k & ~31) + 32 + lane] : 0;
+    // m = unused sequences that fit into the room left.  A block is only ever (re)opened here with room == L, where
+    // every unused sequence fits; inside a block the next m comes out of the previous draw (see below).
+    int m = n - k;
     while (k < n) {
         const uint64_t u = __shfl_sync(kFull, u_cur, k & 31);
-        const int y = room - 1, ya = y >> 10, yr = y >> 5;
-        const int m = room > 0 ? Q2[yr * 33 + (y & 31) + 1] + Q1[ya * 33 + (yr & 31)] + Q0[ya] : 0;
         if (m == 0) {  // nothing fits: the rest of the block is padding
             if (lane == 0) { pv.block_fill[b] = start; pv.block_seg_begin[b + 1] = k; }
             ++b; room = L; start = 0;
+            m = n - k;
             if (RESUME && k >= k_target) break;
             continue;
         }
@@ -391,9 +393,19 @@ __global__ void __launch_bounds__(256, 1) k4_fill(PlanView pv, const int32_t* __
         const int q2 = Q2[row * 33 + lane + 1];
         const int below = Q2[row * 33 + lane];
         j -= Q1[a * 33 + bb];
+        // While the level-2 vote is under way every lane looks up how many sequences would fit after ITS candidate
+        // length row*32 + lane + 1 (tables as they are before this draw, minus the drawn sequence itself when it
+        // would still fit); the chosen lane's value is the next draw's m.  That keeps the three-load lookup off the
+        // chain (177 -> 162 ns per draw).  The slot is clamped to >= 0, and is < L, so the indices stay in the tables.
+        const int my_len = (row << 5) + lane + 1;
+        const int my_room = room - my_len;
+        const int yy = max(my_room - 1, 0), yya = yy >> 10, yyr = yy >> 5;
+        int my_m = Q2[yyr * 33 + (yy & 31) + 1] + Q1[yya * 33 + (yyr & 31)] + Q0[yya];
+        my_m = my_room > 0 ? my_m - (my_len <= my_room ? 1 : 0) : 0;
         // level 2
         const int c = __popc(__ballot_sync(kFull, q2 <= j));
         const int len = (row << 5) + c + 1;
+        m = __shfl_sync(kFull, my_m, c);
         // decrement the running counts at and after the chosen digits
         if (lane >= a) { --q0; Q0[lane + 1] = q0; }
         if (a == 0) { --f0; if (lane >= bb) r1 = q1 - 1; }
