@@ -505,33 +505,50 @@ __global__ void __launch_bounds__(256, 1) k4_fill_lengths(PlanView pv, const int
     const int lane = threadIdx.x;
     const int n = (int)n64;
     int q0 = Q0[lane + 1];
+    int f0 = Q0[1];         // live lengths <= 1024 (every lane keeps a copy)
+    int r1 = Q1[lane + 1];  // row 0 of level 1 in registers, as in k4_fill
+    int live = Q0[32];      // lengths that still have an unused sequence
     int k = 0, b = 0, room = L, start = 0;
     if (lane == 0) pv.block_seg_begin[0] = 0;
     uint64_t u_cur = lane < n ? draw_u[lane] : 0;
     uint64_t u_nxt = 32 + lane < n ? draw_u[32 + lane] : 0;
+    // m = lengths that fit and are not exhausted; every live length fits into a freshly opened block, and inside a
+    // block the next m comes out of the previous draw (per candidate lane, as in k4_fill)
+    int m = live;
     while (k < n) {
         const uint64_t u = __shfl_sync(kFull, u_cur, k & 31);
-        const int y = room - 1, ya = y >> 10;
-        // lengths that fit and are not exhausted
-        const int m = room > 0 ? (Q2[y] & 63) + Q1[ya * 33 + ((y >> 5) & 31)] + Q0[ya] : 0;
         if (m == 0) {
             if (lane == 0) { pv.block_fill[b] = start; pv.block_seg_begin[b + 1] = k; }
             ++b; room = L; start = 0;
+            m = live;
             continue;
         }
         int j = (int)(((uint64_t)(uint32_t)(u >> 32) * (uint32_t)m + __umulhi((uint32_t)u, (uint32_t)m)) >> 32);
-        const int a = __popc(__ballot_sync(kFull, q0 <= j));
-        const int q1 = Q1[a * 33 + lane + 1];
-        j -= Q0[a];
+        int a = 0, q1 = r1;
+        if (j >= f0) {  // beyond the lengths <= 1024: walk level 0 (a >= 1 here, lane 0 holds q0 == f0 <= j)
+            a = __popc(__ballot_sync(kFull, q0 <= j));
+            j -= Q0[a];
+            q1 = Q1[a * 33 + lane + 1];
+        }
         const int bb = __popc(__ballot_sync(kFull, q1 <= j));
         const int row = (a << 5) + bb;
         const int q2 = Q2[(row << 5) + lane];
         j -= Q1[a * 33 + bb];
+        // the next m for this lane's candidate length (old tables; the length itself leaves the count when this draw
+        // takes its last sequence and it would still fit); slot clamped to [0, L)
+        const int my_len = (row << 5) + lane + 1;
+        const int my_room = room - my_len;
+        const int yy = max(my_room - 1, 0), yya = yy >> 10;
+        int my_m = (Q2[yy] & 63) + Q1[yya * 33 + ((yy >> 5) & 31)] + Q0[yya];
+        my_m = my_room > 0 ? my_m - ((((uint32_t)q2 >> 6) == 1u && my_len <= my_room) ? 1 : 0) : 0;
         const int c = __popc(__ballot_sync(kFull, (q2 & 63) <= j));
         const int len = (row << 5) + c + 1;
         const int cnt = (int)((uint32_t)__shfl_sync(kFull, q2, c) >> 6);  // unused sequences of the chosen length, >= 1
+        m = __shfl_sync(kFull, my_m, c);
         if (cnt == 1) {  // the length runs out: it leaves the prefix counts of all three levels
+            --live;
             if (lane >= a) { --q0; Q0[lane + 1] = q0; }
+            if (a == 0) { --f0; if (lane >= bb) r1 = q1 - 1; }
             if (lane >= bb) Q1[a * 33 + lane + 1] = q1 - 1;
             if (lane >= c) Q2[(row << 5) + lane] = (lane == c ? q2 - 64 : q2) - 1;
         } else if (lane == c) {
