@@ -660,8 +660,8 @@ def run_gpu(args, w) -> dict:
 TRAFFIC: dict = {
     # scaled by frames from the N=1,500 capture (profiles/k7_copy_small_cases_ncu_full.md): reads equal the
     # algorithmic bytes, writes are slightly below them (tail of the output still in L2 at kernel end)
-    ("heavy_tail_bf16", "k7_copy<unpack>"): 18.27e9,
-    ("heavy_tail_bf16", "k7_copy<pack>"): 9.09e9,
+    ("heavy_tail_bf16", "k7_copy<unpack>"): 18.29e9,
+    ("heavy_tail_bf16", "k7_copy<pack>"): 9.08e9,
 }
 
 
