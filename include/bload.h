@@ -155,7 +155,7 @@ BLOAD_API int bload_plan_finish(const void* d_plan, void* stream, bload_plan_inf
  *     bload_plan(policy BLOAD_POLICY_UNIFORM_SEQUENCES) ; bload_pack(blocks 0 .. block_capacity) ;
  *     bload_unpack(blocks 0 .. block_capacity)
  * but the fill rule (a chain of dependent draws that keeps one warp busy and leaves the memory system idle) runs
- * in chunks of about 1,250 draws on `stream`, and as soon as a chunk has closed its blocks their tables, metadata,
+ * in chunks of about 1,800 draws (at most 12, or io->chunks) on `stream`, and as soon as a chunk has closed its blocks their tables, metadata,
  * pack and unpack are issued on `side_stream`, under the next chunk of the chain.  Only launch-order dependencies
  * (events) are used; no kernel waits for another.  The paper has no counterpart (it builds blocks on the host).
  *
@@ -189,7 +189,8 @@ typedef struct {
     void* d_ragged_out;
     int64_t block_capacity;
     uint8_t pad_byte;
-    uint8_t reserved_[7];
+    uint8_t chunks;      /* launches of the fill rule: 0 = chosen by the library, else 1..32 */
+    uint8_t reserved_[6];
 } bload_epoch_io_t;
 BLOAD_API int bload_epoch(const int32_t* d_lengths, int64_t n, int32_t t_block, uint64_t seed, void* d_plan,
                           size_t plan_bytes, void* d_work, size_t work_bytes, const bload_epoch_io_t* io, void* stream,

@@ -49,7 +49,7 @@ class EpochIO(C.Structure):
     _fields_ = [("d_store", C.c_void_p), ("frame_bytes", C.c_int64), ("d_dense", C.c_void_p),
                 ("d_seq_id", C.c_void_p), ("d_pos", C.c_void_p), ("d_reset", C.c_void_p), ("d_valid", C.c_void_p),
                 ("d_dense_out", C.c_void_p), ("out_frame_bytes", C.c_int64), ("d_ragged_out", C.c_void_p),
-                ("block_capacity", C.c_int64), ("pad_byte", C.c_uint8), ("reserved_", C.c_uint8 * 7)]
+                ("block_capacity", C.c_int64), ("pad_byte", C.c_uint8), ("chunks", C.c_uint8), ("reserved_", C.c_uint8 * 6)]
 
 
 class VarInfo(C.Structure):
@@ -202,7 +202,7 @@ def bload_plan(lengths, t_block: int, seed: int, policy: int = 0, stream=None, w
 def bload_epoch(lengths, t_block: int, seed: int, block_capacity: int, store=None, frame_bytes: int = 0, dense=None,
                 seq_id=None, pos=None, reset=None, valid=None, pad_byte: int = 0, dense_out=None,
                 out_frame_bytes: int = 0, ragged_out=None, stream=None, side_stream=None, work=None, plan_buf=None,
-                check: bool = True) -> Plan:
+                check: bool = True, chunks: int = 0) -> Plan:
     """Plan, metadata, pack and unpack of a whole epoch in one call; the copies of finished blocks run on
     `side_stream` while the plan is still being built on `stream`.  Same results as bload_plan + bload_pack +
     bload_unpack over blocks [0, block_capacity).  All outputs are complete when the call returns."""
@@ -216,7 +216,7 @@ def bload_epoch(lengths, t_block: int, seed: int, block_capacity: int, store=Non
     if work is None:
         work = torch.empty(sizes.work_bytes, dtype=torch.uint8, device=lengths.device)
     io = EpochIO(_ptr(store), frame_bytes, _ptr(dense), _ptr(seq_id), _ptr(pos), _ptr(reset), _ptr(valid),
-                 _ptr(dense_out), out_frame_bytes, _ptr(ragged_out), block_capacity, pad_byte)
+                 _ptr(dense_out), out_frame_bytes, _ptr(ragged_out), block_capacity, pad_byte, chunks)
     info = PlanInfo()
     side = None if side_stream is None else (side_stream.cuda_stream or None)
     rc = load().bload_epoch(lengths.data_ptr(), n, t_block, seed, plan_buf.data_ptr(), plan_buf.numel(),
