@@ -32,3 +32,47 @@ def test_pack_unpack_round_trip(t_block, data, seed, fb, pad):
     out = np.zeros_like(store)
     O.unpack(p, dense, fb, 0, p.n_blocks + 1, out)
     assert np.array_equal(out, store)
+
+
+@settings(max_examples=60, deadline=None)
+@given(st.integers(1, 30), st.data(), st.integers(0, 2**32), st.integers(1, 24), st.integers(0, 255))
+def test_carry_prev_and_repeat_last_properties(t_block, data, seed, fb, fill):
+    T = np.array(data.draw(st.lists(st.integers(1, t_block), min_size=1, max_size=40)), np.int32)
+    p = O.plan(T, t_block, seed)
+    nb = p.n_blocks + 1
+    store = np.random.default_rng(seed).integers(0, 256, size=(p.sum_t, fb), dtype=np.uint8)
+    dense = O.pack(p, store, fb, 0, nb, fill)
+    seq_id, pos, reset, valid = O.metadata(p, 0, nb)
+    # what a slot receives is the frame before it in the ragged store, or the fill byte at a sequence start / padding
+    prev = O.carry_prev(p, dense, fb, 0, nb, fill)
+    cont = (valid == 1) & (reset == 0)
+    src = p.offsets[np.maximum(seq_id, 0)] + pos - 1
+    assert np.array_equal(prev[cont], store[src[cont]]) and np.all(prev[~cont] == fill)
+    # repeat-last padding changes nothing but the padding of blocks that hold a frame
+    rep = O.pack_repeat_last(p, store, fb, 0, nb, fill)
+    assert np.array_equal(rep[valid == 1], dense[valid == 1])
+    for q in range(nb):
+        k = int(valid[q].sum())
+        want = dense[q, k - 1] if k else np.full(fb, fill, np.uint8)
+        assert np.all(rep[q, k:] == want)
+
+
+@settings(max_examples=60, deadline=None)
+@given(st.integers(1, 20), st.data(), st.integers(0, 2**32), st.integers(0, 255))
+def test_var_frames_round_trip_and_padding(t_block, data, seed, pad):
+    n = data.draw(st.integers(1, 30))
+    T = np.array(data.draw(st.lists(st.integers(1, t_block), min_size=n, max_size=n)), np.int32)
+    F = np.array(data.draw(st.lists(st.integers(1, 20), min_size=n, max_size=n)), np.int32)
+    slot = int(F.max()) + data.draw(st.integers(0, 5))
+    p = O.plan(T, t_block, seed)
+    boff = O.byte_offsets(T, F)
+    store = np.random.default_rng(seed).integers(0, 256, size=int(boff[-1]), dtype=np.uint8)
+    nb = p.n_blocks + 1
+    dense = O.pack_var(p, store, F, slot, 0, nb, pad)
+    seq_id, _, _, valid = O.metadata(p, 0, nb)
+    used = np.where(valid == 1, F[np.maximum(seq_id, 0)], 0)               # bytes of every slot that hold a frame
+    is_pad = np.arange(slot)[None, None, :] >= used[:, :, None]
+    assert np.all(dense[is_pad] == pad) and int((~is_pad).sum()) == int(boff[-1])
+    back = np.zeros_like(store)
+    O.unpack_var(p, dense, F, slot, 0, nb, back)
+    assert np.array_equal(back, store)
