@@ -97,3 +97,41 @@ def test_full_size_tokens():
 
 def test_full_size_heavy_tail_bf16_with_fp32_outputs():
     _run("heavy_tail_bf16", 6)
+
+
+@pytest.mark.parametrize("name", ["tokens", "heavy_tail_bf16"])
+def test_full_size_epoch_call_equals_the_separate_calls(name):
+    """bload_epoch at full size, in the configuration the benchmark times (two streams, the chain's stream with the
+    higher priority): every table and every output byte equals what the separate calls give, which the tests above
+    compare with the oracle."""
+    w = W.WORKLOADS[name]
+    T = W.lengths(w)
+    d_len = torch.from_numpy(T).to(G.DEV)
+    fb, ofb, tb = w.frame_bytes, w.out_frame_bytes, w.t_block
+    ref = B.bload_plan(d_len, tb, w.seed)
+    nb = ref.n_blocks
+    store = W.payload_torch(w, ref.sum_t, G.DEV).view(torch.uint8).reshape(-1)
+    dense_out = torch.randint(0, 256, (nb * tb * ofb,), dtype=torch.uint8, device=G.DEV)
+    want_dense = torch.empty(nb * tb * fb, dtype=torch.uint8, device=G.DEV)
+    want_meta = [torch.empty(nb * tb, dtype=d, device=G.DEV) for d in (torch.int32, torch.int32, torch.uint8, torch.uint8)]
+    want_rag = torch.empty(ref.sum_t * ofb, dtype=torch.uint8, device=G.DEV)
+    B.bload_pack(ref, store, fb, 0, nb, dense=want_dense, seq_id=want_meta[0], pos=want_meta[1], reset=want_meta[2],
+                 valid=want_meta[3])
+    B.bload_unpack(ref, dense_out, ofb, 0, nb, want_rag)
+    got_dense = G.Guarded(nb * tb * fb)
+    got_meta = [torch.full_like(x, 0x11) for x in want_meta]
+    got_rag = G.Guarded(ref.sum_t * ofb, 0x5A)
+    chain, side = torch.cuda.Stream(priority=-1), torch.cuda.Stream()
+    chain.wait_stream(torch.cuda.current_stream())
+    plan = B.bload_epoch(d_len, tb, w.seed, nb, store=store, frame_bytes=fb, dense=got_dense.t, seq_id=got_meta[0],
+                         pos=got_meta[1], reset=got_meta[2], valid=got_meta[3], dense_out=dense_out, out_frame_bytes=ofb,
+                         ragged_out=got_rag.t, stream=chain, side_stream=side)
+    torch.cuda.synchronize()
+    got_dense.check(); got_rag.check()
+    assert plan.info.checksum == ref.info.checksum and plan.n_blocks == nb
+    for k, t in plan.tables().items():
+        assert torch.equal(t, ref.tables()[k]), k
+    assert torch.equal(got_dense.t, want_dense)
+    for a, b in zip(got_meta, want_meta):
+        assert torch.equal(a, b)
+    assert torch.equal(got_rag.t, want_rag)
