@@ -28,6 +28,8 @@
  *   byte_offsets       numpy.cumsum of T_i * F_i
  *   pack_var/unpack_var  equal frame sizes reduce to pack/unpack; per-slot numpy construction from
  *                      H_i x W_i images; round trip; padding bytes
+ *   pack_var2d/unpack_var2d  numpy canvases (canvas[:H_i, :W_i] = image); one row per image reduces to
+ *                      pack_var; round trip
  *   carry_prev         shifting every sequence by one frame in the ragged store and
  *                      packing that gives the same bytes
  *   reset_state        a running sum carried through the slots with resets equals the
@@ -460,6 +462,78 @@ int oracle_unpack_var(const oracle_tables_t *t, const uint8_t *dense_out, const 
             size_t have = (size_t)frame_bytes[sid[s]];
             memcpy(ragged_out + (size_t)byte_offsets[sid[s]] + (size_t)ps[s] * have,
                    dense_out + ((size_t)q * (size_t)t->t_block + (size_t)s) * (size_t)slot_bytes, have);
+        }
+    }
+    free(sid); free(ps); free(rs); free(vd);
+    return ORACLE_OK;
+}
+
+/* Frames as images of rows_i rows of row_bytes_i bytes (H_i x W_i of the problem statement): a slot is a
+ * canvas of rows_max rows of row_stride bytes, an image sits in its top left corner, the rest is padding.
+ * Sequence i holds T_i images of rows_i * row_bytes_i bytes back to back at byte_offsets[i]. */
+void oracle_byte_offsets2d(const int32_t *lengths, const int32_t *rows, const int32_t *row_bytes, int64_t n,
+                           int64_t *byte_offsets)
+{
+    int64_t run = 0;
+    for (int64_t i = 0; i < n; ++i) {
+        byte_offsets[i] = run;
+        run += (int64_t)lengths[i] * (int64_t)rows[i] * (int64_t)row_bytes[i];
+    }
+    byte_offsets[n] = run;
+}
+
+static int var2d_args_ok(const oracle_tables_t *t, const int32_t *rows, const int32_t *row_bytes, int64_t rows_max,
+                         int64_t row_stride)
+{
+    if (rows_max < 1 || row_stride < 1) return 0;
+    for (int64_t i = 0; i < t->n; ++i)
+        if (rows[i] < 1 || rows[i] > rows_max || row_bytes[i] < 1 || row_bytes[i] > row_stride) return 0;
+    return 1;
+}
+
+int oracle_pack_var2d(const oracle_tables_t *t, const uint8_t *store, const int32_t *rows, const int32_t *row_bytes,
+                      const int64_t *byte_offsets, int64_t rows_max, int64_t row_stride, int64_t block_begin,
+                      int64_t block_count, uint8_t *dense, uint8_t pad_byte)
+{
+    if (block_begin < 0 || block_count < 0 || !var2d_args_ok(t, rows, row_bytes, rows_max, row_stride)) return ORACLE_ERR_ARG;
+    const size_t canvas = (size_t)rows_max * (size_t)row_stride;
+    int32_t *sid = (int32_t *)malloc(sizeof(int32_t) * (size_t)t->t_block);
+    int32_t *ps = (int32_t *)malloc(sizeof(int32_t) * (size_t)t->t_block);
+    uint8_t *rs = (uint8_t *)malloc((size_t)t->t_block), *vd = (uint8_t *)malloc((size_t)t->t_block);
+    if (!sid || !ps || !rs || !vd) { free(sid); free(ps); free(rs); free(vd); return ORACLE_ERR_NOMEM; }
+    for (int64_t q = 0; q < block_count; ++q) {
+        oracle_metadata(t, block_begin + q, 1, sid, ps, rs, vd);
+        for (int32_t s = 0; s < t->t_block; ++s) {
+            uint8_t *dst = dense + ((size_t)q * (size_t)t->t_block + (size_t)s) * canvas;
+            memset(dst, pad_byte, canvas);
+            if (!vd[s]) continue;
+            const size_t h = (size_t)rows[sid[s]], w = (size_t)row_bytes[sid[s]];
+            const uint8_t *img = store + (size_t)byte_offsets[sid[s]] + (size_t)ps[s] * h * w;
+            for (size_t r = 0; r < h; ++r) memcpy(dst + r * (size_t)row_stride, img + r * w, w);
+        }
+    }
+    free(sid); free(ps); free(rs); free(vd);
+    return ORACLE_OK;
+}
+
+int oracle_unpack_var2d(const oracle_tables_t *t, const uint8_t *dense_out, const int32_t *rows, const int32_t *row_bytes,
+                        const int64_t *byte_offsets, int64_t rows_max, int64_t row_stride, int64_t block_begin,
+                        int64_t block_count, uint8_t *ragged_out)
+{
+    if (block_begin < 0 || block_count < 0 || !var2d_args_ok(t, rows, row_bytes, rows_max, row_stride)) return ORACLE_ERR_ARG;
+    const size_t canvas = (size_t)rows_max * (size_t)row_stride;
+    int32_t *sid = (int32_t *)malloc(sizeof(int32_t) * (size_t)t->t_block);
+    int32_t *ps = (int32_t *)malloc(sizeof(int32_t) * (size_t)t->t_block);
+    uint8_t *rs = (uint8_t *)malloc((size_t)t->t_block), *vd = (uint8_t *)malloc((size_t)t->t_block);
+    if (!sid || !ps || !rs || !vd) { free(sid); free(ps); free(rs); free(vd); return ORACLE_ERR_NOMEM; }
+    for (int64_t q = 0; q < block_count; ++q) {
+        oracle_metadata(t, block_begin + q, 1, sid, ps, rs, vd);
+        for (int32_t s = 0; s < t->t_block; ++s) {
+            if (!vd[s]) continue;
+            const uint8_t *src = dense_out + ((size_t)q * (size_t)t->t_block + (size_t)s) * canvas;
+            const size_t h = (size_t)rows[sid[s]], w = (size_t)row_bytes[sid[s]];
+            uint8_t *img = ragged_out + (size_t)byte_offsets[sid[s]] + (size_t)ps[s] * h * w;
+            for (size_t r = 0; r < h; ++r) memcpy(img + r * w, src + r * (size_t)row_stride, w);
         }
     }
     free(sid); free(ps); free(rs); free(vd);

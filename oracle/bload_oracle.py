@@ -90,6 +90,14 @@ def lib():
         L.oracle_unpack_var.argtypes = [C.POINTER(_TablesStruct), C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64,
                                         C.c_int64, C.c_int64, C.c_void_p]
         L.oracle_unpack_var.restype = C.c_int
+        L.oracle_byte_offsets2d.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p]
+        L.oracle_byte_offsets2d.restype = None
+        L.oracle_pack_var2d.argtypes = [C.POINTER(_TablesStruct), C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
+                                        C.c_int64, C.c_int64, C.c_int64, C.c_int64, C.c_void_p, C.c_uint8]
+        L.oracle_pack_var2d.restype = C.c_int
+        L.oracle_unpack_var2d.argtypes = [C.POINTER(_TablesStruct), C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
+                                          C.c_int64, C.c_int64, C.c_int64, C.c_int64, C.c_void_p]
+        L.oracle_unpack_var2d.restype = C.c_int
         L.oracle_carry_prev.argtypes = [C.POINTER(_TablesStruct), C.c_void_p, C.c_int64, C.c_int64, C.c_int64,
                                         C.c_void_p, C.c_uint8]
         L.oracle_carry_prev.restype = C.c_int
@@ -266,6 +274,46 @@ def unpack_var(p: OraclePlan, dense_out: np.ndarray, frame_bytes: np.ndarray, sl
     t = p._tables()
     rc = lib().oracle_unpack_var(C.byref(t), _p(dense_out), _p(frame_bytes), _p(boff), slot_bytes, block_begin,
                                  block_count, _p(ragged_out))
+    assert rc == 0, rc
+    return ragged_out
+
+
+def byte_offsets2d(lengths: np.ndarray, rows: np.ndarray, row_bytes: np.ndarray) -> np.ndarray:
+    lengths = np.ascontiguousarray(lengths, dtype=np.int32)
+    rows = np.ascontiguousarray(rows, dtype=np.int32)
+    row_bytes = np.ascontiguousarray(row_bytes, dtype=np.int32)
+    out = np.zeros(lengths.size + 1, dtype=np.int64)
+    lib().oracle_byte_offsets2d(_p(lengths), _p(rows), _p(row_bytes), lengths.size, _p(out))
+    return out
+
+
+def pack_var2d(p: OraclePlan, store: np.ndarray, rows: np.ndarray, row_bytes: np.ndarray, rows_max: int,
+               row_stride: int, block_begin: int, block_count: int, pad_byte: int = 0) -> np.ndarray:
+    """Images of rows[i] x row_bytes[i] bytes in the top left corner of canvases of rows_max x row_stride bytes."""
+    rows = np.ascontiguousarray(rows, dtype=np.int32)
+    row_bytes = np.ascontiguousarray(row_bytes, dtype=np.int32)
+    boff = byte_offsets2d(p.lengths, rows, row_bytes)
+    store = np.ascontiguousarray(store).view(np.uint8).reshape(-1)
+    assert store.size == int(boff[-1])
+    dense = np.empty((block_count, p.t_block, rows_max, row_stride), np.uint8)
+    t = p._tables()
+    rc = lib().oracle_pack_var2d(C.byref(t), _p(store), _p(rows), _p(row_bytes), _p(boff), rows_max, row_stride,
+                                 block_begin, block_count, _p(dense), pad_byte)
+    assert rc == 0, rc
+    return dense
+
+
+def unpack_var2d(p: OraclePlan, dense_out: np.ndarray, rows: np.ndarray, row_bytes: np.ndarray, rows_max: int,
+                 row_stride: int, block_begin: int, block_count: int, ragged_out: np.ndarray) -> np.ndarray:
+    rows = np.ascontiguousarray(rows, dtype=np.int32)
+    row_bytes = np.ascontiguousarray(row_bytes, dtype=np.int32)
+    boff = byte_offsets2d(p.lengths, rows, row_bytes)
+    dense_out = np.ascontiguousarray(dense_out).view(np.uint8).reshape(-1)
+    assert dense_out.size == block_count * p.t_block * rows_max * row_stride
+    assert ragged_out.dtype == np.uint8 and ragged_out.flags.c_contiguous and ragged_out.size == int(boff[-1])
+    t = p._tables()
+    rc = lib().oracle_unpack_var2d(C.byref(t), _p(dense_out), _p(rows), _p(row_bytes), _p(boff), rows_max, row_stride,
+                                   block_begin, block_count, _p(ragged_out))
     assert rc == 0, rc
     return ragged_out
 

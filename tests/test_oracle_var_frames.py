@@ -69,3 +69,40 @@ def test_pack_var_places_every_image_at_the_start_of_its_slot(n, tb, fmax):
     for k in range(p.block_seg_begin[0], p.block_seg_begin[1]):
         i = int(p.seg_seq[k]); inside[boff[i]:boff[i + 1]] = True
     assert np.array_equal(part[inside], store[inside]) and np.all(part[~inside] == 0x99)
+
+
+@pytest.mark.parametrize("n,tb,hmax,wmax", [(8, 6, 3, 5), (50, 20, 6, 16), (120, 40, 4, 9)])
+def test_pack_var2d_places_every_image_in_the_top_left_corner_of_its_canvas(n, tb, hmax, wmax):
+    rng = np.random.default_rng(n + hmax)
+    T = rng.integers(1, tb + 1, size=n).astype(np.int32)
+    H = rng.integers(1, hmax + 1, size=n).astype(np.int32)
+    Wd = rng.integers(1, wmax + 1, size=n).astype(np.int32)
+    p = O.plan(T, tb, 70 + n)
+    videos = [rng.integers(0, 256, size=(int(T[i]), int(H[i]), int(Wd[i])), dtype=np.uint8) for i in range(n)]
+    store = np.concatenate([v.reshape(-1) for v in videos])
+    assert np.array_equal(O.byte_offsets2d(T, H, Wd),
+                          np.concatenate([[0], np.cumsum(T.astype(np.int64) * H * Wd)]))
+    nb = p.n_blocks + 1
+    stride = wmax + 3
+    got = O.pack_var2d(p, store, H, Wd, hmax, stride, 0, nb, 0xEE)
+    seq_id, pos, _, valid = O.metadata(p, 0, nb)
+    want = np.full((nb, tb, hmax, stride), 0xEE, np.uint8)
+    for q in range(nb):
+        for s in range(tb):
+            if valid[q, s]:
+                img = videos[seq_id[q, s]][pos[q, s]]
+                want[q, s, :img.shape[0], :img.shape[1]] = img
+    assert np.array_equal(got, want)
+    assert np.array_equal(O.pack_var2d(p, store, H, Wd, hmax, stride, 1, 2, 0xEE), want[1:3])
+    back = np.full(store.size, 0x99, np.uint8)
+    O.unpack_var2d(p, got, H, Wd, hmax, stride, 0, nb, back)
+    assert np.array_equal(back, store)
+
+
+def test_one_row_per_image_reduces_to_pack_var():
+    p, T, F, rng = _case(90, 25, 4, 30)
+    store = rng.integers(0, 256, size=int(O.byte_offsets(T, F)[-1]), dtype=np.uint8)
+    ones = np.ones(p.n, np.int32)
+    nb = p.n_blocks + 1
+    a = O.pack_var2d(p, store, ones, F, 1, 33, 0, nb, 5).reshape(nb, p.t_block, 33)
+    assert np.array_equal(a, O.pack_var(p, store, F, 33, 0, nb, 5))
