@@ -269,7 +269,8 @@ BLOAD_API int bload_unpack(const void* d_plan, const bload_plan_info_t* info, co
 typedef struct {
     int64_t total_bytes;     /* bytes of the ragged store */
     int64_t max_frame_bytes; /* largest F_i: the smallest slot_bytes that holds every frame */
-    int64_t first_bad_index; /* first i with F_i < 1, else -1 */
+    int64_t first_bad_index; /* first i with F_i < 1 (or rows_i < 1), else -1 */
+    int64_t max_rows;        /* most rows of any image (1 for the calls without rows) */
 } bload_var_info_t;
 BLOAD_API int bload_var_offsets(const int32_t* d_lengths, const int32_t* d_frame_bytes, int64_t n,
                                 int64_t* d_byte_offsets, void* stream, bload_var_info_t* info);
@@ -279,6 +280,29 @@ BLOAD_API int bload_pack_var(const void* d_plan, const bload_plan_info_t* info, 
 BLOAD_API int bload_unpack_var(const void* d_plan, const bload_plan_info_t* info, const void* d_dense_out,
                                const int32_t* d_frame_bytes, const int64_t* d_byte_offsets, int64_t slot_bytes,
                                int64_t block_begin, int64_t block_count, void* d_ragged_out, void* stream);
+
+/*
+ * The same with frames as images (the H x W of the paper's problem statement): every frame of sequence i has
+ * d_rows[i] rows of d_row_bytes[i] bytes (row major, rows back to back in the store).  A slot is a canvas of
+ * rows_max rows of row_stride bytes, so d_dense is [block_count, t_block, rows_max, row_stride]; an image sits in
+ * the top left corner of its canvas, and the bytes to its right and below it are pad_byte.  With one row per image
+ * and rows_max == 1 these calls are bload_pack_var / bload_unpack_var.
+ *
+ * bload_var_offsets2d -- d_byte_offsets[i] = sum over j < i of T_j * rows_j * row_bytes_j.  The array needs n + 4
+ * elements: [n] total bytes, [n+1] largest row size, [n+2] first i with a size < 1 or -1, [n+3] most rows; the same
+ * values come back in `info`.  Precondition of the pack / unpack calls: 1 <= rows_i <= rows_max and
+ * 1 <= row_bytes_i <= row_stride (clamped on the device otherwise, as above).  Errors as for the calls above.
+ */
+BLOAD_API int bload_var_offsets2d(const int32_t* d_lengths, const int32_t* d_rows, const int32_t* d_row_bytes, int64_t n,
+                                  int64_t* d_byte_offsets, void* stream, bload_var_info_t* info);
+BLOAD_API int bload_pack_var2d(const void* d_plan, const bload_plan_info_t* info, const void* d_store,
+                               const int32_t* d_rows, const int32_t* d_row_bytes, const int64_t* d_byte_offsets,
+                               int64_t rows_max, int64_t row_stride, int64_t block_begin, int64_t block_count,
+                               void* d_dense, uint8_t pad_byte, void* stream);
+BLOAD_API int bload_unpack_var2d(const void* d_plan, const bload_plan_info_t* info, const void* d_dense_out,
+                                 const int32_t* d_rows, const int32_t* d_row_bytes, const int64_t* d_byte_offsets,
+                                 int64_t rows_max, int64_t row_stride, int64_t block_begin, int64_t block_count,
+                                 void* d_ragged_out, void* stream);
 
 /*
  * Consumer side of the start table (paper, Methods, second paragraph, and its figure of the DDS

@@ -18,7 +18,8 @@ ERR_UNSUPPORTED, ERR_CUDA, ERR_TIMEOUT, ERR_PLAN = -6, -7, -8, -9
 MAX_T_BLOCK = 32768
 
 EXPORTS = ("bload_plan_sizes", "bload_plan", "bload_plan_async", "bload_plan_finish", "bload_rank_range", "bload_pack", "bload_unpack", "bload_stats", "bload_epoch", "bload_epoch_stage_times",
-           "bload_pack_repeat_last", "bload_var_offsets", "bload_pack_var", "bload_unpack_var", "bload_carry_prev", "bload_reset_state", "bload_valid_sum",
+           "bload_pack_repeat_last", "bload_var_offsets", "bload_pack_var", "bload_unpack_var", "bload_var_offsets2d", "bload_pack_var2d",
+           "bload_unpack_var2d", "bload_carry_prev", "bload_reset_state", "bload_valid_sum",
            "bload_set_plan_timing", "bload_plan_stage_times", "bload_kernel_launches", "bload_strerror",
            "bload_version")
 
@@ -53,7 +54,8 @@ class EpochIO(C.Structure):
 
 
 class VarInfo(C.Structure):
-    _fields_ = [("total_bytes", C.c_int64), ("max_frame_bytes", C.c_int64), ("first_bad_index", C.c_int64)]
+    _fields_ = [("total_bytes", C.c_int64), ("max_frame_bytes", C.c_int64), ("first_bad_index", C.c_int64),
+                ("max_rows", C.c_int64)]
 
 
 class BloadError(RuntimeError):
@@ -96,6 +98,9 @@ def load() -> C.CDLL:
     L.bload_var_offsets.argtypes = [vp, vp, i64, vp, vp, C.POINTER(VarInfo)]
     L.bload_pack_var.argtypes = [vp, C.POINTER(PlanInfo), vp, vp, vp, i64, i64, i64, vp, u8, vp]
     L.bload_unpack_var.argtypes = [vp, C.POINTER(PlanInfo), vp, vp, vp, i64, i64, i64, vp, vp]
+    L.bload_var_offsets2d.argtypes = [vp, vp, vp, i64, vp, vp, C.POINTER(VarInfo)]
+    L.bload_pack_var2d.argtypes = [vp, C.POINTER(PlanInfo), vp, vp, vp, vp, i64, i64, i64, i64, vp, u8, vp]
+    L.bload_unpack_var2d.argtypes = [vp, C.POINTER(PlanInfo), vp, vp, vp, vp, i64, i64, i64, i64, vp, vp]
     L.bload_carry_prev.argtypes = [vp, C.POINTER(PlanInfo), vp, i64, i64, i64, vp, u8, vp]
     L.bload_reset_state.argtypes = [vp, C.POINTER(PlanInfo), i64, i64, i32, vp, i64, vp, vp]
     L.bload_valid_sum.argtypes = [vp, C.POINTER(PlanInfo), vp, i64, i64, vp, vp, vp]
@@ -317,6 +322,40 @@ def bload_unpack_var(plan: Plan, dense_out, frame_bytes, byte_offsets, slot_byte
                                  _stream(stream))
     if rc:
         raise BloadError(rc, "bload_unpack_var")
+
+
+def bload_var_offsets2d(lengths, rows, row_bytes, stream=None):
+    """Byte offsets of a store whose sequence i holds lengths[i] images of rows[i] x row_bytes[i] bytes.
+    Returns (byte_offsets int64 CUDA tensor [n+4], VarInfo)."""
+    import torch
+    n = lengths.numel()
+    out = torch.empty(n + 4, dtype=torch.int64, device=lengths.device)
+    info = VarInfo()
+    rc = load().bload_var_offsets2d(lengths.data_ptr(), rows.data_ptr(), row_bytes.data_ptr(), n, out.data_ptr(),
+                                    _stream(stream), C.byref(info))
+    if rc:
+        err = BloadError(rc, "bload_var_offsets2d")
+        err.info = info
+        raise err
+    return out, info
+
+
+def bload_pack_var2d(plan: Plan, store, rows, row_bytes, byte_offsets, rows_max: int, row_stride: int,
+                     block_begin: int, block_count: int, dense, pad_byte: int = 0, stream=None) -> None:
+    rc = load().bload_pack_var2d(plan.buf.data_ptr(), C.byref(plan.info), _ptr(store), _ptr(rows), _ptr(row_bytes),
+                                 _ptr(byte_offsets), rows_max, row_stride, block_begin, block_count, _ptr(dense),
+                                 pad_byte, _stream(stream))
+    if rc:
+        raise BloadError(rc, "bload_pack_var2d")
+
+
+def bload_unpack_var2d(plan: Plan, dense_out, rows, row_bytes, byte_offsets, rows_max: int, row_stride: int,
+                       block_begin: int, block_count: int, ragged_out, stream=None) -> None:
+    rc = load().bload_unpack_var2d(plan.buf.data_ptr(), C.byref(plan.info), _ptr(dense_out), _ptr(rows),
+                                   _ptr(row_bytes), _ptr(byte_offsets), rows_max, row_stride, block_begin, block_count,
+                                   _ptr(ragged_out), _stream(stream))
+    if rc:
+        raise BloadError(rc, "bload_unpack_var2d")
 
 
 def bload_carry_prev(plan: Plan, dense, frame_bytes: int, block_begin: int, block_count: int, prev,

@@ -447,61 +447,92 @@ int bload_unpack(const void* d_plan, const bload_plan_info_t* info, const void* 
     return BLOAD_OK;
 }
 
-int bload_var_offsets(const int32_t* d_lengths, const int32_t* d_frame_bytes, int64_t n, int64_t* d_byte_offsets,
-                      void* stream, bload_var_info_t* info)
+int bload_var_offsets2d(const int32_t* d_lengths, const int32_t* d_rows, const int32_t* d_row_bytes, int64_t n,
+                        int64_t* d_byte_offsets, void* stream, bload_var_info_t* info)
 {
     if (!info) return BLOAD_ERR_NULL;
     memset(info, 0, sizeof *info);
     info->first_bad_index = -1;
-    if (!d_lengths || !d_frame_bytes || !d_byte_offsets) return BLOAD_ERR_NULL;
+    if (!d_lengths || !d_row_bytes || !d_byte_offsets) return BLOAD_ERR_NULL;
     if (n < 1 || n >= (1LL << 31)) return BLOAD_ERR_ARG;
-    if (!aligned(d_lengths, 4) || !aligned(d_frame_bytes, 4) || !aligned(d_byte_offsets, 8)) return BLOAD_ERR_ALIGN;
+    if (!aligned(d_lengths, 4) || !aligned(d_rows, 4) || !aligned(d_row_bytes, 4) || !aligned(d_byte_offsets, 8))
+        return BLOAD_ERR_ALIGN;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    cudaError_t ce = launch_var_offsets(d_lengths, d_frame_bytes, n, d_byte_offsets, st);
-    int64_t tail[3] = {0, 0, -1};
-    if (ce == cudaSuccess) ce = cudaMemcpyAsync(tail, d_byte_offsets + n, sizeof tail, cudaMemcpyDeviceToHost, st);
+    // the tail of the array: [n] total bytes, [n+1] largest row size, [n+2] first bad index, and with rows [n+3] most rows
+    cudaError_t ce = launch_var_offsets(d_lengths, d_rows, d_row_bytes, n, d_byte_offsets,
+                                        d_rows ? d_byte_offsets + n + 3 : nullptr, st);
+    int64_t tail[4] = {0, 0, -1, 1};
+    if (ce == cudaSuccess)
+        ce = cudaMemcpyAsync(tail, d_byte_offsets + n, (d_rows ? 4 : 3) * sizeof(int64_t), cudaMemcpyDeviceToHost, st);
     if (ce == cudaSuccess) ce = cudaStreamSynchronize(st);
     if (ce != cudaSuccess) { (void)cudaGetLastError(); return BLOAD_ERR_CUDA; }
     info->total_bytes = tail[0];
     info->max_frame_bytes = tail[1];
     info->first_bad_index = tail[2];
+    info->max_rows = tail[3];
     return tail[2] >= 0 ? BLOAD_ERR_ARG : BLOAD_OK;
 }
+
+int bload_var_offsets(const int32_t* d_lengths, const int32_t* d_frame_bytes, int64_t n, int64_t* d_byte_offsets,
+                      void* stream, bload_var_info_t* info)
+{
+    return bload_var_offsets2d(d_lengths, nullptr, d_frame_bytes, n, d_byte_offsets, stream, info);
+}
+
+namespace {
+int copy_var(bool unpack, const void* d_plan, const bload_plan_info_t* info, const void* d_src, const int32_t* d_rows,
+             const int32_t* d_row_bytes, const int64_t* d_byte_offsets, int64_t rows_max, int64_t row_stride,
+             int64_t block_begin, int64_t block_count, void* d_dst, uint8_t pad_byte, void* stream)
+{
+    int rc = check_plan_args(d_plan, info, row_stride, block_begin, block_count);
+    if (rc) return rc;
+    if (rows_max < 1 || rows_max > 0x7fffffffLL) return BLOAD_ERR_ARG;
+    if (block_count == 0) return BLOAD_OK;
+    if (!d_src || !d_dst || !d_row_bytes || !d_byte_offsets) return BLOAD_ERR_NULL;
+    if (!aligned(d_src, 16) || !aligned(d_dst, 16) || !aligned(d_rows, 4) || !aligned(d_row_bytes, 4) ||
+        !aligned(d_byte_offsets, 8))
+        return BLOAD_ERR_ALIGN;
+    cudaError_t ce = launch_copy_var(unpack, plan_view(const_cast<void*>(d_plan), info->n), info->t_block, (int32_t)rows_max,
+                                     row_stride, block_begin, block_count, d_rows, d_row_bytes, d_byte_offsets,
+                                     static_cast<const uint8_t*>(d_src), static_cast<uint8_t*>(d_dst), pad_byte,
+                                     static_cast<cudaStream_t>(stream));
+    if (ce != cudaSuccess) { (void)cudaGetLastError(); return BLOAD_ERR_CUDA; }
+    return BLOAD_OK;
+}
+}  // namespace
 
 int bload_pack_var(const void* d_plan, const bload_plan_info_t* info, const void* d_store, const int32_t* d_frame_bytes,
                    const int64_t* d_byte_offsets, int64_t slot_bytes, int64_t block_begin, int64_t block_count,
                    void* d_dense, uint8_t pad_byte, void* stream)
 {
-    int rc = check_plan_args(d_plan, info, slot_bytes, block_begin, block_count);
-    if (rc) return rc;
-    if (block_count == 0) return BLOAD_OK;
-    if (!d_store || !d_dense || !d_frame_bytes || !d_byte_offsets) return BLOAD_ERR_NULL;
-    if (!aligned(d_dense, 16) || !aligned(d_store, 16) || !aligned(d_frame_bytes, 4) || !aligned(d_byte_offsets, 8))
-        return BLOAD_ERR_ALIGN;
-    cudaError_t ce = launch_copy_var(false, plan_view(const_cast<void*>(d_plan), info->n), info->t_block, slot_bytes,
-                                     block_begin, block_count, d_frame_bytes, d_byte_offsets,
-                                     static_cast<const uint8_t*>(d_store), static_cast<uint8_t*>(d_dense), pad_byte,
-                                     static_cast<cudaStream_t>(stream));
-    if (ce != cudaSuccess) { (void)cudaGetLastError(); return BLOAD_ERR_CUDA; }
-    return BLOAD_OK;
+    return copy_var(false, d_plan, info, d_store, nullptr, d_frame_bytes, d_byte_offsets, 1, slot_bytes, block_begin,
+                    block_count, d_dense, pad_byte, stream);
 }
 
 int bload_unpack_var(const void* d_plan, const bload_plan_info_t* info, const void* d_dense_out,
                      const int32_t* d_frame_bytes, const int64_t* d_byte_offsets, int64_t slot_bytes, int64_t block_begin,
                      int64_t block_count, void* d_ragged_out, void* stream)
 {
-    int rc = check_plan_args(d_plan, info, slot_bytes, block_begin, block_count);
-    if (rc) return rc;
-    if (block_count == 0) return BLOAD_OK;
-    if (!d_dense_out || !d_ragged_out || !d_frame_bytes || !d_byte_offsets) return BLOAD_ERR_NULL;
-    if (!aligned(d_dense_out, 16) || !aligned(d_ragged_out, 16) || !aligned(d_frame_bytes, 4) || !aligned(d_byte_offsets, 8))
-        return BLOAD_ERR_ALIGN;
-    cudaError_t ce = launch_copy_var(true, plan_view(const_cast<void*>(d_plan), info->n), info->t_block, slot_bytes,
-                                     block_begin, block_count, d_frame_bytes, d_byte_offsets,
-                                     static_cast<const uint8_t*>(d_dense_out), static_cast<uint8_t*>(d_ragged_out), 0,
-                                     static_cast<cudaStream_t>(stream));
-    if (ce != cudaSuccess) { (void)cudaGetLastError(); return BLOAD_ERR_CUDA; }
-    return BLOAD_OK;
+    return copy_var(true, d_plan, info, d_dense_out, nullptr, d_frame_bytes, d_byte_offsets, 1, slot_bytes, block_begin,
+                    block_count, d_ragged_out, 0, stream);
+}
+
+int bload_pack_var2d(const void* d_plan, const bload_plan_info_t* info, const void* d_store, const int32_t* d_rows,
+                     const int32_t* d_row_bytes, const int64_t* d_byte_offsets, int64_t rows_max, int64_t row_stride,
+                     int64_t block_begin, int64_t block_count, void* d_dense, uint8_t pad_byte, void* stream)
+{
+    if (!d_rows) return BLOAD_ERR_NULL;
+    return copy_var(false, d_plan, info, d_store, d_rows, d_row_bytes, d_byte_offsets, rows_max, row_stride, block_begin,
+                    block_count, d_dense, pad_byte, stream);
+}
+
+int bload_unpack_var2d(const void* d_plan, const bload_plan_info_t* info, const void* d_dense_out, const int32_t* d_rows,
+                       const int32_t* d_row_bytes, const int64_t* d_byte_offsets, int64_t rows_max, int64_t row_stride,
+                       int64_t block_begin, int64_t block_count, void* d_ragged_out, void* stream)
+{
+    if (!d_rows) return BLOAD_ERR_NULL;
+    return copy_var(true, d_plan, info, d_dense_out, d_rows, d_row_bytes, d_byte_offsets, rows_max, row_stride, block_begin,
+                    block_count, d_ragged_out, 0, stream);
 }
 
 int bload_carry_prev(const void* d_plan, const bload_plan_info_t* info, const void* d_dense, int64_t frame_bytes,

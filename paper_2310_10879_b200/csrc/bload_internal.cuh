@@ -142,10 +142,11 @@ cudaError_t launch_copy_range(bool unpack, const PlanView& pv, int32_t t_block, 
                               uint8_t* dst, int64_t src_total_bytes, uint8_t pad_byte, const int32_t* d_range,
                               cudaStream_t st);
 
-cudaError_t launch_var_offsets(const int32_t* lengths, const int32_t* frame_bytes, int64_t n, int64_t* out, cudaStream_t st);
-cudaError_t launch_copy_var(bool unpack, const PlanView& pv, int32_t t_block, int64_t slot_bytes, int64_t block_begin,
-                            int64_t block_count, const int32_t* frame_bytes, const int64_t* byte_offsets,
-                            const uint8_t* src, uint8_t* dst, uint8_t pad_byte, cudaStream_t st);
+cudaError_t launch_var_offsets(const int32_t* lengths, const int32_t* rows, const int32_t* frame_bytes, int64_t n,
+                               int64_t* out, int64_t* max_rows, cudaStream_t st);
+cudaError_t launch_copy_var(bool unpack, const PlanView& pv, int32_t t_block, int32_t rows_max, int64_t row_stride,
+                            int64_t block_begin, int64_t block_count, const int32_t* seq_rows, const int32_t* frame_bytes,
+                            const int64_t* byte_offsets, const uint8_t* src, uint8_t* dst, uint8_t pad_byte, cudaStream_t st);
 cudaError_t launch_carry_prev(const PlanView& pv, int32_t t_block, int64_t frame_bytes, int64_t block_begin,
                               int64_t block_count, const uint8_t* dense, uint8_t* prev, uint8_t fill_byte, cudaStream_t st,
                               int64_t n, int64_t sum_t);

@@ -3,8 +3,9 @@
 // largest frame, and a smaller frame sits at the start of its slot, followed by padding.
 //   k15_var_offsets  byte offset of every sequence in such a store (exclusive scan of T_i * F_i), with the
 //                    largest frame size and the first invalid size;
-//   k16_copy_var     pack / unpack with per-sequence frame sizes: the decomposition of the fixed-size copy
-//                    kernel (a warp owns a sub-tile of the dense side), walking slots inside each segment.
+//   k16_copy_var     pack / unpack with per-sequence frame sizes, optionally as images of rows x row bytes on a
+//                    canvas: the decomposition of the fixed-size copy kernel (a warp owns a sub-tile of the dense
+//                    side), walking the canvas rows inside each segment.
 #include "bload_internal.cuh"
 #include "bload_warp_copy.cuh"
 
@@ -19,25 +20,28 @@ constexpr int kScanThreads = 1024;
 // One CTA walks the sequences in chunks of kScanThreads with a running carry.  out[0..n) = first byte of each
 // sequence, out[n] = total bytes, out[n+1] = largest frame size, out[n+2] = first i with F_i < 1 (or -1).
 __global__ void __launch_bounds__(kScanThreads) k15_var_offsets(const int32_t* __restrict__ lengths,
+                                                                const int32_t* __restrict__ rows /*null: one row*/,
                                                                 const int32_t* __restrict__ frame_bytes, int64_t n,
-                                                                int64_t* __restrict__ out)
+                                                                int64_t* __restrict__ out, int64_t* __restrict__ max_rows)
 {
     __shared__ int64_t warp_sum[kScanThreads / 32];
     __shared__ int64_t carry_sh;
-    __shared__ int max_sh;
+    __shared__ int max_sh, max_rows_sh;
     __shared__ unsigned long long bad_sh;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    if (threadIdx.x == 0) { carry_sh = 0; max_sh = 0; bad_sh = ~0ULL; }
+    if (threadIdx.x == 0) { carry_sh = 0; max_sh = 0; max_rows_sh = 0; bad_sh = ~0ULL; }
     __syncthreads();
-    int my_max = 0;
+    int my_max = 0, my_rows = 0;
     for (int64_t base = 0; base < n; base += kScanThreads) {
         const int64_t i = base + threadIdx.x;
         int64_t v = 0;
         if (i < n) {
             const int f = frame_bytes[i];
-            if (f < 1) atomicMin(&bad_sh, (unsigned long long)i);
+            const int h = rows ? rows[i] : 1;
+            if (f < 1 || h < 1) atomicMin(&bad_sh, (unsigned long long)i);
             my_max = max(my_max, f);
-            v = (int64_t)lengths[i] * (int64_t)max(f, 0);
+            my_rows = max(my_rows, h);
+            v = (int64_t)lengths[i] * (int64_t)max(h, 0) * (int64_t)max(f, 0);
         }
         int64_t incl = v;  // inclusive scan inside the warp
 #pragma unroll
@@ -65,19 +69,26 @@ __global__ void __launch_bounds__(kScanThreads) k15_var_offsets(const int32_t* _
         __syncthreads();
     }
     atomicMax(&max_sh, my_max);
+    atomicMax(&max_rows_sh, my_rows);
     __syncthreads();
     if (threadIdx.x == 0) {
+        if (max_rows) *max_rows = max_rows_sh;
         out[n] = carry_sh;
         out[n + 1] = max_sh;
         out[n + 2] = bad_sh == ~0ULL ? -1 : (int64_t)bad_sh;
     }
 }
 
-// A frame size is clamped to the slot size on the device, so a caller that breaks the documented precondition
-// (F_i <= slot_bytes) gets truncated frames but never an access outside the buffers.
+// Frames are images of `rows` rows of `frame_bytes` (row) bytes; a slot is a canvas of rows_max rows of row_stride
+// bytes and an image sits in its top left corner (one row per frame and rows_max == 1 give the plain
+// per-sequence frame size).  The dense side is walked row by row of the canvases ("sub-slots" of row_stride
+// bytes).  Row counts and row sizes are clamped to the canvas on the device, so a caller that breaks the documented
+// precondition gets truncated images but never an access outside the buffers.
 template <bool UNPACK>
-__global__ void __launch_bounds__(256, 2) k16_copy_var(PlanView pv, int32_t t_block, int64_t slot_bytes, int64_t block_begin,
-                                                       int64_t block_count, const int32_t* __restrict__ frame_bytes,
+__global__ void __launch_bounds__(256, 2) k16_copy_var(PlanView pv, int32_t t_block, int32_t rows_max, int64_t row_stride,
+                                                       int64_t block_begin, int64_t block_count,
+                                                       const int32_t* __restrict__ seq_rows /*null: one row*/,
+                                                       const int32_t* __restrict__ frame_bytes,
                                                        const int64_t* __restrict__ byte_offsets,
                                                        const uint8_t* __restrict__ src_base, uint8_t* __restrict__ dst_base,
                                                        int64_t sub_bytes, int64_t subs_per_block, uint8_t pad)
@@ -85,6 +96,7 @@ __global__ void __launch_bounds__(256, 2) k16_copy_var(PlanView pv, int32_t t_bl
     const int lane = threadIdx.x & 31;
     const int64_t warps = ((int64_t)gridDim.x * blockDim.x) >> 5;
     const int64_t items = block_count * subs_per_block;
+    const int64_t slot_bytes = (int64_t)rows_max * row_stride;
     const int64_t block_bytes = (int64_t)t_block * slot_bytes;
     const int64_t n_blocks = pv.hdr->n_blocks;
     const int64_t ragged_total = byte_offsets[pv.hdr->n];
@@ -101,18 +113,21 @@ __global__ void __launch_bounds__(256, 2) k16_copy_var(PlanView pv, int32_t t_bl
             const int k0 = pv.block_seg_begin[b], k1 = pv.block_seg_begin[b + 1];
             const int fill = pv.block_fill[b];
             if (cur < (int64_t)fill * slot_bytes) {
+                // position inside the block: slot, canvas row, byte inside the row
                 int slot = (int)(cur / slot_bytes);
-                int64_t in = cur - (int64_t)slot * slot_bytes;  // offset inside the slot
+                int r = (int)((cur - (int64_t)slot * slot_bytes) / row_stride);
+                int64_t in = cur - (int64_t)slot * slot_bytes - (int64_t)r * row_stride;
                 int k = warp_find_segment(pv.seg_start, k0, k1, slot, lane);
-                int kw = k;  // lanes hold start slot, frame size and first byte of segments kw .. kw+31
-                int w_st = fill, w_fb = 1;
+                int kw = k;  // lanes hold start slot, rows, row size and first byte of segments kw .. kw+31
+                int w_st = fill, w_fb = 1, w_rows = 1;
                 int64_t w_off = 0;
                 auto load_window = [&]() {
-                    w_st = fill; w_fb = 1; w_off = 0;
+                    w_st = fill; w_fb = 1; w_rows = 1; w_off = 0;
                     if (kw + lane < k1) {
                         const int id = pv.seg_seq[kw + lane];
                         w_st = pv.seg_start[kw + lane];
-                        w_fb = (int)min((int64_t)max(frame_bytes[id], 1), slot_bytes);
+                        w_fb = (int)min((int64_t)max(frame_bytes[id], 1), row_stride);
+                        w_rows = seq_rows ? min(max(seq_rows[id], 1), rows_max) : 1;
                         w_off = byte_offsets[id];
                     }
                 };
@@ -122,32 +137,39 @@ __global__ void __launch_bounds__(256, 2) k16_copy_var(PlanView pv, int32_t t_bl
                     const int st = __shfl_sync(kFull, w_st, k - kw);
                     const int nx = __shfl_sync(kFull, w_st, k - kw + 1);
                     const int64_t fb = __shfl_sync(kFull, w_fb, k - kw);
+                    const int rows = __shfl_sync(kFull, w_rows, k - kw);
                     const int64_t off = __shfl_sync(kFull, w_off, k - kw);
                     const int64_t seg_e = min((int64_t)nx * slot_bytes, hi);
-                    if (fb == slot_bytes) {  // frames fill their slots: the rest of the segment is one run
+                    if (fb == row_stride && rows == rows_max) {  // images fill their canvases: the segment is one run
                         const int64_t rag = off + (cur - (int64_t)st * slot_bytes);
                         if (UNPACK) warp_copy<true>(dst_base + rag, src_base + dense_off + cur, seg_e - cur, s_limit, lane);
                         else warp_copy<false>(dst_base + dense_off + cur, src_base + rag, seg_e - cur, s_limit, lane);
-                        in = 0;  // a segment ends on a slot boundary unless the tile ends first
                         cur = seg_e;
                     } else {
                         while (cur < seg_e) {
-                            if (in < fb) {
+                            if (r < rows && in < fb) {  // the image's part of this canvas row
                                 const int64_t len = min(fb - in, seg_e - cur);
-                                const int64_t rag = off + (int64_t)(slot - st) * fb + in;
+                                const int64_t rag = off + ((int64_t)(slot - st) * rows + r) * fb + in;
                                 if (UNPACK) warp_copy<true>(dst_base + rag, src_base + dense_off + cur, len, s_limit, lane);
                                 else warp_copy<false>(dst_base + dense_off + cur, src_base + rag, len, s_limit, lane);
                                 cur += len; in += len;
                             }
-                            if (cur < seg_e) {  // the padding behind the frame
-                                const int64_t len = min(slot_bytes - in, seg_e - cur);
+                            if (cur < seg_e) {
+                                // padding: the rest of this row, or, below the image, the rest of the canvas
+                                const int64_t room = r < rows ? row_stride - in : (int64_t)(rows_max - r) * row_stride - in;
+                                const int64_t len = min(room, seg_e - cur);
                                 if (!UNPACK) warp_fill(dst_base + dense_off + cur, len, pad, lane);
                                 cur += len; in += len;
                             }
-                            if (in == slot_bytes) { in = 0; ++slot; }
+                            if (in >= row_stride) {  // on to the next canvas row(s)
+                                const int adv = (int)(in / row_stride);
+                                in -= (int64_t)adv * row_stride;
+                                r += adv;
+                                if (r >= rows_max) { r = 0; ++slot; }
+                            }
                         }
                     }
-                    if (cur == (int64_t)nx * slot_bytes) { ++k; slot = nx; in = 0; }
+                    if (cur == (int64_t)nx * slot_bytes) { ++k; slot = nx; r = 0; in = 0; }
                 }
             }
         }
@@ -157,30 +179,31 @@ __global__ void __launch_bounds__(256, 2) k16_copy_var(PlanView pv, int32_t t_bl
 
 }  // namespace
 
-cudaError_t launch_var_offsets(const int32_t* lengths, const int32_t* frame_bytes, int64_t n, int64_t* out, cudaStream_t st)
+cudaError_t launch_var_offsets(const int32_t* lengths, const int32_t* rows, const int32_t* frame_bytes, int64_t n,
+                               int64_t* out, int64_t* max_rows, cudaStream_t st)
 {
     count_launches(1);
-    k15_var_offsets<<<1, kScanThreads, 0, st>>>(lengths, frame_bytes, n, out);
+    k15_var_offsets<<<1, kScanThreads, 0, st>>>(lengths, rows, frame_bytes, n, out, max_rows);
     return cudaPeekAtLastError();
 }
 
-cudaError_t launch_copy_var(bool unpack, const PlanView& pv, int32_t t_block, int64_t slot_bytes, int64_t block_begin,
-                            int64_t block_count, const int32_t* frame_bytes, const int64_t* byte_offsets,
-                            const uint8_t* src, uint8_t* dst, uint8_t pad_byte, cudaStream_t st)
+cudaError_t launch_copy_var(bool unpack, const PlanView& pv, int32_t t_block, int32_t rows_max, int64_t row_stride,
+                            int64_t block_begin, int64_t block_count, const int32_t* seq_rows, const int32_t* frame_bytes,
+                            const int64_t* byte_offsets, const uint8_t* src, uint8_t* dst, uint8_t pad_byte, cudaStream_t st)
 {
     if (block_count == 0) return cudaSuccess;
-    const int64_t block_bytes = (int64_t)t_block * slot_bytes;
+    const int64_t block_bytes = (int64_t)t_block * rows_max * row_stride;
     const int64_t sub = 16384;
     const int64_t spb = (block_bytes + sub - 1) / sub;
     const int64_t want = (block_count * spb + 7) / 8;
     const unsigned grid = (unsigned)(want < 0x7fffffffLL ? want : 0x7fffffffLL);
     count_launches(1);
     if (unpack)
-        k16_copy_var<true><<<grid, 256, 0, st>>>(pv, t_block, slot_bytes, block_begin, block_count, frame_bytes, byte_offsets,
-                                                  src, dst, sub, spb, pad_byte);
+        k16_copy_var<true><<<grid, 256, 0, st>>>(pv, t_block, rows_max, row_stride, block_begin, block_count, seq_rows,
+                                                  frame_bytes, byte_offsets, src, dst, sub, spb, pad_byte);
     else
-        k16_copy_var<false><<<grid, 256, 0, st>>>(pv, t_block, slot_bytes, block_begin, block_count, frame_bytes, byte_offsets,
-                                                   src, dst, sub, spb, pad_byte);
+        k16_copy_var<false><<<grid, 256, 0, st>>>(pv, t_block, rows_max, row_stride, block_begin, block_count, seq_rows,
+                                                   frame_bytes, byte_offsets, src, dst, sub, spb, pad_byte);
     return cudaPeekAtLastError();
 }
 

@@ -119,3 +119,65 @@ def test_var_calls_reject_bad_arguments():
         with pytest.raises(B.BloadError) as e:
             B.bload_unpack_var(plan, *args)
         assert e.value.code == code
+
+
+def _parity2d(T, H, Wb, tb, seed, hmax, stride, pad=0x6B):
+    T = np.ascontiguousarray(T, np.int32); H = np.ascontiguousarray(H, np.int32); Wb = np.ascontiguousarray(Wb, np.int32)
+    op = O.plan(T, tb, seed)
+    plan = G.gpu_plan(T, tb, seed)
+    d_T, d_H, d_W = (torch.from_numpy(x).to(G.DEV) for x in (T, H, Wb))
+    boff, info = B.bload_var_offsets2d(d_T, d_H, d_W)
+    want_off = O.byte_offsets2d(T, H, Wb)
+    assert np.array_equal(boff[:T.size + 1].cpu().numpy(), want_off)
+    assert (info.total_bytes, info.max_frame_bytes, info.max_rows, info.first_bad_index) == \
+        (int(want_off[-1]), int(Wb.max()), int(H.max()), -1)
+    total = int(want_off[-1])
+    g = torch.Generator(device=G.DEV); g.manual_seed(seed)
+    store = torch.randint(0, 256, (total,), dtype=torch.uint8, device=G.DEV, generator=g)
+    store_h = store.cpu().numpy()
+    canvas = hmax * stride
+    for b0, cnt in ((0, op.n_blocks + 2), (1, max(op.n_blocks - 1, 1))):
+        dense = G.Guarded(cnt * tb * canvas)
+        B.bload_pack_var2d(plan, store, d_H, d_W, boff, hmax, stride, b0, cnt, dense.t, pad_byte=pad)
+        torch.cuda.synchronize(); dense.check()
+        d = G.first_diff(dense.t.cpu().numpy(), O.pack_var2d(op, store_h, H, Wb, hmax, stride, b0, cnt, pad))
+        assert d is None, "pack_var2d %dx%d blocks [%d,+%d): %s" % (hmax, stride, b0, cnt, d)
+        dense_out = torch.randint(0, 256, (cnt * tb * canvas,), dtype=torch.uint8, device=G.DEV, generator=g)
+        rag = G.Guarded(total, 0x5A)
+        B.bload_unpack_var2d(plan, dense_out, d_H, d_W, boff, hmax, stride, b0, cnt, rag.t)
+        torch.cuda.synchronize(); rag.check()
+        want = np.full(total, 0x5A, np.uint8)
+        O.unpack_var2d(op, dense_out.cpu().numpy(), H, Wb, hmax, stride, b0, cnt, want)
+        d = G.first_diff(rag.t.cpu().numpy(), want)
+        assert d is None, "unpack_var2d %dx%d blocks [%d,+%d): %s" % (hmax, stride, b0, cnt, d)
+
+
+@pytest.mark.parametrize("hmax,wmax,extra", [(1, 7, 0), (3, 5, 2), (4, 16, 0), (7, 33, 5), (16, 100, 0), (40, 700, 4),
+                                             (224, 672, 0)])
+def test_images_on_canvases(hmax, wmax, extra):
+    rng = np.random.default_rng(hmax * 1000 + wmax)
+    tb = int(rng.integers(3, 30))
+    n = int(rng.integers(2, 60))
+    T = rng.integers(1, tb + 1, size=n)
+    H = rng.integers(1, hmax + 1, size=n)
+    Wb = rng.integers(1, wmax + 1, size=n)
+    H[0], Wb[0] = hmax, wmax  # one image fills its canvas (when extra == 0): the contiguous path
+    _parity2d(T, H, Wb, tb, 5 + hmax, hmax, wmax + extra)
+
+
+def test_canvases_of_equal_images_match_the_fixed_size_pack():
+    rng = np.random.default_rng(8)
+    tb, h, wb = 30, 6, 48
+    T = rng.integers(1, tb + 1, size=100).astype(np.int32)
+    plan = G.gpu_plan(T, tb, 2)
+    d_T = torch.from_numpy(T).to(G.DEV)
+    d_H = torch.full((T.size,), h, dtype=torch.int32, device=G.DEV)
+    d_W = torch.full((T.size,), wb, dtype=torch.int32, device=G.DEV)
+    boff, info = B.bload_var_offsets2d(d_T, d_H, d_W)
+    store = torch.randint(0, 256, (info.total_bytes,), dtype=torch.uint8, device=G.DEV)
+    nb = plan.n_blocks + 1
+    a = torch.empty(nb * tb * h * wb, dtype=torch.uint8, device=G.DEV); b = torch.empty_like(a)
+    B.bload_pack_var2d(plan, store, d_H, d_W, boff, h, wb, 0, nb, a, pad_byte=3)
+    B.bload_pack(plan, store, h * wb, 0, nb, dense=b, pad_byte=3)
+    torch.cuda.synchronize()
+    assert torch.equal(a, b)
