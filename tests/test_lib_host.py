@@ -87,3 +87,50 @@ def test_null_and_range_errors_without_a_device():
     assert L.bload_pack(264, C.byref(ok), None, 1, 0, 1, None, None, None, None, None, 0, None) == _lib.ERR_ALIGN
     out = (C.c_float * 4)()
     assert L.bload_plan_stage_times(C.byref(out)) == _lib.ERR_PLAN
+
+
+def test_newer_entry_points_reject_bad_arguments_before_any_launch():
+    """Errors the host can see return before the library touches the device, so they can be checked without one."""
+    L = B.load()
+    E = _lib
+    ok = B.PlanInfo(status=0, t_block=4, n=5, n_blocks=2, sum_t=7, t_max=3)
+    p = C.byref(ok)
+    # consumer side
+    assert L.bload_carry_prev(None, p, 256, 4, 0, 1, 512, 0, None) == E.ERR_NULL
+    assert L.bload_carry_prev(256, p, None, 4, 0, 1, 512, 0, None) == E.ERR_NULL
+    assert L.bload_carry_prev(256, p, 512, 4, 0, 1, 512, 0, None) == E.ERR_ARG       # in place
+    assert L.bload_carry_prev(256, p, 512, 0, 0, 1, 1024, 0, None) == E.ERR_ARG      # frame size
+    assert L.bload_carry_prev(256, p, 520, 4, 0, 1, 1024, 0, None) == E.ERR_ALIGN
+    assert L.bload_reset_state(256, p, 0, 1, 4, 512, 16, None, None) == E.ERR_ARG    # slot == t_block
+    assert L.bload_reset_state(256, p, 0, 1, 0, None, 16, None, None) == E.ERR_NULL
+    assert L.bload_reset_state(256, p, 0, 1, 0, 512, 16, 8, None) == E.ERR_ALIGN     # init not 16-byte aligned
+    assert L.bload_valid_sum(256, p, None, 0, 1, 512, None, None) == E.ERR_NULL
+    assert L.bload_valid_sum(256, p, 512, 0, -1, 512, None, None) == E.ERR_ARG
+    assert L.bload_valid_sum(256, p, 512, 0, 1, 516, None, None) == E.ERR_ALIGN
+    # per-sample frame sizes
+    vi = E.VarInfo()
+    assert L.bload_var_offsets(None, 512, 5, 1024, None, C.byref(vi)) == E.ERR_NULL
+    assert L.bload_var_offsets(256, 512, 0, 1024, None, C.byref(vi)) == E.ERR_ARG
+    assert L.bload_var_offsets(256, 512, 5, 1028, None, C.byref(vi)) == E.ERR_ALIGN
+    assert L.bload_var_offsets(256, 512, 5, 1024, None, None) == E.ERR_NULL
+    assert L.bload_pack_var(256, p, 512, None, 1024, 16, 0, 1, 2048, 0, None) == E.ERR_NULL
+    assert L.bload_pack_var(256, p, 512, 768, 1024, 0, 0, 1, 2048, 0, None) == E.ERR_ARG
+    assert L.bload_unpack_var(256, p, 520, 768, 1024, 16, 0, 1, 2048, None) == E.ERR_ALIGN
+    assert L.bload_pack_var2d(256, p, 512, None, 768, 1024, 2, 16, 0, 1, 2048, 0, None) == E.ERR_NULL  # rows missing
+    assert L.bload_pack_var2d(256, p, 512, 640, 768, 1024, 0, 16, 0, 1, 2048, 0, None) == E.ERR_ARG    # rows_max
+    # the whole step in one call
+    io = E.EpochIO(512, 4, 1024, None, None, None, None, None, 0, None, 8, 0, 0)
+    info = B.PlanInfo()
+    assert L.bload_epoch(None, 5, 4, 0, 256, 1 << 20, 512, 1 << 20, C.byref(io), None, None, C.byref(info)) == E.ERR_NULL
+    assert L.bload_epoch(256, 5, 4, 0, 256, 1 << 20, 512, 1 << 20, None, None, None, C.byref(info)) == E.ERR_NULL
+    assert L.bload_epoch(256, 0, 4, 0, 256, 1 << 20, 512, 1 << 20, C.byref(io), None, None, C.byref(info)) == E.ERR_ARG
+    assert L.bload_epoch(256, 5, 4, 0, 256, 16, 512, 1 << 20, C.byref(io), None, None, C.byref(info)) == E.ERR_WORKSPACE
+    bad = E.EpochIO(None, 4, 1024, None, None, None, None, None, 0, None, 8, 0, 0)          # dense without a store
+    assert L.bload_epoch(256, 5, 4, 0, 256, 1 << 20, 512, 1 << 20, C.byref(bad), None, None, C.byref(info)) == E.ERR_NULL
+    bad = E.EpochIO(512, 4, 1024, None, None, None, None, None, 0, None, 0, 0, 0)           # no rows for the outputs
+    assert L.bload_epoch(256, 5, 4, 0, 256, 1 << 20, 512, 1 << 20, C.byref(bad), None, None, C.byref(info)) == E.ERR_ARG
+    bad = E.EpochIO(512, 4, 1024, None, None, None, None, None, 0, None, 8, 0, 33)          # too many chunks
+    assert L.bload_epoch(256, 5, 4, 0, 256, 1 << 20, 512, 1 << 20, C.byref(bad), None, None, C.byref(info)) == E.ERR_ARG
+    out5 = (C.c_float * 5)()
+    assert L.bload_epoch_stage_times(C.byref(out5)) == E.ERR_PLAN
+    assert L.bload_pack_repeat_last(None, p, None, 1, 0, 1, None, None, None, None, None, 0, None) == E.ERR_NULL
