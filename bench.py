@@ -20,6 +20,7 @@ import subprocess
 import sys
 import threading
 import time
+from types import SimpleNamespace
 
 ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
@@ -221,101 +222,10 @@ def config_of(w, extra) -> dict:
 
 
 # ----------------------------------------------------------------------------------------------
-def run_gpu(args, w) -> dict:
-    import torch
-    import torch.distributed as dist
-
-    import paper_2310_10879_b200 as B
-    from paper_2310_10879_b200 import workloads as W
-
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
-    if not torch.cuda.is_available():
-        raise RuntimeError("bench.py needs a CUDA device: there is no CPU fallback of the packing path")
-    B.load()
-    torch.cuda.set_device(local)
-    dev = torch.device("cuda", local)
-    if world > 1 and not dist.is_initialized():
-        dist.init_process_group("nccl", device_id=dev)
-
-    T = W.lengths(w)
-    fb, ofb, tb = w.frame_bytes, w.out_frame_bytes, w.t_block
-    d_len = torch.from_numpy(T).to(dev)
-    sizes = B.bload_plan_sizes(T.size, tb)
-    plan_buf = torch.empty(sizes.plan_bytes, dtype=torch.uint8, device=dev)
-    work = torch.empty(sizes.work_bytes, dtype=torch.uint8, device=dev)
-    plan = B.bload_plan(d_len, tb, w.seed, policy=args.policy, work=work, plan_buf=plan_buf)
-    nb, sum_t = plan.n_blocks, plan.sum_t
-    by = algorithmic_bytes(sum_t, nb, tb, fb, ofb)
-
-    store = W.payload_torch(w, sum_t, dev).view(torch.uint8).reshape(-1)
-    dense = torch.empty(nb * tb * fb, dtype=torch.uint8, device=dev)
-    seq_id = torch.empty(nb * tb, dtype=torch.int32, device=dev)
-    pos = torch.empty(nb * tb, dtype=torch.int32, device=dev)
-    reset = torch.empty(nb * tb, dtype=torch.uint8, device=dev)
-    valid = torch.empty(nb * tb, dtype=torch.uint8, device=dev)
-    dense_out = W.payload_torch(w, nb * tb, dev, out=True).view(torch.uint8).reshape(-1)
-    ragged_out = torch.empty(sum_t * ofb, dtype=torch.uint8, device=dev)
-
-    ev = lambda: torch.cuda.Event(enable_timing=True)
-
-    def step(rec=None):
-        e = [ev() for _ in range(5)] if rec is not None else None
-        if e: e[0].record()
-        p = B.bload_plan(d_len, tb, w.seed, policy=args.policy, work=work, plan_buf=plan_buf)
-        if e: e[1].record()
-        B.bload_pack(p, None, fb, 0, nb, seq_id=seq_id, pos=pos, reset=reset, valid=valid)
-        if e: e[2].record()
-        B.bload_pack(p, store, fb, 0, nb, dense=dense)
-        if e: e[3].record()
-        B.bload_unpack(p, dense_out, ofb, 0, nb, ragged_out)
-        if e: e[4].record()
-        st = B.bload_stats(p.info)
-        if rec is not None:
-            rec.append((e, st))
-        return st
-
-    def barrier():
-        if world > 1:
-            dist.barrier()
-        torch.cuda.synchronize()
-
-    sampler = ClockSampler(local)
-    sampler.start()
-    for _ in range(args.warmup):
-        step()
-    barrier()
-    launches0 = B.bload_kernel_launches()
-    rec = []
-    t_begin, t_end = ev(), ev()
-    barrier()
-    sampler.mark()
-    t_begin.record()
-    for _ in range(args.steps):
-        stats = step(rec)
-    t_end.record()
-    barrier()
-    launches = B.bload_kernel_launches() - launches0
-    # planner stage times from a few extra, untimed plans (the library's stage events stay out of the timed steps)
-    B.bload_set_plan_timing(True)
-    stage_runs = []
-    for _ in range(5):
-        B.bload_plan(d_len, tb, w.seed, policy=args.policy, work=work, plan_buf=plan_buf)
-        stage_runs.append(B.bload_plan_stage_times())
-    B.bload_set_plan_timing(False)
-    seconds = dist_max(t_begin.elapsed_time(t_end) / 1e3, dev)
-    clocks = sampler.stop()
-
-    def avg(i):
-        return sum(r[0][i].elapsed_time(r[0][i + 1]) for r in rec) / len(rec)
-    plan_ms, meta_ms, pack_ms, unpack_ms = avg(0), avg(1), avg(2), avg(3)
-    stage = [sum(r[i] for r in stage_runs) / len(stage_runs) for i in range(4)]
-    step_s = seconds / args.steps
-    value = aggregate(by["pack"] + by["unpack"], world, step_s) / 1e9
-
-    # ---- the same work as a two-stage pipeline: the plan of epoch e+1 runs on a side stream (one warp of one SM)
-    # under the metadata/pack/unpack traffic of epoch e; and eight plans side by side on eight streams
+# ---- the same work as a two-stage pipeline: the plan of epoch e+1 runs on a side stream (one warp of one SM)
+# under the metadata/pack/unpack traffic of epoch e; and eight plans side by side on eight streams
+def _time_pipelined(c):
+    torch, B, W, args, w, T, fb, ofb, tb, d_len, sizes, plan_buf, work, plan, nb, sum_t, by, store, dense, seq_id, pos, reset, valid, dense_out, ragged_out, ev, barrier, world, dev = (c.torch, c.B, c.W, c.args, c.w, c.T, c.fb, c.ofb, c.tb, c.d_len, c.sizes, c.plan_buf, c.work, c.plan, c.nb, c.sum_t, c.by, c.store, c.dense, c.seq_id, c.pos, c.reset, c.valid, c.dense_out, c.ragged_out, c.ev, c.barrier, c.world, c.dev)
     pipelined = None
     if not args.no_pipeline:
         side = torch.cuda.Stream(priority=-1)   # the planner's small kernels go ahead of queued copy CTAs
@@ -366,9 +276,13 @@ def run_gpu(args, w) -> dict:
                              "plans, packs and unpacks one whole epoch)",
                      "eight_plans_side_by_side_ms": t8, "plans_per_s": 8e3 / t8}
         del bufs, work2, jobs8
+    return pipelined
 
-    # ---- the whole step as ONE call (bload_epoch): the fill rule in chunks on this stream, tables, metadata, pack and
-    # unpack of the blocks each chunk has closed on a side stream under the next chunk
+
+# ---- the whole step as ONE call (bload_epoch): the fill rule in chunks on this stream, tables, metadata, pack and
+# unpack of the blocks each chunk has closed on a side stream under the next chunk
+def _time_fused_epoch(c):
+    torch, B, W, args, w, T, fb, ofb, tb, d_len, sizes, plan_buf, work, plan, nb, sum_t, by, store, dense, seq_id, pos, reset, valid, dense_out, ragged_out, ev, barrier, world, dev = (c.torch, c.B, c.W, c.args, c.w, c.T, c.fb, c.ofb, c.tb, c.d_len, c.sizes, c.plan_buf, c.work, c.plan, c.nb, c.sum_t, c.by, c.store, c.dense, c.seq_id, c.pos, c.reset, c.valid, c.dense_out, c.ragged_out, c.ev, c.barrier, c.world, c.dev)
     fused = None
     if not args.no_fused:
         side2 = torch.cuda.Stream()
@@ -400,9 +314,13 @@ def run_gpu(args, w) -> dict:
                          "finished blocks on a side stream while the fill rule is still running",
                  "stage_ms_summed_over_chunks": {"fill": st_ms[0], "tables": st_ms[1], "metadata": st_ms[2],
                                                  "pack": st_ms[3], "unpack": st_ms[4]}}
+    return fused
 
-    # ---- batch-by-batch use: one pack call (metadata + dense) per training batch of w.batch_blocks blocks,
-    # the last batch rounded up with filler blocks; the output buffers of one batch are reused
+
+# ---- batch-by-batch use: one pack call (metadata + dense) per training batch of w.batch_blocks blocks,
+# the last batch rounded up with filler blocks; the output buffers of one batch are reused
+def _time_per_batch(c):
+    torch, B, W, args, w, T, fb, ofb, tb, d_len, sizes, plan_buf, work, plan, nb, sum_t, by, store, dense, seq_id, pos, reset, valid, dense_out, ragged_out, ev, barrier, world, dev = (c.torch, c.B, c.W, c.args, c.w, c.T, c.fb, c.ofb, c.tb, c.d_len, c.sizes, c.plan_buf, c.work, c.plan, c.nb, c.sum_t, c.by, c.store, c.dense, c.seq_id, c.pos, c.reset, c.valid, c.dense_out, c.ragged_out, c.ev, c.barrier, c.world, c.dev)
     bb = w.batch_blocks
     n_batches = (nb + bb - 1) // bb
     per_batch = None
@@ -445,9 +363,13 @@ def run_gpu(args, w) -> dict:
             per_batch["graph_us_per_call"] = None
             per_batch["graph_error"] = str(exc)[:200]
         del b_dense, b_meta
+    return per_batch
 
-    # ---- consumer side of the start table (not part of the step): the shifted copy over the whole epoch, the
-    # masked sum of a per-slot loss, and the per-slot state reset of a batch
+
+# ---- consumer side of the start table (not part of the step): the shifted copy over the whole epoch, the
+# masked sum of a per-slot loss, and the per-slot state reset of a batch
+def _time_consumer(c):
+    torch, B, W, args, w, T, fb, ofb, tb, d_len, sizes, plan_buf, work, plan, nb, sum_t, by, store, dense, seq_id, pos, reset, valid, dense_out, ragged_out, ev, barrier, world, dev = (c.torch, c.B, c.W, c.args, c.w, c.T, c.fb, c.ofb, c.tb, c.d_len, c.sizes, c.plan_buf, c.work, c.plan, c.nb, c.sum_t, c.by, c.store, c.dense, c.seq_id, c.pos, c.reset, c.valid, c.dense_out, c.ragged_out, c.ev, c.barrier, c.world, c.dev)
     consumer = None
     if not args.no_consumer:
         def timed(fn, reps):
@@ -500,8 +422,12 @@ def run_gpu(args, w) -> dict:
                     "reset_state": {"us_per_call": ms_reset * 1e3, "batch_blocks": bb, "state_bytes": 4096},
                     "var_frames": var}
         del vals, bsum, tot, state
+    return consumer
 
-    # ---- end to end through the same calls with HOST buffers (pinned), copies inside the timed region
+
+# ---- end to end through the same calls with HOST buffers (pinned), copies inside the timed region
+def _time_end_to_end(c):
+    torch, B, W, args, w, T, fb, ofb, tb, d_len, sizes, plan_buf, work, plan, nb, sum_t, by, store, dense, seq_id, pos, reset, valid, dense_out, ragged_out, ev, barrier, world, dev = (c.torch, c.B, c.W, c.args, c.w, c.T, c.fb, c.ofb, c.tb, c.d_len, c.sizes, c.plan_buf, c.work, c.plan, c.nb, c.sum_t, c.by, c.store, c.dense, c.seq_id, c.pos, c.reset, c.valid, c.dense_out, c.ragged_out, c.ev, c.barrier, c.world, c.dev)
     e2e = None
     e2e_need = T.size * 4 + store.numel() + dense_out.numel() + dense.numel() + 10 * nb * tb + ragged_out.numel()
     e2e_second_set = 1.05 * (store.numel() + dense_out.numel() + dense.numel() + 10 * nb * tb + ragged_out.numel())
@@ -608,7 +534,111 @@ def run_gpu(args, w) -> dict:
                       "overlap the downloads of step i; timed from the first upload to the last download of the last step"}
         del sets
         del h_store, h_dense, h_dense_out, h_ragged_out
+    return e2e
 
+
+def run_gpu(args, w) -> dict:
+    import torch
+    import torch.distributed as dist
+
+    import paper_2310_10879_b200 as B
+    from paper_2310_10879_b200 import workloads as W
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: there is no CPU fallback of the packing path")
+    B.load()
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1 and not dist.is_initialized():
+        dist.init_process_group("nccl", device_id=dev)
+
+    T = W.lengths(w)
+    fb, ofb, tb = w.frame_bytes, w.out_frame_bytes, w.t_block
+    d_len = torch.from_numpy(T).to(dev)
+    sizes = B.bload_plan_sizes(T.size, tb)
+    plan_buf = torch.empty(sizes.plan_bytes, dtype=torch.uint8, device=dev)
+    work = torch.empty(sizes.work_bytes, dtype=torch.uint8, device=dev)
+    plan = B.bload_plan(d_len, tb, w.seed, policy=args.policy, work=work, plan_buf=plan_buf)
+    nb, sum_t = plan.n_blocks, plan.sum_t
+    by = algorithmic_bytes(sum_t, nb, tb, fb, ofb)
+
+    store = W.payload_torch(w, sum_t, dev).view(torch.uint8).reshape(-1)
+    dense = torch.empty(nb * tb * fb, dtype=torch.uint8, device=dev)
+    seq_id = torch.empty(nb * tb, dtype=torch.int32, device=dev)
+    pos = torch.empty(nb * tb, dtype=torch.int32, device=dev)
+    reset = torch.empty(nb * tb, dtype=torch.uint8, device=dev)
+    valid = torch.empty(nb * tb, dtype=torch.uint8, device=dev)
+    dense_out = W.payload_torch(w, nb * tb, dev, out=True).view(torch.uint8).reshape(-1)
+    ragged_out = torch.empty(sum_t * ofb, dtype=torch.uint8, device=dev)
+
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+
+    def step(rec=None):
+        e = [ev() for _ in range(5)] if rec is not None else None
+        if e: e[0].record()
+        p = B.bload_plan(d_len, tb, w.seed, policy=args.policy, work=work, plan_buf=plan_buf)
+        if e: e[1].record()
+        B.bload_pack(p, None, fb, 0, nb, seq_id=seq_id, pos=pos, reset=reset, valid=valid)
+        if e: e[2].record()
+        B.bload_pack(p, store, fb, 0, nb, dense=dense)
+        if e: e[3].record()
+        B.bload_unpack(p, dense_out, ofb, 0, nb, ragged_out)
+        if e: e[4].record()
+        st = B.bload_stats(p.info)
+        if rec is not None:
+            rec.append((e, st))
+        return st
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    sampler = ClockSampler(local)
+    sampler.start()
+    for _ in range(args.warmup):
+        step()
+    barrier()
+    launches0 = B.bload_kernel_launches()
+    rec = []
+    t_begin, t_end = ev(), ev()
+    barrier()
+    sampler.mark()
+    t_begin.record()
+    for _ in range(args.steps):
+        stats = step(rec)
+    t_end.record()
+    barrier()
+    launches = B.bload_kernel_launches() - launches0
+    # planner stage times from a few extra, untimed plans (the library's stage events stay out of the timed steps)
+    B.bload_set_plan_timing(True)
+    stage_runs = []
+    for _ in range(5):
+        B.bload_plan(d_len, tb, w.seed, policy=args.policy, work=work, plan_buf=plan_buf)
+        stage_runs.append(B.bload_plan_stage_times())
+    B.bload_set_plan_timing(False)
+    seconds = dist_max(t_begin.elapsed_time(t_end) / 1e3, dev)
+    clocks = sampler.stop()
+
+    def avg(i):
+        return sum(r[0][i].elapsed_time(r[0][i + 1]) for r in rec) / len(rec)
+    plan_ms, meta_ms, pack_ms, unpack_ms = avg(0), avg(1), avg(2), avg(3)
+    stage = [sum(r[i] for r in stage_runs) / len(stage_runs) for i in range(4)]
+    step_s = seconds / args.steps
+    value = aggregate(by["pack"] + by["unpack"], world, step_s) / 1e9
+
+    c = SimpleNamespace(torch=torch, B=B, W=W, args=args, w=w, T=T, fb=fb, ofb=ofb, tb=tb, d_len=d_len, sizes=sizes,
+                        plan_buf=plan_buf, work=work, plan=plan, nb=nb, sum_t=sum_t, by=by, store=store, dense=dense,
+                        seq_id=seq_id, pos=pos, reset=reset, valid=valid, dense_out=dense_out, ragged_out=ragged_out,
+                        ev=ev, barrier=barrier, world=world, dev=dev)
+    pipelined = _time_pipelined(c)
+    fused = _time_fused_epoch(c)
+    per_batch = _time_per_batch(c)
+    consumer = _time_consumer(c)
+    e2e = _time_end_to_end(c)
     if rank != 0:
         return {}
 
