@@ -110,3 +110,32 @@ def test_epoch_capacity_too_small_and_bad_arguments():
     with pytest.raises(B.BloadError) as e:
         B.bload_epoch(torch.from_numpy(bad).to(G.DEV), 30, 9, cap, store=store, frame_bytes=fb, dense=dense.t)
     assert e.value.code == -3 and e.value.info.first_bad_index == 77
+
+
+@pytest.mark.parametrize("chunks", [1, 2, 7, 32])
+def test_epoch_with_any_number_of_chunks(chunks):
+    # the number of launches of the fill rule changes where the chain pauses, never what it computes: few draws per
+    # chunk (chunks that end after one block), chunks that find the plan already finished, a single chunk
+    rng = np.random.default_rng(chunks)
+    tb = 64
+    T = np.minimum(rng.geometric(1.0 / 9, size=700), tb).astype(np.int32)
+    op = O.plan(T, tb, 5)
+    cap = op.n_blocks + 1
+    fb = 32
+    store = torch.randint(0, 256, (op.sum_t * fb,), dtype=torch.uint8, device=G.DEV)
+    dense = G.Guarded(cap * tb * fb)
+    valid = torch.empty(cap * tb, dtype=torch.uint8, device=G.DEV)
+    plan = B.bload_epoch(torch.from_numpy(T).to(G.DEV), tb, 5, cap, store=store, frame_bytes=fb, dense=dense.t,
+                         valid=valid, side_stream=torch.cuda.Stream(), chunks=chunks)
+    dense.check()
+    G.assert_plan_equal(plan, op)
+    assert np.array_equal(dense.t.cpu().numpy().reshape(cap, tb, fb), O.pack(op, store.cpu().numpy(), fb, 0, cap, 0))
+    assert np.array_equal(valid.cpu().numpy().reshape(cap, tb), O.metadata(op, 0, cap)[3])
+    # a tiny problem with more chunks than sequences
+    T2 = np.array([3, 1, 2], np.int32)
+    op2 = O.plan(T2, 3, 1)
+    d2 = torch.empty(op2.n_blocks * 3 * 8, dtype=torch.uint8, device=G.DEV)
+    s2 = torch.randint(0, 256, (op2.sum_t * 8,), dtype=torch.uint8, device=G.DEV)
+    p2 = B.bload_epoch(torch.from_numpy(T2).to(G.DEV), 3, 1, op2.n_blocks, store=s2, frame_bytes=8, dense=d2, chunks=chunks)
+    G.assert_plan_equal(p2, op2)
+    assert np.array_equal(d2.cpu().numpy().reshape(op2.n_blocks, 3, 8), O.pack(op2, s2.cpu().numpy(), 8, 0, op2.n_blocks, 0))
