@@ -20,6 +20,9 @@
  *                      (reachable set, exact probabilities, chi-square),
  *                      maximality and no-drop/no-split invariants, the toy
  *                      dataset of the paper (8 videos, lengths 2..6)
+ *   plan digest        recomputed from the segment list with Python integers (MurmurHash3's
+ *                      published finaliser typed in the test), on plans whose block and
+ *                      sequence numbers pass 2^16; field swaps and reorderings
  *   stats              closed forms; the paper's Table I "0 padding" count
  *   metadata/pack/unpack  numpy fancy-index gather built from the tables,
  *                      round trip, pad bytes

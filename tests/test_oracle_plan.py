@@ -301,3 +301,51 @@ def test_policy1_random_small_cases_stay_in_reachable_set():
             p = O.plan(T, tb, seed, policy=1)
             _check(p)
             assert brute.outcome_of_plan(T, p.n_blocks, p.seg_seq, p.block_seg_begin) in dist
+
+
+# ---- the plan digest, recomputed with Python integers ----
+
+def _digest_with_python_integers(seg_block, seg_start, seg_seq):
+    """Wrapping 64-bit sum, over the segments, of the 64-bit finaliser of MurmurHash3 (Appleby's public-domain
+    fmix64: xor-shift 33, multiply, xor-shift 33, multiply, xor-shift 33) applied to
+    (block << 32 | start) * golden-ratio constant + sequence.  Arbitrary-precision integers masked to 64 bits."""
+    M = (1 << 64) - 1
+    total = 0
+    for b, s, q in zip(seg_block.tolist(), seg_start.tolist(), seg_seq.tolist()):
+        k = ((((b & 0xFFFFFFFF) << 32) | (s & 0xFFFFFFFF)) * 0x9E3779B97F4A7C15 + (q & 0xFFFFFFFF)) & M
+        k ^= k >> 33
+        k = (k * 0xFF51AFD7ED558CCD) & M
+        k ^= k >> 33
+        k = (k * 0xC4CEB9FE1A85EC53) & M
+        k ^= k >> 33
+        total = (total + k) & M
+    return total
+
+
+@pytest.mark.parametrize("policy", [0, 1, 2])
+def test_checksum_equals_a_big_integer_recomputation(policy):
+    for name in ("toy_video", "features_fp16", "video_dataset_shape"):
+        w = W.WORKLOADS[name]
+        p = O.plan(W.lengths(w), w.t_block, seed=w.seed, policy=policy)
+        assert p.checksum == _digest_with_python_integers(p.seg_block, p.seg_start, p.seg_seq), name
+
+
+def test_checksum_with_block_and_sequence_numbers_beyond_16_bits():
+    # 70,000 sequences of 3 or 4 frames in blocks of 4: one sequence per block, so block and sequence numbers pass
+    # 2^16 and a digest that truncated either of them, or swapped block and start, would differ
+    rng = np.random.default_rng(7)
+    T = rng.integers(3, 5, size=70000).astype(np.int32)
+    p = O.plan(T, 4, seed=11)
+    assert p.n_blocks == 70000 and int(p.seg_block.max()) >= 1 << 16 and int(p.seg_seq.max()) >= 1 << 16
+    want = _digest_with_python_integers(p.seg_block, p.seg_start, p.seg_seq)
+    assert p.checksum == want
+    # the digest depends on each of the three fields, and not on the order of the segments
+    perm = rng.permutation(T.size)
+    assert _digest_with_python_integers(p.seg_block[perm], p.seg_start[perm], p.seg_seq[perm]) == want
+    assert _digest_with_python_integers(p.seg_block[::-1].copy(), p.seg_start, p.seg_seq) != want
+    assert _digest_with_python_integers(p.seg_start, p.seg_block, p.seg_seq) != want
+    # a plan with non-zero start slots (several sequences per block)
+    T2 = rng.integers(1, 9, size=3000).astype(np.int32)
+    p2 = O.plan(T2, 16, seed=5)
+    assert int(p2.seg_start.max()) > 0
+    assert p2.checksum == _digest_with_python_integers(p2.seg_block, p2.seg_start, p2.seg_seq)
