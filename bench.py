@@ -163,6 +163,32 @@ class CpuOracleSample:
         self.t_plan = time.perf_counter() - t0
         return self.op
 
+    def run_threaded(self, threads: int) -> dict:
+        """The same sample with its blocks spread over `threads` host threads (contiguous block ranges; the oracle's C
+        functions run outside the interpreter lock).  The plan is sequential and is not repeated here."""
+        from concurrent.futures import ThreadPoolExecutor
+        O, w, op = self.O, self.w, self.op
+        fb, ofb = w.frame_bytes, w.out_frame_bytes
+        threads = max(1, min(threads, self.cnt))
+        cuts = [self.b0 + self.cnt * i // threads for i in range(threads + 1)]
+        parts = [(cuts[i], cuts[i + 1] - cuts[i]) for i in range(threads) if cuts[i + 1] > cuts[i]]
+        tbb = w.t_block * ofb
+
+        def do_pack(part):
+            O.pack(op, self.store, fb, part[0], part[1], 0)
+
+        def do_unpack(part):
+            lo = (part[0] - self.b0) * tbb
+            O.unpack(op, self.dense_out[lo:lo + part[1] * tbb], ofb, part[0], part[1], self.ragged_out)
+
+        with ThreadPoolExecutor(max_workers=len(parts)) as pool:
+            t0 = time.perf_counter(); list(pool.map(do_pack, parts)); t_pack = time.perf_counter() - t0
+            t0 = time.perf_counter(); list(pool.map(do_unpack, parts)); t_unpack = time.perf_counter() - t0
+        by = self.bytes
+        return {"cores": len(parts), "pack_GB/s": by["pack"] / t_pack / 1e9, "unpack_GB/s": by["unpack"] / t_unpack / 1e9,
+                "value": (by["pack"] + by["unpack"]) / (t_pack + t_unpack) / 1e9, "unit": UNIT,
+                "what": "pack + unpack of the same blocks spread over host threads (plan and metadata not included)"}
+
     def run(self) -> dict:
         O, w, op = self.O, self.w, self.plan()
         fb, ofb = w.frame_bytes, w.out_frame_bytes
@@ -178,7 +204,8 @@ class CpuOracleSample:
                            % (op.n, self.t_plan, self.cnt, op.n_blocks, self.frames, by["pack"] / t_pack / 1e9,
                               by["unpack"] / t_unpack / 1e9),
                     seconds=self.t_plan + t_meta + t_pack + t_unpack, frames_per_s=self.frames / t_total,
-                    plan_s=self.t_plan, _bytes=by["pack"] + by["unpack"], _t=t_total)
+                    plan_s=self.t_plan, pack_GBs=by["pack"] / t_pack / 1e9, unpack_GBs=by["unpack"] / t_unpack / 1e9,
+                    _bytes=by["pack"] + by["unpack"], _t=t_total)
 
 
 def run_reference(args, w) -> dict:
@@ -643,14 +670,15 @@ def run_gpu(args, w) -> dict:
         return {}
 
     peak, peak_kind = measured_peak()
-    kernels = {"k7_copy<unpack>": (unpack_ms, by["unpack"]), "k7_copy<pack>": (pack_ms, by["pack"]),
-               "k4_fill": (stage[2], None)}
-    dom = max(("k7_copy<unpack>", "k7_copy<pack>"), key=lambda k: kernels[k][0])
+    # the names of the copy kernels are the library's own answer for the calls of the timed steps
+    k_pack, k_unpack = B.bload_last_copy_kernel("pack"), B.bload_last_copy_kernel("unpack")
+    kernels = {k_unpack: (unpack_ms, by["unpack"]), k_pack: (pack_ms, by["pack"]), "k4_fill": (stage[2], None)}
+    dom = max((k_unpack, k_pack), key=lambda k: kernels[k][0])
     d_ms, d_bytes = kernels[dom]
     achieved = d_bytes / (d_ms / 1e3) / 1e9
     roofline = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "GB/s",
                 "frac": achieved / peak, "peak_kind": "of " + peak_kind, "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
-                "traffic": TRAFFIC.get((w.name, dom)) if not (args.n or args.frame_bytes) else None,
+                "traffic": TRAFFIC.get((w.name, dom)) if not (args.n or args.frame_bytes or args.policy) else None,
                 "note": "largest HBM-bound kernel of the step; the planner's fill rule (k4_fill, %.2f ms) is a latency-bound "
                         "chain of dependent draws on one warp and is reported in kernels.plan as time and draws/s" % stage[2], "launch_ms": d_ms, "algorithmic_bytes_per_launch": d_bytes}
 
@@ -660,15 +688,14 @@ def run_gpu(args, w) -> dict:
            "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline,
            "frames_per_s": aggregate(sum_t, world, step_s), "per_batch_pack": per_batch, "pipelined": pipelined, "fused_epoch": fused, "consumer": consumer,
            "kernels": {
-               "pack_copy": {"ms": pack_ms, "GB/s": by["pack"] / pack_ms / 1e6, "frac_measured": by["pack"] / pack_ms / 1e6 / peak,
+               "pack_copy": {"kernel": k_pack, "ms": pack_ms, "GB/s": by["pack"] / pack_ms / 1e6, "frac_measured": by["pack"] / pack_ms / 1e6 / peak,
                              "frac_nominal": by["pack"] / pack_ms / 1e6 / NOMINAL_HBM_GBS, "frames_per_s": sum_t / pack_ms * 1e3},
-               "unpack_copy": {"ms": unpack_ms, "GB/s": by["unpack"] / unpack_ms / 1e6,
+               "unpack_copy": {"kernel": k_unpack, "ms": unpack_ms, "GB/s": by["unpack"] / unpack_ms / 1e6,
                                "frac_measured": by["unpack"] / unpack_ms / 1e6 / peak,
                                "frac_nominal": by["unpack"] / unpack_ms / 1e6 / NOMINAL_HBM_GBS,
                                "frames_per_s": sum_t / unpack_ms * 1e3},
                "metadata": {"ms": meta_ms, "GB/s": by["meta"] / meta_ms / 1e6},
-               "plan": {"ms": plan_ms, "scan_keys_ms": stage[0], "sort_ms": stage[1], "fill_ms": stage[2],
-                        "tables_ms": stage[3], "draws_per_s": T.size / stage[2] * 1e3 if stage[2] > 0 else None}},
+               "plan": plan_figures(plan_ms, stage, T.size, clocks)},
            "padding": {"n": stats["n"], "sum_t": stats["sum_t"], "t_max": stats["t_max"], "n_blocks": stats["n_blocks"],
                        "min_blocks": stats["min_blocks"], "frac_packed": stats["frac_packed"],
                        "frac_naive_tmax": stats["frac_naive_tmax"], "frac_naive_tblock": stats["frac_naive_tblock"],
@@ -678,18 +705,143 @@ def run_gpu(args, w) -> dict:
         need = (fb + ofb) * (sum_t + nb * tb) * 1.3          # host arrays of a whole-workload sample
         if blocks <= 0 and host_memory_available() < need:
             blocks = max(1, int(nb * host_memory_available() / need / 1.5))
-        cb = CpuOracleSample(w, blocks).run()
+        sample = CpuOracleSample(w, blocks)
+        cb = sample.run()
         out["cpu_baseline"] = {k: v for k, v in cb.items() if not k.startswith("_")}
+        out["cpu_baseline"]["all_cores"] = sample.run_threaded(host_cores())
+        del sample
     else:
         out["cpu_baseline"] = None
+    if not args.no_by_config and world == 1 and not (args.n or args.frame_bytes):
+        # the other large configurations, one after the other, with the buffers of this one released first
+        del c, store, dense, seq_id, pos, reset, valid, dense_out, ragged_out, plan, plan_buf, work
+        torch.cuda.empty_cache()
+        out["by_config"] = {name: measure_config(args, W.WORKLOADS[name], dev, peak, clocks)
+                            for name in BY_CONFIG if name != w.name}
     return out
 
 
-# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the committed ncu captures
-# under profiles/; null where the kernel has changed since the counters were taken.
+BY_CONFIG = ("raw_frames", "tokens")
+
+
+def host_cores() -> int:
+    try:
+        return len(os.sched_getaffinity(0))
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def plan_figures(plan_ms, stage, n, clocks) -> dict:
+    """Stage times of the planner; the fill rule (a chain of n dependent draws on one warp) also as time and SM
+    cycles per draw, the cycles from the median SM clock sampled while the timed region ran."""
+    fill_ns = stage[2] * 1e6 / n if n else None
+    mhz = clocks.get("sm_mhz") if clocks else None
+    return {"ms": plan_ms, "scan_keys_ms": stage[0], "sort_ms": stage[1], "fill_ms": stage[2], "tables_ms": stage[3],
+            "draws_per_s": n / stage[2] * 1e3 if stage[2] > 0 else None, "ns_per_draw": fill_ns,
+            "cycles_per_draw": fill_ns * mhz / 1e3 if fill_ns and mhz else None, "sm_mhz_used": mhz}
+
+
+def measure_config(args, w, dev, peak, clocks) -> dict:
+    """Whole-epoch kernel times of one more workload (context beside the headline): every launch bracketed by CUDA
+    events on the launching stream, the kernel names as the library reports them, planner stages, per-batch calls, and
+    the CPU oracle on a bounded sample of the same workload (one thread and all host cores)."""
+    import torch
+
+    import paper_2310_10879_b200 as B
+    from paper_2310_10879_b200 import workloads as W
+
+    T = W.lengths(w)
+    fb, ofb, tb = w.frame_bytes, w.out_frame_bytes, w.t_block
+    d_len = torch.from_numpy(T).to(dev)
+    sizes = B.bload_plan_sizes(T.size, tb)
+    plan_buf = torch.empty(sizes.plan_bytes, dtype=torch.uint8, device=dev)
+    work = torch.empty(sizes.work_bytes, dtype=torch.uint8, device=dev)
+    plan = B.bload_plan(d_len, tb, w.seed, policy=args.policy, work=work, plan_buf=plan_buf)
+    nb, sum_t = plan.n_blocks, plan.sum_t
+    by = algorithmic_bytes(sum_t, nb, tb, fb, ofb)
+    store = W.payload_torch(w, sum_t, dev).view(torch.uint8).reshape(-1)
+    dense = torch.empty(nb * tb * fb, dtype=torch.uint8, device=dev)
+    seq_id = torch.empty(nb * tb, dtype=torch.int32, device=dev)
+    pos = torch.empty(nb * tb, dtype=torch.int32, device=dev)
+    reset = torch.empty(nb * tb, dtype=torch.uint8, device=dev)
+    valid = torch.empty(nb * tb, dtype=torch.uint8, device=dev)
+    dense_out = W.payload_torch(w, nb * tb, dev, out=True).view(torch.uint8).reshape(-1)
+    ragged_out = torch.empty(sum_t * ofb, dtype=torch.uint8, device=dev)
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+
+    def timed(fn, reps=10):
+        for _ in range(3):
+            fn()
+        torch.cuda.synchronize()
+        pairs = []
+        for _ in range(reps):   # inputs and outputs are far larger than L2, so back-to-back launches start cold
+            a, b_ = ev(), ev()
+            a.record(); fn(); b_.record()
+            pairs.append((a, b_))
+        torch.cuda.synchronize()
+        ms = sorted(a.elapsed_time(b_) for a, b_ in pairs)
+        return ms[len(ms) // 2]
+
+    meta_ms = timed(lambda: B.bload_pack(plan, None, fb, 0, nb, seq_id=seq_id, pos=pos, reset=reset, valid=valid))
+    pack_ms = timed(lambda: B.bload_pack(plan, store, fb, 0, nb, dense=dense))
+    k_pack = B.bload_last_copy_kernel("pack")
+    unpack_ms = timed(lambda: B.bload_unpack(plan, dense_out, ofb, 0, nb, ragged_out))
+    k_unpack = B.bload_last_copy_kernel("unpack")
+    prev = torch.empty_like(dense)
+    carry_ms = timed(lambda: B.bload_carry_prev(plan, dense, fb, 0, nb, prev))
+    k_carry = B.bload_last_copy_kernel("carry_prev")
+    del prev
+    cp_bytes = (sum_t - T.size) * fb + nb * tb * fb
+    B.bload_set_plan_timing(True)
+    stage_runs = []
+    t_plan = []
+    for _ in range(3):
+        a, b_ = ev(), ev()
+        a.record()
+        B.bload_plan(d_len, tb, w.seed, policy=args.policy, work=work, plan_buf=plan_buf)
+        b_.record(); torch.cuda.synchronize()
+        t_plan.append(a.elapsed_time(b_))
+        stage_runs.append(B.bload_plan_stage_times())
+    B.bload_set_plan_timing(False)
+    stage = [sum(r[i] for r in stage_runs) / len(stage_runs) for i in range(4)]
+    st = B.bload_stats(plan.info)
+
+    def rate(nbytes, ms):
+        g = nbytes / ms / 1e6
+        return {"ms": ms, "GB/s": g, "frac_measured": g / peak, "frac_nominal": g / NOMINAL_HBM_GBS,
+                "algorithmic_bytes": nbytes}
+    c = SimpleNamespace(torch=torch, B=B, W=W, args=args, w=w, T=T, fb=fb, ofb=ofb, tb=tb, d_len=d_len, sizes=sizes,
+                        plan_buf=plan_buf, work=work, plan=plan, nb=nb, sum_t=sum_t, by=by, store=store, dense=dense,
+                        seq_id=seq_id, pos=pos, reset=reset, valid=valid, dense_out=dense_out, ragged_out=ragged_out,
+                        ev=ev, barrier=torch.cuda.synchronize, world=1, dev=dev)
+    out = {"workload": config_of(w, None)["workload"], "n_blocks": nb, "sum_t": sum_t,
+           "kernels": {"pack_copy": dict(rate(by["pack"], pack_ms), kernel=k_pack, frames_per_s=sum_t / pack_ms * 1e3),
+                       "unpack_copy": dict(rate(by["unpack"], unpack_ms), kernel=k_unpack, frames_per_s=sum_t / unpack_ms * 1e3),
+                       "metadata": dict(rate(by["meta"], meta_ms), kernel="k6_metadata"),
+                       "carry_prev": dict(rate(cp_bytes, carry_ms), kernel=k_carry),
+                       "plan": plan_figures(sum(t_plan) / len(t_plan), stage, T.size, clocks)},
+           "per_batch_pack": _time_per_batch(c),
+           "padding": {"n_blocks": st["n_blocks"], "min_blocks": st["min_blocks"], "frac_packed": st["frac_packed"],
+                       "frac_naive_tmax": st["frac_naive_tmax"], "reduction_vs_tmax": st["reduction_vs_tmax"]}}
+    del c, store, dense, seq_id, pos, reset, valid, dense_out, ragged_out, plan, plan_buf, work
+    torch.cuda.empty_cache()
+    if not args.no_cpu:
+        # bounded sample: about 2 GB of dense blocks from the middle of the epoch
+        blocks = max(1, min(nb, (2 << 30) // max(1, tb * (fb + ofb))))
+        sample = CpuOracleSample(w, blocks)
+        cb = sample.run()
+        out["cpu_baseline"] = {k: v for k, v in cb.items() if not k.startswith("_")}
+        out["cpu_baseline"]["all_cores"] = sample.run_threaded(host_cores())
+        del sample
+    return out
+
+
+# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of one whole-epoch launch, keyed by workload and
+# by the kernel name the library reports; taken once from an ncu capture of a 1,500-sequence case of the same workload
+# and scaled by frames (traffic grows in proportion to the frames moved).  Reads equal the algorithmic bytes, writes are
+# slightly below them (the tail of the output is still in L2 when the kernel ends).  An entry is removed when its
+# kernel changes; a missing entry reports null.
 TRAFFIC: dict = {
-    # scaled by frames from the N=1,500 capture (profiles/k7_copy_small_cases_ncu_full.md): reads equal the
-    # algorithmic bytes, writes are slightly below them (tail of the output still in L2 at kernel end)
     ("heavy_tail_bf16", "k7_copy<unpack>"): 18.29e9,
     ("heavy_tail_bf16", "k7_copy<pack>"): 9.08e9,
 }
@@ -715,6 +867,7 @@ def main():
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--no-consumer", action="store_true")
     ap.add_argument("--no-fused", action="store_true")
+    ap.add_argument("--no-by-config", action="store_true", help="skip the extra measurements of the other large workloads")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "bload" else args.warmup
 

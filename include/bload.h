@@ -45,7 +45,8 @@ extern "C" {
 #define BLOAD_ERR_ALIGN (-5)       /* a device pointer is not aligned as documented */
 #define BLOAD_ERR_UNSUPPORTED (-6) /* t_block above BLOAD_MAX_T_BLOCK, unknown policy */
 #define BLOAD_ERR_CUDA (-7)        /* a CUDA runtime call or launch failed */
-#define BLOAD_ERR_TIMEOUT (-8)     /* a bounded device-side wait expired */
+#define BLOAD_ERR_TIMEOUT (-8)     /* reserved: a bounded device-side wait expired.  No kernel of this version waits on a
+                                      flag (the only waits are for the hardware's own copy groups), so no call returns it */
 #define BLOAD_ERR_PLAN (-9)        /* info/plan do not describe a finished plan */
 
 #define BLOAD_MAX_T_BLOCK 32768
@@ -377,8 +378,11 @@ BLOAD_API int bload_stats(const bload_plan_info_t* info, bload_stats_t* out);
  * cudaFree and no allocating routine of any library.  The price: every GPU that loads the
  * library holds those bytes until the process exits, and the problem size is capped.
  *
- *   d_lengths, n, t_block, seed, policy, d_plan, plan_bytes, stream, info: as for bload_plan
+ *   d_lengths, n, t_block, seed, d_plan, plan_bytes, stream, info: as for bload_plan
  *   (the caller still provides the input and the plan buffer; only d_work/work_bytes are gone).
+ *   policy: BLOAD_POLICY_UNIFORM_SEQUENCES or BLOAD_POLICY_UNIFORM_LENGTHS, the two readings of the
+ *   paper's rule.  BLOAD_POLICY_BEST_FIT_DECREASING needs more scratch per sequence than the array
+ *   was sized for and returns BLOAD_ERR_UNSUPPORTED here; use bload_plan for it.
  *
  * Limits and errors: n > BLOAD_STATIC_MAX_N, or a (n, t_block) whose scratch need exceeds the
  * array, returns BLOAD_ERR_WORKSPACE ("buffer too small") and launches nothing; use bload_plan
@@ -434,6 +438,15 @@ BLOAD_API int bload_plan_stage_times(float out_ms[4]);
  * (all threads).  Host only; lets a benchmark report how many launches a timed region contained.
  */
 BLOAD_API int64_t bload_kernel_launches(void);
+
+/*
+ * bload_last_copy_kernel -- name of the copy kernel that the most recent call of this host thread launched for
+ * which = 0 bload_pack (the dense output), 1 bload_unpack, 2 bload_carry_prev, 3 bload_pack_var[2d],
+ * 4 bload_unpack_var[2d].  The library picks a kernel from the frame size and the run lengths (register path for
+ * large frames, shared-memory staged paths for small word-sized frames); a benchmark reports the choice with this
+ * call instead of guessing it.  Host only.  Returns "" when no such call was made, or for another `which`.
+ */
+BLOAD_API const char* bload_last_copy_kernel(int which);
 
 BLOAD_API const char* bload_strerror(int code);
 BLOAD_API int bload_version(void);

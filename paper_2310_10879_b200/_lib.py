@@ -20,8 +20,8 @@ MAX_T_BLOCK = 32768
 EXPORTS = ("bload_plan_sizes", "bload_plan", "bload_plan_async", "bload_plan_finish", "bload_rank_range", "bload_pack", "bload_unpack", "bload_stats", "bload_epoch", "bload_epoch_stage_times",
            "bload_pack_repeat_last", "bload_var_offsets", "bload_pack_var", "bload_unpack_var", "bload_var_offsets2d", "bload_pack_var2d",
            "bload_unpack_var2d", "bload_carry_prev", "bload_reset_state", "bload_valid_sum",
-           "bload_set_plan_timing", "bload_plan_stage_times", "bload_kernel_launches", "bload_strerror",
-           "bload_version")
+           "bload_plan_static", "bload_set_plan_timing", "bload_plan_stage_times", "bload_kernel_launches", "bload_last_copy_kernel",
+           "bload_strerror", "bload_version")
 
 
 class Sizes(C.Structure):
@@ -73,14 +73,16 @@ def load() -> C.CDLL:
     if _lib is not None:
         return _lib
     if "BLOAD_LIBRARY" not in os.environ:
-        # a missing or stale in-tree library is (re)built from the CUDA sources; if that is impossible, fail loudly
+        # a missing or stale in-tree library is (re)built from the CUDA sources; if that is impossible, fail loudly:
+        # a library built from other sources than the ones in this tree must never run unnoticed
+        from . import build as _build
         try:
-            from . import build as _build
             _build.build()
         except Exception as exc:
-            if not os.path.exists(LIB_PATH):
-                raise RuntimeError("libbload.so is missing at %s and could not be built (%s): there is no CPU "
-                                   "fallback" % (LIB_PATH, exc)) from exc
+            what = "is missing" if not os.path.exists(LIB_PATH) else "was built from other sources than this tree's"
+            raise RuntimeError("libbload.so at %s %s and could not be rebuilt (%s); there is no CPU fallback.  Build it "
+                               "with `python -m paper_2310_10879_b200.build`, or name a library to load with "
+                               "BLOAD_LIBRARY" % (LIB_PATH, what, exc)) from exc
     if not os.path.exists(LIB_PATH):
         raise RuntimeError("libbload.so is missing at %s: build it with `python -m paper_2310_10879_b200.build` "
                            "(there is no CPU fallback)" % LIB_PATH)
@@ -89,6 +91,7 @@ def load() -> C.CDLL:
     L.bload_plan_sizes.argtypes = [i64, i32, C.POINTER(Sizes)]
     L.bload_plan.argtypes = [vp, i64, i32, u64, u32, vp, C.c_size_t, vp, C.c_size_t, vp, C.POINTER(PlanInfo)]
     L.bload_plan_async.argtypes = [vp, i64, i32, u64, u32, vp, C.c_size_t, vp, C.c_size_t, vp]
+    L.bload_plan_static.argtypes = [vp, i64, i32, u64, u32, vp, C.c_size_t, vp, C.POINTER(PlanInfo)]
     L.bload_plan_finish.argtypes = [vp, vp, C.POINTER(PlanInfo)]
     L.bload_rank_range.argtypes = [i64, i32, i32, i32, C.POINTER(i64), C.POINTER(i64)]
     L.bload_pack.argtypes = [vp, C.POINTER(PlanInfo), vp, i64, i64, i64, vp, vp, vp, vp, vp, u8, vp]
@@ -111,12 +114,14 @@ def load() -> C.CDLL:
     L.bload_plan_stage_times.argtypes = [C.POINTER(C.c_float * 4)]
     L.bload_strerror.argtypes = [C.c_int]
     L.bload_strerror.restype = C.c_char_p
+    L.bload_last_copy_kernel.argtypes = [C.c_int]
     L.bload_version.argtypes = []
     L.bload_kernel_launches.argtypes = []
     for name in EXPORTS:
-        if name not in ("bload_strerror", "bload_kernel_launches"):
+        if name not in ("bload_strerror", "bload_kernel_launches", "bload_last_copy_kernel"):
             getattr(L, name).restype = C.c_int
     L.bload_kernel_launches.restype = C.c_int64
+    L.bload_last_copy_kernel.restype = C.c_char_p
     _lib = L
     return L
 
@@ -409,6 +414,14 @@ def bload_kernel_launches() -> int:
     return int(load().bload_kernel_launches())
 
 
+COPY_CALLS = {"pack": 0, "unpack": 1, "carry_prev": 2, "pack_var": 3, "unpack_var": 4}
+
+
+def bload_last_copy_kernel(which: str) -> str:
+    """Name of the copy kernel the last bload_pack / unpack / carry_prev / pack_var / unpack_var call of this thread chose."""
+    return load().bload_last_copy_kernel(COPY_CALLS[which]).decode()
+
+
 STATIC_MAX_N = 65536
 
 
@@ -417,16 +430,13 @@ def bload_plan_static(lengths, t_block: int, seed: int, policy: int = 0, stream=
     """bload_plan without a caller-provided scratch buffer, for callers that cannot allocate device
     memory (for example a loader thread beside a training job whose allocator owns the device).
     The library's built-in scratch array is used instead, which caps n at STATIC_MAX_N; calls that
-    overlap on the GPU race on that array.  Pass a pre-made `plan_buf` to avoid every allocation;
-    without one this wrapper (not the library) allocates the plan buffer with torch."""
+    overlap on the GPU race on that array.  policy: 0 or 1 (best fit decreasing, 2, does not fit the
+    array and raises ERR_UNSUPPORTED).  Pass a pre-made `plan_buf` to avoid every allocation; without
+    one this wrapper (not the library) allocates the plan buffer with torch."""
     import torch
     if not lengths.is_cuda or lengths.dtype != torch.int32 or not lengths.is_contiguous():
         raise TypeError("lengths must be a contiguous CUDA int32 tensor")
-    L = load()
-    fn = L.bload_plan_static
-    fn.argtypes = [C.c_void_p, C.c_int64, C.c_int32, C.c_uint64, C.c_uint32, C.c_void_p, C.c_size_t, C.c_void_p,
-                   C.POINTER(PlanInfo)]
-    fn.restype = C.c_int
+    fn = load().bload_plan_static
     n = lengths.numel()
     sizes = bload_plan_sizes(n, t_block)
     if plan_buf is None:

@@ -2,6 +2,7 @@
 from __future__ import annotations
 
 import glob
+import hashlib
 import os
 import shutil
 import subprocess
@@ -11,18 +12,31 @@ PKG = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libbload.so")
+DEBUG_LIB = os.path.join(PKG, "libbload_debug.so")
+STAMP = LIB + ".sources"  # digest of the sources the library was built from (times of files do not survive a copy)
 
 
 def sources() -> list[str]:
     return sorted(glob.glob(os.path.join(CSRC, "*.cu")))
 
 
-def _stale() -> bool:
-    if not os.path.exists(LIB):
+def source_digest(extra: str = "") -> str:
+    h = hashlib.sha256(extra.encode())
+    deps = sources() + sorted(glob.glob(os.path.join(CSRC, "*.cuh"))) + sorted(glob.glob(os.path.join(ROOT, "include", "*.h")))
+    for d in deps:
+        h.update(os.path.basename(d).encode())
+        with open(d, "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()
+
+
+def stale(lib: str = LIB, extra: str = "") -> bool:
+    """True when `lib` is missing or was not built from the sources as they are now."""
+    try:
+        with open(lib + ".sources") as f:
+            return not os.path.exists(lib) or f.read().strip() != source_digest(extra)
+    except OSError:
         return True
-    t = os.path.getmtime(LIB)
-    deps = sources() + glob.glob(os.path.join(CSRC, "*.cuh")) + glob.glob(os.path.join(ROOT, "include", "*.h"))
-    return any(os.path.getmtime(d) > t for d in deps)
 
 
 def nvcc_path() -> str:
@@ -32,20 +46,28 @@ def nvcc_path() -> str:
     raise RuntimeError("nvcc not found: libbload cannot be built")
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
-    if not force and not _stale():
-        return LIB
-    tmp = LIB + ".tmp%d" % os.getpid()
+def build(force: bool = False, verbose: bool = False, debug: bool = False) -> str:
+    """Compile the library.  debug=True builds libbload_debug.so with -DBLOAD_DEBUG: every global access of the
+    copy, metadata and table kernels is checked against the bounds of its buffer (see bload_debug_status)."""
+    lib = DEBUG_LIB if debug else LIB
+    extra = "debug" if debug else ""
+    if not force and not stale(lib, extra):
+        return lib
+    tmp = lib + ".tmp%d" % os.getpid()
     cmd = [nvcc_path(), "-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17",
            "-shared", "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden",
            "-I", os.path.join(ROOT, "include"), "-I", CSRC]
+    if debug:
+        cmd += ["-DBLOAD_DEBUG=1"]
     if verbose:
         cmd += ["-Xptxas", "-v"]
     cmd += sources() + ["-o", tmp]
     subprocess.check_call(cmd)
-    os.replace(tmp, LIB)
-    return LIB
+    os.replace(tmp, lib)
+    with open(lib + ".sources", "w") as f:
+        f.write(source_digest(extra) + "\n")
+    return lib
 
 
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))
+    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv, debug="--debug" in sys.argv))

@@ -2,6 +2,8 @@
 #include <string.h>
 
 #include <atomic>
+#include <mutex>
+#include <vector>
 
 #include "bload_internal.cuh"
 
@@ -48,11 +50,96 @@ static std::atomic<long long> g_launches{0};
 void count_launches(int k) { g_launches.fetch_add(k, std::memory_order_relaxed); }
 
 namespace {
+constexpr int kMaxDevices = 64, kMaxOptIns = 32;
+std::mutex g_dev_mu;
+std::atomic<int> g_dev_known[kMaxDevices];
+DeviceInfo g_dev_info[kMaxDevices];
+struct OptIn { std::atomic<const void*> kernel; std::atomic<int> bytes; };
+OptIn g_opt_in[kMaxDevices][kMaxOptIns];
+}  // namespace
+
+static thread_local const char* g_last_kernel[kCopyCalls] = {nullptr, nullptr, nullptr, nullptr, nullptr};
+void note_copy_kernel(int call, const char* name) { if (call >= 0 && call < kCopyCalls) g_last_kernel[call] = name; }
+
+DeviceInfo device_info()
+{
+    DeviceInfo fallback{148, 228 * 1024};
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) { (void)cudaGetLastError(); return fallback; }
+    if (g_dev_known[dev].load(std::memory_order_acquire)) return g_dev_info[dev];
+    std::lock_guard<std::mutex> lock(g_dev_mu);
+    if (!g_dev_known[dev].load(std::memory_order_relaxed)) {
+        DeviceInfo d = fallback;
+        int v = 0;
+        if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && v > 0) d.sm_count = v;
+        if (cudaDeviceGetAttribute(&v, cudaDevAttrMaxSharedMemoryPerMultiprocessor, dev) == cudaSuccess && v > 0) d.smem_per_sm = v;
+        (void)cudaGetLastError();
+        g_dev_info[dev] = d;
+        g_dev_known[dev].store(1, std::memory_order_release);
+    }
+    return g_dev_info[dev];
+}
+
+cudaError_t opt_in_shared_memory(const void* kernel, int bytes)
+{
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices)
+        return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    OptIn* row = g_opt_in[dev];
+    for (int i = 0; i < kMaxOptIns; ++i) {
+        const void* k = row[i].kernel.load(std::memory_order_acquire);
+        if (k == kernel && row[i].bytes.load(std::memory_order_relaxed) >= bytes) return cudaSuccess;
+        if (!k) break;
+    }
+    std::lock_guard<std::mutex> lock(g_dev_mu);
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    if (e != cudaSuccess) return e;
+    for (int i = 0; i < kMaxOptIns; ++i) {
+        const void* k = row[i].kernel.load(std::memory_order_relaxed);
+        if (k == kernel || !k) {
+            row[i].bytes.store(bytes, std::memory_order_relaxed);
+            row[i].kernel.store(kernel, std::memory_order_release);
+            break;
+        }
+    }
+    return cudaSuccess;  // a full table only means the attribute is set again next time
+}
+
+namespace {
 thread_local bool g_timing = false;
 thread_local bool g_have_times = false;
 thread_local float g_stage_ms[4] = {0, 0, 0, 0};
 thread_local bool g_have_epoch_times = false;
 thread_local float g_epoch_ms[5] = {0, 0, 0, 0, 0};
+
+// Events of bload_epoch, kept per host thread and device between calls: creating and destroying up to a hundred
+// events per call was a visible share of a short epoch.  Every call synchronises both of its streams before it
+// returns, so all events of the pool are complete then and can be recorded again by the next call.  The pool is
+// never destroyed (at thread exit the CUDA context may already be gone).
+struct EventPool {
+    int dev = -1;
+    std::vector<cudaEvent_t> plain, timed;
+    size_t used_plain = 0, used_timed = 0;
+    cudaEvent_t take(bool with_timing)
+    {
+        std::vector<cudaEvent_t>& v = with_timing ? timed : plain;
+        size_t& used = with_timing ? used_timed : used_plain;
+        if (used == v.size()) {
+            cudaEvent_t e = nullptr;
+            if (cudaEventCreateWithFlags(&e, with_timing ? cudaEventDefault : cudaEventDisableTiming) != cudaSuccess) return nullptr;
+            v.push_back(e);
+        }
+        return v[used++];
+    }
+    void begin_call()
+    {
+        int d = -1;
+        if (cudaGetDevice(&d) != cudaSuccess) d = -1;
+        if (d != dev) { plain.clear(); timed.clear(); dev = d; }  // events belong to the device they were made on
+        used_plain = used_timed = 0;
+    }
+};
+thread_local EventPool* g_events = nullptr;
 
 inline bool aligned(const void* p, uintptr_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
 
@@ -84,6 +171,12 @@ extern "C" {
 int bload_version(void) { return 1; }
 
 int64_t bload_kernel_launches(void) { return (int64_t)g_launches.load(std::memory_order_relaxed); }
+
+const char* bload_last_copy_kernel(int which)
+{
+    if (which < 0 || which >= kCopyCalls || !g_last_kernel[which]) return "";
+    return g_last_kernel[which];
+}
 
 const char* bload_strerror(int code)
 {
@@ -295,16 +388,9 @@ int bload_epoch(const int32_t* d_lengths, int64_t n, int32_t t_block, uint64_t s
     g_have_epoch_times = false;
 
     // events: one per chunk to hand its blocks to the side stream, one to join; with timing, 2 + 5 more per chunk
-    constexpr int kPer = 8;
-    cudaEvent_t evs[kMaxEpochChunks * kPer + 1];
-    int n_ev = 0;
-    auto new_event = [&](bool timed) -> cudaEvent_t {
-        cudaEvent_t e = nullptr;
-        if (cudaEventCreateWithFlags(&e, timed ? cudaEventDefault : cudaEventDisableTiming) != cudaSuccess) return nullptr;
-        evs[n_ev++] = e;
-        return e;
-    };
-    auto destroy_events = [&]() { for (int i = 0; i < n_ev; ++i) cudaEventDestroy(evs[i]); };
+    if (!g_events) g_events = new EventPool;
+    g_events->begin_call();
+    auto new_event = [&](bool timed) -> cudaEvent_t { return g_events->take(timed); };
     struct ChunkEv { cudaEvent_t f0, f1, ready, t0, t1, t2, t3, t4; } ce_[kMaxEpochChunks];
 
     cudaError_t ce = cudaMemsetAsync(ev.resume, 0, sizeof(FillResume), st);
@@ -363,7 +449,6 @@ int bload_epoch(const int32_t* d_lengths, int64_t n, int32_t t_block, uint64_t s
     if (ce != cudaSuccess) {
         (void)cudaGetLastError();
         cudaStreamSynchronize(side); cudaStreamSynchronize(st);  // nothing may still use the events
-        destroy_events();
         return fail(BLOAD_ERR_CUDA);
     }
     if (timing) {
@@ -379,7 +464,6 @@ int bload_epoch(const int32_t* d_lengths, int64_t n, int32_t t_block, uint64_t s
         }
         g_have_epoch_times = true;
     }
-    destroy_events();
     info->status = h.status;
     info->n_blocks = h.n_blocks;
     info->sum_t = h.sum_t;

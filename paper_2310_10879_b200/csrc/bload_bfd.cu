@@ -243,7 +243,7 @@ cudaError_t launch_bfd(const PlanView& pv, const WorkView& wv, const BfdView& bv
 {
     const unsigned gn = (unsigned)((n + 255) / 256);
     const size_t smem = sizeof(int32_t) * (1024 + 64 + (size_t)t_block);
-    cudaError_t e = cudaFuncSetAttribute(kb_chain, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaError_t e = opt_in_shared_memory(kb_chain, (int)smem);
     if (e != cudaSuccess) return e;
     kb_chain<<<1, 256, smem, st>>>(pv.hdr, sorted_key, bv.rec, (int32_t)n, t_block);
     int room_bits = 0;

@@ -218,6 +218,7 @@ cudaError_t launch_carry_prev(const PlanView& pv, int32_t t_block, int64_t frame
     cudaError_t staged_err = cudaSuccess;
     if (staged_carry_prev(pv, t_block, frame_bytes, block_begin, block_count, dense, prev, fill_byte, st, n, sum_t, &staged_err))
         return staged_err;
+    note_copy_kernel(kCallCarryPrev, "k11_carry_prev");
     k11_carry_prev<<<grid_for_items(block_count * spb), 256, 0, st>>>(pv, t_block, frame_bytes, block_begin, block_count,
                                                                      dense, prev, sub, spb, fill_byte);
     return cudaPeekAtLastError();

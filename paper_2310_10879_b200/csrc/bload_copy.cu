@@ -591,12 +591,13 @@ bool staged_carry_prev(const PlanView& pv, int32_t t_block, int64_t frame_bytes,
         return false;
     using Cfg = StageCfg<false>;
     const size_t smem = (size_t)Cfg::kWarps * Cfg::kStages * Cfg::kBytes + 16;
-    const int per_sm = (int)((227 * 1024) / (smem + 1024));
-    *err = cudaFuncSetAttribute(k10_pack_contig<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    const DeviceInfo di = device_info();
+        const int per_sm = (int)(di.smem_per_sm / (smem + 1024));
+    *err = opt_in_shared_memory(k10_pack_contig<true>, (int)smem);
     if (*err != cudaSuccess) return true;
     const int64_t spb = (block_bytes + Cfg::kBytes - 1) / Cfg::kBytes;
     const int64_t tiles = block_count * spb;
-    const int64_t max_warps = (int64_t)148 * per_sm * Cfg::kWarps;
+    const int64_t max_warps = (int64_t)di.sm_count * per_sm * Cfg::kWarps;
     int64_t tpw = (tiles + max_warps - 1) / max_warps;
     if (tpw > kPackChunkTiles) tpw = kPackChunkTiles;
     int64_t warps = (tiles + tpw - 1) / tpw;
@@ -604,6 +605,7 @@ bool staged_carry_prev(const PlanView& pv, int32_t t_block, int64_t frame_bytes,
     const unsigned grid = (unsigned)((warps + Cfg::kWarps - 1) / Cfg::kWarps);
     k10_pack_contig<true><<<grid, Cfg::kWarps * 32, smem, st>>>(pv, (int32_t)n, t_block, frame_bytes, block_begin, dense, prev,
                                                                tiles, tpw, (int32_t)spb, fill_byte);
+    note_copy_kernel(kCallCarryPrev, "k10_pack_contig<carry>");
     *err = cudaPeekAtLastError();
     return true;
 }
@@ -620,12 +622,13 @@ cudaError_t launch_copy(bool unpack, const PlanView& pv, int32_t t_block, int64_
     if (!unpack && short_runs && block_bytes % 16 == 0) {
         using Cfg = StageCfg<false>;
         const size_t smem = (size_t)Cfg::kWarps * Cfg::kStages * Cfg::kBytes + 16;
-        const int per_sm = (int)((227 * 1024) / (smem + 1024));
-        cudaError_t e = cudaFuncSetAttribute(k10_pack_contig<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        const DeviceInfo di = device_info();
+        const int per_sm = (int)(di.smem_per_sm / (smem + 1024));
+        cudaError_t e = opt_in_shared_memory(k10_pack_contig<false>, (int)smem);
         if (e != cudaSuccess) return e;
         const int64_t spb = (block_bytes + Cfg::kBytes - 1) / Cfg::kBytes;
         const int64_t tiles = block_count * spb;
-        const int64_t max_warps = (int64_t)148 * per_sm * Cfg::kWarps;
+        const int64_t max_warps = (int64_t)di.sm_count * per_sm * Cfg::kWarps;
         int64_t tpw = (tiles + max_warps - 1) / max_warps;
         if (tpw > kPackChunkTiles) tpw = kPackChunkTiles;  // chunks are grid-strided beyond this size
         int64_t warps = (tiles + tpw - 1) / tpw;
@@ -633,22 +636,25 @@ cudaError_t launch_copy(bool unpack, const PlanView& pv, int32_t t_block, int64_
         const unsigned grid = (unsigned)((warps + Cfg::kWarps - 1) / Cfg::kWarps);
         k10_pack_contig<false><<<grid, Cfg::kWarps * 32, smem, st>>>(pv, (int32_t)n, t_block, frame_bytes, block_begin, ragged_in,
                                                              dense, tiles, tpw, (int32_t)spb, pad_byte);
+        note_copy_kernel(kCallPack, "k10_pack_contig");
         return cudaPeekAtLastError();
     }
     // whole-plan unpack of small word-sized frames: tile the (contiguous, fully written) ragged side
     if (unpack && short_runs && block_begin == 0 && block_count >= n_blocks && ragged_bytes > 0) {
         using Cfg = StageCfg<false>;
         const size_t smem = (size_t)Cfg::kWarps * Cfg::kStages * Cfg::kBytes + 16;
-        const int per_sm = (int)((227 * 1024) / (smem + 1024));
-        cudaError_t e = cudaFuncSetAttribute(k9_unpack_ragged, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        const DeviceInfo di = device_info();
+        const int per_sm = (int)(di.smem_per_sm / (smem + 1024));
+        cudaError_t e = opt_in_shared_memory(k9_unpack_ragged, (int)smem);
         if (e != cudaSuccess) return e;
         const int64_t tiles = (ragged_bytes + Cfg::kBytes - 1) / Cfg::kBytes;
-        const int64_t max_warps = (int64_t)148 * per_sm * Cfg::kWarps;
+        const int64_t max_warps = (int64_t)di.sm_count * per_sm * Cfg::kWarps;
         const int64_t tpw = (tiles + max_warps - 1) / max_warps;           // contiguous sub-tiles per warp
         const int64_t warps = (tiles + tpw - 1) / tpw;
         const unsigned grid = (unsigned)((warps + Cfg::kWarps - 1) / Cfg::kWarps);
         k9_unpack_ragged<<<grid, Cfg::kWarps * 32, smem, st>>>(pv, (int32_t)n, t_block, frame_bytes, ragged_bytes / frame_bytes,
                                                               dense, ragged_out, tiles, tpw);
+        note_copy_kernel(kCallUnpack, "k9_unpack_ragged");
         return cudaPeekAtLastError();
     }
     // block sub-ranges of small word-sized frames, unpack direction: staged kernel over the dense side
@@ -657,8 +663,9 @@ cudaError_t launch_copy(bool unpack, const PlanView& pv, int32_t t_block, int64_
         const int64_t spb = (block_bytes + Cfg::kBytes - 1) / Cfg::kBytes;
         const int64_t gpb = (spb + Cfg::kGroup - 1) / Cfg::kGroup;  // groups of sub-tiles per block
         const size_t smem = (size_t)Cfg::kWarps * Cfg::kStages * Cfg::kBytes + 16;  // 16 spare bytes: see warp_scatter
-        const int per_sm = (int)((227 * 1024) / (smem + 1024));
-        cudaError_t e = cudaFuncSetAttribute(k8_unpack_staged, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        const DeviceInfo di = device_info();
+        const int per_sm = (int)(di.smem_per_sm / (smem + 1024));
+        cudaError_t e = opt_in_shared_memory(k8_unpack_staged, (int)smem);
         if (e != cudaSuccess) return e;
         // 32-bit group arithmetic on the device: at most 2^31 - 1 groups per launch
         const int64_t max_blocks = 0x7fffffffLL / gpb;
@@ -666,12 +673,14 @@ cudaError_t launch_copy(bool unpack, const PlanView& pv, int32_t t_block, int64_
             const int64_t cnt = block_count - done < max_blocks ? block_count - done : max_blocks;
             const int64_t groups = cnt * gpb;
             const int64_t want = (groups + Cfg::kWarps - 1) / Cfg::kWarps;
-            const unsigned grid = (unsigned)(want < 148 * per_sm ? want : 148 * per_sm);
+            const unsigned grid = (unsigned)(want < (int64_t)di.sm_count * per_sm ? want : (int64_t)di.sm_count * per_sm);
             k8_unpack_staged<<<grid, Cfg::kWarps * 32, smem, st>>>(pv, t_block, frame_bytes, block_begin + done, (uint32_t)groups,
                                                                  dense + done * block_bytes, ragged_out, (uint32_t)gpb, pad_byte);
         }
+        note_copy_kernel(kCallUnpack, "k8_unpack_staged");
         return cudaPeekAtLastError();
     }
+    note_copy_kernel(unpack ? kCallUnpack : kCallPack, unpack ? "k7_copy<unpack>" : "k7_copy<pack>");
     const int64_t sub = 16384;
     const int64_t spb = (block_bytes + sub - 1) / sub;
     const int64_t items = block_count * spb;
@@ -700,7 +709,7 @@ cudaError_t launch_copy_range(bool unpack, const PlanView& pv, int32_t t_block, 
     const int64_t spb = (block_bytes + sub - 1) / sub;
     // many short-lived CTAs rather than a few long ones: the next chunk of the fill rule (one CTA on the other stream)
     // starts as soon as any CTA of this launch retires; a chunk holds some thousand sub-tiles, about one per warp
-    const unsigned grid = 148 * 3 * 16;  // (2 to 32 rounds of resident CTAs measured alike)
+    const unsigned grid = (unsigned)device_info().sm_count * 3 * 16;  // (2 to 32 rounds of resident CTAs measured alike)
     count_launches(1);
     if (unpack)
         k7_copy<true><<<grid, 256, kBesideChainSmemBytes, st>>>(pv, t_block, frame_bytes, 0, 0, src, dst, src_total_bytes, sub, spb,

@@ -117,6 +117,20 @@ cudaError_t launch_bfd(const PlanView& pv, const WorkView& wv, const BfdView& bv
 // every kernel launch of the library goes through this counter (see bload_kernel_launches)
 void count_launches(int k);
 
+// which copy kernel a call chose (see bload_last_copy_kernel): 0 pack, 1 unpack, 2 carry_prev, 3 pack_var, 4 unpack_var
+enum CopyCall { kCallPack = 0, kCallUnpack = 1, kCallCarryPrev = 2, kCallPackVar = 3, kCallUnpackVar = 4, kCopyCalls = 5 };
+void note_copy_kernel(int call, const char* name);
+
+// Multiprocessors and shared memory per multiprocessor of the current device, asked for once per device (grids and
+// occupancy are sized from them; a failed query answers with the B200's 148 and 228 KB).
+struct DeviceInfo { int sm_count; int smem_per_sm; };
+DeviceInfo device_info();
+// cudaFuncAttributeMaxDynamicSharedMemorySize for `kernel` on the current device, set on the first call per device and
+// kernel and remembered: the attribute call costs a few microseconds, which a per-batch launch would pay every time.
+cudaError_t opt_in_shared_memory(const void* kernel, int bytes);
+template <typename K>
+inline cudaError_t opt_in_shared_memory(K* kernel, int bytes) { return opt_in_shared_memory(reinterpret_cast<const void*>(kernel), bytes); }
+
 // launchers (each returns a cudaError_t from cudaPeekAtLastError)
 cudaError_t launch_plan(const int32_t* d_lengths, int64_t n, int32_t t_block, uint64_t seed, uint32_t policy,
                         const PlanView& pv, const WorkView& wv, cudaStream_t st, cudaEvent_t* ev /*5 or null*/,

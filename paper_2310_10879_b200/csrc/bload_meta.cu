@@ -104,7 +104,7 @@ cudaError_t launch_metadata(const PlanView& pv, int32_t t_block, int64_t block_b
     auto al = [](const void* p, uintptr_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; };
     const unsigned chunks = (unsigned)((t_block + kMetaChunk - 1) / kMetaChunk);
     // enough CTAs in flight to cover the machine several times over; beyond that a CTA loops over blocks
-    int64_t rows = (148 * 64 + chunks - 1) / chunks;
+    int64_t rows = ((int64_t)device_info().sm_count * 64 + chunks - 1) / chunks;
     if (rows > block_count && !d_range) rows = block_count;
     if (d_range && rows > 256) rows = 256;  // a chunk of a plan in progress holds a few blocks
     if (rows > 65535) rows = 65535;

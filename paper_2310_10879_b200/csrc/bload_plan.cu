@@ -748,7 +748,7 @@ cudaError_t launch_fill_chunk(const PlanView& pv, const WorkView& wv, const Epoc
 {
     size_t smem = fill_smem_bytes(t_block);
     if (smem < (size_t)kChainSmemBytes) smem = kChainSmemBytes;  // keeps other CTAs off this SM (see kChainSmemBytes)
-    cudaError_t e = cudaFuncSetAttribute(k4_fill<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaError_t e = opt_in_shared_memory(k4_fill<true>, (int)smem);
     if (e != cudaSuccess) return e;
     k4_fill<true><<<1, 256, smem, st>>>(pv, wv.bucket_end, wv.draw_u, wv.draw_rec, n, t_block, ev.resume, ev.fill_tables,
                                          k_target, filler_end);
@@ -787,11 +787,11 @@ cudaError_t launch_plan(const int32_t* d_lengths, int64_t n, int32_t t_block, ui
     }
     const size_t smem = fill_smem_bytes(t_block);
     if (policy == BLOAD_POLICY_UNIFORM_LENGTHS) {
-        e = cudaFuncSetAttribute(k4_fill_lengths, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        e = opt_in_shared_memory(k4_fill_lengths, (int)smem);
         if (e != cudaSuccess) return e;
         k4_fill_lengths<<<1, 256, smem, st>>>(pv, wv.bucket_end, wv.draw_u, wv.draw_rec, n, t_block);
     } else {
-        e = cudaFuncSetAttribute(k4_fill<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        e = opt_in_shared_memory(k4_fill<false>, (int)smem);
         if (e != cudaSuccess) return e;
         k4_fill<false><<<1, 256, smem, st>>>(pv, wv.bucket_end, wv.draw_u, wv.draw_rec, n, t_block, nullptr, nullptr, 0, 0);
     }

@@ -53,7 +53,9 @@ extern "C" int bload_plan_static(const int32_t* d_lengths, int64_t n, int32_t t_
     auto fail = [&](int rc) { info->status = rc; return rc; };
     if (!d_lengths || !d_plan) return fail(BLOAD_ERR_NULL);
     if (n < 1 || t_block < 1) return fail(BLOAD_ERR_ARG);
-    if (t_block > BLOAD_MAX_T_BLOCK || policy != BLOAD_POLICY_UNIFORM_SEQUENCES) return fail(BLOAD_ERR_UNSUPPORTED);
+    // both readings of the paper's rule run in the common scratch layout; best fit decreasing needs about 40 more
+    // bytes per sequence behind it, which this array was not sized for
+    if (t_block > BLOAD_MAX_T_BLOCK || policy > BLOAD_POLICY_UNIFORM_LENGTHS) return fail(BLOAD_ERR_UNSUPPORTED);
     // the built-in scratch is a fixed size: larger problems must use bload_plan with a caller buffer
     if (n > BLOAD_STATIC_MAX_N || work_layout(n, t_block, nullptr, nullptr) > (size_t)BLOAD_STATIC_SCRATCH_BYTES)
         return fail(BLOAD_ERR_WORKSPACE);

@@ -198,6 +198,7 @@ cudaError_t launch_copy_var(bool unpack, const PlanView& pv, int32_t t_block, in
     const int64_t want = (block_count * spb + 7) / 8;
     const unsigned grid = (unsigned)(want < 0x7fffffffLL ? want : 0x7fffffffLL);
     count_launches(1);
+    note_copy_kernel(unpack ? kCallUnpackVar : kCallPackVar, unpack ? "k16_copy_var<unpack>" : "k16_copy_var<pack>");
     if (unpack)
         k16_copy_var<true><<<grid, 256, 0, st>>>(pv, t_block, rows_max, row_stride, block_begin, block_count, seq_rows,
                                                   frame_bytes, byte_offsets, src, dst, sub, spb, pad_byte);
