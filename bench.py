@@ -362,12 +362,14 @@ def _time_per_batch(c):
                              reset=b_meta[2], valid=b_meta[3])
         batch_loop()
         torch.cuda.synchronize()
+        l0 = B.bload_kernel_launches()
         a, b_ = ev(), ev()
         a.record(); batch_loop(); b_.record()
         torch.cuda.synchronize()
         ms = a.elapsed_time(b_)
         per_batch = {"batch_blocks": bb, "batches_timed": reps, "us_per_call": ms * 1e3 / reps,
-                     "GB/s": (2 * bb * tb * fb) * reps / ms / 1e6, "launches_per_call": 2}
+                     "GB/s": (2 * bb * tb * fb) * reps / ms / 1e6,
+                     "launches_per_call": (B.bload_kernel_launches() - l0) / reps, "kernel": B.bload_last_copy_kernel("pack")}
         # the same loop captured once in a CUDA graph and replayed (the calls are asynchronous and allocate nothing)
         try:
             side = torch.cuda.Stream()

@@ -39,6 +39,11 @@
  *                      per-sequence numpy.cumsum after unpacking
  *   valid_sum          packing per-frame integers and summing the frames equals the sum
  *                      over the ragged array (exact in double)
+ *   chunks             closed forms with numpy (sum of ceil / floor of T_i / c, T_i mod c), every kept frame
+ *                      in exactly one chunk, chunks of one sequence in order; a chunk length that
+ *                      covers every sequence reduces to the paper's naive padding (Table I,
+ *                      "0 padding" = 534831); chunk pack/unpack/metadata against the ordinary
+ *                      functions run on the derived one-chunk-per-block plan, and against numpy
  *   Parity unpinned: the paper's "block_pad" padding count of Table I (block
  *   length of that run is not stated and the rule is random) and its
  *   time-per-epoch figures.
@@ -169,6 +174,17 @@ static uint64_t fmix64(uint64_t x)
     return x;
 }
 
+/* Order-independent 64-bit digest of a segment list (block, start slot, sequence per segment). */
+uint64_t oracle_digest(const int32_t *seg_block, const int32_t *seg_start, const int32_t *seg_seq, int64_t n)
+{
+    uint64_t sum = 0;
+    for (int64_t q = 0; q < n; ++q) {
+        uint64_t where = ((uint64_t)(uint32_t)seg_block[q] << 32) | (uint64_t)(uint32_t)seg_start[q];
+        sum += fmix64(where * 0x9E3779B97F4A7C15ULL + (uint64_t)(uint32_t)seg_seq[q]);
+    }
+    return sum;
+}
+
 int oracle_plan(oracle_plan_t *p)
 {
     const int64_t n = p->n;
@@ -297,13 +313,7 @@ int oracle_plan(oracle_plan_t *p)
     if (p->policy != 2) p->block_seg_begin[b] = (int32_t)k;
     p->n_blocks = b;
 
-    /* Order-independent 64-bit digest of the segment list. */
-    uint64_t sum = 0;
-    for (int64_t q = 0; q < n; ++q) {
-        uint64_t where = ((uint64_t)(uint32_t)p->seg_block[q] << 32) | (uint64_t)(uint32_t)p->seg_start[q];
-        sum += fmix64(where * 0x9E3779B97F4A7C15ULL + (uint64_t)(uint32_t)p->seg_seq[q]);
-    }
-    p->checksum = sum;
+    p->checksum = oracle_digest(p->seg_block, p->seg_start, p->seg_seq, n);
 
     free(dict); free(first); free(unused);
     return ORACLE_OK;
@@ -639,5 +649,118 @@ int oracle_stats(oracle_stats_t *s)
     s->frac_naive_tblock = (double)s->pad_naive_tblock / (double)(s->n * s->t_block);
     s->reduction_vs_tmax = s->pad_packed > 0 ? (double)s->pad_naive_tmax / (double)s->pad_packed : 0.0;
     s->mean_segs_per_block = s->n_blocks ? (double)s->n / (double)s->n_blocks : 0.0;
+    return ORACLE_OK;
+}
+
+/* ------------------------------------------------------------------------ */
+/* The chunking strategy the paper compares with (section "Problem Statement  */
+/* and Current Limitations": each sample is broken into chunks of T_block      */
+/* frames and each chunk is treated as an individual sample; figure "Sampling  */
+/* solution"; Table I, column "sampling": no padding, frames deleted).         */
+/* Sequence i is cut at frames 0, c, 2c, ...  With tail == 0 the last, shorter */
+/* chunk is kept (and padded when it becomes a block); with tail == 1 only     */
+/* full chunks are kept and the remaining T_i mod c frames are deleted, which  */
+/* is the reading that gives the table's zero padding.  Chunks are listed in   */
+/* order of (sequence, position); chunk j becomes block j.                     */
+/* ------------------------------------------------------------------------ */
+typedef struct {
+    const int32_t *lengths;
+    int64_t n;
+    int32_t t_chunk;
+    uint32_t tail;
+    int64_t capacity;      /* room in the three arrays below (0 with NULL arrays: count only) */
+    int32_t *chunk_seq;    /* sequence the chunk was cut from */
+    int32_t *chunk_first;  /* its first frame inside that sequence */
+    int32_t *chunk_len;    /* its frames, 1..t_chunk */
+    int64_t n_chunks, frames_kept, frames_deleted, pad_frames, sum_t, t_max, first_bad;
+} oracle_chunks_t;
+
+int oracle_chunks(oracle_chunks_t *p)
+{
+    p->n_chunks = p->frames_kept = p->frames_deleted = p->pad_frames = p->sum_t = p->t_max = 0;
+    p->first_bad = -1;
+    if (p->n < 1 || p->t_chunk < 1 || p->tail > 1) return ORACLE_ERR_ARG;
+    for (int64_t i = 0; i < p->n; ++i)
+        if (p->lengths[i] < 1) { p->first_bad = i; return ORACLE_ERR_LENGTH; }
+    for (int64_t i = 0; i < p->n; ++i) {
+        int32_t t = p->lengths[i];
+        p->sum_t += t;
+        if (t > p->t_max) p->t_max = t;
+        for (int32_t first = 0; first < t; first += p->t_chunk) {
+            int32_t len = t - first < p->t_chunk ? t - first : p->t_chunk;
+            if (len < p->t_chunk && p->tail == 1) { p->frames_deleted += len; continue; }
+            if (p->chunk_seq) {
+                if (p->n_chunks >= p->capacity) return ORACLE_ERR_ARG;
+                p->chunk_seq[p->n_chunks] = (int32_t)i;
+                p->chunk_first[p->n_chunks] = first;
+                p->chunk_len[p->n_chunks] = len;
+            }
+            p->n_chunks += 1;
+            p->frames_kept += len;
+            p->pad_frames += p->t_chunk - len;
+        }
+    }
+    return ORACLE_OK;
+}
+
+typedef struct {
+    int64_t n_chunks;
+    int32_t t_chunk;
+    const int64_t *offsets;   /* of the ORIGINAL sequences in the store */
+    const int32_t *chunk_seq, *chunk_first, *chunk_len;
+} oracle_chunk_tables_t;
+
+/* Every chunk is a sample of its own: its id is the chunk number, positions count from the chunk's first frame. */
+int oracle_chunk_metadata(const oracle_chunk_tables_t *t, int64_t block_begin, int64_t block_count,
+                          int32_t *seq_id, int32_t *pos, uint8_t *reset, uint8_t *valid)
+{
+    if (block_begin < 0 || block_count < 0) return ORACLE_ERR_ARG;
+    for (int64_t q = 0; q < block_count; ++q) {
+        int64_t j = block_begin + q;
+        for (int32_t s = 0; s < t->t_chunk; ++s) {
+            int64_t o = q * t->t_chunk + s;
+            int is_frame = j < t->n_chunks && s < t->chunk_len[j];
+            seq_id[o] = is_frame ? (int32_t)j : -1;
+            pos[o] = is_frame ? s : -1;
+            reset[o] = (uint8_t)(is_frame && s == 0);
+            valid[o] = (uint8_t)is_frame;
+        }
+    }
+    return ORACLE_OK;
+}
+
+int oracle_chunk_pack(const oracle_chunk_tables_t *t, const uint8_t *store, int64_t frame_bytes, int64_t block_begin,
+                      int64_t block_count, uint8_t *dense, uint8_t pad_byte)
+{
+    if (block_begin < 0 || block_count < 0 || frame_bytes < 1) return ORACLE_ERR_ARG;
+    for (int64_t q = 0; q < block_count; ++q) {
+        int64_t j = block_begin + q;
+        for (int32_t s = 0; s < t->t_chunk; ++s) {
+            uint8_t *dst = dense + ((size_t)q * (size_t)t->t_chunk + (size_t)s) * (size_t)frame_bytes;
+            if (j < t->n_chunks && s < t->chunk_len[j]) {
+                int64_t frame = t->offsets[t->chunk_seq[j]] + t->chunk_first[j] + s;
+                memcpy(dst, store + (size_t)frame * (size_t)frame_bytes, (size_t)frame_bytes);
+            } else {
+                memset(dst, pad_byte, (size_t)frame_bytes);
+            }
+        }
+    }
+    return ORACLE_OK;
+}
+
+/* Frames that the strategy deleted have no slot anywhere and stay untouched in ragged_out. */
+int oracle_chunk_unpack(const oracle_chunk_tables_t *t, const uint8_t *dense_out, int64_t frame_bytes, int64_t block_begin,
+                        int64_t block_count, uint8_t *ragged_out)
+{
+    if (block_begin < 0 || block_count < 0 || frame_bytes < 1) return ORACLE_ERR_ARG;
+    for (int64_t q = 0; q < block_count; ++q) {
+        int64_t j = block_begin + q;
+        if (j >= t->n_chunks) continue;
+        for (int32_t s = 0; s < t->chunk_len[j]; ++s) {
+            int64_t frame = t->offsets[t->chunk_seq[j]] + t->chunk_first[j] + s;
+            memcpy(ragged_out + (size_t)frame * (size_t)frame_bytes,
+                   dense_out + ((size_t)q * (size_t)t->t_chunk + (size_t)s) * (size_t)frame_bytes, (size_t)frame_bytes);
+        }
+    }
     return ORACLE_OK;
 }

@@ -55,6 +55,18 @@ class _StatsStruct(C.Structure):
                                           "reduction_vs_tmax", "mean_segs_per_block")]
 
 
+class _ChunksStruct(C.Structure):
+    _fields_ = [("lengths", C.c_void_p), ("n", C.c_int64), ("t_chunk", C.c_int32), ("tail", C.c_uint32),
+                ("capacity", C.c_int64), ("chunk_seq", C.c_void_p), ("chunk_first", C.c_void_p), ("chunk_len", C.c_void_p),
+                ("n_chunks", C.c_int64), ("frames_kept", C.c_int64), ("frames_deleted", C.c_int64),
+                ("pad_frames", C.c_int64), ("sum_t", C.c_int64), ("t_max", C.c_int64), ("first_bad", C.c_int64)]
+
+
+class _ChunkTablesStruct(C.Structure):
+    _fields_ = [("n_chunks", C.c_int64), ("t_chunk", C.c_int32), ("offsets", C.c_void_p), ("chunk_seq", C.c_void_p),
+                ("chunk_first", C.c_void_p), ("chunk_len", C.c_void_p)]
+
+
 def lib():
     global _lib
     if _lib is None:
@@ -107,6 +119,18 @@ def lib():
         L.oracle_valid_sum.argtypes = [C.POINTER(_TablesStruct), C.c_int64, C.c_int64, C.c_void_p,
                                        C.POINTER(C.c_double), C.POINTER(C.c_int64)]
         L.oracle_valid_sum.restype = C.c_int
+        L.oracle_digest.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64]
+        L.oracle_digest.restype = C.c_uint64
+        L.oracle_chunks.argtypes = [C.POINTER(_ChunksStruct)]
+        L.oracle_chunks.restype = C.c_int
+        L.oracle_chunk_metadata.argtypes = [C.POINTER(_ChunkTablesStruct), C.c_int64, C.c_int64] + [C.c_void_p] * 4
+        L.oracle_chunk_metadata.restype = C.c_int
+        L.oracle_chunk_pack.argtypes = [C.POINTER(_ChunkTablesStruct), C.c_void_p, C.c_int64, C.c_int64, C.c_int64,
+                                        C.c_void_p, C.c_uint8]
+        L.oracle_chunk_pack.restype = C.c_int
+        L.oracle_chunk_unpack.argtypes = [C.POINTER(_ChunkTablesStruct), C.c_void_p, C.c_int64, C.c_int64, C.c_int64,
+                                          C.c_void_p]
+        L.oracle_chunk_unpack.restype = C.c_int
         L.oracle_stats.argtypes = [C.POINTER(_StatsStruct)]
         L.oracle_stats.restype = C.c_int
         _lib = L
@@ -362,3 +386,98 @@ def stats(n: int, sum_t: int, t_max: int, t_block: int, n_blocks: int) -> dict:
     rc = lib().oracle_stats(C.byref(s))
     assert rc == 0, rc
     return {k: getattr(s, k) for k, _ in _StatsStruct._fields_}
+
+
+# ---- the chunking strategy (a comparison system of the paper): every chunk of t_chunk frames is a sample and a block ----
+
+KEEP_TAIL, DROP_TAIL = 0, 1
+
+
+@dataclass
+class OracleChunks:
+    status: int
+    n: int                 # sequences the chunks were cut from
+    t_chunk: int
+    tail: int
+    n_chunks: int
+    frames_kept: int
+    frames_deleted: int
+    pad_frames: int
+    sum_t: int
+    t_max: int
+    first_bad: int
+    lengths: np.ndarray
+    offsets: np.ndarray    # int64[n+1] of the original sequences
+    chunk_seq: np.ndarray
+    chunk_first: np.ndarray
+    chunk_len: np.ndarray
+
+    def _tables(self) -> _ChunkTablesStruct:
+        return _ChunkTablesStruct(self.n_chunks, self.t_chunk, _p(self.offsets), _p(self.chunk_seq), _p(self.chunk_first),
+                                  _p(self.chunk_len))
+
+    def as_plan(self) -> OraclePlan:
+        """The same chunks written as plan tables: chunk j is "sequence" j and fills block j from slot 0; its entry of
+        `offsets` is its first frame in the original store ([n_chunks] = all frames of that store)."""
+        m = self.n_chunks
+        ar = np.arange(m, dtype=np.int32)
+        zeros = np.zeros(m, np.int32)
+        off = np.empty(m + 1, np.int64)
+        off[:m] = self.offsets[self.chunk_seq.astype(np.int64)] + self.chunk_first
+        off[m] = self.sum_t
+        digest = int(lib().oracle_digest(_p(ar), _p(zeros), _p(ar), m))
+        return OraclePlan(status=self.status, n=m, t_block=self.t_chunk, seed=0, n_blocks=m, sum_t=self.sum_t,
+                          t_max=self.t_max, first_bad=self.first_bad, checksum=digest, max_segs_per_block=1 if m else 0,
+                          lengths=self.chunk_len.copy(), offsets=off, seg_seq=ar.copy(), seg_block=ar.copy(),
+                          seg_start=zeros.copy(), block_seg_begin=np.arange(m + 1, dtype=np.int32),
+                          block_fill=self.chunk_len.copy(), seq_block=ar.copy(), seq_start=zeros.copy())
+
+
+def chunks(lengths: np.ndarray, t_chunk: int, tail: int = KEEP_TAIL) -> OracleChunks:
+    lengths = np.ascontiguousarray(lengths, dtype=np.int32)
+    n = int(lengths.size)
+    s = _ChunksStruct(lengths=_p(lengths), n=n, t_chunk=t_chunk, tail=tail, capacity=0)
+    rc = lib().oracle_chunks(C.byref(s))                      # first pass: count
+    m = int(s.n_chunks) if rc == 0 else 0
+    seq, first, ln = (np.zeros(max(m, 1), np.int32) for _ in range(3))
+    if rc == 0:
+        s = _ChunksStruct(lengths=_p(lengths), n=n, t_chunk=t_chunk, tail=tail, capacity=m, chunk_seq=_p(seq),
+                          chunk_first=_p(first), chunk_len=_p(ln))
+        rc = lib().oracle_chunks(C.byref(s))
+    return OracleChunks(status=rc, n=n, t_chunk=t_chunk, tail=tail, n_chunks=m, frames_kept=int(s.frames_kept),
+                        frames_deleted=int(s.frames_deleted), pad_frames=int(s.pad_frames), sum_t=int(s.sum_t),
+                        t_max=int(s.t_max), first_bad=int(s.first_bad), lengths=lengths,
+                        offsets=offsets(lengths) if n else np.zeros(1, np.int64), chunk_seq=seq[:m], chunk_first=first[:m],
+                        chunk_len=ln[:m])
+
+
+def chunk_metadata(c: OracleChunks, block_begin: int, block_count: int):
+    shape = (block_count, c.t_chunk)
+    seq_id = np.empty(shape, np.int32); pos = np.empty(shape, np.int32)
+    reset = np.empty(shape, np.uint8); valid = np.empty(shape, np.uint8)
+    t = c._tables()
+    rc = lib().oracle_chunk_metadata(C.byref(t), block_begin, block_count, _p(seq_id), _p(pos), _p(reset), _p(valid))
+    assert rc == 0, rc
+    return seq_id, pos, reset, valid
+
+
+def chunk_pack(c: OracleChunks, store: np.ndarray, frame_bytes: int, block_begin: int, block_count: int,
+               pad_byte: int = 0) -> np.ndarray:
+    store = np.ascontiguousarray(store).view(np.uint8).reshape(-1)
+    assert store.size == c.sum_t * frame_bytes
+    dense = np.empty((block_count, c.t_chunk, frame_bytes), np.uint8)
+    t = c._tables()
+    rc = lib().oracle_chunk_pack(C.byref(t), _p(store), frame_bytes, block_begin, block_count, _p(dense), pad_byte)
+    assert rc == 0, rc
+    return dense
+
+
+def chunk_unpack(c: OracleChunks, dense_out: np.ndarray, frame_bytes: int, block_begin: int, block_count: int,
+                 ragged_out: np.ndarray) -> np.ndarray:
+    dense_out = np.ascontiguousarray(dense_out).view(np.uint8).reshape(-1)
+    assert dense_out.size == block_count * c.t_chunk * frame_bytes
+    assert ragged_out.dtype == np.uint8 and ragged_out.flags.c_contiguous and ragged_out.size == c.sum_t * frame_bytes
+    t = c._tables()
+    rc = lib().oracle_chunk_unpack(C.byref(t), _p(dense_out), frame_bytes, block_begin, block_count, _p(ragged_out))
+    assert rc == 0, rc
+    return ragged_out

@@ -489,7 +489,16 @@ int bload_pack(const void* d_plan, const bload_plan_info_t* info, const void* d_
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     PlanView pv = plan_view(const_cast<void*>(d_plan), info->n);
     cudaError_t ce = cudaSuccess;
-    if (d_seq_id || d_pos || d_reset || d_valid)
+    const bool want_meta = d_seq_id || d_pos || d_reset || d_valid;
+    // a small call for dense blocks and metadata of small frames: one launch does both
+    if (want_meta && d_dense &&
+        staged_pack_with_metadata(pv, info->t_block, frame_bytes, block_begin, block_count, static_cast<const uint8_t*>(d_store),
+                                  static_cast<uint8_t*>(d_dense), d_seq_id, d_pos, d_reset, d_valid,
+                                  info->sum_t * frame_bytes, pad_byte, st, info->n, &ce)) {
+        if (ce != cudaSuccess) { (void)cudaGetLastError(); return BLOAD_ERR_CUDA; }
+        return BLOAD_OK;
+    }
+    if (want_meta)
         ce = launch_metadata(pv, info->t_block, block_begin, block_count, d_seq_id, d_pos, d_reset, d_valid, st);
     if (ce == cudaSuccess && d_dense)
         ce = launch_copy(false, pv, info->t_block, frame_bytes, block_begin, block_count,

@@ -71,6 +71,72 @@ __global__ void __launch_bounds__(256, 3) k11_carry_prev(PlanView pv, int32_t t_
     }
 }
 
+// The same result for short runs (many segments per sub-tile).  Inside the occupied part of a block, prev is the
+// dense input moved up by one frame -- the segments only matter at their first frames.  So a warp copies the
+// occupied part of its sub-tile as ONE shifted run, whatever the segments are (no per-segment alignment work, the
+// bytes in flight of a long run), fills the padding behind it, and then overwrites the first frame of every segment
+// that starts inside the sub-tile with the fill byte: one lane per segment for small frames, the whole warp per
+// segment for larger ones.  The patches are ordered after the copy's stores by a warp barrier.
+__global__ void __launch_bounds__(256, 3) k11_carry_shift(PlanView pv, int32_t t_block, int64_t frame_bytes, int64_t block_begin,
+                                                       int64_t block_count, const uint8_t* __restrict__ dense,
+                                                       uint8_t* __restrict__ prev, int64_t sub_bytes, int64_t subs_per_block,
+                                                       uint8_t fill_byte)
+{
+    const int lane = threadIdx.x & 31;
+    const int64_t warps = ((int64_t)gridDim.x * blockDim.x) >> 5;
+    const int64_t items = block_count * subs_per_block;
+    const int64_t block_bytes = (int64_t)t_block * frame_bytes;
+    const int64_t n_blocks = pv.hdr->n_blocks;
+    const uint8_t* s_limit = dense + block_count * block_bytes;
+    const uint32_t f4 = 0x01010101u * fill_byte;
+
+    for (int64_t item = (((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5); item < items; item += warps) {
+        const int64_t q = item / subs_per_block;
+        const int64_t lo = (item - q * subs_per_block) * sub_bytes;
+        const int64_t hi = min(lo + sub_bytes, block_bytes);
+        const int64_t b = block_begin + q;
+        uint8_t* out = prev + q * block_bytes;
+        int k0 = 0, k1 = 0;
+        int64_t valid_e = lo;  // end of the occupied part of [lo, hi)
+        if (b < n_blocks) {
+            k0 = pv.block_seg_begin[b]; k1 = pv.block_seg_begin[b + 1];
+            valid_e = max(lo, min(hi, (int64_t)pv.block_fill[b] * frame_bytes));
+        }
+        const int64_t c0 = max(lo, frame_bytes);  // slot 0 has no slot before it (and always starts a segment)
+        if (c0 < valid_e) warp_copy<true>(out + c0, dense + q * block_bytes + c0 - frame_bytes, valid_e - c0, s_limit, lane);
+        if (valid_e < hi) warp_fill(out + valid_e, hi - valid_e, fill_byte, lane);
+        if (lo >= valid_e) continue;
+        __syncwarp();
+        // first frames of the segments that reach into [lo, valid_e): segment ka holds the slot of byte lo
+        const int ka = warp_find_segment(pv.seg_start, k0, k1, (int)(lo / frame_bytes), lane);
+        for (int base = ka; base < k1; base += 32) {
+            const int kk = base + lane;
+            int64_t a = valid_e, e = valid_e;  // this lane's patch [a, e), empty by default
+            if (kk < k1) {
+                const int64_t fa = (int64_t)pv.seg_start[kk] * frame_bytes;
+                a = min(max(fa, lo), valid_e);
+                e = min(max(fa + frame_bytes, lo), valid_e);
+            }
+            if (frame_bytes <= 64) {
+                if (((a | e | reinterpret_cast<uintptr_t>(out)) & 3) == 0)
+                    for (int64_t x = a; x < e; x += 4) *reinterpret_cast<uint32_t*>(out + x) = f4;
+                else
+                    for (int64_t x = a; x < e; ++x) out[x] = fill_byte;
+            } else {
+                const unsigned live = __ballot_sync(kFull, a < e);
+                for (unsigned m = live; m; m &= m - 1) {
+                    const int src_lane = __ffs(m) - 1;
+                    const int64_t pa = __shfl_sync(kFull, a, src_lane), pe = __shfl_sync(kFull, e, src_lane);
+                    warp_fill(out + pa, pe - pa, fill_byte, lane);
+                }
+            }
+            // segments are in slot order: once one starts at or behind the end of the range, the rest do too
+            const bool beyond = kk >= k1 || (int64_t)pv.seg_start[kk] * frame_bytes >= valid_e;
+            if (__any_sync(kFull, beyond)) break;
+        }
+    }
+}
+
 // A warp owns `sub_bytes` of one row of the state.  It decides from the plan whether a sequence continues at
 // `slot` of the row's block (then the row is left alone) and otherwise writes the initial state over its part.
 __global__ void __launch_bounds__(256) k12_reset_state(PlanView pv, int64_t block_begin, int64_t block_count, int32_t slot,
@@ -214,10 +280,13 @@ cudaError_t launch_carry_prev(const PlanView& pv, int32_t t_block, int64_t frame
     const int64_t sub = 16384;
     const int64_t spb = (block_bytes + sub - 1) / sub;
     count_launches(1);
-    // small word-sized frames in short runs: the staged pack kernel with the dense input as its source
-    cudaError_t staged_err = cudaSuccess;
-    if (staged_carry_prev(pv, t_block, frame_bytes, block_begin, block_count, dense, prev, fill_byte, st, n, sum_t, &staged_err))
-        return staged_err;
+    // short runs (many segments per sub-tile): one shifted copy per sub-tile and patches at the segment starts
+    if (n > 0 && sum_t * frame_bytes / n <= 16384) {
+        note_copy_kernel(kCallCarryPrev, "k11_carry_shift");
+        k11_carry_shift<<<grid_for_items(block_count * spb), 256, 0, st>>>(pv, t_block, frame_bytes, block_begin, block_count,
+                                                                          dense, prev, sub, spb, fill_byte);
+        return cudaPeekAtLastError();
+    }
     note_copy_kernel(kCallCarryPrev, "k11_carry_prev");
     k11_carry_prev<<<grid_for_items(block_count * spb), 256, 0, st>>>(pv, t_block, frame_bytes, block_begin, block_count,
                                                                      dense, prev, sub, spb, fill_byte);

@@ -15,6 +15,7 @@
 // 16, e.g. 4-byte tokens) each output vector is assembled from two aligned source vectors with
 // funnel shifts.
 #include "bload_internal.cuh"
+#include "bload_meta.cuh"
 #include "bload_warp_copy.cuh"
 
 namespace bload {
@@ -471,22 +472,42 @@ __global__ void __launch_bounds__(StageCfg<false>::kWarps * 32) k9_unpack_ragged
 // twin of k9_unpack_ragged): the warp locates its first segment once and then walks forward through
 // the segment list, which runs on from one block to the next; only `fill` and the segment end of each
 // new block are read, one block ahead.  Blocks at or beyond n_blocks are written as padding.
-// CARRY: the same walk produces bload_carry_prev for small frames (source = the dense input, one frame back).
-template <bool CARRY>
+// META: the per-slot metadata of the same blocks comes out of the same launch.  The first `pack_ctas` CTAs pack; every
+// further CTA writes the metadata of 4 x blockDim.x consecutive slots of one block (the code of the metadata kernel).
+// A call for one training batch of small frames moves about a megabyte and is bound by launch overhead, so one launch
+// instead of two is the gain; the two kinds of CTA run side by side on the machine.
+struct MetaOut {
+    int32_t* seq_id; int32_t* pos; uint8_t* reset; uint8_t* valid;
+    uint32_t pack_ctas;        // CTAs of the grid that pack; the rest write metadata
+    int32_t chunks_per_block;  // metadata CTAs per block
+    int32_t vec;               // t_block % 4 == 0 and aligned outputs: vector stores
+};
+template <bool META>
 __global__ void __launch_bounds__(StageCfg<false>::kWarps * 32) k10_pack_contig(PlanView pv, int32_t n, int32_t t_block,
                                                                               int64_t frame_bytes, int64_t block_begin,
                                                                               const uint8_t* __restrict__ store,
                                                                               uint8_t* __restrict__ dense, int64_t tiles,
                                                                               int64_t tiles_per_warp, int32_t subs_per_block,
-                                                                              uint8_t pad)
+                                                                              uint8_t pad, MetaOut mo)
 {
     using Cfg = StageCfg<false>;
     constexpr int NST = Cfg::kStages, kStageBytes = Cfg::kBytes, kStageWarps = Cfg::kWarps;
+    if (META && blockIdx.x >= mo.pack_ctas) {
+        const uint32_t m = blockIdx.x - mo.pack_ctas;
+        const uint32_t q = m / (uint32_t)mo.chunks_per_block;
+        const int s0 = (int)(m - q * (uint32_t)mo.chunks_per_block) * (kStageWarps * 32 * 4) + (int)threadIdx.x * 4;
+        if (s0 < t_block) {
+            const int64_t o = (int64_t)q * t_block + s0;
+            if (mo.vec) metadata_quad<true>(pv, t_block, block_begin + q, pv.hdr->n_blocks, s0, o, mo.seq_id, mo.pos, mo.reset, mo.valid);
+            else metadata_quad<false>(pv, t_block, block_begin + q, pv.hdr->n_blocks, s0, o, mo.seq_id, mo.pos, mo.reset, mo.valid);
+        }
+        return;
+    }
     extern __shared__ __align__(128) uint8_t stage_mem[];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     uint8_t* my_stages = stage_mem + (size_t)warp * NST * kStageBytes;
     const int64_t gw = (int64_t)blockIdx.x * kStageWarps + warp;
-    const int64_t n_warps = (int64_t)gridDim.x * kStageWarps;
+    const int64_t n_warps = (int64_t)(META ? mo.pack_ctas : gridDim.x) * kStageWarps;
     const int fb = (int)frame_bytes;
     const int block_bytes = t_block * fb;
     const int64_t n_blocks = pv.hdr->n_blocks;
@@ -538,17 +559,7 @@ __global__ void __launch_bounds__(StageCfg<false>::kWarps * 32) k10_pack_contig(
             const int64_t src = __shfl_sync(kFull, w_src, k - kw);
             const int seg_e = (k + 1 < k1) ? nx * fb : fill_bytes;  // the block's last run ends where its frames end
             const int pe = min(seg_e, hi);
-            if (CARRY) {
-                // `store` is the dense input: the first frame of a segment receives the fill pattern, every later byte
-                // the byte one frame before it in the same block
-                const int fe = min(st * fb + fb, pe);
-                for (int o = cur + 4 * lane; o < fe; o += 128) *reinterpret_cast<uint32_t*>(stage + (o - lo)) = p4;
-                cur = max(cur, fe);
-                if (cur < pe)
-                    warp_gather_async(sa + (uint32_t)(cur - lo), store + q * (int64_t)block_bytes + (cur - fb), pe - cur, lane);
-            } else {
-                warp_gather_async(sa + (uint32_t)(cur - lo), store + src * fb + (cur - st * fb), pe - cur, lane);
-            }
+            warp_gather_async(sa + (uint32_t)(cur - lo), store + src * fb + (cur - st * fb), pe - cur, lane);
             cur = pe;
             if (pe == seg_e) ++k;
         }
@@ -580,21 +591,24 @@ __global__ void __launch_bounds__(StageCfg<false>::kWarps * 32) k10_pack_contig(
 
 }  // namespace
 
-// bload_carry_prev through the staged pack kernel; false when the frame size or the run lengths do not suit it.
-bool staged_carry_prev(const PlanView& pv, int32_t t_block, int64_t frame_bytes, int64_t block_begin, int64_t block_count,
-                       const uint8_t* dense, uint8_t* prev, uint8_t fill_byte, cudaStream_t st, int64_t n, int64_t sum_t,
-                       cudaError_t* err)
+// Pack and per-slot metadata of a few blocks of small word-sized frames in ONE launch (see k10_pack_contig<true>);
+// false when the call does not suit the staged pack kernel or is large enough for two full-speed launches.
+bool staged_pack_with_metadata(const PlanView& pv, int32_t t_block, int64_t frame_bytes, int64_t block_begin,
+                               int64_t block_count, const uint8_t* store, uint8_t* dense, int32_t* seq_id, int32_t* pos,
+                               uint8_t* reset, uint8_t* valid, int64_t ragged_bytes, uint8_t pad_byte, cudaStream_t st,
+                               int64_t n, cudaError_t* err)
 {
-    const int64_t block_bytes = (int64_t)t_block * frame_bytes;
-    if (!(frame_bytes % 4 == 0 && n > 0 && sum_t * frame_bytes / n <= kStagedMaxRunBytes && block_bytes < (1LL << 31) &&
-          block_bytes % 16 == 0))
-        return false;
     using Cfg = StageCfg<false>;
+    const int64_t block_bytes = (int64_t)t_block * frame_bytes;
+    constexpr int64_t kMaxFusedSlots = 1 << 22;  // beyond this the metadata kernel's own launch shape is faster
+    if (!(frame_bytes % 4 == 0 && n > 0 && ragged_bytes / n <= kStagedMaxRunBytes && block_bytes < (1LL << 31) &&
+          block_bytes % 16 == 0 && block_count * t_block <= kMaxFusedSlots))
+        return false;
     const size_t smem = (size_t)Cfg::kWarps * Cfg::kStages * Cfg::kBytes + 16;
-    const DeviceInfo di = device_info();
-        const int per_sm = (int)(di.smem_per_sm / (smem + 1024));
     *err = opt_in_shared_memory(k10_pack_contig<true>, (int)smem);
     if (*err != cudaSuccess) return true;
+    const DeviceInfo di = device_info();
+    const int per_sm = (int)(di.smem_per_sm / (smem + 1024));
     const int64_t spb = (block_bytes + Cfg::kBytes - 1) / Cfg::kBytes;
     const int64_t tiles = block_count * spb;
     const int64_t max_warps = (int64_t)di.sm_count * per_sm * Cfg::kWarps;
@@ -602,10 +616,17 @@ bool staged_carry_prev(const PlanView& pv, int32_t t_block, int64_t frame_bytes,
     if (tpw > kPackChunkTiles) tpw = kPackChunkTiles;
     int64_t warps = (tiles + tpw - 1) / tpw;
     if (warps > max_warps) warps = max_warps;
-    const unsigned grid = (unsigned)((warps + Cfg::kWarps - 1) / Cfg::kWarps);
-    k10_pack_contig<true><<<grid, Cfg::kWarps * 32, smem, st>>>(pv, (int32_t)n, t_block, frame_bytes, block_begin, dense, prev,
-                                                               tiles, tpw, (int32_t)spb, fill_byte);
-    note_copy_kernel(kCallCarryPrev, "k10_pack_contig<carry>");
+    auto al = [](const void* p, uintptr_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; };
+    MetaOut mo;
+    mo.seq_id = seq_id; mo.pos = pos; mo.reset = reset; mo.valid = valid;
+    mo.pack_ctas = (uint32_t)((warps + Cfg::kWarps - 1) / Cfg::kWarps);
+    mo.chunks_per_block = (int32_t)((t_block + Cfg::kWarps * 128 - 1) / (Cfg::kWarps * 128));
+    mo.vec = t_block % 4 == 0 && al(seq_id, 16) && al(pos, 16) && al(reset, 4) && al(valid, 4);
+    const int64_t grid = (int64_t)mo.pack_ctas + block_count * mo.chunks_per_block;
+    count_launches(1);
+    note_copy_kernel(kCallPack, "k10_pack_contig<metadata>");
+    k10_pack_contig<true><<<(unsigned)grid, Cfg::kWarps * 32, smem, st>>>(pv, (int32_t)n, t_block, frame_bytes, block_begin, store,
+                                                                        dense, tiles, tpw, (int32_t)spb, pad_byte, mo);
     *err = cudaPeekAtLastError();
     return true;
 }
@@ -635,7 +656,7 @@ cudaError_t launch_copy(bool unpack, const PlanView& pv, int32_t t_block, int64_
         if (warps > max_warps) warps = max_warps;
         const unsigned grid = (unsigned)((warps + Cfg::kWarps - 1) / Cfg::kWarps);
         k10_pack_contig<false><<<grid, Cfg::kWarps * 32, smem, st>>>(pv, (int32_t)n, t_block, frame_bytes, block_begin, ragged_in,
-                                                             dense, tiles, tpw, (int32_t)spb, pad_byte);
+                                                             dense, tiles, tpw, (int32_t)spb, pad_byte, MetaOut{});
         note_copy_kernel(kCallPack, "k10_pack_contig");
         return cudaPeekAtLastError();
     }

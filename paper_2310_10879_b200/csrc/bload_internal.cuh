@@ -164,9 +164,10 @@ cudaError_t launch_copy_var(bool unpack, const PlanView& pv, int32_t t_block, in
 cudaError_t launch_carry_prev(const PlanView& pv, int32_t t_block, int64_t frame_bytes, int64_t block_begin,
                               int64_t block_count, const uint8_t* dense, uint8_t* prev, uint8_t fill_byte, cudaStream_t st,
                               int64_t n, int64_t sum_t);
-bool staged_carry_prev(const PlanView& pv, int32_t t_block, int64_t frame_bytes, int64_t block_begin, int64_t block_count,
-                       const uint8_t* dense, uint8_t* prev, uint8_t fill_byte, cudaStream_t st, int64_t n, int64_t sum_t,
-                       cudaError_t* err);
+bool staged_pack_with_metadata(const PlanView& pv, int32_t t_block, int64_t frame_bytes, int64_t block_begin,
+                               int64_t block_count, const uint8_t* store, uint8_t* dense, int32_t* seq_id, int32_t* pos,
+                               uint8_t* reset, uint8_t* valid, int64_t ragged_bytes, uint8_t pad_byte, cudaStream_t st,
+                               int64_t n, cudaError_t* err);
 cudaError_t launch_reset_state(const PlanView& pv, int64_t block_begin, int64_t block_count, int32_t slot, uint8_t* state,
                                int64_t state_bytes, const uint8_t* init, cudaStream_t st);
 cudaError_t launch_repeat_last(const PlanView& pv, int32_t t_block, int64_t frame_bytes, int64_t block_begin,

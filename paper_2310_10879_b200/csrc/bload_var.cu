@@ -79,21 +79,40 @@ __global__ void __launch_bounds__(kScanThreads) k15_var_offsets(const int32_t* _
     }
 }
 
+// Division of a 32-bit unsigned number by a divisor fixed at launch: a multiply-high and two shifts
+// (Granlund and Montgomery, "Division by invariant integers using multiplication", PLDI 1994).
+struct FastDiv { uint32_t mul, sh1, sh2, d; };
+__device__ __forceinline__ uint32_t fast_div(uint32_t n, const FastDiv& f)
+{
+    const uint32_t t = __umulhi(f.mul, n);
+    return (t + ((n - t) >> f.sh1)) >> f.sh2;
+}
+
 // Frames are images of `rows` rows of `frame_bytes` (row) bytes; a slot is a canvas of rows_max rows of row_stride
 // bytes and an image sits in its top left corner (one row per frame and rows_max == 1 give the plain
 // per-sequence frame size).  The dense side is walked row by row of the canvases ("sub-slots" of row_stride
 // bytes).  Row counts and row sizes are clamped to the canvas on the device, so a caller that breaks the documented
 // precondition gets truncated images but never an access outside the buffers.
+#ifndef BLOAD_VAR_MIN_CTAS
+#define BLOAD_VAR_MIN_CTAS 2
+#endif
+#ifndef BLOAD_VAR_UNROLL
+#define BLOAD_VAR_UNROLL 4
+#endif
 template <bool UNPACK>
-__global__ void __launch_bounds__(256, 2) k16_copy_var(PlanView pv, int32_t t_block, int32_t rows_max, int64_t row_stride,
+__global__ void __launch_bounds__(256, BLOAD_VAR_MIN_CTAS) k16_copy_var(PlanView pv, int32_t t_block, int32_t rows_max, int64_t row_stride,
                                                        int64_t block_begin, int64_t block_count,
                                                        const int32_t* __restrict__ seq_rows /*null: one row*/,
                                                        const int32_t* __restrict__ frame_bytes,
                                                        const int64_t* __restrict__ byte_offsets,
                                                        const uint8_t* __restrict__ src_base, uint8_t* __restrict__ dst_base,
-                                                       int64_t sub_bytes, int64_t subs_per_block, uint8_t pad)
+                                                       int64_t sub_bytes, int64_t subs_per_block, uint8_t pad,
+                                                       FastDiv div_vpr /*by row_stride / 16*/, FastDiv div_rows /*by rows_max*/)
 {
     const int lane = threadIdx.x & 31;
+    const bool rows_aligned = (row_stride & 15) == 0;  // every canvas row starts on a 16-byte boundary
+    const uint32_t p4 = 0x01010101u * pad;
+    const uint4 padv = make_uint4(p4, p4, p4, p4);
     const int64_t warps = ((int64_t)gridDim.x * blockDim.x) >> 5;
     const int64_t items = block_count * subs_per_block;
     const int64_t slot_bytes = (int64_t)rows_max * row_stride;
@@ -144,6 +163,54 @@ __global__ void __launch_bounds__(256, 2) k16_copy_var(PlanView pv, int32_t t_bl
                         const int64_t rag = off + (cur - (int64_t)st * slot_bytes);
                         if (UNPACK) warp_copy<true>(dst_base + rag, src_base + dense_off + cur, seg_e - cur, s_limit, lane);
                         else warp_copy<false>(dst_base + dense_off + cur, src_base + rag, seg_e - cur, s_limit, lane);
+                        cur = seg_e;
+                    } else if (rows_aligned && ((fb | off) & 15) == 0) {
+                        // Rows of the store and of the canvases all start on 16-byte boundaries: one flat loop over the
+                        // 16-byte vectors of [cur, seg_e) on the dense side.  A vector lies in canvas row `rr` of slot
+                        // `sr` (both by the launch-constant divisions) and is either image data, which has its fixed
+                        // place in the store, or padding; four independent vectors per lane are in flight.
+                        const uint32_t nvec = (uint32_t)((seg_e - cur) >> 4);
+                        const uint32_t c0 = (uint32_t)(in >> 4), fbv = (uint32_t)(fb >> 4), vpr = div_vpr.d;
+                        const int64_t slot_rel0 = slot - st;
+                        uint4* __restrict__ dv = reinterpret_cast<uint4*>((UNPACK ? const_cast<uint8_t*>(src_base) : dst_base) + dense_off + cur);
+                        uint8_t* rag_seg = (UNPACK ? dst_base : const_cast<uint8_t*>(src_base)) + off;
+                        auto locate = [&](uint32_t i, bool& data) -> uint4* {
+                            const uint32_t ca = c0 + i;
+                            const uint32_t jr = fast_div(ca, div_vpr);
+                            const uint32_t c = ca - jr * vpr;
+                            const uint32_t ra = (uint32_t)r + jr;
+                            const uint32_t sr = fast_div(ra, div_rows);
+                            const uint32_t rr = ra - sr * (uint32_t)rows_max;
+                            data = rr < (uint32_t)rows && c < fbv;
+                            return reinterpret_cast<uint4*>(rag_seg + ((slot_rel0 + sr) * rows + rr) * fb + 16 * (int64_t)c);
+                        };
+                        uint32_t i = lane;
+                        constexpr int U = BLOAD_VAR_UNROLL;
+                        for (; i + 32 * (U - 1) < nvec; i += 32 * U) {
+                            uint4 v[U]; uint4* rp[U]; bool data[U];
+#pragma unroll
+                            for (int u = 0; u < U; ++u) {
+                                rp[u] = locate(i + 32 * u, data[u]);
+                                v[u] = padv;
+                                if (data[u]) v[u] = ld_stream(UNPACK ? dv + i + 32 * u : rp[u]);
+                            }
+#pragma unroll
+                            for (int u = 0; u < U; ++u) {
+                                if (!UNPACK) st_stream(dv + i + 32 * u, v[u]);
+                                else if (data[u]) st_stream(rp[u], v[u]);
+                            }
+                        }
+                        for (; i < nvec; i += 32) {
+                            bool data;
+                            uint4* rp = locate(i, data);
+                            if (!UNPACK) st_stream(dv + i, data ? ld_stream(rp) : padv);
+                            else if (data) st_stream(rp, ld_stream(dv + i));
+                        }
+                        // where the walk stands after nvec vectors
+                        const uint32_t ca = c0 + nvec, jr = fast_div(ca, div_vpr), ra = (uint32_t)r + jr, sr = fast_div(ra, div_rows);
+                        in = (int64_t)(ca - jr * vpr) << 4;
+                        r = (int)(ra - sr * (uint32_t)rows_max);
+                        slot += (int)sr;
                         cur = seg_e;
                     } else {
                         while (cur < seg_e) {
@@ -197,14 +264,27 @@ cudaError_t launch_copy_var(bool unpack, const PlanView& pv, int32_t t_block, in
     const int64_t spb = (block_bytes + sub - 1) / sub;
     const int64_t want = (block_count * spb + 7) / 8;
     const unsigned grid = (unsigned)(want < 0x7fffffffLL ? want : 0x7fffffffLL);
+    // divisors of the kernel's flat vector loop (used when row_stride is a multiple of 16)
+    auto make_div = [](uint32_t d) {
+        FastDiv f;
+        uint32_t l = 0;
+        while ((1ull << l) < d) ++l;
+        f.mul = (uint32_t)((((1ull << l) - d) << 32) / d + 1);
+        f.sh1 = l < 1 ? l : 1;
+        f.sh2 = l > 0 ? l - 1 : 0;
+        f.d = d;
+        return f;
+    };
+    const FastDiv div_vpr = make_div((uint32_t)(row_stride >= 16 && row_stride / 16 < 0x7fffffffLL ? row_stride / 16 : 1));
+    const FastDiv div_rows = make_div((uint32_t)rows_max);
     count_launches(1);
     note_copy_kernel(unpack ? kCallUnpackVar : kCallPackVar, unpack ? "k16_copy_var<unpack>" : "k16_copy_var<pack>");
     if (unpack)
         k16_copy_var<true><<<grid, 256, 0, st>>>(pv, t_block, rows_max, row_stride, block_begin, block_count, seq_rows,
-                                                  frame_bytes, byte_offsets, src, dst, sub, spb, pad_byte);
+                                                  frame_bytes, byte_offsets, src, dst, sub, spb, pad_byte, div_vpr, div_rows);
     else
         k16_copy_var<false><<<grid, 256, 0, st>>>(pv, t_block, rows_max, row_stride, block_begin, block_count, seq_rows,
-                                                   frame_bytes, byte_offsets, src, dst, sub, spb, pad_byte);
+                                                   frame_bytes, byte_offsets, src, dst, sub, spb, pad_byte, div_vpr, div_rows);
     return cudaPeekAtLastError();
 }
 

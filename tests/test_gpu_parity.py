@@ -238,6 +238,40 @@ def test_small_word_sized_frames_take_the_staged_path(tb, fb, tmax):
         assert np.array_equal(res["dense"], O.pack(op, store.cpu().numpy(), fb, 1, 2, 0))
 
 
+@pytest.mark.parametrize("tb,fb,tmax", [(4096, 4, 4096), (64, 4, 64), (1000, 16, 9), (700, 256, 60), (36, 12, 36)])
+def test_one_launch_for_dense_blocks_and_metadata_of_small_frames(tb, fb, tmax):
+    """A pack call that asks for dense blocks and metadata of small word-sized frames is ONE launch (some CTAs pack, the
+    others write metadata).  Its outputs equal those of the two separate calls and the oracle's: sub-ranges, filler
+    blocks behind the plan, a metadata array left out, metadata pointers that force the scalar stores."""
+    rng = np.random.default_rng(tb * 7 + fb)
+    n = int(min(3000, max(3, 3_000_000 // (tmax * fb))))
+    T = rng.integers(1, tmax + 1, size=n).astype(np.int32)
+    op = O.plan(T, tb, 17); plan = G.gpu_plan(T, tb, 17)
+    store = torch.randint(0, 256, (op.sum_t * fb,), dtype=torch.uint8, device=G.DEV)
+    store_h = store.cpu().numpy()
+    nb = op.n_blocks
+    for b0, cnt in [(0, nb + 2), (0, 1), (max(nb // 2, 0), min(3, nb)), (nb - 1, 4), (nb + 1, 2)]:
+        before = B.bload_kernel_launches()
+        res, _ = G.gpu_pack_all(plan, store, fb, b0, cnt, 0x3C)
+        assert B.bload_kernel_launches() - before == 1
+        assert B.bload_last_copy_kernel("pack") == "k10_pack_contig<metadata>"
+        assert np.array_equal(res["dense"], O.pack(op, store_h, fb, b0, cnt, 0x3C))
+        for name, want in zip(("seq_id", "pos", "reset", "valid"), O.metadata(op, b0, cnt)):
+            assert np.array_equal(res[name], want), name
+    # only two of the four arrays, at addresses that are not vector aligned
+    cnt = min(nb, 5)
+    raw_pos = torch.full((cnt * tb + 3,), 77, dtype=torch.int32, device=G.DEV)
+    raw_valid = torch.full((cnt * tb + 3,), 77, dtype=torch.uint8, device=G.DEV)
+    dense = G.Guarded(cnt * tb * fb)
+    B.bload_pack(plan, store, fb, 0, cnt, dense=dense.t, pos=raw_pos[1:1 + cnt * tb], valid=raw_valid[1:1 + cnt * tb])
+    torch.cuda.synchronize(); dense.check()
+    want = O.metadata(op, 0, cnt)
+    assert np.array_equal(raw_pos[1:1 + cnt * tb].cpu().numpy().reshape(cnt, tb), want[1])
+    assert np.array_equal(raw_valid[1:1 + cnt * tb].cpu().numpy().reshape(cnt, tb), want[3])
+    assert int(raw_pos[0]) == 77 and int(raw_pos[-1]) == 77 and int(raw_valid[0]) == 77 and int(raw_valid[-1]) == 77
+    assert np.array_equal(dense.t.cpu().numpy().reshape(cnt, tb, fb), O.pack(op, store_h, fb, 0, cnt, 0))
+
+
 @pytest.mark.parametrize("tb,fb,lengths", [(6, 4, [2, 2, 3, 3, 4, 5, 6, 6]), (7, 12, [1]), (9, 20, [9, 1, 1]),
                                            (5, 4, [1, 1, 1]), (3000, 4, None), (1234, 36, None)])
 def test_whole_plan_unpack_of_word_sized_frames(tb, fb, lengths):

@@ -181,3 +181,29 @@ def test_canvases_of_equal_images_match_the_fixed_size_pack():
     B.bload_pack(plan, store, h * wb, 0, nb, dense=b, pad_byte=3)
     torch.cuda.synchronize()
     assert torch.equal(a, b)
+
+
+@pytest.mark.parametrize("unit,kmax,extra", [(16, 1, 0), (16, 9, 16), (64, 16, 0), (256, 16, 48), (1024, 4, 0), (1024, 40, 1024)])
+def test_frame_sizes_that_are_multiples_of_16_bytes(unit, kmax, extra):
+    """Frames and slots whose sizes are multiples of 16 bytes take the kernel's flat vector loop; a few sizes that are
+    not are mixed in, so that one launch holds segments of both kinds."""
+    rng = np.random.default_rng(unit + kmax)
+    tb = int(rng.integers(4, 70))
+    n = int(rng.integers(20, 200))
+    T = rng.integers(1, tb + 1, size=n)
+    F = rng.integers(1, kmax + 1, size=n) * unit
+    F[-3:] = np.maximum(F[-3:] - 4, 4)           # the last sequences: word-aligned but not vector-aligned sizes and offsets
+    _parity(T, F, tb, 21 + unit, slot=unit * kmax + extra)
+
+
+@pytest.mark.parametrize("hmax,unit,kmax,extra", [(1, 16, 8, 16), (3, 16, 5, 0), (5, 32, 9, 32), (12, 128, 6, 0), (40, 16, 50, 16)])
+def test_images_whose_rows_are_multiples_of_16_bytes(hmax, unit, kmax, extra):
+    rng = np.random.default_rng(hmax * 100 + kmax)
+    tb = int(rng.integers(3, 40))
+    n = int(rng.integers(5, 80))
+    T = rng.integers(1, tb + 1, size=n)
+    H = rng.integers(1, hmax + 1, size=n)
+    Wb = rng.integers(1, kmax + 1, size=n) * unit
+    H[0], Wb[0] = hmax, kmax * unit
+    Wb[-1] = max(4, Wb[-1] - 8)                  # the last sequence is off the vector path
+    _parity2d(T, H, Wb, tb, 9 + hmax, hmax, kmax * unit + extra)
