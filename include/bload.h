@@ -53,6 +53,8 @@ extern "C" {
 #define BLOAD_POLICY_UNIFORM_SEQUENCES 0u /* every unused sequence that fits is equally likely */
 #define BLOAD_POLICY_BEST_FIT_DECREASING 2u /* NOT the paper's rule: the textbook best-fit-decreasing heuristic, a
                                              deterministic low-padding comparison (seed only orders equal lengths) */
+#define BLOAD_POLICY_CHUNKS_KEEP_TAIL 3u /* written into info.policy by bload_plan_chunks (not accepted by bload_plan) */
+#define BLOAD_POLICY_CHUNKS_DROP_TAIL 4u
 #define BLOAD_POLICY_UNIFORM_LENGTHS 1u   /* every length (key of L_dict) that fits and is not exhausted is equally
                                              likely, then the next unused sequence of that length; needs n < 2^26 */
 
@@ -86,7 +88,7 @@ typedef struct {
     int64_t max_segs_per_block;
     uint64_t seed;
     uint32_t policy;
-    uint32_t reserved_;
+    uint32_t n_source;       /* plans made by bload_plan_chunks: the sequences the chunks were cut from; else 0 */
 } bload_plan_info_t;
 
 typedef struct {
@@ -101,6 +103,7 @@ typedef struct {
     double reduction_vs_tmax; /* pad_naive_tmax / pad_packed (0 when pad_packed == 0) */
     double mean_segs_per_block;
     int64_t max_segs_per_block;
+    int64_t frames_deleted;   /* 0 except for plans of bload_plan_chunks with BLOAD_CHUNKS_DROP_TAIL */
 } bload_stats_t;
 
 /*
@@ -361,8 +364,63 @@ BLOAD_API int bload_valid_sum(const void* d_plan, const bload_plan_info_t* info,
 /*
  * bload_stats -- padding statistics from the scalars of a plan (host only; closed forms).
  * pad_naive_tmax is the "0 padding" row of the paper's Table I, pad_packed its "block_pad" row.
+ * For a plan of bload_plan_chunks the samples are the chunks: n = n_chunks = n_blocks, t_max = longest chunk,
+ * pad_packed = n_chunks * t_chunk - frames kept, frames_deleted = frames of the store - frames kept, and the
+ * naive-padding fields describe padding every chunk to the longest chunk.
  */
 BLOAD_API int bload_stats(const bload_plan_info_t* info, bload_stats_t* out);
+
+/*
+ * The chunking strategy that the paper compares BLoad with (section "Problem Statement and Current Limitations":
+ * every sample is broken into chunks of T_block frames and every chunk is treated as an individual sample; figure
+ * "Sampling solution"; Table I, column "sampling").  Built as a planner only, so that its padding and deleted frames
+ * can be put beside BLoad's on the same data and its batches come out of the same kernels.
+ *
+ * Sequence i (any T_i >= 1; it may be longer than t_chunk) is cut at frames 0, t_chunk, 2 t_chunk, ...
+ *   BLOAD_CHUNKS_KEEP_TAIL  the last, shorter chunk is kept and padded: nothing is deleted
+ *   BLOAD_CHUNKS_DROP_TAIL  only full chunks are kept: no padding, the last T_i mod t_chunk frames of every sequence
+ *                           are deleted (the reading under which the table's "sampling" column has zero padding and
+ *                           a count of deleted frames)
+ * Chunks are numbered in order of (sequence, position).  The plan that bload_plan_chunks writes is an ordinary plan
+ * of n_chunks "sequences" in blocks of t_chunk slots: chunk j is sequence j, alone in block j from slot 0, and its
+ * entry of the offsets table is its first frame in the ORIGINAL ragged store ([n_chunks] = all frames of that store),
+ * so bload_pack, bload_unpack (deleted frames are never touched), bload_carry_prev, bload_reset_state,
+ * bload_valid_sum and bload_stats take it as it is.  Per-slot metadata then names chunks: seq_id = chunk number,
+ * pos = position inside the chunk, reset = 1 at slot 0 of every block -- which is the strategy's weakness the paper
+ * points out: state cannot be carried from one chunk of a sequence to the next.  d_chunk_seq / d_chunk_first
+ * (int32[n_chunks], each may be NULL) receive the sequence each chunk was cut from and its first frame there.
+ * The calls for per-sequence frame sizes (bload_pack_var ...) do not accept such a plan (BLOAD_ERR_UNSUPPORTED).
+ *
+ * bload_chunk_count   the totals, after one synchronisation of `stream`; needs them before the plan can be sized
+ * bload_plan_chunks   the plan; n_chunks as counted (BLOAD_ERR_ARG if the lengths give another number); plan_bytes at
+ *                     least bload_plan_sizes(n_chunks, t_chunk).plan_bytes; one synchronisation of `stream`
+ * d_work: device scratch of bload_chunk_work_bytes(n) bytes, 256-byte aligned (both calls).
+ * Errors: NULL, ARG (n < 1, t_chunk < 1, unknown tail, n_chunks < 1: with DROP_TAIL every sequence may be shorter
+ * than a chunk, then there is nothing to plan), UNSUPPORTED (t_chunk > BLOAD_MAX_T_BLOCK), LENGTH (some T_i < 1, index
+ * in first_bad_index), WORKSPACE, ALIGN, CUDA.
+ */
+#define BLOAD_CHUNKS_KEEP_TAIL 0u
+#define BLOAD_CHUNKS_DROP_TAIL 1u
+typedef struct {
+    int32_t status;
+    uint32_t tail;
+    int32_t t_chunk;
+    int32_t reserved_;
+    int64_t n;               /* sequences */
+    int64_t n_chunks;        /* = blocks */
+    int64_t frames_kept;
+    int64_t frames_deleted;  /* Table I, row "# frames deleted" */
+    int64_t pad_frames;      /* Table I, row "padding amount": n_chunks * t_chunk - frames_kept */
+    int64_t sum_t;           /* frames of the ragged store */
+    int64_t t_max;           /* longest sequence */
+    int64_t first_bad_index; /* first i with T_i < 1, else -1 */
+} bload_chunk_info_t;
+BLOAD_API size_t bload_chunk_work_bytes(int64_t n);
+BLOAD_API int bload_chunk_count(const int32_t* d_lengths, int64_t n, int32_t t_chunk, uint32_t tail, void* d_work,
+                                size_t work_bytes, void* stream, bload_chunk_info_t* out);
+BLOAD_API int bload_plan_chunks(const int32_t* d_lengths, int64_t n, int32_t t_chunk, uint32_t tail, int64_t n_chunks,
+                                void* d_plan, size_t plan_bytes, void* d_work, size_t work_bytes, int32_t* d_chunk_seq,
+                                int32_t* d_chunk_first, void* stream, bload_plan_info_t* info);
 
 /*
  * bload_plan_static -- bload_plan for callers that must not, or cannot, allocate device memory.
@@ -438,6 +496,17 @@ BLOAD_API int bload_plan_stage_times(float out_ms[4]);
  * (all threads).  Host only; lets a benchmark report how many launches a timed region contained.
  */
 BLOAD_API int64_t bload_kernel_launches(void);
+
+/*
+ * bload_debug_status -- what the bounds-checking build of the library has seen.  That build (compiled with
+ * -DBLOAD_DEBUG as libbload_debug.so) checks every global-memory access of its copy, metadata and table kernels
+ * against the buffer ranges of the call, skips an access that lies outside them and records it; nothing traps.
+ * out[0] = accesses refused since the last clear, out[1] = number of the kernel with the first one (5 tables,
+ * 6 metadata, 7 to 11 and 16 the copy kernels, 12 state reset, 14 repeat-last), out[2] = 0 read / 1 write,
+ * out[3] = its address.  Synchronises the device.  `clear` != 0 resets the record.  The ordinary build returns
+ * BLOAD_ERR_UNSUPPORTED and zeros.  Calls that run kernels on two streams at once (bload_epoch) are not checked.
+ */
+BLOAD_API int bload_debug_status(uint64_t out[4], int clear);
 
 /*
  * bload_last_copy_kernel -- name of the copy kernel that the most recent call of this host thread launched for

@@ -427,7 +427,8 @@ class OracleChunks:
         off[m] = self.sum_t
         digest = int(lib().oracle_digest(_p(ar), _p(zeros), _p(ar), m))
         return OraclePlan(status=self.status, n=m, t_block=self.t_chunk, seed=0, n_blocks=m, sum_t=self.sum_t,
-                          t_max=self.t_max, first_bad=self.first_bad, checksum=digest, max_segs_per_block=1 if m else 0,
+                          t_max=int(self.chunk_len.max()) if m else 0, first_bad=self.first_bad, checksum=digest,
+                          max_segs_per_block=1 if m else 0,
                           lengths=self.chunk_len.copy(), offsets=off, seg_seq=ar.copy(), seg_block=ar.copy(),
                           seg_start=zeros.copy(), block_seg_begin=np.arange(m + 1, dtype=np.int32),
                           block_fill=self.chunk_len.copy(), seq_block=ar.copy(), seq_start=zeros.copy())

@@ -7,6 +7,6 @@
 
 The shared library is loaded on first use; nothing here computes on the CPU.
 """
-from ._lib import (BloadError, Plan, PlanInfo, Sizes, bload_pack, bload_plan, bload_plan_static, bload_plan_async, bload_plan_finish, bload_plan_sizes, bload_rank_range,  # noqa: F401
+from ._lib import (BloadError, Plan, PlanInfo, Sizes, bload_pack, bload_plan, bload_plan_static, bload_plan_chunks, ChunkInfo, bload_plan_async, bload_plan_finish, bload_plan_sizes, bload_rank_range,  # noqa: F401
                    bload_epoch, bload_epoch_stage_times, bload_carry_prev, bload_reset_state, bload_valid_sum, bload_var_offsets, bload_pack_var, bload_unpack_var, bload_var_offsets2d, bload_pack_var2d, bload_unpack_var2d,
-                   bload_kernel_launches, bload_last_copy_kernel, bload_plan_stage_times, bload_set_plan_timing, bload_stats, bload_unpack, load, strerror)
+                   bload_kernel_launches, bload_last_copy_kernel, bload_debug_status, bload_plan_stage_times, bload_set_plan_timing, bload_stats, bload_unpack, load, strerror)

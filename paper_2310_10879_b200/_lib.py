@@ -20,7 +20,7 @@ MAX_T_BLOCK = 32768
 EXPORTS = ("bload_plan_sizes", "bload_plan", "bload_plan_async", "bload_plan_finish", "bload_rank_range", "bload_pack", "bload_unpack", "bload_stats", "bload_epoch", "bload_epoch_stage_times",
            "bload_pack_repeat_last", "bload_var_offsets", "bload_pack_var", "bload_unpack_var", "bload_var_offsets2d", "bload_pack_var2d",
            "bload_unpack_var2d", "bload_carry_prev", "bload_reset_state", "bload_valid_sum",
-           "bload_plan_static", "bload_set_plan_timing", "bload_plan_stage_times", "bload_kernel_launches", "bload_last_copy_kernel",
+           "bload_plan_static", "bload_chunk_work_bytes", "bload_chunk_count", "bload_plan_chunks", "bload_set_plan_timing", "bload_plan_stage_times", "bload_kernel_launches", "bload_last_copy_kernel", "bload_debug_status",
            "bload_strerror", "bload_version")
 
 
@@ -35,7 +35,7 @@ class PlanInfo(C.Structure):
     _fields_ = [("status", C.c_int32), ("t_block", C.c_int32), ("n", C.c_int64), ("n_blocks", C.c_int64),
                 ("sum_t", C.c_int64), ("t_max", C.c_int64), ("first_bad_index", C.c_int64),
                 ("checksum", C.c_uint64), ("max_segs_per_block", C.c_int64), ("seed", C.c_uint64),
-                ("policy", C.c_uint32), ("reserved_", C.c_uint32)]
+                ("policy", C.c_uint32), ("n_source", C.c_uint32)]
 
 
 class Stats(C.Structure):
@@ -43,7 +43,7 @@ class Stats(C.Structure):
                                           "pad_naive_tmax", "pad_naive_tblock", "min_blocks")] + \
                [(k, C.c_double) for k in ("frac_packed", "frac_naive_tmax", "frac_naive_tblock",
                                           "reduction_vs_tmax", "mean_segs_per_block")] + \
-               [("max_segs_per_block", C.c_int64)]
+               [("max_segs_per_block", C.c_int64), ("frames_deleted", C.c_int64)]
 
 
 class EpochIO(C.Structure):
@@ -51,6 +51,12 @@ class EpochIO(C.Structure):
                 ("d_seq_id", C.c_void_p), ("d_pos", C.c_void_p), ("d_reset", C.c_void_p), ("d_valid", C.c_void_p),
                 ("d_dense_out", C.c_void_p), ("out_frame_bytes", C.c_int64), ("d_ragged_out", C.c_void_p),
                 ("block_capacity", C.c_int64), ("pad_byte", C.c_uint8), ("chunks", C.c_uint8), ("reserved_", C.c_uint8 * 6)]
+
+
+class ChunkInfo(C.Structure):
+    _fields_ = [("status", C.c_int32), ("tail", C.c_uint32), ("t_chunk", C.c_int32), ("reserved_", C.c_int32)] + \
+               [(k, C.c_int64) for k in ("n", "n_chunks", "frames_kept", "frames_deleted", "pad_frames", "sum_t", "t_max",
+                                          "first_bad_index")]
 
 
 class VarInfo(C.Structure):
@@ -91,6 +97,9 @@ def load() -> C.CDLL:
     L.bload_plan_sizes.argtypes = [i64, i32, C.POINTER(Sizes)]
     L.bload_plan.argtypes = [vp, i64, i32, u64, u32, vp, C.c_size_t, vp, C.c_size_t, vp, C.POINTER(PlanInfo)]
     L.bload_plan_async.argtypes = [vp, i64, i32, u64, u32, vp, C.c_size_t, vp, C.c_size_t, vp]
+    L.bload_chunk_work_bytes.argtypes = [i64]
+    L.bload_chunk_count.argtypes = [vp, i64, i32, u32, vp, C.c_size_t, vp, C.POINTER(ChunkInfo)]
+    L.bload_plan_chunks.argtypes = [vp, i64, i32, u32, i64, vp, C.c_size_t, vp, C.c_size_t, vp, vp, vp, C.POINTER(PlanInfo)]
     L.bload_plan_static.argtypes = [vp, i64, i32, u64, u32, vp, C.c_size_t, vp, C.POINTER(PlanInfo)]
     L.bload_plan_finish.argtypes = [vp, vp, C.POINTER(PlanInfo)]
     L.bload_rank_range.argtypes = [i64, i32, i32, i32, C.POINTER(i64), C.POINTER(i64)]
@@ -115,12 +124,14 @@ def load() -> C.CDLL:
     L.bload_strerror.argtypes = [C.c_int]
     L.bload_strerror.restype = C.c_char_p
     L.bload_last_copy_kernel.argtypes = [C.c_int]
+    L.bload_debug_status.argtypes = [C.POINTER(C.c_uint64 * 4), C.c_int]
     L.bload_version.argtypes = []
     L.bload_kernel_launches.argtypes = []
     for name in EXPORTS:
-        if name not in ("bload_strerror", "bload_kernel_launches", "bload_last_copy_kernel"):
+        if name not in ("bload_strerror", "bload_kernel_launches", "bload_last_copy_kernel", "bload_debug_status", "bload_chunk_work_bytes"):
             getattr(L, name).restype = C.c_int
     L.bload_kernel_launches.restype = C.c_int64
+    L.bload_chunk_work_bytes.restype = C.c_size_t
     L.bload_last_copy_kernel.restype = C.c_char_p
     _lib = L
     return L
@@ -412,6 +423,59 @@ def bload_plan_stage_times() -> list[float]:
 
 def bload_kernel_launches() -> int:
     return int(load().bload_kernel_launches())
+
+
+def bload_debug_status(clear: bool = False):
+    """[refused accesses, kernel number of the first, 0 read / 1 write, address] of the bounds-checking build
+    (BLOAD_LIBRARY=.../libbload_debug.so); None from the ordinary build."""
+    out = (C.c_uint64 * 4)()
+    rc = load().bload_debug_status(C.byref(out), 1 if clear else 0)
+    if rc == ERR_UNSUPPORTED:
+        return None
+    if rc:
+        raise BloadError(rc, "bload_debug_status")
+    return [int(x) for x in out]
+
+
+KEEP_TAIL, DROP_TAIL = 0, 1
+
+
+def bload_plan_chunks(lengths, t_chunk: int, tail: int = KEEP_TAIL, stream=None, check: bool = True):
+    """The chunking strategy of the paper's comparison ("sampling"): every chunk of t_chunk frames of every sequence is a
+    sample and a block.  Returns (Plan over the chunks, ChunkInfo, chunk_seq, chunk_first); the two int32 CUDA tensors
+    name, per chunk, the sequence it was cut from and its first frame there.  Two calls into the library: the count
+    (the plan cannot be sized before it), then the plan."""
+    import torch
+    if not lengths.is_cuda or lengths.dtype != torch.int32 or not lengths.is_contiguous():
+        raise TypeError("lengths must be a contiguous CUDA int32 tensor")
+    n = lengths.numel()
+    L = load()
+    work = torch.empty(max(int(L.bload_chunk_work_bytes(n)), 256), dtype=torch.uint8, device=lengths.device)
+    ci = ChunkInfo()
+    rc = L.bload_chunk_count(lengths.data_ptr(), n, t_chunk, tail, work.data_ptr(), work.numel(), _stream(stream), C.byref(ci))
+    if rc:
+        err = BloadError(rc, "bload_chunk_count")
+        err.info = ci
+        if check:
+            raise err
+        return None, ci, None, None
+    m = int(ci.n_chunks)
+    if m < 1:
+        if check:
+            raise BloadError(ERR_ARG, "bload_plan_chunks (no chunk is kept)")
+        return None, ci, None, None
+    sizes = bload_plan_sizes(m, t_chunk)
+    plan_buf = torch.empty(sizes.plan_bytes, dtype=torch.uint8, device=lengths.device)
+    chunk_seq = torch.empty(m, dtype=torch.int32, device=lengths.device)
+    chunk_first = torch.empty(m, dtype=torch.int32, device=lengths.device)
+    info = PlanInfo()
+    rc = L.bload_plan_chunks(lengths.data_ptr(), n, t_chunk, tail, m, plan_buf.data_ptr(), plan_buf.numel(), work.data_ptr(),
+                             work.numel(), chunk_seq.data_ptr(), chunk_first.data_ptr(), _stream(stream), C.byref(info))
+    if rc and check:
+        err = BloadError(rc, "bload_plan_chunks")
+        err.info = info
+        raise err
+    return Plan(plan_buf, info, sizes), ci, chunk_seq, chunk_first
 
 
 COPY_CALLS = {"pack": 0, "unpack": 1, "carry_prev": 2, "pack_var": 3, "unpack_var": 4}

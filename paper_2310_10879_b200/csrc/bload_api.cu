@@ -5,9 +5,22 @@
 #include <mutex>
 #include <vector>
 
+#include "bload_debug.cuh"
 #include "bload_internal.cuh"
 
 namespace bload {
+
+#ifdef BLOAD_DEBUG
+namespace dbg {
+// every translation unit that holds checked kernels adds its reader here (during static initialisation)
+static std::vector<void (*)(unsigned long long[4], bool)>& collectors()
+{
+    static std::vector<void (*)(unsigned long long[4], bool)> v;
+    return v;
+}
+void register_collector(void (*fn)(unsigned long long[4], bool)) { collectors().push_back(fn); }
+}  // namespace dbg
+#endif
 
 void plan_layout(int64_t n, bload_sizes_t* s)
 {
@@ -171,6 +184,22 @@ extern "C" {
 int bload_version(void) { return 1; }
 
 int64_t bload_kernel_launches(void) { return (int64_t)g_launches.load(std::memory_order_relaxed); }
+
+int bload_debug_status(uint64_t out[4], int clear)
+{
+    if (!out) return BLOAD_ERR_NULL;
+    out[0] = out[1] = out[2] = out[3] = 0;
+#ifdef BLOAD_DEBUG
+    if (cudaDeviceSynchronize() != cudaSuccess) { (void)cudaGetLastError(); return BLOAD_ERR_CUDA; }
+    unsigned long long s[4] = {0, 0, 0, 0};
+    for (auto fn : dbg::collectors()) fn(s, clear != 0);
+    for (int i = 0; i < 4; ++i) out[i] = s[i];
+    return BLOAD_OK;
+#else
+    (void)clear;
+    return BLOAD_ERR_UNSUPPORTED;
+#endif
+}
 
 const char* bload_last_copy_kernel(int which)
 {
@@ -535,7 +564,7 @@ int bload_unpack(const void* d_plan, const bload_plan_info_t* info, const void* 
     cudaError_t ce = launch_copy(true, pv, info->t_block, out_frame_bytes, block_begin, block_count, nullptr,
                                  const_cast<uint8_t*>(static_cast<const uint8_t*>(d_dense_out)),
                                  static_cast<uint8_t*>(d_ragged_out), info->sum_t * out_frame_bytes, 0, st, info->n,
-                                 info->n_blocks);
+                                 info->n_blocks, info->policy == BLOAD_POLICY_CHUNKS_DROP_TAIL);
     if (ce != cudaSuccess) { (void)cudaGetLastError(); return BLOAD_ERR_CUDA; }
     return BLOAD_OK;
 }
@@ -579,6 +608,7 @@ int copy_var(bool unpack, const void* d_plan, const bload_plan_info_t* info, con
 {
     int rc = check_plan_args(d_plan, info, row_stride, block_begin, block_count);
     if (rc) return rc;
+    if (info->policy >= BLOAD_POLICY_CHUNKS_KEEP_TAIL) return BLOAD_ERR_UNSUPPORTED;  // sizes are per sequence, chunks are not sequences
     if (rows_max < 1 || rows_max > 0x7fffffffLL) return BLOAD_ERR_ARG;
     if (block_count == 0) return BLOAD_OK;
     if (!d_src || !d_dst || !d_row_bytes || !d_byte_offsets) return BLOAD_ERR_NULL;
@@ -702,7 +732,10 @@ int bload_stats(const bload_plan_info_t* info, bload_stats_t* out)
     memset(out, 0, sizeof *out);
     if (info->status != BLOAD_OK || info->n < 1 || info->t_block < 1 || info->n_blocks < 1 || info->sum_t < 1)
         return BLOAD_ERR_PLAN;
-    const int64_t n = info->n, s = info->sum_t, tb = info->t_block, nb = info->n_blocks, tm = info->t_max;
+    const int64_t n = info->n, tb = info->t_block, nb = info->n_blocks, tm = info->t_max;
+    // frames that sit in blocks: all of the store, except under the chunking strategy that keeps only full chunks
+    const int64_t s = info->policy == BLOAD_POLICY_CHUNKS_DROP_TAIL ? nb * tb : info->sum_t;
+    out->frames_deleted = info->sum_t - s;
     out->n = n; out->sum_t = s; out->t_max = tm; out->t_block = tb; out->n_blocks = nb;
     out->pad_packed = nb * tb - s;
     out->pad_naive_tmax = n * tm - s;

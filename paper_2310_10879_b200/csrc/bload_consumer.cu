@@ -119,9 +119,9 @@ __global__ void __launch_bounds__(256, 3) k11_carry_shift(PlanView pv, int32_t t
             }
             if (frame_bytes <= 64) {
                 if (((a | e | reinterpret_cast<uintptr_t>(out)) & 3) == 0)
-                    for (int64_t x = a; x < e; x += 4) *reinterpret_cast<uint32_t*>(out + x) = f4;
+                    for (int64_t x = a; x < e; x += 4) put_word(out + x, f4);
                 else
-                    for (int64_t x = a; x < e; ++x) out[x] = fill_byte;
+                    for (int64_t x = a; x < e; ++x) put_byte(out + x, fill_byte);
             } else {
                 const unsigned live = __ballot_sync(kFull, a < e);
                 for (unsigned m = live; m; m &= m - 1) {
@@ -280,6 +280,7 @@ cudaError_t launch_carry_prev(const PlanView& pv, int32_t t_block, int64_t frame
     const int64_t sub = 16384;
     const int64_t spb = (block_bytes + sub - 1) / sub;
     count_launches(1);
+    BLOAD_DBG_EXPECT(st, dbg::kCarry, {{dense, (size_t)(block_count * block_bytes)}}, {{prev, (size_t)(block_count * block_bytes)}});
     // short runs (many segments per sub-tile): one shifted copy per sub-tile and patches at the segment starts
     if (n > 0 && sum_t * frame_bytes / n <= 16384) {
         note_copy_kernel(kCallCarryPrev, "k11_carry_shift");
@@ -300,6 +301,7 @@ cudaError_t launch_reset_state(const PlanView& pv, int64_t block_begin, int64_t 
     const int64_t sub = 16384;
     const int64_t spr = (state_bytes + sub - 1) / sub;
     count_launches(1);
+    BLOAD_DBG_EXPECT(st, dbg::kResetState, {{init, (size_t)state_bytes}}, {{state, (size_t)(block_count * state_bytes)}});
     k12_reset_state<<<grid_for_items(block_count * spr), 256, 0, st>>>(pv, block_begin, block_count, slot, state, state_bytes,
                                                                       init, sub, spr);
     return cudaPeekAtLastError();
@@ -313,6 +315,7 @@ cudaError_t launch_repeat_last(const PlanView& pv, int32_t t_block, int64_t fram
     const int64_t sub = 16384;
     const int64_t spb = (block_bytes + sub - 1) / sub;
     count_launches(1);
+    BLOAD_DBG_EXPECT(st, dbg::kRepeatLast, {{dense, (size_t)(block_count * block_bytes)}}, {{dense, (size_t)(block_count * block_bytes)}});
     k14_repeat_last<<<grid_for_items(block_count * spb), 256, 0, st>>>(pv, t_block, frame_bytes, block_begin, block_count,
                                                                       dense, sub, spb);
     return cudaPeekAtLastError();

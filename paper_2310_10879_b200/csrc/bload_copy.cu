@@ -144,10 +144,12 @@ constexpr int64_t kPackChunkTiles = BLOAD_PACK_CHUNK_TILES;  // consecutive sub-
 __device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 __device__ __forceinline__ void cp_async4(uint32_t s, const void* g)
 {
+    if (!BLOAD_MAY_READ(g, 4)) return;
     asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(s), "l"(g) : "memory");
 }
 __device__ __forceinline__ void cp_async16(uint32_t s, const void* g)
 {
+    if (!BLOAD_MAY_READ(g, 16)) return;
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(s), "l"(g) : "memory");
 }
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
@@ -156,6 +158,7 @@ __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_gr
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void bulk_store(void* g, uint32_t s, uint32_t bytes)
 {
+    if (!BLOAD_MAY_WRITE(g, bytes)) return;
     asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(g), "r"(s), "r"(bytes) : "memory");
 }
 __device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
@@ -164,6 +167,7 @@ __device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.w
 
 // four copies of `sz` bytes, 32 lanes apart, with immediate offsets
 #define BLOAD_CP4X(op, sz, s, g, st)                                                                                \
+    if (BLOAD_MAY_READ(g, sz) && BLOAD_MAY_READ((g) + 3 * st, sz))                                                  \
     asm volatile(op " [%0], [%1], " #sz ";\n\t" op " [%0+" #st "], [%1+" #st "], " #sz ";\n\t"                       \
                  op " [%0+2*" #st "], [%1+2*" #st "], " #sz ";\n\t" op " [%0+3*" #st "], [%1+3*" #st "], " #sz ";"   \
                  ::"r"(s), "l"(g) : "memory")
@@ -216,7 +220,7 @@ __device__ __forceinline__ void warp_scatter(uint8_t* __restrict__ gd, const uin
 {
     int hw = (int)(((16u - (unsigned)(reinterpret_cast<uintptr_t>(gd) & 15u)) & 15u) >> 2);
     if (hw * 4 > n) hw = n >> 2;
-    if (lane < hw) reinterpret_cast<uint32_t*>(gd)[lane] = reinterpret_cast<const uint32_t*>(ss)[lane];
+    if (lane < hw) put_word(gd + 4 * lane, reinterpret_cast<const uint32_t*>(ss)[lane]);
     gd += 4 * hw; ss += 4 * hw; n -= 4 * hw;
     const int nv = n >> 4;
     uint4* d = reinterpret_cast<uint4*>(gd);
@@ -229,7 +233,7 @@ __device__ __forceinline__ void warp_scatter(uint8_t* __restrict__ gd, const uin
         default: scatter_vectors<3>(d, a, nv, lane); break;
     }
     const int tw = (n - (nv << 4)) >> 2;
-    if (lane < tw) reinterpret_cast<uint32_t*>(gd + (nv << 4))[lane] = reinterpret_cast<const uint32_t*>(ss + (nv << 4))[lane];
+    if (lane < tw) put_word(gd + (nv << 4) + 4 * lane, reinterpret_cast<const uint32_t*>(ss + (nv << 4))[lane]);
 }
 
 // What a warp has to remember about a sub-tile between its two phases.
@@ -431,7 +435,7 @@ __global__ void __launch_bounds__(StageCfg<false>::kWarps * 32) k9_unpack_ragged
         __syncwarp();
         const int n16 = nbytes & ~15;
         if (lane == 0 && n16) { bulk_store(ragged + lo, smem_addr(stage), (uint32_t)n16); bulk_commit(); }
-        if (lane < nbytes - n16) ragged[lo + n16 + lane] = stage[n16 + lane];  // last tile only: total % 16 bytes
+        if (lane < nbytes - n16) put_byte(ragged + lo + n16 + lane, stage[n16 + lane]);  // last tile only: total % 16 bytes
     };
     for (int64_t t = t_begin; t < t_end; ++t) {
         uint8_t* stage = my_stages + (size_t)s * kStageBytes;
@@ -624,6 +628,11 @@ bool staged_pack_with_metadata(const PlanView& pv, int32_t t_block, int64_t fram
     mo.vec = t_block % 4 == 0 && al(seq_id, 16) && al(pos, 16) && al(reset, 4) && al(valid, 4);
     const int64_t grid = (int64_t)mo.pack_ctas + block_count * mo.chunks_per_block;
     count_launches(1);
+    {
+        const size_t slots = (size_t)block_count * (size_t)t_block;
+        BLOAD_DBG_EXPECT(st, dbg::kPackContig, {{store, (size_t)ragged_bytes}},
+                         {{dense, (size_t)(block_count * block_bytes)}, {seq_id, 4 * slots}, {pos, 4 * slots}, {reset, slots}, {valid, slots}});
+    }
     note_copy_kernel(kCallPack, "k10_pack_contig<metadata>");
     k10_pack_contig<true><<<(unsigned)grid, Cfg::kWarps * 32, smem, st>>>(pv, (int32_t)n, t_block, frame_bytes, block_begin, store,
                                                                         dense, tiles, tpw, (int32_t)spb, pad_byte, mo);
@@ -633,11 +642,13 @@ bool staged_pack_with_metadata(const PlanView& pv, int32_t t_block, int64_t fram
 
 cudaError_t launch_copy(bool unpack, const PlanView& pv, int32_t t_block, int64_t frame_bytes, int64_t block_begin,
                         int64_t block_count, const uint8_t* ragged_in, uint8_t* dense, uint8_t* ragged_out,
-                        int64_t ragged_bytes, uint8_t pad_byte, cudaStream_t st, int64_t n, int64_t n_blocks)
+                        int64_t ragged_bytes, uint8_t pad_byte, cudaStream_t st, int64_t n, int64_t n_blocks, bool gaps)
 {
     if (block_count == 0) return cudaSuccess;
     const int64_t block_bytes = (int64_t)t_block * frame_bytes;
     count_launches(1);
+    if (unpack) BLOAD_DBG_EXPECT(st, dbg::kCopy, {{dense, (size_t)(block_count * block_bytes)}}, {{ragged_out, (size_t)ragged_bytes}});
+    else BLOAD_DBG_EXPECT(st, dbg::kCopy, {{ragged_in, (size_t)ragged_bytes}}, {{dense, (size_t)(block_count * block_bytes)}});
     // pack of small word-sized frames: contiguous ranges of dense sub-tiles per warp
     const bool short_runs = frame_bytes % 4 == 0 && n > 0 && ragged_bytes / n <= kStagedMaxRunBytes && block_bytes < (1LL << 31);
     if (!unpack && short_runs && block_bytes % 16 == 0) {
@@ -661,7 +672,8 @@ cudaError_t launch_copy(bool unpack, const PlanView& pv, int32_t t_block, int64_
         return cudaPeekAtLastError();
     }
     // whole-plan unpack of small word-sized frames: tile the (contiguous, fully written) ragged side
-    if (unpack && short_runs && block_begin == 0 && block_count >= n_blocks && ragged_bytes > 0) {
+    // (not when frames between the plan's sequences belong to nobody: this path writes the whole ragged buffer)
+    if (unpack && short_runs && !gaps && block_begin == 0 && block_count >= n_blocks && ragged_bytes > 0) {
         using Cfg = StageCfg<false>;
         const size_t smem = (size_t)Cfg::kWarps * Cfg::kStages * Cfg::kBytes + 16;
         const DeviceInfo di = device_info();
@@ -732,6 +744,7 @@ cudaError_t launch_copy_range(bool unpack, const PlanView& pv, int32_t t_block, 
     // starts as soon as any CTA of this launch retires; a chunk holds some thousand sub-tiles, about one per warp
     const unsigned grid = (unsigned)device_info().sm_count * 3 * 16;  // (2 to 32 rounds of resident CTAs measured alike)
     count_launches(1);
+    BLOAD_DBG_UNCHECKED(st);  // runs beside launches of another stream, on a block range only the device knows
     if (unpack)
         k7_copy<true><<<grid, 256, kBesideChainSmemBytes, st>>>(pv, t_block, frame_bytes, 0, 0, src, dst, src_total_bytes, sub, spb,
                                                                 pad_byte, d_range, 0);

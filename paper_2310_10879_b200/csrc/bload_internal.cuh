@@ -140,7 +140,8 @@ cudaError_t launch_metadata(const PlanView& pv, int32_t t_block, int64_t block_b
                             const int32_t* d_range = nullptr);
 cudaError_t launch_copy(bool unpack, const PlanView& pv, int32_t t_block, int64_t frame_bytes, int64_t block_begin,
                         int64_t block_count, const uint8_t* ragged_in, uint8_t* dense, uint8_t* ragged_out,
-                        int64_t ragged_bytes, uint8_t pad_byte, cudaStream_t st, int64_t n, int64_t n_blocks);
+                        int64_t ragged_bytes, uint8_t pad_byte, cudaStream_t st, int64_t n, int64_t n_blocks,
+                        bool gaps = false /*the plan's sequences do not tile the ragged buffer (chunks with deleted frames)*/);
 // The pieces of the planner and the copies that bload_epoch strings together on two streams.  `d_range` points to
 // {first block, end block, end of the real blocks} in device memory: the blocks a launch covers are decided on the
 // device, so these launches use fixed grids whose CTAs loop.

@@ -50,6 +50,12 @@ cudaError_t launch_metadata(const PlanView& pv, int32_t t_block, int64_t block_b
     if (rows > 65535) rows = 65535;
     const dim3 grid(chunks, (unsigned)rows);
     const size_t smem = d_range ? kBesideChainSmemBytes : 0;  // beside a running fill rule: stay off its SM
+    if (d_range) {
+        BLOAD_DBG_UNCHECKED(st);
+    } else {
+        const size_t slots = (size_t)block_count * (size_t)t_block;
+        BLOAD_DBG_EXPECT(st, dbg::kMetadata, {}, {{seq_id, 4 * slots}, {pos, 4 * slots}, {reset, slots}, {valid, slots}});
+    }
     if (t_block % 4 == 0 && al(seq_id, 16) && al(pos, 16) && al(reset, 4) && al(valid, 4))
         k6_metadata<true><<<grid, kMetaThreads, smem, st>>>(pv, t_block, block_begin, (int32_t)block_count, seq_id, pos, reset, valid, d_range);
     else

@@ -1,6 +1,7 @@
 // Per-slot metadata of four consecutive slots of one block, shared by the metadata kernel and by the pack kernel that
 // writes metadata from some of its CTAs.  Device code only.
 #pragma once
+#include "bload_debug.cuh"
 #include "bload_internal.cuh"
 
 namespace bload {
@@ -58,18 +59,18 @@ __device__ __forceinline__ void metadata_quad(const PlanView& pv, int32_t t_bloc
         }
     }
     if (VEC) {  // t_block % 4 == 0 and aligned outputs: one vector per array
-        if (seq_id) __stcs(reinterpret_cast<int4*>(seq_id + o), make_int4(sid[0], sid[1], sid[2], sid[3]));
-        if (pos) __stcs(reinterpret_cast<int4*>(pos + o), make_int4(ps[0], ps[1], ps[2], ps[3]));
-        if (reset) __stcs(reinterpret_cast<unsigned*>(reset + o), rs);
-        if (valid) __stcs(reinterpret_cast<unsigned*>(valid + o), vd);
+        if (seq_id && BLOAD_MAY_WRITE(seq_id + o, 16)) __stcs(reinterpret_cast<int4*>(seq_id + o), make_int4(sid[0], sid[1], sid[2], sid[3]));
+        if (pos && BLOAD_MAY_WRITE(pos + o, 16)) __stcs(reinterpret_cast<int4*>(pos + o), make_int4(ps[0], ps[1], ps[2], ps[3]));
+        if (reset && BLOAD_MAY_WRITE(reset + o, 4)) __stcs(reinterpret_cast<unsigned*>(reset + o), rs);
+        if (valid && BLOAD_MAY_WRITE(valid + o, 4)) __stcs(reinterpret_cast<unsigned*>(valid + o), vd);
     } else {
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
             if (s0 + e < t_block) {
-                if (seq_id) seq_id[o + e] = sid[e];
-                if (pos) pos[o + e] = ps[e];
-                if (reset) reset[o + e] = (uint8_t)((rs >> (8 * e)) & 1u);
-                if (valid) valid[o + e] = (uint8_t)((vd >> (8 * e)) & 1u);
+                if (seq_id && BLOAD_MAY_WRITE(seq_id + o + e, 4)) seq_id[o + e] = sid[e];
+                if (pos && BLOAD_MAY_WRITE(pos + o + e, 4)) pos[o + e] = ps[e];
+                if (reset && BLOAD_MAY_WRITE(reset + o + e, 1)) reset[o + e] = (uint8_t)((rs >> (8 * e)) & 1u);
+                if (valid && BLOAD_MAY_WRITE(valid + o + e, 1)) valid[o + e] = (uint8_t)((vd >> (8 * e)) & 1u);
             }
         }
     }

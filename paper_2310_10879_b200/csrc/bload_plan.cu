@@ -12,6 +12,7 @@
 //   4. a parallel pass that resolves draws to sequence ids and writes the inverse tables.
 #include <limits.h>
 
+#include "bload_debug.cuh"
 #include "bload_internal.cuh"
 
 namespace bload {
@@ -597,8 +598,14 @@ __global__ void __launch_bounds__(256) k5_tables(PlanView pv, const int4* __rest
     unsigned long long term = 0;
     int segs = 0;
     for (int64_t k = k_lo + (int64_t)blockIdx.x * 256 + threadIdx.x; k < k_hi; k += (int64_t)gridDim.x * 256) {
+        if (!BLOAD_MAY_READ(draw_rec + k, 16)) continue;
         int4 r = draw_rec[k];
+        if (!BLOAD_MAY_READ(bucket_end + r.x, 4) || !BLOAD_MAY_READ(sorted_id + (bucket_end[r.x] - r.y), 4)) continue;
         int id = sorted_id[bucket_end[r.x] - r.y];
+        if (!(BLOAD_MAY_WRITE(pv.seg_seq + k, 4) && BLOAD_MAY_WRITE(pv.seg_block + k, 4) && BLOAD_MAY_WRITE(pv.seg_start + k, 4) &&
+              BLOAD_MAY_WRITE(pv.seg_src + k, 8) && BLOAD_MAY_READ(pv.offsets + id, 8) && BLOAD_MAY_WRITE(pv.seq_block + id, 4) &&
+              BLOAD_MAY_WRITE(pv.seq_start + id, 4)))
+            continue;
         pv.seg_seq[k] = id;
         pv.seg_block[k] = r.z;
         pv.seg_start[k] = r.w;
@@ -759,8 +766,9 @@ cudaError_t launch_fill_chunk(const PlanView& pv, const WorkView& wv, const Epoc
 cudaError_t launch_tables_chunk(const PlanView& pv, const WorkView& wv, const int32_t* sorted_id, int64_t n,
                                 const int32_t* d_draw_range, cudaStream_t st)
 {
-    const int64_t want = (n + 255) / 256;
-    k5_tables<<<(unsigned)(want < 592 ? want : 592), 256, kBesideChainSmemBytes, st>>>(pv, wv.draw_rec, wv.bucket_end, sorted_id, n,
+    const int64_t want = (n + 255) / 256, cap = (int64_t)device_info().sm_count * 4;
+    BLOAD_DBG_UNCHECKED(st);  // runs beside launches of another stream
+    k5_tables<<<(unsigned)(want < cap ? want : cap), 256, kBesideChainSmemBytes, st>>>(pv, wv.draw_rec, wv.bucket_end, sorted_id, n,
                                                                                         d_draw_range);
     count_launches(1);
     return cudaPeekAtLastError();
@@ -797,6 +805,12 @@ cudaError_t launch_plan(const int32_t* d_lengths, int64_t n, int32_t t_block, ui
     }
     if (ev) cudaEventRecord(ev[3], st);
 
+    {   // the table kernel may touch the plan buffer and the scratch buffer, nothing else
+        bload_sizes_t sz;
+        plan_layout(n, &sz);
+        const size_t work_bytes = work_layout(n, t_block, nullptr, nullptr);
+        BLOAD_DBG_EXPECT(st, dbg::kTables, {{pv.hdr, sz.plan_bytes}, {wv.key_a, work_bytes}}, {{pv.hdr, sz.plan_bytes}});
+    }
     k5_tables<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(pv, wv.draw_rec, wv.bucket_end, iin, n, nullptr);
     k5_finish<<<1, 32, 0, st>>>(pv.hdr);
     count_launches(1 + 2);

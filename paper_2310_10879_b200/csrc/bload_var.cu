@@ -93,8 +93,12 @@ __device__ __forceinline__ uint32_t fast_div(uint32_t n, const FastDiv& f)
 // per-sequence frame size).  The dense side is walked row by row of the canvases ("sub-slots" of row_stride
 // bytes).  Row counts and row sizes are clamped to the canvas on the device, so a caller that breaks the documented
 // precondition gets truncated images but never an access outside the buffers.
+// Four CTAs per SM: with more registers per thread (two CTAs) the kernel was measured at 5.7 / 5.2 TB/s (pack / unpack,
+// frame sizes of 1 to 4 KB in 4 KB slots) with 21 % of the warp slots in use and its warps waiting on loads; capped at
+// 64 registers it reaches 6.3 / 6.2 TB/s, the few spills sit in the unaligned fallback path.  (3 CTAs and 8 vectors in
+// flight per lane: 6.4 / 5.9.)
 #ifndef BLOAD_VAR_MIN_CTAS
-#define BLOAD_VAR_MIN_CTAS 2
+#define BLOAD_VAR_MIN_CTAS 4
 #endif
 #ifndef BLOAD_VAR_UNROLL
 #define BLOAD_VAR_UNROLL 4
@@ -278,6 +282,17 @@ cudaError_t launch_copy_var(bool unpack, const PlanView& pv, int32_t t_block, in
     const FastDiv div_vpr = make_div((uint32_t)(row_stride >= 16 && row_stride / 16 < 0x7fffffffLL ? row_stride / 16 : 1));
     const FastDiv div_rows = make_div((uint32_t)rows_max);
     count_launches(1);
+#ifdef BLOAD_DEBUG
+    {   // the size of the store is the last entry of the offsets on the device: the checking build may wait for it
+        int64_t n = 0, total = 0;
+        (void)cudaStreamSynchronize(st);
+        (void)cudaMemcpy(&n, &pv.hdr->n, sizeof n, cudaMemcpyDeviceToHost);
+        (void)cudaMemcpy(&total, byte_offsets + n, sizeof total, cudaMemcpyDeviceToHost);
+        const size_t dense_bytes = (size_t)(block_count * block_bytes);
+        if (unpack) BLOAD_DBG_EXPECT(st, dbg::kCopyVar, {{src, dense_bytes}}, {{dst, (size_t)total}});
+        else BLOAD_DBG_EXPECT(st, dbg::kCopyVar, {{src, (size_t)total}}, {{dst, dense_bytes}});
+    }
+#endif
     note_copy_kernel(unpack ? kCallUnpackVar : kCallPackVar, unpack ? "k16_copy_var<unpack>" : "k16_copy_var<pack>");
     if (unpack)
         k16_copy_var<true><<<grid, 256, 0, st>>>(pv, t_block, rows_max, row_stride, block_begin, block_count, seq_rows,

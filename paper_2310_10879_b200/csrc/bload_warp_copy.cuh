@@ -5,13 +5,20 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include "bload_debug.cuh"
+
 namespace bload {
 namespace wc {
 
 constexpr unsigned kFull = 0xffffffffu;
 
-__device__ __forceinline__ uint4 ld_stream(const uint4* p) { return __ldcs(p); }
-__device__ __forceinline__ void st_stream(uint4* p, uint4 v) { __stcs(p, v); }
+// Every data access goes through these few functions; in a bounds-checking build (bload_debug.cuh) each asks first
+// whether its address lies in a range the launcher registered, and a refused access is skipped.
+__device__ __forceinline__ uint4 ld_stream(const uint4* p) { return BLOAD_MAY_READ(p, 16) ? __ldcs(p) : make_uint4(0, 0, 0, 0); }
+__device__ __forceinline__ void st_stream(uint4* p, uint4 v) { if (BLOAD_MAY_WRITE(p, 16)) __stcs(p, v); }
+__device__ __forceinline__ void copy_byte(uint8_t* d, const uint8_t* s) { if (BLOAD_MAY_READ(s, 1) && BLOAD_MAY_WRITE(d, 1)) *d = *s; }
+__device__ __forceinline__ void put_byte(uint8_t* d, uint8_t v) { if (BLOAD_MAY_WRITE(d, 1)) *d = v; }
+__device__ __forceinline__ void put_word(uint8_t* d, uint32_t v) { if (BLOAD_MAY_WRITE(d, 4)) *reinterpret_cast<uint32_t*>(d) = v; }
 
 template <int U>
 __device__ __forceinline__ void warp_copy_aligned(uint4* __restrict__ d, const uint4* __restrict__ s, int64_t nv, int lane)
@@ -44,7 +51,11 @@ __device__ __forceinline__ uint4 splice(uint4 a, uint4 b, int bits)
 // sectors.  Measured on B200 with 64..1028-byte frames: letting them allocate in L1 helps when the source is
 // the dense side (unpack, +3..6 %) and costs when it is the ragged store (pack, -3..5 %), so the direction chooses.
 template <bool CACHED>
-__device__ __forceinline__ uint4 ld_shared_sector(const uint4* p) { return CACHED ? __ldg(p) : __ldcs(p); }
+__device__ __forceinline__ uint4 ld_shared_sector(const uint4* p)
+{
+    if (!BLOAD_MAY_READ(p, 16)) return make_uint4(0, 0, 0, 0);
+    return CACHED ? __ldg(p) : __ldcs(p);
+}
 
 template <int WS, int U, bool CACHED>
 __device__ __forceinline__ void warp_copy_shifted(uint4* __restrict__ d, const uint4* __restrict__ a, int64_t nv, int bits, int lane)
@@ -67,7 +78,7 @@ __device__ __forceinline__ void warp_copy(uint8_t* __restrict__ d, const uint8_t
 {
     int head = (int)((16u - (unsigned)(reinterpret_cast<uintptr_t>(d) & 15u)) & 15u);
     if ((int64_t)head > n) head = (int)n;
-    if (lane < head) d[lane] = s[lane];
+    if (lane < head) copy_byte(d + lane, s + lane);
     d += head; s += head; n -= head;
     int64_t nv = n >> 4;
     const int sh = (int)(reinterpret_cast<uintptr_t>(s) & 15u);
@@ -87,21 +98,21 @@ __device__ __forceinline__ void warp_copy(uint8_t* __restrict__ d, const uint8_t
             default: warp_copy_shifted<3, 4, CACHED>(dv, av, nv, bits, lane); break;
         }
     }
-    for (int64_t t = (nv << 4) + lane; t < n; t += 32) d[t] = s[t];
+    for (int64_t t = (nv << 4) + lane; t < n; t += 32) copy_byte(d + t, s + t);
 }
 
 __device__ __forceinline__ void warp_fill(uint8_t* __restrict__ d, int64_t n, uint8_t pad, int lane)
 {
     int head = (int)((16u - (unsigned)(reinterpret_cast<uintptr_t>(d) & 15u)) & 15u);
     if ((int64_t)head > n) head = (int)n;
-    if (lane < head) d[lane] = pad;
+    if (lane < head) put_byte(d + lane, pad);
     d += head; n -= head;
     const int64_t nv = n >> 4;
     const uint32_t p4 = 0x01010101u * pad;
     const uint4 v = make_uint4(p4, p4, p4, p4);
     uint4* dv = reinterpret_cast<uint4*>(d);
     for (int64_t i = lane; i < nv; i += 32) st_stream(dv + i, v);
-    for (int64_t t = (nv << 4) + lane; t < n; t += 32) d[t] = pad;
+    for (int64_t t = (nv << 4) + lane; t < n; t += 32) put_byte(d + t, pad);
 }
 
 // Largest k in [k0, k1) with seg_start[k] <= slot (seg_start[k0] == 0 <= slot always holds).

@@ -20,7 +20,7 @@ def host_tables(plan) -> dict:
     return {k: v.cpu().numpy() for k, v in plan.tables().items()}
 
 
-def assert_plan_equal(plan, op, maximal=None):
+def assert_plan_equal(plan, op, maximal=None, invariants_too=True):
     """GPU plan vs oracle plan: every table and scalar, bit exact; plus the validity checker."""
     i = plan.info
     assert i.status == 0 and op.status == 0
@@ -36,6 +36,8 @@ def assert_plan_equal(plan, op, maximal=None):
             raise AssertionError("%s differs first at %d: gpu %s oracle %s" % (name, bad, a[bad], b[bad]))
     assert np.array_equal(t["seg_src"], op.offsets[op.seg_seq.astype(np.int64)])
     assert i.checksum == op.checksum and i.max_segs_per_block == op.max_segs_per_block
+    if not invariants_too:                 # e.g. chunks with deleted frames: the "sequences" do not tile the store
+        return
     if maximal is None:
         maximal = i.policy != 2            # best fit decreasing keeps several blocks open
     invariants.check_plan(op.lengths, i.t_block, i.n_blocks, t["offsets"], t["seg_seq"], t["seg_block"],

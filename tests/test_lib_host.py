@@ -32,6 +32,13 @@ def test_library_exports_every_declared_symbol():
     assert B.strerror(0) == "ok" and "length" in B.strerror(_lib.ERR_LENGTH)
 
 
+def test_bounds_checking_build_compiles_and_exports_the_same_symbols():
+    from paper_2310_10879_b200 import build
+    L = C.CDLL(build.build(debug=True))
+    for n in _declared():
+        assert hasattr(L, n), n
+
+
 def test_plan_sizes_layout():
     for n, tb in [(1, 1), (8, 6), (1000, 1000), (1_000_000, 4096), (20_000, 10_000)]:
         s = B.bload_plan_sizes(n, tb)

@@ -37,8 +37,11 @@ def _same_plan(a, b):
 
 
 def _memory_state():
-    """What an allocation anywhere would change: torch's allocator counters and the driver's free bytes."""
-    return (torch.cuda.memory_allocated(DEV), torch.cuda.memory_reserved(DEV), torch.cuda.mem_get_info(DEV)[0])
+    """What an allocation anywhere would change: the number of blocks torch's allocator has ever handed out, the number
+    of segments it has ever taken from the driver (both only grow; tensors of earlier tests that are freed meanwhile do
+    not move them), and the driver's free bytes."""
+    st = torch.cuda.memory_stats(DEV)
+    return (st["allocation.all.allocated"], st["segment.all.allocated"], torch.cuda.mem_get_info(DEV)[0])
 
 
 @pytest.mark.parametrize("policy", [0, 1])
