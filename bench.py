@@ -238,8 +238,9 @@ def run_reference(args, w) -> dict:
 
 
 def config_of(w, extra) -> dict:
-    c = {"workload": "configs[%d] %s: N=%d, lengths %s, frame %d B (%s), T_block=%d, unpack of %d B/frame outputs; "
-                     "one whole-epoch call per direction" % (w.index, w.name, w.n, w.dist, w.frame_bytes, w.payload,
+    which = "configs[%d]" % w.index if 0 <= w.index <= 4 else "extra workload (not an evaluation configuration)"
+    c = {"workload": "%s %s: N=%d, lengths %s, frame %d B (%s), T_block=%d, unpack of %d B/frame outputs; "
+                     "one whole-epoch call per direction" % (which, w.name, w.n, w.dist, w.frame_bytes, w.payload,
                                                              w.t_block, w.out_frame_bytes),
          "batch_blocks": w.batch_blocks, "l2": "inputs larger than L2 (no flush needed)", "seed": w.seed,
          "policy": POLICY}

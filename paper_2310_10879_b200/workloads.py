@@ -6,7 +6,8 @@ two can be compared on identical data.  The five workloads follow the shapes of
 the evaluation configurations (toy video, per-frame features, raw frames,
 token sequences, heavy-tailed feature sequences); a sixth has the shape of the
 video dataset used in the paper's experiments (N=7,464 clips of 3..94 frames)
-and is a synthetic stand-in, not that dataset.
+and is a synthetic stand-in, not that dataset; a seventh ("random_chunks") is a
+probe of the memory system, not a workload of the paper.
 """
 from __future__ import annotations
 
@@ -45,6 +46,11 @@ WORKLOADS = {
     # shape of the paper's training set (Experiments section): N clips, 3..94 frames, mean about 22.3
     "video_dataset_shape": Workload("video_dataset_shape", 5, 7464, 94, 64, 64, 8,
                                     "3 + geometric(mean 19.3) clip [3,94]", "u8"),
+    # Not one of the evaluation configurations: a probe of the memory system.  Every sequence is one frame and every block
+    # one slot, so the plan is a random permutation and pack / unpack copy equal-sized, 16-byte aligned chunks in random
+    # order.  It measures what a copy of chunks of that size can reach on the device, whichever kernel moves them; other
+    # chunk sizes with bench.py's --frame-bytes (and --n to keep the total at a few GB).
+    "random_chunks": Workload("random_chunks", 6, 262_144, 1, 16384, 16384, 256, "all 1 (one frame per sequence and block)", "u8"),
 }
 
 # The toy dataset of the paper's problem statement: 8 videos of 2..6 frames, two of
@@ -75,6 +81,8 @@ def lengths(w: Workload, seed: int | None = None) -> np.ndarray:
         t = np.clip(np.floor(20.0 * (1.0 + rng.pareto(1.5, size=n))), 1, 10_000)
     elif w.name == "video_dataset_shape":
         t = np.clip(2 + rng.geometric(1.0 / 20.3, size=n), 3, 94)
+    elif w.name == "random_chunks":
+        t = np.ones(n)
     else:
         raise KeyError(w.name)
     t = np.minimum(t, w.t_block)

@@ -57,7 +57,7 @@ def test_dataset_shaped_lengths():
     plan, op = G.full_parity(W.lengths(w), w.t_block, w.seed, w.frame_bytes)
     s = B.bload_stats(plan.info)
     assert s == {**O.stats(op.n, op.sum_t, op.t_max, op.t_block, op.n_blocks),
-                 "max_segs_per_block": op.max_segs_per_block}
+                 "max_segs_per_block": op.max_segs_per_block, "frames_deleted": 0}
 
 
 @pytest.mark.parametrize("fb", [1, 2, 3, 4, 6, 8, 12, 20, 24, 48, 100, 1000, 4100])
