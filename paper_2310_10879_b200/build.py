@@ -46,11 +46,13 @@ def nvcc_path() -> str:
     raise RuntimeError("nvcc not found: libbload cannot be built")
 
 
-def build(force: bool = False, verbose: bool = False, debug: bool = False) -> str:
+def build(force: bool = False, verbose: bool = False, debug: bool = False, defines: tuple = (), out: str | None = None) -> str:
     """Compile the library.  debug=True builds libbload_debug.so with -DBLOAD_DEBUG: every global access of the
-    copy, metadata and table kernels is checked against the bounds of its buffer (see bload_debug_status)."""
-    lib = DEBUG_LIB if debug else LIB
-    extra = "debug" if debug else ""
+    copy, metadata and table kernels is checked against the bounds of its buffer (see bload_debug_status).
+    defines / out: a variant with other tuning constants (e.g. ("BLOAD_STAGED_MAX_RUN=-1",) sends every frame size
+    through the register-path copy kernel) written to `out`; load it with BLOAD_LIBRARY to compare."""
+    lib = out or (DEBUG_LIB if debug else LIB)
+    extra = ("debug" if debug else "") + " ".join(defines)
     if not force and not stale(lib, extra):
         return lib
     tmp = lib + ".tmp%d" % os.getpid()
@@ -59,6 +61,7 @@ def build(force: bool = False, verbose: bool = False, debug: bool = False) -> st
            "-I", os.path.join(ROOT, "include"), "-I", CSRC]
     if debug:
         cmd += ["-DBLOAD_DEBUG=1"]
+    cmd += ["-D" + d for d in defines]
     if verbose:
         cmd += ["-Xptxas", "-v"]
     cmd += sources() + ["-o", tmp]
@@ -70,4 +73,9 @@ def build(force: bool = False, verbose: bool = False, debug: bool = False) -> st
 
 
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv, debug="--debug" in sys.argv))
+    argv = sys.argv[1:]
+    defs = tuple(argv[i + 1] for i, a in enumerate(argv[:-1]) if a == "--define")
+    out_path = next((argv[i + 1] for i, a in enumerate(argv[:-1]) if a == "--out"), None)
+    if defs and not out_path:
+        sys.exit("--define needs --out: the in-tree library is always built with the default constants")
+    print(build(force="--force" in argv, verbose="-v" in argv, debug="--debug" in argv, defines=defs, out=out_path))

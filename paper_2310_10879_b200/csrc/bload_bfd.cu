@@ -28,7 +28,7 @@ __global__ void __launch_bounds__(256, 1) kb_chain(const PlanHeader* hdr, const 
                                                    int2* __restrict__ rec, int32_t n, int32_t L)
 {
     extern __shared__ __align__(16) int32_t sm[];
-    const int words = (L + 31) >> 5;                       // rooms 1..L map to bits 0..L-1
+    // rooms 1..L map to bits 0..L-1 of B2
     uint32_t* B2 = reinterpret_cast<uint32_t*>(sm);        // [1024] bit set: some open block has that room
     int2* ring = reinterpret_cast<int2*>(sm + 1024);       // [32] records of the last items
     int32_t* cnt = sm + 1024 + 64;                         // [L] open blocks per room

@@ -135,7 +135,10 @@ template <bool UNPACK> struct StageCfg : StageCfgT<BLOAD_PACK_BYTES, BLOAD_PACK_
 template <> struct StageCfg<true> : StageCfgT<BLOAD_UNPACK_BYTES, BLOAD_UNPACK_WARPS, BLOAD_UNPACK_STAGES, BLOAD_UNPACK_GROUP> {};
 // the staged kernels win while the average run (T_i * frame_bytes) is short; measured cross-over on B200 at about
 // 16 KB (1.4 KB runs: 6.0 against 3.8 TB/s; 14 KB: 5.9 against 5.8; 23 KB: 6.15 against 6.36)
-constexpr int64_t kStagedMaxRunBytes = 16384;
+#ifndef BLOAD_STAGED_MAX_RUN
+#define BLOAD_STAGED_MAX_RUN 16384
+#endif
+constexpr int64_t kStagedMaxRunBytes = BLOAD_STAGED_MAX_RUN;  // (-1: every frame size through the register path, to compare)
 #ifndef BLOAD_PACK_CHUNK_TILES
 #define BLOAD_PACK_CHUNK_TILES 4
 #endif
@@ -629,7 +632,7 @@ bool staged_pack_with_metadata(const PlanView& pv, int32_t t_block, int64_t fram
     const int64_t grid = (int64_t)mo.pack_ctas + block_count * mo.chunks_per_block;
     count_launches(1);
     {
-        const size_t slots = (size_t)block_count * (size_t)t_block;
+        [[maybe_unused]] const size_t slots = (size_t)block_count * (size_t)t_block;
         BLOAD_DBG_EXPECT(st, dbg::kPackContig, {{store, (size_t)ragged_bytes}},
                          {{dense, (size_t)(block_count * block_bytes)}, {seq_id, 4 * slots}, {pos, 4 * slots}, {reset, slots}, {valid, slots}});
     }

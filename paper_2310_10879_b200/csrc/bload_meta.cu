@@ -53,7 +53,7 @@ cudaError_t launch_metadata(const PlanView& pv, int32_t t_block, int64_t block_b
     if (d_range) {
         BLOAD_DBG_UNCHECKED(st);
     } else {
-        const size_t slots = (size_t)block_count * (size_t)t_block;
+        [[maybe_unused]] const size_t slots = (size_t)block_count * (size_t)t_block;
         BLOAD_DBG_EXPECT(st, dbg::kMetadata, {}, {{seq_id, 4 * slots}, {pos, 4 * slots}, {reset, slots}, {valid, slots}});
     }
     if (t_block % 4 == 0 && al(seq_id, 16) && al(pos, 16) && al(reset, 4) && al(valid, 4))
