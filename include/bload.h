@@ -517,6 +517,14 @@ BLOAD_API int bload_debug_status(uint64_t out[4], int clear);
  */
 BLOAD_API const char* bload_last_copy_kernel(int which);
 
+/*
+ * bload_bulk_copy_timeouts -- for builds with -DBLOAD_BULK_COPY=1 only (a measurement variant that sends large frames
+ * through the bulk-copy engine and waits on mbarriers; the default library has no such wait and returns 0): the number
+ * of mbarrier waits that gave up after their poll limit since the library was loaded.  A warp that gives up stops
+ * copying, so any value but 0 means incomplete outputs.  Synchronises the device.  Host only.
+ */
+BLOAD_API int64_t bload_bulk_copy_timeouts(void);
+
 BLOAD_API const char* bload_strerror(int code);
 BLOAD_API int bload_version(void);
 

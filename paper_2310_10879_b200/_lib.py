@@ -20,7 +20,7 @@ MAX_T_BLOCK = 32768
 EXPORTS = ("bload_plan_sizes", "bload_plan", "bload_plan_async", "bload_plan_finish", "bload_rank_range", "bload_pack", "bload_unpack", "bload_stats", "bload_epoch", "bload_epoch_stage_times",
            "bload_pack_repeat_last", "bload_var_offsets", "bload_pack_var", "bload_unpack_var", "bload_var_offsets2d", "bload_pack_var2d",
            "bload_unpack_var2d", "bload_carry_prev", "bload_reset_state", "bload_valid_sum",
-           "bload_plan_static", "bload_chunk_work_bytes", "bload_chunk_count", "bload_plan_chunks", "bload_set_plan_timing", "bload_plan_stage_times", "bload_kernel_launches", "bload_last_copy_kernel", "bload_debug_status",
+           "bload_plan_static", "bload_chunk_work_bytes", "bload_chunk_count", "bload_plan_chunks", "bload_set_plan_timing", "bload_plan_stage_times", "bload_kernel_launches", "bload_last_copy_kernel", "bload_debug_status", "bload_bulk_copy_timeouts",
            "bload_strerror", "bload_version")
 
 
@@ -128,9 +128,11 @@ def load() -> C.CDLL:
     L.bload_version.argtypes = []
     L.bload_kernel_launches.argtypes = []
     for name in EXPORTS:
-        if name not in ("bload_strerror", "bload_kernel_launches", "bload_last_copy_kernel", "bload_debug_status", "bload_chunk_work_bytes"):
+        if name not in ("bload_strerror", "bload_kernel_launches", "bload_last_copy_kernel", "bload_debug_status", "bload_bulk_copy_timeouts", "bload_chunk_work_bytes"):
             getattr(L, name).restype = C.c_int
     L.bload_kernel_launches.restype = C.c_int64
+    L.bload_bulk_copy_timeouts.argtypes = []
+    L.bload_bulk_copy_timeouts.restype = C.c_int64
     L.bload_chunk_work_bytes.restype = C.c_size_t
     L.bload_last_copy_kernel.restype = C.c_char_p
     _lib = L

@@ -201,6 +201,8 @@ int bload_debug_status(uint64_t out[4], int clear)
 #endif
 }
 
+int64_t bload_bulk_copy_timeouts(void) { return (int64_t)bulk_copy_timeouts(); }
+
 const char* bload_last_copy_kernel(int which)
 {
     if (which < 0 || which >= kCopyCalls || !g_last_kernel[which]) return "";

@@ -135,6 +135,9 @@ template <bool UNPACK> struct StageCfg : StageCfgT<BLOAD_PACK_BYTES, BLOAD_PACK_
 template <> struct StageCfg<true> : StageCfgT<BLOAD_UNPACK_BYTES, BLOAD_UNPACK_WARPS, BLOAD_UNPACK_STAGES, BLOAD_UNPACK_GROUP> {};
 // the staged kernels win while the average run (T_i * frame_bytes) is short; measured cross-over on B200 at about
 // 16 KB (1.4 KB runs: 6.0 against 3.8 TB/s; 14 KB: 5.9 against 5.8; 23 KB: 6.15 against 6.36)
+#ifndef BLOAD_BULK_COPY
+#define BLOAD_BULK_COPY 0
+#endif
 #ifndef BLOAD_STAGED_MAX_RUN
 #define BLOAD_STAGED_MAX_RUN 16384
 #endif
@@ -596,6 +599,182 @@ __global__ void __launch_bounds__(StageCfg<false>::kWarps * 32) k10_pack_contig(
     if (lane == 0) bulk_wait_read<0>();
 }
 
+
+// ------------------------------------------------------------------------------------------------
+// Measurement variant, compiled only with -DBLOAD_BULK_COPY=1 (never in the default library): the large-frame path
+// through the bulk-copy engine instead of registers.  Frames whose size is a multiple of 16 bytes; a warp owns a ring
+// of shared-memory stages, each the image of one sub-tile of the dense side.  Pack: every run piece of the sub-tile
+// arrives by one cp.async.bulk (global -> shared, completion counted in bytes on the stage's mbarrier), padding is
+// written with shared stores, the sub-tile leaves with ONE bulk store.  Unpack: the occupied part of the sub-tile
+// arrives by ONE bulk load and leaves with one bulk store per run piece.  It exists so that the comparison "bulk
+// engine against register path" can be repeated from this source; on B200 the register path is faster (see the
+// measurements next to launch_copy).  The only waits are on the warp's own mbarriers and bulk groups; the mbarrier
+// wait gives up after a fixed number of polls, counts the event (bload_bulk_copy_timeouts) and lets the warp finish.
+#if BLOAD_BULK_COPY
+#ifndef BLOAD_BULK_BYTES
+#define BLOAD_BULK_BYTES 8192
+#endif
+#ifndef BLOAD_BULK_WARPS
+#define BLOAD_BULK_WARPS 4
+#endif
+#ifndef BLOAD_BULK_STAGES
+#define BLOAD_BULK_STAGES 3
+#endif
+static __device__ unsigned int g_bulk_timeouts;
+
+__device__ __forceinline__ void mbar_init(uint32_t bar)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(1) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void bulk_load(uint32_t smem_dst, const void* g, uint32_t bytes, uint32_t bar)
+{
+    if (!BLOAD_MAY_READ(g, bytes)) return;
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(smem_dst), "l"(g), "r"(bytes), "r"(bar) : "memory");
+}
+// true when the phase with this parity has completed; gives up after kPolls polls
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity)
+{
+    constexpr int kPolls = 1 << 22;
+    for (int i = 0; i < kPolls; ++i) {
+        uint32_t done;
+        asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                     : "=r"(done) : "r"(bar), "r"(parity) : "memory");
+        if (done) return true;
+    }
+    atomicAdd(&g_bulk_timeouts, 1u);
+    return false;
+}
+
+template <bool UNPACK>
+__global__ void __launch_bounds__(BLOAD_BULK_WARPS * 32) k7b_copy_bulk(PlanView pv, int32_t t_block, int64_t frame_bytes,
+                                                                      int64_t block_begin, int64_t block_count,
+                                                                      const uint8_t* __restrict__ src_base,
+                                                                      uint8_t* __restrict__ dst_base, int64_t subs_per_block,
+                                                                      uint8_t pad)
+{
+    constexpr int NST = BLOAD_BULK_STAGES, kBytes = BLOAD_BULK_BYTES, kWarps = BLOAD_BULK_WARPS;
+    extern __shared__ __align__(128) uint8_t stage_mem[];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    uint8_t* my_stages = stage_mem + (size_t)warp * NST * kBytes;
+    const uint32_t my_bars = smem_addr(stage_mem + (size_t)kWarps * NST * kBytes) + (uint32_t)warp * NST * 8;
+    if (lane == 0) {
+        for (int i = 0; i < NST; ++i) mbar_init(my_bars + 8 * i);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncwarp();
+    const int64_t warps = (int64_t)gridDim.x * kWarps;
+    const int64_t items = block_count * subs_per_block;
+    const int64_t block_bytes = (int64_t)t_block * frame_bytes;
+    const int64_t n_blocks = pv.hdr->n_blocks;
+    const uint32_t p4 = 0x01010101u * pad;
+    uint32_t parity_bits = 0;  // bit i: parity of the phase stage i's barrier is in
+
+    // what the second phase of an item needs
+    struct Pending { int64_t dense_off; int64_t b; int lo; int nbytes; int valid; int k; int k1; int fill; bool wait; };
+    Pending prev{};
+    bool have_prev = false, alive = true;
+    int s = 0, s_prev = 0;
+
+    // second phase: the loads of the item have landed in `stage`
+    auto complete = [&](const Pending& it, uint8_t* stage, int st_idx) {
+        if (it.wait) {
+            bool ok = true;
+            if (lane == 0) ok = mbar_wait(my_bars + 8 * st_idx, (parity_bits >> st_idx) & 1u);
+            ok = __shfl_sync(kFull, ok, 0);
+            parity_bits ^= 1u << st_idx;
+            if (!ok) { alive = false; return; }
+        }
+        fence_proxy_async();  // shared stores of padding before the bulk store reads them
+        __syncwarp();
+        if (!UNPACK) {
+            if (lane == 0) bulk_store(dst_base + it.dense_off, smem_addr(stage), (uint32_t)it.nbytes);
+        } else if (it.valid > 0) {
+            // one bulk store per run piece of the occupied part
+            int k = it.k, kw = it.k;
+            int w_st = (kw + lane < it.k1) ? pv.seg_start[kw + lane] : it.fill;
+            int64_t w_src = (kw + lane < it.k1) ? pv.seg_src[kw + lane] : 0;
+            int64_t cur = it.lo;
+            const int64_t hi = (int64_t)it.lo + it.valid;
+            while (cur < hi && k < it.k1) {
+                if (k - kw == 31) {
+                    kw = k;
+                    w_st = (kw + lane < it.k1) ? pv.seg_start[kw + lane] : it.fill;
+                    w_src = (kw + lane < it.k1) ? pv.seg_src[kw + lane] : 0;
+                }
+                const int st = __shfl_sync(kFull, w_st, k - kw);
+                const int nx = __shfl_sync(kFull, w_st, k - kw + 1);
+                const int64_t src_frame = __shfl_sync(kFull, w_src, k - kw);
+                const int64_t pe = min((int64_t)nx * frame_bytes, hi);
+                const int64_t rag = src_frame * frame_bytes + (cur - (int64_t)st * frame_bytes);
+                if (lane == 0) bulk_store(dst_base + rag, smem_addr(stage) + (uint32_t)(cur - it.lo), (uint32_t)(pe - cur));
+                cur = pe;
+                ++k;
+            }
+        }
+        if (lane == 0) bulk_commit();
+    };
+
+    for (int64_t item = (int64_t)blockIdx.x * kWarps + warp; item < items && alive; item += warps) {
+        const int64_t q = item / subs_per_block;
+        Pending it{};
+        it.lo = (int)((item - q * subs_per_block) * kBytes);
+        it.nbytes = (int)min((int64_t)kBytes, block_bytes - it.lo);
+        it.b = block_begin + q;
+        it.dense_off = q * block_bytes + it.lo;
+        int k0 = 0;
+        if (it.b < n_blocks) { k0 = pv.block_seg_begin[it.b]; it.k1 = pv.block_seg_begin[it.b + 1]; it.fill = pv.block_fill[it.b]; }
+        const int64_t fill_bytes = (int64_t)it.fill * frame_bytes;
+        it.valid = it.lo < fill_bytes ? (int)min((int64_t)it.nbytes, fill_bytes - it.lo) : 0;
+        it.wait = it.valid > 0;
+        it.k = it.valid > 0 ? warp_find_segment(pv.seg_start, k0, it.k1, (int)(it.lo / frame_bytes), lane) : k0;
+        uint8_t* stage = my_stages + (size_t)s * kBytes;
+        const uint32_t sa = smem_addr(stage), bar = my_bars + 8 * s;
+        if (lane == 0) bulk_wait_read<NST - 2>();  // the stores that last read this stage have finished reading
+        __syncwarp();
+        if (it.valid > 0) {
+            if (lane == 0) mbar_expect_tx(bar, (uint32_t)it.valid);
+            if (UNPACK) {
+                if (lane == 0) bulk_load(sa, src_base + it.dense_off, (uint32_t)it.valid, bar);
+            } else {
+                int k = it.k, kw = it.k;
+                int w_st = (kw + lane < it.k1) ? pv.seg_start[kw + lane] : it.fill;
+                int64_t w_src = (kw + lane < it.k1) ? pv.seg_src[kw + lane] : 0;
+                int64_t cur = it.lo;
+                const int64_t hi = (int64_t)it.lo + it.valid;
+                while (cur < hi && k < it.k1) {
+                    if (k - kw == 31) {
+                        kw = k;
+                        w_st = (kw + lane < it.k1) ? pv.seg_start[kw + lane] : it.fill;
+                        w_src = (kw + lane < it.k1) ? pv.seg_src[kw + lane] : 0;
+                    }
+                    const int st = __shfl_sync(kFull, w_st, k - kw);
+                    const int nx = __shfl_sync(kFull, w_st, k - kw + 1);
+                    const int64_t src_frame = __shfl_sync(kFull, w_src, k - kw);
+                    const int64_t pe = min((int64_t)nx * frame_bytes, hi);
+                    const int64_t rag = src_frame * frame_bytes + (cur - (int64_t)st * frame_bytes);
+                    if (lane == 0) bulk_load(sa + (uint32_t)(cur - it.lo), src_base + rag, (uint32_t)(pe - cur), bar);
+                    cur = pe;
+                    ++k;
+                }
+            }
+        }
+        if (!UNPACK)  // padding behind the frames (valid and nbytes are multiples of 16 here)
+            for (int o = it.valid + 16 * lane; o < it.nbytes; o += 512) *reinterpret_cast<uint4*>(stage + o) = make_uint4(p4, p4, p4, p4);
+        if (have_prev) complete(prev, my_stages + (size_t)s_prev * kBytes, s_prev);
+        prev = it; have_prev = true; s_prev = s;
+        s = (s + 1 == NST) ? 0 : s + 1;
+    }
+    if (have_prev && alive) complete(prev, my_stages + (size_t)s_prev * kBytes, s_prev);
+    __syncwarp();
+    if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");  // the warp's own stores are complete
+}
+#endif  // BLOAD_BULK_COPY
+
 }  // namespace
 
 // Pack and per-slot metadata of a few blocks of small word-sized frames in ONE launch (see k10_pack_contig<true>);
@@ -716,6 +895,27 @@ cudaError_t launch_copy(bool unpack, const PlanView& pv, int32_t t_block, int64_
         note_copy_kernel(kCallUnpack, "k8_unpack_staged");
         return cudaPeekAtLastError();
     }
+#if BLOAD_BULK_COPY
+    if (frame_bytes % 16 == 0) {  // the measurement variant through the bulk-copy engine
+        constexpr int kB = BLOAD_BULK_BYTES, kW = BLOAD_BULK_WARPS, kS = BLOAD_BULK_STAGES;
+        const size_t smem = (size_t)kW * kS * kB + (size_t)kW * kS * 8;
+        const DeviceInfo di = device_info();
+        const int per_sm = (int)(di.smem_per_sm / (smem + 1024));
+        const int64_t spb_b = (block_bytes + kB - 1) / kB;
+        const int64_t want_b = (block_count * spb_b + kW - 1) / kW, cap = (int64_t)di.sm_count * (per_sm > 0 ? per_sm : 1);
+        const unsigned grid_b = (unsigned)(want_b < cap ? want_b : cap);
+        cudaError_t e = opt_in_shared_memory(unpack ? k7b_copy_bulk<true> : k7b_copy_bulk<false>, (int)smem);
+        if (e != cudaSuccess) return e;
+        note_copy_kernel(unpack ? kCallUnpack : kCallPack, unpack ? "k7b_copy_bulk<unpack>" : "k7b_copy_bulk<pack>");
+        if (unpack)
+            k7b_copy_bulk<true><<<grid_b, kW * 32, smem, st>>>(pv, t_block, frame_bytes, block_begin, block_count, dense, ragged_out,
+                                                              spb_b, pad_byte);
+        else
+            k7b_copy_bulk<false><<<grid_b, kW * 32, smem, st>>>(pv, t_block, frame_bytes, block_begin, block_count, ragged_in, dense,
+                                                               spb_b, pad_byte);
+        return cudaPeekAtLastError();
+    }
+#endif
     note_copy_kernel(unpack ? kCallUnpack : kCallPack, unpack ? "k7_copy<unpack>" : "k7_copy<pack>");
     const int64_t sub = 16384;
     const int64_t spb = (block_bytes + sub - 1) / sub;
@@ -755,6 +955,22 @@ cudaError_t launch_copy_range(bool unpack, const PlanView& pv, int32_t t_block, 
         k7_copy<false><<<grid, 256, kBesideChainSmemBytes, st>>>(pv, t_block, frame_bytes, 0, 0, src, dst, src_total_bytes, sub, spb,
                                                                  pad_byte, d_range, 0);
     return cudaPeekAtLastError();
+}
+
+
+// mbarrier waits that gave up in the bulk-copy measurement variant since the library was loaded (0 in the default build)
+unsigned int bulk_copy_timeouts()
+{
+#if BLOAD_BULK_COPY
+    unsigned int v = 0;
+    if (cudaDeviceSynchronize() != cudaSuccess || cudaMemcpyFromSymbol(&v, g_bulk_timeouts, sizeof v) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return ~0u;
+    }
+    return v;
+#else
+    return 0;
+#endif
 }
 
 }  // namespace bload

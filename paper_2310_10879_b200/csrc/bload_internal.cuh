@@ -121,6 +121,8 @@ void count_launches(int k);
 enum CopyCall { kCallPack = 0, kCallUnpack = 1, kCallCarryPrev = 2, kCallPackVar = 3, kCallUnpackVar = 4, kCopyCalls = 5 };
 void note_copy_kernel(int call, const char* name);
 
+unsigned int bulk_copy_timeouts();  // see bload_bulk_copy_timeouts
+
 // Multiprocessors and shared memory per multiprocessor of the current device, asked for once per device (grids and
 // occupancy are sized from them; a failed query answers with the B200's 148 and 228 KB).
 struct DeviceInfo { int sm_count; int smem_per_sm; };
