@@ -18,8 +18,14 @@ import sys
 import pytest
 rc = pytest.main(["-x", "-q", "-m", "gpu", "-p", "no:cacheprovider", "-k",
                   "frame_sizes or config_ or toy8 or degenerate or block_ranges", "tests/test_gpu_parity.py"])
+import torch
 import paper_2310_10879_b200 as B
-assert B.bload_last_copy_kernel("pack").startswith("k7b_copy_bulk") or B.bload_last_copy_kernel("unpack").startswith("k7b_copy_bulk")
+plan = B.bload_plan(torch.full((40,), 50, dtype=torch.int32, device="cuda:0"), 64, 1)   # runs of 50 KB: the large-frame path
+store = torch.zeros(plan.sum_t * 1024, dtype=torch.uint8, device="cuda:0")
+dense = torch.empty(plan.n_blocks * 64 * 1024, dtype=torch.uint8, device="cuda:0")
+B.bload_pack(plan, store, 1024, 0, plan.n_blocks, dense=dense)
+B.bload_unpack(plan, dense, 1024, 0, plan.n_blocks, store)
+assert B.bload_last_copy_kernel("pack") == "k7b_copy_bulk<pack>" and B.bload_last_copy_kernel("unpack") == "k7b_copy_bulk<unpack>"
 timeouts = B.load().bload_bulk_copy_timeouts()
 print("bulk copy timeouts:", timeouts)
 sys.exit(int(rc) or (1 if timeouts else 0))
