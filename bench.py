@@ -702,7 +702,8 @@ def run_gpu(args, w) -> dict:
            "padding": {"n": stats["n"], "sum_t": stats["sum_t"], "t_max": stats["t_max"], "n_blocks": stats["n_blocks"],
                        "min_blocks": stats["min_blocks"], "frac_packed": stats["frac_packed"],
                        "frac_naive_tmax": stats["frac_naive_tmax"], "frac_naive_tblock": stats["frac_naive_tblock"],
-                       "reduction_vs_tmax": stats["reduction_vs_tmax"]}}
+                       "reduction_vs_tmax": stats["reduction_vs_tmax"],
+                       "chunking_strategy": chunk_strategy_figures(B, torch, d_len, tb)}}
     if not args.no_cpu and world == 1:
         blocks = args.ref_blocks
         need = (fb + ofb) * (sum_t + nb * tb) * 1.3          # host arrays of a whole-workload sample
@@ -732,6 +733,27 @@ def host_cores() -> int:
         return len(os.sched_getaffinity(0))
     except Exception:
         return os.cpu_count() or 1
+
+
+def chunk_strategy_figures(B, torch, d_len, t_block) -> dict:
+    """The chunking strategy the paper compares with, as a planner on the same lengths (context for the padding figures):
+    chunks of an eighth of the block length, tails kept and tails dropped; device time of count + plan per variant."""
+    out = {}
+    c = max(1, t_block // 8)
+    for name, tail in (("keep_tail", 0), ("drop_tail", 1)):
+        try:
+            B.bload_plan_chunks(d_len, c, tail)                      # warm-up
+            a, b_ = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            plan, ci, _, _ = B.bload_plan_chunks(d_len, c, tail)
+            b_.record(); torch.cuda.synchronize()
+            out[name] = {"t_chunk": c, "n_chunks": int(ci.n_chunks), "pad_frames": int(ci.pad_frames),
+                         "frames_deleted": int(ci.frames_deleted), "frac_padding": ci.pad_frames / max(1, ci.n_chunks * c),
+                         "frac_deleted": ci.frames_deleted / max(1, ci.sum_t), "count_and_plan_ms": a.elapsed_time(b_)}
+            del plan
+        except Exception as exc:                                     # e.g. nothing is kept when every sequence is shorter
+            out[name] = {"t_chunk": c, "error": str(exc)[:120]}
+    return out
 
 
 def plan_figures(plan_ms, stage, n, clocks) -> dict:
@@ -825,7 +847,8 @@ def measure_config(args, w, dev, peak, clocks) -> dict:
                        "plan": plan_figures(sum(t_plan) / len(t_plan), stage, T.size, clocks)},
            "per_batch_pack": _time_per_batch(c),
            "padding": {"n_blocks": st["n_blocks"], "min_blocks": st["min_blocks"], "frac_packed": st["frac_packed"],
-                       "frac_naive_tmax": st["frac_naive_tmax"], "reduction_vs_tmax": st["reduction_vs_tmax"]}}
+                       "frac_naive_tmax": st["frac_naive_tmax"], "reduction_vs_tmax": st["reduction_vs_tmax"],
+                       "chunking_strategy": chunk_strategy_figures(B, torch, d_len, tb)}}
     del c, store, dense, seq_id, pos, reset, valid, dense_out, ragged_out, plan, plan_buf, work
     torch.cuda.empty_cache()
     if not args.no_cpu:

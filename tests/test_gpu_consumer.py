@@ -253,8 +253,10 @@ def test_pack_repeat_last_workloads():
 @pytest.mark.parametrize("fb,tb", [(4, 16), (4, 4096), (8, 64), (12, 1000), (16, 64), (32, 500), (100, 64), (256, 48),
                                    (4, 8192)])
 def test_carry_prev_small_word_sized_frames_take_the_staged_kernel(fb, tb):
-    # frame sizes that are multiples of 4 in short runs with 16-byte block rows: stages of 8 KB, several per block or
-    # several blocks per stage, segments that start inside a stage, first frames that straddle two stages
+    # (the name is historical: these cases used to go through the staged pack kernel; short runs now take the shifted
+    # copy, k11_carry_shift)  frame sizes that are multiples of 4 in short runs with 16-byte block rows: several
+    # sub-tiles per block or several blocks per sub-tile, segments that start inside a sub-tile, first frames that
+    # straddle two sub-tiles
     rng = np.random.default_rng(fb * 1000 + tb)
     n = int(rng.integers(50, 600))
     T = np.minimum(rng.geometric(1.0 / max(2, tb // 6), size=n), tb).astype(np.int32)
@@ -264,3 +266,21 @@ def test_carry_prev_small_word_sized_frames_take_the_staged_kernel(fb, tb):
     if op.n_blocks > 4:
         _carry_prev_parity(plan, op, fb, 3, op.n_blocks - 4, 0x5E)
         _carry_prev_parity(plan, op, fb, op.n_blocks - 1, 5, 0x01)
+
+
+@pytest.mark.parametrize("fb,tb,tmax", [(1, 40, 9), (3, 50, 50), (7, 3000, 40), (10, 64, 8), (130, 64, 20), (1000, 12, 5),
+                                        (4096, 30, 3), (20, 20000, 600), (6, 16384, 300)])
+def test_carry_prev_short_runs_take_the_shifted_copy(fb, tb, tmax):
+    """Short runs (16 KB or less on average), any frame size: one shifted copy per sub-tile and fill patches at the first
+    frame of every segment -- one lane per segment for frames up to 64 bytes, the whole warp per segment above; frame
+    sizes that are not multiples of 4 or 16, first frames that straddle sub-tiles, more than 32 segments per sub-tile,
+    blocks that end inside a sub-tile, filler blocks, sub-ranges."""
+    rng = np.random.default_rng(fb * 77 + tb)
+    n = int(min(3000, max(4, 4_000_000 // (tmax * fb))))
+    T = rng.integers(1, tmax + 1, size=n).astype(np.int32)
+    plan, op = _both_plans(T, tb, 31)
+    _carry_prev_parity(plan, op, fb, 0, op.n_blocks + 2, 0x00)
+    assert B.bload_last_copy_kernel("carry_prev") == "k11_carry_shift"
+    _carry_prev_parity(plan, op, fb, 0, op.n_blocks, 0xC3, seed=9)
+    if op.n_blocks > 3:
+        _carry_prev_parity(plan, op, fb, 1, op.n_blocks - 2, 0x5E)
