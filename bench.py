@@ -883,7 +883,9 @@ def main():
     ap.add_argument("--n", type=int, default=0, help="override the number of sequences (small profiling cases)")
     ap.add_argument("--policy", type=int, default=0, help="fill policy: 0 uniform over sequences, 1 uniform over lengths")
     ap.add_argument("--frame-bytes", type=int, default=0, help="override the frame size of the workload (experiments)")
-    ap.add_argument("--e2e-steps", type=int, default=6)
+    ap.add_argument("--e2e-steps", type=int, default=12,
+                    help="steps of the end-to-end leg (the pipeline over PCIe fills and drains once: about 200 ms that "
+                         "are shared by these steps)")
     ap.add_argument("--ref-blocks", type=int, default=0,
                     help="blocks in the CPU oracle's sample (0 = all blocks for the CPU baseline; sized from a "
                          "calibration run for --impl reference)")
