@@ -126,3 +126,37 @@ def test_full_size_epoch_call_equals_the_separate_calls(name):
     for a, b in zip(got_meta, want_meta):
         assert torch.equal(a, b)
     assert torch.equal(got_rag.t, want_rag)
+
+
+@pytest.mark.parametrize("tail", [O.KEEP_TAIL, O.DROP_TAIL])
+def test_full_size_chunking_planner_on_the_token_lengths(tail):
+    """The chunking planner at a million sequences (2.4 / 1.6 million chunks of 512 tokens): totals, every table and the
+    digest against the oracle, and the packed bytes of every block through the ordinary pack call, slab by slab."""
+    w = W.WORKLOADS["tokens"]
+    T = W.lengths(w)
+    c, fb = 512, w.frame_bytes
+    ch = O.chunks(T, c, tail)
+    plan, ci, cseq, cfirst = B.bload_plan_chunks(torch.from_numpy(T).to(G.DEV), c, tail)
+    assert (ci.n_chunks, ci.frames_kept, ci.frames_deleted, ci.pad_frames, ci.sum_t) == \
+        (ch.n_chunks, ch.frames_kept, ch.frames_deleted, ch.pad_frames, ch.sum_t)
+    assert np.array_equal(cseq.cpu().numpy(), ch.chunk_seq) and np.array_equal(cfirst.cpu().numpy(), ch.chunk_first)
+    G.assert_plan_equal(plan, ch.as_plan(), maximal=False, invariants_too=tail == O.KEEP_TAIL)
+    store = W.payload_torch(w, ch.sum_t, G.DEV).view(torch.uint8).reshape(-1)
+    nb = ch.n_chunks
+    dense = G.Guarded(nb * c * fb)
+    B.bload_pack(plan, store, fb, 0, nb, dense=dense.t)
+    torch.cuda.synchronize(); dense.check()
+    store_h = store.cpu().numpy()
+    d2 = dense.t.view(nb, c * fb)
+    for lo, cnt in _slabs(nb, c * fb):
+        _assert_same(d2[lo:lo + cnt], O.chunk_pack(ch, store_h, fb, lo, cnt, 0), "chunk blocks %d..%d" % (lo, lo + cnt))
+    # unpack: kept frames come back, deleted frames keep the canary value
+    back = G.Guarded(ch.sum_t * fb, 0x5A)
+    B.bload_unpack(plan, dense.t, fb, 0, nb, back.t)
+    torch.cuda.synchronize(); back.check()
+    want = np.full(ch.sum_t * fb, 0x5A, np.uint8)
+    for lo, cnt in _slabs(nb, c * fb):
+        O.chunk_unpack(ch, d2[lo:lo + cnt].cpu().numpy(), fb, lo, cnt, want)
+    step = 1 << 30
+    for lo in range(0, want.size, step):
+        _assert_same(back.t[lo:lo + step], want[lo:lo + step], "unpacked bytes from %d" % lo)
