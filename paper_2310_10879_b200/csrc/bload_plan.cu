@@ -428,21 +428,25 @@ __global__ void __launch_bounds__(256, 1) k4_fill(PlanView pv, const int32_t* __
         u_nxt = k + 32 + lane < n ? draw_u[k + 32 + lane] : 0;
         __syncwarp();
     };
-    // The loop is unrolled over the 32 places of a group: ring entry and word lane become constants, and the
-    // flush test and the loop branch come once per group (measured 162 -> 142 ns per draw on heavy-tailed lengths,
-    // 184 -> 155 ns on token lengths; unrolled 8 times: 148 / 162).  Draws before the first group boundary (a
-    // resumed chain) and after the last whole group go one by one.
+    // The loop is unrolled over half a group: ring entry and word lane become a base plus a constant, and the flush
+    // test and the loop branch come once per 16 draws.  Measured per draw, heavy-tailed / token lengths: rolled loop
+    // 162 / 184 ns, unrolled 4 times 153 / 166, 8 times 148 / 162, 16 times 147 / 160, 32 times 142 / 155 -- but the
+    // last figure moved between 142 and 159 ns from one build or process to the next (the body of 32 draws no longer
+    // fits the innermost instruction cache), while 8 and 16 repeated to the tenth of a nanosecond.  Draws before the
+    // first boundary (a resumed chain) and after the last whole half group go one by one.
+    constexpr int kUnroll = 16;
     bool stop = false;
-    while (!stop && k < n && (k & 31) != 0) {
+    while (!stop && k < n && (k & (kUnroll - 1)) != 0) {
         stop = draw(k & 31);
         if (!stop && (k & 31) == 0) flush_group();
     }
-    while (!stop && k + 32 <= n) {
+    while (!stop && k + kUnroll <= n) {
+        const int base = k & 31;
 #pragma unroll
-        for (int i = 0; i < 32; ++i) {
-            if (draw(i)) { stop = true; break; }
+        for (int i = 0; i < kUnroll; ++i) {
+            if (draw(base + i)) { stop = true; break; }
         }
-        if (!stop) flush_group();
+        if (!stop && (k & 31) == 0) flush_group();
     }
     while (!stop && k < n) {
         stop = draw(k & 31);
@@ -589,12 +593,16 @@ __global__ void __launch_bounds__(256, 1) k4_fill_lengths(PlanView pv, const int
         u_nxt = k + 32 + lane < n ? draw_u[k + 32 + lane] : 0;
         __syncwarp();
     };
-    while (k + 32 <= n) {  // unrolled over the 32 places of a group, as in k4_fill
+    while (k + 16 <= n) {  // unrolled over half a group, as in k4_fill
+        const int base = k & 31;
 #pragma unroll
-        for (int i = 0; i < 32; ++i) draw(i);
-        flush_group();
+        for (int i = 0; i < 16; ++i) draw(base + i);
+        if ((k & 31) == 0) flush_group();
     }
-    while (k < n) draw(k & 31);
+    while (k < n) {
+        draw(k & 31);
+        if ((k & 31) == 0) flush_group();
+    }
     __syncwarp();
     if (lane < (n & 31)) draw_rec[(n & ~31) + lane] = ring[lane];
     if (lane == 0) {
