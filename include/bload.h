@@ -215,7 +215,10 @@ BLOAD_API int bload_epoch_stage_times(float out_ms[5]);
  * round an epoch up to whole batches.  d_store is the flat ragged store (sum_t * frame_bytes bytes,
  * sequence i at frame offsets[i]); d_dense is [block_count, t_block, frame_bytes] row major.
  * d_store and d_dense must be 16-byte aligned.  d_dense and each of the four metadata outputs may be
- * NULL (that output is skipped).  Asynchronous on `stream`; no host synchronisation.
+ * NULL (that output is skipped).  Asynchronous on `stream`; no host synchronisation.  Launches: one kernel for the
+ * metadata and one for the dense blocks; a call that asks for both, for small word-sized frames (frame_bytes a multiple
+ * of 4, runs of at most 16 KB on average, t_block * frame_bytes a multiple of 16) and at most 4 Mi slots, is a single
+ * launch -- the call a training loop makes per batch of token-sized frames is bound by launch overhead, not by bytes.
  * Errors: NULL plan/info/store (when d_dense is given), ARG (frame_bytes < 1, negative range,
  * block_begin + block_count >= 2^31), ALIGN, PLAN (info->status != 0), CUDA.
  */
