@@ -126,11 +126,13 @@ __global__ void __launch_bounds__(256) k7_copy(PlanView pv, int32_t t_block, int
 #ifndef BLOAD_UNPACK_GROUP
 #define BLOAD_UNPACK_GROUP 4
 #endif
+#pragma nv_diag_suppress 177  // (the pack configuration never reads kGroup)
 template <int BYTES, int WARPS, int STAGES, int GROUP>
 struct StageCfgT {
     static constexpr int kBytes = BYTES, kWarps = WARPS, kStages = STAGES, kGroup = GROUP;
     static_assert(BYTES % 512 == 0 && STAGES >= 2 && GROUP >= 1, "stage configuration");
 };
+#pragma nv_diag_default 177
 template <bool UNPACK> struct StageCfg : StageCfgT<BLOAD_PACK_BYTES, BLOAD_PACK_WARPS, BLOAD_PACK_STAGES, 2> {};
 template <> struct StageCfg<true> : StageCfgT<BLOAD_UNPACK_BYTES, BLOAD_UNPACK_WARPS, BLOAD_UNPACK_STAGES, BLOAD_UNPACK_GROUP> {};
 // the staged kernels win while the average run (T_i * frame_bytes) is short; measured cross-over on B200 at about
@@ -152,6 +154,11 @@ __device__ __forceinline__ void cp_async4(uint32_t s, const void* g)
 {
     if (!BLOAD_MAY_READ(g, 4)) return;
     asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(s), "l"(g) : "memory");
+}
+__device__ __forceinline__ void cp_async8(uint32_t s, const void* g)
+{
+    if (!BLOAD_MAY_READ(g, 8)) return;
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"(s), "l"(g) : "memory");
 }
 __device__ __forceinline__ void cp_async16(uint32_t s, const void* g)
 {
@@ -196,6 +203,18 @@ __device__ __forceinline__ void warp_gather_async(uint32_t sd, const uint8_t* __
         }
         const int tw = (n - (nv << 4)) >> 2;
         if (lane < tw) cp_async4(sd + (nv << 4) + 4 * lane, gs + (nv << 4) + 4 * lane);
+    } else if (((sd ^ (uint32_t)reinterpret_cast<uintptr_t>(gs)) & 7u) == 0) {
+        // source and stage agree modulo 8: one leading word to reach an 8-byte boundary, then 8-byte copies
+        const int hw = (n >= 4) ? (int)((sd >> 2) & 1u) : 0;
+        if (hw && lane == 0) cp_async4(sd, gs);
+        if (hw) { sd += 4; gs += 4; n -= 4; }
+        const int nd = n >> 3;
+        uint32_t s = sd + 8 * lane;
+        const uint8_t* g = gs + 8 * lane;
+        int rem = nd - lane;  // double words left for this lane, 32 apart
+        for (; rem > 96; rem -= 128, s += 1024, g += 1024) BLOAD_CP4X("cp.async.ca.shared.global", 8, s, g, 256);
+        for (; rem > 0; rem -= 32, s += 256, g += 256) cp_async8(s, g);
+        if ((n & 4) && lane == 0) cp_async4(sd + (nd << 3), gs + (nd << 3));
     } else {
         uint32_t s = sd + 4 * lane;
         const uint8_t* g = gs + 4 * lane;
