@@ -668,6 +668,19 @@ def run_gpu(args, w) -> dict:
     fused = _time_fused_epoch(c)
     per_batch = _time_per_batch(c)
     consumer = _time_consumer(c)
+
+    def timed_launch(fn, reps=10):
+        for _ in range(3):
+            fn()
+        torch.cuda.synchronize()
+        a, b_ = ev(), ev()
+        a.record()
+        for _ in range(reps):
+            fn()
+        b_.record()
+        torch.cuda.synchronize()
+        return a.elapsed_time(b_) / reps
+    rank_share = rank_share_figures(c, timed_launch) if not args.no_consumer else None
     e2e = _time_end_to_end(c)
     if rank != 0:
         return {}
@@ -690,6 +703,7 @@ def run_gpu(args, w) -> dict:
            "dtype": "u8", "data": "synthetic", "config": config_of(w, {"parallelism": "replicas only"}),
            "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline,
            "frames_per_s": aggregate(sum_t, world, step_s), "per_batch_pack": per_batch, "pipelined": pipelined, "fused_epoch": fused, "consumer": consumer,
+           "one_rank_of_eight": rank_share,
            "kernels": {
                "pack_copy": {"kernel": k_pack, "ms": pack_ms, "GB/s": by["pack"] / pack_ms / 1e6, "frac_measured": by["pack"] / pack_ms / 1e6 / peak,
                              "frac_nominal": by["pack"] / pack_ms / 1e6 / NOMINAL_HBM_GBS, "frames_per_s": sum_t / pack_ms * 1e3},
@@ -754,6 +768,26 @@ def chunk_strategy_figures(B, torch, d_len, t_block) -> dict:
         except Exception as exc:                                     # e.g. nothing is kept when every sequence is shorter
             out[name] = {"t_chunk": c, "error": str(exc)[:120]}
     return out
+
+
+def rank_share_figures(c, timed) -> dict:
+    """What ONE of eight data-parallel ranks does per epoch (the paper's setting; every rank computes the same plan and
+    takes its own contiguous block range, bload_rank_range): pack and unpack of that range, whole-range launches."""
+    B, torch = c.B, c.torch
+    b0, cnt = B.bload_rank_range(c.nb, 8, 3, c.w.batch_blocks)
+    real = max(0, min(c.nb, b0 + cnt) - b0)
+    fill = int(c.plan.tables()["block_fill"][b0:b0 + real].to(torch.int64).sum().item())
+    bb = c.tb * c.fb
+    dense = c.dense[:min(cnt, c.nb) * bb] if cnt * bb <= c.dense.numel() else torch.empty(cnt * bb, dtype=torch.uint8, device=c.dev)
+    ms_p = timed(lambda: B.bload_pack(c.plan, c.store, c.fb, b0, cnt, dense=dense))
+    k_p = B.bload_last_copy_kernel("pack")
+    obb = c.tb * c.ofb
+    dout = c.dense_out[:cnt * obb] if cnt * obb <= c.dense_out.numel() else torch.empty(cnt * obb, dtype=torch.uint8, device=c.dev)
+    ms_u = timed(lambda: B.bload_unpack(c.plan, dout, c.ofb, b0, cnt, c.ragged_out))
+    k_u = B.bload_last_copy_kernel("unpack")
+    return {"world": 8, "rank": 3, "block_begin": b0, "block_count": cnt, "frames": fill,
+            "pack": {"kernel": k_p, "ms": ms_p, "GB/s": (fill * c.fb + cnt * bb) / ms_p / 1e6},
+            "unpack": {"kernel": k_u, "ms": ms_u, "GB/s": 2 * fill * c.ofb / ms_u / 1e6}}
 
 
 def plan_figures(plan_ms, stage, n, clocks) -> dict:
@@ -846,6 +880,7 @@ def measure_config(args, w, dev, peak, clocks) -> dict:
                        "carry_prev": dict(rate(cp_bytes, carry_ms), kernel=k_carry),
                        "plan": plan_figures(sum(t_plan) / len(t_plan), stage, T.size, clocks)},
            "per_batch_pack": _time_per_batch(c),
+           "one_rank_of_eight": rank_share_figures(c, timed),
            "padding": {"n_blocks": st["n_blocks"], "min_blocks": st["min_blocks"], "frac_packed": st["frac_packed"],
                        "frac_naive_tmax": st["frac_naive_tmax"], "reduction_vs_tmax": st["reduction_vs_tmax"],
                        "chunking_strategy": chunk_strategy_figures(B, torch, d_len, tb)}}

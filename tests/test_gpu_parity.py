@@ -272,6 +272,47 @@ def test_one_launch_for_dense_blocks_and_metadata_of_small_frames(tb, fb, tmax):
     assert np.array_equal(dense.t.cpu().numpy().reshape(cnt, tb, fb), O.pack(op, store_h, fb, 0, cnt, 0))
 
 
+@pytest.mark.parametrize("tb,fb,kind", [(4096, 4, "tokens"), (2048, 8, "half"), (3072, 4, "half"), (1024, 16, "few_long"),
+                                        (4096, 4, "all_long"), (8192, 4, "four_per_block"), (1000, 20, "around_512"),
+                                        (333, 48, "half")])
+def test_unpack_of_block_ranges_of_small_frames(tb, fb, kind):
+    """Unpack of a block sub-range of small word-sized frames (the staged kernel over the dense side): run pieces of
+    512 bytes or more leave the stage with one bulk store from a place aligned like their destination, their first and
+    last words are copied directly, shorter pieces are scattered from the image of the sub-tile.  Plans that mix the
+    two kinds in every proportion, pieces just below and above the threshold, pieces cut by sub-tile ends, ranges that
+    start and end anywhere, filler blocks; every byte against the oracle, canaries around the output."""
+    rng = np.random.default_rng(tb * 3 + fb)
+    blocks = (24 << 20) // (tb * fb)
+    if kind == "tokens":
+        T = W.lengths(W.scaled(W.WORKLOADS["tokens"], int(blocks * 4.7)))
+    elif kind == "half":
+        T = np.where(rng.random(blocks) < 0.5, tb, rng.integers(1, 40, size=blocks))
+        T = np.concatenate([T, rng.integers(1, 40, size=blocks * 20)])
+    elif kind == "few_long":
+        T = np.concatenate([rng.integers(1, 24, size=blocks * 90), np.full(blocks // 50, tb)])
+    elif kind == "all_long":
+        T = np.full(blocks, tb)
+    elif kind == "four_per_block":
+        T = np.full(4 * blocks, tb // 4)
+    else:                                                   # run lengths around 512 bytes
+        T = rng.integers(max(1, 480 // fb), 560 // fb + 1, size=blocks * (tb * fb // 520))
+    T = rng.permutation(np.minimum(np.asarray(T), tb)).astype(np.int32)
+    op = O.plan(T, tb, 6); plan = G.gpu_plan(T, tb, 6)
+    nb = op.n_blocks
+    g = torch.Generator(device=G.DEV); g.manual_seed(tb)
+    for b0, cnt in ((1, nb - 2), (0, 3), (nb // 3, nb // 2), (nb - 2, 5)):
+        cnt = max(cnt, 1)
+        dense_out = torch.randint(0, 256, (cnt * tb * fb,), dtype=torch.uint8, device=G.DEV, generator=g)
+        rag = G.Guarded(op.sum_t * fb, 0x5A)
+        B.bload_unpack(plan, dense_out, fb, b0, cnt, rag.t)
+        torch.cuda.synchronize(); rag.check()
+        assert B.bload_last_copy_kernel("unpack") == "k8_unpack_staged"
+        want = np.full(op.sum_t * fb, 0x5A, np.uint8)
+        O.unpack(op, dense_out.cpu().numpy(), fb, b0, cnt, want)
+        d = G.first_diff(rag.t.cpu().numpy(), want)
+        assert d is None, "blocks [%d, +%d): %s" % (b0, cnt, d)
+
+
 @pytest.mark.parametrize("tb,fb,lengths", [(6, 4, [2, 2, 3, 3, 4, 5, 6, 6]), (7, 12, [1]), (9, 20, [9, 1, 1]),
                                            (5, 4, [1, 1, 1]), (3000, 4, None), (1234, 36, None)])
 def test_whole_plan_unpack_of_word_sized_frames(tb, fb, lengths):
