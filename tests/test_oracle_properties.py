@@ -76,3 +76,37 @@ def test_var_frames_round_trip_and_padding(t_block, data, seed, pad):
     back = np.zeros_like(store)
     O.unpack_var(p, dense, F, slot, 0, nb, back)
     assert np.array_equal(back, store)
+
+
+@settings(max_examples=120, deadline=None)
+@given(st.integers(1, 40), st.data(), st.integers(0, 1), st.integers(1, 12), st.integers(0, 2**32))
+def test_chunking_strategy_properties(t_chunk, data, tail, fb, seed):
+    """Any lengths and chunk length: every kept frame sits in exactly one chunk at the slot its position says, chunks
+    never cross a sequence, the two tails differ exactly by the short last chunks, and pack followed by unpack returns
+    the kept frames and leaves the deleted ones alone."""
+    T = np.array(data.draw(st.lists(st.integers(1, 3 * t_chunk + 2), min_size=1, max_size=40)), np.int32)
+    ch = O.chunks(T, t_chunk, tail)
+    assert ch.status == 0
+    T64 = T.astype(np.int64)
+    assert ch.frames_kept + ch.frames_deleted == int(T64.sum()) and ch.n_chunks * t_chunk == ch.frames_kept + ch.pad_frames
+    assert bool((ch.chunk_len >= 1).all()) and bool((ch.chunk_len <= t_chunk).all()) if ch.n_chunks else True
+    assert bool((ch.chunk_first % t_chunk == 0).all()) and bool((ch.chunk_first + ch.chunk_len <= T[ch.chunk_seq]).all())
+    if tail == O.DROP_TAIL:
+        assert ch.pad_frames == 0 and ch.frames_deleted == int((T64 % t_chunk).sum())
+    else:
+        assert ch.frames_deleted == 0 and ch.pad_frames == int(((-T64) % t_chunk).sum())
+    store = np.random.default_rng(seed).integers(0, 256, size=ch.sum_t * fb, dtype=np.uint8)
+    dense = O.chunk_pack(ch, store, fb, 0, ch.n_chunks + 1, 0xEE)
+    sid, pos, reset, valid = O.chunk_metadata(ch, 0, ch.n_chunks + 1)
+    assert int(valid.sum()) == ch.frames_kept and int(reset.sum()) == ch.n_chunks
+    assert np.all(dense[valid == 0] == 0xEE)
+    back = np.full(ch.sum_t * fb, 0x5A, np.uint8)
+    O.chunk_unpack(ch, dense, fb, 0, ch.n_chunks + 1, back)
+    kept = np.zeros(ch.sum_t, bool)
+    for j in range(ch.n_chunks):
+        a = int(ch.offsets[ch.chunk_seq[j]]) + int(ch.chunk_first[j])
+        assert not kept[a:a + ch.chunk_len[j]].any()
+        kept[a:a + ch.chunk_len[j]] = True
+    assert int(kept.sum()) == ch.frames_kept
+    b2, s2 = back.reshape(-1, fb), store.reshape(-1, fb)
+    assert np.array_equal(b2[kept], s2[kept]) and bool((b2[~kept] == 0x5A).all())
