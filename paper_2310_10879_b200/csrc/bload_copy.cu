@@ -101,7 +101,7 @@ __global__ void __launch_bounds__(256) k7_copy(PlanView pv, int32_t t_block, int
 //                      with 16-byte cp.async, scatter it to the ragged side with 16-byte stores.
 // The loads of item i are in flight while item i-1 is completed, and nothing waits on a flag: the only
 // waits are cp.async.wait_group / cp.async.bulk.wait_group, which end when the hardware copies end.
-// Requires frame_bytes % 4 == 0 (and, on the dense side, (t_block * frame_bytes) % 16 == 0).
+// Requires frame_bytes % 4 == 0 (and, for k8_unpack_staged, (t_block * frame_bytes) % 16 == 0).
 // Tuning of the two directions (swept on B200 with the 4-byte token workload): bytes per stage, warps
 // per CTA, stages per warp, consecutive sub-tiles of a block handled by one warp.  More, smaller stages
 // mean more resident warps; the kernels are limited by per-warp instruction latency, not by bytes in flight.
@@ -498,9 +498,11 @@ __global__ void __launch_bounds__(StageCfg<false>::kWarps * 32) k9_unpack_ragged
 
 // ------------------------------------------------------------------------------------------------
 // Pack for small word-sized frames with a contiguous range of dense sub-tiles per warp (the pack-side
-// twin of k9_unpack_ragged): the warp locates its first segment once and then walks forward through
-// the segment list, which runs on from one block to the next; only `fill` and the segment end of each
-// new block are read, one block ahead.  Blocks at or beyond n_blocks are written as padding.
+// twin of k9_unpack_ragged).  The dense side of the call is cut into sub-tiles as ONE array, whatever the
+// size of a block: a sub-tile may hold the end of one block, several whole small blocks and the start of
+// another, and a block may begin at any 4-byte offset.  The warp locates its first segment once and then
+// walks forward through the segment list, which runs on from one block to the next; only `fill` and the
+// segment end of each new block are read, one block ahead.  Blocks at or beyond n_blocks are written as padding.
 // META: the per-slot metadata of the same blocks comes out of the same launch.  The first `pack_ctas` CTAs pack; every
 // further CTA writes the metadata of 4 x blockDim.x consecutive slots of one block (the code of the metadata kernel).
 // A call for one training batch of small frames moves about a megabyte and is bound by launch overhead, so one launch
@@ -516,7 +518,7 @@ __global__ void __launch_bounds__(StageCfg<false>::kWarps * 32) k10_pack_contig(
                                                                               int64_t frame_bytes, int64_t block_begin,
                                                                               const uint8_t* __restrict__ store,
                                                                               uint8_t* __restrict__ dense, int64_t tiles,
-                                                                              int64_t tiles_per_warp, int32_t subs_per_block,
+                                                                              int64_t tiles_per_warp, int64_t total,
                                                                               uint8_t pad, MetaOut mo)
 {
     using Cfg = StageCfg<false>;
@@ -545,24 +547,36 @@ __global__ void __launch_bounds__(StageCfg<false>::kWarps * 32) k10_pack_contig(
     int64_t prev_off = 0;
     int prev_n = 0, s = 0, s_prev = 0;
     bool have_prev = false;
+    // a finished sub-tile leaves with one bulk copy; only the very last sub-tile of a call can end off a 16-byte
+    // boundary (total % 16 != 0), and its last words leave with plain stores
     auto complete = [&](int64_t off, int nbytes, uint8_t* stage) {
         fence_proxy_async();
         __syncwarp();
-        if (lane == 0) { bulk_store(dense + off, smem_addr(stage), (uint32_t)nbytes); bulk_commit(); }
+        const int nb16 = nbytes & ~15;
+        if (lane == 0 && nb16) { bulk_store(dense + off, smem_addr(stage), (uint32_t)nb16); bulk_commit(); }
+        if (lane < ((nbytes - nb16) >> 2)) put_word(dense + off + nb16 + 4 * lane, *reinterpret_cast<const uint32_t*>(stage + nb16 + 4 * lane));
     };
     const uint32_t p4 = 0x01010101u * pad;
+    // padding bytes [p, pe) of a stage (both multiples of 4): words up to a 16-byte boundary, vectors, words
+    auto fill_pad = [&](uint8_t* stage, int p, int pe) {
+        const int a = min((p + 15) & ~15, pe);
+        if (lane < ((a - p) >> 2)) *reinterpret_cast<uint32_t*>(stage + p + 4 * lane) = p4;
+        const int bnd = max(a, pe & ~15);
+        for (int o = a + 16 * lane; o < bnd; o += 512) *reinterpret_cast<uint4*>(stage + o) = make_uint4(p4, p4, p4, p4);
+        if (lane < ((pe - bnd) >> 2)) *reinterpret_cast<uint32_t*>(stage + bnd + 4 * lane) = p4;
+    };
     // the warp takes chunks of `tiles_per_warp` consecutive sub-tiles, chunk after chunk, grid-strided
     for (int64_t t_begin = gw * tiles_per_warp; t_begin < tiles; t_begin += n_warps * tiles_per_warp) {
     const int64_t t_end = min(t_begin + tiles_per_warp, tiles);
-    int64_t q = t_begin / subs_per_block;            // block of this call the warp is in
-    int sub = (int)(t_begin - q * subs_per_block);   // sub-tile inside it
+    const int64_t lo0 = t_begin * kStageBytes;
+    int64_t q = lo0 / block_bytes;                   // block of this call the warp starts in
+    int bo = (int)(q * block_bytes - lo0);           // where that block begins, relative to the sub-tile (<= 0 here)
     // current block: end of its segments and occupied bytes; the same two scalars of the next block
     int k1 = seg_end_of(block_begin + q), fill_bytes = fill_of(block_begin + q);
     int k1_next = seg_end_of(block_begin + q + 1), fill_next = fill_of(block_begin + q + 1);
     // position in the segment list and a window of 32 segments from kw (raw start slots, source frames)
     int k = (block_begin + q) < n_blocks ? pv.block_seg_begin[block_begin + q] : 0;
-    if (sub != 0 && sub * kStageBytes < fill_bytes)
-        k = warp_find_segment(pv.seg_start, k, k1, (sub * kStageBytes) / fb, lane);
+    if (bo != 0 && -bo < fill_bytes) k = warp_find_segment(pv.seg_start, k, k1, (-bo) / fb, lane);
     int kw = k, w_st = 0;
     int64_t w_src = 0;
     auto load_window = [&]() {
@@ -574,41 +588,45 @@ __global__ void __launch_bounds__(StageCfg<false>::kWarps * 32) k10_pack_contig(
     for (int64_t t = t_begin; t < t_end; ++t) {
         uint8_t* stage = my_stages + (size_t)s * kStageBytes;
         const uint32_t sa = smem_addr(stage);
-        const int lo = sub * kStageBytes;
-        const int nbytes = min(kStageBytes, block_bytes - lo);
-        const int valid = lo < fill_bytes ? min(nbytes, fill_bytes - lo) : 0;
+        const int64_t lo = t * kStageBytes;
+        const int nbytes = (int)min((int64_t)kStageBytes, total - lo);
         if (lane == 0) bulk_wait_read<NST - 2>();  // the store that last read this stage has finished reading
         __syncwarp();
-        int cur = lo;
-        const int hi = lo + valid;
-        while (cur < hi) {
-            if ((unsigned)(k - kw) >= 31u) { kw = k; load_window(); }
-            const int st = __shfl_sync(kFull, w_st, k - kw);
-            int nx = __shfl_sync(kFull, w_st, k - kw + 1);
-            const int64_t src = __shfl_sync(kFull, w_src, k - kw);
-            const int seg_e = (k + 1 < k1) ? nx * fb : fill_bytes;  // the block's last run ends where its frames end
-            const int pe = min(seg_e, hi);
-            warp_gather_async(sa + (uint32_t)(cur - lo), store + src * fb + (cur - st * fb), pe - cur, lane);
-            cur = pe;
-            if (pe == seg_e) ++k;
+        int p = 0;  // position in the sub-tile; the loop ends because every turn moves p or closes a block (block_bytes > 0)
+        while (p < nbytes) {
+            const int hi = min(bo + fill_bytes, nbytes);  // end of the block's frames, clipped
+            while (p < hi) {
+                if ((unsigned)(k - kw) >= 31u) { kw = k; load_window(); }
+                const int st = __shfl_sync(kFull, w_st, k - kw);
+                const int nx = __shfl_sync(kFull, w_st, k - kw + 1);
+                const int64_t src = __shfl_sync(kFull, w_src, k - kw);
+                const int seg_e = bo + ((k + 1 < k1) ? nx * fb : fill_bytes);  // the block's last run ends where its frames end
+                const int pe = min(seg_e, hi);
+                warp_gather_async(sa + (uint32_t)p, store + src * fb + (p - bo - st * fb), pe - p, lane);
+                p = pe;
+                if (pe == seg_e) ++k;
+            }
+            if (p < nbytes || bo + block_bytes == nbytes) {  // padding up to the end of the block, then the next block
+                const int blk_end = bo + block_bytes;
+                const int pe = min(blk_end, nbytes);
+                fill_pad(stage, p, pe);
+                p = pe;
+                if (pe == blk_end) {  // the next block's segments follow directly in the list
+                    ++q; bo = blk_end;
+                    k = k1;  // (already there unless the warp started inside the padding of the block it leaves)
+                    k1 = k1_next; fill_bytes = fill_next;
+                    k1_next = seg_end_of(block_begin + q + 1); fill_next = fill_of(block_begin + q + 1);
+                }
+            }
         }
-        // padding: words up to the next 16-byte boundary, then vectors (valid % 4 == 0, nbytes % 16 == 0)
-        const int firstv = min((valid + 15) & ~15, nbytes);
-        if (lane < ((firstv - valid) >> 2)) *reinterpret_cast<uint32_t*>(stage + valid + 4 * lane) = p4;
-        for (int o = firstv + 16 * lane; o < nbytes; o += 512) *reinterpret_cast<uint4*>(stage + o) = make_uint4(p4, p4, p4, p4);
+        bo -= nbytes;
         cp_async_commit();
         if (have_prev) {
             cp_async_wait<1>();
             complete(prev_off, prev_n, my_stages + (size_t)s_prev * kStageBytes);
         }
-        prev_off = q * (int64_t)block_bytes + lo; prev_n = nbytes; have_prev = true; s_prev = s;
+        prev_off = lo; prev_n = nbytes; have_prev = true; s_prev = s;
         s = (s + 1 == NST) ? 0 : s + 1;
-        if (++sub == subs_per_block) {  // next block: its segments follow directly in the list
-            sub = 0; ++q;
-            k = k1;  // (already there unless the warp started inside the padding of the block it leaves)
-            k1 = k1_next; fill_bytes = fill_next;
-            k1_next = seg_end_of(block_begin + q + 1); fill_next = fill_of(block_begin + q + 1);
-        }
     }
     }
     if (!have_prev) return;
@@ -806,16 +824,16 @@ bool staged_pack_with_metadata(const PlanView& pv, int32_t t_block, int64_t fram
     using Cfg = StageCfg<false>;
     const int64_t block_bytes = (int64_t)t_block * frame_bytes;
     constexpr int64_t kMaxFusedSlots = 1 << 22;  // beyond this the metadata kernel's own launch shape is faster
-    if (!(frame_bytes % 4 == 0 && n > 0 && ragged_bytes / n <= kStagedMaxRunBytes && block_bytes < (1LL << 31) &&
-          block_bytes % 16 == 0 && block_count * t_block <= kMaxFusedSlots))
+    if (!(frame_bytes % 4 == 0 && n > 0 && ragged_bytes / n <= kStagedMaxRunBytes && block_bytes < (1LL << 30) &&
+          block_count * t_block <= kMaxFusedSlots))
         return false;
     const size_t smem = (size_t)Cfg::kWarps * Cfg::kStages * Cfg::kBytes + 16;
     *err = opt_in_shared_memory(k10_pack_contig<true>, (int)smem);
     if (*err != cudaSuccess) return true;
     const DeviceInfo di = device_info();
     const int per_sm = (int)(di.smem_per_sm / (smem + 1024));
-    const int64_t spb = (block_bytes + Cfg::kBytes - 1) / Cfg::kBytes;
-    const int64_t tiles = block_count * spb;
+    const int64_t total = block_count * block_bytes;
+    const int64_t tiles = (total + Cfg::kBytes - 1) / Cfg::kBytes;
     const int64_t max_warps = (int64_t)di.sm_count * per_sm * Cfg::kWarps;
     int64_t tpw = (tiles + max_warps - 1) / max_warps;
     if (tpw > kPackChunkTiles) tpw = kPackChunkTiles;
@@ -836,7 +854,7 @@ bool staged_pack_with_metadata(const PlanView& pv, int32_t t_block, int64_t fram
     }
     note_copy_kernel(kCallPack, "k10_pack_contig<metadata>");
     k10_pack_contig<true><<<(unsigned)grid, Cfg::kWarps * 32, smem, st>>>(pv, (int32_t)n, t_block, frame_bytes, block_begin, store,
-                                                                        dense, tiles, tpw, (int32_t)spb, pad_byte, mo);
+                                                                        dense, tiles, tpw, total, pad_byte, mo);
     *err = cudaPeekAtLastError();
     return true;
 }
@@ -851,16 +869,16 @@ cudaError_t launch_copy(bool unpack, const PlanView& pv, int32_t t_block, int64_
     if (unpack) BLOAD_DBG_EXPECT(st, dbg::kCopy, {{dense, (size_t)(block_count * block_bytes)}}, {{ragged_out, (size_t)ragged_bytes}});
     else BLOAD_DBG_EXPECT(st, dbg::kCopy, {{ragged_in, (size_t)ragged_bytes}}, {{dense, (size_t)(block_count * block_bytes)}});
     // pack of small word-sized frames: contiguous ranges of dense sub-tiles per warp
-    const bool short_runs = frame_bytes % 4 == 0 && n > 0 && ragged_bytes / n <= kStagedMaxRunBytes && block_bytes < (1LL << 31);
-    if (!unpack && short_runs && block_bytes % 16 == 0) {
+    const bool short_runs = frame_bytes % 4 == 0 && n > 0 && ragged_bytes / n <= kStagedMaxRunBytes && block_bytes < (1LL << 30);
+    if (!unpack && short_runs) {
         using Cfg = StageCfg<false>;
         const size_t smem = (size_t)Cfg::kWarps * Cfg::kStages * Cfg::kBytes + 16;
         const DeviceInfo di = device_info();
         const int per_sm = (int)(di.smem_per_sm / (smem + 1024));
         cudaError_t e = opt_in_shared_memory(k10_pack_contig<false>, (int)smem);
         if (e != cudaSuccess) return e;
-        const int64_t spb = (block_bytes + Cfg::kBytes - 1) / Cfg::kBytes;
-        const int64_t tiles = block_count * spb;
+        const int64_t total = block_count * block_bytes;
+        const int64_t tiles = (total + Cfg::kBytes - 1) / Cfg::kBytes;  // of the dense side as one array: blocks begin anywhere
         const int64_t max_warps = (int64_t)di.sm_count * per_sm * Cfg::kWarps;
         int64_t tpw = (tiles + max_warps - 1) / max_warps;
         if (tpw > kPackChunkTiles) tpw = kPackChunkTiles;  // chunks are grid-strided beyond this size
@@ -868,7 +886,7 @@ cudaError_t launch_copy(bool unpack, const PlanView& pv, int32_t t_block, int64_
         if (warps > max_warps) warps = max_warps;
         const unsigned grid = (unsigned)((warps + Cfg::kWarps - 1) / Cfg::kWarps);
         k10_pack_contig<false><<<grid, Cfg::kWarps * 32, smem, st>>>(pv, (int32_t)n, t_block, frame_bytes, block_begin, ragged_in,
-                                                             dense, tiles, tpw, (int32_t)spb, pad_byte, MetaOut{});
+                                                             dense, tiles, tpw, total, pad_byte, MetaOut{});
         note_copy_kernel(kCallPack, "k10_pack_contig");
         return cudaPeekAtLastError();
     }

@@ -238,7 +238,32 @@ def test_small_word_sized_frames_take_the_staged_path(tb, fb, tmax):
         assert np.array_equal(res["dense"], O.pack(op, store.cpu().numpy(), fb, 1, 2, 0))
 
 
-@pytest.mark.parametrize("tb,fb,tmax", [(4096, 4, 4096), (64, 4, 64), (1000, 16, 9), (700, 256, 60), (36, 12, 36)])
+@pytest.mark.parametrize("tb,fb,tmax", [(94, 12, 94), (7, 12, 7), (94, 20, 94), (94, 100, 60), (5, 4, 5), (1, 4, 1), (3, 4, 3),
+                                        (1234, 36, 600), (4097, 4, 4097), (10001, 12, 2000), (2049, 8, 2049)])
+def test_pack_of_small_frames_in_blocks_of_any_size(tb, fb, tmax):
+    """The staged pack kernel cuts the dense side of a call into sub-tiles as one array, so blocks need not be multiples
+    of 16 bytes: blocks of 4 to 120,012 bytes that begin at every 4-byte offset, hundreds of blocks per sub-tile, blocks
+    cut by sub-tile ends inside their frames and inside their padding, calls whose total is not a multiple of 16 bytes
+    (the last words leave with plain stores), filler blocks, sub-ranges."""
+    assert (tb * fb) % 16 != 0
+    rng = np.random.default_rng(tb * 977 + fb)
+    n = int(min(6000, max(3, 6_000_000 // (tmax * fb))))
+    T = rng.integers(1, tmax + 1, size=n).astype(np.int32)
+    T[rng.integers(0, n)] = tmax
+    plan, op = G.full_parity(T, tb, 8, fb, out_fb=fb, pad=0x6B, extra_blocks=3)
+    assert B.bload_last_copy_kernel("pack").startswith("k10_pack_contig")
+    store = torch.randint(0, 256, (op.sum_t * fb,), dtype=torch.uint8, device=G.DEV)
+    store_h = store.cpu().numpy()
+    nb = op.n_blocks
+    for b0, cnt in [(0, 1), (1, 1), (nb // 2, 3), (nb - 1, 2), (0, nb), (nb // 3, nb // 2 + 1), (nb, 1)]:
+        res, _ = G.gpu_pack_all(plan, store, fb, b0, cnt, 0xD2, meta=False)
+        assert B.bload_last_copy_kernel("pack") == "k10_pack_contig"
+        d = G.first_diff(res["dense"].reshape(-1), O.pack(op, store_h, fb, b0, cnt, 0xD2).reshape(-1))
+        assert d is None, "blocks [%d, +%d): %s" % (b0, cnt, d)
+
+
+@pytest.mark.parametrize("tb,fb,tmax", [(4096, 4, 4096), (64, 4, 64), (1000, 16, 9), (700, 256, 60), (36, 12, 36), (94, 12, 94),
+                                        (5, 4, 5)])
 def test_one_launch_for_dense_blocks_and_metadata_of_small_frames(tb, fb, tmax):
     """A pack call that asks for dense blocks and metadata of small word-sized frames is ONE launch (some CTAs pack, the
     others write metadata).  Its outputs equal those of the two separate calls and the oracle's: sub-ranges, filler
@@ -276,11 +301,9 @@ def test_one_launch_for_dense_blocks_and_metadata_of_small_frames(tb, fb, tmax):
                                         (4096, 4, "all_long"), (8192, 4, "four_per_block"), (1000, 20, "around_512"),
                                         (333, 48, "half")])
 def test_unpack_of_block_ranges_of_small_frames(tb, fb, kind):
-    """Unpack of a block sub-range of small word-sized frames (the staged kernel over the dense side): run pieces of
-    512 bytes or more leave the stage with one bulk store from a place aligned like their destination, their first and
-    last words are copied directly, shorter pieces are scattered from the image of the sub-tile.  Plans that mix the
-    two kinds in every proportion, pieces just below and above the threshold, pieces cut by sub-tile ends, ranges that
-    start and end anywhere, filler blocks; every byte against the oracle, canaries around the output."""
+    """Unpack of a block sub-range of small word-sized frames (the staged kernel over the dense side).  Plans that mix
+    runs as long as a block and runs of a few frames in every proportion, runs around 512 bytes, runs cut by sub-tile
+    ends, ranges that start and end anywhere, filler blocks; every byte against the oracle, canaries around the output."""
     rng = np.random.default_rng(tb * 3 + fb)
     blocks = (24 << 20) // (tb * fb)
     if kind == "tokens":
