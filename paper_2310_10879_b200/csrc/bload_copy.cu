@@ -638,6 +638,257 @@ __global__ void __launch_bounds__(StageCfg<false>::kWarps * 32) k10_pack_contig(
 
 
 // ------------------------------------------------------------------------------------------------
+// Runs of a few hundred bytes or less (short sentences of token ids, per-frame labels of short clips).  The kernels
+// above hand one run at a time to the whole warp; with 40-word runs most lanes idle and the run's bookkeeping costs
+// more than its copy.  Here the sub-tile is walked by WORDS instead: lane l takes the words l, l+32, ... of the
+// stage-side array and finds the run of each of its words itself, in a window of 32 runs that the warp builds with one
+// lane per run and keeps in shared memory.  A window entry holds where the run begins and ends in the stage-side
+// array (relative to the first byte of the warp's range, clamped) and the distance from there to its source; a lane
+// only ever moves forward in the window.  Every word costs the same dozen instructions whatever the run lengths are.
+// Stages, completion and the sub-tile ranges per warp are those of k10_pack_contig / k9_unpack_ragged.
+constexpr int kShortWindowBytes = 32 * 16;
+constexpr int kFar = 0x7fffffff;  // "beyond the warp's range"
+#ifndef BLOAD_SHORT_RUN_WORDS
+#define BLOAD_SHORT_RUN_WORDS 128
+#endif
+#ifndef BLOAD_SHORT_CHUNK_TILES
+#define BLOAD_SHORT_CHUNK_TILES 4
+#endif
+constexpr int64_t kShortChunkTiles = BLOAD_SHORT_CHUNK_TILES;  // consecutive sub-tiles a warp packs before it jumps ahead
+// The word-wise kernels take the calls whose average run is at most this many words of 8 or 4 bytes, and every call of
+// the staged path whose frames are multiples of 16 bytes.  Measured on B200 against k10_pack_contig / k9_unpack_ragged
+// (pack / unpack, TB/s): 4-byte frames in 232-byte runs 2.66 / 3.30 against 2.41 / 2.27 and in 3.5 KB runs 4.4 / 5.3
+// against 5.9 / 6.1; 12-byte frames in 696-byte runs 3.7 / 4.5 against 4.7 / 4.6; 8-byte frames in 176-byte runs
+// 2.8 / 3.3 against 1.5 / 1.9, in 464-byte runs 4.1 / 4.3 against 3.9 / 3.9, in 6.9 KB runs 5.4 / 5.8 against 5.9 / 5.8;
+// 16-byte frames in 352-byte runs 4.6 / 5.0 against 3.0 / 3.5, 32-byte frames in 704-byte runs 5.6 / 5.5 against
+// 4.8 / 5.4, 16-byte frames in 14 KB runs 6.0 / 5.8 against 5.9 / 5.9.
+inline bool runs_are_short(int64_t ragged_bytes, int64_t n, int64_t frame_bytes)
+{
+    if (frame_bytes % 16 == 0) return true;
+    return ragged_bytes / n <= (int64_t)BLOAD_SHORT_RUN_WORDS * (frame_bytes % 8 == 0 ? 8 : 4);
+}
+__device__ __forceinline__ int clamp_far(int64_t v) { return v < 0 ? 0 : (v > (int64_t)kFar ? kFar : (int)v); }
+
+// words [p0, p1) of the range, for the stage that images the range from t0; win[r] = {begin, end, source minus
+// stage-side position (64 bit)}; r, e, delta, dn are the lane's place in the window.  A word is W = 16, 8 or 4 bytes, the
+// largest of them that divides the frame size: every run then begins and ends on a word boundary on both sides.
+template <int W>
+__device__ __forceinline__ void cp_async_word(uint32_t s, const void* g)
+{
+    if (W == 16) cp_async16(s, g);
+    else if (W == 8) cp_async8(s, g);
+    else cp_async4(s, g);
+}
+template <bool PAD, int W>
+__device__ __forceinline__ void walk_words(const int4* __restrict__ win, int& r, int& e, int64_t& delta, int& dn, int p0, int p1,
+                                           int t0, uint8_t* stage, const uint8_t* __restrict__ src, uint32_t p4, int lane)
+{
+    const uint32_t sa = smem_addr(stage);
+    for (int p = p0 + W * lane; p < p1; p += 32 * W) {
+        while (p >= dn) {  // (p < p1 <= begin of the window's last entry, so r + 1 <= 31)
+            ++r;
+            const int4 w = win[r];
+            e = w.y; delta = (int64_t)(((uint64_t)(uint32_t)w.w << 32) | (uint32_t)w.z);
+            dn = win[r + 1].x;
+        }
+        if (!PAD || p < e) cp_async_word<W>(sa + (uint32_t)(p - t0), src + delta + p);
+        else if (W == 16) *reinterpret_cast<uint4*>(stage + (p - t0)) = make_uint4(p4, p4, p4, p4);
+        else if (W == 8) *reinterpret_cast<uint2*>(stage + (p - t0)) = make_uint2(p4, p4);
+        else *reinterpret_cast<uint32_t*>(stage + (p - t0)) = p4;
+    }
+}
+
+template <bool META, int W>
+__global__ void __launch_bounds__(StageCfg<false>::kWarps * 32) k17_pack_short_runs(PlanView pv, int32_t n, int32_t t_block,
+                                                                                  int64_t frame_bytes, int64_t block_begin,
+                                                                                  const uint8_t* __restrict__ store,
+                                                                                  uint8_t* __restrict__ dense, int64_t tiles,
+                                                                                  int64_t tiles_per_warp, int64_t total,
+                                                                                  uint8_t pad, MetaOut mo)
+{
+    using Cfg = StageCfg<false>;
+    constexpr int NST = Cfg::kStages, kStageBytes = Cfg::kBytes, kStageWarps = Cfg::kWarps;
+    if (META && blockIdx.x >= mo.pack_ctas) {
+        const uint32_t m = blockIdx.x - mo.pack_ctas;
+        const uint32_t q = m / (uint32_t)mo.chunks_per_block;
+        const int s0 = (int)(m - q * (uint32_t)mo.chunks_per_block) * (kStageWarps * 32 * 4) + (int)threadIdx.x * 4;
+        if (s0 < t_block) {
+            const int64_t o = (int64_t)q * t_block + s0;
+            if (mo.vec) metadata_quad<true>(pv, t_block, block_begin + q, pv.hdr->n_blocks, s0, o, mo.seq_id, mo.pos, mo.reset, mo.valid);
+            else metadata_quad<false>(pv, t_block, block_begin + q, pv.hdr->n_blocks, s0, o, mo.seq_id, mo.pos, mo.reset, mo.valid);
+        }
+        return;
+    }
+    extern __shared__ __align__(128) uint8_t stage_mem[];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    uint8_t* my_stages = stage_mem + (size_t)warp * NST * kStageBytes;
+    int4* win = reinterpret_cast<int4*>(stage_mem + (size_t)kStageWarps * NST * kStageBytes + 16 + (size_t)warp * kShortWindowBytes);
+    const int64_t gw = (int64_t)blockIdx.x * kStageWarps + warp;
+    const int64_t n_warps = (int64_t)(META ? mo.pack_ctas : gridDim.x) * kStageWarps;
+    const int fb = (int)frame_bytes;
+    const int64_t block_bytes = (int64_t)t_block * fb;
+    const int64_t n_blocks = pv.hdr->n_blocks;
+    int64_t prev_off = 0;
+    int prev_n = 0, s = 0, s_prev = 0;
+    bool have_prev = false;
+    auto complete = [&](int64_t off, int nbytes, uint8_t* stage) {
+        fence_proxy_async();
+        __syncwarp();
+        const int nb16 = nbytes & ~15;
+        if (lane == 0 && nb16) { bulk_store(dense + off, smem_addr(stage), (uint32_t)nb16); bulk_commit(); }
+        if (lane < ((nbytes - nb16) >> 2)) put_word(dense + off + nb16 + 4 * lane, *reinterpret_cast<const uint32_t*>(stage + nb16 + 4 * lane));
+    };
+    const uint32_t p4 = 0x01010101u * pad;
+    for (int64_t t_begin = gw * tiles_per_warp; t_begin < tiles; t_begin += n_warps * tiles_per_warp) {
+        const int64_t t_end = min(t_begin + tiles_per_warp, tiles);
+        const int64_t lo0 = t_begin * kStageBytes;  // positions below are relative to this byte of the call's dense side
+        // the run that holds lo0 or, when lo0 lies in padding, the last run before it
+        int kw;
+        {
+            const int64_t q = lo0 / block_bytes, b = block_begin + q;
+            if (b >= n_blocks) kw = n - 1;
+            else {
+                const int k0 = pv.block_seg_begin[b], k1 = pv.block_seg_begin[b + 1];
+                const int64_t r0 = lo0 - q * block_bytes;
+                kw = r0 < (int64_t)pv.block_fill[b] * fb ? warp_find_segment(pv.seg_start, k0, k1, (int)(r0 / fb), lane) : k1 - 1;
+            }
+        }
+        int r = 0, e = 0, dn = 0, d_last = 0;
+        int64_t delta = 0;
+        // one lane per run: its place in the dense side, its length (up to the next run of the block, or to the end of the
+        // block's frames) and its source
+        auto load_window = [&]() {
+            const int k = kw + lane;
+            int4 w = make_int4(kFar, kFar, 0, 0);
+            if (k < n) {
+                const int blk = pv.seg_block[k], st = pv.seg_start[k];
+                const int nst = k + 1 < n ? pv.seg_start[k + 1] : 0;  // a later run of the same block starts later
+                const int e_slot = nst > st ? nst : pv.block_fill[blk];
+                const int64_t d_flat = (blk - block_begin) * block_bytes + (int64_t)st * fb - lo0;
+                const int64_t dl = pv.seg_src[k] * fb - d_flat;
+                w = make_int4(clamp_far(d_flat), clamp_far(d_flat + (int64_t)(e_slot - st) * fb), (int)(uint32_t)(uint64_t)dl,
+                              (int)(uint32_t)((uint64_t)dl >> 32));
+            }
+            __syncwarp();  // every lane has left the previous window
+            win[lane] = w;
+            __syncwarp();
+            const int4 w0 = win[0];
+            r = 0; e = w0.y; delta = (int64_t)(((uint64_t)(uint32_t)w0.w << 32) | (uint32_t)w0.z);
+            dn = win[1].x; d_last = win[31].x;
+        };
+        load_window();
+        for (int64_t t = t_begin; t < t_end; ++t) {
+            uint8_t* stage = my_stages + (size_t)s * kStageBytes;
+            const int64_t lo = t * kStageBytes;
+            const int nbytes = (int)min((int64_t)kStageBytes, total - lo);
+            const int t0 = (int)(lo - lo0), t1 = t0 + nbytes;
+            if (lane == 0) bulk_wait_read<NST - 2>();  // the store that last read this stage has finished reading
+            __syncwarp();
+            int done = t0;
+            while (done < t1) {  // ends: a turn reaches t1 or moves the window on by 31 runs that begin ever later
+                const int limit = min(t1, d_last);
+                walk_words<true, W>(win, r, e, delta, dn, done, limit, t0, stage, store, p4, lane);
+                done = limit;
+                if (limit == d_last) { kw += 31; load_window(); }
+            }
+            cp_async_commit();
+            if (have_prev) {
+                cp_async_wait<1>();
+                complete(prev_off, prev_n, my_stages + (size_t)s_prev * kStageBytes);
+            }
+            prev_off = lo; prev_n = nbytes; have_prev = true; s_prev = s;
+            s = (s + 1 == NST) ? 0 : s + 1;
+        }
+    }
+    if (!have_prev) return;
+    cp_async_wait<0>();
+    complete(prev_off, prev_n, my_stages + (size_t)s_prev * kStageBytes);
+    __syncwarp();
+    if (lane == 0) bulk_wait_read<0>();
+}
+
+// whole-plan unpack, the ragged side walked by words (see k9_unpack_ragged for the tiling): a window entry is one
+// sequence, which ends where the next begins
+template <int W>
+__global__ void __launch_bounds__(StageCfg<false>::kWarps * 32) k18_unpack_short_runs(PlanView pv, int32_t n, int32_t t_block,
+                                                                                    int64_t frame_bytes, int64_t sum_t,
+                                                                                    const uint8_t* __restrict__ dense,
+                                                                                    uint8_t* __restrict__ ragged,
+                                                                                    int64_t tiles, int64_t tiles_per_warp)
+{
+    using Cfg = StageCfg<false>;
+    constexpr int NST = Cfg::kStages, kStageBytes = Cfg::kBytes, kStageWarps = Cfg::kWarps;
+    extern __shared__ __align__(128) uint8_t stage_mem[];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    uint8_t* my_stages = stage_mem + (size_t)warp * NST * kStageBytes;
+    int4* win = reinterpret_cast<int4*>(stage_mem + (size_t)kStageWarps * NST * kStageBytes + 16 + (size_t)warp * kShortWindowBytes);
+    const int64_t gw = (int64_t)blockIdx.x * kStageWarps + warp;
+    const int64_t t_begin = gw * tiles_per_warp;
+    const int64_t t_end = min(t_begin + tiles_per_warp, tiles);
+    if (t_begin >= t_end) return;
+    const int64_t total = sum_t * frame_bytes;
+    const int64_t lo0 = t_begin * kStageBytes;  // positions below are relative to this byte of the ragged side
+    const int64_t block_bytes = (int64_t)t_block * frame_bytes;
+
+    int kw = warp_find_sequence(pv.offsets, n, lo0 / frame_bytes, lane);
+    int r = 0, e = 0, dn = 0, d_last = 0;
+    int64_t delta = 0;
+    auto load_window = [&]() {
+        const int i = kw + lane;
+        int4 w = make_int4(kFar, kFar, 0, 0);
+        if (i < n) {
+            const int64_t d_flat = pv.offsets[i] * frame_bytes - lo0;
+            const int64_t dl = pv.seq_block[i] * block_bytes + pv.seq_start[i] * frame_bytes - d_flat;
+            w = make_int4(clamp_far(d_flat), kFar, (int)(uint32_t)(uint64_t)dl, (int)(uint32_t)((uint64_t)dl >> 32));
+        }
+        __syncwarp();  // every lane has left the previous window
+        win[lane] = w;
+        __syncwarp();
+        const int4 w0 = win[0];
+        r = 0; e = w0.y; delta = (int64_t)(((uint64_t)(uint32_t)w0.w << 32) | (uint32_t)w0.z);
+        dn = win[1].x; d_last = win[31].x;
+    };
+    load_window();
+
+    int64_t prev_lo = 0;
+    int prev_n = 0, s = 0, s_prev = 0;
+    bool have_prev = false;
+    auto complete = [&](int64_t lo, int nbytes, uint8_t* stage) {
+        fence_proxy_async();
+        __syncwarp();
+        const int n16 = nbytes & ~15;
+        if (lane == 0 && n16) { bulk_store(ragged + lo, smem_addr(stage), (uint32_t)n16); bulk_commit(); }
+        if (lane < ((nbytes - n16) >> 2)) put_word(ragged + lo + n16 + 4 * lane, *reinterpret_cast<const uint32_t*>(stage + n16 + 4 * lane));
+    };
+    for (int64_t t = t_begin; t < t_end; ++t) {
+        uint8_t* stage = my_stages + (size_t)s * kStageBytes;
+        const int64_t lo = t * kStageBytes;
+        const int nbytes = (int)min((int64_t)kStageBytes, total - lo);
+        const int t0 = (int)(lo - lo0), t1 = t0 + nbytes;
+        if (lane == 0) bulk_wait_read<NST - 2>();  // the store that last read this stage has finished reading
+        __syncwarp();
+        int done = t0;
+        while (done < t1) {
+            const int limit = min(t1, d_last);
+            walk_words<false, W>(win, r, e, delta, dn, done, limit, t0, stage, dense, 0u, lane);
+            done = limit;
+            if (limit == d_last) { kw += 31; load_window(); }
+        }
+        cp_async_commit();
+        if (have_prev) {
+            cp_async_wait<1>();
+            complete(prev_lo, prev_n, my_stages + (size_t)s_prev * kStageBytes);
+        }
+        prev_lo = lo; prev_n = nbytes; have_prev = true; s_prev = s;
+        s = (s + 1 == NST) ? 0 : s + 1;
+    }
+    cp_async_wait<0>();
+    complete(prev_lo, prev_n, my_stages + (size_t)s_prev * kStageBytes);
+    __syncwarp();
+    if (lane == 0) bulk_wait_read<0>();
+}
+
+// ------------------------------------------------------------------------------------------------
 // Measurement variant, compiled only with -DBLOAD_BULK_COPY=1 (never in the default library): the large-frame path
 // through the bulk-copy engine instead of registers.  Frames whose size is a multiple of 16 bytes; a warp owns a ring
 // of shared-memory stages, each the image of one sub-tile of the dense side.  Pack: every run piece of the sub-tile
@@ -827,8 +1078,13 @@ bool staged_pack_with_metadata(const PlanView& pv, int32_t t_block, int64_t fram
     if (!(frame_bytes % 4 == 0 && n > 0 && ragged_bytes / n <= kStagedMaxRunBytes && block_bytes < (1LL << 30) &&
           block_count * t_block <= kMaxFusedSlots))
         return false;
-    const size_t smem = (size_t)Cfg::kWarps * Cfg::kStages * Cfg::kBytes + 16;
-    *err = opt_in_shared_memory(k10_pack_contig<true>, (int)smem);
+    const bool by_words = runs_are_short(ragged_bytes, n, frame_bytes);  // very short runs: the word-wise kernel
+    const size_t smem = (size_t)Cfg::kWarps * Cfg::kStages * Cfg::kBytes + 16 + (by_words ? (size_t)Cfg::kWarps * kShortWindowBytes : 0);
+    using PackKernel = void (*)(PlanView, int32_t, int32_t, int64_t, int64_t, const uint8_t*, uint8_t*, int64_t, int64_t, int64_t, uint8_t, MetaOut);
+    const PackKernel kernel = !by_words ? k10_pack_contig<true>
+                              : frame_bytes % 16 == 0 ? k17_pack_short_runs<true, 16>
+                              : frame_bytes % 8 == 0 ? k17_pack_short_runs<true, 8> : k17_pack_short_runs<true, 4>;
+    *err = opt_in_shared_memory(kernel, (int)smem);
     if (*err != cudaSuccess) return true;
     const DeviceInfo di = device_info();
     const int per_sm = (int)(di.smem_per_sm / (smem + 1024));
@@ -836,7 +1092,7 @@ bool staged_pack_with_metadata(const PlanView& pv, int32_t t_block, int64_t fram
     const int64_t tiles = (total + Cfg::kBytes - 1) / Cfg::kBytes;
     const int64_t max_warps = (int64_t)di.sm_count * per_sm * Cfg::kWarps;
     int64_t tpw = (tiles + max_warps - 1) / max_warps;
-    if (tpw > kPackChunkTiles) tpw = kPackChunkTiles;
+    if (tpw > (by_words ? kShortChunkTiles : kPackChunkTiles)) tpw = by_words ? kShortChunkTiles : kPackChunkTiles;
     int64_t warps = (tiles + tpw - 1) / tpw;
     if (warps > max_warps) warps = max_warps;
     auto al = [](const void* p, uintptr_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; };
@@ -852,9 +1108,9 @@ bool staged_pack_with_metadata(const PlanView& pv, int32_t t_block, int64_t fram
         BLOAD_DBG_EXPECT(st, dbg::kPackContig, {{store, (size_t)ragged_bytes}},
                          {{dense, (size_t)(block_count * block_bytes)}, {seq_id, 4 * slots}, {pos, 4 * slots}, {reset, slots}, {valid, slots}});
     }
-    note_copy_kernel(kCallPack, "k10_pack_contig<metadata>");
-    k10_pack_contig<true><<<(unsigned)grid, Cfg::kWarps * 32, smem, st>>>(pv, (int32_t)n, t_block, frame_bytes, block_begin, store,
-                                                                        dense, tiles, tpw, total, pad_byte, mo);
+    note_copy_kernel(kCallPack, by_words ? "k17_pack_short_runs<metadata>" : "k10_pack_contig<metadata>");
+    kernel<<<(unsigned)grid, Cfg::kWarps * 32, smem, st>>>(pv, (int32_t)n, t_block, frame_bytes, block_begin, store, dense, tiles, tpw,
+                                                         total, pad_byte, mo);
     *err = cudaPeekAtLastError();
     return true;
 }
@@ -872,38 +1128,63 @@ cudaError_t launch_copy(bool unpack, const PlanView& pv, int32_t t_block, int64_
     const bool short_runs = frame_bytes % 4 == 0 && n > 0 && ragged_bytes / n <= kStagedMaxRunBytes && block_bytes < (1LL << 30);
     if (!unpack && short_runs) {
         using Cfg = StageCfg<false>;
-        const size_t smem = (size_t)Cfg::kWarps * Cfg::kStages * Cfg::kBytes + 16;
+        const bool by_words = runs_are_short(ragged_bytes, n, frame_bytes);  // very short runs: the word-wise kernel
+        const size_t smem = (size_t)Cfg::kWarps * Cfg::kStages * Cfg::kBytes + 16 + (by_words ? (size_t)Cfg::kWarps * kShortWindowBytes : 0);
         const DeviceInfo di = device_info();
         const int per_sm = (int)(di.smem_per_sm / (smem + 1024));
-        cudaError_t e = opt_in_shared_memory(k10_pack_contig<false>, (int)smem);
+        using PackKernel = void (*)(PlanView, int32_t, int32_t, int64_t, int64_t, const uint8_t*, uint8_t*, int64_t, int64_t, int64_t, uint8_t, MetaOut);
+        const PackKernel kernel = !by_words ? k10_pack_contig<false>
+                                  : frame_bytes % 16 == 0 ? k17_pack_short_runs<false, 16>
+                                  : frame_bytes % 8 == 0 ? k17_pack_short_runs<false, 8> : k17_pack_short_runs<false, 4>;
+        cudaError_t e = opt_in_shared_memory(kernel, (int)smem);
         if (e != cudaSuccess) return e;
         const int64_t total = block_count * block_bytes;
         const int64_t tiles = (total + Cfg::kBytes - 1) / Cfg::kBytes;  // of the dense side as one array: blocks begin anywhere
         const int64_t max_warps = (int64_t)di.sm_count * per_sm * Cfg::kWarps;
         int64_t tpw = (tiles + max_warps - 1) / max_warps;
-        if (tpw > kPackChunkTiles) tpw = kPackChunkTiles;  // chunks are grid-strided beyond this size
+        if (tpw > (by_words ? kShortChunkTiles : kPackChunkTiles)) tpw = by_words ? kShortChunkTiles : kPackChunkTiles;  // grid-strided beyond
         int64_t warps = (tiles + tpw - 1) / tpw;
         if (warps > max_warps) warps = max_warps;
         const unsigned grid = (unsigned)((warps + Cfg::kWarps - 1) / Cfg::kWarps);
-        k10_pack_contig<false><<<grid, Cfg::kWarps * 32, smem, st>>>(pv, (int32_t)n, t_block, frame_bytes, block_begin, ragged_in,
-                                                             dense, tiles, tpw, total, pad_byte, MetaOut{});
-        note_copy_kernel(kCallPack, "k10_pack_contig");
+        kernel<<<grid, Cfg::kWarps * 32, smem, st>>>(pv, (int32_t)n, t_block, frame_bytes, block_begin, ragged_in, dense, tiles, tpw, total,
+                                                   pad_byte, MetaOut{});
+        note_copy_kernel(kCallPack, by_words ? "k17_pack_short_runs" : "k10_pack_contig");
         return cudaPeekAtLastError();
     }
     // whole-plan unpack of small word-sized frames: tile the (contiguous, fully written) ragged side
     // (not when frames between the plan's sequences belong to nobody: this path writes the whole ragged buffer)
     if (unpack && short_runs && !gaps && block_begin == 0 && block_count >= n_blocks && ragged_bytes > 0) {
         using Cfg = StageCfg<false>;
-        const size_t smem = (size_t)Cfg::kWarps * Cfg::kStages * Cfg::kBytes + 16;
+        const int64_t tiles = (ragged_bytes + Cfg::kBytes - 1) / Cfg::kBytes;
         const DeviceInfo di = device_info();
-        const int per_sm = (int)(di.smem_per_sm / (smem + 1024));
+        auto shape = [&](size_t smem, int64_t* tpw) {  // contiguous sub-tiles per warp; CTAs
+            const int per_sm = (int)(di.smem_per_sm / (smem + 1024));
+            const int64_t max_warps = (int64_t)di.sm_count * per_sm * Cfg::kWarps;
+            *tpw = (tiles + max_warps - 1) / max_warps;
+            const int64_t warps = (tiles + *tpw - 1) / *tpw;
+            return (unsigned)((warps + Cfg::kWarps - 1) / Cfg::kWarps);
+        };
+        size_t smem = (size_t)Cfg::kWarps * Cfg::kStages * Cfg::kBytes + 16;
+        int64_t tpw = 0;
+        // very short runs: the word-wise kernel (32-bit positions inside a warp's range)
+        if (runs_are_short(ragged_bytes, n, frame_bytes)) {
+            const size_t smem_w = smem + (size_t)Cfg::kWarps * kShortWindowBytes;
+            const unsigned grid = shape(smem_w, &tpw);
+            if (tpw * Cfg::kBytes < (1LL << 30)) {
+                using UnpackKernel = void (*)(PlanView, int32_t, int32_t, int64_t, int64_t, const uint8_t*, uint8_t*, int64_t, int64_t);
+                const UnpackKernel kernel = frame_bytes % 16 == 0 ? k18_unpack_short_runs<16>
+                                            : frame_bytes % 8 == 0 ? k18_unpack_short_runs<8> : k18_unpack_short_runs<4>;
+                cudaError_t e = opt_in_shared_memory(kernel, (int)smem_w);
+                if (e != cudaSuccess) return e;
+                kernel<<<grid, Cfg::kWarps * 32, smem_w, st>>>(pv, (int32_t)n, t_block, frame_bytes, ragged_bytes / frame_bytes, dense,
+                                                             ragged_out, tiles, tpw);
+                note_copy_kernel(kCallUnpack, "k18_unpack_short_runs");
+                return cudaPeekAtLastError();
+            }
+        }
         cudaError_t e = opt_in_shared_memory(k9_unpack_ragged, (int)smem);
         if (e != cudaSuccess) return e;
-        const int64_t tiles = (ragged_bytes + Cfg::kBytes - 1) / Cfg::kBytes;
-        const int64_t max_warps = (int64_t)di.sm_count * per_sm * Cfg::kWarps;
-        const int64_t tpw = (tiles + max_warps - 1) / max_warps;           // contiguous sub-tiles per warp
-        const int64_t warps = (tiles + tpw - 1) / tpw;
-        const unsigned grid = (unsigned)((warps + Cfg::kWarps - 1) / Cfg::kWarps);
+        const unsigned grid = shape(smem, &tpw);
         k9_unpack_ragged<<<grid, Cfg::kWarps * 32, smem, st>>>(pv, (int32_t)n, t_block, frame_bytes, ragged_bytes / frame_bytes,
                                                               dense, ragged_out, tiles, tpw);
         note_copy_kernel(kCallUnpack, "k9_unpack_ragged");

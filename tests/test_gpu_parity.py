@@ -238,6 +238,48 @@ def test_small_word_sized_frames_take_the_staged_path(tb, fb, tmax):
         assert np.array_equal(res["dense"], O.pack(op, store.cpu().numpy(), fb, 1, 2, 0))
 
 
+def _runs_are_short(sum_t, n, fb):
+    """Among the calls of the staged path the word-wise kernels take those whose frames are multiples of 16 bytes and
+    those whose runs average 128 words (of 8 or 4 bytes, whichever divides the frame size) or less."""
+    return fb % 16 == 0 or sum_t * fb // n <= 128 * (8 if fb % 8 == 0 else 4)
+
+
+@pytest.mark.parametrize("tb,fb,kind", [(4096, 4, "ones"), (4096, 4, "few_words"), (10000, 4, "heavy_tail"), (94, 8, "clips"),
+                                        (94, 12, "clips"), (512, 36, "few_words"), (64, 256, "ones"), (4096, 4, "some_long"),
+                                        (33, 4, "few_words"), (1000, 16, "one_sequence")])
+def test_runs_of_a_few_words(tb, fb, kind):
+    """Calls whose runs average 128 words or less take the word-wise kernels (a lane finds the run of each of its words
+    in a window of 32 runs): runs of one word (a window lasts 31 words), a few words, clip- and sentence-like lengths, a
+    few runs as long as a block among thousands of tiny ones, windows that end inside a sub-tile and at its end, warps
+    that start inside padding and inside filler blocks, totals that are not multiples of 16 bytes, sub-ranges."""
+    rng = np.random.default_rng(tb * 31 + fb)
+    if kind == "ones":
+        T = np.ones(30011, np.int64)
+    elif kind == "few_words":
+        T = rng.integers(1, 6, size=40003)
+    elif kind == "heavy_tail":
+        T = W.lengths(W.scaled(W.WORKLOADS["heavy_tail_bf16"], 60000))
+    elif kind == "clips":
+        T = W.lengths(W.scaled(W.WORKLOADS["video_dataset_shape"], 50000))
+    elif kind == "some_long":
+        T = np.concatenate([rng.integers(1, 9, size=60000), np.full(25, tb), rng.integers(tb // 2, tb, size=20)])
+    else:
+        T = np.array([7])
+    T = rng.permutation(np.minimum(T, tb)).astype(np.int32)
+    assert _runs_are_short(int(T.sum()), len(T), fb)
+    plan, op = G.full_parity(T, tb, 21, fb, out_fb=fb, pad=0xE1, extra_blocks=3)
+    assert B.bload_last_copy_kernel("pack").startswith("k17_pack_short_runs")
+    assert B.bload_last_copy_kernel("unpack") == "k18_unpack_short_runs"
+    store = torch.randint(0, 256, (op.sum_t * fb,), dtype=torch.uint8, device=G.DEV)
+    store_h = store.cpu().numpy()
+    nb = op.n_blocks
+    for b0, cnt in [(0, 1), (nb // 2, 3), (nb - 1, 3), (nb + 2, 2), (1, max(nb - 2, 1))]:
+        res, _ = G.gpu_pack_all(plan, store, fb, b0, cnt, 0x4D, meta=False)
+        assert B.bload_last_copy_kernel("pack") == "k17_pack_short_runs"
+        d = G.first_diff(res["dense"].reshape(-1), O.pack(op, store_h, fb, b0, cnt, 0x4D).reshape(-1))
+        assert d is None, "blocks [%d, +%d): %s" % (b0, cnt, d)
+
+
 @pytest.mark.parametrize("tb,fb,tmax", [(94, 12, 94), (7, 12, 7), (94, 20, 94), (94, 100, 60), (5, 4, 5), (1, 4, 1), (3, 4, 3),
                                         (1234, 36, 600), (4097, 4, 4097), (10001, 12, 2000), (2049, 8, 2049)])
 def test_pack_of_small_frames_in_blocks_of_any_size(tb, fb, tmax):
@@ -251,13 +293,15 @@ def test_pack_of_small_frames_in_blocks_of_any_size(tb, fb, tmax):
     T = rng.integers(1, tmax + 1, size=n).astype(np.int32)
     T[rng.integers(0, n)] = tmax
     plan, op = G.full_parity(T, tb, 8, fb, out_fb=fb, pad=0x6B, extra_blocks=3)
-    assert B.bload_last_copy_kernel("pack").startswith("k10_pack_contig")
+    short = _runs_are_short(op.sum_t, len(T), fb)
+    staged = "k17_pack_short_runs" if short else "k10_pack_contig"
+    assert B.bload_last_copy_kernel("pack").startswith(staged)
     store = torch.randint(0, 256, (op.sum_t * fb,), dtype=torch.uint8, device=G.DEV)
     store_h = store.cpu().numpy()
     nb = op.n_blocks
     for b0, cnt in [(0, 1), (1, 1), (nb // 2, 3), (nb - 1, 2), (0, nb), (nb // 3, nb // 2 + 1), (nb, 1)]:
         res, _ = G.gpu_pack_all(plan, store, fb, b0, cnt, 0xD2, meta=False)
-        assert B.bload_last_copy_kernel("pack") == "k10_pack_contig"
+        assert B.bload_last_copy_kernel("pack") == staged
         d = G.first_diff(res["dense"].reshape(-1), O.pack(op, store_h, fb, b0, cnt, 0xD2).reshape(-1))
         assert d is None, "blocks [%d, +%d): %s" % (b0, cnt, d)
 
@@ -279,7 +323,7 @@ def test_one_launch_for_dense_blocks_and_metadata_of_small_frames(tb, fb, tmax):
         before = B.bload_kernel_launches()
         res, _ = G.gpu_pack_all(plan, store, fb, b0, cnt, 0x3C)
         assert B.bload_kernel_launches() - before == 1
-        assert B.bload_last_copy_kernel("pack") == "k10_pack_contig<metadata>"
+        assert B.bload_last_copy_kernel("pack") == ("k17_pack_short_runs" if _runs_are_short(op.sum_t, len(T), fb) else "k10_pack_contig") + "<metadata>"
         assert np.array_equal(res["dense"], O.pack(op, store_h, fb, b0, cnt, 0x3C))
         for name, want in zip(("seq_id", "pos", "reset", "valid"), O.metadata(op, b0, cnt)):
             assert np.array_equal(res[name], want), name
