@@ -240,15 +240,15 @@ def test_small_word_sized_frames_take_the_staged_path(tb, fb, tmax):
 
 def _runs_are_short(sum_t, n, fb):
     """Among the calls of the staged path the word-wise kernels take those whose frames are multiples of 16 bytes and
-    those whose runs average 128 words (of 8 or 4 bytes, whichever divides the frame size) or less."""
-    return fb % 16 == 0 or sum_t * fb // n <= 128 * (8 if fb % 8 == 0 else 4)
+    those whose runs average 768 bytes or less."""
+    return fb % 16 == 0 or sum_t * fb // n <= 768
 
 
 @pytest.mark.parametrize("tb,fb,kind", [(4096, 4, "ones"), (4096, 4, "few_words"), (10000, 4, "heavy_tail"), (94, 8, "clips"),
                                         (94, 12, "clips"), (512, 36, "few_words"), (64, 256, "ones"), (4096, 4, "some_long"),
                                         (33, 4, "few_words"), (1000, 16, "one_sequence")])
 def test_runs_of_a_few_words(tb, fb, kind):
-    """Calls whose runs average 128 words or less take the word-wise kernels (a lane finds the run of each of its words
+    """Calls whose runs are short on average take the word-wise kernels (a lane finds the run of each of its words
     in a window of 32 runs): runs of one word (a window lasts 31 words), a few words, clip- and sentence-like lengths, a
     few runs as long as a block among thousands of tiny ones, windows that end inside a sub-tile and at its end, warps
     that start inside padding and inside filler blocks, totals that are not multiples of 16 bytes, sub-ranges."""
@@ -278,6 +278,17 @@ def test_runs_of_a_few_words(tb, fb, kind):
         assert B.bload_last_copy_kernel("pack") == "k17_pack_short_runs"
         d = G.first_diff(res["dense"].reshape(-1), O.pack(op, store_h, fb, b0, cnt, 0x4D).reshape(-1))
         assert d is None, "blocks [%d, +%d): %s" % (b0, cnt, d)
+        # the same range back: the word-wise walk along the dense side, canaries around the output
+        dense_out = torch.randint(0, 256, (cnt * tb * fb,), dtype=torch.uint8, device=G.DEV)
+        rag = G.Guarded(op.sum_t * fb, 0x5A)
+        B.bload_unpack(plan, dense_out, fb, b0, cnt, rag.t)
+        torch.cuda.synchronize(); rag.check()
+        if not (b0 == 0 and cnt >= nb):
+            assert B.bload_last_copy_kernel("unpack") == "k19_unpack_range_short_runs"
+        want = np.full(op.sum_t * fb, 0x5A, np.uint8)
+        O.unpack(op, dense_out.cpu().numpy(), fb, b0, cnt, want)
+        d = G.first_diff(rag.t.cpu().numpy(), want)
+        assert d is None, "unpack of blocks [%d, +%d): %s" % (b0, cnt, d)
 
 
 @pytest.mark.parametrize("tb,fb,tmax", [(94, 12, 94), (7, 12, 7), (94, 20, 94), (94, 100, 60), (5, 4, 5), (1, 4, 1), (3, 4, 3),
@@ -345,7 +356,8 @@ def test_one_launch_for_dense_blocks_and_metadata_of_small_frames(tb, fb, tmax):
                                         (4096, 4, "all_long"), (8192, 4, "four_per_block"), (1000, 20, "around_512"),
                                         (333, 48, "half")])
 def test_unpack_of_block_ranges_of_small_frames(tb, fb, kind):
-    """Unpack of a block sub-range of small word-sized frames (the staged kernel over the dense side).  Plans that mix
+    """Unpack of a block sub-range of small word-sized frames (the staged kernel over the dense side or, for short runs
+    and for frames that are multiples of 16 bytes, the word-wise walk along it).  Plans that mix
     runs as long as a block and runs of a few frames in every proportion, runs around 512 bytes, runs cut by sub-tile
     ends, ranges that start and end anywhere, filler blocks; every byte against the oracle, canaries around the output."""
     rng = np.random.default_rng(tb * 3 + fb)
@@ -373,7 +385,8 @@ def test_unpack_of_block_ranges_of_small_frames(tb, fb, kind):
         rag = G.Guarded(op.sum_t * fb, 0x5A)
         B.bload_unpack(plan, dense_out, fb, b0, cnt, rag.t)
         torch.cuda.synchronize(); rag.check()
-        assert B.bload_last_copy_kernel("unpack") == "k8_unpack_staged"
+        assert B.bload_last_copy_kernel("unpack") == ("k19_unpack_range_short_runs" if _runs_are_short(op.sum_t, len(T), fb)
+                                                      else "k8_unpack_staged")
         want = np.full(op.sum_t * fb, 0x5A, np.uint8)
         O.unpack(op, dense_out.cpu().numpy(), fb, b0, cnt, want)
         d = G.first_diff(rag.t.cpu().numpy(), want)
