@@ -902,6 +902,66 @@ def measure_config(args, w, dev, peak, clocks) -> dict:
 # and scaled by frames (traffic grows in proportion to the frames moved).  Reads equal the algorithmic bytes, writes are
 # slightly below them (the tail of the output is still in L2 when the kernel ends).  An entry is removed when its
 # kernel changes; a missing entry reports null.
+def frame_sweep(args) -> dict:
+    """Pack, whole-plan unpack and sub-range unpack across frame sizes and three shapes of length distribution (token
+    lengths, the heavy-tailed lengths, the clip lengths of the paper's dataset), about 1.5 GB per direction and case: which
+    kernel the library chooses and what it reaches.  Not a step of the benchmark; printed as its own JSON line."""
+    import torch
+    import paper_2310_10879_b200 as B
+    from paper_2310_10879_b200 import workloads as W
+    dev = torch.device("cuda:0")
+    peak, _ = measured_peak()
+    mean_len = {"tokens": 868.0, "heavy_tail_bf16": 57.8, "video_dataset_shape": 22.3}
+    sizes = [int(x) for x in args.frame_sweep.split(",")] if args.frame_sweep != "default" else \
+        [1, 2, 4, 6, 8, 12, 16, 20, 24, 32, 48, 64, 100, 128, 250, 256, 512, 1024, 4096, 4100, 12288, 150528]
+
+    def timed(fn, reps=5):
+        for _ in range(3):
+            fn()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        a.record()
+        for _ in range(reps):
+            fn()
+        b.record()
+        torch.cuda.synchronize()
+        return a.elapsed_time(b) / reps
+
+    rows = []
+    for name in ("tokens", "heavy_tail_bf16", "video_dataset_shape"):
+        base = W.WORKLOADS[name]
+        for fb in sizes:
+            n = int(min(2_000_000, max(16, 1.5e9 / (mean_len[name] * fb))))
+            w = W.scaled(base, n)
+            T = W.lengths(w)
+            tb = w.t_block
+            if int(T.sum()) * fb < 2.5e8:  # below twice the L2 size the figures say little about HBM
+                continue
+            plan = B.bload_plan(torch.from_numpy(T).to(dev), tb, w.seed)
+            nb, st = plan.n_blocks, plan.sum_t
+            g = torch.Generator(device=dev)
+            g.manual_seed(fb)
+            store = torch.randint(0, 256, (st * fb,), dtype=torch.uint8, device=dev, generator=g)
+            dense = torch.empty(nb * tb * fb, dtype=torch.uint8, device=dev)
+            back = torch.zeros_like(store)
+            ms_p = timed(lambda: B.bload_pack(plan, store, fb, 0, nb, dense=dense))
+            k_p = B.bload_last_copy_kernel("pack")
+            ms_u = timed(lambda: B.bload_unpack(plan, dense, fb, 0, nb, back))
+            k_u = B.bload_last_copy_kernel("unpack")
+            row = {"lengths": name, "frame_bytes": fb, "n": n, "n_blocks": nb, "mean_run_bytes": round(st * fb / n),
+                   "store_MB": round(st * fb / 1e6), "round_trip_ok": bool(torch.equal(back, store)),
+                   "pack": {"kernel": k_p, "GB/s": round((st * fb + nb * tb * fb) / ms_p / 1e6), "frac_measured": round((st * fb + nb * tb * fb) / ms_p / 1e6 / peak, 3)},
+                   "unpack": {"kernel": k_u, "GB/s": round(2 * st * fb / ms_u / 1e6), "frac_measured": round(2 * st * fb / ms_u / 1e6 / peak, 3)}}
+            if nb > 2 and (tb * fb) % 16 == 0:  # all blocks but the first (the buffer of a sub-range is 16-byte aligned)
+                ms_s = timed(lambda: B.bload_unpack(plan, dense[tb * fb:], fb, 1, nb - 1, back))
+                gbs = 2 * st * fb * (nb - 1) / nb / ms_s / 1e6
+                row["unpack_sub_range"] = {"kernel": B.bload_last_copy_kernel("unpack"), "GB/s": round(gbs), "frac_measured": round(gbs / peak, 3)}
+            rows.append(row)
+            del store, dense, back, plan
+            torch.cuda.empty_cache()
+    return {"frame_sweep": rows, "peak_GB/s": peak, "unit": "GB/s of algorithmic bytes (pack: frames read + blocks written; unpack: frames read + written)"}
+
+
 TRAFFIC: dict = {
     ("heavy_tail_bf16", "k7_copy<unpack>"): 18.29e9,
     ("heavy_tail_bf16", "k7_copy<pack>"): 9.08e9,
@@ -931,7 +991,13 @@ def main():
     ap.add_argument("--no-consumer", action="store_true")
     ap.add_argument("--no-fused", action="store_true")
     ap.add_argument("--no-by-config", action="store_true", help="skip the extra measurements of the other large workloads")
+    ap.add_argument("--frame-sweep", default="", metavar="SIZES",
+                    help="instead of the benchmark: pack / unpack throughput and the kernel chosen across frame sizes "
+                         "('default' or a comma-separated list of bytes) and three length distributions; one JSON line")
     args = ap.parse_args()
+    if args.frame_sweep:
+        print(json.dumps(frame_sweep(args)), flush=True)
+        return
     args.warmup = max(args.warmup, 3) if args.impl == "bload" else args.warmup
 
     global POLICY

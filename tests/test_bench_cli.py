@@ -22,3 +22,20 @@ def test_reference_arm_prints_one_json_line():
     assert d["cpu_baseline"]["kind"] == "oracle" and d["cpu_baseline"]["cores"] == 1 and "sample" in d["cpu_baseline"]
     assert d["e2e"]["h2d_bytes_per_step"] == 0 and d["e2e"]["value"] == d["value"]
     assert "workload" in d["config"] and d["steps"] == 2
+
+
+import pytest
+
+
+@pytest.mark.gpu
+def test_frame_sweep_prints_one_json_line():
+    """`bench.py --frame-sweep SIZES` replaces the benchmark by a sweep over frame sizes; every case round-trips."""
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--frame-sweep", "8,256"], capture_output=True,
+                         text=True, timeout=600)
+    assert out.returncode == 0, out.stderr[-2000:]
+    lines = [l for l in out.stdout.splitlines() if l.strip()]
+    assert len(lines) == 1
+    rows = json.loads(lines[0])["frame_sweep"]
+    assert len(rows) >= 5 and all(r["round_trip_ok"] for r in rows)
+    assert {r["frame_bytes"] for r in rows} == {8, 256}
+    assert all(r["pack"]["GB/s"] > 0 and r["unpack"]["GB/s"] > 0 for r in rows)
