@@ -680,7 +680,7 @@ inline bool runs_are_short(int64_t ragged_bytes, int64_t n, int64_t frame_bytes)
 }
 __device__ __forceinline__ int clamp_far(int64_t v) { return v < 0 ? 0 : (v > (int64_t)kFar ? kFar : (int)v); }
 
-// words [p0, p1) of the range, for the stage that images the range from t0; win[r] = {begin, end, source minus
+// words [p0, p1) of the range, for the stage that images the range from t0; win[r] = {begin of run r+1, end, source minus
 // stage-side position (64 bit)}; r, e, delta, dn are the lane's place in the window.  A word is W = 16, 8 or 4 bytes, the
 // largest of them that divides the frame size: every run then begins and ends on a word boundary on both sides.
 template <int W>
@@ -696,11 +696,10 @@ __device__ __forceinline__ void walk_words(const int4* __restrict__ win, int& r,
 {
     const uint32_t sa = smem_addr(stage);
     for (int p = p0 + W * lane; p < p1; p += 32 * W) {
-        while (p >= dn) {  // (p < p1 <= begin of the window's last entry, so r + 1 <= 31)
+        while (p >= dn) {  // (p < p1 <= begin of the window's last entry, so r stays below 31)
             ++r;
-            const int4 w = win[r];
-            e = w.y; delta = (int64_t)(((uint64_t)(uint32_t)w.w << 32) | (uint32_t)w.z);
-            dn = win[r + 1].x;
+            const int4 w = win[r];  // {begin of the next run, end, source minus position}
+            dn = w.x; e = w.y; delta = (int64_t)(((uint64_t)(uint32_t)w.w << 32) | (uint32_t)w.z);
         }
         if (!PAD || p < e) cp_async_word<W>(sa + (uint32_t)(p - t0), src + delta + p);
         else if (W == 16) *reinterpret_cast<uint4*>(stage + (p - t0)) = make_uint4(p4, p4, p4, p4);
@@ -785,11 +784,11 @@ __global__ void __launch_bounds__(ShortCfg<W>::kWarps * 32) k17_pack_short_runs(
         auto load_window = [&]() {  // one lane per run
             const int4 w = dense_side_entry(pv, n, kw + lane, block_begin, block_bytes, fb, lo0);
             __syncwarp();  // every lane has left the previous window
-            win[lane] = w;
+            d_last = __shfl_sync(kFull, w.x, 31);
+            win[lane] = make_int4(__shfl_down_sync(kFull, w.x, 1), w.y, w.z, w.w);  // (lane 31's entry is never walked)
             __syncwarp();
             const int4 w0 = win[0];
-            r = 0; e = w0.y; delta = (int64_t)(((uint64_t)(uint32_t)w0.w << 32) | (uint32_t)w0.z);
-            dn = win[1].x; d_last = win[31].x;
+            r = 0; dn = w0.x; e = w0.y; delta = (int64_t)(((uint64_t)(uint32_t)w0.w << 32) | (uint32_t)w0.z);
         };
         load_window();
         for (int64_t t = t_begin; t < t_end; ++t) {
@@ -857,11 +856,11 @@ __global__ void __launch_bounds__(ShortCfg<W>::kWarps * 32) k18_unpack_short_run
             w = make_int4(clamp_far(d_flat), kFar, (int)(uint32_t)(uint64_t)dl, (int)(uint32_t)((uint64_t)dl >> 32));
         }
         __syncwarp();  // every lane has left the previous window
-        win[lane] = w;
+        d_last = __shfl_sync(kFull, w.x, 31);
+        win[lane] = make_int4(__shfl_down_sync(kFull, w.x, 1), w.y, w.z, w.w);  // (lane 31's entry is never walked)
         __syncwarp();
         const int4 w0 = win[0];
-        r = 0; e = w0.y; delta = (int64_t)(((uint64_t)(uint32_t)w0.w << 32) | (uint32_t)w0.z);
-        dn = win[1].x; d_last = win[31].x;
+        r = 0; dn = w0.x; e = w0.y; delta = (int64_t)(((uint64_t)(uint32_t)w0.w << 32) | (uint32_t)w0.z);
     };
     load_window();
 
@@ -945,11 +944,11 @@ __global__ void __launch_bounds__(256) k19_unpack_range_short_runs(PlanView pv, 
         auto load_window = [&]() {  // one lane per run
             const int4 w = dense_side_entry(pv, n, kw + lane, block_begin, block_bytes, fb, lo0);
             __syncwarp();  // every lane has left the previous window
-            win[lane] = w;
+            d_last = __shfl_sync(kFull, w.x, 31);
+            win[lane] = make_int4(__shfl_down_sync(kFull, w.x, 1), w.y, w.z, w.w);  // (lane 31's entry is never walked)
             __syncwarp();
             const int4 w0 = win[0];
-            r = 0; e = w0.y; delta = (int64_t)(((uint64_t)(uint32_t)w0.w << 32) | (uint32_t)w0.z);
-            dn = win[1].x; d_last = win[31].x;
+            r = 0; dn = w0.x; e = w0.y; delta = (int64_t)(((uint64_t)(uint32_t)w0.w << 32) | (uint32_t)w0.z);
         };
         load_window();
         const uint8_t* src = dense + lo0;
@@ -965,11 +964,10 @@ __global__ void __launch_bounds__(256) k19_unpack_range_short_runs(PlanView pv, 
                     const int q = p + u * 32 * W;
                     ok[u] = false;
                     if (q < limit) {
-                        while (q >= dn) {  // (q < limit <= begin of the window's last entry, so r + 1 <= 31)
+                        while (q >= dn) {  // (q < limit <= begin of the window's last entry, so r stays below 31)
                             ++r;
-                            const int4 w = win[r];
-                            e = w.y; delta = (int64_t)(((uint64_t)(uint32_t)w.w << 32) | (uint32_t)w.z);
-                            dn = win[r + 1].x;
+                            const int4 w = win[r];  // {begin of the next run, end, source minus position}
+                            dn = w.x; e = w.y; delta = (int64_t)(((uint64_t)(uint32_t)w.w << 32) | (uint32_t)w.z);
                         }
                         ok[u] = q < e;
                         to[u] = delta + q;
