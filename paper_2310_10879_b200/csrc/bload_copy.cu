@@ -1170,7 +1170,7 @@ bool staged_pack_with_metadata(const PlanView& pv, int32_t t_block, int64_t fram
 {
     const int64_t block_bytes = (int64_t)t_block * frame_bytes;
     constexpr int64_t kMaxFusedSlots = 1 << 22;  // beyond this the metadata kernel's own launch shape is faster
-    if (!(frame_bytes % 4 == 0 && n > 0 && ragged_bytes / n <= kStagedMaxRunBytes && block_bytes < (1LL << 30) &&
+    if (!(frame_bytes % 4 == 0 && n > 0 && n < 0x7fffff00LL && ragged_bytes / n <= kStagedMaxRunBytes && block_bytes < (1LL << 30) &&
           block_count * t_block <= kMaxFusedSlots))
         return false;
     const bool by_words = runs_are_short(ragged_bytes, n, frame_bytes);  // very short runs: the word-wise kernel
@@ -1221,7 +1221,9 @@ cudaError_t launch_copy(bool unpack, const PlanView& pv, int32_t t_block, int64_
     if (unpack) BLOAD_DBG_EXPECT(st, dbg::kCopy, {{dense, (size_t)(block_count * block_bytes)}}, {{ragged_out, (size_t)ragged_bytes}});
     else BLOAD_DBG_EXPECT(st, dbg::kCopy, {{ragged_in, (size_t)ragged_bytes}}, {{dense, (size_t)(block_count * block_bytes)}});
     // pack of small word-sized frames: contiguous ranges of dense sub-tiles per warp
-    const bool short_runs = frame_bytes % 4 == 0 && n > 0 && ragged_bytes / n <= kStagedMaxRunBytes && block_bytes < (1LL << 30);
+    // (the staged kernels index windows of 32 runs past a 32-bit position in the segment list)
+    const bool short_runs = frame_bytes % 4 == 0 && n > 0 && n < 0x7fffff00LL && ragged_bytes / n <= kStagedMaxRunBytes &&
+                            block_bytes < (1LL << 30);
     if (!unpack && short_runs) {
         const bool by_words = runs_are_short(ragged_bytes, n, frame_bytes);  // very short runs: the word-wise kernel
         const StagedShape Cfg = !by_words ? shape_of<StageCfg<false>>() : frame_bytes % 16 == 0 ? shape_of<ShortCfg<16>>() : shape_of<ShortCfg<4>>();
