@@ -217,7 +217,7 @@ BLOAD_API int bload_epoch_stage_times(float out_ms[5]);
  * d_store and d_dense must be 16-byte aligned.  d_dense and each of the four metadata outputs may be
  * NULL (that output is skipped).  Asynchronous on `stream`; no host synchronisation.  Launches: one kernel for the
  * metadata and one for the dense blocks; a call that asks for both, for small word-sized frames (frame_bytes a multiple
- * of 4, runs of at most 16 KB on average, t_block * frame_bytes a multiple of 16) and at most 4 Mi slots, is a single
+ * of 4, runs of at most 16 KB on average, blocks of less than 1 GiB) and at most 4 Mi slots, is a single
  * launch -- the call a training loop makes per batch of token-sized frames is bound by launch overhead, not by bytes.
  * Errors: NULL plan/info/store (when d_dense is given), ARG (frame_bytes < 1, negative range,
  * block_begin + block_count >= 2^31), ALIGN, PLAN (info->status != 0), CUDA.
@@ -515,7 +515,8 @@ BLOAD_API int bload_debug_status(uint64_t out[4], int clear);
  * bload_last_copy_kernel -- name of the copy kernel that the most recent call of this host thread launched for
  * which = 0 bload_pack (the dense output), 1 bload_unpack, 2 bload_carry_prev, 3 bload_pack_var[2d],
  * 4 bload_unpack_var[2d].  The library picks a kernel from the frame size and the run lengths (register path for
- * large frames, shared-memory staged paths for small word-sized frames); a benchmark reports the choice with this
+ * large frames, shared-memory staged paths for small word-sized frames, run by run or -- for short runs -- word by
+ * word); a benchmark reports the choice with this
  * call instead of guessing it.  Host only.  Returns "" when no such call was made, or for another `which`.
  */
 BLOAD_API const char* bload_last_copy_kernel(int which);
