@@ -663,9 +663,10 @@ constexpr int kFar = 0x7fffffff;  // "beyond the warp's range"
 #define BLOAD_SHORT_CHUNK_TILES 4
 #endif
 constexpr int64_t kShortChunkTiles = BLOAD_SHORT_CHUNK_TILES;  // consecutive sub-tiles a warp packs before it jumps ahead
-// The word-wise kernels take every call of the staged path whose frames are multiples of 16 bytes and, for narrower
-// words, the calls whose average run is at most BLOAD_SHORT_RUN bytes.  Measured on B200 against k10_pack_contig /
-// k9_unpack_ragged (pack / unpack, TB/s; word-wise first):
+// Short runs for the staged kernels: the word-wise ones (k17, k18) instead of the run-by-run ones (k10, k9).  Frames that
+// are multiples of 8 bytes no longer reach these kernels through bload_pack / bload_unpack without metadata (the unstaged
+// walks below are faster: see walks_unstaged); the single-launch pack with metadata still uses k17 for them, with 16-
+// or 8-byte words.  Measured on B200 against k10_pack_contig / k9_unpack_ragged (pack / unpack, TB/s; word-wise first):
 //   16-byte words: 16-byte frames in 352-byte runs 4.6 / 5.0 against 3.0 / 3.5, 32-byte frames in 704-byte runs 5.6 / 5.5
 //     against 4.8 / 5.4, 64-byte frames in 3.7 KB runs 6.0 / 5.9 against 5.9 / 5.8, 16-byte frames in 14 KB runs 6.0 / 5.8
 //     against 5.9 / 5.9;
@@ -902,10 +903,14 @@ __global__ void __launch_bounds__(ShortCfg<W>::kWarps * 32) k18_unpack_short_run
     if (lane == 0) bulk_wait_read<0>();
 }
 
-// Unpack of a block sub-range with short runs: the same walk along the dense side, without a stage.  A lane loads
-// each of its words from the dense side (lanes read consecutive words: coalesced) and stores it to the word's place in
-// the ragged output (consecutive inside a run); words of padding are skipped.
+// The same walk along the dense side without a stage, in either direction.  Unpack (block sub-ranges with short runs):
+// a lane loads each of its words from the dense side (lanes read consecutive words: coalesced) and stores it to the
+// word's place in the ragged output (consecutive inside a run); words of padding are skipped.  Pack: the word comes from
+// its place in the ragged store, or is padding, and goes to the dense side.  Words of 2 bytes and 1 byte serve frames
+// that are not multiples of 4 bytes, which cp.async (4 bytes at least) cannot move.
 template <int W> struct WordOf { using type = uint32_t; };
+template <> struct WordOf<1> { using type = unsigned char; };
+template <> struct WordOf<2> { using type = unsigned short; };
 template <> struct WordOf<8> { using type = uint2; };
 template <> struct WordOf<16> { using type = uint4; };
 template <int W>
@@ -920,12 +925,20 @@ __device__ __forceinline__ void store_word(uint8_t* p, typename WordOf<W>::type 
     using T = typename WordOf<W>::type;
     if (BLOAD_MAY_WRITE(p, W)) __stcs(reinterpret_cast<T*>(p), v);
 }
+template <int W>
+__device__ __forceinline__ typename WordOf<W>::type pad_word(uint32_t p4)
+{
+    using T = typename WordOf<W>::type;
+    if constexpr (W == 16) return make_uint4(p4, p4, p4, p4);
+    else if constexpr (W == 8) return make_uint2(p4, p4);
+    else return (T)p4;
+}
 
 constexpr int kRangeChunkBytes = 16384;  // of the dense side per warp and turn
-template <int W>
-__global__ void __launch_bounds__(256) k19_unpack_range_short_runs(PlanView pv, int32_t n, int32_t t_block, int64_t frame_bytes,
-                                                                   int64_t block_begin, const uint8_t* __restrict__ dense,
-                                                                   uint8_t* __restrict__ ragged, int64_t total)
+template <int W, bool PACK>
+__global__ void __launch_bounds__(256) k19_walk_dense_side(PlanView pv, int32_t n, int32_t t_block, int64_t frame_bytes,
+                                                           int64_t block_begin, const uint8_t* __restrict__ from,
+                                                           uint8_t* __restrict__ to_base, int64_t total, uint8_t pad)
 {
     __shared__ int4 windows[8][32];
     constexpr int U = W == 16 ? 4 : 8;  // words in flight per lane (4-byte words, 232-byte runs: 2 -> 2.54, 4 -> 2.68, 8 -> 2.78 TB/s)
@@ -935,6 +948,7 @@ __global__ void __launch_bounds__(256) k19_unpack_range_short_runs(PlanView pv, 
     const int64_t block_bytes = (int64_t)t_block * fb;
     const int64_t n_blocks = pv.hdr->n_blocks;
     const int64_t chunks = (total + kRangeChunkBytes - 1) / kRangeChunkBytes;
+    const uint32_t p4 = 0x01010101u * pad;
     for (int64_t c = (int64_t)blockIdx.x * 8 + warp; c < chunks; c += (int64_t)gridDim.x * 8) {
         const int64_t lo0 = c * kRangeChunkBytes;  // positions below are relative to this byte of the call's dense side
         const int p_end = (int)min((int64_t)kRangeChunkBytes, total - lo0);
@@ -951,13 +965,15 @@ __global__ void __launch_bounds__(256) k19_unpack_range_short_runs(PlanView pv, 
             r = 0; dn = w0.x; e = w0.y; delta = (int64_t)(((uint64_t)(uint32_t)w0.w << 32) | (uint32_t)w0.z);
         };
         load_window();
-        const uint8_t* src = dense + lo0;
+        // the dense side of the chunk is read (unpack) or written (pack); the ragged side is the other one
+        const uint8_t* dense_in = from + lo0;
+        uint8_t* dense_out = to_base + lo0;
         int done = 0;
         while (done < p_end) {  // ends: a turn reaches p_end or moves the window on by 31 runs that begin ever later
             const int limit = min(p_end, d_last);
             for (int p = done + W * lane; p < limit; p += 32 * W * U) {
-                int64_t to[U];
-                bool ok[U];
+                int64_t at[U];   // the word's place on the ragged side
+                bool ok[U];      // the word belongs to a run
                 typename WordOf<W>::type v[U];
 #pragma unroll
                 for (int u = 0; u < U; ++u) {
@@ -970,18 +986,131 @@ __global__ void __launch_bounds__(256) k19_unpack_range_short_runs(PlanView pv, 
                             dn = w.x; e = w.y; delta = (int64_t)(((uint64_t)(uint32_t)w.w << 32) | (uint32_t)w.z);
                         }
                         ok[u] = q < e;
-                        to[u] = delta + q;
+                        at[u] = delta + q;
                     }
                 }
+                if (PACK) {
 #pragma unroll
-                for (int u = 0; u < U; ++u) if (ok[u]) v[u] = load_word<W>(src + p + u * 32 * W);
+                    for (int u = 0; u < U; ++u) v[u] = ok[u] ? load_word<W>(from + at[u]) : pad_word<W>(p4);
 #pragma unroll
-                for (int u = 0; u < U; ++u) if (ok[u]) store_word<W>(ragged + to[u], v[u]);
+                    for (int u = 0; u < U; ++u) if (p + u * 32 * W < limit) store_word<W>(dense_out + p + u * 32 * W, v[u]);
+                } else {
+#pragma unroll
+                    for (int u = 0; u < U; ++u) if (ok[u]) v[u] = load_word<W>(dense_in + p + u * 32 * W);
+#pragma unroll
+                    for (int u = 0; u < U; ++u) if (ok[u]) store_word<W>(to_base + at[u], v[u]);
+                }
             }
             done = limit;
             if (limit == d_last) { kw += 31; load_window(); }
         }
     }
+}
+// Whole-plan unpack by the same unstaged walk, along the RAGGED side: a window entry is one sequence (it ends where the
+// next begins), a lane loads each of its words from the word's place in the dense buffer and stores it in place; the
+// stores are contiguous across the warp, the loads inside a run.
+template <int W>
+__global__ void __launch_bounds__(256) k21_unpack_walk_ragged(PlanView pv, int32_t n, int32_t t_block, int64_t frame_bytes,
+                                                              int64_t sum_t, const uint8_t* __restrict__ dense,
+                                                              uint8_t* __restrict__ ragged)
+{
+    __shared__ int4 windows[8][32];
+    constexpr int U = W == 16 ? 4 : 8;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    int4* win = windows[warp];
+    const int64_t total = sum_t * frame_bytes;
+    const int64_t block_bytes = (int64_t)t_block * frame_bytes;
+    const int64_t chunks = (total + kRangeChunkBytes - 1) / kRangeChunkBytes;
+    for (int64_t c = (int64_t)blockIdx.x * 8 + warp; c < chunks; c += (int64_t)gridDim.x * 8) {
+        const int64_t lo0 = c * kRangeChunkBytes;  // positions below are relative to this byte of the ragged side
+        const int p_end = (int)min((int64_t)kRangeChunkBytes, total - lo0);
+        int kw = warp_find_sequence(pv.offsets, n, lo0 / frame_bytes, lane);
+        int r = 0, dn = 0, d_last = 0;
+        int64_t delta = 0;
+        auto load_window = [&]() {  // one lane per sequence
+            const int i = kw + lane;
+            int4 w = make_int4(kFar, kFar, 0, 0);
+            if (i < n) {
+                const int64_t d_flat = pv.offsets[i] * frame_bytes - lo0;
+                const int64_t dl = pv.seq_block[i] * block_bytes + pv.seq_start[i] * frame_bytes - d_flat;
+                w = make_int4(clamp_far(d_flat), kFar, (int)(uint32_t)(uint64_t)dl, (int)(uint32_t)((uint64_t)dl >> 32));
+            }
+            __syncwarp();  // every lane has left the previous window
+            d_last = __shfl_sync(kFull, w.x, 31);
+            win[lane] = make_int4(__shfl_down_sync(kFull, w.x, 1), w.y, w.z, w.w);  // (lane 31's entry is never walked)
+            __syncwarp();
+            const int4 w0 = win[0];
+            r = 0; dn = w0.x; delta = (int64_t)(((uint64_t)(uint32_t)w0.w << 32) | (uint32_t)w0.z);
+        };
+        load_window();
+        uint8_t* out = ragged + lo0;
+        int done = 0;
+        while (done < p_end) {  // ends: a turn reaches p_end or moves the window on by 31 sequences that begin ever later
+            const int limit = min(p_end, d_last);
+            for (int p = done + W * lane; p < limit; p += 32 * W * U) {
+                int64_t at[U];
+                typename WordOf<W>::type v[U];
+#pragma unroll
+                for (int u = 0; u < U; ++u) {
+                    const int q = p + u * 32 * W;
+                    if (q < limit) {
+                        while (q >= dn) {  // (q < limit <= begin of the window's last entry, so r stays below 31)
+                            ++r;
+                            const int4 w = win[r];
+                            dn = w.x; delta = (int64_t)(((uint64_t)(uint32_t)w.w << 32) | (uint32_t)w.z);
+                        }
+                        at[u] = delta + q;
+                    }
+                }
+#pragma unroll
+                for (int u = 0; u < U; ++u) if (p + u * 32 * W < limit) v[u] = load_word<W>(dense + at[u]);
+#pragma unroll
+                for (int u = 0; u < U; ++u) if (p + u * 32 * W < limit) store_word<W>(out + p + u * 32 * W, v[u]);
+            }
+            done = limit;
+            if (limit == d_last) { kw += 31; load_window(); }
+        }
+    }
+}
+using WalkRaggedKernel = void (*)(PlanView, int32_t, int32_t, int64_t, int64_t, const uint8_t*, uint8_t*);
+inline WalkRaggedKernel walk_ragged_kernel_for(int64_t frame_bytes)
+{
+    return frame_bytes % 16 == 0 ? k21_unpack_walk_ragged<16> : frame_bytes % 8 == 0 ? k21_unpack_walk_ragged<8>
+           : frame_bytes % 4 == 0 ? k21_unpack_walk_ragged<4> : frame_bytes % 2 == 0 ? k21_unpack_walk_ragged<2>
+                                                                                     : k21_unpack_walk_ragged<1>;
+}
+
+using WalkKernel = void (*)(PlanView, int32_t, int32_t, int64_t, int64_t, const uint8_t*, uint8_t*, int64_t, uint8_t);
+template <bool PACK>
+WalkKernel walk_kernel_for(int64_t frame_bytes)
+{
+    return frame_bytes % 16 == 0 ? k19_walk_dense_side<16, PACK> : frame_bytes % 8 == 0 ? k19_walk_dense_side<8, PACK>
+           : frame_bytes % 4 == 0 ? k19_walk_dense_side<4, PACK> : frame_bytes % 2 == 0 ? k19_walk_dense_side<2, PACK>
+                                                                                        : k19_walk_dense_side<1, PACK>;
+}
+// Which calls take the unstaged walks (k19 along the dense side: pack and block sub-ranges; k21 along the ragged side:
+// whole-plan unpack).  Measured on B200 over three length distributions, about 1.5 GB per case (TB/s, pack / whole-plan
+// unpack, walk against the best of the staged kernels or the register path):
+//   16-byte words: 16-byte frames in 352-byte runs 5.04 / 4.91 against 4.59 / 4.96; 32-byte frames in 1.9 KB runs
+//     6.03 / 6.08 against 5.86 / 5.56; 256-byte frames in 15 KB runs 6.28 / 6.45 against 5.96 / 6.24; 16-byte frames in 14 KB
+//     runs 6.22 / 6.37 against 5.88 / 6.06
+//   8-byte words: 8-byte frames in 176-byte runs 3.92 / 3.83 against 3.36 / 3.40, in 464-byte runs 5.07 / 5.00 against
+//     4.45 / 4.42, in 6.9 KB runs 6.22 / 6.20 against 5.83 / 5.75; 24-byte frames in 1.4 KB runs 5.90 / 5.80 against 5.58 / 5.37
+//   4-byte words: 4-byte frames in 232-byte runs 3.61 / 3.66 against 3.59 / 3.65 (word-wise staged), 20-byte frames in
+//     1.2 KB runs 4.93 / 4.98 against 5.25 / 5.25 (run by run), 4-byte frames in 3.5 KB runs 5.19 / 5.30 against 5.87 / 6.08:
+//     the staged kernels keep the frames that are multiples of 4 but not of 8 bytes
+//   2-byte words (frames that are even but not multiples of 4; against the register path): 6-byte frames in 133-byte runs
+//     2.24 / 2.23 against 0.46 / 0.71, in 346-byte runs 2.85 / 2.95 against 1.26 / 1.88; 30-byte frames in 669-byte runs
+//     3.16 / 3.24 against 1.68 / 2.34, in 1.7 KB runs 3.34 / 3.52 against 3.06 / 3.79; 2-byte frames in 1.7 KB runs 3.36 / 3.55
+//     against 3.66 / 4.20
+//   1-byte words (odd frame sizes): 3-byte frames in 173-byte runs 1.49 / 1.56 against 0.73 / 1.15; 1-byte frames in
+//     870-byte runs 1.87 / 2.07 against 2.51 / 3.23
+inline bool walks_unstaged(int64_t frame_bytes, int64_t mean_run, bool unpack)
+{
+    if (frame_bytes % 8 == 0) return mean_run <= kStagedMaxRunBytes;
+    if (frame_bytes % 4 == 0) return false;
+    if (frame_bytes % 2 == 0) return mean_run <= (unpack ? 1024 : 1536);
+    return mean_run <= 384;
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -1220,20 +1349,46 @@ cudaError_t launch_copy(bool unpack, const PlanView& pv, int32_t t_block, int64_
     count_launches(1);
     if (unpack) BLOAD_DBG_EXPECT(st, dbg::kCopy, {{dense, (size_t)(block_count * block_bytes)}}, {{ragged_out, (size_t)ragged_bytes}});
     else BLOAD_DBG_EXPECT(st, dbg::kCopy, {{ragged_in, (size_t)ragged_bytes}}, {{dense, (size_t)(block_count * block_bytes)}});
+    // Which family moves the frames (measured cross-overs beside walks_unstaged and runs_are_short):
+    //   unstaged word-wise walks   frames that are multiples of 8 bytes in runs of at most 16 KB on average; frames that
+    //                              are not multiples of 4 bytes in short runs; 4-byte-word frames in short runs when a
+    //                              block sub-range is unpacked
+    //   staged, word by word       frames that are multiples of 4 (not 8) bytes in runs of at most 768 bytes
+    //   staged, run by run         the other frames that are multiples of 4 bytes, in runs of at most 16 KB
+    //   register path              everything else
+    // (the staged kernels and the walks index windows of 32 runs past a 32-bit position in the segment list)
+    const bool indexable = n > 0 && n < 0x7fffff00LL && block_bytes < (1LL << 30);
+    const int64_t mean_run = n > 0 ? ragged_bytes / n : 0;
+    const bool short_runs = frame_bytes % 4 == 0 && indexable && mean_run <= kStagedMaxRunBytes;
+    const bool whole_plan = unpack && !gaps && block_begin == 0 && block_count >= n_blocks && ragged_bytes > 0;
+    const bool by_words = short_runs && runs_are_short(ragged_bytes, n, frame_bytes);
+    if (indexable && (walks_unstaged(frame_bytes, mean_run, unpack) || (by_words && unpack && !whole_plan))) {
+        const int64_t cap = (int64_t)device_info().sm_count * 32;
+        if (whole_plan) {  // along the ragged side, which is contiguous and written completely
+            const WalkRaggedKernel kernel = walk_ragged_kernel_for(frame_bytes);
+            const int64_t want = ((ragged_bytes + kRangeChunkBytes - 1) / kRangeChunkBytes + 7) / 8;
+            kernel<<<(unsigned)(want < cap ? want : cap), 256, 0, st>>>(pv, (int32_t)n, t_block, frame_bytes, ragged_bytes / frame_bytes,
+                                                                        dense, ragged_out);
+            note_copy_kernel(kCallUnpack, "k21_unpack_walk_ragged");
+            return cudaPeekAtLastError();
+        }
+        const WalkKernel kernel = unpack ? walk_kernel_for<false>(frame_bytes) : walk_kernel_for<true>(frame_bytes);
+        const int64_t total = block_count * block_bytes;
+        const int64_t want = ((total + kRangeChunkBytes - 1) / kRangeChunkBytes + 7) / 8;
+        kernel<<<(unsigned)(want < cap ? want : cap), 256, 0, st>>>(pv, (int32_t)n, t_block, frame_bytes, block_begin,
+                                                                    unpack ? dense : ragged_in, unpack ? ragged_out : dense, total, pad_byte);
+        note_copy_kernel(unpack ? kCallUnpack : kCallPack, unpack ? "k19_unpack_walk_dense" : "k19_pack_walk_dense");
+        return cudaPeekAtLastError();
+    }
     // pack of small word-sized frames: contiguous ranges of dense sub-tiles per warp
-    // (the staged kernels index windows of 32 runs past a 32-bit position in the segment list)
-    const bool short_runs = frame_bytes % 4 == 0 && n > 0 && n < 0x7fffff00LL && ragged_bytes / n <= kStagedMaxRunBytes &&
-                            block_bytes < (1LL << 30);
     if (!unpack && short_runs) {
-        const bool by_words = runs_are_short(ragged_bytes, n, frame_bytes);  // very short runs: the word-wise kernel
-        const StagedShape Cfg = !by_words ? shape_of<StageCfg<false>>() : frame_bytes % 16 == 0 ? shape_of<ShortCfg<16>>() : shape_of<ShortCfg<4>>();
+        // (frames that are multiples of 8 bytes went to the walks above: words of 4 bytes here)
+        const StagedShape Cfg = by_words ? shape_of<ShortCfg<4>>() : shape_of<StageCfg<false>>();
         const size_t smem = (size_t)Cfg.kWarps * Cfg.kStages * Cfg.kBytes + 16 + (by_words ? (size_t)Cfg.kWarps * kShortWindowBytes : 0);
         const DeviceInfo di = device_info();
         const int per_sm = (int)(di.smem_per_sm / (smem + 1024));
         using PackKernel = void (*)(PlanView, int32_t, int32_t, int64_t, int64_t, const uint8_t*, uint8_t*, int64_t, int64_t, int64_t, uint8_t, MetaOut);
-        const PackKernel kernel = !by_words ? k10_pack_contig<false>
-                                  : frame_bytes % 16 == 0 ? k17_pack_short_runs<false, 16>
-                                  : frame_bytes % 8 == 0 ? k17_pack_short_runs<false, 8> : k17_pack_short_runs<false, 4>;
+        const PackKernel kernel = by_words ? k17_pack_short_runs<false, 4> : k10_pack_contig<false>;
         cudaError_t e = opt_in_shared_memory(kernel, (int)smem);
         if (e != cudaSuccess) return e;
         const int64_t total = block_count * block_bytes;
@@ -1251,58 +1406,28 @@ cudaError_t launch_copy(bool unpack, const PlanView& pv, int32_t t_block, int64_
     }
     // whole-plan unpack of small word-sized frames: tile the (contiguous, fully written) ragged side
     // (not when frames between the plan's sequences belong to nobody: this path writes the whole ragged buffer)
-    if (unpack && short_runs && !gaps && block_begin == 0 && block_count >= n_blocks && ragged_bytes > 0) {
+    if (whole_plan && short_runs) {
         const DeviceInfo di = device_info();
-        int64_t tiles = 0, tpw = 0;
-        auto shape = [&](const StagedShape& c, size_t smem) {  // sub-tiles, contiguous sub-tiles per warp; returns the CTAs
-            tiles = (ragged_bytes + c.kBytes - 1) / c.kBytes;
-            const int per_sm = (int)(di.smem_per_sm / (smem + 1024));
-            const int64_t max_warps = (int64_t)di.sm_count * per_sm * c.kWarps;
-            tpw = (tiles + max_warps - 1) / max_warps;
-            const int64_t warps = (tiles + tpw - 1) / tpw;
-            return (unsigned)((warps + c.kWarps - 1) / c.kWarps);
-        };
-        // very short runs: the word-wise kernel (32-bit positions inside a warp's range); with 16-byte words and runs of
-        // 2 KB or more the unstaged walk along the dense side (below) is 2-4 % faster still
-        if (runs_are_short(ragged_bytes, n, frame_bytes) && !(frame_bytes % 16 == 0 && ragged_bytes / n >= 2048)) {
-            const StagedShape c = frame_bytes % 16 == 0 ? shape_of<ShortCfg<16>>() : shape_of<ShortCfg<4>>();
-            const size_t smem_w = (size_t)c.kWarps * c.kStages * c.kBytes + 16 + (size_t)c.kWarps * kShortWindowBytes;
-            const unsigned grid = shape(c, smem_w);
-            if (tpw * c.kBytes < (1LL << 30)) {
-                using UnpackKernel = void (*)(PlanView, int32_t, int32_t, int64_t, int64_t, const uint8_t*, uint8_t*, int64_t, int64_t);
-                const UnpackKernel kernel = frame_bytes % 16 == 0 ? k18_unpack_short_runs<16>
-                                            : frame_bytes % 8 == 0 ? k18_unpack_short_runs<8> : k18_unpack_short_runs<4>;
-                cudaError_t e = opt_in_shared_memory(kernel, (int)smem_w);
-                if (e != cudaSuccess) return e;
-                kernel<<<grid, c.kWarps * 32, smem_w, st>>>(pv, (int32_t)n, t_block, frame_bytes, ragged_bytes / frame_bytes, dense,
-                                                          ragged_out, tiles, tpw);
-                note_copy_kernel(kCallUnpack, "k18_unpack_short_runs");
-                return cudaPeekAtLastError();
-            }
-        }
-        if (!runs_are_short(ragged_bytes, n, frame_bytes)) {
-            const StagedShape c = shape_of<StageCfg<false>>();
-            const size_t smem = (size_t)c.kWarps * c.kStages * c.kBytes + 16;
-            cudaError_t e = opt_in_shared_memory(k9_unpack_ragged, (int)smem);
+        const StagedShape c = by_words ? shape_of<ShortCfg<4>>() : shape_of<StageCfg<false>>();
+        const size_t smem = (size_t)c.kWarps * c.kStages * c.kBytes + 16 + (by_words ? (size_t)c.kWarps * kShortWindowBytes : 0);
+        const int64_t tiles = (ragged_bytes + c.kBytes - 1) / c.kBytes;
+        const int per_sm = (int)(di.smem_per_sm / (smem + 1024));
+        const int64_t max_warps = (int64_t)di.sm_count * per_sm * c.kWarps;
+        const int64_t tpw = (tiles + max_warps - 1) / max_warps;  // contiguous sub-tiles per warp
+        const int64_t warps = (tiles + tpw - 1) / tpw;
+        const unsigned grid = (unsigned)((warps + c.kWarps - 1) / c.kWarps);
+        // (the word-wise kernel keeps 32-bit positions inside a warp's range)
+        const bool words = by_words && tpw * c.kBytes < (1LL << 30);
+        using UnpackKernel = void (*)(PlanView, int32_t, int32_t, int64_t, int64_t, const uint8_t*, uint8_t*, int64_t, int64_t);
+        const UnpackKernel kernel = words ? k18_unpack_short_runs<4> : k9_unpack_ragged;
+        if (words || !by_words) {
+            cudaError_t e = opt_in_shared_memory(kernel, (int)smem);
             if (e != cudaSuccess) return e;
-            const unsigned grid = shape(c, smem);
-            k9_unpack_ragged<<<grid, c.kWarps * 32, smem, st>>>(pv, (int32_t)n, t_block, frame_bytes, ragged_bytes / frame_bytes,
-                                                               dense, ragged_out, tiles, tpw);
-            note_copy_kernel(kCallUnpack, "k9_unpack_ragged");
+            kernel<<<grid, c.kWarps * 32, smem, st>>>(pv, (int32_t)n, t_block, frame_bytes, ragged_bytes / frame_bytes, dense, ragged_out,
+                                                    tiles, tpw);
+            note_copy_kernel(kCallUnpack, words ? "k18_unpack_short_runs" : "k9_unpack_ragged");
             return cudaPeekAtLastError();
         }
-    }
-    // block sub-ranges with short runs, unpack direction: word-wise walk along the dense side
-    if (unpack && short_runs && runs_are_short(ragged_bytes, n, frame_bytes)) {
-        using RangeKernel = void (*)(PlanView, int32_t, int32_t, int64_t, int64_t, const uint8_t*, uint8_t*, int64_t);
-        const RangeKernel kernel = frame_bytes % 16 == 0 ? k19_unpack_range_short_runs<16>
-                                   : frame_bytes % 8 == 0 ? k19_unpack_range_short_runs<8> : k19_unpack_range_short_runs<4>;
-        const int64_t total = block_count * block_bytes;
-        const int64_t want = ((total + kRangeChunkBytes - 1) / kRangeChunkBytes + 7) / 8;
-        const int64_t cap = (int64_t)device_info().sm_count * 32;
-        kernel<<<(unsigned)(want < cap ? want : cap), 256, 0, st>>>(pv, (int32_t)n, t_block, frame_bytes, block_begin, dense, ragged_out, total);
-        note_copy_kernel(kCallUnpack, "k19_unpack_range_short_runs");
-        return cudaPeekAtLastError();
     }
     // block sub-ranges of small word-sized frames, unpack direction: staged kernel over the dense side
     if (unpack && short_runs && block_bytes % 16 == 0) {

@@ -130,3 +130,26 @@ def full_parity(lengths: np.ndarray, t_block: int, seed: int, fb: int, out_fb: i
     back.check()
     assert torch.equal(back.t, store)
     return plan, op
+
+
+def expected_copy_kernels(sum_t: int, n: int, fb: int, t_block: int) -> dict:
+    """Which kernel the library is documented to choose for a call (the rules stated beside launch_copy): `pack` and
+    `unpack` for whole-plan calls without metadata, `unpack_range` for a block sub-range, `pack_meta` for a pack call
+    that also asks for metadata and holds at most 4 Mi slots."""
+    run = sum_t * fb // n
+    if fb % 4 == 0 and run <= 16384:
+        words = run <= 768
+        if fb % 8 == 0:
+            plain = dict(pack="k19_pack_walk_dense", unpack="k21_unpack_walk_ragged", unpack_range="k19_unpack_walk_dense")
+        elif words:
+            plain = dict(pack="k17_pack_short_runs", unpack="k18_unpack_short_runs", unpack_range="k19_unpack_walk_dense")
+        else:
+            plain = dict(pack="k10_pack_contig", unpack="k9_unpack_ragged",
+                         unpack_range="k8_unpack_staged" if (t_block * fb) % 16 == 0 else "k7_copy<unpack>")
+        plain["pack_meta"] = ("k17_pack_short_runs" if (fb % 16 == 0 or words) else "k10_pack_contig") + "<metadata>"
+        return plain
+    if fb % 4 != 0 and ((fb % 2 == 0 and run <= 1536) or run <= 384):
+        up = run <= (1024 if fb % 2 == 0 else 384)
+        return dict(pack="k19_pack_walk_dense", unpack="k21_unpack_walk_ragged" if up else "k7_copy<unpack>",
+                    unpack_range="k19_unpack_walk_dense" if up else "k7_copy<unpack>", pack_meta="k19_pack_walk_dense")
+    return dict(pack="k7_copy<pack>", unpack="k7_copy<unpack>", unpack_range="k7_copy<unpack>", pack_meta="k7_copy<pack>")

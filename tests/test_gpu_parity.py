@@ -238,12 +238,6 @@ def test_small_word_sized_frames_take_the_staged_path(tb, fb, tmax):
         assert np.array_equal(res["dense"], O.pack(op, store.cpu().numpy(), fb, 1, 2, 0))
 
 
-def _runs_are_short(sum_t, n, fb):
-    """Among the calls of the staged path the word-wise kernels take those whose frames are multiples of 16 bytes and
-    those whose runs average 768 bytes or less."""
-    return fb % 16 == 0 or sum_t * fb // n <= 768
-
-
 @pytest.mark.parametrize("tb,fb,kind", [(4096, 4, "ones"), (4096, 4, "few_words"), (10000, 4, "heavy_tail"), (94, 8, "clips"),
                                         (94, 12, "clips"), (512, 36, "few_words"), (64, 256, "ones"), (4096, 4, "some_long"),
                                         (33, 4, "few_words"), (1000, 16, "one_sequence")])
@@ -266,16 +260,17 @@ def test_runs_of_a_few_words(tb, fb, kind):
     else:
         T = np.array([7])
     T = rng.permutation(np.minimum(T, tb)).astype(np.int32)
-    assert _runs_are_short(int(T.sum()), len(T), fb)
+    want_k = G.expected_copy_kernels(int(T.sum()), len(T), fb, tb)
+    assert want_k["pack_meta"] == "k17_pack_short_runs<metadata>"
     plan, op = G.full_parity(T, tb, 21, fb, out_fb=fb, pad=0xE1, extra_blocks=3)
-    assert B.bload_last_copy_kernel("pack").startswith("k17_pack_short_runs")
-    assert B.bload_last_copy_kernel("unpack") == "k18_unpack_short_runs"
+    assert B.bload_last_copy_kernel("pack") == want_k["pack_meta"]
+    assert B.bload_last_copy_kernel("unpack") == want_k["unpack"]
     store = torch.randint(0, 256, (op.sum_t * fb,), dtype=torch.uint8, device=G.DEV)
     store_h = store.cpu().numpy()
     nb = op.n_blocks
     for b0, cnt in [(0, 1), (nb // 2, 3), (nb - 1, 3), (nb + 2, 2), (1, max(nb - 2, 1))]:
         res, _ = G.gpu_pack_all(plan, store, fb, b0, cnt, 0x4D, meta=False)
-        assert B.bload_last_copy_kernel("pack") == "k17_pack_short_runs"
+        assert B.bload_last_copy_kernel("pack") == want_k["pack"]
         d = G.first_diff(res["dense"].reshape(-1), O.pack(op, store_h, fb, b0, cnt, 0x4D).reshape(-1))
         assert d is None, "blocks [%d, +%d): %s" % (b0, cnt, d)
         # the same range back: the word-wise walk along the dense side, canaries around the output
@@ -283,8 +278,40 @@ def test_runs_of_a_few_words(tb, fb, kind):
         rag = G.Guarded(op.sum_t * fb, 0x5A)
         B.bload_unpack(plan, dense_out, fb, b0, cnt, rag.t)
         torch.cuda.synchronize(); rag.check()
-        if not (b0 == 0 and cnt >= nb):
-            assert B.bload_last_copy_kernel("unpack") == "k19_unpack_range_short_runs"
+        assert B.bload_last_copy_kernel("unpack") == (want_k["unpack"] if b0 == 0 and cnt >= nb else want_k["unpack_range"])
+        want = np.full(op.sum_t * fb, 0x5A, np.uint8)
+        O.unpack(op, dense_out.cpu().numpy(), fb, b0, cnt, want)
+        d = G.first_diff(rag.t.cpu().numpy(), want)
+        assert d is None, "unpack of blocks [%d, +%d): %s" % (b0, cnt, d)
+
+
+@pytest.mark.parametrize("tb,fb,tmax", [(94, 6, 94), (94, 3, 94), (4096, 2, 300), (4096, 1, 200), (1000, 30, 40), (33, 10, 33),
+                                        (7, 1, 7), (1, 3, 1), (5000, 2, 1500), (640, 6, 400), (2000, 1, 700), (3000, 3, 600)])
+def test_frames_that_are_not_multiples_of_4_bytes(tb, fb, tmax):
+    """Even frame sizes that are not multiples of 4 take the unstaged walks with 2-byte words while their runs average at
+    most 1.5 KB (pack) or 1 KB (unpack), odd sizes with 1-byte words up to 384 bytes; above that the register path.
+    Blocks of 3 bytes to 30 KB, runs of 1 byte and up, padding, filler blocks, sub-ranges, canaries around every output;
+    the last three cases sit at and above the cross-overs."""
+    rng = np.random.default_rng(tb * 53 + fb)
+    n = int(min(8000, max(3, 3_000_000 // (tmax * fb))))
+    T = rng.integers(1, tmax + 1, size=n).astype(np.int32)
+    T[rng.integers(0, n)] = tmax
+    want_k = G.expected_copy_kernels(int(T.sum()), n, fb, tb)
+    plan, op = G.full_parity(T, tb, 33, fb, out_fb=fb, pad=0x9C, extra_blocks=2)
+    assert B.bload_last_copy_kernel("pack") == want_k["pack"] and B.bload_last_copy_kernel("unpack") == want_k["unpack"]
+    store = torch.randint(0, 256, (op.sum_t * fb,), dtype=torch.uint8, device=G.DEV)
+    store_h = store.cpu().numpy()
+    nb = op.n_blocks
+    for b0, cnt in [(0, 1), (nb // 2, 2), (nb - 1, 3), (nb, 2)]:
+        res, _ = G.gpu_pack_all(plan, store, fb, b0, cnt, 0x21, meta=False)
+        d = G.first_diff(res["dense"].reshape(-1), O.pack(op, store_h, fb, b0, cnt, 0x21).reshape(-1))
+        assert d is None, "blocks [%d, +%d): %s" % (b0, cnt, d)
+        rag = G.Guarded(op.sum_t * fb, 0x5A)
+        # (a block range must start 16-byte aligned in the caller's buffer: a fresh buffer per range)
+        dense_out = torch.randint(0, 256, (cnt * tb * fb,), dtype=torch.uint8, device=G.DEV)
+        B.bload_unpack(plan, dense_out, fb, b0, cnt, rag.t)
+        torch.cuda.synchronize(); rag.check()
+        assert B.bload_last_copy_kernel("unpack") == (want_k["unpack"] if b0 == 0 and cnt >= nb else want_k["unpack_range"])
         want = np.full(op.sum_t * fb, 0x5A, np.uint8)
         O.unpack(op, dense_out.cpu().numpy(), fb, b0, cnt, want)
         d = G.first_diff(rag.t.cpu().numpy(), want)
@@ -304,15 +331,14 @@ def test_pack_of_small_frames_in_blocks_of_any_size(tb, fb, tmax):
     T = rng.integers(1, tmax + 1, size=n).astype(np.int32)
     T[rng.integers(0, n)] = tmax
     plan, op = G.full_parity(T, tb, 8, fb, out_fb=fb, pad=0x6B, extra_blocks=3)
-    short = _runs_are_short(op.sum_t, len(T), fb)
-    staged = "k17_pack_short_runs" if short else "k10_pack_contig"
-    assert B.bload_last_copy_kernel("pack").startswith(staged)
+    want_k = G.expected_copy_kernels(op.sum_t, len(T), fb, tb)
+    assert B.bload_last_copy_kernel("pack") == want_k["pack_meta"] and want_k["pack"] != "k7_copy<pack>"
     store = torch.randint(0, 256, (op.sum_t * fb,), dtype=torch.uint8, device=G.DEV)
     store_h = store.cpu().numpy()
     nb = op.n_blocks
     for b0, cnt in [(0, 1), (1, 1), (nb // 2, 3), (nb - 1, 2), (0, nb), (nb // 3, nb // 2 + 1), (nb, 1)]:
         res, _ = G.gpu_pack_all(plan, store, fb, b0, cnt, 0xD2, meta=False)
-        assert B.bload_last_copy_kernel("pack") == staged
+        assert B.bload_last_copy_kernel("pack") == want_k["pack"]
         d = G.first_diff(res["dense"].reshape(-1), O.pack(op, store_h, fb, b0, cnt, 0xD2).reshape(-1))
         assert d is None, "blocks [%d, +%d): %s" % (b0, cnt, d)
 
@@ -334,7 +360,7 @@ def test_one_launch_for_dense_blocks_and_metadata_of_small_frames(tb, fb, tmax):
         before = B.bload_kernel_launches()
         res, _ = G.gpu_pack_all(plan, store, fb, b0, cnt, 0x3C)
         assert B.bload_kernel_launches() - before == 1
-        assert B.bload_last_copy_kernel("pack") == ("k17_pack_short_runs" if _runs_are_short(op.sum_t, len(T), fb) else "k10_pack_contig") + "<metadata>"
+        assert B.bload_last_copy_kernel("pack") == G.expected_copy_kernels(op.sum_t, len(T), fb, tb)["pack_meta"]
         assert np.array_equal(res["dense"], O.pack(op, store_h, fb, b0, cnt, 0x3C))
         for name, want in zip(("seq_id", "pos", "reset", "valid"), O.metadata(op, b0, cnt)):
             assert np.array_equal(res[name], want), name
@@ -385,8 +411,7 @@ def test_unpack_of_block_ranges_of_small_frames(tb, fb, kind):
         rag = G.Guarded(op.sum_t * fb, 0x5A)
         B.bload_unpack(plan, dense_out, fb, b0, cnt, rag.t)
         torch.cuda.synchronize(); rag.check()
-        assert B.bload_last_copy_kernel("unpack") == ("k19_unpack_range_short_runs" if _runs_are_short(op.sum_t, len(T), fb)
-                                                      else "k8_unpack_staged")
+        assert B.bload_last_copy_kernel("unpack") == G.expected_copy_kernels(op.sum_t, len(T), fb, tb)["unpack_range"]
         want = np.full(op.sum_t * fb, 0x5A, np.uint8)
         O.unpack(op, dense_out.cpu().numpy(), fb, b0, cnt, want)
         d = G.first_diff(rag.t.cpu().numpy(), want)
