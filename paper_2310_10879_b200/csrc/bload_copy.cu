@@ -1105,6 +1105,11 @@ WalkKernel walk_kernel_for(int64_t frame_bytes)
 //     against 3.66 / 4.20
 //   1-byte words (odd frame sizes): 3-byte frames in 173-byte runs 1.49 / 1.56 against 0.73 / 1.15; 1-byte frames in
 //     870-byte runs 1.87 / 2.07 against 2.51 / 3.23
+// Tried for the 4-byte words and dropped: the ragged-side walk in 16-byte groups (four 4-byte loads and one 16-byte store
+// per group that lies inside one run, word by word for the groups that hold a run's end).  Whole-plan unpack, TB/s,
+// against the staged kernels: 4-byte frames in 3.5 KB runs 5.86 against 6.10, 12-byte frames in 10 KB runs 6.07 against
+// 6.06, 100-byte frames in 5.8 KB runs 5.99 against 6.04, 4-byte frames in 232-byte runs 3.75 against 3.65, 12-byte frames
+// in 696-byte runs 4.97 against 4.70: within 6 % either way, so the staged kernels stayed.
 inline bool walks_unstaged(int64_t frame_bytes, int64_t mean_run, bool unpack)
 {
     if (frame_bytes % 8 == 0) return mean_run <= kStagedMaxRunBytes;
