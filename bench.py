@@ -956,10 +956,26 @@ def frame_sweep(args) -> dict:
                 ms_s = timed(lambda: B.bload_unpack(plan, dense[tb * fb:], fb, 1, nb - 1, back))
                 gbs = 2 * st * fb * (nb - 1) / nb / ms_s / 1e6
                 row["unpack_sub_range"] = {"kernel": B.bload_last_copy_kernel("unpack"), "GB/s": round(gbs), "frac_measured": round(gbs / peak, 3)}
+            # the consumer-side shifted copy over the same blocks, and the per-slot metadata of the call
+            prev = back = None
+            prev = torch.empty_like(dense)
+            ms_c = timed(lambda: B.bload_carry_prev(plan, dense, fb, 0, nb, prev, 0))
+            gbs = ((st - n) * fb + nb * tb * fb) / ms_c / 1e6
+            row["carry_prev"] = {"kernel": B.bload_last_copy_kernel("carry_prev"), "GB/s": round(gbs), "frac_measured": round(gbs / peak, 3)}
+            del prev
+            if nb * tb >= 1 << 22:  # (smaller calls are bound by the launch, not by the 10 bytes per slot)
+                ids = torch.empty((2, nb * tb), dtype=torch.int32, device=dev)
+                flags = torch.empty((2, nb * tb), dtype=torch.uint8, device=dev)
+                ms_m = timed(lambda: B.bload_pack(plan, None, fb, 0, nb, seq_id=ids[0], pos=ids[1], reset=flags[0], valid=flags[1]))
+                row["metadata"] = {"GB/s": round(nb * tb * 10 / ms_m / 1e6), "frac_measured": round(nb * tb * 10 / ms_m / 1e6 / peak, 3),
+                                   "slots": nb * tb, "t_block": tb}
+                del ids, flags
             rows.append(row)
             del store, dense, back, plan
             torch.cuda.empty_cache()
-    return {"frame_sweep": rows, "peak_GB/s": peak, "unit": "GB/s of algorithmic bytes (pack: frames read + blocks written; unpack: frames read + written)"}
+    return {"frame_sweep": rows, "peak_GB/s": peak,
+            "unit": "GB/s of algorithmic bytes (pack: frames read + blocks written; unpack: frames read + written; carry_prev: "
+                    "frames but the first of every sequence read + blocks written; metadata: 10 bytes per slot written)"}
 
 
 TRAFFIC: dict = {

@@ -10,12 +10,14 @@
 //                    in double precision and in a fixed order, plus their total.
 #include "bload_internal.cuh"
 #include "bload_warp_copy.cuh"
+#include "bload_walk.cuh"
 
 namespace bload {
 
 namespace {
 
 using namespace wc;
+using namespace walk;
 
 // Same decomposition as the pack kernel: the output is cut into sub-tiles of `sub_bytes`, a warp owns one.
 // Inside a segment that occupies bytes [seg_b, seg_e) of its block, the first frame receives the fill byte and
@@ -263,6 +265,100 @@ __global__ void __launch_bounds__(kSumThreads) k13_total(PlanView pv, int64_t bl
     if (threadIdx.x == 0) { total[0] = ts; total[1] = tc; }
 }
 
+// The shifted copy as a word-wise walk along the dense side (see bload_walk.cuh), for short runs and small blocks: lane l
+// takes the words l, l+32, ... of 16 KB of the output and finds the run of each of its words in a window of 32 runs.  A
+// word of a run's first frame, of padding or of a filler block receives the fill byte, every other word x receives
+// dense[x - frame_bytes]: loads and stores of a warp are contiguous.  A window entry: {begin of the next run, end of this
+// run, begin of this run}, relative to the first byte of the warp's piece.
+template <int W>
+__global__ void __launch_bounds__(256) k23_carry_walk(PlanView pv, int32_t n, int32_t t_block, int64_t frame_bytes,
+                                                      int64_t block_begin, const uint8_t* __restrict__ dense,
+                                                      uint8_t* __restrict__ prev, int64_t total, uint8_t fill)
+{
+    __shared__ int4 windows[8][32];
+    constexpr int U = W == 16 ? 4 : 8;  // words in flight per lane
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    int4* win = windows[warp];
+    const int fb = (int)frame_bytes;
+    const int64_t block_bytes = (int64_t)t_block * fb;
+    const int64_t n_blocks = pv.hdr->n_blocks;
+    const int64_t chunks = (total + kRangeChunkBytes - 1) / kRangeChunkBytes;
+    const uint32_t f4 = 0x01010101u * fill;
+    for (int64_t c = (int64_t)blockIdx.x * 8 + warp; c < chunks; c += (int64_t)gridDim.x * 8) {
+        const int64_t lo0 = c * kRangeChunkBytes;  // positions below are relative to this byte of the call's dense side
+        const int p_end = (int)min((int64_t)kRangeChunkBytes, total - lo0);
+        int kw = first_run_at(pv, n, block_begin, n_blocks, lo0, block_bytes, fb, lane);
+        int r = 0, e = 0, b = 0, dn = 0, d_last = 0;
+        auto load_window = [&]() {  // one lane per run
+            const int k = kw + lane;
+            int4 w = make_int4(kFar, kFar, 0, 0);
+            if (k < n) {
+                const int blk = pv.seg_block[k], st = pv.seg_start[k];
+                const int nst = k + 1 < n ? pv.seg_start[k + 1] : 0;  // a later run of the same block starts later
+                const int e_slot = nst > st ? nst : pv.block_fill[blk];
+                const int64_t d_flat = (blk - block_begin) * block_bytes + (int64_t)st * fb - lo0;
+                // (a run that began before this piece began inside the same block: more than -2^30; one that lies before
+                // the call's blocks is clamped, its end is 0 and its begin is never looked at)
+                const int64_t b_true = d_flat < -(1LL << 30) ? -(1LL << 30) : d_flat;
+                w = make_int4(clamp_far(d_flat), clamp_far(d_flat + (int64_t)(e_slot - st) * fb), b_true > (int64_t)kFar ? kFar : (int)b_true, 0);
+            }
+            __syncwarp();  // every lane has left the previous window
+            d_last = __shfl_sync(kFull, w.x, 31);
+            win[lane] = make_int4(__shfl_down_sync(kFull, w.x, 1), w.y, w.z, 0);  // (lane 31's entry is never walked)
+            __syncwarp();
+            const int4 w0 = win[0];
+            r = 0; dn = w0.x; e = w0.y; b = w0.z;
+        };
+        load_window();
+        const uint8_t* src = dense + lo0 - fb;  // the word at position q comes from position q - frame_bytes
+        uint8_t* out = prev + lo0;
+        int done = 0;
+        while (done < p_end) {  // ends: a turn reaches p_end or moves the window on by 31 runs that begin ever later
+            const int limit = min(p_end, d_last);
+            for (int p = done + W * lane; p < limit; p += 32 * W * U) {
+                bool carried[U];
+                typename WordOf<W>::type v[U];
+#pragma unroll
+                for (int u = 0; u < U; ++u) {
+                    const int q = p + u * 32 * W;
+                    carried[u] = false;
+                    if (q < limit) {
+                        while (q >= dn) {  // (q < limit <= begin of the window's last entry, so r stays below 31)
+                            ++r;
+                            const int4 w = win[r];
+                            dn = w.x; e = w.y; b = w.z;
+                        }
+                        carried[u] = q < e && q - b >= fb;
+                    }
+                }
+#pragma unroll
+                for (int u = 0; u < U; ++u) v[u] = carried[u] ? load_word<W>(src + p + u * 32 * W) : pad_word<W>(f4);
+#pragma unroll
+                for (int u = 0; u < U; ++u) if (p + u * 32 * W < limit) store_word<W>(out + p + u * 32 * W, v[u]);
+            }
+            done = limit;
+            if (limit == d_last) { kw += 31; load_window(); }
+        }
+    }
+}
+using CarryWalkKernel = void (*)(PlanView, int32_t, int32_t, int64_t, int64_t, const uint8_t*, uint8_t*, int64_t, uint8_t);
+inline CarryWalkKernel carry_walk_kernel_for(int64_t frame_bytes)
+{
+    return frame_bytes % 16 == 0 ? k23_carry_walk<16> : frame_bytes % 8 == 0 ? k23_carry_walk<8>
+           : frame_bytes % 4 == 0 ? k23_carry_walk<4> : frame_bytes % 2 == 0 ? k23_carry_walk<2> : k23_carry_walk<1>;
+}
+// When the walk replaces the sub-tile kernels.  Measured on B200 (TB/s, walk against k11_carry_shift; clips = blocks of 94
+// frames in runs of 22): 8-byte frames of clips 4.87 against 1.33, 16-byte 5.85 against 2.41, 64-byte 6.21 against 4.31,
+// 256-byte 6.36 against 5.43, 6-byte 2.72 against 1.07 (the sub-tile kernels take a block per warp at least: 752 bytes);
+// blocks of 10,000 frames in runs of 58: 16-byte frames 6.25 against 5.47, 64-byte 6.29 against 6.11, 256-byte (15 KB
+// runs) 6.41 against 6.51, 8-byte 5.86 against 5.90, 4-byte 4.59 against 5.33, 6-byte 3.29 against 5.19; token lengths:
+// 8- and 16-byte frames level, 4-byte 5.91 against 6.26, 64-byte and larger 2-3 % behind.
+inline bool carry_walks(int64_t frame_bytes, int64_t mean_run, int64_t block_bytes)
+{
+    if (block_bytes <= 4096) return true;
+    return frame_bytes % 8 == 0 && (mean_run <= 8192 || block_bytes <= 32768) && mean_run <= 16384;
+}
+
 unsigned grid_for_items(int64_t items)
 {
     const int64_t want = (items + 7) / 8;  // CTAs of 8 warps, one item per warp
@@ -281,6 +377,15 @@ cudaError_t launch_carry_prev(const PlanView& pv, int32_t t_block, int64_t frame
     const int64_t spb = (block_bytes + sub - 1) / sub;
     count_launches(1);
     BLOAD_DBG_EXPECT(st, dbg::kCarry, {{dense, (size_t)(block_count * block_bytes)}}, {{prev, (size_t)(block_count * block_bytes)}});
+    if (n > 0 && n < 0x7fffff00LL && block_bytes < (1LL << 30) && carry_walks(frame_bytes, sum_t * frame_bytes / n, block_bytes)) {
+        const int64_t total = block_count * block_bytes;
+        const int64_t want = ((total + kRangeChunkBytes - 1) / kRangeChunkBytes + 7) / 8;
+        const int64_t cap = (int64_t)device_info().sm_count * 32;
+        note_copy_kernel(kCallCarryPrev, "k23_carry_walk");
+        carry_walk_kernel_for(frame_bytes)<<<(unsigned)(want < cap ? want : cap), 256, 0, st>>>(pv, (int32_t)n, t_block, frame_bytes, block_begin,
+                                                                                                dense, prev, total, fill_byte);
+        return cudaPeekAtLastError();
+    }
     // short runs (many segments per sub-tile): one shifted copy per sub-tile and patches at the segment starts
     if (n > 0 && sum_t * frame_bytes / n <= 16384) {
         note_copy_kernel(kCallCarryPrev, "k11_carry_shift");

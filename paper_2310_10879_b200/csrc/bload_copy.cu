@@ -17,12 +17,14 @@
 #include "bload_internal.cuh"
 #include "bload_meta.cuh"
 #include "bload_warp_copy.cuh"
+#include "bload_walk.cuh"
 
 namespace bload {
 
 namespace {
 
 using namespace wc;
+using namespace walk;
 
 // `range` (device, or null): {first block, end block, end of the real blocks} replaces block_begin / block_count /
 // n_blocks when the blocks of a launch are decided on the device (a plan that is still being built); `out_base` is
@@ -655,7 +657,6 @@ __global__ void __launch_bounds__(StageCfg<false>::kWarps * 32) k10_pack_contig(
 template <int W> struct ShortCfg : StageCfgT<4096, 8, 2, 2> {};
 template <> struct ShortCfg<16> : StageCfgT<8192, 4, 2, 2> {};
 constexpr int kShortWindowBytes = 32 * 16;
-constexpr int kFar = 0x7fffffff;  // "beyond the warp's range"
 #ifndef BLOAD_SHORT_RUN
 #define BLOAD_SHORT_RUN 768
 #endif
@@ -679,7 +680,6 @@ inline bool runs_are_short(int64_t ragged_bytes, int64_t n, int64_t frame_bytes)
 {
     return frame_bytes % 16 == 0 || ragged_bytes / n <= BLOAD_SHORT_RUN;
 }
-__device__ __forceinline__ int clamp_far(int64_t v) { return v < 0 ? 0 : (v > (int64_t)kFar ? kFar : (int)v); }
 
 // words [p0, p1) of the range, for the stage that images the range from t0; win[r] = {begin of run r+1, end, source minus
 // stage-side position (64 bit)}; r, e, delta, dn are the lane's place in the window.  A word is W = 16, 8 or 4 bytes, the
@@ -707,32 +707,6 @@ __device__ __forceinline__ void walk_words(const int4* __restrict__ win, int& r,
         else if (W == 8) *reinterpret_cast<uint2*>(stage + (p - t0)) = make_uint2(p4, p4);
         else *reinterpret_cast<uint32_t*>(stage + (p - t0)) = p4;
     }
-}
-
-// the run that holds byte lo0 of the call's dense side or, when lo0 lies in padding or in a filler block, the last run before it
-__device__ __forceinline__ int first_run_at(const PlanView& pv, int n, int64_t block_begin, int64_t n_blocks, int64_t lo0,
-                                            int64_t block_bytes, int fb, int lane)
-{
-    const int64_t q = lo0 / block_bytes, b = block_begin + q;
-    if (b >= n_blocks) return n - 1;
-    const int k0 = pv.block_seg_begin[b], k1 = pv.block_seg_begin[b + 1];
-    const int64_t r0 = lo0 - q * block_bytes;
-    return r0 < (int64_t)pv.block_fill[b] * fb ? warp_find_segment(pv.seg_start, k0, k1, (int)(r0 / fb), lane) : k1 - 1;
-}
-// window entry of run k for a walk along the dense side: where the run begins and ends there, relative to byte lo0 of the
-// call's dense side and clamped to [0, kFar], and its place in the ragged store minus its (unclamped) begin.  A run ends
-// where the next run of its block begins, or where the block's frames end.
-__device__ __forceinline__ int4 dense_side_entry(const PlanView& pv, int n, int k, int64_t block_begin, int64_t block_bytes, int fb,
-                                                 int64_t lo0)
-{
-    if (k >= n) return make_int4(kFar, kFar, 0, 0);
-    const int blk = pv.seg_block[k], st = pv.seg_start[k];
-    const int nst = k + 1 < n ? pv.seg_start[k + 1] : 0;  // a later run of the same block starts later
-    const int e_slot = nst > st ? nst : pv.block_fill[blk];
-    const int64_t d_flat = (blk - block_begin) * block_bytes + (int64_t)st * fb - lo0;
-    const int64_t dl = pv.seg_src[k] * fb - d_flat;
-    return make_int4(clamp_far(d_flat), clamp_far(d_flat + (int64_t)(e_slot - st) * fb), (int)(uint32_t)(uint64_t)dl,
-                     (int)(uint32_t)((uint64_t)dl >> 32));
 }
 
 template <bool META, int W>
@@ -908,33 +882,6 @@ __global__ void __launch_bounds__(ShortCfg<W>::kWarps * 32) k18_unpack_short_run
 // word's place in the ragged output (consecutive inside a run); words of padding are skipped.  Pack: the word comes from
 // its place in the ragged store, or is padding, and goes to the dense side.  Words of 2 bytes and 1 byte serve frames
 // that are not multiples of 4 bytes, which cp.async (4 bytes at least) cannot move.
-template <int W> struct WordOf { using type = uint32_t; };
-template <> struct WordOf<1> { using type = unsigned char; };
-template <> struct WordOf<2> { using type = unsigned short; };
-template <> struct WordOf<8> { using type = uint2; };
-template <> struct WordOf<16> { using type = uint4; };
-template <int W>
-__device__ __forceinline__ typename WordOf<W>::type load_word(const uint8_t* p)
-{
-    using T = typename WordOf<W>::type;
-    return BLOAD_MAY_READ(p, W) ? __ldcs(reinterpret_cast<const T*>(p)) : T{};
-}
-template <int W>
-__device__ __forceinline__ void store_word(uint8_t* p, typename WordOf<W>::type v)
-{
-    using T = typename WordOf<W>::type;
-    if (BLOAD_MAY_WRITE(p, W)) __stcs(reinterpret_cast<T*>(p), v);
-}
-template <int W>
-__device__ __forceinline__ typename WordOf<W>::type pad_word(uint32_t p4)
-{
-    using T = typename WordOf<W>::type;
-    if constexpr (W == 16) return make_uint4(p4, p4, p4, p4);
-    else if constexpr (W == 8) return make_uint2(p4, p4);
-    else return (T)p4;
-}
-
-constexpr int kRangeChunkBytes = 16384;  // of the dense side per warp and turn
 template <int W, bool PACK>
 __global__ void __launch_bounds__(256) k19_walk_dense_side(PlanView pv, int32_t n, int32_t t_block, int64_t frame_bytes,
                                                            int64_t block_begin, const uint8_t* __restrict__ from,

@@ -34,6 +34,79 @@ __global__ void __launch_bounds__(kMetaThreads) k6_metadata(PlanView pv, int32_t
     }
 }
 
+// The same outputs for blocks that are short or not a multiple of 4 slots long (the paper's own block of 94 frames): a
+// thread produces 4 consecutive slots of the call's blocks taken as ONE array, wherever the blocks end, so every thread
+// of a CTA has work (the kernel above gives a block a CTA of 1,024 slots at least: 9 % of it for 94 slots) and the ids
+// leave in 16-byte vectors whatever t_block is.  A quad that runs into the next block carries on with its first segment.
+template <bool VEC>
+__global__ void __launch_bounds__(kMetaThreads) k6_metadata_flat(PlanView pv, int32_t t_block, int64_t block_begin, int64_t total,
+                                                                 int32_t* __restrict__ seq_id, int32_t* __restrict__ pos,
+                                                                 uint8_t* __restrict__ reset, uint8_t* __restrict__ valid)
+{
+    const int64_t n_blocks = pv.hdr->n_blocks;
+    const int32_t* __restrict__ seg_start = pv.seg_start;
+    for (int64_t o = ((int64_t)blockIdx.x * kMetaThreads + threadIdx.x) * 4; o < total; o += (int64_t)gridDim.x * kMetaThreads * 4) {
+        int64_t q = o / t_block;
+        int s = (int)(o - q * t_block);
+        int sid[4] = {-1, -1, -1, -1}, ps[4] = {-1, -1, -1, -1};
+        unsigned rs = 0, vd = 0;  // one flag byte per slot
+        int fill = 0, k = 0, k1 = 0, st = 0, nx = 0, id = 0;
+        auto open_block = [&](int64_t b) {  // header of block b; its first segment starts at slot 0
+            fill = 0; k = 0; k1 = 0;
+            if (b < n_blocks) { k = __ldg(pv.block_seg_begin + b); k1 = __ldg(pv.block_seg_begin + b + 1); fill = __ldg(pv.block_fill + b); }
+        };
+        auto open_segment = [&]() {
+            st = __ldg(seg_start + k);
+            nx = (k + 1 < k1) ? __ldg(seg_start + k + 1) : fill;
+            id = __ldg(pv.seg_seq + k);
+        };
+        open_block(block_begin + q);
+        if (s < fill) {  // last segment of the block that starts at or before s
+            int lo = k, hi = k1;
+            while (hi - lo > 1) {
+                const int mid = (lo + hi) >> 1;
+                if (__ldg(seg_start + mid) <= s) lo = mid; else hi = mid;
+            }
+            k = lo;
+            open_segment();
+        }
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            if (o + e < total) {
+                if (s == t_block) {
+                    ++q; s = 0;
+                    open_block(block_begin + q);
+                    if (fill > 0) open_segment();
+                }
+                if (s < fill) {
+                    if (s >= nx) { ++k; open_segment(); }
+                    sid[e] = id;
+                    ps[e] = s - st;
+                    vd |= 1u << (8 * e);
+                    if (s == st) rs |= 1u << (8 * e);
+                }
+                ++s;
+            }
+        }
+        if (VEC && o + 4 <= total) {
+            if (seq_id && BLOAD_MAY_WRITE(seq_id + o, 16)) __stcs(reinterpret_cast<int4*>(seq_id + o), make_int4(sid[0], sid[1], sid[2], sid[3]));
+            if (pos && BLOAD_MAY_WRITE(pos + o, 16)) __stcs(reinterpret_cast<int4*>(pos + o), make_int4(ps[0], ps[1], ps[2], ps[3]));
+            if (reset && BLOAD_MAY_WRITE(reset + o, 4)) __stcs(reinterpret_cast<unsigned*>(reset + o), rs);
+            if (valid && BLOAD_MAY_WRITE(valid + o, 4)) __stcs(reinterpret_cast<unsigned*>(valid + o), vd);
+        } else {
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                if (o + e < total) {
+                    if (seq_id && BLOAD_MAY_WRITE(seq_id + o + e, 4)) seq_id[o + e] = sid[e];
+                    if (pos && BLOAD_MAY_WRITE(pos + o + e, 4)) pos[o + e] = ps[e];
+                    if (reset && BLOAD_MAY_WRITE(reset + o + e, 1)) reset[o + e] = (uint8_t)((rs >> (8 * e)) & 1u);
+                    if (valid && BLOAD_MAY_WRITE(valid + o + e, 1)) valid[o + e] = (uint8_t)((vd >> (8 * e)) & 1u);
+                }
+            }
+        }
+    }
+}
+
 }  // namespace
 
 cudaError_t launch_metadata(const PlanView& pv, int32_t t_block, int64_t block_begin, int64_t block_count,
@@ -55,6 +128,18 @@ cudaError_t launch_metadata(const PlanView& pv, int32_t t_block, int64_t block_b
     } else {
         [[maybe_unused]] const size_t slots = (size_t)block_count * (size_t)t_block;
         BLOAD_DBG_EXPECT(st, dbg::kMetadata, {}, {{seq_id, 4 * slots}, {pos, 4 * slots}, {reset, slots}, {valid, slots}});
+    }
+    // blocks that leave a CTA of the chunked kernel mostly idle, or whose length rules out its vector stores
+    if (!d_range && (t_block % 4 != 0 || (int64_t)chunks * kMetaChunk * 4 > (int64_t)t_block * 5)) {
+        const int64_t total = block_count * t_block;
+        const int64_t want = (total + kMetaChunk - 1) / kMetaChunk, cap = (int64_t)device_info().sm_count * 64;
+        const unsigned flat_grid = (unsigned)(want < cap ? want : cap);
+        if (al(seq_id, 16) && al(pos, 16) && al(reset, 4) && al(valid, 4))
+            k6_metadata_flat<true><<<flat_grid, kMetaThreads, 0, st>>>(pv, t_block, block_begin, total, seq_id, pos, reset, valid);
+        else
+            k6_metadata_flat<false><<<flat_grid, kMetaThreads, 0, st>>>(pv, t_block, block_begin, total, seq_id, pos, reset, valid);
+        count_launches(1);
+        return cudaPeekAtLastError();
     }
     if (t_block % 4 == 0 && al(seq_id, 16) && al(pos, 16) && al(reset, 4) && al(valid, 4))
         k6_metadata<true><<<grid, kMetaThreads, smem, st>>>(pv, t_block, block_begin, (int32_t)block_count, seq_id, pos, reset, valid, d_range);

@@ -268,6 +268,39 @@ def test_carry_prev_small_word_sized_frames_take_the_staged_kernel(fb, tb):
         _carry_prev_parity(plan, op, fb, op.n_blocks - 1, 5, 0x01)
 
 
+def _expected_carry_kernel(sum_t, n, fb, tb):
+    """The rule stated beside launch_carry_prev: the word-wise walk for blocks of at most 4 KB and, when the frames are
+    multiples of 8 bytes, for runs of at most 8 KB (or blocks of at most 32 KB) on average; else the shifted copy per
+    sub-tile up to 16 KB runs; else the segment-by-segment kernel."""
+    run, block = sum_t * fb // n, tb * fb
+    if block <= 4096 or (fb % 8 == 0 and (run <= 8192 or block <= 32768) and run <= 16384):
+        return "k23_carry_walk"
+    return "k11_carry_shift" if run <= 16384 else "k11_carry_prev"
+
+
+@pytest.mark.parametrize("fb,tb,tmax", [(8, 94, 94), (16, 94, 94), (64, 94, 94), (6, 94, 94), (1, 7, 7), (12, 94, 94), (256, 94, 60),
+                                        (32, 10000, 300), (8, 4096, 2000), (4, 1, 1), (2, 2047, 700)])
+def test_carry_prev_by_the_word_wise_walk(fb, tb, tmax):
+    """Small blocks (the paper's own block of 94 frames with per-frame records of a few bytes) and short runs of frames
+    that are multiples of 8 bytes take the word-wise walk: words of 16, 8, 4, 2 and 1 bytes, blocks of 4 bytes to 320 KB,
+    runs that begin before the warp's piece, pieces that begin in padding and in filler blocks, sub-ranges; the
+    previous frame of every frame, the fill byte on first frames and padding."""
+    rng = np.random.default_rng(fb * 19 + tb)
+    n = int(min(6000, max(4, 3_000_000 // (tmax * fb))))
+    T = rng.integers(1, tmax + 1, size=n).astype(np.int32)
+    T[rng.integers(0, n)] = tmax
+    plan, op = _both_plans(T, tb, 13)
+    assert _expected_carry_kernel(op.sum_t, n, fb, tb) == "k23_carry_walk"
+    _carry_prev_parity(plan, op, fb, 0, op.n_blocks + 3, 0x00)
+    assert B.bload_last_copy_kernel("carry_prev") == "k23_carry_walk"
+    _carry_prev_parity(plan, op, fb, 0, op.n_blocks, 0xB4, seed=3)
+    if op.n_blocks > 3:
+        _carry_prev_parity(plan, op, fb, 1, op.n_blocks - 2, 0x5E)
+        _carry_prev_parity(plan, op, fb, op.n_blocks // 2, 2, 0x01)
+    _carry_prev_parity(plan, op, fb, op.n_blocks - 1, 4, 0x77)
+    _carry_prev_parity(plan, op, fb, op.n_blocks + 1, 2, 0x12)
+
+
 @pytest.mark.parametrize("fb,tb,tmax", [(1, 40, 9), (3, 50, 50), (7, 3000, 40), (10, 64, 8), (130, 64, 20), (1000, 12, 5),
                                         (4096, 30, 3), (20, 20000, 600), (6, 16384, 300)])
 def test_carry_prev_short_runs_take_the_shifted_copy(fb, tb, tmax):
@@ -280,7 +313,7 @@ def test_carry_prev_short_runs_take_the_shifted_copy(fb, tb, tmax):
     T = rng.integers(1, tmax + 1, size=n).astype(np.int32)
     plan, op = _both_plans(T, tb, 31)
     _carry_prev_parity(plan, op, fb, 0, op.n_blocks + 2, 0x00)
-    assert B.bload_last_copy_kernel("carry_prev") == "k11_carry_shift"
+    assert B.bload_last_copy_kernel("carry_prev") == _expected_carry_kernel(op.sum_t, n, fb, tb)
     _carry_prev_parity(plan, op, fb, 0, op.n_blocks, 0xC3, seed=9)
     if op.n_blocks > 3:
         _carry_prev_parity(plan, op, fb, 1, op.n_blocks - 2, 0x5E)

@@ -20,7 +20,7 @@ def test_small_cases_under_the_bounds_checking_build():
     files = ["tests/test_gpu_fuzz.py", "tests/test_gpu_parity.py", "tests/test_gpu_var_frames.py", "tests/test_gpu_consumer.py",
              "tests/test_gpu_chunks.py"]
     select = ("fuzz or frame_sizes or staged or degenerate or toy8 or one_launch or whole_plan_unpack or block_ranges or "
-              "metadata_only or blocks_of_any_size or few_words or not_multiples_of_4 or random_frame_sizes or multiples_of_16 or images or carry_prev or reset_state or repeat_last or "
+              "metadata_only or blocks_of_any_size or blocks_of_any_length or few_words or not_multiples_of_4 or by_the_word_wise_walk or random_frame_sizes or multiples_of_16 or images or carry_prev or reset_state or repeat_last or "
               "chunk_plans")
     r = subprocess.run([sys.executable, "-m", "pytest", "-x", "-q", "-m", "gpu", "-k", select, "-p", "no:cacheprovider"] + files,
                        cwd=ROOT, env=env, capture_output=True, text=True, timeout=1500)

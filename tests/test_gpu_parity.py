@@ -145,6 +145,40 @@ def test_metadata_only_and_dense_only_calls():
                           O.metadata(op, 0, op.n_blocks)[2])
 
 
+@pytest.mark.parametrize("tb", [1, 2, 3, 5, 6, 94, 96, 777, 1023, 1024, 1025, 1300, 2500, 4097, 10001])
+def test_metadata_for_blocks_of_any_length(tb):
+    """Metadata-only calls over block lengths around the kernels' shapes: blocks shorter than a CTA's 1,024 slots and blocks
+    whose length is not a multiple of 4 take the kernel that treats the call's blocks as one array (quads that run through
+    the ends of one to four blocks), the others the chunked kernel; whole plans with filler blocks, sub-ranges that start
+    anywhere, unaligned output pointers, a subset of the four arrays; canaries around every output."""
+    rng = np.random.default_rng(tb)
+    n = int(min(4000, max(6, 400_000 // tb)))
+    T = rng.integers(1, tb + 1, size=n).astype(np.int32)
+    op = O.plan(T, tb, 12); plan = G.gpu_plan(T, tb, 12)
+    nb = op.n_blocks
+    for b0, cnt in [(0, nb + 3), (1, max(nb - 2, 1)), (nb // 2, 1), (nb - 1, 3), (nb + 1, 2)]:
+        slots = cnt * tb
+        outs = dict(seq_id=G.Guarded(slots * 4, 0x11), pos=G.Guarded(slots * 4, 0x11), reset=G.Guarded(slots, 0x11),
+                    valid=G.Guarded(slots, 0x11))
+        B.bload_pack(plan, None, 8, b0, cnt, seq_id=outs["seq_id"].t.view(torch.int32), pos=outs["pos"].t.view(torch.int32),
+                     reset=outs["reset"].t, valid=outs["valid"].t)
+        torch.cuda.synchronize()
+        want = O.metadata(op, b0, cnt)
+        for (name, g), w in zip(outs.items(), want):
+            g.check()
+            got = g.t.view(torch.int32) if name in ("seq_id", "pos") else g.t
+            assert np.array_equal(got.cpu().numpy().reshape(cnt, tb), w), (name, b0, cnt)
+    # two of the four arrays at addresses that rule out vector stores
+    cnt = min(nb, 7)
+    raw_pos = torch.full((cnt * tb + 3,), 77, dtype=torch.int32, device=G.DEV)
+    raw_reset = torch.full((cnt * tb + 3,), 77, dtype=torch.uint8, device=G.DEV)
+    B.bload_pack(plan, None, 8, 0, cnt, pos=raw_pos[1:1 + cnt * tb], reset=raw_reset[1:1 + cnt * tb])
+    want = O.metadata(op, 0, cnt)
+    assert np.array_equal(raw_pos[1:1 + cnt * tb].cpu().numpy().reshape(cnt, tb), want[1])
+    assert np.array_equal(raw_reset[1:1 + cnt * tb].cpu().numpy().reshape(cnt, tb), want[2])
+    assert int(raw_pos[0]) == 77 and int(raw_pos[-1]) == 77 and int(raw_reset[0]) == 77 and int(raw_reset[-2]) == 77
+
+
 def test_bad_lengths_are_reported_not_faulted():
     for T, tb, bad in [([3, 0, 2], 4, 1), ([3, 4, 5, 2], 4, 2), ([3, -1], 4, 1)]:
         plan = G.gpu_plan(np.array(T, np.int32), tb, 0, check=False)
