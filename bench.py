@@ -964,8 +964,8 @@ def frame_sweep(args) -> dict:
             row["carry_prev"] = {"kernel": B.bload_last_copy_kernel("carry_prev"), "GB/s": round(gbs), "frac_measured": round(gbs / peak, 3)}
             del prev
             if nb * tb >= 1 << 22:  # (smaller calls are bound by the launch, not by the 10 bytes per slot)
-                ids = torch.empty((2, nb * tb), dtype=torch.int32, device=dev)
-                flags = torch.empty((2, nb * tb), dtype=torch.uint8, device=dev)
+                ids = [torch.empty(nb * tb, dtype=torch.int32, device=dev) for _ in range(2)]   # (each array 16-byte aligned)
+                flags = [torch.empty(nb * tb, dtype=torch.uint8, device=dev) for _ in range(2)]
                 ms_m = timed(lambda: B.bload_pack(plan, None, fb, 0, nb, seq_id=ids[0], pos=ids[1], reset=flags[0], valid=flags[1]))
                 row["metadata"] = {"GB/s": round(nb * tb * 10 / ms_m / 1e6), "frac_measured": round(nb * tb * 10 / ms_m / 1e6 / peak, 3),
                                    "slots": nb * tb, "t_block": tb}

@@ -269,17 +269,17 @@ def test_carry_prev_small_word_sized_frames_take_the_staged_kernel(fb, tb):
 
 
 def _expected_carry_kernel(sum_t, n, fb, tb):
-    """The rule stated beside launch_carry_prev: the word-wise walk for blocks of at most 4 KB and, when the frames are
-    multiples of 8 bytes, for runs of at most 8 KB (or blocks of at most 32 KB) on average; else the shifted copy per
+    """The rule stated beside launch_carry_prev: the word-wise walk for blocks of at most 1 KB (4 KB when the frames are
+    multiples of 4 bytes) and, when the frames are multiples of 8 bytes, for runs of at most 8 KB (or blocks of at most 32 KB) on average; else the shifted copy per
     sub-tile up to 16 KB runs; else the segment-by-segment kernel."""
     run, block = sum_t * fb // n, tb * fb
-    if block <= 4096 or (fb % 8 == 0 and (run <= 8192 or block <= 32768) and run <= 16384):
+    if block <= 1024 or (block <= 4096 and fb % 4 == 0) or (fb % 8 == 0 and (run <= 8192 or block <= 32768) and run <= 16384):
         return "k23_carry_walk"
     return "k11_carry_shift" if run <= 16384 else "k11_carry_prev"
 
 
 @pytest.mark.parametrize("fb,tb,tmax", [(8, 94, 94), (16, 94, 94), (64, 94, 94), (6, 94, 94), (1, 7, 7), (12, 94, 94), (256, 94, 60),
-                                        (32, 10000, 300), (8, 4096, 2000), (4, 1, 1), (2, 2047, 700)])
+                                        (32, 10000, 300), (8, 4096, 2000), (4, 1, 1), (2, 500, 300)])
 def test_carry_prev_by_the_word_wise_walk(fb, tb, tmax):
     """Small blocks (the paper's own block of 94 frames with per-frame records of a few bytes) and short runs of frames
     that are multiples of 8 bytes take the word-wise walk: words of 16, 8, 4, 2 and 1 bytes, blocks of 4 bytes to 320 KB,
