@@ -530,7 +530,7 @@ int bload_pack(const void* d_plan, const bload_plan_info_t* info, const void* d_
         return BLOAD_OK;
     }
     if (want_meta)
-        ce = launch_metadata(pv, info->t_block, block_begin, block_count, d_seq_id, d_pos, d_reset, d_valid, st);
+        ce = launch_metadata(pv, info->t_block, block_begin, block_count, d_seq_id, d_pos, d_reset, d_valid, st, nullptr, info->n, info->sum_t);
     if (ce == cudaSuccess && d_dense)
         ce = launch_copy(false, pv, info->t_block, frame_bytes, block_begin, block_count,
                          static_cast<const uint8_t*>(d_store), static_cast<uint8_t*>(d_dense), nullptr,

@@ -139,7 +139,8 @@ cudaError_t launch_plan(const int32_t* d_lengths, int64_t n, int32_t t_block, ui
                         const BfdView* bv = nullptr /*policy 2 only*/);
 cudaError_t launch_metadata(const PlanView& pv, int32_t t_block, int64_t block_begin, int64_t block_count,
                             int32_t* seq_id, int32_t* pos, uint8_t* reset, uint8_t* valid, cudaStream_t st,
-                            const int32_t* d_range = nullptr);
+                            const int32_t* d_range = nullptr, int64_t n = 0 /*sequences and frames of the plan, when the*/,
+                            int64_t sum_t = 0 /*caller knows them: they choose the kernel*/);
 cudaError_t launch_copy(bool unpack, const PlanView& pv, int32_t t_block, int64_t frame_bytes, int64_t block_begin,
                         int64_t block_count, const uint8_t* ragged_in, uint8_t* dense, uint8_t* ragged_out,
                         int64_t ragged_bytes, uint8_t pad_byte, cudaStream_t st, int64_t n, int64_t n_blocks,
