@@ -14,6 +14,17 @@
 // destination are then misaligned relative to each other (frame sizes that are not multiples of
 // 16, e.g. 4-byte tokens) each output vector is assembled from two aligned source vectors with
 // funnel shifts.
+//
+// In this file, in order:
+//   k7_copy                      the register path described above (large frames, long runs)
+//   k10 / k9 / k8                small word-sized frames, run by run through shared-memory stages (cp.async in, one bulk
+//                                store out): pack, whole-plan unpack, unpack of a block sub-range
+//   k17 / k18                    the same stages, word by word: runs of a few hundred bytes (a lane finds the run of each
+//                                of its words in a window of 32 runs)
+//   k19 / k21                    word by word without a stage: frames that are multiples of 8 bytes, and frames that are
+//                                not multiples of 4 bytes in short runs
+//   k7b_copy_bulk                a measurement variant (large frames through the bulk-copy engine), off by default
+//   launch_copy and friends      which kernel takes which call, with the measurements the rules come from
 #include "bload_internal.cuh"
 #include "bload_meta.cuh"
 #include "bload_warp_copy.cuh"
