@@ -28,7 +28,10 @@ def _assert_same(got: torch.Tensor, want: np.ndarray, what: str):
 
 
 def _run(name):
-    w = W.WORKLOADS[name]
+    _run_workload(W.WORKLOADS[name])
+
+
+def _run_workload(w, carry=False):
     T = W.lengths(w)
     op = O.plan(T, w.t_block, w.seed)
     plan = G.gpu_plan(T, w.t_block, w.seed)
@@ -76,6 +79,15 @@ def _run(name):
         _assert_same(rag.t[lo:lo + step], want[lo:lo + step], "unpacked bytes from %d" % lo)
     st = B.bload_stats(plan.info)
     assert st["pad_packed"] == nb * tb - op.sum_t and st["pad_naive_tmax"] == op.n * op.t_max - op.sum_t
+    if carry:  # the consumer-side shifted copy of the same per-frame outputs, every block
+        del rag, want
+        prev = G.Guarded(nb * tb * ofb, 0x3C)
+        B.bload_carry_prev(plan, out_u8.reshape(-1), ofb, 0, nb, prev.t, fill_byte=0xE7)
+        torch.cuda.synchronize(); prev.check()
+        p3 = prev.t.view(nb, tb * ofb)
+        for lo, cnt in _slabs(nb, tb * ofb):
+            _assert_same(p3[lo:lo + cnt], O.carry_prev(op, out_u8[lo:lo + cnt].cpu().numpy().reshape(-1), ofb, lo, cnt, 0xE7),
+                         "carry_prev of blocks %d..%d" % (lo, lo + cnt))
 
 
 def test_full_size_raw_frames():
@@ -88,6 +100,19 @@ def test_full_size_tokens():
 
 def test_full_size_heavy_tail_bf16_with_fp32_outputs():
     _run("heavy_tail_bf16")
+
+
+@pytest.mark.parametrize("name,n,fb", [("video_dataset_shape", 1_000_000, 8), ("heavy_tail_bf16", 1_000_000, 4),
+                                       ("video_dataset_shape", 600_000, 6), ("tokens", 120_000, 16),
+                                       ("video_dataset_shape", 400_000, 12)])
+def test_a_million_short_runs(name, n, fb):
+    """The word-wise kernels at scale: a million clips of 22 frames with 8-byte records (blocks of 94 slots), a million
+    heavy-tailed sequences of 4-byte frames, 6-byte and 12-byte records, 16-byte frames with token lengths.  Plan, packed
+    bytes, metadata, unpacked bytes and the shifted copy of every block against the oracle; thousands of windows per
+    warp, warps that begin inside runs, padding and the filler tail."""
+    from dataclasses import replace
+    w = replace(W.scaled(W.WORKLOADS[name], n), frame_bytes=fb, out_frame_bytes=fb, payload="u8")
+    _run_workload(w, carry=True)
 
 
 @pytest.mark.parametrize("name", ["tokens", "heavy_tail_bf16"])
