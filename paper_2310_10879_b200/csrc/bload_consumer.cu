@@ -199,6 +199,48 @@ __global__ void __launch_bounds__(256) k14_repeat_last(PlanView pv, int32_t t_bl
     }
 }
 
+// The same for small frames (below 512 bytes), where a copy per padding frame costs more than the frame: the padding
+// part of the sub-tile is written word by word, lane l the words l, l+32, ...; a word at byte x of the padding comes from
+// byte x mod frame_bytes of the last frame.  A word is the largest of 16, 8, 4, 2 and 1 bytes that divides the frame.
+template <int W>
+__global__ void __launch_bounds__(256) k14_repeat_last_words(PlanView pv, int32_t t_block, int64_t frame_bytes, int64_t block_begin,
+                                                             int64_t block_count, uint8_t* __restrict__ dense, int64_t sub_bytes,
+                                                             int64_t subs_per_block)
+{
+    const int lane = threadIdx.x & 31;
+    const int64_t warps = ((int64_t)gridDim.x * blockDim.x) >> 5;
+    const int64_t items = block_count * subs_per_block;
+    const int64_t block_bytes = (int64_t)t_block * frame_bytes;
+    const int64_t n_blocks = pv.hdr->n_blocks;
+    const int fb = (int)frame_bytes;
+    for (int64_t item = (((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5); item < items; item += warps) {
+        const int64_t q = item / subs_per_block;
+        const int64_t b = block_begin + q;
+        if (b >= n_blocks) continue;  // a filler block has no frame to repeat
+        const int64_t pad_lo = (int64_t)pv.block_fill[b] * frame_bytes;
+        const int64_t lo = (item - q * subs_per_block) * sub_bytes;
+        const int64_t hi = min(lo + sub_bytes, block_bytes);
+        const int64_t cur = max(lo, pad_lo);
+        if (cur >= hi || pad_lo == 0) continue;
+        uint8_t* row = dense + q * block_bytes;
+        const uint8_t* last = row + pad_lo - frame_bytes;
+        // (pad_lo, lo and frame_bytes are multiples of W: so are cur and every offset below)
+        int off = (int)((cur - pad_lo + (int64_t)W * lane) % fb);  // offset of this lane's first word inside the frame
+        const int step = (32 * W) % fb;
+        for (int64_t x = cur + (int64_t)W * lane; x < hi; x += 32 * W) {
+            store_word<W>(row + x, load_word<W>(last + off));
+            off += step;
+            if (off >= fb) off -= fb;
+        }
+    }
+}
+using RepeatWordsKernel = void (*)(PlanView, int32_t, int64_t, int64_t, int64_t, uint8_t*, int64_t, int64_t);
+inline RepeatWordsKernel repeat_words_kernel_for(int64_t frame_bytes)
+{
+    return frame_bytes % 16 == 0 ? k14_repeat_last_words<16> : frame_bytes % 8 == 0 ? k14_repeat_last_words<8>
+           : frame_bytes % 4 == 0 ? k14_repeat_last_words<4> : frame_bytes % 2 == 0 ? k14_repeat_last_words<2> : k14_repeat_last_words<1>;
+}
+
 constexpr int kSumThreads = 256;
 
 // Fixed-order sum of one double per thread over a CTA of kSumThreads threads; the result is valid in thread 0.
@@ -454,8 +496,12 @@ cudaError_t launch_repeat_last(const PlanView& pv, int32_t t_block, int64_t fram
     const int64_t spb = (block_bytes + sub - 1) / sub;
     count_launches(1);
     BLOAD_DBG_EXPECT(st, dbg::kRepeatLast, {{dense, (size_t)(block_count * block_bytes)}}, {{dense, (size_t)(block_count * block_bytes)}});
-    k14_repeat_last<<<grid_for_items(block_count * spb), 256, 0, st>>>(pv, t_block, frame_bytes, block_begin, block_count,
-                                                                      dense, sub, spb);
+    if (frame_bytes < 512)
+        repeat_words_kernel_for(frame_bytes)<<<grid_for_items(block_count * spb), 256, 0, st>>>(pv, t_block, frame_bytes, block_begin,
+                                                                                                block_count, dense, sub, spb);
+    else
+        k14_repeat_last<<<grid_for_items(block_count * spb), 256, 0, st>>>(pv, t_block, frame_bytes, block_begin, block_count,
+                                                                          dense, sub, spb);
     return cudaPeekAtLastError();
 }
 
