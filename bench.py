@@ -216,8 +216,8 @@ def run_reference(args, w) -> dict:
     if blocks <= 0:
         cal = CpuOracleSample(w, 2).run()
         per_block = max(cal["seconds"] - cal["plan_s"], 1e-3) / 2
-        budget = 100.0 / max(1, args.warmup + args.steps) - cal["plan_s"]
-        blocks = int(max(1, min(budget / per_block, 64)))
+        seconds_per_step = 100.0 / max(1, args.warmup + args.steps) - cal["plan_s"]
+        blocks = int(max(1, min(seconds_per_step / per_block, 64)))
     sample = CpuOracleSample(w, blocks)
     times, last = [], None
     for i in range(args.warmup + args.steps):
