@@ -159,7 +159,8 @@ BLOAD_API int bload_plan_finish(const void* d_plan, void* stream, bload_plan_inf
  *     bload_plan(policy BLOAD_POLICY_UNIFORM_SEQUENCES) ; bload_pack(blocks 0 .. block_capacity) ;
  *     bload_unpack(blocks 0 .. block_capacity)
  * but the fill rule (a chain of dependent draws that keeps one warp busy and leaves the memory system idle) runs
- * in chunks of about 1,800 draws (at most 12, or io->chunks) on `stream`, and as soon as a chunk has closed its blocks their tables, metadata,
+ * in chunks (about 1,800 draws each on average, at most 10, every chunk 1.25 times as long as the one before; or io->chunks
+ * equal chunks) on `stream`, and as soon as a chunk has closed its blocks their tables, metadata,
  * pack and unpack are issued on `side_stream`, under the next chunk of the chain.  Only launch-order dependencies
  * (events) are used; no kernel waits for another.  The paper has no counterpart (it builds blocks on the host).
  *
