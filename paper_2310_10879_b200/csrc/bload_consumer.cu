@@ -348,7 +348,7 @@ __global__ void __launch_bounds__(kSumThreads) k13_total(PlanView pv, int64_t bl
 template <int W>
 __global__ void __launch_bounds__(256) k23_carry_walk(PlanView pv, int32_t n, int32_t t_block, int64_t frame_bytes,
                                                       int64_t block_begin, const uint8_t* __restrict__ dense,
-                                                      uint8_t* __restrict__ prev, int64_t total, uint8_t fill)
+                                                      uint8_t* __restrict__ prev, int64_t total, uint8_t fill, int32_t piece)
 {
     __shared__ int4 windows[8][32];
     constexpr int U = W == 16 ? 4 : 8;  // words in flight per lane
@@ -357,11 +357,11 @@ __global__ void __launch_bounds__(256) k23_carry_walk(PlanView pv, int32_t n, in
     const int fb = (int)frame_bytes;
     const int64_t block_bytes = (int64_t)t_block * fb;
     const int64_t n_blocks = pv.hdr->n_blocks;
-    const int64_t chunks = (total + kRangeChunkBytes - 1) / kRangeChunkBytes;
+    const int64_t chunks = (total + piece - 1) / piece;
     const uint32_t f4 = 0x01010101u * fill;
     for (int64_t c = (int64_t)blockIdx.x * 8 + warp; c < chunks; c += (int64_t)gridDim.x * 8) {
-        const int64_t lo0 = c * kRangeChunkBytes;  // positions below are relative to this byte of the call's dense side
-        const int p_end = (int)min((int64_t)kRangeChunkBytes, total - lo0);
+        const int64_t lo0 = c * (int64_t)piece;  // positions below are relative to this byte of the call's dense side
+        const int p_end = (int)min((int64_t)piece, total - lo0);
         int kw = first_run_at(pv, n, block_begin, n_blocks, lo0, block_bytes, fb, lane);
         int r = 0, e = 0, b = 0, dn = 0, d_last = 0;
         auto load_window = [&]() {  // one lane per run
@@ -416,7 +416,7 @@ __global__ void __launch_bounds__(256) k23_carry_walk(PlanView pv, int32_t n, in
         }
     }
 }
-using CarryWalkKernel = void (*)(PlanView, int32_t, int32_t, int64_t, int64_t, const uint8_t*, uint8_t*, int64_t, uint8_t);
+using CarryWalkKernel = void (*)(PlanView, int32_t, int32_t, int64_t, int64_t, const uint8_t*, uint8_t*, int64_t, uint8_t, int32_t);
 inline CarryWalkKernel carry_walk_kernel_for(int64_t frame_bytes)
 {
     return frame_bytes % 16 == 0 ? k23_carry_walk<16> : frame_bytes % 8 == 0 ? k23_carry_walk<8>
@@ -454,11 +454,12 @@ cudaError_t launch_carry_prev(const PlanView& pv, int32_t t_block, int64_t frame
     BLOAD_DBG_EXPECT(st, dbg::kCarry, {{dense, (size_t)(block_count * block_bytes)}}, {{prev, (size_t)(block_count * block_bytes)}});
     if (n > 0 && n < 0x7fffff00LL && block_bytes < (1LL << 30) && carry_walks(frame_bytes, sum_t * frame_bytes / n, block_bytes)) {
         const int64_t total = block_count * block_bytes;
-        const int64_t want = ((total + kRangeChunkBytes - 1) / kRangeChunkBytes + 7) / 8;
+        const int piece = walk_piece_bytes(total, device_info().sm_count);
+        const int64_t want = ((total + piece - 1) / piece + 7) / 8;
         const int64_t cap = (int64_t)device_info().sm_count * 32;
         note_copy_kernel(kCallCarryPrev, "k23_carry_walk");
         carry_walk_kernel_for(frame_bytes)<<<(unsigned)(want < cap ? want : cap), 256, 0, st>>>(pv, (int32_t)n, t_block, frame_bytes, block_begin,
-                                                                                                dense, prev, total, fill_byte);
+                                                                                                dense, prev, total, fill_byte, piece);
         return cudaPeekAtLastError();
     }
     // short runs (many segments per sub-tile): one shifted copy per sub-tile and patches at the segment starts

@@ -894,9 +894,9 @@ __global__ void __launch_bounds__(ShortCfg<W>::kWarps * 32) k18_unpack_short_run
 // its place in the ragged store, or is padding, and goes to the dense side.  Words of 2 bytes and 1 byte serve frames
 // that are not multiples of 4 bytes, which cp.async (4 bytes at least) cannot move.
 template <int W, bool PACK>
-__global__ void __launch_bounds__(256) k19_walk_dense_side(PlanView pv, int32_t n, int32_t t_block, int64_t frame_bytes,
+__global__ void __launch_bounds__(256, 4) k19_walk_dense_side(PlanView pv, int32_t n, int32_t t_block, int64_t frame_bytes,
                                                            int64_t block_begin, const uint8_t* __restrict__ from,
-                                                           uint8_t* __restrict__ to_base, int64_t total, uint8_t pad)
+                                                           uint8_t* __restrict__ to_base, int64_t total, uint8_t pad, int32_t piece)
 {
     __shared__ int4 windows[8][32];
     constexpr int U = W == 16 ? 4 : 8;  // words in flight per lane (4-byte words, 232-byte runs: 2 -> 2.54, 4 -> 2.68, 8 -> 2.78 TB/s)
@@ -905,11 +905,11 @@ __global__ void __launch_bounds__(256) k19_walk_dense_side(PlanView pv, int32_t 
     const int fb = (int)frame_bytes;
     const int64_t block_bytes = (int64_t)t_block * fb;
     const int64_t n_blocks = pv.hdr->n_blocks;
-    const int64_t chunks = (total + kRangeChunkBytes - 1) / kRangeChunkBytes;
+    const int64_t chunks = (total + piece - 1) / piece;
     const uint32_t p4 = 0x01010101u * pad;
     for (int64_t c = (int64_t)blockIdx.x * 8 + warp; c < chunks; c += (int64_t)gridDim.x * 8) {
-        const int64_t lo0 = c * kRangeChunkBytes;  // positions below are relative to this byte of the call's dense side
-        const int p_end = (int)min((int64_t)kRangeChunkBytes, total - lo0);
+        const int64_t lo0 = c * (int64_t)piece;  // positions below are relative to this byte of the call's dense side
+        const int p_end = (int)min((int64_t)piece, total - lo0);
         int kw = first_run_at(pv, n, block_begin, n_blocks, lo0, block_bytes, fb, lane);
         int r = 0, e = 0, dn = 0, d_last = 0;
         int64_t delta = 0;
@@ -968,9 +968,9 @@ __global__ void __launch_bounds__(256) k19_walk_dense_side(PlanView pv, int32_t 
 // next begins), a lane loads each of its words from the word's place in the dense buffer and stores it in place; the
 // stores are contiguous across the warp, the loads inside a run.
 template <int W>
-__global__ void __launch_bounds__(256) k21_unpack_walk_ragged(PlanView pv, int32_t n, int32_t t_block, int64_t frame_bytes,
+__global__ void __launch_bounds__(256, 4) k21_unpack_walk_ragged(PlanView pv, int32_t n, int32_t t_block, int64_t frame_bytes,
                                                               int64_t sum_t, const uint8_t* __restrict__ dense,
-                                                              uint8_t* __restrict__ ragged)
+                                                              uint8_t* __restrict__ ragged, int32_t piece)
 {
     __shared__ int4 windows[8][32];
     constexpr int U = W == 16 ? 4 : 8;
@@ -978,10 +978,10 @@ __global__ void __launch_bounds__(256) k21_unpack_walk_ragged(PlanView pv, int32
     int4* win = windows[warp];
     const int64_t total = sum_t * frame_bytes;
     const int64_t block_bytes = (int64_t)t_block * frame_bytes;
-    const int64_t chunks = (total + kRangeChunkBytes - 1) / kRangeChunkBytes;
+    const int64_t chunks = (total + piece - 1) / piece;
     for (int64_t c = (int64_t)blockIdx.x * 8 + warp; c < chunks; c += (int64_t)gridDim.x * 8) {
-        const int64_t lo0 = c * kRangeChunkBytes;  // positions below are relative to this byte of the ragged side
-        const int p_end = (int)min((int64_t)kRangeChunkBytes, total - lo0);
+        const int64_t lo0 = c * (int64_t)piece;  // positions below are relative to this byte of the ragged side
+        const int p_end = (int)min((int64_t)piece, total - lo0);
         int kw = warp_find_sequence(pv.offsets, n, lo0 / frame_bytes, lane);
         int r = 0, dn = 0, d_last = 0;
         int64_t delta = 0;
@@ -1030,7 +1030,7 @@ __global__ void __launch_bounds__(256) k21_unpack_walk_ragged(PlanView pv, int32
         }
     }
 }
-using WalkRaggedKernel = void (*)(PlanView, int32_t, int32_t, int64_t, int64_t, const uint8_t*, uint8_t*);
+using WalkRaggedKernel = void (*)(PlanView, int32_t, int32_t, int64_t, int64_t, const uint8_t*, uint8_t*, int32_t);
 inline WalkRaggedKernel walk_ragged_kernel_for(int64_t frame_bytes)
 {
     return frame_bytes % 16 == 0 ? k21_unpack_walk_ragged<16> : frame_bytes % 8 == 0 ? k21_unpack_walk_ragged<8>
@@ -1038,7 +1038,7 @@ inline WalkRaggedKernel walk_ragged_kernel_for(int64_t frame_bytes)
                                                                                      : k21_unpack_walk_ragged<1>;
 }
 
-using WalkKernel = void (*)(PlanView, int32_t, int32_t, int64_t, int64_t, const uint8_t*, uint8_t*, int64_t, uint8_t);
+using WalkKernel = void (*)(PlanView, int32_t, int32_t, int64_t, int64_t, const uint8_t*, uint8_t*, int64_t, uint8_t, int32_t);
 template <bool PACK>
 WalkKernel walk_kernel_for(int64_t frame_bytes)
 {
@@ -1329,17 +1329,19 @@ cudaError_t launch_copy(bool unpack, const PlanView& pv, int32_t t_block, int64_
         const int64_t cap = (int64_t)device_info().sm_count * 32;
         if (whole_plan) {  // along the ragged side, which is contiguous and written completely
             const WalkRaggedKernel kernel = walk_ragged_kernel_for(frame_bytes);
-            const int64_t want = ((ragged_bytes + kRangeChunkBytes - 1) / kRangeChunkBytes + 7) / 8;
+            const int piece = walk_piece_bytes(ragged_bytes, device_info().sm_count);
+            const int64_t want = ((ragged_bytes + piece - 1) / piece + 7) / 8;
             kernel<<<(unsigned)(want < cap ? want : cap), 256, 0, st>>>(pv, (int32_t)n, t_block, frame_bytes, ragged_bytes / frame_bytes,
-                                                                        dense, ragged_out);
+                                                                        dense, ragged_out, piece);
             note_copy_kernel(kCallUnpack, "k21_unpack_walk_ragged");
             return cudaPeekAtLastError();
         }
         const WalkKernel kernel = unpack ? walk_kernel_for<false>(frame_bytes) : walk_kernel_for<true>(frame_bytes);
         const int64_t total = block_count * block_bytes;
-        const int64_t want = ((total + kRangeChunkBytes - 1) / kRangeChunkBytes + 7) / 8;
+        const int piece = walk_piece_bytes(total, device_info().sm_count);
+        const int64_t want = ((total + piece - 1) / piece + 7) / 8;
         kernel<<<(unsigned)(want < cap ? want : cap), 256, 0, st>>>(pv, (int32_t)n, t_block, frame_bytes, block_begin,
-                                                                    unpack ? dense : ragged_in, unpack ? ragged_out : dense, total, pad_byte);
+                                                                    unpack ? dense : ragged_in, unpack ? ragged_out : dense, total, pad_byte, piece);
         note_copy_kernel(unpack ? kCallUnpack : kCallPack, unpack ? "k19_unpack_walk_dense" : "k19_pack_walk_dense");
         return cudaPeekAtLastError();
     }

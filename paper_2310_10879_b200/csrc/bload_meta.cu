@@ -114,21 +114,21 @@ __global__ void __launch_bounds__(kMetaThreads) k6_metadata_flat(PlanView pv, in
 // run of its quad in a window of 32 runs that the warp builds with one lane per run -- {begin of the next run, end,
 // begin, sequence id} in slots relative to the warp's piece -- and only moves forward in it.  A quad inside one run (or
 // inside padding) needs no search and no table load at all; a quad that holds the end of a run goes slot by slot.
-constexpr int kMetaWalkSlots = 4096;
+constexpr int kMetaWalkSlots = 4096;  // slots per warp and turn, for calls that fill the machine
 template <bool VEC>
 __global__ void __launch_bounds__(256) k6_metadata_walk(PlanView pv, int32_t n, int32_t t_block, int64_t block_begin, int64_t total,
                                                         int32_t* __restrict__ seq_id, int32_t* __restrict__ pos,
-                                                        uint8_t* __restrict__ reset, uint8_t* __restrict__ valid)
+                                                        uint8_t* __restrict__ reset, uint8_t* __restrict__ valid, int32_t piece)
 {
     using namespace walk;
     __shared__ int4 windows[8][32];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     int4* win = windows[warp];
     const int64_t n_blocks = pv.hdr->n_blocks;
-    const int64_t chunks = (total + kMetaWalkSlots - 1) / kMetaWalkSlots;
+    const int64_t chunks = (total + piece - 1) / piece;
     for (int64_t c = (int64_t)blockIdx.x * 8 + warp; c < chunks; c += (int64_t)gridDim.x * 8) {
-        const int64_t lo0 = c * kMetaWalkSlots;  // positions below are slots relative to this slot of the call
-        const int p_end = (int)min((int64_t)kMetaWalkSlots, total - lo0);
+        const int64_t lo0 = c * (int64_t)piece;  // positions below are slots relative to this slot of the call
+        const int p_end = (int)min((int64_t)piece, total - lo0);
         int kw = first_run_at(pv, n, block_begin, n_blocks, lo0, t_block, 1, lane);
         int r = 0, dn = 0, e = 0, b = 0, id = 0, d_last = 0, my_begin = 0;
         auto load_window = [&]() {  // one lane per run
@@ -246,12 +246,15 @@ cudaError_t launch_metadata(const PlanView& pv, int32_t t_block, int64_t block_b
     constexpr int64_t kMetaWalkRun = 256;  // slots per run, on average, up to which the walk is used
     if (!d_range && n > 0 && n < 0x7fffff00LL && sum_t / n <= kMetaWalkRun) {
         const int64_t total = block_count * t_block;
-        const int64_t want = ((total + kMetaWalkSlots - 1) / kMetaWalkSlots + 7) / 8, cap = (int64_t)device_info().sm_count * 32;
+        // (a piece of 4,096 slots per warp when that fills the machine, else a multiple of 512 slots, 512 at least)
+        const int64_t per_warp = total / ((int64_t)device_info().sm_count * 32);
+        const int piece = per_warp >= kMetaWalkSlots ? kMetaWalkSlots : (int)(per_warp < 512 ? 512 : ((per_warp + 511) / 512) * 512);
+        const int64_t want = ((total + piece - 1) / piece + 7) / 8, cap = (int64_t)device_info().sm_count * 32;
         const unsigned walk_grid = (unsigned)(want < cap ? want : cap);
         if (al(seq_id, 16) && al(pos, 16) && al(reset, 4) && al(valid, 4))
-            k6_metadata_walk<true><<<walk_grid, 256, 0, st>>>(pv, (int32_t)n, t_block, block_begin, total, seq_id, pos, reset, valid);
+            k6_metadata_walk<true><<<walk_grid, 256, 0, st>>>(pv, (int32_t)n, t_block, block_begin, total, seq_id, pos, reset, valid, piece);
         else
-            k6_metadata_walk<false><<<walk_grid, 256, 0, st>>>(pv, (int32_t)n, t_block, block_begin, total, seq_id, pos, reset, valid);
+            k6_metadata_walk<false><<<walk_grid, 256, 0, st>>>(pv, (int32_t)n, t_block, block_begin, total, seq_id, pos, reset, valid, piece);
         count_launches(1);
         return cudaPeekAtLastError();
     }

@@ -71,7 +71,16 @@ __device__ __forceinline__ typename WordOf<W>::type pad_word(uint32_t p4)
     else return (T)p4;
 }
 
-constexpr int kRangeChunkBytes = 16384;  // of the dense side per warp and turn
+constexpr int kRangeChunkBytes = 16384;  // of the walked side per warp and turn, for calls that fill the machine
+// The piece a warp takes per turn: 16 KB when that still gives every SM a few CTAs of 8 warps, else smaller (a multiple
+// of 2 KB) so that a call of a few MB is spread over the machine instead of a handful of warps.
+inline int walk_piece_bytes(int64_t total, int sm_count)
+{
+    const int64_t per_warp = total / ((int64_t)sm_count * 32);
+    if (per_warp >= kRangeChunkBytes) return kRangeChunkBytes;
+    const int64_t p = ((per_warp + 2047) / 2048) * 2048;
+    return (int)(p < 2048 ? 2048 : p);
+}
 
 }  // namespace walk
 }  // namespace bload
