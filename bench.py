@@ -979,8 +979,8 @@ def frame_sweep(args) -> dict:
 
 
 TRAFFIC: dict = {
-    ("heavy_tail_bf16", "k7_copy<unpack>"): 18.29e9,
-    ("heavy_tail_bf16", "k7_copy<pack>"): 9.08e9,
+    ("heavy_tail_bf16", "k7_copy<unpack>"): 18.27e9,
+    ("heavy_tail_bf16", "k7_copy<pack>"): 9.09e9,
 }
 
 
