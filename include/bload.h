@@ -220,6 +220,9 @@ BLOAD_API int bload_epoch_stage_times(float out_ms[5]);
  * metadata and one for the dense blocks; a call that asks for both, for small word-sized frames (frame_bytes a multiple
  * of 4, runs of at most 16 KB on average, blocks of less than 1 GiB) and at most 4 Mi slots, is a single
  * launch -- the call a training loop makes per batch of token-sized frames is bound by launch overhead, not by bytes.
+ * With large frames the two kernels run side by side (the second is a programmatic dependent launch that does not wait
+ * for the first to end: their outputs are disjoint); whatever follows in `stream` still starts after both have ended.
+ * So the dense buffer and the metadata arrays of one call must not overlap each other.
  * Errors: NULL plan/info/store (when d_dense is given), ARG (frame_bytes < 1, negative range,
  * block_begin + block_count >= 2^31), ALIGN, PLAN (info->status != 0), CUDA.
  */

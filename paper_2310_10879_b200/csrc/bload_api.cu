@@ -548,7 +548,7 @@ int bload_pack(const void* d_plan, const bload_plan_info_t* info, const void* d_
     if (ce == cudaSuccess && d_dense)
         ce = launch_copy(false, pv, info->t_block, frame_bytes, block_begin, block_count,
                          static_cast<const uint8_t*>(d_store), static_cast<uint8_t*>(d_dense), nullptr,
-                         info->sum_t * frame_bytes, pad_byte, st, info->n, info->n_blocks);
+                         info->sum_t * frame_bytes, pad_byte, st, info->n, info->n_blocks, false, want_meta);
     if (ce != cudaSuccess) { (void)cudaGetLastError(); return BLOAD_ERR_CUDA; }
     return BLOAD_OK;
 }

@@ -98,6 +98,7 @@ __global__ void __launch_bounds__(256) k7_copy(PlanView pv, int32_t t_block, int
         }
         if (!UNPACK && cur < hi) warp_fill(dst_base + dense_off + cur, hi - cur, pad, lane);
     }
+    if (!UNPACK) wait_for_prerequisites();  // (a pack launched beside the call's metadata kernel ends after it)
 }
 
 
@@ -1305,7 +1306,8 @@ bool staged_pack_with_metadata(const PlanView& pv, int32_t t_block, int64_t fram
 
 cudaError_t launch_copy(bool unpack, const PlanView& pv, int32_t t_block, int64_t frame_bytes, int64_t block_begin,
                         int64_t block_count, const uint8_t* ragged_in, uint8_t* dense, uint8_t* ragged_out,
-                        int64_t ragged_bytes, uint8_t pad_byte, cudaStream_t st, int64_t n, int64_t n_blocks, bool gaps)
+                        int64_t ragged_bytes, uint8_t pad_byte, cudaStream_t st, int64_t n, int64_t n_blocks, bool gaps,
+                        bool beside_previous)
 {
     if (block_count == 0) return cudaSuccess;
     const int64_t block_bytes = (int64_t)t_block * frame_bytes;
@@ -1450,7 +1452,19 @@ cudaError_t launch_copy(bool unpack, const PlanView& pv, int32_t t_block, int64_
     if (unpack)
         k7_copy<true><<<grid, 256, 0, st>>>(pv, t_block, frame_bytes, block_begin, block_count, dense, ragged_out,
                                              block_count * block_bytes, sub, spb, pad_byte, nullptr, block_begin);
-    else
+    else if (beside_previous && !dbg::kChecked) {
+        // measured on B200, per-batch calls (dense blocks + metadata, two launches): 8 blocks of 41 MB 112.0 -> 105.5 us
+        // per call (107.4 -> 102.9 replayed from a graph), 4 blocks of 135 MB 168.8 -> 163.2 us (164.4 -> 160.2)
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(grid); cfg.blockDim = dim3(256); cfg.dynamicSmemBytes = 0; cfg.stream = st;
+        cudaLaunchAttribute at[1];
+        at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        at[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = at; cfg.numAttrs = 1;
+        const int32_t* no_range = nullptr;
+        return cudaLaunchKernelEx(&cfg, k7_copy<false>, pv, t_block, frame_bytes, block_begin, block_count, ragged_in,
+                                  dense, ragged_bytes, sub, spb, pad_byte, no_range, block_begin);
+    } else
         k7_copy<false><<<grid, 256, 0, st>>>(pv, t_block, frame_bytes, block_begin, block_count, ragged_in, dense,
                                               ragged_bytes, sub, spb, pad_byte, nullptr, block_begin);
     return cudaPeekAtLastError();

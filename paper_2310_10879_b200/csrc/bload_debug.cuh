@@ -20,6 +20,13 @@ namespace dbg {
 enum KernelId { kNone = 0, kCopy = 7, kUnpackStaged = 8, kUnpackRagged = 9, kPackContig = 10, kCarry = 11, kResetState = 12,
                 kRepeatLast = 14, kCopyVar = 16, kMetadata = 6, kTables = 5 };
 
+// (the checker keeps one set of ranges per device: launches of a checked build never overlap each other)
+#ifdef BLOAD_DEBUG
+constexpr bool kChecked = true;
+#else
+constexpr bool kChecked = false;
+#endif
+
 #ifdef BLOAD_DEBUG
 constexpr int kRanges = 6;
 struct Ranges {

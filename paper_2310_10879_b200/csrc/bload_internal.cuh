@@ -137,6 +137,15 @@ inline cudaError_t opt_in_shared_memory(K* kernel, int bytes) { return opt_in_sh
 cudaError_t launch_plan(const int32_t* d_lengths, int64_t n, int32_t t_block, uint64_t seed, uint32_t policy,
                         const PlanView& pv, const WorkView& wv, cudaStream_t st, cudaEvent_t* ev /*5 or null*/,
                         const BfdView* bv = nullptr /*policy 2 only*/);
+// Programmatic dependent launch, used where one call issues two kernels that touch disjoint buffers (per-slot metadata,
+// then the dense blocks): the first releases its dependents as soon as it runs, the second is launched with the
+// programmatic-serialisation attribute and so starts beside it instead of behind it, and waits for it only at its own
+// end, so that "the second has finished" still means "both have finished" for whatever comes next in the stream.
+// Both instructions do nothing in a kernel that was launched the ordinary way.
+#ifdef __CUDACC__
+__device__ __forceinline__ void release_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void wait_for_prerequisites() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+#endif
 cudaError_t launch_metadata(const PlanView& pv, int32_t t_block, int64_t block_begin, int64_t block_count,
                             int32_t* seq_id, int32_t* pos, uint8_t* reset, uint8_t* valid, cudaStream_t st,
                             const int32_t* d_range = nullptr, int64_t n = 0 /*sequences and frames of the plan, when the*/,
@@ -144,7 +153,9 @@ cudaError_t launch_metadata(const PlanView& pv, int32_t t_block, int64_t block_b
 cudaError_t launch_copy(bool unpack, const PlanView& pv, int32_t t_block, int64_t frame_bytes, int64_t block_begin,
                         int64_t block_count, const uint8_t* ragged_in, uint8_t* dense, uint8_t* ragged_out,
                         int64_t ragged_bytes, uint8_t pad_byte, cudaStream_t st, int64_t n, int64_t n_blocks,
-                        bool gaps = false /*the plan's sequences do not tile the ragged buffer (chunks with deleted frames)*/);
+                        bool gaps = false /*the plan's sequences do not tile the ragged buffer (chunks with deleted frames)*/,
+                        bool beside_previous = false /*the launch before this one in `st` is the call's own metadata kernel,
+                                                       which touches none of this launch's buffers: start beside it*/);
 // The pieces of the planner and the copies that bload_epoch strings together on two streams.  `d_range` points to
 // {first block, end block, end of the real blocks} in device memory: the blocks a launch covers are decided on the
 // device, so these launches use fixed grids whose CTAs loop.

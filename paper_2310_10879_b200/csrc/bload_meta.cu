@@ -22,6 +22,7 @@ __global__ void __launch_bounds__(kMetaThreads) k6_metadata(PlanView pv, int32_t
                                                             int32_t* __restrict__ pos, uint8_t* __restrict__ reset,
                                                             uint8_t* __restrict__ valid, const int32_t* __restrict__ range)
 {
+    release_dependents();
     const int s0 = (int)blockIdx.x * kMetaChunk + (int)threadIdx.x * 4;
     if (s0 >= t_block) return;
     // `range` (device, or null): {first block, end block, end of the real blocks} of a plan that is still being built;
@@ -44,6 +45,7 @@ __global__ void __launch_bounds__(kMetaThreads) k6_metadata_flat(PlanView pv, in
                                                                  int32_t* __restrict__ seq_id, int32_t* __restrict__ pos,
                                                                  uint8_t* __restrict__ reset, uint8_t* __restrict__ valid)
 {
+    release_dependents();
     const int64_t n_blocks = pv.hdr->n_blocks;
     const int32_t* __restrict__ seg_start = pv.seg_start;
     for (int64_t o = ((int64_t)blockIdx.x * kMetaThreads + threadIdx.x) * 4; o < total; o += (int64_t)gridDim.x * kMetaThreads * 4) {
@@ -120,6 +122,7 @@ __global__ void __launch_bounds__(256) k6_metadata_walk(PlanView pv, int32_t n, 
                                                         int32_t* __restrict__ seq_id, int32_t* __restrict__ pos,
                                                         uint8_t* __restrict__ reset, uint8_t* __restrict__ valid, int32_t piece)
 {
+    release_dependents();
     using namespace walk;
     __shared__ int4 windows[8][32];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
