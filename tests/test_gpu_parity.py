@@ -546,3 +546,37 @@ def test_rank_ranges_pack_and_unpack_like_the_whole():
         covered += cnt
     torch.cuda.synchronize()
     assert covered >= op.n_blocks and torch.equal(back, store)
+
+
+def test_reader_behind_a_pack_of_large_frames_sees_dense_blocks_and_metadata():
+    """Large frames: the pack kernel is launched beside the call's metadata kernel, not behind it.  Whatever the stream
+    runs next must still find both outputs complete -- here copies enqueued on the same side stream straight after
+    the call, with no synchronisation in between, call after call on the same output buffers (so a late metadata
+    kernel of call i would also be caught overwriting the results of call i+1)."""
+    rng = np.random.default_rng(99)
+    tb, fb = 2000, 4096
+    T = rng.integers(1, 40, size=6000).astype(np.int32)
+    plan = G.gpu_plan(T, tb, 3)
+    op = O.plan(T, tb, 3)
+    store = torch.randint(0, 256, (op.sum_t * fb,), dtype=torch.uint8, device=G.DEV)
+    assert G.expected_copy_kernels(op.sum_t, T.size, fb, tb)["pack"] == "k7_copy<pack>"
+    cnt = 3
+    dense = torch.empty(cnt * tb * fb, dtype=torch.uint8, device=G.DEV)
+    seq_id = torch.empty(cnt * tb, dtype=torch.int32, device=G.DEV)
+    pos = torch.empty_like(seq_id)
+    reset = torch.empty(cnt * tb, dtype=torch.uint8, device=G.DEV)
+    valid = torch.empty_like(reset)
+    s = torch.cuda.Stream()
+    s.wait_stream(torch.cuda.current_stream())
+    got = []
+    with torch.cuda.stream(s):
+        for b0 in range(0, min(op.n_blocks, 4 * cnt), cnt):
+            B.bload_pack(plan, store, fb, b0, cnt, dense=dense, seq_id=seq_id, pos=pos, reset=reset, valid=valid, pad_byte=0x5C)
+            got.append((b0, dense.clone(), seq_id.clone(), pos.clone(), reset.clone(), valid.clone()))
+    s.synchronize()
+    assert B.bload_last_copy_kernel("pack") == "k7_copy<pack>"
+    h_store = store.cpu().numpy()
+    for b0, d, si, po, re, va in got:
+        assert np.array_equal(d.cpu().numpy().reshape(cnt, tb, fb), O.pack(op, h_store, fb, b0, cnt, 0x5C)), b0
+        for name, arr, want in zip(("seq_id", "pos", "reset", "valid"), (si, po, re, va), O.metadata(op, b0, cnt)):
+            assert np.array_equal(arr.cpu().numpy().reshape(cnt, tb), want), (b0, name)
