@@ -23,6 +23,7 @@
 //                                of its words in a window of 32 runs)
 //   k19 / k21                    word by word without a stage: frames that are multiples of 8 bytes, and frames that are
 //                                not multiples of 4 bytes in short runs
+//   k24                          pack of frames of 1 to 3 bytes in runs of 0.4 to 4 KB: the walk in granules of 16 bytes
 //   k7b_copy_bulk                a measurement variant (large frames through the bulk-copy engine), off by default
 //   launch_copy and friends      which kernel takes which call, with the measurements the rules come from
 #include "bload_internal.cuh"
@@ -965,6 +966,142 @@ __global__ void __launch_bounds__(256, 4) k19_walk_dense_side(PlanView pv, int32
         }
     }
 }
+// Pack of frames that are not multiples of 4 bytes in runs too long for the 2- and 1-byte words above: the same walk
+// along the dense side in granules of 16 bytes.  A granule that lies inside one run -- nearly all of them, when runs
+// last a kilobyte -- is two aligned 16-byte loads from wherever its source happens to begin, a byte shift and one
+// 16-byte store; a granule of padding is one store; a granule that holds a run's end or begin is put together byte
+// by byte from the window.  Against the register path the gain is in the short runs between the long ones: there a
+// warp handles one run at a time and waits for its loads, here every lane has U granules of any runs in flight.
+// A window is left at the last whole granule below its last entry and the next one starts at the run that holds that
+// byte (a search, not a step of 31 runs); where 31 runs fill less than one granule, lanes 0..15 resolve that granule's
+// bytes through the plan's tables directly.
+__device__ __forceinline__ uint4 shift_bytes(uint4 a, uint4 b, int sh)  // bytes [sh, sh + 16) of a followed by b, 0 < sh < 16
+{
+    const int bits = (sh & 3) * 8;
+    switch (sh >> 2) {
+        case 0: return splice<0>(a, b, bits);
+        case 1: return splice<1>(a, b, bits);
+        case 2: return splice<2>(a, b, bits);
+        default: return splice<3>(a, b, bits);
+    }
+}
+// the byte at position `pos` of the call's dense side, from the tables alone (any lane, no window)
+__device__ __forceinline__ uint8_t dense_byte(const PlanView& pv, int64_t block_begin, int64_t n_blocks, int64_t block_bytes, int fb,
+                                              int64_t pos, const uint8_t* __restrict__ from, uint8_t pad)
+{
+    const int64_t q = pos / block_bytes, b = block_begin + q;
+    if (b >= n_blocks) return pad;
+    const int64_t in_block = pos - q * block_bytes;
+    const int slot = (int)(in_block / fb);
+    if (slot >= pv.block_fill[b]) return pad;
+    int lo = pv.block_seg_begin[b], hi = pv.block_seg_begin[b + 1];  // the last run of the block that starts at or before slot
+    while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if (pv.seg_start[mid] <= slot) lo = mid; else hi = mid;
+    }
+    const uint8_t* s = from + (pv.seg_src[lo] + (slot - pv.seg_start[lo])) * (int64_t)fb + (in_block - (int64_t)slot * fb);
+    return BLOAD_MAY_READ(s, 1) ? *s : (uint8_t)0;
+}
+__global__ void __launch_bounds__(256, 4) k24_pack_granules(PlanView pv, int32_t n, int32_t t_block, int64_t frame_bytes,
+                                                            int64_t block_begin, const uint8_t* __restrict__ from,
+                                                            uint8_t* __restrict__ to_base, int64_t total, int64_t from_bytes,
+                                                            uint8_t pad, int32_t piece)
+{
+    __shared__ int4 windows[8][32];
+    constexpr int U = 4;  // granules in flight per lane
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    int4* win = windows[warp];
+    const int fb = (int)frame_bytes;
+    const int64_t block_bytes = (int64_t)t_block * fb;
+    const int64_t n_blocks = pv.hdr->n_blocks;
+    const int64_t chunks = (total + piece - 1) / piece;
+    const uint32_t p4 = 0x01010101u * pad;
+    const uint4 pad16 = make_uint4(p4, p4, p4, p4);
+    const uint8_t* from_end = from + from_bytes;
+    for (int64_t c = (int64_t)blockIdx.x * 8 + warp; c < chunks; c += (int64_t)gridDim.x * 8) {
+        const int64_t lo0 = c * (int64_t)piece;  // positions below are relative to this byte of the call's dense side
+        const int p_end = (int)min((int64_t)piece, total - lo0);
+        uint8_t* dense_out = to_base + lo0;
+        int r = 0, e = 0, dn = 0, d_last = 0;
+        int64_t delta = 0;
+        auto load_window = [&](int kw) {  // one lane per run
+            const int4 w = dense_side_entry(pv, n, kw + lane, block_begin, block_bytes, fb, lo0);
+            __syncwarp();  // every lane has left the previous window
+            d_last = __shfl_sync(kFull, w.x, 31);
+            win[lane] = make_int4(__shfl_down_sync(kFull, w.x, 1), w.y, w.z, w.w);  // (lane 31's entry is never walked)
+            __syncwarp();
+            const int4 w0 = win[0];
+            r = 0; dn = w0.x; e = w0.y; delta = (int64_t)(((uint64_t)(uint32_t)w0.w << 32) | (uint32_t)w0.z);
+        };
+        int done = 0;
+        while (done < p_end) {
+            load_window(first_run_at(pv, n, block_begin, n_blocks, lo0 + done, block_bytes, fb, lane));
+            const int lim = min(p_end, d_last);
+            const int lim_g = lim == p_end ? p_end : (lim & ~15);  // whole granules below the window's last entry
+            if (lim_g <= done) {  // 31 runs inside one granule: its bytes one by one, from the tables
+                const int cnt = min(16, p_end - done);
+                if (lane < cnt) wc::put_byte(dense_out + done + lane, dense_byte(pv, block_begin, n_blocks, block_bytes, fb, lo0 + done + lane, from, pad));
+                done += cnt;
+                continue;
+            }
+            for (int p = done + 16 * lane; p < lim_g; p += 32 * 16 * U) {
+                uint4 v0[U], v1[U];
+                int kind[U];  // 0 nothing, 1 aligned source, 2 shifted source, 3 padding, 4 byte by byte
+                int shv[U];   // kind 2: the source's offset in its 16-byte vector; kind 4: the window entry of the granule's first byte
+#pragma unroll
+                for (int u = 0; u < U; ++u) {
+                    const int q = p + u * 512;
+                    kind[u] = 0; shv[u] = 0;
+                    if (q < lim_g) {
+                        while (q >= dn) {  // (q < lim_g <= begin of the window's last entry, so r stays below 31)
+                            ++r;
+                            const int4 w = win[r];
+                            dn = w.x; e = w.y; delta = (int64_t)(((uint64_t)(uint32_t)w.w << 32) | (uint32_t)w.z);
+                        }
+                        const uint8_t* s = from + (delta + q);
+                        const int sh = (int)(reinterpret_cast<uintptr_t>(s) & 15u);
+                        if (q + 16 <= e && q + 16 <= p_end) {
+                            if (sh == 0) { kind[u] = 1; v0[u] = wc::ld_stream(reinterpret_cast<const uint4*>(s)); }
+                            else if (s - sh + 32 <= from_end) {
+                                kind[u] = 2; shv[u] = sh;
+                                v0[u] = wc::ld_shared_sector<false>(reinterpret_cast<const uint4*>(s - sh));
+                                v1[u] = wc::ld_shared_sector<false>(reinterpret_cast<const uint4*>(s - sh) + 1);
+                            } else { kind[u] = 4; shv[u] = r; }
+                        } else if (q >= e && q + 16 <= dn && q + 16 <= p_end) kind[u] = 3;
+                        else { kind[u] = 4; shv[u] = r; }
+                    }
+                }
+#pragma unroll
+                for (int u = 0; u < U; ++u) {
+                    const int q = p + u * 512;
+                    uint4* d = reinterpret_cast<uint4*>(dense_out + q);
+                    if (kind[u] == 1) wc::st_stream(d, v0[u]);
+                    else if (kind[u] == 2) wc::st_stream(d, shift_bytes(v0[u], v1[u], shv[u]));
+                    else if (kind[u] == 3) wc::st_stream(d, pad16);
+                }
+                // the granules that hold a run's begin or end: byte by byte, with a walk of their own from the granule's entry
+#pragma unroll
+                for (int u = 0; u < U; ++u) {
+                    if (kind[u] != 4) continue;
+                    int rr = shv[u];
+                    int4 w = win[rr];
+                    int ddn = w.x, ee = w.y;
+                    int64_t dd = (int64_t)(((uint64_t)(uint32_t)w.w << 32) | (uint32_t)w.z);
+                    const int q = p + u * 512, q_end = min(q + 16, p_end);
+                    for (int x = q; x < q_end; ++x) {
+                        while (x >= ddn) {
+                            ++rr; w = win[rr];
+                            ddn = w.x; ee = w.y; dd = (int64_t)(((uint64_t)(uint32_t)w.w << 32) | (uint32_t)w.z);
+                        }
+                        if (x < ee) wc::copy_byte(dense_out + x, from + (dd + x));
+                        else wc::put_byte(dense_out + x, pad);
+                    }
+                }
+            }
+            done = lim_g;
+        }
+    }
+}
 // Whole-plan unpack by the same unstaged walk, along the RAGGED side: a window entry is one sequence (it ends where the
 // next begins), a lane loads each of its words from the word's place in the dense buffer and stores it in place; the
 // stores are contiguous across the warp, the loads inside a run.
@@ -1069,6 +1206,19 @@ WalkKernel walk_kernel_for(int64_t frame_bytes)
 // against the staged kernels: 4-byte frames in 3.5 KB runs 5.86 against 6.10, 12-byte frames in 10 KB runs 6.07 against
 // 6.06, 100-byte frames in 5.8 KB runs 5.99 against 6.04, 4-byte frames in 232-byte runs 3.75 against 3.65, 12-byte frames
 // in 696-byte runs 4.97 against 4.70: within 6 % either way, so the staged kernels stayed.
+#ifndef BLOAD_GRANULE_MAX_RUN
+#define BLOAD_GRANULE_MAX_RUN 4096
+#endif
+#ifndef BLOAD_GRANULE_MAX_FRAME
+#define BLOAD_GRANULE_MAX_FRAME 3
+#endif
+// Pack of frames of 1 to 3 bytes (per-token masks, 16-bit ids or scalars) in runs beyond the 2- and 1-byte walks and up
+// to 4 KB on average: k24_pack_granules instead of the register path.  Measured on B200 (TB/s, granules against the
+// register path; about 1.5 GB per case): token lengths, 1-byte frames (870-byte runs) 3.70 against 2.52, 2-byte frames
+// (1.7 KB) 4.43 against 3.66, 3-byte frames (2.6 KB) 4.56 against 4.28; beyond that the register path is as fast
+// or faster: 6-byte frames (5.2 KB) 4.96 against 4.93, 10-byte (8.7 KB) 5.21 against 5.42, 30-byte (26 KB) 5.54 against
+// 6.00; 30-byte frames in heavy-tailed 1.7 KB runs 2.98 against 3.07, 250-byte frames in 5.5 KB clips 4.47 against 4.28.
+constexpr int64_t kGranuleMaxRun = BLOAD_GRANULE_MAX_RUN, kGranuleMaxFrame = BLOAD_GRANULE_MAX_FRAME;
 inline bool walks_unstaged(int64_t frame_bytes, int64_t mean_run, bool unpack)
 {
     if (frame_bytes % 8 == 0) return mean_run <= kStagedMaxRunBytes;
@@ -1320,6 +1470,7 @@ cudaError_t launch_copy(bool unpack, const PlanView& pv, int32_t t_block, int64_
     //                              block sub-range is unpacked
     //   staged, word by word       frames that are multiples of 4 (not 8) bytes in runs of at most 768 bytes
     //   staged, run by run         the other frames that are multiples of 4 bytes, in runs of at most 16 KB
+    //   granules of 16 bytes       pack of frames of 1 to 3 bytes in runs beyond the walks, up to 4 KB on average
     //   register path              everything else
     // (the staged kernels and the walks index windows of 32 runs past a 32-bit position in the segment list)
     const bool indexable = n > 0 && n < 0x7fffff00LL && block_bytes < (1LL << 30);
@@ -1417,6 +1568,17 @@ cudaError_t launch_copy(bool unpack, const PlanView& pv, int32_t t_block, int64_
                                                                  dense + done * block_bytes, ragged_out, (uint32_t)gpb, pad_byte);
         }
         note_copy_kernel(kCallUnpack, "k8_unpack_staged");
+        return cudaPeekAtLastError();
+    }
+    // pack of frames that are not multiples of 4 bytes, in runs beyond the 2- and 1-byte walks: granules of 16 bytes
+    if (!unpack && indexable && frame_bytes % 4 != 0 && frame_bytes <= kGranuleMaxFrame && mean_run <= kGranuleMaxRun) {
+        const int64_t cap = (int64_t)device_info().sm_count * 32;
+        const int64_t total = block_count * block_bytes;
+        const int piece = walk_piece_bytes(total, device_info().sm_count);
+        const int64_t want = ((total + piece - 1) / piece + 7) / 8;
+        k24_pack_granules<<<(unsigned)(want < cap ? want : cap), 256, 0, st>>>(pv, (int32_t)n, t_block, frame_bytes, block_begin, ragged_in,
+                                                                                dense, total, ragged_bytes, pad_byte, piece);
+        note_copy_kernel(kCallPack, "k24_pack_granules");
         return cudaPeekAtLastError();
     }
 #if BLOAD_BULK_COPY

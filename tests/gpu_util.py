@@ -152,4 +152,6 @@ def expected_copy_kernels(sum_t: int, n: int, fb: int, t_block: int) -> dict:
         up = run <= (1024 if fb % 2 == 0 else 384)
         return dict(pack="k19_pack_walk_dense", unpack="k21_unpack_walk_ragged" if up else "k7_copy<unpack>",
                     unpack_range="k19_unpack_walk_dense" if up else "k7_copy<unpack>", pack_meta="k19_pack_walk_dense")
+    if fb < 4 and run <= 4096:  # frames of 1 to 3 bytes in runs beyond the word-wise walks: 16-byte granules (pack only)
+        return dict(pack="k24_pack_granules", unpack="k7_copy<unpack>", unpack_range="k7_copy<unpack>", pack_meta="k24_pack_granules")
     return dict(pack="k7_copy<pack>", unpack="k7_copy<unpack>", unpack_range="k7_copy<unpack>", pack_meta="k7_copy<pack>")

@@ -580,3 +580,34 @@ def test_reader_behind_a_pack_of_large_frames_sees_dense_blocks_and_metadata():
         assert np.array_equal(d.cpu().numpy().reshape(cnt, tb, fb), O.pack(op, h_store, fb, b0, cnt, 0x5C)), b0
         for name, arr, want in zip(("seq_id", "pos", "reset", "valid"), (si, po, re, va), O.metadata(op, b0, cnt)):
             assert np.array_equal(arr.cpu().numpy().reshape(cnt, tb), want), (b0, name)
+
+
+@pytest.mark.parametrize("tb,fb,kind", [(4096, 1, "token_like"), (4096, 2, "token_like"), (4096, 3, "token_like"),
+                                        (333, 3, "uniform"), (2047, 2, "uniform"), (5000, 1, "ones_and_long"),
+                                        (3100, 1, "ones_and_long"), (901, 3, "uniform")])
+def test_frames_of_one_to_three_bytes_in_runs_up_to_4_kb_are_packed_in_granules(tb, fb, kind):
+    """Frames shorter than a word (masks, 16-bit ids) in runs beyond the word-wise walks: the pack kernel that moves
+    16-byte granules.  Lengths with the shape of the token workload (many runs of 8 frames between runs as long as a
+    block), blocks whose size is not a multiple of 16 bytes (the last granule of the call is partial), and thousands of
+    one-frame runs between long ones, which the fill rule collects at the ends of the blocks: dozens of runs inside one
+    granule, more than a window of 32 holds.  Whole plan with filler blocks, sub-ranges, a non-zero pad byte."""
+    rng = np.random.default_rng(tb * 7 + fb)
+    if kind == "token_like":
+        T = np.concatenate([np.full(900, 8), np.full(350 // fb, tb), rng.integers(9, tb // fb, size=900)]).astype(np.int32)
+    elif kind == "uniform":
+        T = rng.integers(1, tb + 1, size=2500).astype(np.int32)
+    else:
+        T = np.concatenate([np.ones(3000, np.int32), np.full(900, tb, np.int32), rng.integers(2, 40, size=300).astype(np.int32)])
+    rng.shuffle(T)
+    want_k = G.expected_copy_kernels(int(T.sum()), T.size, fb, tb)
+    assert want_k["pack"] == "k24_pack_granules", (int(T.sum()) * fb // T.size)
+    plan, op = G.full_parity(T, tb, 41, fb, out_fb=fb, pad=0xC3, extra_blocks=3)
+    assert B.bload_last_copy_kernel("pack") == "k24_pack_granules"
+    store = torch.randint(0, 256, (op.sum_t * fb,), dtype=torch.uint8, device=G.DEV)
+    store_h = store.cpu().numpy()
+    nb = op.n_blocks
+    for b0, cnt in [(0, 1), (1, 1), (nb // 3, 5), (nb - 2, 4), (nb, 1)]:
+        res, _ = G.gpu_pack_all(plan, store, fb, b0, cnt, 0x3D, meta=True)
+        d = G.first_diff(res["dense"].reshape(-1), O.pack(op, store_h, fb, b0, cnt, 0x3D).reshape(-1))
+        assert d is None, "blocks [%d, +%d): %s" % (b0, cnt, d)
+    assert B.bload_last_copy_kernel("pack") == "k24_pack_granules"
