@@ -23,7 +23,8 @@
 //                                of its words in a window of 32 runs)
 //   k19 / k21                    word by word without a stage: frames that are multiples of 8 bytes, and frames that are
 //                                not multiples of 4 bytes in short runs
-//   k24                          pack of frames of 1 to 3 bytes in runs of 0.4 to 4 KB: the walk in granules of 16 bytes
+//   k24 / k25                    pack and whole-plan unpack of frames of 1 to 3 bytes in runs of 0.4 to 4 KB: the walk in
+//                                granules of 16 bytes
 //   k7b_copy_bulk                a measurement variant (large frames through the bulk-copy engine), off by default
 //   launch_copy and friends      which kernel takes which call, with the measurements the rules come from
 #include "bload_internal.cuh"
@@ -1168,6 +1169,118 @@ __global__ void __launch_bounds__(256, 4) k21_unpack_walk_ragged(PlanView pv, in
         }
     }
 }
+// Whole-plan unpack of the same frames in granules of 16 bytes, along the ragged side (which has no padding: every byte
+// belongs to a sequence).  The stores are the aligned side here, the loads from the blocks the shifted one.
+__device__ __forceinline__ uint8_t ragged_byte(const PlanView& pv, int n, int64_t block_bytes, int fb, int64_t pos,
+                                               const uint8_t* __restrict__ dense)
+{
+    const int64_t f = pos / fb;
+    int lo = 0, hi = n;  // the last sequence that begins at or before frame f
+    while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if (pv.offsets[mid] <= f) lo = mid; else hi = mid;
+    }
+    const uint8_t* s = dense + pv.seq_block[lo] * block_bytes + (pv.seq_start[lo] + (f - pv.offsets[lo])) * (int64_t)fb + (pos - f * fb);
+    return BLOAD_MAY_READ(s, 1) ? *s : (uint8_t)0;
+}
+__global__ void __launch_bounds__(256, 4) k25_unpack_granules(PlanView pv, int32_t n, int32_t t_block, int64_t frame_bytes,
+                                                              int64_t sum_t, const uint8_t* __restrict__ dense,
+                                                              uint8_t* __restrict__ ragged, int64_t dense_bytes, int32_t piece)
+{
+    __shared__ int4 windows[8][32];
+    constexpr int U = 4;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    int4* win = windows[warp];
+    const int fb = (int)frame_bytes;
+    const int64_t total = sum_t * frame_bytes;
+    const int64_t block_bytes = (int64_t)t_block * frame_bytes;
+    const int64_t chunks = (total + piece - 1) / piece;
+    const uint8_t* dense_end = dense + dense_bytes;
+    for (int64_t c = (int64_t)blockIdx.x * 8 + warp; c < chunks; c += (int64_t)gridDim.x * 8) {
+        const int64_t lo0 = c * (int64_t)piece;  // positions below are relative to this byte of the ragged side
+        const int p_end = (int)min((int64_t)piece, total - lo0);
+        uint8_t* out = ragged + lo0;
+        int r = 0, dn = 0, d_last = 0;
+        int64_t delta = 0;
+        auto load_window = [&](int kw) {  // one lane per sequence
+            const int i = kw + lane;
+            int4 w = make_int4(kFar, kFar, 0, 0);
+            if (i < n) {
+                const int64_t d_flat = pv.offsets[i] * frame_bytes - lo0;
+                const int64_t dl = pv.seq_block[i] * block_bytes + pv.seq_start[i] * frame_bytes - d_flat;
+                w = make_int4(clamp_far(d_flat), kFar, (int)(uint32_t)(uint64_t)dl, (int)(uint32_t)((uint64_t)dl >> 32));
+            }
+            __syncwarp();  // every lane has left the previous window
+            d_last = __shfl_sync(kFull, w.x, 31);
+            win[lane] = make_int4(__shfl_down_sync(kFull, w.x, 1), w.y, w.z, w.w);  // (lane 31's entry is never walked)
+            __syncwarp();
+            const int4 w0 = win[0];
+            r = 0; dn = w0.x; delta = (int64_t)(((uint64_t)(uint32_t)w0.w << 32) | (uint32_t)w0.z);
+        };
+        int done = 0;
+        while (done < p_end) {
+            load_window(warp_find_sequence(pv.offsets, n, (lo0 + done) / frame_bytes, lane));
+            const int lim = min(p_end, d_last);
+            const int lim_g = lim == p_end ? p_end : (lim & ~15);  // whole granules below the window's last entry
+            if (lim_g <= done) {  // 31 sequences inside one granule: its bytes one by one, from the tables
+                const int cnt = min(16, p_end - done);
+                if (lane < cnt) wc::put_byte(out + done + lane, ragged_byte(pv, n, block_bytes, fb, lo0 + done + lane, dense));
+                done += cnt;
+                continue;
+            }
+            for (int p = done + 16 * lane; p < lim_g; p += 32 * 16 * U) {
+                uint4 v0[U], v1[U];
+                int kind[U];  // 0 nothing, 1 aligned source, 2 shifted source, 4 byte by byte
+                int shv[U];   // kind 2: the source's offset in its 16-byte vector; kind 4: the window entry of the granule's first byte
+#pragma unroll
+                for (int u = 0; u < U; ++u) {
+                    const int q = p + u * 512;
+                    kind[u] = 0; shv[u] = 0;
+                    if (q < lim_g) {
+                        while (q >= dn) {  // (q < lim_g <= begin of the window's last entry, so r stays below 31)
+                            ++r;
+                            const int4 w = win[r];
+                            dn = w.x; delta = (int64_t)(((uint64_t)(uint32_t)w.w << 32) | (uint32_t)w.z);
+                        }
+                        const uint8_t* s = dense + (delta + q);
+                        const int sh = (int)(reinterpret_cast<uintptr_t>(s) & 15u);
+                        if (q + 16 <= dn && q + 16 <= p_end) {
+                            if (sh == 0) { kind[u] = 1; v0[u] = wc::ld_stream(reinterpret_cast<const uint4*>(s)); }
+                            else if (s - sh + 32 <= dense_end) {
+                                kind[u] = 2; shv[u] = sh;
+                                v0[u] = wc::ld_shared_sector<true>(reinterpret_cast<const uint4*>(s - sh));
+                                v1[u] = wc::ld_shared_sector<true>(reinterpret_cast<const uint4*>(s - sh) + 1);
+                            } else { kind[u] = 4; shv[u] = r; }
+                        } else { kind[u] = 4; shv[u] = r; }
+                    }
+                }
+#pragma unroll
+                for (int u = 0; u < U; ++u) {
+                    uint4* d = reinterpret_cast<uint4*>(out + p + u * 512);
+                    if (kind[u] == 1) wc::st_stream(d, v0[u]);
+                    else if (kind[u] == 2) wc::st_stream(d, shift_bytes(v0[u], v1[u], shv[u]));
+                }
+#pragma unroll
+                for (int u = 0; u < U; ++u) {
+                    if (kind[u] != 4) continue;
+                    int rr = shv[u];
+                    int4 w = win[rr];
+                    int ddn = w.x;
+                    int64_t dd = (int64_t)(((uint64_t)(uint32_t)w.w << 32) | (uint32_t)w.z);
+                    const int q = p + u * 512, q_end = min(q + 16, p_end);
+                    for (int x = q; x < q_end; ++x) {
+                        while (x >= ddn) {
+                            ++rr; w = win[rr];
+                            ddn = w.x; dd = (int64_t)(((uint64_t)(uint32_t)w.w << 32) | (uint32_t)w.z);
+                        }
+                        wc::copy_byte(out + x, dense + (dd + x));
+                    }
+                }
+            }
+            done = lim_g;
+        }
+    }
+}
 using WalkRaggedKernel = void (*)(PlanView, int32_t, int32_t, int64_t, int64_t, const uint8_t*, uint8_t*, int32_t);
 inline WalkRaggedKernel walk_ragged_kernel_for(int64_t frame_bytes)
 {
@@ -1209,6 +1322,9 @@ WalkKernel walk_kernel_for(int64_t frame_bytes)
 #ifndef BLOAD_GRANULE_MAX_RUN
 #define BLOAD_GRANULE_MAX_RUN 4096
 #endif
+#ifndef BLOAD_GRANULE_UNPACK
+#define BLOAD_GRANULE_UNPACK 1  // 0: whole-plan unpack of these frames stays on the register path (to compare)
+#endif
 #ifndef BLOAD_GRANULE_MAX_FRAME
 #define BLOAD_GRANULE_MAX_FRAME 3
 #endif
@@ -1218,6 +1334,8 @@ WalkKernel walk_kernel_for(int64_t frame_bytes)
 // (1.7 KB) 4.43 against 3.66, 3-byte frames (2.6 KB) 4.56 against 4.28; beyond that the register path is as fast
 // or faster: 6-byte frames (5.2 KB) 4.96 against 4.93, 10-byte (8.7 KB) 5.21 against 5.42, 30-byte (26 KB) 5.54 against
 // 6.00; 30-byte frames in heavy-tailed 1.7 KB runs 2.98 against 3.07, 250-byte frames in 5.5 KB clips 4.47 against 4.28.
+// Whole-plan unpack of the same frames along the ragged side (k25_unpack_granules), same cases: 3.67 against 3.23, 4.71
+// against 4.19, 5.02 against 4.6.
 constexpr int64_t kGranuleMaxRun = BLOAD_GRANULE_MAX_RUN, kGranuleMaxFrame = BLOAD_GRANULE_MAX_FRAME;
 inline bool walks_unstaged(int64_t frame_bytes, int64_t mean_run, bool unpack)
 {
@@ -1470,7 +1588,8 @@ cudaError_t launch_copy(bool unpack, const PlanView& pv, int32_t t_block, int64_
     //                              block sub-range is unpacked
     //   staged, word by word       frames that are multiples of 4 (not 8) bytes in runs of at most 768 bytes
     //   staged, run by run         the other frames that are multiples of 4 bytes, in runs of at most 16 KB
-    //   granules of 16 bytes       pack of frames of 1 to 3 bytes in runs beyond the walks, up to 4 KB on average
+    //   granules of 16 bytes       pack and whole-plan unpack of frames of 1 to 3 bytes in runs beyond the walks, up to
+    //                              4 KB on average
     //   register path              everything else
     // (the staged kernels and the walks index windows of 32 runs past a 32-bit position in the segment list)
     const bool indexable = n > 0 && n < 0x7fffff00LL && block_bytes < (1LL << 30);
@@ -1568,6 +1687,16 @@ cudaError_t launch_copy(bool unpack, const PlanView& pv, int32_t t_block, int64_
                                                                  dense + done * block_bytes, ragged_out, (uint32_t)gpb, pad_byte);
         }
         note_copy_kernel(kCallUnpack, "k8_unpack_staged");
+        return cudaPeekAtLastError();
+    }
+    // whole-plan unpack of the same frames, along the ragged side
+    if (BLOAD_GRANULE_UNPACK && whole_plan && indexable && frame_bytes % 4 != 0 && frame_bytes <= kGranuleMaxFrame && mean_run <= kGranuleMaxRun) {
+        const int64_t cap = (int64_t)device_info().sm_count * 32;
+        const int piece = walk_piece_bytes(ragged_bytes, device_info().sm_count);
+        const int64_t want = ((ragged_bytes + piece - 1) / piece + 7) / 8;
+        k25_unpack_granules<<<(unsigned)(want < cap ? want : cap), 256, 0, st>>>(pv, (int32_t)n, t_block, frame_bytes, ragged_bytes / frame_bytes,
+                                                                                  dense, ragged_out, block_count * block_bytes, piece);
+        note_copy_kernel(kCallUnpack, "k25_unpack_granules");
         return cudaPeekAtLastError();
     }
     // pack of frames that are not multiples of 4 bytes, in runs beyond the 2- and 1-byte walks: granules of 16 bytes

@@ -148,10 +148,12 @@ def expected_copy_kernels(sum_t: int, n: int, fb: int, t_block: int) -> dict:
                          unpack_range="k8_unpack_staged" if (t_block * fb) % 16 == 0 else "k7_copy<unpack>")
         plain["pack_meta"] = ("k17_pack_short_runs" if (fb % 16 == 0 or words) else "k10_pack_contig") + "<metadata>"
         return plain
+    gran = fb < 4 and run <= 4096  # frames of 1 to 3 bytes in runs beyond the word-wise walks: 16-byte granules
     if fb % 4 != 0 and ((fb % 2 == 0 and run <= 1536) or run <= 384):
         up = run <= (1024 if fb % 2 == 0 else 384)
-        return dict(pack="k19_pack_walk_dense", unpack="k21_unpack_walk_ragged" if up else "k7_copy<unpack>",
+        return dict(pack="k19_pack_walk_dense",
+                    unpack="k21_unpack_walk_ragged" if up else ("k25_unpack_granules" if gran else "k7_copy<unpack>"),
                     unpack_range="k19_unpack_walk_dense" if up else "k7_copy<unpack>", pack_meta="k19_pack_walk_dense")
-    if fb < 4 and run <= 4096:  # frames of 1 to 3 bytes in runs beyond the word-wise walks: 16-byte granules (pack only)
-        return dict(pack="k24_pack_granules", unpack="k7_copy<unpack>", unpack_range="k7_copy<unpack>", pack_meta="k24_pack_granules")
+    if gran:  # (whole-plan unpack; block sub-ranges stay on the register path)
+        return dict(pack="k24_pack_granules", unpack="k25_unpack_granules", unpack_range="k7_copy<unpack>", pack_meta="k24_pack_granules")
     return dict(pack="k7_copy<pack>", unpack="k7_copy<unpack>", unpack_range="k7_copy<unpack>", pack_meta="k7_copy<pack>")

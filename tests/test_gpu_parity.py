@@ -585,9 +585,9 @@ def test_reader_behind_a_pack_of_large_frames_sees_dense_blocks_and_metadata():
 @pytest.mark.parametrize("tb,fb,kind", [(4096, 1, "token_like"), (4096, 2, "token_like"), (4096, 3, "token_like"),
                                         (333, 3, "uniform"), (2047, 2, "uniform"), (5000, 1, "ones_and_long"),
                                         (3100, 1, "ones_and_long"), (901, 3, "uniform")])
-def test_frames_of_one_to_three_bytes_in_runs_up_to_4_kb_are_packed_in_granules(tb, fb, kind):
-    """Frames shorter than a word (masks, 16-bit ids) in runs beyond the word-wise walks: the pack kernel that moves
-    16-byte granules.  Lengths with the shape of the token workload (many runs of 8 frames between runs as long as a
+def test_frames_of_one_to_three_bytes_in_runs_up_to_4_kb_move_in_granules(tb, fb, kind):
+    """Frames shorter than a word (masks, 16-bit ids) in runs beyond the word-wise walks: the pack and whole-plan unpack
+    kernels that move 16-byte granules.  Lengths with the shape of the token workload (many runs of 8 frames between runs as long as a
     block), blocks whose size is not a multiple of 16 bytes (the last granule of the call is partial), and thousands of
     one-frame runs between long ones, which the fill rule collects at the ends of the blocks: dozens of runs inside one
     granule, more than a window of 32 holds.  Whole plan with filler blocks, sub-ranges, a non-zero pad byte."""
@@ -602,7 +602,7 @@ def test_frames_of_one_to_three_bytes_in_runs_up_to_4_kb_are_packed_in_granules(
     want_k = G.expected_copy_kernels(int(T.sum()), T.size, fb, tb)
     assert want_k["pack"] == "k24_pack_granules", (int(T.sum()) * fb // T.size)
     plan, op = G.full_parity(T, tb, 41, fb, out_fb=fb, pad=0xC3, extra_blocks=3)
-    assert B.bload_last_copy_kernel("pack") == "k24_pack_granules"
+    assert B.bload_last_copy_kernel("pack") == "k24_pack_granules" and B.bload_last_copy_kernel("unpack") == "k25_unpack_granules"
     store = torch.randint(0, 256, (op.sum_t * fb,), dtype=torch.uint8, device=G.DEV)
     store_h = store.cpu().numpy()
     nb = op.n_blocks
