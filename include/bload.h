@@ -520,7 +520,8 @@ BLOAD_API int bload_debug_status(uint64_t out[4], int clear);
  * which = 0 bload_pack (the dense output), 1 bload_unpack, 2 bload_carry_prev, 3 bload_pack_var[2d],
  * 4 bload_unpack_var[2d].  The library picks a kernel from the frame size and the run lengths (register path for
  * large frames, shared-memory staged paths for small word-sized frames, run by run or -- for short runs -- word by
- * word); a benchmark reports the choice with this
+ * word, unstaged walks word by word or, for frames of 1 to 3 bytes, in granules of 16 bytes); a benchmark reports the
+ * choice with this
  * call instead of guessing it.  Host only.  Returns "" when no such call was made, or for another `which`.
  */
 BLOAD_API const char* bload_last_copy_kernel(int which);
