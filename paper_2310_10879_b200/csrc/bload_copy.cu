@@ -1322,6 +1322,9 @@ WalkKernel walk_kernel_for(int64_t frame_bytes)
 #ifndef BLOAD_GRANULE_MAX_RUN
 #define BLOAD_GRANULE_MAX_RUN 4096
 #endif
+#ifndef BLOAD_ODD_WALKS
+#define BLOAD_ODD_WALKS 1  // 0: no 2- and 1-byte word walks (to compare the granule kernels with them)
+#endif
 #ifndef BLOAD_GRANULE_UNPACK
 #define BLOAD_GRANULE_UNPACK 1  // 0: whole-plan unpack of these frames stays on the register path (to compare)
 #endif
@@ -1336,11 +1339,15 @@ WalkKernel walk_kernel_for(int64_t frame_bytes)
 // 6.00; 30-byte frames in heavy-tailed 1.7 KB runs 2.98 against 3.07, 250-byte frames in 5.5 KB clips 4.47 against 4.28.
 // Whole-plan unpack of the same frames along the ragged side (k25_unpack_granules), same cases: 3.67 against 3.23, 4.71
 // against 4.19, 5.02 against 4.6.
+// In short runs the word-wise walks stay (granules against them, pack / unpack): 6-byte frames in 346-byte runs 1.44 /
+// 1.83 against 2.87 / 3.02, 3-byte frames in 173-byte runs 1.01 / 1.32 against 1.49 / 1.60, 30-byte frames in 663-byte
+// runs 2.09 / 2.60 against 3.19 / 3.35: a granule that holds a run's end is moved byte by byte.
 constexpr int64_t kGranuleMaxRun = BLOAD_GRANULE_MAX_RUN, kGranuleMaxFrame = BLOAD_GRANULE_MAX_FRAME;
 inline bool walks_unstaged(int64_t frame_bytes, int64_t mean_run, bool unpack)
 {
     if (frame_bytes % 8 == 0) return mean_run <= kStagedMaxRunBytes;
     if (frame_bytes % 4 == 0) return false;
+    if (!BLOAD_ODD_WALKS) return false;
     if (frame_bytes % 2 == 0) return mean_run <= (unpack ? 1024 : 1536);
     return mean_run <= 384;
 }
